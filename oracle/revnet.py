@@ -1,0 +1,318 @@
+"""Float64 CPU oracle: reversible block, Algorithm 1, and a classification stack.
+
+TEST INFRASTRUCTURE ONLY (see the package docstring).  All tensors are NCHW
+numpy float64; convolution weights are [Cout, Cin, kh, kw].
+
+Structures (plain Python, built by the caller):
+  layer    = {"name": str, "gamma": [Cin], "beta": [Cin], "W": [Cout,Cin,k,k], "stride": int (default 1)}
+  function = list of layers, applied first to last; each layer is conv(relu(bn(.)))   (Section 2.2, Eq. 2)
+  block    = (F, G)                                                                     (Section 3.1)
+  net      = {"stem": {"name","W","stride","pad"}, "maxpool": bool,
+              "stages": [{"trans": layer or None, "c": int, "units": [block, ...]}],
+              "fc": {"name","W":[K,C],"b":[K]}, "eps": float}
+"""
+import ctypes
+import os
+
+import numpy as np
+
+from . import build as _build
+
+_lib = None
+_D = ctypes.POINTER(ctypes.c_double)
+_I = ctypes.POINTER(ctypes.c_int)
+
+# running count of dense multiply-add work issued through the conv primitives (2 flops per MAC)
+FLOPS = {"conv": 0}
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(_build.build())
+        for fn in ("oracle_conv_fwd", "oracle_conv_dgrad", "oracle_conv_wgrad"):
+            getattr(_lib, fn).argtypes = [_D, _D, _D] + [ctypes.c_int] * 8
+            getattr(_lib, fn).restype = None
+        _lib.oracle_maxpool_fwd.argtypes = [_D, _D, _I] + [ctypes.c_int] * 7
+        _lib.oracle_maxpool_bwd.argtypes = [_D, _I, _D] + [ctypes.c_int] * 6
+    return _lib
+
+
+def _p(x):
+    return x.ctypes.data_as(_D)
+
+
+def _c(x):
+    return np.ascontiguousarray(x, dtype=np.float64)
+
+
+def _osz(n, k, s, p):
+    return (n + 2 * p - k) // s + 1
+
+
+# --------------------------------------------------------------------------- primitives
+
+def conv_fwd(a, w, stride=1, pad=None):
+    """out[n,co,i,j] = sum_{ci,kh,kw} w[co,ci,kh,kw] a[n,ci,i*s+kh-p,j*s+kw-p]  (Eq. 2, Conv_kxk)."""
+    a, w = _c(a), _c(w)
+    N, Ci, H, W = a.shape
+    Co, _, k, _ = w.shape
+    p = k // 2 if pad is None else pad
+    out = np.empty((N, Co, _osz(H, k, stride, p), _osz(W, k, stride, p)))
+    _load().oracle_conv_fwd(_p(a), _p(w), _p(out), N, Ci, H, W, Co, k, stride, p)
+    FLOPS["conv"] += 2 * out.size * Ci * k * k
+    return out
+
+
+def conv_dgrad(dout, w, in_hw, stride=1, pad=None):
+    """Adjoint of conv_fwd with respect to its input."""
+    dout, w = _c(dout), _c(w)
+    N, Co = dout.shape[:2]
+    _, Ci, k, _ = w.shape
+    p = k // 2 if pad is None else pad
+    H, W = in_hw
+    da = np.empty((N, Ci, H, W))
+    _load().oracle_conv_dgrad(_p(dout), _p(w), _p(da), N, Ci, H, W, Co, k, stride, p)
+    FLOPS["conv"] += 2 * dout.size * Ci * k * k
+    return da
+
+
+def conv_wgrad(dout, a, k, stride=1, pad=None):
+    """Adjoint of conv_fwd with respect to its weights."""
+    dout, a = _c(dout), _c(a)
+    N, Ci, H, W = a.shape
+    Co = dout.shape[1]
+    p = k // 2 if pad is None else pad
+    dw = np.empty((Co, Ci, k, k))
+    _load().oracle_conv_wgrad(_p(dout), _p(a), _p(dw), N, Ci, H, W, Co, k, stride, p)
+    FLOPS["conv"] += 2 * dout.size * Ci * k * k
+    return dw
+
+
+def maxpool_fwd(a, k=3, s=2, p=1):
+    a = _c(a)
+    N, C, H, W = a.shape
+    Ho, Wo = _osz(H, k, s, p), _osz(W, k, s, p)
+    out = np.empty((N, C, Ho, Wo))
+    idx = np.empty((N, C, Ho, Wo), dtype=np.int32)
+    _load().oracle_maxpool_fwd(_p(a), _p(out), idx.ctypes.data_as(_I), N, C, H, W, k, s, p)
+    return out, idx
+
+
+def maxpool_bwd(dout, idx, in_hw):
+    dout = _c(dout)
+    N, C, Ho, Wo = dout.shape
+    H, W = in_hw
+    da = np.empty((N, C, H, W))
+    _load().oracle_maxpool_bwd(_p(dout), idx.ctypes.data_as(_I), _p(da), N, C, H, W, Ho, Wo)
+    return da
+
+
+def bn_relu_fwd(t, gamma, beta, eps):
+    """a(x) = ReLU(BN(x)) with train-mode batch statistics (Eq. 2): per channel over (n,h,w),
+    biased variance.  Returns a and what the backward needs."""
+    mu = t.mean(axis=(0, 2, 3), keepdims=True)
+    var = ((t - mu) ** 2).mean(axis=(0, 2, 3), keepdims=True)
+    r = 1.0 / np.sqrt(var + eps)
+    xhat = (t - mu) * r
+    b = gamma.reshape(1, -1, 1, 1) * xhat + beta.reshape(1, -1, 1, 1)
+    a = np.maximum(b, 0.0)
+    return a, (xhat, r, b > 0.0, gamma)
+
+
+def bn_relu_bwd(da, cache):
+    """Backprop through ReLU then train-mode BN, differentiating through the batch mean and variance.
+    ReLU'(0) = 0."""
+    xhat, r, mask, gamma = cache
+    M = xhat.shape[0] * xhat.shape[2] * xhat.shape[3]
+    db = da * mask
+    dbeta = db.sum(axis=(0, 2, 3))
+    dgamma = (db * xhat).sum(axis=(0, 2, 3))
+    g = gamma.reshape(1, -1, 1, 1)
+    dt = (g * r / M) * (M * db - dbeta.reshape(1, -1, 1, 1) - xhat * dgamma.reshape(1, -1, 1, 1))
+    return dt, dgamma, dbeta
+
+
+# --------------------------------------------------------------------------- residual functions
+
+def fn_fwd(u, layers, eps):
+    """Residual function: chain of c_k(x) = Conv(ReLU(BN(x))) layers (Eq. 2: Basic = c3(c3(x)),
+    Bottleneck = c1(c3(c1(x)))).  Returns the value and per-layer caches."""
+    caches = []
+    t = u
+    for L in layers:
+        a, bn = bn_relu_fwd(t, np.asarray(L["gamma"], np.float64), np.asarray(L["beta"], np.float64), eps)
+        w = np.asarray(L["W"], np.float64)
+        s = L.get("stride", 1)
+        caches.append((bn, a, w, s, t.shape[2:], L["name"]))
+        t = conv_fwd(a, w, stride=s)
+    return t, caches
+
+
+def fn_bwd(g, caches, grads):
+    """Ordinary backprop (Eq. 1) through a residual function; parameter gradients go into `grads`."""
+    for bn, a, w, s, in_hw, name in reversed(caches):
+        grads[name + ".W"] = conv_wgrad(g, a, w.shape[2], stride=s)
+        da = conv_dgrad(g, w, in_hw, stride=s)
+        g, dgamma, dbeta = bn_relu_bwd(da, bn)
+        grads[name + ".gamma"] = dgamma
+        grads[name + ".beta"] = dbeta
+    return g
+
+
+# --------------------------------------------------------------------------- reversible block
+
+def block_fwd(x1, x2, F, G, eps, keep=False):
+    """y1 = x1 + F(x2); y2 = x2 + G(y1)   (Section 3.1)."""
+    f, cF = fn_fwd(x2, F, eps)
+    y1 = x1 + f
+    g, cG = fn_fwd(y1, G, eps)
+    y2 = x2 + g
+    return (y1, y2, (cF, cG)) if keep else (y1, y2)
+
+
+def block_inverse(y1, y2, F, G, eps):
+    """x2 = y2 - G(y1); x1 = y1 - F(x2)   (Section 3.1)."""
+    x2 = y2 - fn_fwd(y1, G, eps)[0]
+    x1 = y1 - fn_fwd(x2, F, eps)[0]
+    return x1, x2
+
+
+def block_bwd_stored(dy1, dy2, caches, grads):
+    """Ordinary backprop through the forward graph with z1 as an explicit node (Eq. 8), using
+    activations kept from the forward pass."""
+    cF, cG = caches
+    dz1 = dy1 + fn_bwd(dy2, cG, grads)
+    dx2 = dy2 + fn_bwd(dz1, cF, grads)
+    dx1 = dz1
+    return dx1, dx2
+
+
+def block_bwd_reconstruct(y1, y2, dy1, dy2, F, G, eps, grads):
+    """Algorithm 1 (BlockReverse): rebuild the inputs from the outputs, then backprop.
+    Batch statistics are recomputed from the reconstructed tensors; nothing is kept per block.
+    The activations computed while reconstructing are reused for the gradient steps (the 4N form,
+    Section 5 "Implementation")."""
+    z1 = y1
+    gz, cG = fn_fwd(z1, G, eps)
+    x2 = y2 - gz
+    fx, cF = fn_fwd(x2, F, eps)
+    x1 = z1 - fx
+    dz1 = dy1 + fn_bwd(dy2, cG, grads)
+    dx2 = dy2 + fn_bwd(dz1, cF, grads)
+    dx1 = dz1
+    return x1, x2, dx1, dx2
+
+
+# --------------------------------------------------------------------------- classification stack
+
+def softmax_ce(logits, labels):
+    """Mean softmax cross-entropy with max-subtracted log-sum-exp; returns loss and dlogits."""
+    N = logits.shape[0]
+    m = logits.max(axis=1, keepdims=True)
+    e = np.exp(logits - m)
+    lse = m[:, 0] + np.log(e.sum(axis=1))
+    loss = float((lse - logits[np.arange(N), labels]).mean())
+    sm = e / e.sum(axis=1, keepdims=True)
+    sm[np.arange(N), labels] -= 1.0
+    return loss, sm / N
+
+
+def stack_train_grads(net, images, labels, mode):
+    """Forward + backward of the whole stack.
+
+    mode "stored": every block's activations are kept (ordinary backprop).
+    mode "reconstruct": only the inputs of non-reversible layers (stem, max-pool, transitions,
+    head) are kept; each stage is reversed block by block with Algorithm 1 (Section 3.2).
+
+    Returns a dict: logits, loss, pred, grads{name: array}, stored_bytes (activation bytes kept
+    between forward and backward), block_inputs (the (x1,x2) each block saw in the forward) and,
+    in reconstruct mode, recovered (the (x1,x2) Algorithm 1 rebuilt), both keyed (stage, unit).
+    """
+    eps = net["eps"]
+    images = np.asarray(images, np.float64)
+    labels = np.asarray(labels).astype(np.int64)
+    grads, stored, block_inputs, recovered = {}, [], {}, {}
+
+    # ---- forward
+    st = net["stem"]
+    wst = np.asarray(st["W"], np.float64)
+    stored.append(images)
+    h = conv_fwd(images, wst, stride=st["stride"], pad=st["pad"])
+    stem_out_hw = h.shape[2:]
+    pool_idx = None
+    if net["maxpool"]:
+        stored.append(h)                      # nothing of h is needed later except its shape/argmax
+        h, pool_idx = maxpool_fwd(h, 3, 2, 1)
+    stage_fw = []
+    for si, S in enumerate(net["stages"]):
+        tcache = None
+        if S["trans"] is not None:
+            stored.append(h)                  # input of a non-reversible layer is kept
+            h, tcache = fn_fwd(h, [S["trans"]], eps)
+        c = S["c"]
+        x1, x2 = h[:, :c].copy(), h[:, c:].copy()
+        bcaches = []
+        for ui, (F, G) in enumerate(S["units"]):
+            block_inputs[(si, ui)] = (x1, x2)
+            if mode == "stored":
+                x1, x2, bc = block_fwd(x1, x2, F, G, eps, keep=True)
+                bcaches.append(bc)
+                stored += [t for fc in bc for (bn, a, *_r) in fc for t in (bn[0], a)]
+            else:
+                x1, x2 = block_fwd(x1, x2, F, G, eps)
+        h = np.concatenate([x1, x2], axis=1)
+        stage_fw.append((tcache, bcaches, x1, x2))
+    stored.append(h)                          # top activations: needed to start the reversal
+    feat = h.mean(axis=(2, 3))
+    fc = net["fc"]
+    wfc, bfc = np.asarray(fc["W"], np.float64), np.asarray(fc["b"], np.float64)
+    logits = feat @ wfc.T + bfc
+    loss, dlogits = softmax_ce(logits, labels)
+    pred = logits.argmax(axis=1).astype(np.int32)
+
+    # ---- backward
+    grads[fc["name"] + ".W"] = dlogits.T @ feat
+    grads[fc["name"] + ".b"] = dlogits.sum(axis=0)
+    dfeat = dlogits @ wfc
+    Hh, Wh = h.shape[2:]
+    dh = np.broadcast_to(dfeat[:, :, None, None] / (Hh * Wh), h.shape).copy()
+    for si in reversed(range(len(net["stages"]))):
+        S = net["stages"][si]
+        tcache, bcaches, y1, y2 = stage_fw[si]
+        c = S["c"]
+        d1, d2 = dh[:, :c].copy(), dh[:, c:].copy()
+        for ui in reversed(range(len(S["units"]))):
+            F, G = S["units"][ui]
+            if mode == "stored":
+                d1, d2 = block_bwd_stored(d1, d2, bcaches[ui], grads)
+            else:
+                y1, y2, d1, d2 = block_bwd_reconstruct(y1, y2, d1, d2, F, G, eps, grads)
+                recovered[(si, ui)] = (y1, y2)
+        dh = np.concatenate([d1, d2], axis=1)
+        if tcache is not None:
+            dh = fn_bwd(dh, tcache, grads)
+    if pool_idx is not None:
+        dh = maxpool_bwd(dh, pool_idx, stem_out_hw)
+    grads[st["name"] + ".W"] = conv_wgrad(dh, images, wst.shape[2], stride=st["stride"], pad=st["pad"])
+
+    seen, nbytes = set(), 0
+    for t in stored:
+        if id(t) not in seen:
+            seen.add(id(t))
+            nbytes += t.size * 4              # counted at the 4-byte storage width of the method
+    return dict(logits=logits, loss=loss, pred=pred, grads=grads, stored_bytes=nbytes,
+                block_inputs=block_inputs, recovered=recovered, top=(stage_fw[-1][2], stage_fw[-1][3]))
+
+
+def sgd_step(params, grads, velocity, lr, momentum, weight_decay, decayed):
+    """v <- mu v + (g + lambda w) ; w <- w - lr v   (Appendix 6.1: momentum 0.9, weight decay on
+    weights named in `decayed` only)."""
+    new_p, new_v = {}, {}
+    for k, w in params.items():
+        w = np.asarray(w, np.float64)
+        g = grads[k] + (weight_decay * w if k in decayed else 0.0)
+        v = momentum * np.asarray(velocity[k], np.float64) + g
+        new_v[k] = v
+        new_p[k] = w - lr * v
+    return new_p, new_v

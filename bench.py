@@ -1,0 +1,263 @@
+#!/usr/bin/env python
+"""Benchmark: RevNet train-step images/sec on B200 (one replica per GPU, no collectives).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config revnet38] [--impl ours|reference]
+
+A step is one whole train step of the stack (forward, reconstructing backward through every
+stage, SGD update) on one synthetic batch.  Prints ONE JSON line (rank 0).
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "revnet_train_step_images_per_sec"
+UNIT = "images/s"
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm=d["hbm_gbs"], tc_burst=d["bf16_tflops"], tc_sustained=d["bf16_tflops_sustained"], source="measured")
+    return dict(hbm=6650.0, tc_burst=1590.0, tc_sustained=1400.0, source="fallback")
+
+
+# fp32 FMA peak of the CUDA cores: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (max SM clock)
+ALU_FP32_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
+
+KERNEL_BOUND = {  # which roofline a kernel class is measured against
+    "conv_fprop_simt": "alu", "conv_dgrad_simt": "alu", "conv_wgrad_simt": "alu",
+    "conv_fprop_tc": "tensor", "conv_dgrad_tc": "tensor", "conv_wgrad_tc": "tensor",
+}
+
+
+class ClockSampler:
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.idx, self.proc = gpu_index, None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits", "-lms", "100",
+                                          "-i", str(self.idx)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if not self.proc:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, mx, reasons = [], [], set()
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return dict(sm_mhz=float(np.median(sm)) if sm else None, sm_max_mhz=max(mx) if mx else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def cpu_baseline(cfg, sample_n, steps=1):
+    """The oracle, as it stands, on a bounded sample of the workload (reduced batch)."""
+    from oracle import revnet as orc
+    from paper_1707_04585_b200 import synthetic as syn
+    from tests import helpers as hp
+    sc = syn.shrink(cfg, N=sample_n)
+    inp = syn.make_stack_inputs(sc)
+    net = hp.oracle_net(sc, inp["params"])
+    vel = {k: np.zeros_like(v, dtype=np.float64) for k, v in inp["params"].items()}
+    times = []
+    for _ in range(steps):
+        t0 = time.perf_counter()
+        r = orc.stack_train_grads(net, inp["images"], inp["labels"], "reconstruct")
+        orc.sgd_step(inp["params"], r["grads"], vel, sc.lr, sc.momentum, sc.weight_decay, hp.decayed_names(sc))
+        times.append(time.perf_counter() - t0)
+    try:
+        cores = len(os.sched_getaffinity(0))
+    except Exception:
+        cores = os.cpu_count()
+    omp = os.environ.get("OMP_NUM_THREADS")
+    if omp:
+        cores = min(cores, int(omp))
+    return dict(value=sample_n / float(np.mean(times)), unit=UNIT, cores=cores, kind="oracle",
+                sample=f"{steps} train step(s) (forward + reconstructing backward + SGD) on batch {sample_n} of {cfg.N}, fp64",
+                seconds_per_step=float(np.mean(times)))
+
+
+def run_reference(args, cfg):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample = max(2, min(cfg.N, args.ref_batch))
+    t0 = time.perf_counter()
+    cb = cpu_baseline(cfg, sample, steps=1)            # untimed warm-up of caches is not separated: the oracle is timed as it stands
+    k = max(1, min(args.steps, int(60.0 / max(cb["seconds_per_step"], 1e-3))))
+    cb = cpu_baseline(cfg, sample, steps=k)
+    line = dict(metric=METRIC, value=cb["value"], unit=UNIT, n_gpus=args.gpus, steps=k, warmup=1,
+                ms_per_step=cb["seconds_per_step"] * 1e3, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic", impl="reference",
+                config=dict(workload=cfg.name, global_batch=cfg.N, sample_batch=sample),
+                cpu_baseline=dict(value=cb["value"], unit=UNIT, cores=cb["cores"], kind="oracle", sample=cb["sample"]),
+                e2e=dict(value=cb["value"], unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                wall_s=time.perf_counter() - t0)
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args, cfg):
+    import torch
+    import torch.distributed as dist
+    from paper_1707_04585_b200 import binding as B, runner as R, synthetic as syn
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    ctx = B.Context(local)
+    # every rank trains its own replica on its own batch (weak scaling, no exchange step)
+    import dataclasses
+    rcfg = dataclasses.replace(cfg, seed=cfg.seed + 1000 * rank)
+    inp = syn.make_stack_inputs(rcfg)
+    run = R.StackRunner(ctx, rcfg, mode=0)
+    run.load(inp["images"], inp["labels"], inp["params"])
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")     # > 126 MB of L2
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        st = run.step(want_logits=False)
+    barrier()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a, b in ev:
+        flush.zero_()                      # evict L2 between timed iterations (outside the timed span)
+        a.record(stream)
+        st = run.step(want_logits=False)
+        b.record(stream)
+    barrier()
+    dev_ms = sum(a.elapsed_time(b) for a, b in ev)
+    launches = int(st.kernel_launches) * args.steps
+
+    # ---- end to end through the host-buffer entry point: pinned H2D of the batch, D2H of loss + predictions
+    h_img = torch.from_numpy(B.to_nhwc(inp["images"])).pin_memory()
+    h_lab = torch.from_numpy(inp["labels"]).pin_memory()
+    h_loss = torch.zeros(1, dtype=torch.float32).pin_memory()
+    h_pred = torch.zeros(rcfg.N, dtype=torch.int32).pin_memory()
+    for _ in range(2):
+        B.revnet_train_step_host(ctx, run.plan, h_img, h_lab, run.images, run.labels, run.params, run.grads, run.momentum,
+                                 run.act, run.ws, run.loss, run.pred, h_loss, h_pred)
+    barrier()
+    e2e_ms = 0.0
+    for _ in range(args.steps):
+        flush.zero_()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        B.revnet_train_step_host(ctx, run.plan, h_img, h_lab, run.images, run.labels, run.params, run.grads, run.momentum,
+                                 run.act, run.ws, run.loss, run.pred, h_loss, h_pred)   # returns after its own stream sync
+        e2e_ms += (time.perf_counter() - t0) * 1e3
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- per-kernel timing with CUDA events on the launching stream (same process, after the timed steps)
+    B.revnet_profile_enable(ctx, True)
+    psteps = 2
+    for _ in range(psteps):
+        run.step(want_logits=False)
+    prof = B.revnet_profile_summary(ctx)
+    B.revnet_profile_enable(ctx, False)
+    final_loss = float(run.loss.item())
+
+    t = torch.tensor([dev_ms, e2e_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dev_ms, e2e_ms = float(t[0]), float(t[1])
+    if rank == 0:
+        peaks = load_peaks()
+        total_images = rcfg.N * world * args.steps
+        tot = sum(v["ms"] for v in prof.values()) or 1.0
+        top = max(prof.items(), key=lambda kv: kv[1]["ms"])
+        name, rec = top
+        bound = KERNEL_BOUND.get(name, "hbm")
+        avg_s = rec["ms"] / rec["launches"] * 1e-3
+        if bound == "hbm":
+            ach, peak, runit = rec["bytes"] / rec["launches"] / avg_s / 1e9, peaks["hbm"], "GB/s"
+        elif bound == "tensor":
+            ach, peak, runit = rec["flops"] / rec["launches"] / avg_s / 1e12, peaks["tc_sustained"], "TFLOP/s"
+        else:
+            ach, peak, runit = rec["flops"] / rec["launches"] / avg_s / 1e12, ALU_FP32_TFLOPS, "TFLOP/s"
+        roof = dict(bound=bound, achieved=ach, peak=peak, unit=runit, frac=ach / peak, traffic=None, kernel=name,
+                    kernel_share=rec["ms"] / tot, avg_launch_us=avg_s * 1e6, peak_source=peaks["source"],
+                    kernels={k: dict(launches=v["launches"] // psteps, ms_per_step=v["ms"] / psteps, share=v["ms"] / tot,
+                                     gbs=(v["bytes"] / (v["ms"] * 1e-3) / 1e9) if v["ms"] > 0 else None,
+                                     tflops=(v["flops"] / (v["ms"] * 1e-3) / 1e12) if v["ms"] > 0 else None)
+                             for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])})
+        img_bytes = h_img.numel() * 4 + h_lab.numel() * 4
+        line = dict(metric=METRIC, value=total_images / (dev_ms * 1e-3), unit=UNIT, n_gpus=world, steps=args.steps,
+                    warmup=args.warmup, ms_per_step=dev_ms / args.steps, higher_is_better=True, scaling="weak",
+                    vs_baseline=None, dtype="bf16", data="synthetic",
+                    config=dict(workload=cfg.name, global_batch=rcfg.N * world, per_gpu_batch=rcfg.N, image=cfg.img,
+                                parallelism=f"replicas x{world}", l2="flushed between timed steps (256 MB write)",
+                                mode="bf16 conv operands, fp32 accumulate and coupling state"),
+                    e2e=dict(value=total_images / (e2e_ms * 1e-3), unit=UNIT, h2d_bytes_per_step=img_bytes,
+                             d2h_bytes_per_step=4 + 4 * rcfg.N, ms_per_step=e2e_ms / args.steps),
+                    gpu_launches=launches, clocks=clocks, roofline=roof,
+                    activation_bytes=int(st.stored_activation_bytes), workspace_bytes=int(st.workspace_peak_bytes),
+                    flops_per_step=int(st.flops_fwd + st.flops_bwd), final_loss=final_loss)
+        if not args.no_cpu and world == 1:
+            line["cpu_baseline"] = {k: v for k, v in cpu_baseline(cfg, min(cfg.N, args.ref_batch)).items() if k != "seconds_per_step"}
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="revnet38")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--ref-batch", type=int, default=32, help="batch of the bounded CPU-oracle sample")
+    ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    from paper_1707_04585_b200 import synthetic as syn
+    cfg = syn.stack_config(args.config)
+    if args.impl == "reference":
+        run_reference(args, cfg)
+    else:
+        run_ours(args, cfg)
+
+
+if __name__ == "__main__":
+    main()

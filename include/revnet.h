@@ -1,0 +1,201 @@
+/*
+ * revnet.h -- C ABI of the reversible residual network library for NVIDIA B200 (sm_100a).
+ *
+ * The calls follow the paper's statement of the problem (arXiv 1707.04585):
+ *   - a reversible block maps (x1, x2) to (y1, y2) with y1 = x1 + F(x2), y2 = x2 + G(y1)
+ *     (Section 3.1), F and G being chains of BN -> ReLU -> conv layers (Section 2.2, Eq. 2);
+ *   - its backward is given only (y1, y2) and (dy1, dy2) and returns (x1, x2), (dx1, dx2) and
+ *     the parameter gradients (Section 3.2, Algorithm 1);
+ *   - a stack of such blocks keeps only the inputs of its non-reversible layers (Section 3.2).
+ *
+ * Conventions that hold for every call
+ *   - All tensor pointers are DEVICE pointers unless a parameter is marked "host".
+ *   - Activations are NHWC float32.  x1 and x2 (and y1, y2, their gradients) are two separate
+ *     contiguous tensors [N,H,W,c]; x1 holds channels [0,c) of the block input, x2 channels [c,2c).
+ *   - Convolution weights are float32 [Cout][kh][kw][Cin], cross-correlation, zero padding k/2,
+ *     no bias.  BN is train-mode (batch statistics over N,H,W, biased variance); no running
+ *     statistics are kept.
+ *   - The caller owns every buffer.  The library allocates no device memory in any call
+ *     below; scratch comes from the workspace the caller passes.
+ *   - Work is enqueued on the caller's stream (a cudaStream_t passed as void*); calls do not
+ *     synchronise unless stated.  Device pointers must be 16-byte aligned, channel counts
+ *     multiples of 4.
+ *   - Aliasing y1==x1, y2==x2 in revnet_block_fwd and x1==y1, x2==y2, dx1==dy1, dx2==dy2 in
+ *     revnet_block_bwd is legal: that is how a stack runs in place.
+ *   - Gradient outputs are overwritten, not accumulated.
+ *   - Every call returns 0 (REVNET_OK) or a negative revnet_status; the text of the last error
+ *     of a context is available from revnet_last_error.  No exception crosses the ABI.
+ *   - mode 0: convolution operands rounded to bf16, products accumulated in fp32 on the tensor
+ *     cores where the shape allows; mode 1: strict fp32 arithmetic throughout (verification).
+ *     The coupling state (x, y and their gradients) is fp32 in both modes.
+ */
+#ifndef REVNET_H_
+#define REVNET_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    REVNET_OK = 0,
+    REVNET_E_INVALID_ARG = -1,
+    REVNET_E_UNSUPPORTED_SHAPE = -2,
+    REVNET_E_WORKSPACE_TOO_SMALL = -3,
+    REVNET_E_MISALIGNED = -4,
+    REVNET_E_CUDA = -5,
+    REVNET_E_TIMEOUT = -6,
+    REVNET_E_INTERNAL = -7
+} revnet_status;
+
+typedef struct revnet_ctx revnet_ctx;
+typedef struct revnet_plan revnet_plan;
+
+/* Create / destroy a context bound to one CUDA device.  Creation allocates a few hundred
+ * bytes of device memory for status words; nothing else is ever allocated by the library. */
+int revnet_create(revnet_ctx **out, int device);
+int revnet_destroy(revnet_ctx *ctx);
+/* Text of the last error recorded on ctx (never NULL; valid until the next failing call). */
+const char *revnet_last_error(const revnet_ctx *ctx);
+
+/* A residual function: n_layers (1..3) layers, each BN -> ReLU -> conv k x k, stride 1
+ * (Section 2.2, Eq. 2: Basic = c3(c3(x)), Bottleneck = c1(c3(c1(x)))).
+ * cin[0] and cout[n_layers-1] must equal the block's half-channel count c. */
+typedef struct {
+    int n_layers;
+    int k[3];
+    int cin[3];
+    int cout[3];
+} revnet_fn_desc;
+
+typedef struct {
+    int N, H, W, c;          /* x1, x2: [N,H,W,c] each */
+    revnet_fn_desc F, G;
+    float eps;               /* BN epsilon */
+    int mode;                /* 0 = bf16 tensor-core operands, 1 = strict fp32 */
+} revnet_block_desc;
+
+/* Parameters of one residual function (device pointers): W[l] is [cout][k][k][cin],
+ * gamma[l], beta[l] are [cin[l]] (the BN in front of conv l). */
+typedef struct {
+    const float *W[3];
+    const float *gamma[3];
+    const float *beta[3];
+} revnet_fn_params;
+
+/* Gradient outputs of one residual function, same shapes as the parameters. */
+typedef struct {
+    float *dW[3];
+    float *dgamma[3];
+    float *dbeta[3];
+} revnet_fn_grads;
+
+/* Workspace (bytes) that revnet_block_fwd / revnet_block_bwd need for this shape. */
+int revnet_block_workspace_bytes(revnet_ctx *ctx, const revnet_block_desc *desc,
+                                 size_t *fwd_bytes, size_t *bwd_bytes);
+
+/* Block forward (Section 3.1): y1 = x1 + F(x2); y2 = x2 + G(y1). */
+int revnet_block_fwd(revnet_ctx *ctx, const revnet_block_desc *desc,
+                     const float *x1, const float *x2,
+                     const revnet_fn_params *F, const revnet_fn_params *G,
+                     float *y1, float *y2,
+                     void *workspace, size_t workspace_bytes, void *stream);
+
+/* Block backward without stored activations (Algorithm 1): from (y1,y2) and (dy1,dy2) compute
+ * x2 = y2 - G(y1), x1 = y1 - F(x2), dx1 = dy1 + (dG/dz1)^T dy2, dx2 = dy2 + (dF/dx2)^T dx1,
+ * and the gradients of the parameters of F and G.  The activations computed while
+ * reconstructing are reused for the gradient steps (four convolution passes per layer in all,
+ * counting the forward: Section 3.2 "Computational overhead", Section 5.1). */
+int revnet_block_bwd(revnet_ctx *ctx, const revnet_block_desc *desc,
+                     const float *y1, const float *y2, const float *dy1, const float *dy2,
+                     const revnet_fn_params *F, const revnet_fn_params *G,
+                     float *x1, float *x2, float *dx1, float *dx2,
+                     const revnet_fn_grads *gF, const revnet_fn_grads *gG,
+                     void *workspace, size_t workspace_bytes, void *stream);
+
+/* ---- classification stack (Section 3.2: only non-reversible layers keep their inputs) ---- */
+
+typedef struct {
+    int units;         /* reversible units in the stage */
+    int c;             /* channels per half */
+    int w;             /* bottleneck width (kind 2), else 0 */
+    int kind;          /* 0: F,G = one conv3x3; 1: basic (3x3,3x3); 2: bottleneck (1x1,3x3,1x1) */
+    int trans_k;       /* stored BN-ReLU-conv transition in front of the stage (0 = none) */
+    int trans_stride;  /* 1 or 2 */
+} revnet_stage_desc;
+
+#define REVNET_MAX_STAGES 8
+
+typedef struct {
+    int N, img, in_ch, n_classes;
+    int stem_k, stem_stride, stem_cout, maxpool;    /* bare conv stem (+ 3x3/2 max-pool) */
+    int n_stages;
+    revnet_stage_desc stage[REVNET_MAX_STAGES];
+    float eps;
+    int mode;
+    float lr, momentum, weight_decay;               /* SGD (Appendix 6.1); decay on conv/FC weights only */
+    int verify_reconstruction;                      /* debug: keep a copy of each stage input and report
+                                                       max |reconstructed - original| per stage */
+} revnet_stack_desc;
+
+typedef struct {
+    uint64_t stored_activation_bytes;  /* activations kept between forward and backward */
+    uint64_t workspace_peak_bytes;     /* high-water mark of scratch use during the step */
+    uint64_t flops_fwd, flops_bwd;     /* dense conv + FC flops issued (2 per multiply-add) */
+    uint64_t kernel_launches;          /* kernels enqueued by the step */
+    float recon_max_abs[REVNET_MAX_STAGES]; /* filled only with verify_reconstruction */
+    int device_status;                 /* 0, or the code a device-side bounded wait reported */
+} revnet_step_stats;
+
+/* Plan a stack: validates the description and sizes the caller's buffers.
+ * param_count: floats in each of params / grads / momentum.  Parameter order is forward order:
+ * stem W; per stage: [transition gamma, beta, W]; per unit: F layers (gamma, beta, W each) then
+ * G layers; FC W [n_classes][C], FC b.  The activation buffer holds the stored tensors (stem /
+ * max-pool output where a transition follows, one (x1,x2) pair per stage); its size does not
+ * depend on the number of units per stage. */
+int revnet_stack_plan(revnet_ctx *ctx, const revnet_stack_desc *desc, revnet_plan **plan,
+                      size_t *param_count, size_t *activation_bytes, size_t *workspace_bytes);
+int revnet_plan_destroy(revnet_plan *plan);
+
+/* One SGD training step: forward, loss, reconstructing backward through every stage
+ * (Algorithm 1 applied block by block from the stage outputs), SGD-with-momentum update.
+ * images: [N,img,img,in_ch] float32; labels: [N] int32 in [0,n_classes).
+ * loss: 1 float (mean softmax cross-entropy); pred: [N] int32 arg-max (lowest index on ties);
+ * logits: [N][n_classes] or NULL.  params/momentum are updated in place, grads overwritten.
+ * stats (host, may be NULL) is filled from host-side accounting; with verify_reconstruction the
+ * call synchronises the stream to read the per-stage error back. */
+int revnet_train_step(revnet_ctx *ctx, revnet_plan *plan,
+                      const float *images, const int32_t *labels,
+                      float *params, float *grads, float *momentum,
+                      void *activations, void *workspace,
+                      float *loss, int32_t *pred, float *logits,
+                      revnet_step_stats *stats, void *stream);
+
+/* Same step fed from HOST memory: copies images_host / labels_host (pinned memory recommended)
+ * into the device staging buffers images_dev / labels_dev, runs revnet_train_step, copies loss
+ * and pred back to loss_host / pred_host and synchronises the stream. */
+int revnet_train_step_host(revnet_ctx *ctx, revnet_plan *plan,
+                           const float *images_host, const int32_t *labels_host,
+                           float *images_dev, int32_t *labels_dev,
+                           float *params, float *grads, float *momentum,
+                           void *activations, void *workspace,
+                           float *loss_dev, int32_t *pred_dev,
+                           float *loss_host, int32_t *pred_host,
+                           revnet_step_stats *stats, void *stream);
+
+/* ---- per-kernel timing (no counterpart in the paper: measurement support) ----
+ * While enabled, every kernel the library launches on behalf of this context is followed by a
+ * CUDA event on the caller's stream.  revnet_profile_summary waits for the last event and writes
+ * one text line per kernel name: "name<TAB>launches<TAB>total_ms<TAB>algorithmic_bytes<TAB>flops".
+ * The time of a launch is the span between the previous event and its own, so the first record
+ * after enabling is only a boundary.  buf may be NULL with buflen 0 to query `needed`.
+ * Enabling (or disabling) clears earlier records. */
+int revnet_profile_enable(revnet_ctx *ctx, int on);
+int revnet_profile_summary(revnet_ctx *ctx, char *buf, size_t buflen, size_t *needed);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* REVNET_H_ */

@@ -1,0 +1,179 @@
+// C ABI: context management and the block-level entry points.
+#include "common.cuh"
+#include <string.h>
+#include <stdio.h>
+
+static int fail(revnet_ctx *ctx, int code, const std::string &msg) { if (ctx) ctx->err = msg; return code; }
+
+extern "C" int revnet_create(revnet_ctx **out, int device) {
+    if (!out) return REVNET_E_INVALID_ARG;
+    revnet_ctx *c = new revnet_ctx();
+    c->device = device;
+    if (device >= 0) {
+        // device < 0 makes a planning-only context: sizes and layouts can be queried without a GPU
+        int sm = 0;
+        if (cudaSetDevice(device) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
+            cudaMalloc(&c->dev_status, 256) != cudaSuccess || cudaMemset(c->dev_status, 0, 256) != cudaSuccess) {
+            cudaGetLastError();
+            delete c;
+            return REVNET_E_CUDA;
+        }
+        c->sm_count = sm;
+    }
+    *out = c;
+    return REVNET_OK;
+}
+
+extern "C" int revnet_destroy(revnet_ctx *ctx) {
+    if (!ctx) return REVNET_OK;
+    for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
+    if (ctx->dev_status) cudaFree(ctx->dev_status);
+    delete ctx;
+    return REVNET_OK;
+}
+
+extern "C" const char *revnet_last_error(const revnet_ctx *ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+static int check_fn(const revnet_fn_desc &f, int c) {
+    if (f.n_layers < 1 || f.n_layers > 3) return 0;
+    for (int l = 0; l < f.n_layers; l++) {
+        if ((f.k[l] != 1 && f.k[l] != 3) || f.cin[l] < 4 || f.cin[l] % 4 || f.cout[l] < 4 || f.cout[l] % 4) return 0;
+        if (l && f.cin[l] != f.cout[l - 1]) return 0;
+    }
+    return f.cin[0] == c && f.cout[f.n_layers - 1] == c;
+}
+static int check_desc(revnet_ctx *ctx, const revnet_block_desc *d) {
+    if (!ctx || !d) return fail(ctx, REVNET_E_INVALID_ARG, "null descriptor");
+    if (d->N < 1 || d->H < 1 || d->W < 1 || d->c < 4 || (d->mode != 0 && d->mode != 1))
+        return fail(ctx, REVNET_E_INVALID_ARG, "block descriptor: N,H,W >= 1, c >= 4, mode in {0,1}");
+    if (d->c % 4 || !check_fn(d->F, d->c) || !check_fn(d->G, d->c))
+        return fail(ctx, REVNET_E_UNSUPPORTED_SHAPE, "block descriptor: channels must be multiples of 4, kernels 1 or 3, F and G must map c -> c");
+    if ((size_t)d->N * d->H * d->W >= (1u << 30)) return fail(ctx, REVNET_E_UNSUPPORTED_SHAPE, "block descriptor: too many pixels");
+    return REVNET_OK;
+}
+
+static std::vector<Layer> layers_of(const revnet_fn_desc &f, const revnet_fn_params *p, const revnet_fn_grads *g) {
+    std::vector<Layer> v(f.n_layers);
+    for (int l = 0; l < f.n_layers; l++) {
+        v[l].cin = f.cin[l]; v[l].cout = f.cout[l]; v[l].k = f.k[l]; v[l].stride = 1;
+        if (p) { v[l].W = p->W[l]; v[l].gamma = p->gamma[l]; v[l].beta = p->beta[l]; }
+        if (g) { v[l].dW = g->dW[l]; v[l].dgamma = g->dgamma[l]; v[l].dbeta = g->dbeta[l]; }
+    }
+    return v;
+}
+
+static bool aligned16(std::initializer_list<const void *> ps) {
+    for (const void *p : ps) if ((uintptr_t)p & 15) return false;
+    return true;
+}
+static bool fn_ptrs_ok(const revnet_fn_desc &f, const revnet_fn_params *p, const revnet_fn_grads *g, bool need_g, bool *misaligned) {
+    if (!p || (need_g && !g)) return false;
+    for (int l = 0; l < f.n_layers; l++) {
+        if (!p->W[l] || !p->gamma[l] || !p->beta[l]) return false;
+        if (!aligned16({p->W[l], p->gamma[l], p->beta[l]})) *misaligned = true;
+        if (need_g) {
+            if (!g->dW[l] || !g->dgamma[l] || !g->dbeta[l]) return false;
+            if (!aligned16({g->dW[l], g->dgamma[l], g->dbeta[l]})) *misaligned = true;
+        }
+    }
+    return true;
+}
+
+extern "C" int revnet_block_workspace_bytes(revnet_ctx *ctx, const revnet_block_desc *d, size_t *fwd_bytes, size_t *bwd_bytes) {
+    int rc = check_desc(ctx, d);
+    if (rc) return rc;
+    Geom g{d->N, d->H, d->W};
+    float *fake = (float *)0x1000;
+    for (int pass = 0; pass < 2; pass++) {
+        Exec ex; ex.ctx = ctx; ex.dry = true; ex.ws.dry = true; ex.mode = d->mode; ex.eps = d->eps;
+        auto F = layers_of(d->F, nullptr, nullptr), G = layers_of(d->G, nullptr, nullptr);
+        if (pass == 0) block_forward(ex, g, d->c, F, G, fake, fake, fake, fake);
+        else block_backward(ex, g, d->c, F, G, fake, fake, fake, fake, fake, fake, fake, fake);
+        size_t *o = pass == 0 ? fwd_bytes : bwd_bytes;
+        if (o) *o = ex.ws.peak + 256;
+    }
+    return REVNET_OK;
+}
+
+static int finish(revnet_ctx *ctx, Exec &ex, const char *who) {
+    if (ex.ws.overflow) return fail(ctx, REVNET_E_WORKSPACE_TOO_SMALL, std::string(who) + ": workspace too small");
+    if (ex.failed) return REVNET_E_CUDA;
+    return REVNET_OK;
+}
+
+extern "C" int revnet_block_fwd(revnet_ctx *ctx, const revnet_block_desc *d, const float *x1, const float *x2,
+                                const revnet_fn_params *Fp, const revnet_fn_params *Gp, float *y1, float *y2,
+                                void *workspace, size_t workspace_bytes, void *stream) {
+    int rc = check_desc(ctx, d);
+    if (rc) return rc;
+    bool mis = false;
+    if (!x1 || !x2 || !y1 || !y2 || !workspace || !fn_ptrs_ok(d->F, Fp, nullptr, false, &mis) || !fn_ptrs_ok(d->G, Gp, nullptr, false, &mis))
+        return fail(ctx, REVNET_E_INVALID_ARG, "revnet_block_fwd: null pointer");
+    if (mis || !aligned16({x1, x2, y1, y2, workspace})) return fail(ctx, REVNET_E_MISALIGNED, "revnet_block_fwd: pointers must be 16-byte aligned");
+    size_t need = 0;
+    revnet_block_workspace_bytes(ctx, d, &need, nullptr);
+    if (workspace_bytes < need) return fail(ctx, REVNET_E_WORKSPACE_TOO_SMALL, "revnet_block_fwd: workspace too small");
+    Exec ex; ex.ctx = ctx; ex.dry = false; ex.mode = d->mode; ex.eps = d->eps; ex.stream = (cudaStream_t)stream;
+    ex.ws.dry = false; ex.ws.base = (char *)workspace; ex.ws.cap = workspace_bytes;
+    block_forward(ex, Geom{d->N, d->H, d->W}, d->c, layers_of(d->F, Fp, nullptr), layers_of(d->G, Gp, nullptr),
+                  (float *)x1, (float *)x2, y1, y2);
+    return finish(ctx, ex, "revnet_block_fwd");
+}
+
+extern "C" int revnet_block_bwd(revnet_ctx *ctx, const revnet_block_desc *d, const float *y1, const float *y2,
+                                const float *dy1, const float *dy2, const revnet_fn_params *Fp, const revnet_fn_params *Gp,
+                                float *x1, float *x2, float *dx1, float *dx2, const revnet_fn_grads *gF, const revnet_fn_grads *gG,
+                                void *workspace, size_t workspace_bytes, void *stream) {
+    int rc = check_desc(ctx, d);
+    if (rc) return rc;
+    bool mis = false;
+    if (!y1 || !y2 || !dy1 || !dy2 || !x1 || !x2 || !dx1 || !dx2 || !workspace ||
+        !fn_ptrs_ok(d->F, Fp, gF, true, &mis) || !fn_ptrs_ok(d->G, Gp, gG, true, &mis))
+        return fail(ctx, REVNET_E_INVALID_ARG, "revnet_block_bwd: null pointer");
+    if (mis || !aligned16({y1, y2, dy1, dy2, x1, x2, dx1, dx2, workspace}))
+        return fail(ctx, REVNET_E_MISALIGNED, "revnet_block_bwd: pointers must be 16-byte aligned");
+    size_t need = 0;
+    revnet_block_workspace_bytes(ctx, d, nullptr, &need);
+    if (workspace_bytes < need) return fail(ctx, REVNET_E_WORKSPACE_TOO_SMALL, "revnet_block_bwd: workspace too small");
+    Exec ex; ex.ctx = ctx; ex.dry = false; ex.mode = d->mode; ex.eps = d->eps; ex.stream = (cudaStream_t)stream;
+    ex.ws.dry = false; ex.ws.base = (char *)workspace; ex.ws.cap = workspace_bytes;
+    block_backward(ex, Geom{d->N, d->H, d->W}, d->c, layers_of(d->F, Fp, gF), layers_of(d->G, Gp, gG),
+                   y1, y2, dy1, dy2, x1, x2, dx1, dx2);
+    return finish(ctx, ex, "revnet_block_bwd");
+}
+
+// ---- per-kernel timing
+extern "C" int revnet_profile_enable(revnet_ctx *ctx, int on) {
+    if (!ctx) return REVNET_E_INVALID_ARG;
+    ctx->profiling = on != 0;
+    ctx->prof.clear();
+    ctx->ev_used = 0;
+    return REVNET_OK;
+}
+
+extern "C" int revnet_profile_summary(revnet_ctx *ctx, char *buf, size_t buflen, size_t *needed) {
+    if (!ctx || (!buf && buflen)) return REVNET_E_INVALID_ARG;
+    struct Acc { std::string name; uint64_t n = 0; double ms = 0, bytes = 0, flops = 0; };
+    std::vector<Acc> acc;
+    if (!ctx->prof.empty() && cudaEventSynchronize(ctx->prof.back().ev) != cudaSuccess)
+        return fail(ctx, REVNET_E_CUDA, std::string("revnet_profile_summary: ") + cudaGetErrorString(cudaGetLastError()));
+    for (size_t i = 1; i < ctx->prof.size(); i++) {
+        const ProfRec &r = ctx->prof[i];
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, ctx->prof[i - 1].ev, r.ev) != cudaSuccess) { cudaGetLastError(); continue; }
+        Acc *a = nullptr;
+        for (auto &x : acc) if (x.name == r.name) { a = &x; break; }
+        if (!a) { acc.push_back(Acc()); a = &acc.back(); a->name = r.name; }
+        a->n++; a->ms += ms; a->bytes += r.bytes; a->flops += r.flops;
+    }
+    std::string out;
+    char line[256];
+    for (auto &a : acc) {
+        snprintf(line, sizeof line, "%s\t%llu\t%.6f\t%.0f\t%.0f\n", a.name.c_str(), (unsigned long long)a.n, a.ms, a.bytes, a.flops);
+        out += line;
+    }
+    if (needed) *needed = out.size() + 1;
+    if (buflen) { size_t n = out.size() < buflen - 1 ? out.size() : buflen - 1; memcpy(buf, out.data(), n); buf[n] = 0; }
+    return REVNET_OK;
+}

@@ -1,0 +1,125 @@
+// Residual-function and reversible-block engine: sequences the kernels for
+//   forward   y1 = x1 + F(x2); y2 = x2 + G(y1)                                   (Section 3.1)
+//   backward  Algorithm 1: x2 = y2 - G(y1); backprop G; x1 = y1 - F(x2); backprop F
+// The tensors a residual function produces while being recomputed stay in the workspace and
+// feed its own backprop, so each conv layer costs four passes per step in all.
+#include "common.cuh"
+
+// dispatch: tensor-core kernels take the shapes they support in mode 0, the fp32 kernels the rest
+bool conv_fprop_tc(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign);
+bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da);
+bool conv_wgrad_tc(Exec &ex, const void *g, const void *a, Geom gi, const Layer &L, float *dW);
+
+static void conv_fprop(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign) {
+    const bool b16 = ex.mode == 0;
+    if (b16 && conv_fprop_tc(ex, a, gi, L, out, partner, sign)) return;
+    conv_fprop_simt(ex, a, b16, gi, L, out, partner, sign);
+}
+static void conv_dgrad(Exec &ex, const void *g, Geom gi, const Layer &L, float *da) {
+    const bool b16 = ex.mode == 0;
+    if (b16 && conv_dgrad_tc(ex, g, gi, L, da)) return;
+    conv_dgrad_simt(ex, g, b16, gi, L, da);
+}
+static void conv_wgrad(Exec &ex, const void *g, const void *a, Geom gi, const Layer &L, float *dW) {
+    const bool b16 = ex.mode == 0;
+    if (b16 && conv_wgrad_tc(ex, g, a, gi, L, dW)) return;
+    conv_wgrad_simt(ex, g, b16, a, b16, gi, L, dW);
+}
+
+static size_t esz(const Exec &ex) { return ex.mode == 0 ? 2 : 4; }
+
+// out = partner + sign * Fn(u).  With `saved`, every layer's activated input, BN input and BN
+// statistics are left in the workspace (the caller releases them after the backward).
+void fn_forward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, Pair partner, Pair out, int sign,
+                FnSaved *saved, bool skip_last_conv) {
+    const int L = (int)layers.size();
+    const bool b16 = ex.mode == 0;
+    size_t outer = ex.ws.mark();
+    Pair t = u;
+    Geom gi = g;
+    if (saved) { saved->a.clear(); saved->t.clear(); saved->bn.clear(); saved->gin = g; }
+    for (int l = 0; l < L; l++) {
+        const Layer &ly = layers[l];
+        const size_t P = gi.P();
+        BnState st = bn_alloc(ex, ly.cin);
+        bn_stats(ex, t, P, ly.gamma, ly.beta, st);
+        void *a = ex.ws.alloc(P * ly.cin * esz(ex));
+        bn_relu_apply(ex, t, P, st, a, b16);
+        Geom go{gi.N, conv_out(gi.H, ly.k, ly.stride), conv_out(gi.W, ly.k, ly.stride)};
+        if (saved) { saved->a.push_back(a); saved->bn.push_back(st); }
+        if (l == L - 1) {
+            if (!skip_last_conv) conv_fprop(ex, a, gi, ly, out, partner, sign);
+        } else {
+            float *tn = ex.ws.get<float>(go.P() * ly.cout);
+            conv_fprop(ex, a, gi, ly, single(tn, ly.cout), Pair{}, 0);
+            if (saved) saved->t.push_back(tn);
+            t = single(tn, ly.cout);
+        }
+        gi = go;
+    }
+    if (!saved) ex.ws.release(outer);
+}
+
+// dgin_out = add + (dFn/du)^T gup ; parameter gradients through the layers' pointers.
+void fn_backward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, FnSaved &saved, Pair gup,
+                 Pair add, Pair dgin_out) {
+    const int L = (int)layers.size();
+    const bool b16 = ex.mode == 0;
+    size_t outer = ex.ws.mark();
+    // geometry of every layer's input
+    std::vector<Geom> gin(L + 1);
+    gin[0] = g;
+    for (int l = 0; l < L; l++)
+        gin[l + 1] = Geom{gin[l].N, conv_out(gin[l].H, layers[l].k, layers[l].stride), conv_out(gin[l].W, layers[l].k, layers[l].stride)};
+    // upstream gradient as one operand tensor
+    const void *gcur;
+    {
+        const int C = gup.C();
+        if (!b16 && gup.c1 == 0) gcur = gup.p0;
+        else {
+            void *buf = ex.ws.alloc(gin[L].P() * C * esz(ex));
+            concat_cast(ex, gup, gin[L].P(), buf, b16);
+            gcur = buf;
+        }
+    }
+    for (int l = L - 1; l >= 0; l--) {
+        const Layer &ly = layers[l];
+        const size_t P = gin[l].P();
+        conv_wgrad(ex, gcur, saved.a[l], gin[l], ly, ly.dW);
+        float *da = ex.ws.get<float>(P * ly.cin);
+        conv_dgrad(ex, gcur, gin[l], ly, da);
+        if (l == 0) {
+            // add.p0 == nullptr: the gradient is stored without a partner (stored transitions)
+            bn_relu_bwd(ex, da, u, P, saved.bn[0], ly.gamma, ly.dgamma, ly.dbeta, nullptr, false, add, dgin_out);
+        } else {
+            void *dt = ex.ws.alloc(P * ly.cin * esz(ex));
+            bn_relu_bwd(ex, da, single(saved.t[l - 1], ly.cin), P, saved.bn[l], ly.gamma, ly.dgamma, ly.dbeta,
+                        dt, b16, Pair{}, Pair{});
+            gcur = dt;
+        }
+    }
+    ex.ws.release(outer);
+}
+
+void block_forward(Exec &ex, Geom g, int c, const std::vector<Layer> &F, const std::vector<Layer> &G,
+                   float *x1, float *x2, float *y1, float *y2) {
+    fn_forward(ex, g, single(x2, c), F, single(x1, c), single(y1, c), +1, nullptr, false);
+    fn_forward(ex, g, single(y1, c), G, single(x2, c), single(y2, c), +1, nullptr, false);
+}
+
+void block_backward(Exec &ex, Geom g, int c, const std::vector<Layer> &F, const std::vector<Layer> &G,
+                    const float *y1, const float *y2, const float *dy1, const float *dy2,
+                    float *x1, float *x2, float *dx1, float *dx2) {
+    FnSaved sv;
+    size_t m = ex.ws.mark();
+    // x2 = y2 - G(z1), z1 = y1
+    fn_forward(ex, g, single((float *)y1, c), G, single((float *)y2, c), single(x2, c), -1, &sv, false);
+    // dz1 = dy1 + (dG/dz1)^T dy2 ; dW_G
+    fn_backward(ex, g, single((float *)y1, c), G, sv, single((float *)dy2, c), single((float *)dy1, c), single(dx1, c));
+    ex.ws.release(m);
+    // x1 = z1 - F(x2)
+    fn_forward(ex, g, single(x2, c), F, single((float *)y1, c), single(x1, c), -1, &sv, false);
+    // dx2 = dy2 + (dF/dx2)^T dz1 ; dW_F ; dx1 = dz1 (already in place)
+    fn_backward(ex, g, single(x2, c), F, sv, single(dx1, c), single((float *)dy2, c), single(dx2, c));
+    ex.ws.release(m);
+}

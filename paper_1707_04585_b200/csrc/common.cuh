@@ -1,0 +1,147 @@
+// Internal declarations shared by the library's translation units.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include <string>
+#include <vector>
+#include "../../include/revnet.h"
+
+typedef __nv_bfloat16 bf16;
+
+// ---------------------------------------------------------------- context
+struct ProfRec { const char *name; double bytes, flops; cudaEvent_t ev; };
+struct revnet_ctx {
+    int device = 0;
+    int sm_count = 148;
+    std::string err;
+    int *dev_status = nullptr;   // device word for bounded-wait time-outs
+    void *encode_tiled = nullptr; // driver entry point for tensor-map encoding
+    // per-kernel timing (revnet_profile_*): one event after every launch while enabled
+    bool profiling = false;
+    std::vector<ProfRec> prof;
+    std::vector<cudaEvent_t> ev_pool;
+    size_t ev_used = 0;
+    cudaEvent_t next_event();
+};
+
+// A tensor of C = c0 + c1 channels stored as two NHWC tensors: channels [0,c0) in p0 (row
+// stride c0) and [c0,c0+c1) in p1 (row stride c1).  c1 == 0: one plain tensor.
+struct Pair {
+    float *p0;
+    float *p1;
+    int c0, c1;
+    __host__ __device__ int C() const { return c0 + c1; }
+    __device__ __forceinline__ float *at(size_t row, int ch) const {
+        return ch < c0 ? p0 + row * c0 + ch : p1 + row * c1 + (ch - c0);
+    }
+};
+static inline Pair single(float *p, int C) { return Pair{p, nullptr, C, 0}; }
+static inline Pair halves(float *a, float *b, int c) { return Pair{a, b, c, c}; }
+
+// Bump allocator over the caller's workspace; in dry mode it only measures.
+struct Arena {
+    char *base = nullptr;
+    size_t off = 0, cap = 0, peak = 0;
+    bool dry = true;
+    bool overflow = false;
+    void *alloc(size_t bytes) {
+        size_t a = (off + 255) & ~size_t(255);
+        off = a + bytes;
+        if (off > peak) peak = off;
+        if (!dry && off > cap) { overflow = true; return nullptr; }
+        return dry ? (void *)(uintptr_t)(0x1000 + a) : base + a;   // non-null fake address in dry mode
+    }
+    template <class T> T *get(size_t n) { return (T *)alloc(n * sizeof(T)); }
+    size_t mark() const { return off; }
+    void release(size_t m) { off = m; }
+};
+
+// Everything a kernel launcher needs.
+struct Exec {
+    revnet_ctx *ctx = nullptr;
+    cudaStream_t stream = nullptr;
+    Arena ws;
+    bool dry = true;       // true: size the workspace and count work, launch nothing
+    int mode = 0;          // 0 bf16 tensor-core operands, 1 strict fp32
+    float eps = 1e-5f;
+    uint64_t flops = 0;    // dense conv/FC flops issued
+    uint64_t launches = 0;
+    bool failed = false;
+    // called after every launch: error check, launch count and (when profiling) an event;
+    // bytes / flops are the algorithmic traffic and work of that launch
+    void check(const char *what, double bytes = 0, double flops = 0);
+    void mark(const char *what);   // profiling boundary that is not a kernel (copies, step start)
+};
+
+// One BN -> ReLU -> conv layer with its parameter and gradient pointers.
+struct Layer {
+    int cin = 0, cout = 0, k = 1, stride = 1;
+    const float *W = nullptr, *gamma = nullptr, *beta = nullptr;
+    float *dW = nullptr, *dgamma = nullptr, *dbeta = nullptr;
+    const bf16 *Wp_fprop = nullptr;   // bf16 [cout][k][k][cin_pad]           (mode 0)
+    const bf16 *Wp_dgrad = nullptr;   // bf16 [cin][k][k][cout_pad], taps mirrored (mode 0)
+};
+
+// Per-BN statistics kept between a layer's forward and its backward.
+struct BnState {
+    float *scale, *shift, *mean, *rstd;   // [C] each
+};
+
+struct Geom { int N, H, W; size_t P() const { return (size_t)N * H * W; } };
+
+// ---------------------------------------------------------------- elementwise.cu
+BnState bn_alloc(Exec &ex, int C);
+// batch statistics of t ([P,C]) -> scale = gamma*rstd, shift = beta - mean*scale, mean, rstd
+void bn_stats(Exec &ex, Pair t, size_t P, const float *gamma, const float *beta, BnState st);
+// a = relu(scale*t + shift) written as one [P,C] tensor of float (strict) or bf16
+void bn_relu_apply(Exec &ex, Pair t, size_t P, BnState st, void *a, bool a_bf16);
+// BN+ReLU backward: da [P,C] fp32; t the BN input; writes dgamma, dbeta and
+//   out = dt                  (out_single: float or bf16 [P,C])   when add.p0 == nullptr
+//   out_pair = add + dt       (fp32 pair)                        otherwise
+void bn_relu_bwd(Exec &ex, const float *da, Pair t, size_t P, BnState st, const float *gamma,
+                 float *dgamma, float *dbeta, void *out_single, bool out_bf16, Pair add, Pair out_pair);
+// copy a pair into one [P,C] tensor of float or bf16
+void concat_cast(Exec &ex, Pair src, size_t P, void *dst, bool dst_bf16);
+void maxpool_fwd(Exec &ex, const float *in, float *out, int N, int H, int W, int C);
+void maxpool_bwd(Exec &ex, const float *in, const float *dout, float *din, int N, int H, int W, int C);
+void head_fwd(Exec &ex, Pair y, int N, int HW, const float *Wfc, const float *bfc, const int32_t *labels,
+              int n_classes, float *feat, float *logits, float *dlogits, float *loss, int32_t *pred);
+void head_bwd(Exec &ex, Pair dy, int N, int HW, const float *Wfc, const float *feat, const float *dlogits,
+              int n_classes, float *dWfc, float *dbfc, float *dfeat);
+void sgd_update(Exec &ex, float *params, const float *grads, float *mom, size_t n,
+                const uint32_t *seg_end, const uint8_t *seg_decay, int n_seg,
+                float lr, float momentum, float wd);
+void max_abs_diff(Exec &ex, const float *a, const float *b, size_t n, float *out /*1 float, pre-zeroed*/);
+void fill_zero(Exec &ex, void *p, size_t bytes);
+
+// ---------------------------------------------------------------- conv_simt.cu
+// Operand element type of the activated tensor / upstream gradient: float or bf16.
+// out = partner + sign*conv(a)   (sign 0: out = conv(a), partner unused)
+void conv_fprop_simt(Exec &ex, const void *a, bool a_bf16, Geom gi, const Layer &L, Pair out, Pair partner, int sign);
+void conv_dgrad_simt(Exec &ex, const void *g, bool g_bf16, Geom gi, const Layer &L, float *da);
+void conv_wgrad_simt(Exec &ex, const void *g, bool g_bf16, const void *a, bool a_bf16, Geom gi, const Layer &L, float *dW);
+
+// ---------------------------------------------------------------- block.cu
+struct FnSaved;   // activations kept from a residual function's (re)computation
+// out = partner + sign * Fn(u); if saved != nullptr the per-layer tensors stay in the workspace
+// skip_last_conv: only rebuild the saved tensors (used to re-derive a stored layer's operands)
+void fn_forward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, Pair partner, Pair out, int sign,
+                FnSaved *saved, bool skip_last_conv);
+// dgin_out = add + (dFn/du)^T gup, parameter gradients written through the layers' pointers
+void fn_backward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, FnSaved &saved, Pair gup,
+                 Pair add, Pair dgin_out);
+struct FnSaved {
+    std::vector<void *> a;        // activated input of each conv
+    std::vector<float *> t;       // BN input of each layer beyond the first (conv outputs)
+    std::vector<BnState> bn;
+    Geom gin;
+};
+void block_forward(Exec &ex, Geom g, int c, const std::vector<Layer> &F, const std::vector<Layer> &G,
+                   float *x1, float *x2, float *y1, float *y2);
+void block_backward(Exec &ex, Geom g, int c, const std::vector<Layer> &F, const std::vector<Layer> &G,
+                    const float *y1, const float *y2, const float *dy1, const float *dy2,
+                    float *x1, float *x2, float *dx1, float *dx2);
+
+static inline int conv_out(int in, int k, int s) { return (in + 2 * (k / 2) - k) / s + 1; }

@@ -1,0 +1,479 @@
+// HBM-bound kernels: BN batch statistics, BN+ReLU apply and backward, concat/cast, max-pool,
+// classification head, SGD.  All reductions are two-stage with a fixed summation order, so a
+// residual function recomputed in the backward pass reproduces the forward bit for bit.
+#include "common.cuh"
+#include <math.h>
+
+cudaEvent_t revnet_ctx::next_event() {
+    if (ev_used == ev_pool.size()) {
+        cudaEvent_t e;
+        cudaEventCreate(&e);
+        ev_pool.push_back(e);
+    }
+    return ev_pool[ev_used++];
+}
+
+void Exec::check(const char *what, double bytes, double flops) {
+    launches++;
+    cudaError_t e = cudaPeekAtLastError();
+    if (e != cudaSuccess && !failed) {
+        failed = true;
+        ctx->err = std::string(what) + ": " + cudaGetErrorString(e);
+    }
+    if (ctx->profiling) {
+        cudaEvent_t ev = ctx->next_event();
+        cudaEventRecord(ev, stream);
+        ctx->prof.push_back(ProfRec{what, bytes, flops, ev});
+    }
+}
+void Exec::mark(const char *what) {
+    if (ctx->profiling && !dry) {
+        cudaEvent_t ev = ctx->next_event();
+        cudaEventRecord(ev, stream);
+        ctx->prof.push_back(ProfRec{what, 0, 0, ev});
+    }
+}
+
+static inline int cdiv(size_t a, size_t b) { return (int)((a + b - 1) / b); }
+
+__device__ __forceinline__ float4 ld4(const float *p) { return *reinterpret_cast<const float4 *>(p); }
+__device__ __forceinline__ void st4(float *p, float4 v) { *reinterpret_cast<float4 *>(p) = v; }
+__device__ __forceinline__ void st4(bf16 *p, float4 v) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+    uint2 u;
+    u.x = *reinterpret_cast<uint32_t *>(&lo);
+    u.y = *reinterpret_cast<uint32_t *>(&hi);
+    *reinterpret_cast<uint2 *>(p) = u;
+}
+
+// ------------------------------------------------------------------ column reductions
+// Shape of the launch used by every per-channel reduction over a [P,C] tensor: a CTA owns a slab
+// of SW channel quads and a range of rows; threadIdx.y strides the rows.
+struct RedShape { int SW, RPP, slabs, chunks, rows_per_cta; };
+static RedShape red_shape(size_t P, int C, int sm) {
+    RedShape r;
+    int C4 = C / 4;
+    r.SW = C4 < 128 ? C4 : 128;
+    r.RPP = 256 / r.SW; if (r.RPP < 1) r.RPP = 1;
+    r.slabs = cdiv(C4, r.SW);
+    size_t want = (size_t)sm * 4 / r.slabs; if (want < 1) want = 1;
+    size_t rows = (P + want - 1) / want;
+    size_t min_rows = (size_t)r.RPP * 8;
+    if (rows < min_rows) rows = min_rows;
+    r.rows_per_cta = (int)rows;
+    r.chunks = cdiv(P, rows);
+    return r;
+}
+
+// part layout: [chunk][2][C]
+template <int MODE>   // 0: sum t, sum t^2 ; 1: sum db, sum db*xhat (BN+ReLU backward)
+__global__ void col_reduce_kernel(Pair t, const float *__restrict__ da, size_t P, int rows_per_cta,
+                                  const float *__restrict__ scale, const float *__restrict__ shift,
+                                  const float *__restrict__ mean, const float *__restrict__ rstd,
+                                  float *__restrict__ part) {
+    extern __shared__ float4 sm4[];
+    const int C = t.C(), C4 = C / 4, SW = blockDim.x, RPP = blockDim.y;
+    const int q = blockIdx.y * SW + threadIdx.x;
+    const bool valid = q < C4;
+    const size_t r0 = (size_t)blockIdx.x * rows_per_cta;
+    size_t r1 = r0 + rows_per_cta; if (r1 > P) r1 = P;
+    float4 s = make_float4(0, 0, 0, 0), ss = s;
+    if (valid) {
+        float4 sc, sh, mu, rs;
+        if (MODE == 1) { sc = ld4(scale + q * 4); sh = ld4(shift + q * 4); mu = ld4(mean + q * 4); rs = ld4(rstd + q * 4); }
+        for (size_t r = r0 + threadIdx.y; r < r1; r += RPP) {
+            float4 v = ld4(t.at(r, q * 4));
+            if (MODE == 0) {
+                s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+                ss.x += v.x * v.x; ss.y += v.y * v.y; ss.z += v.z * v.z; ss.w += v.w * v.w;
+            } else {
+                float4 g = ld4(da + r * C + q * 4);
+                float dx = fmaf(sc.x, v.x, sh.x) > 0.f ? g.x : 0.f, dy = fmaf(sc.y, v.y, sh.y) > 0.f ? g.y : 0.f;
+                float dz = fmaf(sc.z, v.z, sh.z) > 0.f ? g.z : 0.f, dw = fmaf(sc.w, v.w, sh.w) > 0.f ? g.w : 0.f;
+                s.x += dx; s.y += dy; s.z += dz; s.w += dw;
+                ss.x += dx * (v.x - mu.x) * rs.x; ss.y += dy * (v.y - mu.y) * rs.y;
+                ss.z += dz * (v.z - mu.z) * rs.z; ss.w += dw * (v.w - mu.w) * rs.w;
+            }
+        }
+    }
+    sm4[(threadIdx.y * SW + threadIdx.x) * 2 + 0] = s;
+    sm4[(threadIdx.y * SW + threadIdx.x) * 2 + 1] = ss;
+    __syncthreads();
+    if (threadIdx.y == 0 && valid) {
+        for (int y = 1; y < RPP; y++) {
+            float4 a = sm4[(y * SW + threadIdx.x) * 2], b = sm4[(y * SW + threadIdx.x) * 2 + 1];
+            s.x += a.x; s.y += a.y; s.z += a.z; s.w += a.w;
+            ss.x += b.x; ss.y += b.y; ss.z += b.z; ss.w += b.w;
+        }
+        st4(part + ((size_t)blockIdx.x * 2 + 0) * C + q * 4, s);
+        st4(part + ((size_t)blockIdx.x * 2 + 1) * C + q * 4, ss);
+    }
+}
+
+__global__ void bn_stats_finalize(const float *__restrict__ part, int chunks, int C, double invP, float eps,
+                                  const float *__restrict__ gamma, const float *__restrict__ beta,
+                                  float *scale, float *shift, float *mean, float *rstd) {
+    int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    double s = 0, ss = 0;
+    for (int i = 0; i < chunks; i++) { s += part[((size_t)i * 2) * C + c]; ss += part[((size_t)i * 2 + 1) * C + c]; }
+    double mu = s * invP, var = ss * invP - mu * mu;
+    if (var < 0) var = 0;
+    float r = (float)(1.0 / sqrt(var + (double)eps));
+    float sc = gamma[c] * r;
+    scale[c] = sc; shift[c] = beta[c] - (float)mu * sc; mean[c] = (float)mu; rstd[c] = r;
+}
+
+// coef: [3][C] = gamma*rstd, gamma*rstd*dbeta/M, gamma*rstd*dgamma/M
+__global__ void bn_bwd_finalize(const float *__restrict__ part, int chunks, int C, double invP,
+                                const float *__restrict__ gamma, const float *__restrict__ rstd,
+                                float *dgamma, float *dbeta, float *coef) {
+    int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C) return;
+    double s = 0, ss = 0;
+    for (int i = 0; i < chunks; i++) { s += part[((size_t)i * 2) * C + c]; ss += part[((size_t)i * 2 + 1) * C + c]; }
+    dbeta[c] = (float)s; dgamma[c] = (float)ss;
+    double gr = (double)gamma[c] * (double)rstd[c];
+    coef[c] = (float)gr; coef[C + c] = (float)(gr * s * invP); coef[2 * C + c] = (float)(gr * ss * invP);
+}
+
+BnState bn_alloc(Exec &ex, int C) {
+    BnState st;
+    float *p = ex.ws.get<float>((size_t)4 * C);
+    st.scale = p; st.shift = p + C; st.mean = p + 2 * C; st.rstd = p + 3 * C;
+    return st;
+}
+
+void bn_stats(Exec &ex, Pair t, size_t P, const float *gamma, const float *beta, BnState st) {
+    const int C = t.C();
+    RedShape r = red_shape(P, C, ex.ctx->sm_count);
+    size_t m = ex.ws.mark();
+    float *part = ex.ws.get<float>((size_t)r.chunks * 2 * C);
+    if (!ex.dry) {
+        dim3 grid(r.chunks, r.slabs), block(r.SW, r.RPP);
+        col_reduce_kernel<0><<<grid, block, (size_t)r.SW * r.RPP * 32, ex.stream>>>(t, nullptr, P, r.rows_per_cta,
+                                                                                 nullptr, nullptr, nullptr, nullptr, part);
+        ex.check("bn_stats_partial", (double)P * C * 4);
+        bn_stats_finalize<<<cdiv(C, 128), 128, 0, ex.stream>>>(part, r.chunks, C, 1.0 / (double)P, ex.eps, gamma, beta,
+                                                              st.scale, st.shift, st.mean, st.rstd);
+        ex.check("bn_stats_finalize");
+    }
+    ex.ws.release(m);
+}
+
+template <class TO>
+__global__ void bn_relu_apply_kernel(Pair t, size_t nquads, int C4, const float *__restrict__ scale,
+                                     const float *__restrict__ shift, TO *__restrict__ a) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
+        size_t row = i / C4; int q = (int)(i - row * C4);
+        float4 v = ld4(t.at(row, q * 4)), sc = ld4(scale + q * 4), sh = ld4(shift + q * 4);
+        v.x = fmaxf(fmaf(sc.x, v.x, sh.x), 0.f); v.y = fmaxf(fmaf(sc.y, v.y, sh.y), 0.f);
+        v.z = fmaxf(fmaf(sc.z, v.z, sh.z), 0.f); v.w = fmaxf(fmaf(sc.w, v.w, sh.w), 0.f);
+        st4(a + i * 4, v);
+    }
+}
+
+static int ew_grid(size_t n, int sm) {
+    size_t g = (n + 255) / 256, cap = (size_t)sm * 8;
+    return (int)(g < cap ? (g ? g : 1) : cap);
+}
+
+void bn_relu_apply(Exec &ex, Pair t, size_t P, BnState st, void *a, bool a_bf16) {
+    if (ex.dry) return;
+    const int C4 = t.C() / 4; size_t nq = P * C4;
+    if (a_bf16) bn_relu_apply_kernel<bf16><<<ew_grid(nq, ex.ctx->sm_count), 256, 0, ex.stream>>>(t, nq, C4, st.scale, st.shift, (bf16 *)a);
+    else bn_relu_apply_kernel<float><<<ew_grid(nq, ex.ctx->sm_count), 256, 0, ex.stream>>>(t, nq, C4, st.scale, st.shift, (float *)a);
+    ex.check("bn_relu_apply", (double)P * t.C() * (a_bf16 ? 6 : 8));
+}
+
+// dt = coef0*db - coef1 - coef2*xhat ; db = da*[scale*t+shift > 0]
+// OUT 0: out[P,C] = dt (float or bf16) ; 1: outp = dt (fp32 pair) ; 2: outp = add + dt
+template <class TO, int OUT>
+__global__ void bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, size_t nquads, int C4,
+                                         const float *__restrict__ scale, const float *__restrict__ shift,
+                                         const float *__restrict__ mean, const float *__restrict__ rstd,
+                                         const float *__restrict__ coef, TO *__restrict__ out, Pair add, Pair outp) {
+    const int C = C4 * 4;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
+        size_t row = i / C4; int q = (int)(i - row * C4), c = q * 4;
+        float4 v = ld4(t.at(row, c)), g = ld4(da + i * 4);
+        float4 sc = ld4(scale + c), sh = ld4(shift + c), mu = ld4(mean + c), rs = ld4(rstd + c);
+        float4 k0 = ld4(coef + c), k1 = ld4(coef + C + c), k2 = ld4(coef + 2 * C + c), o;
+        o.x = k0.x * (fmaf(sc.x, v.x, sh.x) > 0.f ? g.x : 0.f) - k1.x - k2.x * ((v.x - mu.x) * rs.x);
+        o.y = k0.y * (fmaf(sc.y, v.y, sh.y) > 0.f ? g.y : 0.f) - k1.y - k2.y * ((v.y - mu.y) * rs.y);
+        o.z = k0.z * (fmaf(sc.z, v.z, sh.z) > 0.f ? g.z : 0.f) - k1.z - k2.z * ((v.z - mu.z) * rs.z);
+        o.w = k0.w * (fmaf(sc.w, v.w, sh.w) > 0.f ? g.w : 0.f) - k1.w - k2.w * ((v.w - mu.w) * rs.w);
+        if (OUT == 2) {
+            float4 p = ld4(add.at(row, c));
+            o.x += p.x; o.y += p.y; o.z += p.z; o.w += p.w;
+        }
+        if (OUT == 0) st4(out + i * 4, o);
+        else st4(outp.at(row, c), o);
+    }
+}
+
+void bn_relu_bwd(Exec &ex, const float *da, Pair t, size_t P, BnState st, const float *gamma,
+                 float *dgamma, float *dbeta, void *out_single, bool out_bf16, Pair add, Pair out_pair) {
+    const int C = t.C(), C4 = C / 4;
+    RedShape r = red_shape(P, C, ex.ctx->sm_count);
+    size_t m = ex.ws.mark();
+    float *part = ex.ws.get<float>((size_t)r.chunks * 2 * C);
+    float *coef = ex.ws.get<float>((size_t)3 * C);
+    if (!ex.dry) {
+        dim3 grid(r.chunks, r.slabs), block(r.SW, r.RPP);
+        col_reduce_kernel<1><<<grid, block, (size_t)r.SW * r.RPP * 32, ex.stream>>>(t, da, P, r.rows_per_cta, st.scale, st.shift,
+                                                                                 st.mean, st.rstd, part);
+        ex.check("bn_bwd_partial", (double)P * C * 8);
+        bn_bwd_finalize<<<cdiv(C, 128), 128, 0, ex.stream>>>(part, r.chunks, C, 1.0 / (double)P, gamma, st.rstd, dgamma, dbeta, coef);
+        ex.check("bn_bwd_finalize");
+        size_t nq = P * C4; int g = ew_grid(nq, ex.ctx->sm_count);
+#define RV_ARGS da, t, nq, C4, st.scale, st.shift, st.mean, st.rstd, coef
+        if (out_pair.p0 && add.p0) bn_relu_bwd_apply_kernel<float, 2><<<g, 256, 0, ex.stream>>>(RV_ARGS, nullptr, add, out_pair);
+        else if (out_pair.p0) bn_relu_bwd_apply_kernel<float, 1><<<g, 256, 0, ex.stream>>>(RV_ARGS, nullptr, add, out_pair);
+        else if (out_bf16) bn_relu_bwd_apply_kernel<bf16, 0><<<g, 256, 0, ex.stream>>>(RV_ARGS, (bf16 *)out_single, add, out_pair);
+        else bn_relu_bwd_apply_kernel<float, 0><<<g, 256, 0, ex.stream>>>(RV_ARGS, (float *)out_single, add, out_pair);
+#undef RV_ARGS
+        ex.check("bn_relu_bwd_apply", (double)P * C * (out_pair.p0 ? (add.p0 ? 16 : 12) : (out_bf16 ? 10 : 12)));
+    }
+    ex.ws.release(m);
+}
+
+template <class TO>
+__global__ void concat_cast_kernel(Pair src, size_t nquads, int C4, TO *__restrict__ dst) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
+        size_t row = i / C4; int q = (int)(i - row * C4);
+        st4(dst + i * 4, ld4(src.at(row, q * 4)));
+    }
+}
+
+void concat_cast(Exec &ex, Pair src, size_t P, void *dst, bool dst_bf16) {
+    if (ex.dry) return;
+    const int C4 = src.C() / 4; size_t nq = P * C4; int g = ew_grid(nq, ex.ctx->sm_count);
+    if (dst_bf16) concat_cast_kernel<bf16><<<g, 256, 0, ex.stream>>>(src, nq, C4, (bf16 *)dst);
+    else concat_cast_kernel<float><<<g, 256, 0, ex.stream>>>(src, nq, C4, (float *)dst);
+    ex.check("concat_cast", (double)P * src.C() * (dst_bf16 ? 6 : 8));
+}
+
+// ------------------------------------------------------------------ max-pool 3x3 stride 2 pad 1 (NHWC)
+__global__ void maxpool_fwd_kernel(const float *__restrict__ in, float *__restrict__ out, int N, int H, int W, int C4, int Ho, int Wo) {
+    size_t n = (size_t)N * Ho * Wo * C4;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        int q = (int)(i % C4); size_t p = i / C4;
+        int j = (int)(p % Wo); p /= Wo; int io = (int)(p % Ho); int b = (int)(p / Ho);
+        float4 m = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+        for (int kh = 0; kh < 3; kh++) for (int kw = 0; kw < 3; kw++) {
+            int y = io * 2 + kh - 1, x = j * 2 + kw - 1;
+            if (y < 0 || y >= H || x < 0 || x >= W) continue;
+            float4 v = ld4(in + (((size_t)b * H + y) * W + x) * C4 * 4 + q * 4);
+            m.x = fmaxf(m.x, v.x); m.y = fmaxf(m.y, v.y); m.z = fmaxf(m.z, v.z); m.w = fmaxf(m.w, v.w);
+        }
+        st4(out + i * 4, m);
+    }
+}
+
+// Gradient goes to the first maximum met in (kh,kw) row-major scan of each window.  Gather form:
+// each input element visits the (at most four) windows that cover it, in a fixed order.
+__global__ void maxpool_bwd_kernel(const float *__restrict__ in, const float *__restrict__ dout, float *__restrict__ din,
+                                   int N, int H, int W, int C, int Ho, int Wo) {
+    size_t n = (size_t)N * H * W * C;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        int c = (int)(i % C); size_t p = i / C;
+        int x = (int)(p % W); p /= W; int y = (int)(p % H); int b = (int)(p / H);
+        const float self = in[i];
+        float acc = 0.f;
+        for (int io = (y + 1 - 2 + 1) / 2; io <= (y + 1) / 2; io++) {
+            if (io < 0 || io >= Ho || io * 2 - 1 > y || io * 2 + 1 < y) continue;
+            for (int j = (x + 1 - 2 + 1) / 2; j <= (x + 1) / 2; j++) {
+                if (j < 0 || j >= Wo || j * 2 - 1 > x || j * 2 + 1 < x) continue;
+                // is (y,x) the first maximum of window (io,j)?
+                bool first = true;
+                for (int kh = 0; kh < 3 && first; kh++) for (int kw = 0; kw < 3; kw++) {
+                    int yy = io * 2 + kh - 1, xx = j * 2 + kw - 1;
+                    if (yy < 0 || yy >= H || xx < 0 || xx >= W) continue;
+                    float v = in[(((size_t)b * H + yy) * W + xx) * C + c];
+                    bool before = (yy < y) || (yy == y && xx < x);
+                    if (v > self || (before && v == self)) { first = false; break; }
+                }
+                if (first) acc += dout[(((size_t)b * Ho + io) * Wo + j) * C + c];
+            }
+        }
+        din[i] = acc;
+    }
+}
+
+void maxpool_fwd(Exec &ex, const float *in, float *out, int N, int H, int W, int C) {
+    if (ex.dry) return;
+    int Ho = conv_out(H, 3, 2), Wo = conv_out(W, 3, 2);
+    size_t n = (size_t)N * Ho * Wo * (C / 4);
+    maxpool_fwd_kernel<<<ew_grid(n, ex.ctx->sm_count), 256, 0, ex.stream>>>(in, out, N, H, W, C / 4, Ho, Wo);
+    ex.check("maxpool_fwd");
+}
+void maxpool_bwd(Exec &ex, const float *in, const float *dout, float *din, int N, int H, int W, int C) {
+    if (ex.dry) return;
+    int Ho = conv_out(H, 3, 2), Wo = conv_out(W, 3, 2);
+    size_t n = (size_t)N * H * W * C;
+    maxpool_bwd_kernel<<<ew_grid(n, ex.ctx->sm_count), 256, 0, ex.stream>>>(in, dout, din, N, H, W, C, Ho, Wo);
+    ex.check("maxpool_bwd");
+}
+
+// ------------------------------------------------------------------ head: avgpool -> FC -> softmax CE -> argmax
+__global__ void avgpool_kernel(Pair y, int HW, float *__restrict__ feat) {
+    extern __shared__ float4 sm4[];
+    const int C = y.C(), C4 = C / 4, SW = blockDim.x, RPP = blockDim.y;
+    const int q = blockIdx.y * SW + threadIdx.x, n = blockIdx.x;
+    const bool valid = q < C4;
+    float4 s = make_float4(0, 0, 0, 0);
+    if (valid)
+        for (int r = threadIdx.y; r < HW; r += RPP) {
+            float4 v = ld4(y.at((size_t)n * HW + r, q * 4));
+            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+        }
+    sm4[threadIdx.y * SW + threadIdx.x] = s;
+    __syncthreads();
+    if (threadIdx.y == 0 && valid) {
+        for (int yy = 1; yy < RPP; yy++) { float4 a = sm4[yy * SW + threadIdx.x]; s.x += a.x; s.y += a.y; s.z += a.z; s.w += a.w; }
+        float inv = 1.f / (float)HW;
+        s.x *= inv; s.y *= inv; s.z *= inv; s.w *= inv;
+        st4(feat + (size_t)n * C + q * 4, s);
+    }
+}
+
+// one warp per (n,k)
+__global__ void fc_fwd_kernel(const float *__restrict__ feat, const float *__restrict__ Wfc, const float *__restrict__ bfc,
+                              int N, int C, int K, float *__restrict__ logits) {
+    int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (warp >= N * K) return;
+    int n = warp / K, k = warp - n * K;
+    float s = 0.f;
+    for (int c = lane; c < C; c += 32) s = fmaf(feat[(size_t)n * C + c], Wfc[(size_t)k * C + c], s);
+    for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) logits[warp] = s + bfc[k];
+}
+
+// one warp per sample: stable log-sum-exp, dlogits = (softmax - onehot)/N, arg-max (lowest index on ties)
+__global__ void softmax_ce_kernel(const float *__restrict__ logits, const int32_t *__restrict__ labels, int N, int K,
+                                  float *__restrict__ dlogits, float *__restrict__ loss_n, int32_t *__restrict__ pred) {
+    int n = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (n >= N) return;
+    const float *z = logits + (size_t)n * K;
+    float m = -INFINITY; int mi = 0x7fffffff;
+    for (int k = lane; k < K; k += 32) { float v = z[k]; if (v > m) { m = v; mi = k; } }
+    for (int o = 16; o; o >>= 1) {
+        float om = __shfl_xor_sync(0xffffffffu, m, o); int oi = __shfl_xor_sync(0xffffffffu, mi, o);
+        if (om > m || (om == m && oi < mi)) { m = om; mi = oi; }
+    }
+    float s = 0.f;
+    for (int k = lane; k < K; k += 32) s += expf(z[k] - m);
+    for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    const int lab = labels[n];
+    const float inv = 1.f / s, invN = 1.f / (float)N;
+    for (int k = lane; k < K; k += 32) dlogits[(size_t)n * K + k] = (expf(z[k] - m) * inv - (k == lab ? 1.f : 0.f)) * invN;
+    if (lane == 0) { loss_n[n] = m + logf(s) - z[lab]; pred[n] = mi; }
+}
+
+__global__ void mean_kernel(const float *__restrict__ v, int N, float *out) {
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        double s = 0; for (int i = 0; i < N; i++) s += v[i];
+        *out = (float)(s / N);
+    }
+}
+
+void head_fwd(Exec &ex, Pair y, int N, int HW, const float *Wfc, const float *bfc, const int32_t *labels,
+              int K, float *feat, float *logits, float *dlogits, float *loss, int32_t *pred) {
+    const int C = y.C();
+    ex.flops += 2ull * N * C * K;
+    size_t m = ex.ws.mark();
+    float *loss_n = ex.ws.get<float>(N);
+    if (!ex.dry) {
+        int C4 = C / 4, SW = C4 < 128 ? C4 : 128, RPP = 256 / SW; if (RPP < 1) RPP = 1;
+        dim3 grid(N, cdiv(C4, SW)), block(SW, RPP);
+        avgpool_kernel<<<grid, block, (size_t)SW * RPP * 16, ex.stream>>>(y, HW, feat);
+        ex.check("avgpool");
+        fc_fwd_kernel<<<cdiv((size_t)N * K * 32, 256), 256, 0, ex.stream>>>(feat, Wfc, bfc, N, C, K, logits);
+        ex.check("fc_fwd");
+        softmax_ce_kernel<<<cdiv((size_t)N * 32, 256), 256, 0, ex.stream>>>(logits, labels, N, K, dlogits, loss_n, pred);
+        ex.check("softmax_ce");
+        mean_kernel<<<1, 32, 0, ex.stream>>>(loss_n, N, loss);
+        ex.check("loss_mean");
+    }
+    ex.ws.release(m);
+}
+
+__global__ void fc_wgrad_kernel(const float *__restrict__ dlogits, const float *__restrict__ feat, int N, int C, int K,
+                                float *__restrict__ dW, float *__restrict__ db) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < (size_t)K * C) {
+        int k = (int)(i / C), c = (int)(i - (size_t)k * C);
+        float s = 0.f;
+        for (int n = 0; n < N; n++) s = fmaf(dlogits[(size_t)n * K + k], feat[(size_t)n * C + c], s);
+        dW[i] = s;
+    }
+    if (i < (size_t)K) { float s = 0.f; for (int n = 0; n < N; n++) s += dlogits[(size_t)n * K + i]; db[i] = s; }
+}
+__global__ void fc_dgrad_kernel(const float *__restrict__ dlogits, const float *__restrict__ Wfc, int N, int C, int K,
+                                float scale, float *__restrict__ dfeat) {
+    size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= (size_t)N * C) return;
+    int n = (int)(i / C), c = (int)(i - (size_t)n * C);
+    float s = 0.f;
+    for (int k = 0; k < K; k++) s = fmaf(dlogits[(size_t)n * K + k], Wfc[(size_t)k * C + c], s);
+    dfeat[i] = s * scale;
+}
+__global__ void avgpool_bwd_kernel(const float *__restrict__ dfeat, Pair dy, size_t nquads, int C4, int HW) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
+        size_t row = i / C4; int q = (int)(i - row * C4); size_t n = row / HW;
+        st4(dy.at(row, q * 4), ld4(dfeat + n * C4 * 4 + q * 4));
+    }
+}
+
+void head_bwd(Exec &ex, Pair dy, int N, int HW, const float *Wfc, const float *feat, const float *dlogits,
+              int K, float *dWfc, float *dbfc, float *dfeat) {
+    const int C = dy.C();
+    ex.flops += 4ull * N * C * K;
+    if (ex.dry) return;
+    fc_wgrad_kernel<<<cdiv((size_t)K * C, 256), 256, 0, ex.stream>>>(dlogits, feat, N, C, K, dWfc, dbfc);
+    ex.check("fc_wgrad");
+    fc_dgrad_kernel<<<cdiv((size_t)N * C, 256), 256, 0, ex.stream>>>(dlogits, Wfc, N, C, K, 1.f / (float)HW, dfeat);
+    ex.check("fc_dgrad");
+    size_t nq = (size_t)N * HW * (C / 4);
+    avgpool_bwd_kernel<<<ew_grid(nq, ex.ctx->sm_count), 256, 0, ex.stream>>>(dfeat, dy, nq, C / 4, HW);
+    ex.check("avgpool_bwd");
+}
+
+// ------------------------------------------------------------------ SGD with momentum and weight decay
+__global__ void sgd_kernel(float *__restrict__ p, const float *__restrict__ g, float *__restrict__ v, size_t n,
+                           const uint32_t *__restrict__ seg_end, const uint8_t *__restrict__ seg_decay, int n_seg,
+                           float lr, float mu, float wd) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        int lo = 0, hi = n_seg - 1;                  // first segment whose end is > i
+        while (lo < hi) { int mid = (lo + hi) >> 1; if (seg_end[mid] > i) hi = mid; else lo = mid + 1; }
+        float w = p[i];
+        float gg = g[i] + (seg_decay[lo] ? wd * w : 0.f);
+        float vv = fmaf(mu, v[i], gg);
+        v[i] = vv;
+        p[i] = w - lr * vv;
+    }
+}
+void sgd_update(Exec &ex, float *params, const float *grads, float *mom, size_t n, const uint32_t *seg_end,
+                const uint8_t *seg_decay, int n_seg, float lr, float momentum, float wd) {
+    if (ex.dry) return;
+    sgd_kernel<<<ew_grid(n, ex.ctx->sm_count), 256, 0, ex.stream>>>(params, grads, mom, n, seg_end, seg_decay, n_seg, lr, momentum, wd);
+    ex.check("sgd", (double)n * 20);
+}
+
+__global__ void max_abs_diff_kernel(const float *__restrict__ a, const float *__restrict__ b, size_t n, float *out) {
+    float m = 0.f;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
+        m = fmaxf(m, fabsf(a[i] - b[i]));
+    for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0) atomicMax(reinterpret_cast<int *>(out), __float_as_int(m));   // m >= 0
+}
+void max_abs_diff(Exec &ex, const float *a, const float *b, size_t n, float *out) {
+    if (ex.dry) return;
+    max_abs_diff_kernel<<<ew_grid(n, ex.ctx->sm_count), 256, 0, ex.stream>>>(a, b, n, out);
+    ex.check("max_abs_diff");
+}
+void fill_zero(Exec &ex, void *p, size_t bytes) {
+    if (ex.dry) return;
+    cudaMemsetAsync(p, 0, bytes, ex.stream);
+}

@@ -1,0 +1,331 @@
+// Stack driver: a classification network of reversible stages that keeps only the inputs of its
+// non-reversible layers (Section 3.2).  Each stage owns ONE (x1,x2) buffer pair; its units run in
+// place on it in the forward pass, and Algorithm 1 walks it back in place in the backward pass,
+// so the activation footprint does not depend on the number of units.
+#include "common.cuh"
+#include <string.h>
+#include <array>
+#include <stdlib.h>
+
+struct LayerSlot { int cin, cout, k, stride; size_t off_gamma, off_beta, off_W; };   // offsets in floats; stem: gamma/beta unused
+
+struct StagePlan {
+    int c, H, units;
+    bool has_trans;
+    LayerSlot trans;
+    std::vector<std::vector<LayerSlot>> F, G;
+    size_t off_x1, off_x2;          // bytes into the activation buffer
+    size_t off_v1, off_v2;          // verify copies (bytes), valid with verify_reconstruction
+};
+
+struct revnet_plan {
+    revnet_ctx *ctx;
+    revnet_stack_desc d;
+    LayerSlot stem;
+    int stemH;                      // stem output resolution
+    int poolH;                      // after max-pool (== stemH without)
+    bool stem_direct;               // stem writes straight into stage 0's pair
+    size_t off_stem_out, off_pool_out;
+    std::vector<StagePlan> st;
+    size_t off_fcW, off_fcb;
+    int feat_C;
+    size_t n_params, act_bytes, ws_bytes;
+    uint64_t stored_bytes;
+    std::vector<uint32_t> seg_end; std::vector<uint8_t> seg_decay;
+    void *pinned = nullptr;         // seg_end then seg_decay, page-locked for async upload
+    bool pinned_is_malloc = false;  // no CUDA device at plan time: plain host memory instead
+};
+
+static std::vector<std::array<int, 3>> fn_shape(int kind, int c, int w) {
+    if (kind == 0) return {{c, c, 3}};
+    if (kind == 1) return {{c, c, 3}, {c, c, 3}};
+    return {{c, w, 1}, {w, w, 3}, {w, c, 1}};
+}
+
+static Layer bind(const LayerSlot &s, float *params, float *grads) {
+    Layer L;
+    L.cin = s.cin; L.cout = s.cout; L.k = s.k; L.stride = s.stride;
+    L.W = params + s.off_W; L.gamma = params + s.off_gamma; L.beta = params + s.off_beta;
+    L.dW = grads + s.off_W; L.dgamma = grads + s.off_gamma; L.dbeta = grads + s.off_beta;
+    return L;
+}
+static std::vector<Layer> bind(const std::vector<LayerSlot> &v, float *params, float *grads) {
+    std::vector<Layer> o;
+    for (auto &s : v) o.push_back(bind(s, params, grads));
+    return o;
+}
+
+// Runs (or, with ex.dry, only sizes) one training step.
+static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32_t *labels, float *params, float *grads,
+                     float *mom, char *act, float *loss, int32_t *pred, float *logits_out, revnet_step_stats *stats,
+                     float **recon_dev) {
+    const revnet_stack_desc &d = pl->d;
+    const int N = d.N, S = d.n_stages;
+    auto actf = [&](size_t off) { return (float *)(act + off); };
+
+    ex.mark("step_begin");
+    // ---- step-long scratch
+    const size_t nseg = pl->seg_end.size();
+    uint32_t *seg_end = ex.ws.get<uint32_t>(nseg);
+    uint8_t *seg_decay = ex.ws.get<uint8_t>(nseg);
+    if (!ex.dry) {
+        cudaMemcpyAsync(seg_end, pl->pinned, nseg * 4, cudaMemcpyHostToDevice, ex.stream);
+        cudaMemcpyAsync(seg_decay, (char *)pl->pinned + nseg * 4, nseg, cudaMemcpyHostToDevice, ex.stream);
+    }
+    size_t gmax = (size_t)N * pl->stemH * pl->stemH * d.stem_cout;           // gradient w.r.t. stem / pool output
+    for (auto &s : pl->st) { size_t e = (size_t)N * s.H * s.H * 2 * s.c; if (e > gmax) gmax = e; }
+    float *gbuf[2] = {ex.ws.get<float>(gmax), ex.ws.get<float>(gmax)};
+    const int K = d.n_classes, FC = pl->feat_C;
+    float *feat = ex.ws.get<float>((size_t)N * FC), *dfeat = ex.ws.get<float>((size_t)N * FC);
+    float *logits = logits_out ? logits_out : ex.ws.get<float>((size_t)N * K);
+    float *dlogits = ex.ws.get<float>((size_t)N * K);
+    float *recon = ex.ws.get<float>(REVNET_MAX_STAGES);
+    if (recon_dev) *recon_dev = recon;
+    if (d.verify_reconstruction) fill_zero(ex, recon, REVNET_MAX_STAGES * sizeof(float));
+
+    // ---- forward
+    Layer stem = bind(pl->stem, params, grads);
+    Geom gimg{N, d.img, d.img};
+    StagePlan &s0 = pl->st[0];
+    if (pl->stem_direct)
+        conv_fprop_simt(ex, images, false, gimg, stem, halves(actf(s0.off_x1), actf(s0.off_x2), s0.c), Pair{}, 0);
+    else
+        conv_fprop_simt(ex, images, false, gimg, stem, single(actf(pl->off_stem_out), d.stem_cout), Pair{}, 0);
+    Pair prev = single(actf(pl->off_stem_out), d.stem_cout);
+    int prevH = pl->stemH;
+    if (d.maxpool) {
+        maxpool_fwd(ex, actf(pl->off_stem_out), actf(pl->off_pool_out), N, pl->stemH, pl->stemH, d.stem_cout);
+        prev = single(actf(pl->off_pool_out), d.stem_cout);
+        prevH = pl->poolH;
+    }
+    for (int si = 0; si < S; si++) {
+        StagePlan &s = pl->st[si];
+        float *x1 = actf(s.off_x1), *x2 = actf(s.off_x2);
+        Geom g{N, s.H, s.H};
+        if (s.has_trans) {
+            std::vector<Layer> T{bind(s.trans, params, grads)};
+            fn_forward(ex, Geom{N, prevH, prevH}, prev, T, Pair{}, halves(x1, x2, s.c), 0, nullptr, false);
+        }
+        if (d.verify_reconstruction && !ex.dry) {
+            size_t b = g.P() * s.c * sizeof(float);
+            cudaMemcpyAsync(actf(s.off_v1), x1, b, cudaMemcpyDeviceToDevice, ex.stream);
+            cudaMemcpyAsync(actf(s.off_v2), x2, b, cudaMemcpyDeviceToDevice, ex.stream);
+        }
+        for (int u = 0; u < s.units; u++)
+            block_forward(ex, g, s.c, bind(s.F[u], params, grads), bind(s.G[u], params, grads), x1, x2, x1, x2);
+        prev = halves(x1, x2, s.c);
+        prevH = s.H;
+    }
+    StagePlan &top = pl->st[S - 1];
+    head_fwd(ex, prev, N, top.H * top.H, params + pl->off_fcW, params + pl->off_fcb, labels, K, feat, logits, dlogits, loss, pred);
+    const uint64_t flops_fwd = ex.flops;
+
+    // ---- backward
+    int gi = (S - 1) & 1;
+    {
+        size_t half = (size_t)N * top.H * top.H * top.c;
+        head_bwd(ex, halves(gbuf[gi], gbuf[gi] + half, top.c), N, top.H * top.H, params + pl->off_fcW, feat, dlogits, K,
+                 grads + pl->off_fcW, grads + pl->off_fcb, dfeat);
+    }
+    for (int si = S - 1; si >= 0; si--) {
+        StagePlan &s = pl->st[si];
+        float *x1 = actf(s.off_x1), *x2 = actf(s.off_x2);
+        Geom g{N, s.H, s.H};
+        size_t half = g.P() * s.c;
+        float *d1 = gbuf[gi], *d2 = gbuf[gi] + half;
+        for (int u = s.units - 1; u >= 0; u--)
+            block_backward(ex, g, s.c, bind(s.F[u], params, grads), bind(s.G[u], params, grads), x1, x2, d1, d2, x1, x2, d1, d2);
+        if (d.verify_reconstruction) {
+            max_abs_diff(ex, x1, actf(s.off_v1), half, recon + si);
+            max_abs_diff(ex, x2, actf(s.off_v2), half, recon + si);
+        }
+        if (s.has_trans) {
+            std::vector<Layer> T{bind(s.trans, params, grads)};
+            Pair tin; int tH; Pair gout;
+            if (si > 0) {
+                StagePlan &p = pl->st[si - 1];
+                tin = halves(actf(p.off_x1), actf(p.off_x2), p.c); tH = p.H;
+                size_t ph = (size_t)N * p.H * p.H * p.c;
+                gout = halves(gbuf[gi ^ 1], gbuf[gi ^ 1] + ph, p.c);
+            } else {
+                tin = single(actf(d.maxpool ? pl->off_pool_out : pl->off_stem_out), d.stem_cout); tH = pl->poolH;
+                gout = single(gbuf[gi ^ 1], d.stem_cout);
+            }
+            FnSaved sv;
+            size_t m = ex.ws.mark();
+            fn_forward(ex, Geom{N, tH, tH}, tin, T, Pair{}, Pair{}, 0, &sv, true);   // rebuild the operands from the stored input
+            fn_backward(ex, Geom{N, tH, tH}, tin, T, sv, halves(d1, d2, s.c), Pair{}, gout);
+            ex.ws.release(m);
+            gi ^= 1;
+        }
+    }
+    // gradient w.r.t. the stem output now sits in gbuf[gi]: a pair if the stem feeds stage 0 directly
+    {
+        size_t m = ex.ws.mark();
+        const float *gstem;
+        size_t Pstem = (size_t)N * pl->stemH * pl->stemH;
+        if (pl->stem_direct) {
+            float *cat = ex.ws.get<float>(Pstem * d.stem_cout);
+            concat_cast(ex, halves(gbuf[gi], gbuf[gi] + Pstem * s0.c, s0.c), Pstem, cat, false);
+            gstem = cat;
+        } else if (d.maxpool) {
+            float *gp = ex.ws.get<float>(Pstem * d.stem_cout);
+            maxpool_bwd(ex, actf(pl->off_stem_out), gbuf[gi], gp, N, pl->stemH, pl->stemH, d.stem_cout);
+            gstem = gp;
+        } else {
+            gstem = gbuf[gi];
+        }
+        conv_wgrad_simt(ex, gstem, false, images, false, gimg, stem, stem.dW);
+        ex.ws.release(m);
+    }
+    sgd_update(ex, params, grads, mom, pl->n_params, seg_end, seg_decay, (int)nseg, d.lr, d.momentum, d.weight_decay);
+
+    if (stats) {
+        stats->stored_activation_bytes = pl->stored_bytes;
+        stats->workspace_peak_bytes = ex.ws.peak;
+        stats->flops_fwd = flops_fwd;
+        stats->flops_bwd = ex.flops - flops_fwd;
+        stats->kernel_launches = ex.launches;
+        stats->device_status = 0;
+        for (int i = 0; i < REVNET_MAX_STAGES; i++) stats->recon_max_abs[i] = 0.f;
+    }
+}
+
+static int fail(revnet_ctx *ctx, int code, const std::string &msg) { if (ctx) ctx->err = msg; return code; }
+
+extern "C" int revnet_stack_plan(revnet_ctx *ctx, const revnet_stack_desc *desc, revnet_plan **plan_out,
+                                 size_t *param_count, size_t *activation_bytes, size_t *workspace_bytes) {
+    if (!ctx || !desc || !plan_out) return fail(ctx, REVNET_E_INVALID_ARG, "revnet_stack_plan: null argument");
+    const revnet_stack_desc &d = *desc;
+    if (d.N < 1 || d.img < 1 || d.in_ch < 1 || d.n_classes < 2 || d.n_stages < 1 || d.n_stages > REVNET_MAX_STAGES)
+        return fail(ctx, REVNET_E_INVALID_ARG, "revnet_stack_plan: bad N/img/in_ch/n_classes/n_stages");
+    if ((d.stem_k != 3 && d.stem_k != 7) || (d.stem_stride != 1 && d.stem_stride != 2) || d.stem_cout % 4)
+        return fail(ctx, REVNET_E_UNSUPPORTED_SHAPE, "revnet_stack_plan: stem must be 3x3 or 7x7, stride 1 or 2, cout % 4 == 0");
+    if (d.mode != 0 && d.mode != 1) return fail(ctx, REVNET_E_INVALID_ARG, "revnet_stack_plan: mode must be 0 or 1");
+    revnet_plan *pl = new revnet_plan();
+    pl->ctx = ctx; pl->d = d;
+    size_t off = 0;
+    auto take = [&](size_t n, bool decay) { size_t o = off; off += n; pl->seg_end.push_back((uint32_t)off); pl->seg_decay.push_back(decay); return o; };
+    auto slot = [&](int cin, int cout, int k, int stride, bool bn) {
+        LayerSlot s{cin, cout, k, stride, 0, 0, 0};
+        if (bn) { s.off_gamma = take(cin, false); s.off_beta = take(cin, false); }
+        s.off_W = take((size_t)cout * k * k * cin, true);
+        return s;
+    };
+    pl->stem = slot(d.in_ch, d.stem_cout, d.stem_k, d.stem_stride, false);
+    pl->stemH = conv_out(d.img, d.stem_k, d.stem_stride);
+    pl->poolH = d.maxpool ? conv_out(pl->stemH, 3, 2) : pl->stemH;
+    int cprev = d.stem_cout, H = pl->poolH;
+    size_t aoff = 0;
+    auto atake = [&](size_t bytes) { size_t o = aoff; aoff += (bytes + 255) & ~size_t(255); return o; };
+    pl->stem_direct = !d.maxpool && d.stage[0].trans_k == 0;
+    pl->stored_bytes = (uint64_t)d.N * d.img * d.img * d.in_ch * 4;
+    pl->off_stem_out = pl->off_pool_out = 0;
+    if (!pl->stem_direct) {
+        size_t b = (size_t)d.N * pl->stemH * pl->stemH * d.stem_cout * 4;
+        pl->off_stem_out = atake(b); pl->stored_bytes += b;
+        if (d.maxpool) { size_t pb = (size_t)d.N * H * H * d.stem_cout * 4; pl->off_pool_out = atake(pb); pl->stored_bytes += pb; }
+    }
+    for (int si = 0; si < d.n_stages; si++) {
+        const revnet_stage_desc &sd = d.stage[si];
+        bool bad = sd.units < 1 || sd.c < 4 || sd.c % 4 || sd.kind < 0 || sd.kind > 2 || (sd.kind == 2 && (sd.w < 4 || sd.w % 4));
+        bad = bad || (sd.trans_k != 0 && sd.trans_k != 1 && sd.trans_k != 3) || (sd.trans_k && sd.trans_stride != 1 && sd.trans_stride != 2);
+        // a stage without a transition is only possible directly behind a stem that needs no pooling
+        bad = bad || (sd.trans_k == 0 && (si > 0 || d.maxpool || cprev != 2 * sd.c));
+        if (bad) { delete pl; return fail(ctx, REVNET_E_UNSUPPORTED_SHAPE, "revnet_stack_plan: unsupported stage " + std::to_string(si)); }
+        StagePlan s;
+        s.c = sd.c; s.units = sd.units; s.has_trans = sd.trans_k != 0;
+        if (s.has_trans) { s.trans = slot(cprev, 2 * sd.c, sd.trans_k, sd.trans_stride, true); H = conv_out(H, sd.trans_k, sd.trans_stride); }
+        s.H = H;
+        for (int u = 0; u < sd.units; u++) {
+            for (int f = 0; f < 2; f++) {
+                std::vector<LayerSlot> v;
+                for (auto &sh : fn_shape(sd.kind, sd.c, sd.w)) v.push_back(slot(sh[0], sh[1], sh[2], 1, true));
+                (f == 0 ? s.F : s.G).push_back(v);
+            }
+        }
+        size_t hb = (size_t)d.N * H * H * sd.c * 4;
+        s.off_x1 = atake(hb); s.off_x2 = atake(hb);
+        pl->stored_bytes += 2 * hb;
+        s.off_v1 = s.off_v2 = 0;
+        pl->st.push_back(s);
+        cprev = 2 * sd.c;
+    }
+    if (d.verify_reconstruction)
+        for (auto &s : pl->st) { size_t hb = (size_t)d.N * s.H * s.H * s.c * 4; s.off_v1 = atake(hb); s.off_v2 = atake(hb); }
+    pl->feat_C = cprev;
+    pl->off_fcW = take((size_t)d.n_classes * cprev, true);
+    pl->off_fcb = take(d.n_classes, false);
+    pl->n_params = off;
+    pl->act_bytes = aoff;
+    if (off >= 0xffffffffull) { delete pl; return fail(ctx, REVNET_E_UNSUPPORTED_SHAPE, "revnet_stack_plan: more than 2^32 parameters"); }
+    size_t nseg = pl->seg_end.size();
+    if (cudaMallocHost(&pl->pinned, nseg * 5) != cudaSuccess) {
+        cudaGetLastError();
+        pl->pinned = malloc(nseg * 5);
+        pl->pinned_is_malloc = true;
+        if (!pl->pinned) { delete pl; return fail(ctx, REVNET_E_INTERNAL, "revnet_stack_plan: out of host memory"); }
+    }
+    memcpy(pl->pinned, pl->seg_end.data(), nseg * 4);
+    memcpy((char *)pl->pinned + nseg * 4, pl->seg_decay.data(), nseg);
+    // size the workspace with a dry run of the very same driver
+    Exec ex; ex.ctx = ctx; ex.dry = true; ex.ws.dry = true; ex.mode = d.mode; ex.eps = d.eps;
+    run_step(pl, ex, nullptr, nullptr, (float *)0x1000, (float *)0x1000, (float *)0x1000, (char *)0x1000, nullptr, nullptr, nullptr, nullptr, nullptr);
+    pl->ws_bytes = ex.ws.peak + 256;
+    if (param_count) *param_count = pl->n_params;
+    if (activation_bytes) *activation_bytes = pl->act_bytes;
+    if (workspace_bytes) *workspace_bytes = pl->ws_bytes;
+    *plan_out = pl;
+    return REVNET_OK;
+}
+
+extern "C" int revnet_plan_destroy(revnet_plan *pl) {
+    if (!pl) return REVNET_OK;
+    if (pl->pinned) { if (pl->pinned_is_malloc) free(pl->pinned); else cudaFreeHost(pl->pinned); }
+    delete pl;
+    return REVNET_OK;
+}
+
+extern "C" int revnet_train_step(revnet_ctx *ctx, revnet_plan *pl, const float *images, const int32_t *labels,
+                                 float *params, float *grads, float *momentum, void *activations, void *workspace,
+                                 float *loss, int32_t *pred, float *logits, revnet_step_stats *stats, void *stream) {
+    if (!ctx || !pl || !images || !labels || !params || !grads || !momentum || !activations || !workspace || !loss || !pred)
+        return fail(ctx, REVNET_E_INVALID_ARG, "revnet_train_step: null argument");
+    const void *ptrs[] = {images, params, grads, momentum, activations, workspace};
+    for (const void *p : ptrs)
+        if ((uintptr_t)p & 15) return fail(ctx, REVNET_E_MISALIGNED, "revnet_train_step: pointers must be 16-byte aligned");
+    Exec ex; ex.ctx = ctx; ex.dry = false; ex.mode = pl->d.mode; ex.eps = pl->d.eps; ex.stream = (cudaStream_t)stream;
+    ex.ws.dry = false; ex.ws.base = (char *)workspace; ex.ws.cap = pl->ws_bytes;
+    float *recon = nullptr;
+    run_step(pl, ex, images, labels, params, grads, momentum, (char *)activations, loss, pred, logits, stats, &recon);
+    if (ex.ws.overflow) return fail(ctx, REVNET_E_WORKSPACE_TOO_SMALL, "revnet_train_step: workspace smaller than planned");
+    if (ex.failed) return REVNET_E_CUDA;
+    if (pl->d.verify_reconstruction && stats) {
+        if (cudaMemcpyAsync(stats->recon_max_abs, recon, sizeof(float) * REVNET_MAX_STAGES, cudaMemcpyDeviceToHost, ex.stream) != cudaSuccess ||
+            cudaStreamSynchronize(ex.stream) != cudaSuccess)
+            return fail(ctx, REVNET_E_CUDA, std::string("revnet_train_step: ") + cudaGetErrorString(cudaGetLastError()));
+    }
+    return REVNET_OK;
+}
+
+extern "C" int revnet_train_step_host(revnet_ctx *ctx, revnet_plan *pl, const float *images_host, const int32_t *labels_host,
+                                      float *images_dev, int32_t *labels_dev, float *params, float *grads, float *momentum,
+                                      void *activations, void *workspace, float *loss_dev, int32_t *pred_dev,
+                                      float *loss_host, int32_t *pred_host, revnet_step_stats *stats, void *stream) {
+    if (!ctx || !pl || !images_host || !labels_host || !images_dev || !labels_dev || !loss_host || !pred_host)
+        return fail(ctx, REVNET_E_INVALID_ARG, "revnet_train_step_host: null argument");
+    cudaStream_t s = (cudaStream_t)stream;
+    const revnet_stack_desc &d = pl->d;
+    size_t ib = (size_t)d.N * d.img * d.img * d.in_ch * sizeof(float);
+    if (cudaMemcpyAsync(images_dev, images_host, ib, cudaMemcpyHostToDevice, s) != cudaSuccess ||
+        cudaMemcpyAsync(labels_dev, labels_host, (size_t)d.N * 4, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return fail(ctx, REVNET_E_CUDA, std::string("revnet_train_step_host: H2D copy: ") + cudaGetErrorString(cudaGetLastError()));
+    int rc = revnet_train_step(ctx, pl, images_dev, labels_dev, params, grads, momentum, activations, workspace,
+                               loss_dev, pred_dev, nullptr, stats, stream);
+    if (rc) return rc;
+    if (cudaMemcpyAsync(loss_host, loss_dev, 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaMemcpyAsync(pred_host, pred_dev, (size_t)d.N * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess)
+        return fail(ctx, REVNET_E_CUDA, std::string("revnet_train_step_host: D2H copy: ") + cudaGetErrorString(cudaGetLastError()));
+    return REVNET_OK;
+}

@@ -1,0 +1,96 @@
+"""Convenience wrappers that own the device buffers of one block / one stack and call the C ABI.
+
+Marshalling only: numpy (NCHW, [Cout,Cin,kh,kw]) in, torch CUDA buffers in the ABI's layouts,
+numpy out.  Used by the tests, the smoke check and the benchmark.
+"""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+from . import binding as B
+from . import synthetic as syn
+
+
+def _dev(a, dtype=torch.float32):
+    return torch.from_numpy(np.ascontiguousarray(a)).to(dtype).cuda()
+
+
+class BlockRunner:
+    def __init__(self, ctx: B.Context, b: syn.BlockCfg, mode: int):
+        self.ctx, self.b, self.mode = ctx, b, mode
+        self.desc = B.block_desc(b, mode)
+        fwd, bwd = B.revnet_block_workspace_bytes(ctx, self.desc)
+        self.ws = torch.empty(max(fwd, bwd), dtype=torch.uint8, device="cuda")
+        self.layers = syn.fn_layers(b.kind, b.c, b.w)
+
+    def _params(self, params, fn):
+        return [dict(W=_dev(B.w_to_abi(params[f"{fn}.l{i}.W"])), gamma=_dev(params[f"{fn}.l{i}.gamma"]),
+                     beta=_dev(params[f"{fn}.l{i}.beta"])) for i in range(len(self.layers))]
+
+    def load(self, params):
+        self.F, self.G = self._params(params, "F"), self._params(params, "G")
+        self.gF = [{k: torch.zeros_like(v) for k, v in l.items()} for l in self.F]
+        self.gG = [{k: torch.zeros_like(v) for k, v in l.items()} for l in self.G]
+
+    def forward(self, x1, x2, inplace=False):
+        """x1, x2: NCHW numpy -> y1, y2 NCHW numpy"""
+        dx1, dx2 = _dev(B.to_nhwc(x1)), _dev(B.to_nhwc(x2))
+        y1, y2 = (dx1, dx2) if inplace else (torch.empty_like(dx1), torch.empty_like(dx2))
+        B.revnet_block_fwd(self.ctx, self.desc, dx1, dx2, self.F, self.G, y1, y2, self.ws)
+        torch.cuda.synchronize()
+        return B.to_nchw(y1.cpu().numpy()), B.to_nchw(y2.cpu().numpy())
+
+    def backward(self, y1, y2, dy1, dy2, inplace=False):
+        ty1, ty2, tdy1, tdy2 = (_dev(B.to_nhwc(t)) for t in (y1, y2, dy1, dy2))
+        if inplace:
+            x1, x2, dx1, dx2 = ty1, ty2, tdy1, tdy2
+        else:
+            x1, x2, dx1, dx2 = (torch.empty_like(ty1) for _ in range(4))
+        B.revnet_block_bwd(self.ctx, self.desc, ty1, ty2, tdy1, tdy2, self.F, self.G, x1, x2, dx1, dx2, self.gF, self.gG, self.ws)
+        torch.cuda.synchronize()
+        grads = {}
+        for fn, gl in (("F", self.gF), ("G", self.gG)):
+            for i, l in enumerate(gl):
+                grads[f"{fn}.l{i}.W"] = B.w_from_abi(l["W"].cpu().numpy())
+                grads[f"{fn}.l{i}.gamma"] = l["gamma"].cpu().numpy()
+                grads[f"{fn}.l{i}.beta"] = l["beta"].cpu().numpy()
+        out = [B.to_nchw(t.cpu().numpy()) for t in (x1, x2, dx1, dx2)]
+        return out[0], out[1], out[2], out[3], grads
+
+
+class StackRunner:
+    def __init__(self, ctx: B.Context, cfg: syn.StackCfg, mode: int, verify_reconstruction: bool = False):
+        self.ctx, self.cfg, self.mode = ctx, cfg, mode
+        self.specs = syn.param_specs(cfg)
+        self.desc = B.stack_desc(cfg, mode, verify_reconstruction)
+        self.plan = B.revnet_stack_plan(ctx, self.desc)
+        n = self.plan.param_count
+        assert n == sum(int(np.prod(s)) for _, s, _ in self.specs)
+        self.params = torch.zeros(n, dtype=torch.float32, device="cuda")
+        self.grads = torch.zeros(n, dtype=torch.float32, device="cuda")
+        self.momentum = torch.zeros(n, dtype=torch.float32, device="cuda")
+        self.act = torch.empty(self.plan.activation_bytes, dtype=torch.uint8, device="cuda")
+        self.ws = torch.empty(self.plan.workspace_bytes, dtype=torch.uint8, device="cuda")
+        self.images = torch.empty((cfg.N, cfg.img, cfg.img, cfg.in_ch), dtype=torch.float32, device="cuda")
+        self.labels = torch.empty((cfg.N,), dtype=torch.int32, device="cuda")
+        self.loss = torch.zeros(1, dtype=torch.float32, device="cuda")
+        self.pred = torch.zeros(cfg.N, dtype=torch.int32, device="cuda")
+        self.logits = torch.zeros((cfg.N, cfg.n_classes), dtype=torch.float32, device="cuda")
+
+    def load(self, images, labels, params):
+        self.images.copy_(torch.from_numpy(B.to_nhwc(images)))
+        self.labels.copy_(torch.from_numpy(np.asarray(labels, np.int32)))
+        self.params.copy_(torch.from_numpy(B.pack_params(self.specs, params)))
+        self.momentum.zero_()
+
+    def step(self, want_logits=True):
+        return B.revnet_train_step(self.ctx, self.plan, self.images, self.labels, self.params, self.grads, self.momentum,
+                                   self.act, self.ws, self.loss, self.pred, self.logits if want_logits else None)
+
+    def results(self):
+        torch.cuda.synchronize()
+        return dict(loss=float(self.loss.item()), pred=self.pred.cpu().numpy(), logits=self.logits.cpu().numpy(),
+                    grads=B.unpack_params(self.specs, self.grads.cpu().numpy()),
+                    params=B.unpack_params(self.specs, self.params.cpu().numpy()),
+                    momentum=B.unpack_params(self.specs, self.momentum.cpu().numpy()))

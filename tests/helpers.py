@@ -43,10 +43,10 @@ def rel_l2(a, b):
 def tiny_stack(kind="basic", maxpool=False, N=4, img=8, units=2, seed=11, n_classes=5):
     """A few-thousand-parameter stack with every kind of layer the big configs have."""
     if kind == "basic":
-        st = (syn.StageCfg(units, 4, 0, "basic", 0, 1), syn.StageCfg(units, 6, 0, "basic", 3, 2))
+        st = (syn.StageCfg(units, 4, 0, "basic", 0, 1), syn.StageCfg(units, 8, 0, "basic", 3, 2))
         stem_c = 8
     else:
-        st = (syn.StageCfg(units, 8, 2, "bottleneck", 3, 1), syn.StageCfg(units, 12, 3, "bottleneck", 3, 2))
-        stem_c = 6
+        st = (syn.StageCfg(units, 8, 4, "bottleneck", 3, 1), syn.StageCfg(units, 12, 4, "bottleneck", 3, 2))
+        stem_c = 8
     return syn.StackCfg(f"tiny_{kind}", N, img * (4 if maxpool else 1), n_classes,
                         7 if maxpool else 3, 2 if maxpool else 1, stem_c, maxpool, st, seed=seed)

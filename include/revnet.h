@@ -25,6 +25,14 @@
  *   - Gradient outputs are overwritten, not accumulated.
  *   - Every call returns 0 (REVNET_OK) or a negative revnet_status; the text of the last error
  *     of a context is available from revnet_last_error.  No exception crosses the ABI.
+ *   - Coupling state.  With state_frac_bits = 0 the tensors x1, x2, y1, y2 (and a stack's stage
+ *     buffers) hold float32 and reconstruction is exact only up to rounding, which low-precision
+ *     residual functions amplify.  With state_frac_bits = k > 0 they hold int32 fixed-point
+ *     numbers (value = i * 2^-k): the residual function's float result is rounded to that grid
+ *     before the add, y = x + round(F * 2^k) is undone exactly by x = y - round(F * 2^k), and the
+ *     reversal returns the forward pass's inputs bit for bit (Section 3.2, "Numerical error":
+ *     fixed point on the x's and y's, floating point inside F and G).  Range |value| < 2^(31-k).
+ *     Gradients are float32 in either format.
  *   - mode 0: convolution operands rounded to bf16, products accumulated in fp32 on the tensor
  *     cores where the shape allows; mode 1: strict fp32 arithmetic throughout (verification).
  *     The coupling state (x, y and their gradients) is fp32 in both modes.
@@ -75,6 +83,8 @@ typedef struct {
     revnet_fn_desc F, G;
     float eps;               /* BN epsilon */
     int mode;                /* 0 = bf16 tensor-core operands, 1 = strict fp32 */
+    int state_frac_bits;     /* 0: x, y are float32.  k in 1..24: x, y are int32 fixed point with k
+                                fractional bits (value = i * 2^-k); see "coupling state" above */
 } revnet_block_desc;
 
 /* Parameters of one residual function (device pointers): W[l] is [cout][k][k][cin],
@@ -98,9 +108,9 @@ int revnet_block_workspace_bytes(revnet_ctx *ctx, const revnet_block_desc *desc,
 
 /* Block forward (Section 3.1): y1 = x1 + F(x2); y2 = x2 + G(y1). */
 int revnet_block_fwd(revnet_ctx *ctx, const revnet_block_desc *desc,
-                     const float *x1, const float *x2,
+                     const void *x1, const void *x2,
                      const revnet_fn_params *F, const revnet_fn_params *G,
-                     float *y1, float *y2,
+                     void *y1, void *y2,
                      void *workspace, size_t workspace_bytes, void *stream);
 
 /* Block backward without stored activations (Algorithm 1): from (y1,y2) and (dy1,dy2) compute
@@ -109,9 +119,9 @@ int revnet_block_fwd(revnet_ctx *ctx, const revnet_block_desc *desc,
  * reconstructing are reused for the gradient steps (four convolution passes per layer in all,
  * counting the forward: Section 3.2 "Computational overhead", Section 5.1). */
 int revnet_block_bwd(revnet_ctx *ctx, const revnet_block_desc *desc,
-                     const float *y1, const float *y2, const float *dy1, const float *dy2,
+                     const void *y1, const void *y2, const float *dy1, const float *dy2,
                      const revnet_fn_params *F, const revnet_fn_params *G,
-                     float *x1, float *x2, float *dx1, float *dx2,
+                     void *x1, void *x2, float *dx1, float *dx2,
                      const revnet_fn_grads *gF, const revnet_fn_grads *gG,
                      void *workspace, size_t workspace_bytes, void *stream);
 
@@ -135,6 +145,7 @@ typedef struct {
     revnet_stage_desc stage[REVNET_MAX_STAGES];
     float eps;
     int mode;
+    int state_frac_bits;                            /* format of the stage buffers, as in revnet_block_desc */
     float lr, momentum, weight_decay;               /* SGD (Appendix 6.1); decay on conv/FC weights only */
     int verify_reconstruction;                      /* debug: keep a copy of each stage input and report
                                                        max |reconstructed - original| per stage */

@@ -133,25 +133,58 @@ def bn_relu_bwd(da, cache):
     return dt, dgamma, dbeta
 
 
+# --------------------------------------------------------------------------- storage formats
+# The definitions above are exact real arithmetic in float64.  Two OPTIONAL storage roundings
+# can be switched on so that the discrete decisions of a low-precision implementation (which
+# side of zero a ReLU input falls on, which grid point a stored value rounds to) are taken at
+# that implementation's precision rather than at float64's:
+#   num["bf16_operands"]: convolution operands (activated input, weights, upstream gradient) are
+#       rounded to bfloat16 (8-bit exponent, 7-bit mantissa, round to nearest even) before each
+#       convolution; products and sums stay float64.
+#   num["frac_bits"] = k > 0: the coupling state is kept on the grid 2^-k: y = x + rint(F 2^k)/2^k,
+#       the fixed-point remedy of Section 3.2 ("Numerical error"); reconstruction is then exact.
+# With num = None (the default everywhere) nothing is rounded.
+
+def round_bf16(x):
+    """Round float64 values to the nearest bfloat16 (ties to even), returned as float64."""
+    x = np.asarray(x, np.float64)
+    m, e = np.frexp(x)                                      # x = m * 2^e, 0.5 <= |m| < 1
+    r = np.rint(m * 256.0) / 256.0                          # 8 significant bits; rint = ties to even
+    out = np.ldexp(r, e)
+    return np.where(np.isfinite(x), out, x)
+
+
+def _rb(x, num):
+    return round_bf16(x) if num and num.get("bf16_operands") else x
+
+
+def quantize_state(v, num):
+    """Residual-function value as it is added to a fixed-point coupling state."""
+    k = num.get("frac_bits", 0) if num else 0
+    return np.rint(v * float(1 << k)) / float(1 << k) if k else v
+
+
 # --------------------------------------------------------------------------- residual functions
 
-def fn_fwd(u, layers, eps):
+def fn_fwd(u, layers, eps, num=None):
     """Residual function: chain of c_k(x) = Conv(ReLU(BN(x))) layers (Eq. 2: Basic = c3(c3(x)),
     Bottleneck = c1(c3(c1(x)))).  Returns the value and per-layer caches."""
     caches = []
     t = u
     for L in layers:
         a, bn = bn_relu_fwd(t, np.asarray(L["gamma"], np.float64), np.asarray(L["beta"], np.float64), eps)
-        w = np.asarray(L["W"], np.float64)
+        a = _rb(a, num)
+        w = _rb(np.asarray(L["W"], np.float64), num)
         s = L.get("stride", 1)
         caches.append((bn, a, w, s, t.shape[2:], L["name"]))
         t = conv_fwd(a, w, stride=s)
     return t, caches
 
 
-def fn_bwd(g, caches, grads):
+def fn_bwd(g, caches, grads, num=None):
     """Ordinary backprop (Eq. 1) through a residual function; parameter gradients go into `grads`."""
     for bn, a, w, s, in_hw, name in reversed(caches):
+        g = _rb(g, num)
         grads[name + ".W"] = conv_wgrad(g, a, w.shape[2], stride=s)
         da = conv_dgrad(g, w, in_hw, stride=s)
         g, dgamma, dbeta = bn_relu_bwd(da, bn)
@@ -162,44 +195,44 @@ def fn_bwd(g, caches, grads):
 
 # --------------------------------------------------------------------------- reversible block
 
-def block_fwd(x1, x2, F, G, eps, keep=False):
+def block_fwd(x1, x2, F, G, eps, keep=False, num=None):
     """y1 = x1 + F(x2); y2 = x2 + G(y1)   (Section 3.1)."""
-    f, cF = fn_fwd(x2, F, eps)
-    y1 = x1 + f
-    g, cG = fn_fwd(y1, G, eps)
-    y2 = x2 + g
+    f, cF = fn_fwd(x2, F, eps, num)
+    y1 = x1 + quantize_state(f, num)
+    g, cG = fn_fwd(y1, G, eps, num)
+    y2 = x2 + quantize_state(g, num)
     return (y1, y2, (cF, cG)) if keep else (y1, y2)
 
 
-def block_inverse(y1, y2, F, G, eps):
+def block_inverse(y1, y2, F, G, eps, num=None):
     """x2 = y2 - G(y1); x1 = y1 - F(x2)   (Section 3.1)."""
-    x2 = y2 - fn_fwd(y1, G, eps)[0]
-    x1 = y1 - fn_fwd(x2, F, eps)[0]
+    x2 = y2 - quantize_state(fn_fwd(y1, G, eps, num)[0], num)
+    x1 = y1 - quantize_state(fn_fwd(x2, F, eps, num)[0], num)
     return x1, x2
 
 
-def block_bwd_stored(dy1, dy2, caches, grads):
+def block_bwd_stored(dy1, dy2, caches, grads, num=None):
     """Ordinary backprop through the forward graph with z1 as an explicit node (Eq. 8), using
     activations kept from the forward pass."""
     cF, cG = caches
-    dz1 = dy1 + fn_bwd(dy2, cG, grads)
-    dx2 = dy2 + fn_bwd(dz1, cF, grads)
+    dz1 = dy1 + fn_bwd(dy2, cG, grads, num)
+    dx2 = dy2 + fn_bwd(dz1, cF, grads, num)
     dx1 = dz1
     return dx1, dx2
 
 
-def block_bwd_reconstruct(y1, y2, dy1, dy2, F, G, eps, grads):
+def block_bwd_reconstruct(y1, y2, dy1, dy2, F, G, eps, grads, num=None):
     """Algorithm 1 (BlockReverse): rebuild the inputs from the outputs, then backprop.
     Batch statistics are recomputed from the reconstructed tensors; nothing is kept per block.
     The activations computed while reconstructing are reused for the gradient steps (the 4N form,
     Section 5 "Implementation")."""
     z1 = y1
-    gz, cG = fn_fwd(z1, G, eps)
-    x2 = y2 - gz
-    fx, cF = fn_fwd(x2, F, eps)
-    x1 = z1 - fx
-    dz1 = dy1 + fn_bwd(dy2, cG, grads)
-    dx2 = dy2 + fn_bwd(dz1, cF, grads)
+    gz, cG = fn_fwd(z1, G, eps, num)
+    x2 = y2 - quantize_state(gz, num)
+    fx, cF = fn_fwd(x2, F, eps, num)
+    x1 = z1 - quantize_state(fx, num)
+    dz1 = dy1 + fn_bwd(dy2, cG, grads, num)
+    dx2 = dy2 + fn_bwd(dz1, cF, grads, num)
     dx1 = dz1
     return x1, x2, dx1, dx2
 
@@ -218,7 +251,7 @@ def softmax_ce(logits, labels):
     return loss, sm / N
 
 
-def stack_train_grads(net, images, labels, mode):
+def stack_train_grads(net, images, labels, mode, num=None):
     """Forward + backward of the whole stack.
 
     mode "stored": every block's activations are kept (ordinary backprop).
@@ -249,18 +282,20 @@ def stack_train_grads(net, images, labels, mode):
         tcache = None
         if S["trans"] is not None:
             stored.append(h)                  # input of a non-reversible layer is kept
-            h, tcache = fn_fwd(h, [S["trans"]], eps)
+            h, tcache = fn_fwd(h, [S["trans"]], eps, num)
         c = S["c"]
+        if si == 0 or S["trans"] is not None:
+            h = quantize_state(h, num)        # the stage buffers hold the coupling state's format
         x1, x2 = h[:, :c].copy(), h[:, c:].copy()
         bcaches = []
         for ui, (F, G) in enumerate(S["units"]):
             block_inputs[(si, ui)] = (x1, x2)
             if mode == "stored":
-                x1, x2, bc = block_fwd(x1, x2, F, G, eps, keep=True)
+                x1, x2, bc = block_fwd(x1, x2, F, G, eps, keep=True, num=num)
                 bcaches.append(bc)
                 stored += [t for fc in bc for (bn, a, *_r) in fc for t in (bn[0], a)]
             else:
-                x1, x2 = block_fwd(x1, x2, F, G, eps)
+                x1, x2 = block_fwd(x1, x2, F, G, eps, num=num)
         h = np.concatenate([x1, x2], axis=1)
         stage_fw.append((tcache, bcaches, x1, x2))
     stored.append(h)                          # top activations: needed to start the reversal
@@ -285,13 +320,13 @@ def stack_train_grads(net, images, labels, mode):
         for ui in reversed(range(len(S["units"]))):
             F, G = S["units"][ui]
             if mode == "stored":
-                d1, d2 = block_bwd_stored(d1, d2, bcaches[ui], grads)
+                d1, d2 = block_bwd_stored(d1, d2, bcaches[ui], grads, num)
             else:
-                y1, y2, d1, d2 = block_bwd_reconstruct(y1, y2, d1, d2, F, G, eps, grads)
+                y1, y2, d1, d2 = block_bwd_reconstruct(y1, y2, d1, d2, F, G, eps, grads, num)
                 recovered[(si, ui)] = (y1, y2)
         dh = np.concatenate([d1, d2], axis=1)
         if tcache is not None:
-            dh = fn_bwd(dh, tcache, grads)
+            dh = fn_bwd(dh, tcache, grads, num)
     if pool_idx is not None:
         dh = maxpool_bwd(dh, pool_idx, stem_out_hw)
     grads[st["name"] + ".W"] = conv_wgrad(dh, images, wst.shape[2], stride=st["stride"], pad=st["pad"])

@@ -30,7 +30,7 @@ class FnDesc(C.Structure):
 
 class BlockDesc(C.Structure):
     _fields_ = [("N", C.c_int), ("H", C.c_int), ("W", C.c_int), ("c", C.c_int), ("F", FnDesc), ("G", FnDesc),
-                ("eps", C.c_float), ("mode", C.c_int)]
+                ("eps", C.c_float), ("mode", C.c_int), ("state_frac_bits", C.c_int)]
 
 
 class FnParams(C.Structure):
@@ -50,7 +50,7 @@ class StackDesc(C.Structure):
     _fields_ = [("N", C.c_int), ("img", C.c_int), ("in_ch", C.c_int), ("n_classes", C.c_int),
                 ("stem_k", C.c_int), ("stem_stride", C.c_int), ("stem_cout", C.c_int), ("maxpool", C.c_int),
                 ("n_stages", C.c_int), ("stage", StageDesc * MAX_STAGES), ("eps", C.c_float), ("mode", C.c_int),
-                ("lr", C.c_float), ("momentum", C.c_float), ("weight_decay", C.c_float),
+                ("state_frac_bits", C.c_int), ("lr", C.c_float), ("momentum", C.c_float), ("weight_decay", C.c_float),
                 ("verify_reconstruction", C.c_int)]
 
 
@@ -128,23 +128,23 @@ def fn_desc(kind: str, c: int, w: int) -> FnDesc:
     return d
 
 
-def block_desc(b: syn.BlockCfg, mode: int) -> BlockDesc:
+def block_desc(b: syn.BlockCfg, mode: int, state_frac_bits: int = 0) -> BlockDesc:
     d = BlockDesc()
     d.N, d.H, d.W, d.c = b.N, b.H, b.W, b.c
     d.F = fn_desc(b.kind, b.c, b.w)
     d.G = fn_desc(b.kind, b.c, b.w)
-    d.eps, d.mode = b.eps, mode
+    d.eps, d.mode, d.state_frac_bits = b.eps, mode, state_frac_bits
     return d
 
 
-def stack_desc(cfg: syn.StackCfg, mode: int, verify_reconstruction: bool = False) -> StackDesc:
+def stack_desc(cfg: syn.StackCfg, mode: int, verify_reconstruction: bool = False, state_frac_bits: int = 0) -> StackDesc:
     d = StackDesc()
     d.N, d.img, d.in_ch, d.n_classes = cfg.N, cfg.img, cfg.in_ch, cfg.n_classes
     d.stem_k, d.stem_stride, d.stem_cout, d.maxpool = cfg.stem_k, cfg.stem_stride, cfg.stem_cout, int(cfg.maxpool)
     d.n_stages = len(cfg.stages)
     for i, s in enumerate(cfg.stages):
         d.stage[i] = StageDesc(s.units, s.c, s.w, KIND[s.kind], s.trans_k, s.trans_stride)
-    d.eps, d.mode = cfg.eps, mode
+    d.eps, d.mode, d.state_frac_bits = cfg.eps, mode, state_frac_bits
     d.lr, d.momentum, d.weight_decay = cfg.lr, cfg.momentum, cfg.weight_decay
     d.verify_reconstruction = int(verify_reconstruction)
     return d

@@ -2,6 +2,7 @@
 #include "common.cuh"
 #include <string.h>
 #include <stdio.h>
+#include <math.h>
 
 static int fail(revnet_ctx *ctx, int code, const std::string &msg) { if (ctx) ctx->err = msg; return code; }
 
@@ -45,8 +46,8 @@ static int check_fn(const revnet_fn_desc &f, int c) {
 }
 static int check_desc(revnet_ctx *ctx, const revnet_block_desc *d) {
     if (!ctx || !d) return fail(ctx, REVNET_E_INVALID_ARG, "null descriptor");
-    if (d->N < 1 || d->H < 1 || d->W < 1 || d->c < 4 || (d->mode != 0 && d->mode != 1))
-        return fail(ctx, REVNET_E_INVALID_ARG, "block descriptor: N,H,W >= 1, c >= 4, mode in {0,1}");
+    if (d->N < 1 || d->H < 1 || d->W < 1 || d->c < 4 || (d->mode != 0 && d->mode != 1) || d->state_frac_bits < 0 || d->state_frac_bits > 24)
+        return fail(ctx, REVNET_E_INVALID_ARG, "block descriptor: N,H,W >= 1, c >= 4, mode in {0,1}, state_frac_bits in [0,24]");
     if (d->c % 4 || !check_fn(d->F, d->c) || !check_fn(d->G, d->c))
         return fail(ctx, REVNET_E_UNSUPPORTED_SHAPE, "block descriptor: channels must be multiples of 4, kernels 1 or 3, F and G must map c -> c");
     if ((size_t)d->N * d->H * d->W >= (1u << 30)) return fail(ctx, REVNET_E_UNSUPPORTED_SHAPE, "block descriptor: too many pixels");
@@ -102,8 +103,8 @@ static int finish(revnet_ctx *ctx, Exec &ex, const char *who) {
     return REVNET_OK;
 }
 
-extern "C" int revnet_block_fwd(revnet_ctx *ctx, const revnet_block_desc *d, const float *x1, const float *x2,
-                                const revnet_fn_params *Fp, const revnet_fn_params *Gp, float *y1, float *y2,
+extern "C" int revnet_block_fwd(revnet_ctx *ctx, const revnet_block_desc *d, const void *x1, const void *x2,
+                                const revnet_fn_params *Fp, const revnet_fn_params *Gp, void *y1, void *y2,
                                 void *workspace, size_t workspace_bytes, void *stream) {
     int rc = check_desc(ctx, d);
     if (rc) return rc;
@@ -115,15 +116,16 @@ extern "C" int revnet_block_fwd(revnet_ctx *ctx, const revnet_block_desc *d, con
     revnet_block_workspace_bytes(ctx, d, &need, nullptr);
     if (workspace_bytes < need) return fail(ctx, REVNET_E_WORKSPACE_TOO_SMALL, "revnet_block_fwd: workspace too small");
     Exec ex; ex.ctx = ctx; ex.dry = false; ex.mode = d->mode; ex.eps = d->eps; ex.stream = (cudaStream_t)stream;
+    ex.q = d->state_frac_bits ? ldexpf(1.f, -d->state_frac_bits) : 0.f;
     ex.ws.dry = false; ex.ws.base = (char *)workspace; ex.ws.cap = workspace_bytes;
     block_forward(ex, Geom{d->N, d->H, d->W}, d->c, layers_of(d->F, Fp, nullptr), layers_of(d->G, Gp, nullptr),
-                  (float *)x1, (float *)x2, y1, y2);
+                  (float *)x1, (float *)x2, (float *)y1, (float *)y2);
     return finish(ctx, ex, "revnet_block_fwd");
 }
 
-extern "C" int revnet_block_bwd(revnet_ctx *ctx, const revnet_block_desc *d, const float *y1, const float *y2,
+extern "C" int revnet_block_bwd(revnet_ctx *ctx, const revnet_block_desc *d, const void *y1, const void *y2,
                                 const float *dy1, const float *dy2, const revnet_fn_params *Fp, const revnet_fn_params *Gp,
-                                float *x1, float *x2, float *dx1, float *dx2, const revnet_fn_grads *gF, const revnet_fn_grads *gG,
+                                void *x1, void *x2, float *dx1, float *dx2, const revnet_fn_grads *gF, const revnet_fn_grads *gG,
                                 void *workspace, size_t workspace_bytes, void *stream) {
     int rc = check_desc(ctx, d);
     if (rc) return rc;
@@ -137,9 +139,10 @@ extern "C" int revnet_block_bwd(revnet_ctx *ctx, const revnet_block_desc *d, con
     revnet_block_workspace_bytes(ctx, d, nullptr, &need);
     if (workspace_bytes < need) return fail(ctx, REVNET_E_WORKSPACE_TOO_SMALL, "revnet_block_bwd: workspace too small");
     Exec ex; ex.ctx = ctx; ex.dry = false; ex.mode = d->mode; ex.eps = d->eps; ex.stream = (cudaStream_t)stream;
+    ex.q = d->state_frac_bits ? ldexpf(1.f, -d->state_frac_bits) : 0.f;
     ex.ws.dry = false; ex.ws.base = (char *)workspace; ex.ws.cap = workspace_bytes;
     block_backward(ex, Geom{d->N, d->H, d->W}, d->c, layers_of(d->F, Fp, gF), layers_of(d->G, Gp, gG),
-                   y1, y2, dy1, dy2, x1, x2, dx1, dx2);
+                   (const float *)y1, (const float *)y2, dy1, dy2, (float *)x1, (float *)x2, dx1, dx2);
     return finish(ctx, ex, "revnet_block_bwd");
 }
 

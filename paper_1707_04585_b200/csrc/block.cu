@@ -103,23 +103,25 @@ void fn_backward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, FnS
 
 void block_forward(Exec &ex, Geom g, int c, const std::vector<Layer> &F, const std::vector<Layer> &G,
                    float *x1, float *x2, float *y1, float *y2) {
-    fn_forward(ex, g, single(x2, c), F, single(x1, c), single(y1, c), +1, nullptr, false);
-    fn_forward(ex, g, single(y1, c), G, single(x2, c), single(y2, c), +1, nullptr, false);
+    const float q = ex.q;
+    fn_forward(ex, g, single(x2, c, q), F, single(x1, c, q), single(y1, c, q), +1, nullptr, false);
+    fn_forward(ex, g, single(y1, c, q), G, single(x2, c, q), single(y2, c, q), +1, nullptr, false);
 }
 
 void block_backward(Exec &ex, Geom g, int c, const std::vector<Layer> &F, const std::vector<Layer> &G,
                     const float *y1, const float *y2, const float *dy1, const float *dy2,
                     float *x1, float *x2, float *dx1, float *dx2) {
     FnSaved sv;
+    const float q = ex.q;   // format of the coupling state; gradients are always float
     size_t m = ex.ws.mark();
     // x2 = y2 - G(z1), z1 = y1
-    fn_forward(ex, g, single((float *)y1, c), G, single((float *)y2, c), single(x2, c), -1, &sv, false);
+    fn_forward(ex, g, single((float *)y1, c, q), G, single((float *)y2, c, q), single(x2, c, q), -1, &sv, false);
     // dz1 = dy1 + (dG/dz1)^T dy2 ; dW_G
-    fn_backward(ex, g, single((float *)y1, c), G, sv, single((float *)dy2, c), single((float *)dy1, c), single(dx1, c));
+    fn_backward(ex, g, single((float *)y1, c, q), G, sv, single((float *)dy2, c), single((float *)dy1, c), single(dx1, c));
     ex.ws.release(m);
     // x1 = z1 - F(x2)
-    fn_forward(ex, g, single(x2, c), F, single((float *)y1, c), single(x1, c), -1, &sv, false);
+    fn_forward(ex, g, single(x2, c, q), F, single((float *)y1, c, q), single(x1, c, q), -1, &sv, false);
     // dx2 = dy2 + (dF/dx2)^T dz1 ; dW_F ; dx1 = dz1 (already in place)
-    fn_backward(ex, g, single(x2, c), F, sv, single(dx1, c), single((float *)dy2, c), single(dx2, c));
+    fn_backward(ex, g, single(x2, c, q), F, sv, single(dx1, c), single((float *)dy2, c), single(dx2, c));
     ex.ws.release(m);
 }

@@ -28,17 +28,40 @@ struct revnet_ctx {
 
 // A tensor of C = c0 + c1 channels stored as two NHWC tensors: channels [0,c0) in p0 (row
 // stride c0) and [c0,c0+c1) in p1 (row stride c1).  c1 == 0: one plain tensor.
+// q == 0: elements are float.  q > 0: elements are int32 fixed point, value = i * q with
+// q = 2^-frac_bits (the exactly invertible coupling state of Section 3.2, "Numerical error").
 struct Pair {
     float *p0;
     float *p1;
     int c0, c1;
+    float q;
     __host__ __device__ int C() const { return c0 + c1; }
     __device__ __forceinline__ float *at(size_t row, int ch) const {
         return ch < c0 ? p0 + row * c0 + ch : p1 + row * c1 + (ch - c0);
     }
+#ifdef __CUDACC__
+    __device__ __forceinline__ float4 ld4(size_t row, int ch) const {
+        const float *p = at(row, ch);
+        if (q == 0.f) return *reinterpret_cast<const float4 *>(p);
+        int4 i = *reinterpret_cast<const int4 *>(p);
+        return make_float4(__int2float_rn(i.x) * q, __int2float_rn(i.y) * q, __int2float_rn(i.z) * q, __int2float_rn(i.w) * q);
+    }
+    // out = partner + sign * v on the stored representation (sign 0: out = v)
+    __device__ __forceinline__ void couple(size_t row, int ch, float v, const Pair &partner, int sign) const {
+        float *o = at(row, ch);
+        if (q == 0.f) {
+            if (sign) { float p = *partner.at(row, ch); v = sign > 0 ? p + v : p - v; }
+            *o = v;
+        } else {
+            int iv = __float2int_rn(v * (1.f / q));
+            if (sign) { int p = *reinterpret_cast<const int *>(partner.at(row, ch)); iv = sign > 0 ? p + iv : p - iv; }
+            *reinterpret_cast<int *>(o) = iv;
+        }
+    }
+#endif
 };
-static inline Pair single(float *p, int C) { return Pair{p, nullptr, C, 0}; }
-static inline Pair halves(float *a, float *b, int c) { return Pair{a, b, c, c}; }
+static inline Pair single(float *p, int C, float q = 0.f) { return Pair{p, nullptr, C, 0, q}; }
+static inline Pair halves(float *a, float *b, int c, float q = 0.f) { return Pair{a, b, c, c, q}; }
 
 // Bump allocator over the caller's workspace; in dry mode it only measures.
 struct Arena {
@@ -66,6 +89,7 @@ struct Exec {
     bool dry = true;       // true: size the workspace and count work, launch nothing
     int mode = 0;          // 0 bf16 tensor-core operands, 1 strict fp32
     float eps = 1e-5f;
+    float q = 0.f;         // coupling-state format: 0 = float, else int32 fixed point with step q
     uint64_t flops = 0;    // dense conv/FC flops issued
     uint64_t launches = 0;
     bool failed = false;
@@ -113,7 +137,8 @@ void head_bwd(Exec &ex, Pair dy, int N, int HW, const float *Wfc, const float *f
 void sgd_update(Exec &ex, float *params, const float *grads, float *mom, size_t n,
                 const uint32_t *seg_end, const uint8_t *seg_decay, int n_seg,
                 float lr, float momentum, float wd);
-void max_abs_diff(Exec &ex, const float *a, const float *b, size_t n, float *out /*1 float, pre-zeroed*/);
+// max |a - b| over n elements of two state tensors (float, or fixed point when q > 0)
+void max_abs_diff(Exec &ex, const float *a, const float *b, size_t n, float q, float *out /*1 float, pre-zeroed*/);
 void fill_zero(Exec &ex, void *p, size_t bytes);
 
 // ---------------------------------------------------------------- conv_simt.cu

@@ -27,10 +27,11 @@ template <class TA> struct FpropA {           // m = output pixel, k = (kh,kw,ci
         return ldf(a + (((size_t)n * g.H + y) * g.W + x) * g.Ci + ci);
     }
 };
+__device__ __forceinline__ float round_w(float w, bool to_bf16) { return to_bf16 ? __bfloat162float(__float2bfloat16_rn(w)) : w; }
 struct FpropB {                               // k = (kh,kw,ci), n = co ; W[co][kh][kw][ci]
-    const float *w; int K;
+    const float *w; int K; bool wb;           // wb: weights take part as bf16 values (mode 0)
     static constexpr bool k_fast = true;
-    __device__ float operator()(int kk, int n) const { return w[(size_t)n * K + kk]; }
+    __device__ float operator()(int kk, int n) const { return round_w(w[(size_t)n * K + kk], wb); }
 };
 template <class TG> struct DgradA {           // m = input pixel, k = (kh,kw,co)
     const TG *gq; ConvGeom g;
@@ -46,11 +47,11 @@ template <class TG> struct DgradA {           // m = input pixel, k = (kh,kw,co)
     }
 };
 struct DgradB {                               // k = (kh,kw,co), n = ci
-    const float *w; ConvGeom g;
+    const float *w; ConvGeom g; bool wb;
     static constexpr bool k_fast = false;
     __device__ float operator()(int kk, int n) const {
         int co = kk % g.Co, tap = kk / g.Co;
-        return w[((size_t)co * g.k * g.k + tap) * g.Ci + n];
+        return round_w(w[((size_t)co * g.k * g.k + tap) * g.Ci + n], wb);
     }
 };
 template <class TG> struct WgradA {           // m = co, k = output pixel
@@ -73,10 +74,7 @@ template <class TA> struct WgradB {           // k = output pixel, n = (kh,kw,ci
 // ---- epilogues
 struct EpiCouple {                            // out = partner + sign*acc (sign 0: plain store); out/partner may be split pairs
     Pair out, partner; int sign;
-    __device__ void operator()(int m, int n, float v, int) const {
-        if (sign) { float p = *partner.at(m, n); v = sign > 0 ? p + v : p - v; }
-        *out.at(m, n) = v;
-    }
+    __device__ void operator()(int m, int n, float v, int) const { out.couple(m, n, v, partner, sign); }
 };
 struct EpiPlain {                             // row-major [M][N] (+ split-K slice)
     float *out; int N; size_t slice;
@@ -164,7 +162,7 @@ void conv_fprop_simt(Exec &ex, const void *a, bool a_bf16, Geom gi, const Layer 
     ex.flops += 2ull * M * N * K;
     if (ex.dry) return;
     EpiCouple ep{out, partner, sign};
-    FpropB bl{L.W, K};
+    FpropB bl{L.W, K, a_bf16};
     const double bytes = (double)g.N * g.H * g.W * g.Ci * (a_bf16 ? 2 : 4) + (double)M * N * (sign ? 8 : 4) + (double)N * K * 4;
     if (a_bf16) launch_gemm(ex, "conv_fprop_simt", FpropA<bf16>{(const bf16 *)a, g}, bl, ep, M, N, K, 1, K, bytes);
     else launch_gemm(ex, "conv_fprop_simt", FpropA<float>{(const float *)a, g}, bl, ep, M, N, K, 1, K, bytes);
@@ -176,7 +174,7 @@ void conv_dgrad_simt(Exec &ex, const void *gq, bool g_bf16, Geom gi, const Layer
     ex.flops += 2ull * g.N * g.Ho * g.Wo * N * K;
     if (ex.dry) return;
     EpiPlain ep{da, N, 0};
-    DgradB bl{L.W, g};
+    DgradB bl{L.W, g, g_bf16};
     const double bytes = (double)g.N * g.Ho * g.Wo * g.Co * (g_bf16 ? 2 : 4) + (double)M * N * 4 + (double)N * K * 4;
     if (g_bf16) launch_gemm(ex, "conv_dgrad_simt", DgradA<bf16>{(const bf16 *)gq, g}, bl, ep, M, N, K, 1, K, bytes);
     else launch_gemm(ex, "conv_dgrad_simt", DgradA<float>{(const float *)gq, g}, bl, ep, M, N, K, 1, K, bytes);

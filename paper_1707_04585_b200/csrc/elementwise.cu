@@ -82,7 +82,7 @@ __global__ void col_reduce_kernel(Pair t, const float *__restrict__ da, size_t P
         float4 sc, sh, mu, rs;
         if (MODE == 1) { sc = ld4(scale + q * 4); sh = ld4(shift + q * 4); mu = ld4(mean + q * 4); rs = ld4(rstd + q * 4); }
         for (size_t r = r0 + threadIdx.y; r < r1; r += RPP) {
-            float4 v = ld4(t.at(r, q * 4));
+            float4 v = t.ld4(r, q * 4);
             if (MODE == 0) {
                 s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
                 ss.x += v.x * v.x; ss.y += v.y * v.y; ss.z += v.z * v.z; ss.w += v.w * v.w;
@@ -166,7 +166,7 @@ __global__ void bn_relu_apply_kernel(Pair t, size_t nquads, int C4, const float 
                                      const float *__restrict__ shift, TO *__restrict__ a) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
         size_t row = i / C4; int q = (int)(i - row * C4);
-        float4 v = ld4(t.at(row, q * 4)), sc = ld4(scale + q * 4), sh = ld4(shift + q * 4);
+        float4 v = t.ld4(row, q * 4), sc = ld4(scale + q * 4), sh = ld4(shift + q * 4);
         v.x = fmaxf(fmaf(sc.x, v.x, sh.x), 0.f); v.y = fmaxf(fmaf(sc.y, v.y, sh.y), 0.f);
         v.z = fmaxf(fmaf(sc.z, v.z, sh.z), 0.f); v.w = fmaxf(fmaf(sc.w, v.w, sh.w), 0.f);
         st4(a + i * 4, v);
@@ -196,7 +196,7 @@ __global__ void bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, s
     const int C = C4 * 4;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
         size_t row = i / C4; int q = (int)(i - row * C4), c = q * 4;
-        float4 v = ld4(t.at(row, c)), g = ld4(da + i * 4);
+        float4 v = t.ld4(row, c), g = ld4(da + i * 4);
         float4 sc = ld4(scale + c), sh = ld4(shift + c), mu = ld4(mean + c), rs = ld4(rstd + c);
         float4 k0 = ld4(coef + c), k1 = ld4(coef + C + c), k2 = ld4(coef + 2 * C + c), o;
         o.x = k0.x * (fmaf(sc.x, v.x, sh.x) > 0.f ? g.x : 0.f) - k1.x - k2.x * ((v.x - mu.x) * rs.x);
@@ -204,7 +204,7 @@ __global__ void bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, s
         o.z = k0.z * (fmaf(sc.z, v.z, sh.z) > 0.f ? g.z : 0.f) - k1.z - k2.z * ((v.z - mu.z) * rs.z);
         o.w = k0.w * (fmaf(sc.w, v.w, sh.w) > 0.f ? g.w : 0.f) - k1.w - k2.w * ((v.w - mu.w) * rs.w);
         if (OUT == 2) {
-            float4 p = ld4(add.at(row, c));
+            float4 p = add.ld4(row, c);
             o.x += p.x; o.y += p.y; o.z += p.z; o.w += p.w;
         }
         if (OUT == 0) st4(out + i * 4, o);
@@ -242,7 +242,7 @@ template <class TO>
 __global__ void concat_cast_kernel(Pair src, size_t nquads, int C4, TO *__restrict__ dst) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
         size_t row = i / C4; int q = (int)(i - row * C4);
-        st4(dst + i * 4, ld4(src.at(row, q * 4)));
+        st4(dst + i * 4, src.ld4(row, q * 4));
     }
 }
 
@@ -325,7 +325,7 @@ __global__ void avgpool_kernel(Pair y, int HW, float *__restrict__ feat) {
     float4 s = make_float4(0, 0, 0, 0);
     if (valid)
         for (int r = threadIdx.y; r < HW; r += RPP) {
-            float4 v = ld4(y.at((size_t)n * HW + r, q * 4));
+            float4 v = y.ld4((size_t)n * HW + r, q * 4);
             s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
         }
     sm4[threadIdx.y * SW + threadIdx.x] = s;
@@ -461,16 +461,18 @@ void sgd_update(Exec &ex, float *params, const float *grads, float *mom, size_t 
     ex.check("sgd", (double)n * 20);
 }
 
-__global__ void max_abs_diff_kernel(const float *__restrict__ a, const float *__restrict__ b, size_t n, float *out) {
+__global__ void max_abs_diff_kernel(const float *__restrict__ a, const float *__restrict__ b, size_t n, float q, float *out) {
     float m = 0.f;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x)
-        m = fmaxf(m, fabsf(a[i] - b[i]));
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        if (q == 0.f) m = fmaxf(m, fabsf(a[i] - b[i]));
+        else m = fmaxf(m, fabsf((float)(reinterpret_cast<const int *>(a)[i] - reinterpret_cast<const int *>(b)[i])) * q);
+    }
     for (int o = 16; o; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
     if ((threadIdx.x & 31) == 0) atomicMax(reinterpret_cast<int *>(out), __float_as_int(m));   // m >= 0
 }
-void max_abs_diff(Exec &ex, const float *a, const float *b, size_t n, float *out) {
+void max_abs_diff(Exec &ex, const float *a, const float *b, size_t n, float q, float *out) {
     if (ex.dry) return;
-    max_abs_diff_kernel<<<ew_grid(n, ex.ctx->sm_count), 256, 0, ex.stream>>>(a, b, n, out);
+    max_abs_diff_kernel<<<ew_grid(n, ex.ctx->sm_count), 256, 0, ex.stream>>>(a, b, n, q, out);
     ex.check("max_abs_diff");
 }
 void fill_zero(Exec &ex, void *p, size_t bytes) {

@@ -6,6 +6,7 @@
 #include <string.h>
 #include <array>
 #include <stdlib.h>
+#include <math.h>
 
 struct LayerSlot { int cin, cout, k, stride; size_t off_gamma, off_beta, off_W; };   // offsets in floats; stem: gamma/beta unused
 
@@ -62,6 +63,7 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
     const revnet_stack_desc &d = pl->d;
     const int N = d.N, S = d.n_stages;
     auto actf = [&](size_t off) { return (float *)(act + off); };
+    const float q = ex.q;   // format of the stage buffers (the coupling state)
 
     ex.mark("step_begin");
     // ---- step-long scratch
@@ -88,7 +90,7 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
     Geom gimg{N, d.img, d.img};
     StagePlan &s0 = pl->st[0];
     if (pl->stem_direct)
-        conv_fprop_simt(ex, images, false, gimg, stem, halves(actf(s0.off_x1), actf(s0.off_x2), s0.c), Pair{}, 0);
+        conv_fprop_simt(ex, images, false, gimg, stem, halves(actf(s0.off_x1), actf(s0.off_x2), s0.c, q), Pair{}, 0);
     else
         conv_fprop_simt(ex, images, false, gimg, stem, single(actf(pl->off_stem_out), d.stem_cout), Pair{}, 0);
     Pair prev = single(actf(pl->off_stem_out), d.stem_cout);
@@ -104,7 +106,7 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
         Geom g{N, s.H, s.H};
         if (s.has_trans) {
             std::vector<Layer> T{bind(s.trans, params, grads)};
-            fn_forward(ex, Geom{N, prevH, prevH}, prev, T, Pair{}, halves(x1, x2, s.c), 0, nullptr, false);
+            fn_forward(ex, Geom{N, prevH, prevH}, prev, T, Pair{}, halves(x1, x2, s.c, q), 0, nullptr, false);
         }
         if (d.verify_reconstruction && !ex.dry) {
             size_t b = g.P() * s.c * sizeof(float);
@@ -113,7 +115,7 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
         }
         for (int u = 0; u < s.units; u++)
             block_forward(ex, g, s.c, bind(s.F[u], params, grads), bind(s.G[u], params, grads), x1, x2, x1, x2);
-        prev = halves(x1, x2, s.c);
+        prev = halves(x1, x2, s.c, q);
         prevH = s.H;
     }
     StagePlan &top = pl->st[S - 1];
@@ -136,15 +138,15 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
         for (int u = s.units - 1; u >= 0; u--)
             block_backward(ex, g, s.c, bind(s.F[u], params, grads), bind(s.G[u], params, grads), x1, x2, d1, d2, x1, x2, d1, d2);
         if (d.verify_reconstruction) {
-            max_abs_diff(ex, x1, actf(s.off_v1), half, recon + si);
-            max_abs_diff(ex, x2, actf(s.off_v2), half, recon + si);
+            max_abs_diff(ex, x1, actf(s.off_v1), half, q, recon + si);
+            max_abs_diff(ex, x2, actf(s.off_v2), half, q, recon + si);
         }
         if (s.has_trans) {
             std::vector<Layer> T{bind(s.trans, params, grads)};
             Pair tin; int tH; Pair gout;
             if (si > 0) {
                 StagePlan &p = pl->st[si - 1];
-                tin = halves(actf(p.off_x1), actf(p.off_x2), p.c); tH = p.H;
+                tin = halves(actf(p.off_x1), actf(p.off_x2), p.c, q); tH = p.H;
                 size_t ph = (size_t)N * p.H * p.H * p.c;
                 gout = halves(gbuf[gi ^ 1], gbuf[gi ^ 1] + ph, p.c);
             } else {
@@ -202,6 +204,7 @@ extern "C" int revnet_stack_plan(revnet_ctx *ctx, const revnet_stack_desc *desc,
     if ((d.stem_k != 3 && d.stem_k != 7) || (d.stem_stride != 1 && d.stem_stride != 2) || d.stem_cout % 4)
         return fail(ctx, REVNET_E_UNSUPPORTED_SHAPE, "revnet_stack_plan: stem must be 3x3 or 7x7, stride 1 or 2, cout % 4 == 0");
     if (d.mode != 0 && d.mode != 1) return fail(ctx, REVNET_E_INVALID_ARG, "revnet_stack_plan: mode must be 0 or 1");
+    if (d.state_frac_bits < 0 || d.state_frac_bits > 24) return fail(ctx, REVNET_E_INVALID_ARG, "revnet_stack_plan: state_frac_bits must be in [0,24]");
     revnet_plan *pl = new revnet_plan();
     pl->ctx = ctx; pl->d = d;
     size_t off = 0;
@@ -270,6 +273,7 @@ extern "C" int revnet_stack_plan(revnet_ctx *ctx, const revnet_stack_desc *desc,
     memcpy((char *)pl->pinned + nseg * 4, pl->seg_decay.data(), nseg);
     // size the workspace with a dry run of the very same driver
     Exec ex; ex.ctx = ctx; ex.dry = true; ex.ws.dry = true; ex.mode = d.mode; ex.eps = d.eps;
+    ex.q = d.state_frac_bits ? ldexpf(1.f, -d.state_frac_bits) : 0.f;
     run_step(pl, ex, nullptr, nullptr, (float *)0x1000, (float *)0x1000, (float *)0x1000, (char *)0x1000, nullptr, nullptr, nullptr, nullptr, nullptr);
     pl->ws_bytes = ex.ws.peak + 256;
     if (param_count) *param_count = pl->n_params;
@@ -295,6 +299,7 @@ extern "C" int revnet_train_step(revnet_ctx *ctx, revnet_plan *pl, const float *
     for (const void *p : ptrs)
         if ((uintptr_t)p & 15) return fail(ctx, REVNET_E_MISALIGNED, "revnet_train_step: pointers must be 16-byte aligned");
     Exec ex; ex.ctx = ctx; ex.dry = false; ex.mode = pl->d.mode; ex.eps = pl->d.eps; ex.stream = (cudaStream_t)stream;
+    ex.q = pl->d.state_frac_bits ? ldexpf(1.f, -pl->d.state_frac_bits) : 0.f;
     ex.ws.dry = false; ex.ws.base = (char *)workspace; ex.ws.cap = pl->ws_bytes;
     float *recon = nullptr;
     run_step(pl, ex, images, labels, params, grads, momentum, (char *)activations, loss, pred, logits, stats, &recon);

@@ -16,10 +16,29 @@ def _dev(a, dtype=torch.float32):
     return torch.from_numpy(np.ascontiguousarray(a)).to(dtype).cuda()
 
 
+DEFAULT_FRAC_BITS = {0: 16, 1: 0}   # bf16 mode runs on the exactly invertible fixed-point state
+
+
+def to_state(x_nchw: np.ndarray, frac_bits: int):
+    """NCHW float array -> device NHWC tensor in the state format (float32, or int32 fixed point)."""
+    x = B.to_nhwc(np.asarray(x_nchw, np.float32))
+    if frac_bits == 0:
+        return torch.from_numpy(x).cuda()
+    return torch.from_numpy(np.rint(x.astype(np.float64) * (1 << frac_bits)).astype(np.int32)).cuda()
+
+
+def from_state(t: torch.Tensor, frac_bits: int) -> np.ndarray:
+    """device NHWC state tensor -> NCHW float64 array (exact for fixed point)."""
+    a = t.cpu().numpy()
+    a = a.astype(np.float64) if frac_bits == 0 else a.astype(np.float64) / (1 << frac_bits)
+    return B.to_nchw(a)
+
+
 class BlockRunner:
-    def __init__(self, ctx: B.Context, b: syn.BlockCfg, mode: int):
+    def __init__(self, ctx: B.Context, b: syn.BlockCfg, mode: int, frac_bits: int = None):
         self.ctx, self.b, self.mode = ctx, b, mode
-        self.desc = B.block_desc(b, mode)
+        self.frac = DEFAULT_FRAC_BITS[mode] if frac_bits is None else frac_bits
+        self.desc = B.block_desc(b, mode, self.frac)
         fwd, bwd = B.revnet_block_workspace_bytes(ctx, self.desc)
         self.ws = torch.empty(max(fwd, bwd), dtype=torch.uint8, device="cuda")
         self.layers = syn.fn_layers(b.kind, b.c, b.w)
@@ -34,19 +53,21 @@ class BlockRunner:
         self.gG = [{k: torch.zeros_like(v) for k, v in l.items()} for l in self.G]
 
     def forward(self, x1, x2, inplace=False):
-        """x1, x2: NCHW numpy -> y1, y2 NCHW numpy"""
-        dx1, dx2 = _dev(B.to_nhwc(x1)), _dev(B.to_nhwc(x2))
+        """x1, x2: NCHW numpy -> y1, y2 NCHW numpy (values of the state format, exact)"""
+        dx1, dx2 = to_state(x1, self.frac), to_state(x2, self.frac)
         y1, y2 = (dx1, dx2) if inplace else (torch.empty_like(dx1), torch.empty_like(dx2))
         B.revnet_block_fwd(self.ctx, self.desc, dx1, dx2, self.F, self.G, y1, y2, self.ws)
         torch.cuda.synchronize()
-        return B.to_nchw(y1.cpu().numpy()), B.to_nchw(y2.cpu().numpy())
+        return from_state(y1, self.frac), from_state(y2, self.frac)
 
     def backward(self, y1, y2, dy1, dy2, inplace=False):
-        ty1, ty2, tdy1, tdy2 = (_dev(B.to_nhwc(t)) for t in (y1, y2, dy1, dy2))
+        ty1, ty2 = to_state(y1, self.frac), to_state(y2, self.frac)
+        tdy1, tdy2 = (_dev(B.to_nhwc(t)) for t in (dy1, dy2))
         if inplace:
             x1, x2, dx1, dx2 = ty1, ty2, tdy1, tdy2
         else:
-            x1, x2, dx1, dx2 = (torch.empty_like(ty1) for _ in range(4))
+            x1, x2 = torch.empty_like(ty1), torch.empty_like(ty2)
+            dx1, dx2 = torch.empty_like(tdy1), torch.empty_like(tdy2)
         B.revnet_block_bwd(self.ctx, self.desc, ty1, ty2, tdy1, tdy2, self.F, self.G, x1, x2, dx1, dx2, self.gF, self.gG, self.ws)
         torch.cuda.synchronize()
         grads = {}
@@ -55,15 +76,17 @@ class BlockRunner:
                 grads[f"{fn}.l{i}.W"] = B.w_from_abi(l["W"].cpu().numpy())
                 grads[f"{fn}.l{i}.gamma"] = l["gamma"].cpu().numpy()
                 grads[f"{fn}.l{i}.beta"] = l["beta"].cpu().numpy()
-        out = [B.to_nchw(t.cpu().numpy()) for t in (x1, x2, dx1, dx2)]
-        return out[0], out[1], out[2], out[3], grads
+        return (from_state(x1, self.frac), from_state(x2, self.frac),
+                B.to_nchw(dx1.cpu().numpy()), B.to_nchw(dx2.cpu().numpy()), grads)
 
 
 class StackRunner:
-    def __init__(self, ctx: B.Context, cfg: syn.StackCfg, mode: int, verify_reconstruction: bool = False):
+    def __init__(self, ctx: B.Context, cfg: syn.StackCfg, mode: int, verify_reconstruction: bool = False,
+                 frac_bits: int = None):
         self.ctx, self.cfg, self.mode = ctx, cfg, mode
+        self.frac = DEFAULT_FRAC_BITS[mode] if frac_bits is None else frac_bits
         self.specs = syn.param_specs(cfg)
-        self.desc = B.stack_desc(cfg, mode, verify_reconstruction)
+        self.desc = B.stack_desc(cfg, mode, verify_reconstruction, self.frac)
         self.plan = B.revnet_stack_plan(ctx, self.desc)
         n = self.plan.param_count
         assert n == sum(int(np.prod(s)) for _, s, _ in self.specs)

@@ -196,6 +196,12 @@ int revnet_train_step_host(revnet_ctx *ctx, revnet_plan *plan,
                            float *loss_host, int32_t *pred_host,
                            revnet_step_stats *stats, void *stream);
 
+/* Waits inside the library's kernels (on shared-memory barriers) are bounded; a kernel whose wait
+ * runs out stops its work, records a status word on the device and exits normally.
+ * revnet_check_device synchronises the stream, returns REVNET_OK or that status (REVNET_E_TIMEOUT)
+ * and clears it.  No counterpart in the paper: failure reporting. */
+int revnet_check_device(revnet_ctx *ctx, void *stream);
+
 /* ---- per-kernel timing (no counterpart in the paper: measurement support) ----
  * While enabled, every kernel the library launches on behalf of this context is followed by a
  * CUDA event on the caller's stream.  revnet_profile_summary waits for the last event and writes

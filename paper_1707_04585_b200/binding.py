@@ -21,7 +21,7 @@ _lib = None
 
 EXPORTS = ["revnet_create", "revnet_destroy", "revnet_last_error", "revnet_block_workspace_bytes",
            "revnet_block_fwd", "revnet_block_bwd", "revnet_stack_plan", "revnet_plan_destroy",
-           "revnet_train_step", "revnet_train_step_host", "revnet_profile_enable", "revnet_profile_summary"]
+           "revnet_train_step", "revnet_train_step_host", "revnet_profile_enable", "revnet_profile_summary", "revnet_check_device"]
 
 
 class FnDesc(C.Structure):
@@ -290,3 +290,8 @@ def revnet_profile_summary(ctx):
         name, n, ms, by, fl = line.split("\t")
         out[name] = dict(launches=int(n), ms=float(ms), bytes=float(by), flops=float(fl))
     return out
+
+
+def revnet_check_device(ctx):
+    """Synchronise and raise if a kernel reported that it gave up a bounded wait."""
+    ctx.check(lib().revnet_check_device(ctx.h, _stream()), "revnet_check_device")

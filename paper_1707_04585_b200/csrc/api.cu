@@ -146,6 +146,23 @@ extern "C" int revnet_block_bwd(revnet_ctx *ctx, const revnet_block_desc *d, con
     return finish(ctx, ex, "revnet_block_bwd");
 }
 
+// ---- device-side status
+extern "C" int revnet_check_device(revnet_ctx *ctx, void *stream) {
+    if (!ctx) return REVNET_E_INVALID_ARG;
+    if (!ctx->dev_status) return REVNET_OK;
+    int st = 0;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (cudaMemcpyAsync(&st, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess ||
+        cudaStreamSynchronize(s) != cudaSuccess)
+        return fail(ctx, REVNET_E_CUDA, std::string("revnet_check_device: ") + cudaGetErrorString(cudaGetLastError()));
+    if (st != 0) {
+        cudaMemsetAsync(ctx->dev_status, 0, sizeof(int), s);
+        cudaStreamSynchronize(s);
+        return fail(ctx, st, "a kernel gave up a bounded wait (device status " + std::to_string(st) + ")");
+    }
+    return REVNET_OK;
+}
+
 // ---- per-kernel timing
 extern "C" int revnet_profile_enable(revnet_ctx *ctx, int on) {
     if (!ctx) return REVNET_E_INVALID_ARG;

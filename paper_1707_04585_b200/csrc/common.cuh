@@ -58,6 +58,27 @@ struct Pair {
             *reinterpret_cast<int *>(o) = iv;
         }
     }
+    // four consecutive channels at once (ch % 4 == 0)
+    __device__ __forceinline__ void couple4(size_t row, int ch, float4 v, const Pair &partner, int sign) const {
+        float *o = at(row, ch);
+        if (q == 0.f) {
+            if (sign) {
+                float4 p = *reinterpret_cast<const float4 *>(partner.at(row, ch));
+                if (sign > 0) { v.x = p.x + v.x; v.y = p.y + v.y; v.z = p.z + v.z; v.w = p.w + v.w; }
+                else { v.x = p.x - v.x; v.y = p.y - v.y; v.z = p.z - v.z; v.w = p.w - v.w; }
+            }
+            *reinterpret_cast<float4 *>(o) = v;
+        } else {
+            const float s = 1.f / q;
+            int4 iv = make_int4(__float2int_rn(v.x * s), __float2int_rn(v.y * s), __float2int_rn(v.z * s), __float2int_rn(v.w * s));
+            if (sign) {
+                int4 p = *reinterpret_cast<const int4 *>(partner.at(row, ch));
+                if (sign > 0) { iv.x = p.x + iv.x; iv.y = p.y + iv.y; iv.z = p.z + iv.z; iv.w = p.w + iv.w; }
+                else { iv.x = p.x - iv.x; iv.y = p.y - iv.y; iv.z = p.z - iv.z; iv.w = p.w - iv.w; }
+            }
+            *reinterpret_cast<int4 *>(o) = iv;
+        }
+    }
 #endif
 };
 static inline Pair single(float *p, int C, float q = 0.f) { return Pair{p, nullptr, C, 0, q}; }

@@ -1,7 +1,350 @@
-// Tensor-core convolution kernels (tcgen05 / TMEM / TMA).  Each entry returns false when it does
-// not take the shape, and the caller then runs the fp32 kernel.
+// Tensor-core convolution for sm_100a: implicit GEMM with bf16 operands, fp32 accumulation in
+// tensor memory (tcgen05.mma), operand tiles staged in shared memory by TMA.
+//
+//   out[p, co] = sum_{tap, ci} a[p (+) tap, ci] * Wp[co, tap, ci]        (Eq. 2, Conv_kxk; stride 1)
+//
+// GEMM view: M = 128 output pixels per CTA (whole image rows, so a tile is one TMA box of the NHWC
+// tensor), N = output channels, K = taps x input channels.  For every tap the A tile is the same
+// box shifted by (kh - pad, kw - pad); TMA zero-fills what falls outside the image, which is
+// exactly the convolution's zero padding because the activated tensor is materialised.
+// dgrad is the same kernel run on the upstream gradient with the tap-mirrored, transposed pack
+// of the weights.  Each entry point returns false for shapes it does not take.
+//
+// Roles inside a CTA (192 threads): warp 0 issues TMA loads, warp 1 allocates tensor memory and
+// issues the MMAs, warps 2..5 drain the accumulator (tcgen05.ld), apply the coupling epilogue
+// (out = partner +/- acc on the float or fixed-point state) and store.
+// Every mbarrier wait is bounded; on expiry the kernel records a status word and leaves.
 #include "common.cuh"
+#include <cuda.h>
 
-bool conv_fprop_tc(Exec &, const void *, Geom, const Layer &, Pair, Pair, int) { return false; }
-bool conv_dgrad_tc(Exec &, const void *, Geom, const Layer &, float *) { return false; }
+namespace {
+
+constexpr int kStages = 4;
+constexpr int kThreads = 192;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any real wait of this kernel
+
+struct TcParams {
+    int taps;        // k*k
+    int k;           // kernel size
+    int chunks;      // channel chunks per tap
+    int KC;          // channels per chunk (16, 32 or 64)
+    int cin_pad;     // chunks * KC
+    int BN;          // N tile
+    int n_cols;      // valid output channels
+    int H, W;        // image size
+    int BH, BIMG;    // tile: BH rows x W columns x BIMG images = 128 pixels
+    Pair out, partner;
+    int sign;
+    int *status;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// bounded wait: false when the limit ran out
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+    const uint32_t addr = smem_u32(bar);
+    unsigned long long t0 = 0;
+    for (uint32_t it = 0;; it++) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+        if (done) return true;
+        if ((it & 63) == 63) {
+            unsigned long long now;
+            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > kWaitLimitNs) return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2, int c3) {
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
+}
+
+// shared-memory matrix descriptor, K-major operand whose rows are `row_bytes` (32/64/128) long and
+// stored with the matching TMA swizzle; 8-row groups are row_bytes*8 apart
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, int row_bytes) {
+    const uint64_t layout = row_bytes == 128 ? 2 : (row_bytes == 64 ? 4 : 6);
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFF) >> 4);                 // start address
+    d |= (uint64_t)1 << 16;                                 // leading byte offset (unused for swizzled K-major)
+    d |= (uint64_t)((row_bytes * 8) >> 4) << 32;            // stride byte offset between 8-row groups
+    d |= (uint64_t)1 << 46;                                 // descriptor version
+    d |= layout << 61;
+    return d;
+}
+
+// instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128
+__device__ __forceinline__ uint32_t instr_desc(int n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+__device__ __forceinline__ void mma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int i = 0; i < 16; i++) v[i] = __uint_as_float(r[i]);
+}
+
+struct __align__(8) TcShared {
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    uint64_t acc_full;
+    uint32_t tmem_base;
+    uint32_t failed;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    // operand stages first (1024-byte aligned for the 128-byte swizzle), bookkeeping behind them
+    uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int a_bytes = 128 * p.KC * 2, b_bytes = p.BN * p.KC * 2;
+    const int b_off = (a_bytes + 1023) & ~1023;
+    const int stage_bytes = b_off + ((b_bytes + 1023) & ~1023);
+    TcShared *sh = (TcShared *)(tiles + kStages * stage_bytes);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int iters = p.taps * p.chunks;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < p.BN) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; s++) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+        mbar_init(&sh->acc_full, 1);
+        sh->failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_d = sh->tmem_base;
+
+    // tile origin: tiles are runs of 128 consecutive pixels in (n, h, w) order
+    const int tiles_per_img = p.BIMG > 1 ? 1 : p.H / p.BH;
+    const int n0 = p.BIMG > 1 ? blockIdx.x * p.BIMG : blockIdx.x / tiles_per_img;
+    const int h0 = p.BIMG > 1 ? 0 : (blockIdx.x % tiles_per_img) * p.BH;
+    const int col0 = blockIdx.y * p.BN;
+    const int pad = p.k / 2;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int it = 0; it < iters; it++) {
+                const int s = it % kStages, round = it / kStages;
+                if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); break; }
+                const int tap = it / p.chunks, ch = it - tap * p.chunks;
+                const int kh = tap / p.k, kw = tap - kh * p.k;
+                uint8_t *sa = tiles + s * stage_bytes;
+                mbar_expect_tx(&sh->full[s], (uint32_t)(a_bytes + b_bytes));
+                tma_load_4d(sa, &map_a, &sh->full[s], ch * p.KC, kw - pad, h0 + kh - pad, n0);
+                tma_load_2d(sa + b_off, &map_b, &sh->full[s], tap * p.cin_pad + ch * p.KC, col0);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(p.BN);
+            const int row_bytes = p.KC * 2;
+            bool ok = true;
+            for (int it = 0; it < iters && ok; it++) {
+                const int s = it % kStages, round = it / kStages;
+                if (!mbar_wait(&sh->full[s], round & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t sa = smem_u32(tiles + s * stage_bytes);
+                for (int kk = 0; kk < p.KC / 16; kk++) {
+                    const uint64_t da = smem_desc(sa + kk * 32, row_bytes);
+                    const uint64_t db = smem_desc(sa + b_off + kk * 32, row_bytes);
+                    mma_bf16(tmem_d, da, db, idesc, (it > 0 || kk > 0) ? 1u : 0u);
+                }
+                mma_commit(&sh->empty[s]);          // frees the stage once these MMAs have read it
+            }
+            mma_commit(&sh->acc_full);              // accumulator complete (also issued after a failure, so nobody waits forever)
+        }
+    } else {
+        // epilogue: warp w owns accumulator lanes 32*(w%4) .. +31 = pixel rows of the tile
+        const int quarter = warp & 3;
+        const bool ok = mbar_wait(&sh->acc_full, 0);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok && sh->failed == 0) {
+            const size_t row = (size_t)blockIdx.x * 128 + quarter * 32 + lane;
+            for (int c = 0; c < p.BN; c += 16) {
+                float v[16];
+                tmem_ld16(tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, v);
+#pragma unroll
+                for (int j = 0; j < 16; j += 4) {
+                    const int col = col0 + c + j;
+                    if (col < p.n_cols) p.out.couple4(row, col, make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]), p.partner, p.sign);
+                }
+            }
+        } else if (lane == 0) {
+            atomicExch(&sh->failed, 1u);
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x == 0 && sh->failed) atomicExch(p.status, (int)REVNET_E_TIMEOUT);
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(tmem_cols) : "memory");
+    }
+}
+
+// ---- weight packs: bf16 [rows_pad][taps][cin_pad]; transposed = true builds the dgrad operand
+// (rows = input channels, columns = output channels, taps mirrored)
+__global__ void pack_weights_kernel(const float *__restrict__ W, bf16 *__restrict__ out, int Co, int Ci, int k,
+                                    int rows_pad, int cols_pad, int transposed) {
+    const int taps = k * k;
+    const size_t n = (size_t)rows_pad * taps * cols_pad;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % cols_pad);
+        const int tap = (int)((i / cols_pad) % taps);
+        const int r = (int)(i / ((size_t)cols_pad * taps));
+        float v = 0.f;
+        if (!transposed) { if (r < Co && c < Ci) v = W[((size_t)r * taps + tap) * Ci + c]; }
+        else { if (r < Ci && c < Co) v = W[((size_t)c * taps + (taps - 1 - tap)) * Ci + r]; }
+        out[i] = __float2bfloat16_rn(v);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encoder(revnet_ctx *ctx) {
+    if (!ctx->encode_tiled) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || qres != cudaDriverEntryPointSuccess)
+            fn = nullptr;
+        ctx->encode_tiled = fn;
+    }
+    return (EncodeTiledFn)ctx->encode_tiled;
+}
+
+int round_up(int x, int m) { return (x + m - 1) / m * m; }
+
+struct TcShape { int KC, cin_pad, chunks, BN, n_tiles, BH, BIMG, smem; };
+
+// Which shapes the kernel takes: stride 1, k in {1,3}; a 128-pixel tile must be whole rows of one
+// image or whole images; channel rows 16-byte aligned for TMA.
+bool tc_shape(Geom g, int cin, int cout, int k, int stride, TcShape &s) {
+    if (stride != 1 || (k != 1 && k != 3) || cin % 8 || cout % 4) return false;
+    const int W = g.W, H = g.H;
+    if (W > 128 || 128 % W) return false;
+    if (H * W >= 128) { if (H % (128 / W)) return false; s.BH = 128 / W; s.BIMG = 1; }
+    else { if (128 % (H * W) || g.N % (128 / (H * W))) return false; s.BH = H; s.BIMG = 128 / (H * W); }
+    s.cin_pad = round_up(cin, 16);
+    s.KC = s.cin_pad % 64 == 0 ? 64 : (s.cin_pad % 32 == 0 ? 32 : 16);
+    s.chunks = s.cin_pad / s.KC;
+    const int cout_pad = round_up(cout, 16);
+    s.BN = cout_pad <= 128 ? cout_pad : 128;
+    s.n_tiles = (cout_pad + s.BN - 1) / s.BN;
+    const int a_bytes = 128 * s.KC * 2, b_bytes = s.BN * s.KC * 2;
+    s.smem = 1024 + kStages * (((a_bytes + 1023) & ~1023) + ((b_bytes + 1023) & ~1023)) + (int)sizeof(TcShared) + 64;
+    return true;
+}
+
+// act: bf16 [N,H,W,cin]; Wsrc: fp32 weights; transposed selects the dgrad pack
+bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom g, int cin, int cout, int k, int stride,
+                 const float *Wsrc, bool transposed, Pair out, Pair partner, int sign) {
+    TcShape s;
+    if (!tc_shape(g, cin, cout, k, stride, s)) return false;
+    const int taps = k * k, cout_pad = round_up(cout, 16);
+    const int rows_pad = s.n_tiles * s.BN;
+    if (!ex.dry && !encoder(ex.ctx)) return false;
+    ex.flops += 2ull * g.P() * cout * cin * taps;
+    size_t m = ex.ws.mark();
+    bf16 *wp = ex.ws.get<bf16>((size_t)rows_pad * taps * s.cin_pad);
+    (void)cout_pad;
+    if (!ex.dry) {
+        EncodeTiledFn enc = encoder(ex.ctx);
+        // the pack is rebuilt from the fp32 master weights on every call
+        {
+            const size_t n = (size_t)rows_pad * taps * s.cin_pad;
+            int grid = (int)((n + 255) / 256); if (grid > ex.ctx->sm_count * 4) grid = ex.ctx->sm_count * 4;
+            if (!transposed) pack_weights_kernel<<<grid, 256, 0, ex.stream>>>(Wsrc, wp, cout, cin, k, rows_pad, s.cin_pad, 0);
+            else pack_weights_kernel<<<grid, 256, 0, ex.stream>>>(Wsrc, wp, cin, cout, k, rows_pad, s.cin_pad, 1);
+            ex.check("pack_weights", (double)n * 6);
+        }
+        CUtensorMap map_a, map_b;
+        const CUtensorMapSwizzle sw = s.KC == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : (s.KC == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+        {
+            cuuint64_t dims[4] = {(cuuint64_t)cin, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N};
+            cuuint64_t strides[3] = {(cuuint64_t)cin * 2, (cuuint64_t)g.W * cin * 2, (cuuint64_t)g.H * g.W * cin * 2};
+            cuuint32_t box[4] = {(cuuint32_t)s.KC, (cuuint32_t)g.W, (cuuint32_t)s.BH, (cuuint32_t)s.BIMG};
+            cuuint32_t es[4] = {1, 1, 1, 1};
+            CUresult r = enc(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void *)act, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                             sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) { ex.failed = true; ex.ctx->err = std::string(what) + ": tensor map (activations) rejected"; ex.ws.release(m); return true; }
+        }
+        {
+            cuuint64_t dims[2] = {(cuuint64_t)taps * s.cin_pad, (cuuint64_t)rows_pad};
+            cuuint64_t strides[1] = {(cuuint64_t)taps * s.cin_pad * 2};
+            cuuint32_t box[2] = {(cuuint32_t)s.KC, (cuuint32_t)s.BN};
+            cuuint32_t es[2] = {1, 1};
+            CUresult r = enc(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void *)wp, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                             sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+            if (r != CUDA_SUCCESS) { ex.failed = true; ex.ctx->err = std::string(what) + ": tensor map (weights) rejected"; ex.ws.release(m); return true; }
+        }
+        TcParams p;
+        p.taps = taps; p.k = k; p.chunks = s.chunks; p.KC = s.KC; p.cin_pad = s.cin_pad; p.BN = s.BN; p.n_cols = cout;
+        p.H = g.H; p.W = g.W; p.BH = s.BH; p.BIMG = s.BIMG; p.out = out; p.partner = partner; p.sign = sign; p.status = ex.ctx->dev_status;
+        static bool attr_set = false;
+        if (!attr_set) { cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); attr_set = true; }
+        dim3 grid((unsigned)(g.P() / 128), (unsigned)s.n_tiles);
+        conv_tc_kernel<<<grid, kThreads, s.smem, ex.stream>>>(map_a, map_b, p);
+        const double bytes = (double)g.P() * cin * 2 + (double)g.P() * cout * (sign ? 8 : 4) + (double)cout * taps * cin * 2;
+        ex.check(what, bytes, 2.0 * g.P() * cout * cin * taps);
+    }
+    ex.ws.release(m);
+    return true;
+}
+
+}  // namespace
+
+bool conv_fprop_tc(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign) {
+    return run_conv_tc(ex, "conv_fprop_tc", a, gi, L.cin, L.cout, L.k, L.stride, L.W, false, out, partner, sign);
+}
+
+// da[q,ci] = sum_{tap,co} g[q (-) tap, co] W[co,tap,ci]: a stride-1 convolution of g with the mirrored, transposed weights
+bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da) {
+    return run_conv_tc(ex, "conv_dgrad_tc", g, gi, L.cout, L.cin, L.k, L.stride, L.W, true, single(da, L.cin), Pair{}, 0);
+}
+
 bool conv_wgrad_tc(Exec &, const void *, const void *, Geom, const Layer &, float *) { return false; }

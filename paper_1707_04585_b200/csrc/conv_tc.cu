@@ -92,9 +92,24 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, int row_bytes) {
     return d;
 }
 
-// instruction descriptor: bf16 x bf16 -> fp32, both operands K-major, M = 128
-__device__ __forceinline__ uint32_t instr_desc(int n) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+// instruction descriptor: bf16 x bf16 -> fp32, M = 128; mn_major: both operands have their M / N
+// index contiguous in shared memory (pixel-major tiles of the weight-gradient GEMM), else K-major
+__device__ __forceinline__ uint32_t instr_desc(int n, bool mn_major = false) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | (mn_major ? (3u << 15) : 0u) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+}
+
+// descriptor of an MN-major operand: rows are K indices, each row holds `row_bytes` (32/64/128) of
+// contiguous M (or N) elements with the matching swizzle; the next block of M / N elements starts
+// `block_bytes` further on, groups of 8 K-rows are row_bytes*8 apart
+__device__ __forceinline__ uint64_t smem_desc_mn(uint32_t addr, int row_bytes, int block_bytes) {
+    const uint64_t layout = row_bytes == 128 ? 2 : (row_bytes == 64 ? 4 : 6);
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3FFFF) >> 4);
+    d |= (uint64_t)((block_bytes >> 4) & 0x3FFF) << 16;     // leading byte offset: between M / N blocks
+    d |= (uint64_t)((row_bytes * 8) >> 4) << 32;            // stride byte offset: between 8-row K groups
+    d |= (uint64_t)1 << 46;
+    d |= layout << 61;
+    return d;
 }
 
 __device__ __forceinline__ void mma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
@@ -336,6 +351,168 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom g, int cin, i
     return true;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Weight gradient:  dW[co, tap, ci] = sum_p g[p, co] * a[p (+) tap, ci]
+// GEMM view: the reduction runs over pixels.  Both operands are pixel-major in memory, so the tiles
+// TMA delivers ([128 pixels][channel block]) are MN-major operands as they stand.  The M side
+// stacks (tap, input-channel block) tiles -- one shifted TMA box each -- 128 rows per MMA group;
+// the N side is a block of output channels.  A CTA owns up to two M groups and one N tile, walks
+// its share of the pixel tiles (split-K) accumulating in tensor memory, and writes an fp32
+// partial; the partials are summed in fixed order by splitk_sum_kernel.
+struct WgParams {
+    int taps, k;
+    int blockC, cblks, cin;      // input-channel block (16/32/64), blocks per tap, valid channels
+    int total_blocks;            // taps * cblks
+    int blockN, BN, cout;        // output-channel block, N tile, valid channels
+    int GM;                      // M groups per CTA (1 or 2)
+    int H, W, BH, BIMG;
+    int n_tiles_px;              // pixel tiles in all
+    int stages;
+    float *partial;              // [splits][cout][taps][cin]
+    size_t slice;                // cout*taps*cin
+    int *status;
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_g, const WgParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int blk_bytes_a = 256 * p.blockC, blk_bytes_b = 256 * p.blockN;   // [128 pixels][block] bf16
+    const int a_region = p.GM * 32768;                                       // 128 M rows x 128 pixels x 2 B per group
+    const int stage_bytes = a_region + ((256 * p.BN + 1023) & ~1023);
+    TcShared *sh = (TcShared *)(tiles + p.stages * stage_bytes);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bpg = 128 / p.blockC;                          // blocks per M group
+    const int first_block = blockIdx.y * p.GM * bpg;
+    int n_blocks = p.total_blocks - first_block; if (n_blocks > p.GM * bpg) n_blocks = p.GM * bpg;
+    const int groups = (n_blocks + bpg - 1) / bpg;
+    const int col0 = blockIdx.z * p.BN;
+    int nb_n = (p.cout - col0 + p.blockN - 1) / p.blockN; if (nb_n > p.BN / p.blockN) nb_n = p.BN / p.blockN;   // N blocks holding valid channels
+    const int my_tiles = (p.n_tiles_px - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < p.GM * p.BN) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; s++) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+        mbar_init(&sh->acc_full, 1);
+        sh->failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem_d = sh->tmem_base;
+    const int pad = p.k / 2;
+    const int tiles_per_img = p.BIMG > 1 ? 1 : p.H / p.BH;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            const uint32_t tx = (uint32_t)(n_blocks * blk_bytes_a + nb_n * blk_bytes_b);
+            for (int it = 0; it < my_tiles; it++) {
+                const int s = it % p.stages, round = it / p.stages;
+                if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); break; }
+                const int t = blockIdx.x + it * gridDim.x;
+                const int n0 = p.BIMG > 1 ? t * p.BIMG : t / tiles_per_img;
+                const int h0 = p.BIMG > 1 ? 0 : (t % tiles_per_img) * p.BH;
+                uint8_t *sa = tiles + s * stage_bytes;
+                mbar_expect_tx(&sh->full[s], tx);
+                for (int b = 0; b < n_blocks; b++) {
+                    const int gb = first_block + b, tap = gb / p.cblks, cb = gb - tap * p.cblks;
+                    const int kh = tap / p.k, kw = tap - kh * p.k;
+                    tma_load_4d(sa + b * blk_bytes_a, &map_a, &sh->full[s], cb * p.blockC, kw - pad, h0 + kh - pad, n0);
+                }
+                for (int b = 0; b < nb_n; b++)
+                    tma_load_4d(sa + a_region + b * blk_bytes_b, &map_g, &sh->full[s], col0 + b * p.blockN, 0, h0, n0);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = instr_desc(p.BN, true);
+            const int rba = p.blockC * 2, rbb = p.blockN * 2;
+            for (int it = 0; it < my_tiles; it++) {
+                const int s = it % p.stages, round = it / p.stages;
+                if (!mbar_wait(&sh->full[s], round & 1)) { atomicExch(&sh->failed, 1u); break; }
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint32_t sa = smem_u32(tiles + s * stage_bytes);
+                for (int g = 0; g < groups; g++)
+                    for (int ks = 0; ks < 8; ks++) {         // 16 pixels per MMA
+                        const uint64_t da = smem_desc_mn(sa + g * 32768 + ks * 16 * rba, rba, blk_bytes_a);
+                        const uint64_t db = smem_desc_mn(sa + a_region + ks * 16 * rbb, rbb, blk_bytes_b);
+                        mma_bf16(tmem_d + (uint32_t)(g * p.BN), da, db, idesc, (it > 0 || ks > 0) ? 1u : 0u);
+                    }
+                mma_commit(&sh->empty[s]);
+            }
+            mma_commit(&sh->acc_full);
+        }
+    } else {
+        const int quarter = warp & 3;
+        const bool ok = mbar_wait(&sh->acc_full, 0);
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        if (ok && sh->failed == 0) {
+            const int m = quarter * 32 + lane;
+            float *dst = p.partial + (size_t)blockIdx.x * p.slice;
+            for (int g = 0; g < groups; g++) {
+                const int gb = first_block + g * bpg + m / p.blockC;
+                const int tap = gb / p.cblks, ci = (gb - tap * p.cblks) * p.blockC + m % p.blockC;
+                const bool row_ok = gb < p.total_blocks && ci < p.cin;
+                for (int c = 0; c < p.BN; c += 16) {
+                    float v[16];
+                    tmem_ld16(tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(g * p.BN + c), v);   // whole warp takes part
+                    if (row_ok) {
+#pragma unroll
+                        for (int j = 0; j < 16; j++) {
+                            const int co = col0 + c + j;
+                            if (co < p.cout) dst[((size_t)co * p.taps + tap) * p.cin + ci] = my_tiles > 0 ? v[j] : 0.f;
+                        }
+                    }
+                }
+            }
+        } else if (lane == 0) {
+            atomicExch(&sh->failed, 1u);
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (threadIdx.x == 0 && sh->failed) atomicExch(p.status, (int)REVNET_E_TIMEOUT);
+    if (warp == 1) {
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(tmem_cols) : "memory");
+    }
+}
+
+__global__ void splitk_sum_kernel(const float *__restrict__ part, size_t n, int splits, float *__restrict__ out) {
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        float s = 0.f;
+        for (int z = 0; z < splits; z++) s += part[(size_t)z * n + i];
+        out[i] = s;
+    }
+}
+
+int pick_block(int c_pad) { return c_pad % 64 == 0 ? 64 : (c_pad % 32 == 0 ? 32 : 16); }
+
+bool tile_shape(Geom g, int &BH, int &BIMG) {
+    const int W = g.W, H = g.H;
+    if (W > 128 || 128 % W) return false;
+    if (H * W >= 128) { if (H % (128 / W)) return false; BH = 128 / W; BIMG = 1; }
+    else { if (128 % (H * W) || g.N % (128 / (H * W))) return false; BH = H; BIMG = 128 / (H * W); }
+    return true;
+}
+
+bool encode_act_map(Exec &ex, CUtensorMap *map, const void *base, Geom g, int C, int box_c, int BH, int BIMG) {
+    const CUtensorMapSwizzle sw = box_c == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : (box_c == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
+    cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N};
+    cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)g.W * C * 2, (cuuint64_t)g.H * g.W * C * 2};
+    cuuint32_t box[4] = {(cuuint32_t)box_c, (cuuint32_t)g.W, (cuuint32_t)BH, (cuuint32_t)BIMG};
+    cuuint32_t es[4] = {1, 1, 1, 1};
+    return encoder(ex.ctx)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void *)base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 bool conv_fprop_tc(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign) {
@@ -347,4 +524,55 @@ bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da) 
     return run_conv_tc(ex, "conv_dgrad_tc", g, gi, L.cout, L.cin, L.k, L.stride, L.W, true, single(da, L.cin), Pair{}, 0);
 }
 
-bool conv_wgrad_tc(Exec &, const void *, const void *, Geom, const Layer &, float *) { return false; }
+
+bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer &L, float *dW) {
+    if (L.stride != 1 || (L.k != 1 && L.k != 3) || L.cin % 8 || L.cout % 8) return false;
+    WgParams p;
+    if (!tile_shape(gi, p.BH, p.BIMG)) return false;
+    if (!ex.dry && !encoder(ex.ctx)) return false;
+    const int taps = L.k * L.k, cin_pad = round_up(L.cin, 16), cout_pad = round_up(L.cout, 16);
+    p.taps = taps; p.k = L.k; p.cin = L.cin; p.cout = L.cout;
+    p.blockC = pick_block(cin_pad); p.cblks = cin_pad / p.blockC; p.total_blocks = taps * p.cblks;
+    p.blockN = pick_block(cout_pad);
+    p.BN = cout_pad <= 128 ? cout_pad : 128;
+    if (p.BN % p.blockN) p.BN = p.blockN;
+    const int bpg = 128 / p.blockC;
+    const int groups_all = (p.total_blocks + bpg - 1) / bpg;
+    p.GM = groups_all >= 2 ? 2 : 1;
+    const int m_chunks = (groups_all + p.GM - 1) / p.GM;
+    const int n_tiles = (cout_pad + p.BN - 1) / p.BN;
+    p.H = gi.H; p.W = gi.W;
+    p.n_tiles_px = (int)(gi.P() / 128);
+    const int stage_bytes = p.GM * 32768 + ((256 * p.BN + 1023) & ~1023);
+    p.stages = (200 * 1024 - 2048) / stage_bytes; if (p.stages > kStages) p.stages = kStages;
+    if (p.stages < 2) return false;
+    // split the pixel reduction so that the grid covers the machine about twice
+    int splits = (2 * ex.ctx->sm_count + m_chunks * n_tiles - 1) / (m_chunks * n_tiles);
+    if (splits > p.n_tiles_px) splits = p.n_tiles_px;
+    if (splits < 1) splits = 1;
+    p.slice = (size_t)L.cout * taps * L.cin;
+    ex.flops += 2ull * gi.P() * L.cout * L.cin * taps;
+    size_t m = ex.ws.mark();
+    float *part = splits > 1 ? ex.ws.get<float>((size_t)splits * p.slice) : dW;
+    if (!ex.dry) {
+        CUtensorMap map_a, map_g;
+        if (!encode_act_map(ex, &map_a, a, gi, L.cin, p.blockC, p.BH, p.BIMG) || !encode_act_map(ex, &map_g, gq, gi, L.cout, p.blockN, p.BH, p.BIMG)) {
+            ex.failed = true; ex.ctx->err = "conv_wgrad_tc: tensor map rejected"; ex.ws.release(m); return true;
+        }
+        p.partial = part; p.status = ex.ctx->dev_status;
+        static bool attr_set = false;
+        if (!attr_set) { cudaFuncSetAttribute(wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); attr_set = true; }
+        const int smem = 1024 + p.stages * stage_bytes + (int)sizeof(TcShared) + 64;
+        dim3 grid((unsigned)splits, (unsigned)m_chunks, (unsigned)n_tiles);
+        wgrad_tc_kernel<<<grid, kThreads, smem, ex.stream>>>(map_a, map_g, p);
+        const double bytes = (double)gi.P() * (L.cin + L.cout) * 2 + (double)p.slice * 4 * (splits > 1 ? splits : 1);
+        ex.check("conv_wgrad_tc", bytes, 2.0 * gi.P() * L.cout * L.cin * taps);
+        if (splits > 1) {
+            int grid2 = (int)((p.slice + 255) / 256); if (grid2 > ex.ctx->sm_count * 8) grid2 = ex.ctx->sm_count * 8;
+            splitk_sum_kernel<<<grid2, 256, 0, ex.stream>>>(part, p.slice, splits, dW);
+            ex.check("splitk_sum", (double)p.slice * 4 * (splits + 1));
+        }
+    }
+    ex.ws.release(m);
+    return true;
+}

@@ -110,31 +110,43 @@ __global__ void col_reduce_kernel(Pair t, const float *__restrict__ da, size_t P
     }
 }
 
+// one warp per channel: lanes stride the per-CTA partials, double accumulation, fixed butterfly order
+__device__ __forceinline__ void warp_sum2(const float *__restrict__ part, int chunks, int C, int c, double &s, double &ss) {
+    const int lane = threadIdx.x & 31;
+    s = 0; ss = 0;
+    for (int i = lane; i < chunks; i += 32) { s += part[((size_t)i * 2) * C + c]; ss += part[((size_t)i * 2 + 1) * C + c]; }
+    for (int o = 16; o; o >>= 1) { s += __shfl_xor_sync(0xffffffffu, s, o); ss += __shfl_xor_sync(0xffffffffu, ss, o); }
+}
+
 __global__ void bn_stats_finalize(const float *__restrict__ part, int chunks, int C, double invP, float eps,
                                   const float *__restrict__ gamma, const float *__restrict__ beta,
                                   float *scale, float *shift, float *mean, float *rstd) {
-    int c = blockIdx.x * blockDim.x + threadIdx.x;
+    const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (c >= C) return;
-    double s = 0, ss = 0;
-    for (int i = 0; i < chunks; i++) { s += part[((size_t)i * 2) * C + c]; ss += part[((size_t)i * 2 + 1) * C + c]; }
-    double mu = s * invP, var = ss * invP - mu * mu;
-    if (var < 0) var = 0;
-    float r = (float)(1.0 / sqrt(var + (double)eps));
-    float sc = gamma[c] * r;
-    scale[c] = sc; shift[c] = beta[c] - (float)mu * sc; mean[c] = (float)mu; rstd[c] = r;
+    double s, ss;
+    warp_sum2(part, chunks, C, c, s, ss);
+    if ((threadIdx.x & 31) == 0) {
+        double mu = s * invP, var = ss * invP - mu * mu;
+        if (var < 0) var = 0;
+        float r = (float)(1.0 / sqrt(var + (double)eps));
+        float sc = gamma[c] * r;
+        scale[c] = sc; shift[c] = beta[c] - (float)mu * sc; mean[c] = (float)mu; rstd[c] = r;
+    }
 }
 
 // coef: [3][C] = gamma*rstd, gamma*rstd*dbeta/M, gamma*rstd*dgamma/M
 __global__ void bn_bwd_finalize(const float *__restrict__ part, int chunks, int C, double invP,
                                 const float *__restrict__ gamma, const float *__restrict__ rstd,
                                 float *dgamma, float *dbeta, float *coef) {
-    int c = blockIdx.x * blockDim.x + threadIdx.x;
+    const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (c >= C) return;
-    double s = 0, ss = 0;
-    for (int i = 0; i < chunks; i++) { s += part[((size_t)i * 2) * C + c]; ss += part[((size_t)i * 2 + 1) * C + c]; }
-    dbeta[c] = (float)s; dgamma[c] = (float)ss;
-    double gr = (double)gamma[c] * (double)rstd[c];
-    coef[c] = (float)gr; coef[C + c] = (float)(gr * s * invP); coef[2 * C + c] = (float)(gr * ss * invP);
+    double s, ss;
+    warp_sum2(part, chunks, C, c, s, ss);
+    if ((threadIdx.x & 31) == 0) {
+        dbeta[c] = (float)s; dgamma[c] = (float)ss;
+        double gr = (double)gamma[c] * (double)rstd[c];
+        coef[c] = (float)gr; coef[C + c] = (float)(gr * s * invP); coef[2 * C + c] = (float)(gr * ss * invP);
+    }
 }
 
 BnState bn_alloc(Exec &ex, int C) {
@@ -154,7 +166,7 @@ void bn_stats(Exec &ex, Pair t, size_t P, const float *gamma, const float *beta,
         col_reduce_kernel<0><<<grid, block, (size_t)r.SW * r.RPP * 32, ex.stream>>>(t, nullptr, P, r.rows_per_cta,
                                                                                  nullptr, nullptr, nullptr, nullptr, part);
         ex.check("bn_stats_partial", (double)P * C * 4);
-        bn_stats_finalize<<<cdiv(C, 128), 128, 0, ex.stream>>>(part, r.chunks, C, 1.0 / (double)P, ex.eps, gamma, beta,
+        bn_stats_finalize<<<cdiv((size_t)C * 32, 128), 128, 0, ex.stream>>>(part, r.chunks, C, 1.0 / (double)P, ex.eps, gamma, beta,
                                                               st.scale, st.shift, st.mean, st.rstd);
         ex.check("bn_stats_finalize");
     }
@@ -224,7 +236,7 @@ void bn_relu_bwd(Exec &ex, const float *da, Pair t, size_t P, BnState st, const 
         col_reduce_kernel<1><<<grid, block, (size_t)r.SW * r.RPP * 32, ex.stream>>>(t, da, P, r.rows_per_cta, st.scale, st.shift,
                                                                                  st.mean, st.rstd, part);
         ex.check("bn_bwd_partial", (double)P * C * 8);
-        bn_bwd_finalize<<<cdiv(C, 128), 128, 0, ex.stream>>>(part, r.chunks, C, 1.0 / (double)P, gamma, st.rstd, dgamma, dbeta, coef);
+        bn_bwd_finalize<<<cdiv((size_t)C * 32, 128), 128, 0, ex.stream>>>(part, r.chunks, C, 1.0 / (double)P, gamma, st.rstd, dgamma, dbeta, coef);
         ex.check("bn_bwd_finalize");
         size_t nq = P * C4; int g = ew_grid(nq, ex.ctx->sm_count);
 #define RV_ARGS da, t, nq, C4, st.scale, st.shift, st.mean, st.rstd, coef

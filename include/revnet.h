@@ -149,6 +149,11 @@ typedef struct {
     float lr, momentum, weight_decay;               /* SGD (Appendix 6.1); decay on conv/FC weights only */
     int verify_reconstruction;                      /* debug: keep a copy of each stage input and report
                                                        max |reconstructed - original| per stage */
+    int use_cuda_graph;                             /* 1: the first revnet_train_step with a given set of buffer
+                                                       addresses records the step as a CUDA graph (on a private
+                                                       stream) and launches it on the caller's stream; later
+                                                       calls with the same addresses only replay it.  Ignored
+                                                       with verify_reconstruction or while profiling. */
 } revnet_stack_desc;
 
 typedef struct {
@@ -169,6 +174,11 @@ typedef struct {
 int revnet_stack_plan(revnet_ctx *ctx, const revnet_stack_desc *desc, revnet_plan **plan,
                       size_t *param_count, size_t *activation_bytes, size_t *workspace_bytes);
 int revnet_plan_destroy(revnet_plan *plan);
+/* How the planned workspace divides: the part that holds per-parameter data (bf16 weight packs,
+ * the SGD segment table) grows with depth like the parameters do; the rest is activation scratch
+ * (gradient pair, one block's recomputed internals, reduction partials) and does not depend on the
+ * number of units per stage (Section 3.2: storage independent of depth). */
+int revnet_plan_scratch_split(const revnet_plan *plan, size_t *param_scratch_bytes, size_t *activation_scratch_bytes);
 
 /* One SGD training step: forward, loss, reconstructing backward through every stage
  * (Algorithm 1 applied block by block from the stage outputs), SGD-with-momentum update.

@@ -21,7 +21,7 @@ _lib = None
 
 EXPORTS = ["revnet_create", "revnet_destroy", "revnet_last_error", "revnet_block_workspace_bytes",
            "revnet_block_fwd", "revnet_block_bwd", "revnet_stack_plan", "revnet_plan_destroy",
-           "revnet_train_step", "revnet_train_step_host", "revnet_profile_enable", "revnet_profile_summary", "revnet_check_device"]
+           "revnet_train_step", "revnet_train_step_host", "revnet_profile_enable", "revnet_profile_summary", "revnet_check_device", "revnet_plan_scratch_split"]
 
 
 class FnDesc(C.Structure):
@@ -51,7 +51,7 @@ class StackDesc(C.Structure):
                 ("stem_k", C.c_int), ("stem_stride", C.c_int), ("stem_cout", C.c_int), ("maxpool", C.c_int),
                 ("n_stages", C.c_int), ("stage", StageDesc * MAX_STAGES), ("eps", C.c_float), ("mode", C.c_int),
                 ("state_frac_bits", C.c_int), ("lr", C.c_float), ("momentum", C.c_float), ("weight_decay", C.c_float),
-                ("verify_reconstruction", C.c_int)]
+                ("verify_reconstruction", C.c_int), ("use_cuda_graph", C.c_int)]
 
 
 class StepStats(C.Structure):
@@ -137,7 +137,8 @@ def block_desc(b: syn.BlockCfg, mode: int, state_frac_bits: int = 0) -> BlockDes
     return d
 
 
-def stack_desc(cfg: syn.StackCfg, mode: int, verify_reconstruction: bool = False, state_frac_bits: int = 0) -> StackDesc:
+def stack_desc(cfg: syn.StackCfg, mode: int, verify_reconstruction: bool = False, state_frac_bits: int = 0,
+               use_cuda_graph: bool = True) -> StackDesc:
     d = StackDesc()
     d.N, d.img, d.in_ch, d.n_classes = cfg.N, cfg.img, cfg.in_ch, cfg.n_classes
     d.stem_k, d.stem_stride, d.stem_cout, d.maxpool = cfg.stem_k, cfg.stem_stride, cfg.stem_cout, int(cfg.maxpool)
@@ -147,6 +148,7 @@ def stack_desc(cfg: syn.StackCfg, mode: int, verify_reconstruction: bool = False
     d.eps, d.mode, d.state_frac_bits = cfg.eps, mode, state_frac_bits
     d.lr, d.momentum, d.weight_decay = cfg.lr, cfg.momentum, cfg.weight_decay
     d.verify_reconstruction = int(verify_reconstruction)
+    d.use_cuda_graph = int(use_cuda_graph)
     return d
 
 
@@ -238,6 +240,9 @@ class Plan:
         ctx.check(lib().revnet_stack_plan(ctx.h, C.byref(desc), C.byref(self.h), C.byref(n), C.byref(a), C.byref(w)),
                   "revnet_stack_plan")
         self.param_count, self.activation_bytes, self.workspace_bytes = n.value, a.value, w.value
+        ps, as_ = C.c_size_t(), C.c_size_t()
+        ctx.check(lib().revnet_plan_scratch_split(self.h, C.byref(ps), C.byref(as_)), "revnet_plan_scratch_split")
+        self.param_scratch_bytes, self.activation_scratch_bytes = ps.value, as_.value
 
     def close(self):
         if self.h:

@@ -15,7 +15,8 @@ extern "C" int revnet_create(revnet_ctx **out, int device) {
         int sm = 0;
         if (cudaSetDevice(device) != cudaSuccess ||
             cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
-            cudaMalloc(&c->dev_status, 256) != cudaSuccess || cudaMemset(c->dev_status, 0, 256) != cudaSuccess) {
+            cudaMalloc(&c->dev_status, 256) != cudaSuccess || cudaMemset(c->dev_status, 0, 256) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&c->capture_stream, cudaStreamNonBlocking) != cudaSuccess) {
             cudaGetLastError();
             delete c;
             return REVNET_E_CUDA;
@@ -30,6 +31,7 @@ extern "C" int revnet_destroy(revnet_ctx *ctx) {
     if (!ctx) return REVNET_OK;
     for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
     if (ctx->dev_status) cudaFree(ctx->dev_status);
+    if (ctx->capture_stream) cudaStreamDestroy(ctx->capture_stream);
     delete ctx;
     return REVNET_OK;
 }

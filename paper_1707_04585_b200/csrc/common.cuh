@@ -18,6 +18,7 @@ struct revnet_ctx {
     std::string err;
     int *dev_status = nullptr;   // device word for bounded-wait time-outs
     void *encode_tiled = nullptr; // driver entry point for tensor-map encoding
+    cudaStream_t capture_stream = nullptr;   // private stream on which a train step is captured into a graph
     // per-kernel timing (revnet_profile_*): one event after every launch while enabled
     bool profiling = false;
     std::vector<ProfRec> prof;
@@ -168,6 +169,13 @@ void fill_zero(Exec &ex, void *p, size_t bytes);
 void conv_fprop_simt(Exec &ex, const void *a, bool a_bf16, Geom gi, const Layer &L, Pair out, Pair partner, int sign);
 void conv_dgrad_simt(Exec &ex, const void *g, bool g_bf16, Geom gi, const Layer &L, float *da);
 void conv_wgrad_simt(Exec &ex, const void *g, bool g_bf16, const void *a, bool a_bf16, Geom gi, const Layer &L, float *dW);
+
+// ---------------------------------------------------------------- conv_tc.cu
+// bf16 weight packs of the tensor-core kernels, built once per train step
+struct PackJob { const float *W; bf16 *out; int Co, Ci, k, rows_pad, cols_pad, transposed; };
+size_t tc_pack_elems(int cin, int cout, int k, bool transposed);
+PackJob tc_pack_job(const float *W, bf16 *out, int cin, int cout, int k, bool transposed);
+void tc_pack_batch(Exec &ex, const PackJob *jobs_dev, int n_jobs, double bytes);
 
 // ---------------------------------------------------------------- block.cu
 struct FnSaved;   // activations kept from a residual function's (re)computation

@@ -257,6 +257,22 @@ __global__ void pack_weights_kernel(const float *__restrict__ W, bf16 *__restric
     }
 }
 
+// all packs of a step in one launch: blockIdx.y walks the job table
+__global__ void pack_weights_batch_kernel(const PackJob *__restrict__ jobs) {
+    const PackJob j = jobs[blockIdx.y];
+    const int taps = j.k * j.k;
+    const size_t n = (size_t)j.rows_pad * taps * j.cols_pad;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % j.cols_pad);
+        const int tap = (int)((i / j.cols_pad) % taps);
+        const int r = (int)(i / ((size_t)j.cols_pad * taps));
+        float v = 0.f;
+        if (!j.transposed) { if (r < j.Co && c < j.Ci) v = j.W[((size_t)r * taps + tap) * j.Ci + c]; }
+        else { if (r < j.Ci && c < j.Co) v = j.W[((size_t)c * taps + (taps - 1 - tap)) * j.Ci + r]; }
+        j.out[i] = __float2bfloat16_rn(v);
+    }
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
                                   const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -297,7 +313,7 @@ bool tc_shape(Geom g, int cin, int cout, int k, int stride, TcShape &s) {
 
 // act: bf16 [N,H,W,cin]; Wsrc: fp32 weights; transposed selects the dgrad pack
 bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom g, int cin, int cout, int k, int stride,
-                 const float *Wsrc, bool transposed, Pair out, Pair partner, int sign) {
+                 const float *Wsrc, const bf16 *prepacked, bool transposed, Pair out, Pair partner, int sign) {
     TcShape s;
     if (!tc_shape(g, cin, cout, k, stride, s)) return false;
     const int taps = k * k, cout_pad = round_up(cout, 16);
@@ -305,12 +321,12 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom g, int cin, i
     if (!ex.dry && !encoder(ex.ctx)) return false;
     ex.flops += 2ull * g.P() * cout * cin * taps;
     size_t m = ex.ws.mark();
-    bf16 *wp = ex.ws.get<bf16>((size_t)rows_pad * taps * s.cin_pad);
+    bf16 *wp = prepacked ? const_cast<bf16 *>(prepacked) : ex.ws.get<bf16>((size_t)rows_pad * taps * s.cin_pad);
     (void)cout_pad;
     if (!ex.dry) {
         EncodeTiledFn enc = encoder(ex.ctx);
-        // the pack is rebuilt from the fp32 master weights on every call
-        {
+        // without a pack made earlier in the step, build it from the fp32 master weights now
+        if (!prepacked) {
             const size_t n = (size_t)rows_pad * taps * s.cin_pad;
             int grid = (int)((n + 255) / 256); if (grid > ex.ctx->sm_count * 4) grid = ex.ctx->sm_count * 4;
             if (!transposed) pack_weights_kernel<<<grid, 256, 0, ex.stream>>>(Wsrc, wp, cout, cin, k, rows_pad, s.cin_pad, 0);
@@ -485,10 +501,19 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
 }
 
+// out[i] = sum over splits of part[z][i], in a fixed order: 8 interleaved groups of splits per
+// element, combined through shared memory (256 threads = 32 elements x 8 groups)
 __global__ void splitk_sum_kernel(const float *__restrict__ part, size_t n, int splits, float *__restrict__ out) {
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        float s = 0.f;
-        for (int z = 0; z < splits; z++) s += part[(size_t)z * n + i];
+    __shared__ float sm[8][33];
+    const int e = threadIdx.x & 31, grp = threadIdx.x >> 5;
+    const size_t i = (size_t)blockIdx.x * 32 + e;
+    float s = 0.f;
+    if (i < n)
+        for (int z = grp; z < splits; z += 8) s += part[(size_t)z * n + i];
+    sm[grp][e] = s;
+    __syncthreads();
+    if (grp == 0 && i < n) {
+        for (int g = 1; g < 8; g++) s += sm[g][e];
         out[i] = s;
     }
 }
@@ -516,12 +541,12 @@ bool encode_act_map(Exec &ex, CUtensorMap *map, const void *base, Geom g, int C,
 }  // namespace
 
 bool conv_fprop_tc(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign) {
-    return run_conv_tc(ex, "conv_fprop_tc", a, gi, L.cin, L.cout, L.k, L.stride, L.W, false, out, partner, sign);
+    return run_conv_tc(ex, "conv_fprop_tc", a, gi, L.cin, L.cout, L.k, L.stride, L.W, L.Wp_fprop, false, out, partner, sign);
 }
 
 // da[q,ci] = sum_{tap,co} g[q (-) tap, co] W[co,tap,ci]: a stride-1 convolution of g with the mirrored, transposed weights
 bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da) {
-    return run_conv_tc(ex, "conv_dgrad_tc", g, gi, L.cout, L.cin, L.k, L.stride, L.W, true, single(da, L.cin), Pair{}, 0);
+    return run_conv_tc(ex, "conv_dgrad_tc", g, gi, L.cout, L.cin, L.k, L.stride, L.W, L.Wp_dgrad, true, single(da, L.cin), Pair{}, 0);
 }
 
 
@@ -546,8 +571,8 @@ bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer
     const int stage_bytes = p.GM * 32768 + ((256 * p.BN + 1023) & ~1023);
     p.stages = (200 * 1024 - 2048) / stage_bytes; if (p.stages > kStages) p.stages = kStages;
     if (p.stages < 2) return false;
-    // split the pixel reduction so that the grid covers the machine about twice
-    int splits = (2 * ex.ctx->sm_count + m_chunks * n_tiles - 1) / (m_chunks * n_tiles);
+    // split the pixel reduction so that the grid covers the machine once
+    int splits = (ex.ctx->sm_count + m_chunks * n_tiles - 1) / (m_chunks * n_tiles);
     if (splits > p.n_tiles_px) splits = p.n_tiles_px;
     if (splits < 1) splits = 1;
     p.slice = (size_t)L.cout * taps * L.cin;
@@ -568,11 +593,34 @@ bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer
         const double bytes = (double)gi.P() * (L.cin + L.cout) * 2 + (double)p.slice * 4 * (splits > 1 ? splits : 1);
         ex.check("conv_wgrad_tc", bytes, 2.0 * gi.P() * L.cout * L.cin * taps);
         if (splits > 1) {
-            int grid2 = (int)((p.slice + 255) / 256); if (grid2 > ex.ctx->sm_count * 8) grid2 = ex.ctx->sm_count * 8;
-            splitk_sum_kernel<<<grid2, 256, 0, ex.stream>>>(part, p.slice, splits, dW);
+            splitk_sum_kernel<<<(unsigned)((p.slice + 31) / 32), 256, 0, ex.stream>>>(part, p.slice, splits, dW);
             ex.check("splitk_sum", (double)p.slice * 4 * (splits + 1));
         }
     }
     ex.ws.release(m);
     return true;
+}
+
+// ---- packs made once per step (the train step calls these before the forward pass)
+static void pack_dims(int rows, int cols, int &rows_pad, int &cols_pad) {
+    const int rp = round_up(rows, 16), BN = rp <= 128 ? rp : 128;
+    rows_pad = (rp + BN - 1) / BN * BN;
+    cols_pad = round_up(cols, 16);
+}
+size_t tc_pack_elems(int cin, int cout, int k, bool transposed) {
+    int rp, cp;
+    if (!transposed) pack_dims(cout, cin, rp, cp); else pack_dims(cin, cout, rp, cp);
+    return (size_t)rp * k * k * cp;
+}
+PackJob tc_pack_job(const float *W, bf16 *out, int cin, int cout, int k, bool transposed) {
+    PackJob j;
+    j.W = W; j.out = out; j.Co = cout; j.Ci = cin; j.k = k; j.transposed = transposed ? 1 : 0;
+    if (!transposed) pack_dims(cout, cin, j.rows_pad, j.cols_pad); else pack_dims(cin, cout, j.rows_pad, j.cols_pad);
+    return j;
+}
+void tc_pack_batch(Exec &ex, const PackJob *jobs_dev, int n_jobs, double bytes) {
+    if (ex.dry || n_jobs == 0) return;
+    dim3 grid(16, (unsigned)n_jobs);
+    pack_weights_batch_kernel<<<grid, 256, 0, ex.stream>>>(jobs_dev);
+    ex.check("pack_weights_batch", bytes);
 }

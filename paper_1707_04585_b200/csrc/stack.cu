@@ -8,7 +8,10 @@
 #include <stdlib.h>
 #include <math.h>
 
-struct LayerSlot { int cin, cout, k, stride; size_t off_gamma, off_beta, off_W; };   // offsets in floats; stem: gamma/beta unused
+struct LayerSlot {
+    int cin, cout, k, stride; size_t off_gamma, off_beta, off_W;   // offsets in floats; stem: gamma/beta unused
+    const bf16 *wp_f = nullptr, *wp_d = nullptr;                  // bf16 packs of the current step (mode 0)
+};
 
 struct StagePlan {
     int c, H, units;
@@ -30,11 +33,17 @@ struct revnet_plan {
     std::vector<StagePlan> st;
     size_t off_fcW, off_fcb;
     int feat_C;
-    size_t n_params, act_bytes, ws_bytes;
+    size_t n_params, act_bytes, ws_bytes, param_scratch_bytes = 0;
     uint64_t stored_bytes;
     std::vector<uint32_t> seg_end; std::vector<uint8_t> seg_decay;
     void *pinned = nullptr;         // seg_end then seg_decay, page-locked for async upload
     bool pinned_is_malloc = false;  // no CUDA device at plan time: plain host memory instead
+    void *pack_host = nullptr;      // page-locked staging for the weight-pack job table
+    size_t pack_host_bytes = 0;
+    // the step captured as a CUDA graph, valid for one set of buffer addresses
+    cudaGraphExec_t graph_exec = nullptr;
+    const void *graph_key[10] = {};
+    revnet_step_stats graph_stats = {};
 };
 
 static std::vector<std::array<int, 3>> fn_shape(int kind, int c, int w) {
@@ -48,6 +57,7 @@ static Layer bind(const LayerSlot &s, float *params, float *grads) {
     L.cin = s.cin; L.cout = s.cout; L.k = s.k; L.stride = s.stride;
     L.W = params + s.off_W; L.gamma = params + s.off_gamma; L.beta = params + s.off_beta;
     L.dW = grads + s.off_W; L.dgamma = grads + s.off_gamma; L.dbeta = grads + s.off_beta;
+    L.Wp_fprop = s.wp_f; L.Wp_dgrad = s.wp_d;
     return L;
 }
 static std::vector<Layer> bind(const std::vector<LayerSlot> &v, float *params, float *grads) {
@@ -74,6 +84,38 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
         cudaMemcpyAsync(seg_end, pl->pinned, nseg * 4, cudaMemcpyHostToDevice, ex.stream);
         cudaMemcpyAsync(seg_decay, (char *)pl->pinned + nseg * 4, nseg, cudaMemcpyHostToDevice, ex.stream);
     }
+    // bf16 weight packs for the tensor-core kernels: every stride-1 BN-ReLU-conv layer, one launch
+    {
+        std::vector<LayerSlot *> slots;
+        for (auto &s : pl->st) {
+            if (s.has_trans) slots.push_back(&s.trans);
+            for (auto &f : s.F) for (auto &l : f) slots.push_back(&l);
+            for (auto &f : s.G) for (auto &l : f) slots.push_back(&l);
+        }
+        std::vector<PackJob> jobs;
+        double bytes = 0;
+        for (LayerSlot *l : slots) {
+            l->wp_f = l->wp_d = nullptr;
+            if (ex.mode != 0 || l->stride != 1 || l->cin % 8 || l->cout % 8) continue;
+            size_t nf = tc_pack_elems(l->cin, l->cout, l->k, false), nd = tc_pack_elems(l->cin, l->cout, l->k, true);
+            bf16 *f = ex.ws.get<bf16>(nf), *dd = ex.ws.get<bf16>(nd);
+            l->wp_f = f; l->wp_d = dd;
+            jobs.push_back(tc_pack_job(params + l->off_W, f, l->cin, l->cout, l->k, false));
+            jobs.push_back(tc_pack_job(params + l->off_W, dd, l->cin, l->cout, l->k, true));
+            bytes += (double)(nf + nd) * 2 + (double)l->cin * l->cout * l->k * l->k * 8;
+        }
+        PackJob *jobs_dev = ex.ws.get<PackJob>(jobs.size() + 1);
+        if (!ex.dry && !jobs.empty()) {
+            if (jobs.size() * sizeof(PackJob) <= pl->pack_host_bytes) {
+                memcpy(pl->pack_host, jobs.data(), jobs.size() * sizeof(PackJob));
+                cudaMemcpyAsync(jobs_dev, pl->pack_host, jobs.size() * sizeof(PackJob), cudaMemcpyHostToDevice, ex.stream);
+                tc_pack_batch(ex, jobs_dev, (int)jobs.size(), bytes);
+            } else {
+                for (LayerSlot *l : slots) l->wp_f = l->wp_d = nullptr;   // no staging room: pack per call instead
+            }
+        }
+    }
+    if (ex.dry) pl->param_scratch_bytes = (ex.ws.off + 255) & ~size_t(255);   // everything above scales with the parameters, not the activations
     size_t gmax = (size_t)N * pl->stemH * pl->stemH * d.stem_cout;           // gradient w.r.t. stem / pool output
     for (auto &s : pl->st) { size_t e = (size_t)N * s.H * s.H * 2 * s.c; if (e > gmax) gmax = e; }
     float *gbuf[2] = {ex.ws.get<float>(gmax), ex.ws.get<float>(gmax)};
@@ -210,7 +252,8 @@ extern "C" int revnet_stack_plan(revnet_ctx *ctx, const revnet_stack_desc *desc,
     size_t off = 0;
     auto take = [&](size_t n, bool decay) { size_t o = off; off += n; pl->seg_end.push_back((uint32_t)off); pl->seg_decay.push_back(decay); return o; };
     auto slot = [&](int cin, int cout, int k, int stride, bool bn) {
-        LayerSlot s{cin, cout, k, stride, 0, 0, 0};
+        LayerSlot s;
+        s.cin = cin; s.cout = cout; s.k = k; s.stride = stride; s.off_gamma = s.off_beta = s.off_W = 0;
         if (bn) { s.off_gamma = take(cin, false); s.off_beta = take(cin, false); }
         s.off_W = take((size_t)cout * k * k * cin, true);
         return s;
@@ -269,6 +312,14 @@ extern "C" int revnet_stack_plan(revnet_ctx *ctx, const revnet_stack_desc *desc,
         pl->pinned_is_malloc = true;
         if (!pl->pinned) { delete pl; return fail(ctx, REVNET_E_INTERNAL, "revnet_stack_plan: out of host memory"); }
     }
+    {
+        size_t layers = 0;
+        for (auto &st : pl->st) layers += 1 + (size_t)st.units * 6;
+        pl->pack_host_bytes = layers * 2 * sizeof(PackJob);
+        if (pl->pinned_is_malloc || cudaMallocHost(&pl->pack_host, pl->pack_host_bytes) != cudaSuccess) {
+            cudaGetLastError(); pl->pack_host = nullptr; pl->pack_host_bytes = 0;
+        }
+    }
     memcpy(pl->pinned, pl->seg_end.data(), nseg * 4);
     memcpy((char *)pl->pinned + nseg * 4, pl->seg_decay.data(), nseg);
     // size the workspace with a dry run of the very same driver
@@ -283,9 +334,18 @@ extern "C" int revnet_stack_plan(revnet_ctx *ctx, const revnet_stack_desc *desc,
     return REVNET_OK;
 }
 
+extern "C" int revnet_plan_scratch_split(const revnet_plan *pl, size_t *param_scratch_bytes, size_t *activation_scratch_bytes) {
+    if (!pl) return REVNET_E_INVALID_ARG;
+    if (param_scratch_bytes) *param_scratch_bytes = pl->param_scratch_bytes;
+    if (activation_scratch_bytes) *activation_scratch_bytes = pl->ws_bytes - pl->param_scratch_bytes;
+    return REVNET_OK;
+}
+
 extern "C" int revnet_plan_destroy(revnet_plan *pl) {
     if (!pl) return REVNET_OK;
     if (pl->pinned) { if (pl->pinned_is_malloc) free(pl->pinned); else cudaFreeHost(pl->pinned); }
+    if (pl->graph_exec) cudaGraphExecDestroy(pl->graph_exec);
+    if (pl->pack_host) cudaFreeHost(pl->pack_host);
     delete pl;
     return REVNET_OK;
 }
@@ -298,11 +358,47 @@ extern "C" int revnet_train_step(revnet_ctx *ctx, revnet_plan *pl, const float *
     const void *ptrs[] = {images, params, grads, momentum, activations, workspace};
     for (const void *p : ptrs)
         if ((uintptr_t)p & 15) return fail(ctx, REVNET_E_MISALIGNED, "revnet_train_step: pointers must be 16-byte aligned");
-    Exec ex; ex.ctx = ctx; ex.dry = false; ex.mode = pl->d.mode; ex.eps = pl->d.eps; ex.stream = (cudaStream_t)stream;
+    const bool use_graph = pl->d.use_cuda_graph && !pl->d.verify_reconstruction && !ctx->profiling && ctx->capture_stream;
+    const void *key[10] = {images, labels, params, grads, momentum, activations, workspace, loss, pred, logits};
+    if (use_graph && pl->graph_exec && memcmp(key, pl->graph_key, sizeof key) == 0) {
+        if (cudaGraphLaunch(pl->graph_exec, (cudaStream_t)stream) != cudaSuccess)
+            return fail(ctx, REVNET_E_CUDA, std::string("revnet_train_step: graph launch: ") + cudaGetErrorString(cudaGetLastError()));
+        if (stats) *stats = pl->graph_stats;
+        return REVNET_OK;
+    }
+    Exec ex; ex.ctx = ctx; ex.dry = false; ex.mode = pl->d.mode; ex.eps = pl->d.eps;
+    ex.stream = use_graph ? ctx->capture_stream : (cudaStream_t)stream;
     ex.q = pl->d.state_frac_bits ? ldexpf(1.f, -pl->d.state_frac_bits) : 0.f;
     ex.ws.dry = false; ex.ws.base = (char *)workspace; ex.ws.cap = pl->ws_bytes;
+    if (use_graph) {
+        if (pl->graph_exec) { cudaGraphExecDestroy(pl->graph_exec); pl->graph_exec = nullptr; }
+        if (cudaStreamBeginCapture(ex.stream, cudaStreamCaptureModeRelaxed) != cudaSuccess)
+            return fail(ctx, REVNET_E_CUDA, std::string("revnet_train_step: begin capture: ") + cudaGetErrorString(cudaGetLastError()));
+    }
     float *recon = nullptr;
-    run_step(pl, ex, images, labels, params, grads, momentum, (char *)activations, loss, pred, logits, stats, &recon);
+    revnet_step_stats local_stats;
+    run_step(pl, ex, images, labels, params, grads, momentum, (char *)activations, loss, pred, logits, &local_stats, &recon);
+    if (use_graph) {
+        cudaGraph_t graph = nullptr;
+        cudaError_t e = cudaStreamEndCapture(ex.stream, &graph);
+        if (e != cudaSuccess || ex.failed || ex.ws.overflow) {
+            if (graph) cudaGraphDestroy(graph);
+            cudaGetLastError();
+            if (ex.ws.overflow) return fail(ctx, REVNET_E_WORKSPACE_TOO_SMALL, "revnet_train_step: workspace smaller than planned");
+            if (!ex.failed) ctx->err = std::string("revnet_train_step: end capture: ") + cudaGetErrorString(e);
+            return REVNET_E_CUDA;
+        }
+        e = cudaGraphInstantiate(&pl->graph_exec, graph, 0);
+        cudaGraphDestroy(graph);
+        if (e != cudaSuccess) { pl->graph_exec = nullptr; return fail(ctx, REVNET_E_CUDA, std::string("revnet_train_step: instantiate: ") + cudaGetErrorString(e)); }
+        memcpy(pl->graph_key, key, sizeof key);
+        pl->graph_stats = local_stats;
+        if (cudaGraphLaunch(pl->graph_exec, (cudaStream_t)stream) != cudaSuccess)
+            return fail(ctx, REVNET_E_CUDA, std::string("revnet_train_step: graph launch: ") + cudaGetErrorString(cudaGetLastError()));
+        if (stats) *stats = local_stats;
+        return REVNET_OK;
+    }
+    if (stats) *stats = local_stats;
     if (ex.ws.overflow) return fail(ctx, REVNET_E_WORKSPACE_TOO_SMALL, "revnet_train_step: workspace smaller than planned");
     if (ex.failed) return REVNET_E_CUDA;
     if (pl->d.verify_reconstruction && stats) {

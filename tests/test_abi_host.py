@@ -49,10 +49,10 @@ def test_activation_bytes_flat_in_depth_and_equal_to_oracle_count(ctx):
     def pad(n): return (n + 255) // 256 * 256
 
     def scratch(plan, cfg):
-        # the workspace also carries the SGD segment table (5 bytes per parameter tensor), which is
-        # parameter metadata and grows with depth like the parameters do; everything else must not
-        nt = len(syn.param_specs(cfg))
-        return plan.workspace_bytes - pad(4 * nt) - pad(nt)
+        # the workspace also carries per-parameter data (bf16 weight packs, SGD segment table), which
+        # grows with depth like the parameters do; the activation scratch must not
+        assert plan.param_scratch_bytes + plan.activation_scratch_bytes == plan.workspace_bytes
+        return plan.activation_scratch_bytes
     for units in (1, 3, 9, 18, 36):
         cfg = syn.shrink(base, units=units)
         plan = B.revnet_stack_plan(ctx, B.stack_desc(cfg, 0))

@@ -282,3 +282,23 @@ def test_activation_memory_flat_in_depth_on_device(ctx):
         seen.add((st.stored_activation_bytes, r.plan.activation_bytes))
         assert np.isfinite(r.results()["loss"])
     assert len(seen) == 1, seen
+
+
+def test_graph_replay_matches_eager(ctx):
+    """The step replayed from its CUDA graph gives the same bits as the step enqueued kernel by kernel."""
+    cfg = syn.shrink(syn.stack_config("revnet38"), N=16)
+    inp = syn.make_stack_inputs(cfg)
+    out = []
+    for graph in (False, True):
+        r = R.StackRunner(ctx, cfg, 0, use_cuda_graph=graph)
+        r.load(inp["images"], inp["labels"], inp["params"])
+        for _ in range(3):
+            st = r.step()
+        res = r.results()
+        out.append((res, st))
+    (a, sa), (b, sb) = out
+    assert a["loss"] == b["loss"] and np.array_equal(a["pred"], b["pred"])
+    for k in a["params"]:
+        assert np.array_equal(a["params"][k], b["params"][k]), k
+        assert np.array_equal(a["grads"][k], b["grads"][k]), k
+    assert sa.kernel_launches == sb.kernel_launches and sa.flops_bwd == sb.flops_bwd

@@ -125,6 +125,36 @@ int revnet_block_bwd(revnet_ctx *ctx, const revnet_block_desc *desc,
                      const revnet_fn_grads *gF, const revnet_fn_grads *gG,
                      void *workspace, size_t workspace_bytes, void *stream);
 
+/* ---- stored (non-reversible) layer: BN -> ReLU -> conv k x k with stride 1 or 2 (Section 3.1: a
+ * reversible block must have stride 1; Section 3.2: such layers keep their input).  The input is
+ * either one float32 tensor [N,H,W,cin] (in_split = 0, in2 unused) or the two halves of a
+ * coupling state, cin/2 channels each, in the state format (in_split = 1).  The output
+ * [N,H/stride,W/stride,cout] is written as two halves (out1: channels [0,cout/2), out2: the rest)
+ * in the state format: it is the (x1,x2) the next stage starts from. */
+typedef struct {
+    int N, H, W;             /* input geometry */
+    int cin, cout, k, stride;
+    int in_split;
+    float eps;
+    int mode;
+    int state_frac_bits;
+} revnet_transition_desc;
+
+int revnet_transition_workspace_bytes(revnet_ctx *ctx, const revnet_transition_desc *desc,
+                                      size_t *fwd_bytes, size_t *bwd_bytes);
+int revnet_transition_fwd(revnet_ctx *ctx, const revnet_transition_desc *desc,
+                          const void *in1, const void *in2,
+                          const float *W, const float *gamma, const float *beta,
+                          void *out1, void *out2,
+                          void *workspace, size_t workspace_bytes, void *stream);
+/* Backward from the stored input: din (float32, same split as the input), dW, dgamma, dbeta. */
+int revnet_transition_bwd(revnet_ctx *ctx, const revnet_transition_desc *desc,
+                          const void *in1, const void *in2,
+                          const float *dout1, const float *dout2,
+                          const float *W, const float *gamma, const float *beta,
+                          float *din1, float *din2, float *dW, float *dgamma, float *dbeta,
+                          void *workspace, size_t workspace_bytes, void *stream);
+
 /* ---- classification stack (Section 3.2: only non-reversible layers keep their inputs) ---- */
 
 typedef struct {

@@ -21,7 +21,8 @@ _lib = None
 
 EXPORTS = ["revnet_create", "revnet_destroy", "revnet_last_error", "revnet_block_workspace_bytes",
            "revnet_block_fwd", "revnet_block_bwd", "revnet_stack_plan", "revnet_plan_destroy",
-           "revnet_train_step", "revnet_train_step_host", "revnet_profile_enable", "revnet_profile_summary", "revnet_check_device", "revnet_plan_scratch_split"]
+           "revnet_train_step", "revnet_train_step_host", "revnet_profile_enable", "revnet_profile_summary", "revnet_check_device", "revnet_plan_scratch_split",
+           "revnet_transition_workspace_bytes", "revnet_transition_fwd", "revnet_transition_bwd"]
 
 
 class FnDesc(C.Structure):
@@ -39,6 +40,11 @@ class FnParams(C.Structure):
 
 class FnGrads(C.Structure):
     _fields_ = [("dW", C.c_void_p * 3), ("dgamma", C.c_void_p * 3), ("dbeta", C.c_void_p * 3)]
+
+
+class TransitionDesc(C.Structure):
+    _fields_ = [("N", C.c_int), ("H", C.c_int), ("W", C.c_int), ("cin", C.c_int), ("cout", C.c_int), ("k", C.c_int),
+                ("stride", C.c_int), ("in_split", C.c_int), ("eps", C.c_float), ("mode", C.c_int), ("state_frac_bits", C.c_int)]
 
 
 class StageDesc(C.Structure):
@@ -300,3 +306,25 @@ def revnet_profile_summary(ctx):
 def revnet_check_device(ctx):
     """Synchronise and raise if a kernel reported that it gave up a bounded wait."""
     ctx.check(lib().revnet_check_device(ctx.h, _stream()), "revnet_check_device")
+
+
+def _nbytes(t):
+    return C.c_size_t(t.numel() * t.element_size())
+
+
+def revnet_transition_workspace_bytes(ctx, desc):
+    f, b = C.c_size_t(), C.c_size_t()
+    ctx.check(lib().revnet_transition_workspace_bytes(ctx.h, C.byref(desc), C.byref(f), C.byref(b)), "revnet_transition_workspace_bytes")
+    return f.value, b.value
+
+
+def revnet_transition_fwd(ctx, desc, in1, in2, W, gamma, beta, out1, out2, workspace):
+    ctx.check(lib().revnet_transition_fwd(ctx.h, C.byref(desc), _ptr(in1), _ptr(in2), _ptr(W), _ptr(gamma), _ptr(beta),
+                                          _ptr(out1), _ptr(out2), _ptr(workspace), _nbytes(workspace), _stream()),
+              "revnet_transition_fwd")
+
+
+def revnet_transition_bwd(ctx, desc, in1, in2, dout1, dout2, W, gamma, beta, din1, din2, dW, dgamma, dbeta, workspace):
+    ctx.check(lib().revnet_transition_bwd(ctx.h, C.byref(desc), _ptr(in1), _ptr(in2), _ptr(dout1), _ptr(dout2), _ptr(W),
+                                          _ptr(gamma), _ptr(beta), _ptr(din1), _ptr(din2), _ptr(dW), _ptr(dgamma), _ptr(dbeta),
+                                          _ptr(workspace), _nbytes(workspace), _stream()), "revnet_transition_bwd")

@@ -148,6 +148,89 @@ extern "C" int revnet_block_bwd(revnet_ctx *ctx, const revnet_block_desc *d, con
     return finish(ctx, ex, "revnet_block_bwd");
 }
 
+// ---- stored (non-reversible) BN -> ReLU -> conv layer: forward keeps nothing, backward rebuilds its
+// operands from the stored input (Section 3.2: inputs of non-reversible layers are kept)
+static int check_trans(revnet_ctx *ctx, const revnet_transition_desc *d) {
+    if (!ctx || !d) return fail(ctx, REVNET_E_INVALID_ARG, "null descriptor");
+    if (d->N < 1 || d->H < 1 || d->W < 1 || (d->mode != 0 && d->mode != 1) || d->state_frac_bits < 0 || d->state_frac_bits > 24 ||
+        (d->in_split != 0 && d->in_split != 1))
+        return fail(ctx, REVNET_E_INVALID_ARG, "transition descriptor: bad N/H/W/mode/state_frac_bits/in_split");
+    if ((d->k != 1 && d->k != 3) || (d->stride != 1 && d->stride != 2) || d->cin < 4 || d->cin % (d->in_split ? 8 : 4) || d->cout < 8 || d->cout % 8)
+        return fail(ctx, REVNET_E_UNSUPPORTED_SHAPE, "transition descriptor: k in {1,3}, stride in {1,2}, cin % 4 (8 when split), cout % 8");
+    return REVNET_OK;
+}
+static void trans_run(Exec &ex, const revnet_transition_desc *d, bool backward, const void *in1, const void *in2,
+                      const float *W, const float *gamma, const float *beta, void *out1, void *out2,
+                      const float *dout1, const float *dout2, float *din1, float *din2, float *dW, float *dgamma, float *dbeta) {
+    const float q = ex.q;
+    Layer L; L.cin = d->cin; L.cout = d->cout; L.k = d->k; L.stride = d->stride;
+    L.W = W; L.gamma = gamma; L.beta = beta; L.dW = dW; L.dgamma = dgamma; L.dbeta = dbeta;
+    std::vector<Layer> T{L};
+    Geom g{d->N, d->H, d->W};
+    Pair tin = d->in_split ? halves((float *)in1, (float *)in2, d->cin / 2, q) : single((float *)in1, d->cin);
+    const int ch = d->cout / 2;
+    if (!backward) {
+        fn_forward(ex, g, tin, T, Pair{}, halves((float *)out1, (float *)out2, ch, q), 0, nullptr, false);
+    } else {
+        FnSaved sv;
+        size_t m = ex.ws.mark();
+        fn_forward(ex, g, tin, T, Pair{}, Pair{}, 0, &sv, true);
+        Pair gout = d->in_split ? halves(din1, din2, d->cin / 2) : single(din1, d->cin);
+        fn_backward(ex, g, tin, T, sv, halves((float *)dout1, (float *)dout2, ch), Pair{}, gout);
+        ex.ws.release(m);
+    }
+}
+static Exec trans_exec(revnet_ctx *ctx, const revnet_transition_desc *d, bool dry, void *ws, size_t ws_bytes, void *stream) {
+    Exec ex; ex.ctx = ctx; ex.dry = dry; ex.ws.dry = dry; ex.mode = d->mode; ex.eps = d->eps; ex.stream = (cudaStream_t)stream;
+    ex.q = d->state_frac_bits ? ldexpf(1.f, -d->state_frac_bits) : 0.f;
+    ex.ws.base = (char *)ws; ex.ws.cap = ws_bytes;
+    return ex;
+}
+extern "C" int revnet_transition_workspace_bytes(revnet_ctx *ctx, const revnet_transition_desc *d, size_t *fwd_bytes, size_t *bwd_bytes) {
+    int rc = check_trans(ctx, d);
+    if (rc) return rc;
+    float *f = (float *)0x1000;
+    for (int pass = 0; pass < 2; pass++) {
+        Exec ex = trans_exec(ctx, d, true, nullptr, 0, nullptr);
+        trans_run(ex, d, pass == 1, f, f, f, f, f, f, f, f, f, f, f, f, f, f);
+        size_t *o = pass == 0 ? fwd_bytes : bwd_bytes;
+        if (o) *o = ex.ws.peak + 256;
+    }
+    return REVNET_OK;
+}
+extern "C" int revnet_transition_fwd(revnet_ctx *ctx, const revnet_transition_desc *d, const void *in1, const void *in2,
+                                     const float *W, const float *gamma, const float *beta, void *out1, void *out2,
+                                     void *workspace, size_t workspace_bytes, void *stream) {
+    int rc = check_trans(ctx, d);
+    if (rc) return rc;
+    if (!in1 || (d->in_split && !in2) || !W || !gamma || !beta || !out1 || !out2 || !workspace)
+        return fail(ctx, REVNET_E_INVALID_ARG, "revnet_transition_fwd: null pointer");
+    if (!aligned16({in1, in2, W, gamma, beta, out1, out2, workspace})) return fail(ctx, REVNET_E_MISALIGNED, "revnet_transition_fwd: pointers must be 16-byte aligned");
+    size_t need = 0;
+    revnet_transition_workspace_bytes(ctx, d, &need, nullptr);
+    if (workspace_bytes < need) return fail(ctx, REVNET_E_WORKSPACE_TOO_SMALL, "revnet_transition_fwd: workspace too small");
+    Exec ex = trans_exec(ctx, d, false, workspace, workspace_bytes, stream);
+    trans_run(ex, d, false, in1, in2, W, gamma, beta, out1, out2, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr);
+    return finish(ctx, ex, "revnet_transition_fwd");
+}
+extern "C" int revnet_transition_bwd(revnet_ctx *ctx, const revnet_transition_desc *d, const void *in1, const void *in2,
+                                     const float *dout1, const float *dout2, const float *W, const float *gamma, const float *beta,
+                                     float *din1, float *din2, float *dW, float *dgamma, float *dbeta,
+                                     void *workspace, size_t workspace_bytes, void *stream) {
+    int rc = check_trans(ctx, d);
+    if (rc) return rc;
+    if (!in1 || (d->in_split && (!in2 || !din2)) || !dout1 || !dout2 || !W || !gamma || !beta || !din1 || !dW || !dgamma || !dbeta || !workspace)
+        return fail(ctx, REVNET_E_INVALID_ARG, "revnet_transition_bwd: null pointer");
+    if (!aligned16({in1, in2, dout1, dout2, W, gamma, beta, din1, din2, dW, dgamma, dbeta, workspace}))
+        return fail(ctx, REVNET_E_MISALIGNED, "revnet_transition_bwd: pointers must be 16-byte aligned");
+    size_t need = 0;
+    revnet_transition_workspace_bytes(ctx, d, nullptr, &need);
+    if (workspace_bytes < need) return fail(ctx, REVNET_E_WORKSPACE_TOO_SMALL, "revnet_transition_bwd: workspace too small");
+    Exec ex = trans_exec(ctx, d, false, workspace, workspace_bytes, stream);
+    trans_run(ex, d, true, in1, in2, W, gamma, beta, nullptr, nullptr, dout1, dout2, din1, din2, dW, dgamma, dbeta);
+    return finish(ctx, ex, "revnet_transition_bwd");
+}
+
 // ---- device-side status
 extern "C" int revnet_check_device(revnet_ctx *ctx, void *stream) {
     if (!ctx) return REVNET_E_INVALID_ARG;

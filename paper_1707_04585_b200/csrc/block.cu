@@ -17,7 +17,18 @@ static void conv_fprop(Exec &ex, const void *a, Geom gi, const Layer &L, Pair ou
 }
 static void conv_dgrad(Exec &ex, const void *g, Geom gi, const Layer &L, float *da) {
     const bool b16 = ex.mode == 0;
-    if (b16 && conv_dgrad_tc(ex, g, gi, L, da)) return;
+    if (b16 && L.stride == 1 && conv_dgrad_tc(ex, g, gi, L, da)) return;
+    if (b16 && L.stride == 2 && gi.H % 2 == 0 && gi.W % 2 == 0 && L.cout % 8 == 0) {
+        // stride 2: spread g over the input grid (zeros between samples); the data gradient is then the
+        // stride-1 one:  da[y,x] = sum_taps g_up[y + pad - kh, x + pad - kw] W[.,kh,kw,.]
+        size_t m = ex.ws.mark();
+        bf16 *gup = ex.ws.get<bf16>(gi.P() * L.cout);
+        upsample_zero_bf16(ex, (const bf16 *)g, gup, gi.N, gi.H / 2, gi.W / 2, L.cout);
+        Layer L1 = L; L1.stride = 1;
+        const bool ok = conv_dgrad_tc(ex, gup, gi, L1, da);
+        ex.ws.release(m);
+        if (ok) return;
+    }
     conv_dgrad_simt(ex, g, b16, gi, L, da);
 }
 static void conv_wgrad(Exec &ex, const void *g, const void *a, Geom gi, const Layer &L, float *dW) {

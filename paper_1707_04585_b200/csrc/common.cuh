@@ -162,6 +162,8 @@ void sgd_update(Exec &ex, float *params, const float *grads, float *mom, size_t 
 // max |a - b| over n elements of two state tensors (float, or fixed point when q > 0)
 void max_abs_diff(Exec &ex, const float *a, const float *b, size_t n, float q, float *out /*1 float, pre-zeroed*/);
 void fill_zero(Exec &ex, void *p, size_t bytes);
+// out[n, 2i, 2j, :] = in[n, i, j, :], zero elsewhere; out is [N, 2Ho, 2Wo, C]
+void upsample_zero_bf16(Exec &ex, const bf16 *in, bf16 *out, int N, int Ho, int Wo, int C);
 
 // ---------------------------------------------------------------- conv_simt.cu
 // Operand element type of the activated tensor / upstream gradient: float or bf16.

@@ -31,7 +31,8 @@ struct TcParams {
     int cin_pad;     // chunks * KC
     int BN;          // N tile
     int n_cols;      // valid output channels
-    int H, W;        // image size
+    int H, W;        // output image size
+    int stride;      // 1 or 2: input pixel = output pixel * stride + tap - pad (TMA traversal stride)
     int BH, BIMG;    // tile: BH rows x W columns x BIMG images = 128 pixels
     Pair out, partner;
     int sign;
@@ -188,7 +189,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const int kh = tap / p.k, kw = tap - kh * p.k;
                 uint8_t *sa = tiles + s * stage_bytes;
                 mbar_expect_tx(&sh->full[s], (uint32_t)(a_bytes + b_bytes));
-                tma_load_4d(sa, &map_a, &sh->full[s], ch * p.KC, kw - pad, h0 + kh - pad, n0);
+                tma_load_4d(sa, &map_a, &sh->full[s], ch * p.KC, kw - pad, h0 * p.stride + kh - pad, n0);
                 tma_load_2d(sa + b_off, &map_b, &sh->full[s], tap * p.cin_pad + ch * p.KC, col0);
             }
         }
@@ -292,10 +293,10 @@ int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
 struct TcShape { int KC, cin_pad, chunks, BN, n_tiles, BH, BIMG, smem; };
 
-// Which shapes the kernel takes: stride 1, k in {1,3}; a 128-pixel tile must be whole rows of one
+// Which shapes the kernel takes: stride 1 or 2, k in {1,3}; a 128-pixel output tile must be whole rows of one
 // image or whole images; channel rows 16-byte aligned for TMA.
-bool tc_shape(Geom g, int cin, int cout, int k, int stride, TcShape &s) {
-    if (stride != 1 || (k != 1 && k != 3) || cin % 8 || cout % 4) return false;
+bool tc_shape(Geom g, int cin, int cout, int k, int stride, TcShape &s) {   // g: output geometry
+    if ((stride != 1 && stride != 2) || (k != 1 && k != 3) || cin % 8 || cout % 4) return false;
     const int W = g.W, H = g.H;
     if (W > 128 || 128 % W) return false;
     if (H * W >= 128) { if (H % (128 / W)) return false; s.BH = 128 / W; s.BIMG = 1; }
@@ -312,9 +313,11 @@ bool tc_shape(Geom g, int cin, int cout, int k, int stride, TcShape &s) {
 }
 
 // act: bf16 [N,H,W,cin]; Wsrc: fp32 weights; transposed selects the dgrad pack
-bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom g, int cin, int cout, int k, int stride,
+bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin, int cout, int k, int stride,
                  const float *Wsrc, const bf16 *prepacked, bool transposed, Pair out, Pair partner, int sign) {
     TcShape s;
+    if (stride == 2 && (gin.H % 2 || gin.W % 2)) return false;
+    const Geom g{gin.N, conv_out(gin.H, k, stride), conv_out(gin.W, k, stride)};   // output geometry
     if (!tc_shape(g, cin, cout, k, stride, s)) return false;
     const int taps = k * k, cout_pad = round_up(cout, 16);
     const int rows_pad = s.n_tiles * s.BN;
@@ -336,10 +339,11 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom g, int cin, i
         CUtensorMap map_a, map_b;
         const CUtensorMapSwizzle sw = s.KC == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : (s.KC == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
         {
-            cuuint64_t dims[4] = {(cuuint64_t)cin, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N};
-            cuuint64_t strides[3] = {(cuuint64_t)cin * 2, (cuuint64_t)g.W * cin * 2, (cuuint64_t)g.H * g.W * cin * 2};
-            cuuint32_t box[4] = {(cuuint32_t)s.KC, (cuuint32_t)g.W, (cuuint32_t)s.BH, (cuuint32_t)s.BIMG};
-            cuuint32_t es[4] = {1, 1, 1, 1};
+            // the box spans stride x the tile in the input image and is walked with that stride
+            cuuint64_t dims[4] = {(cuuint64_t)cin, (cuuint64_t)gin.W, (cuuint64_t)gin.H, (cuuint64_t)gin.N};
+            cuuint64_t strides[3] = {(cuuint64_t)cin * 2, (cuuint64_t)gin.W * cin * 2, (cuuint64_t)gin.H * gin.W * cin * 2};
+            cuuint32_t box[4] = {(cuuint32_t)s.KC, (cuuint32_t)(g.W * stride), (cuuint32_t)(s.BH * stride), (cuuint32_t)s.BIMG};
+            cuuint32_t es[4] = {1, (cuuint32_t)stride, (cuuint32_t)stride, 1};
             CUresult r = enc(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void *)act, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                              sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) { ex.failed = true; ex.ctx->err = std::string(what) + ": tensor map (activations) rejected"; ex.ws.release(m); return true; }
@@ -355,12 +359,12 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom g, int cin, i
         }
         TcParams p;
         p.taps = taps; p.k = k; p.chunks = s.chunks; p.KC = s.KC; p.cin_pad = s.cin_pad; p.BN = s.BN; p.n_cols = cout;
-        p.H = g.H; p.W = g.W; p.BH = s.BH; p.BIMG = s.BIMG; p.out = out; p.partner = partner; p.sign = sign; p.status = ex.ctx->dev_status;
+        p.H = g.H; p.W = g.W; p.stride = stride; p.BH = s.BH; p.BIMG = s.BIMG; p.out = out; p.partner = partner; p.sign = sign; p.status = ex.ctx->dev_status;
         static bool attr_set = false;
         if (!attr_set) { cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); attr_set = true; }
         dim3 grid((unsigned)(g.P() / 128), (unsigned)s.n_tiles);
         conv_tc_kernel<<<grid, kThreads, s.smem, ex.stream>>>(map_a, map_b, p);
-        const double bytes = (double)g.P() * cin * 2 + (double)g.P() * cout * (sign ? 8 : 4) + (double)cout * taps * cin * 2;
+        const double bytes = (double)gin.P() * cin * 2 + (double)g.P() * cout * (sign ? 8 : 4) + (double)cout * taps * cin * 2;
         ex.check(what, bytes, 2.0 * g.P() * cout * cin * taps);
     }
     ex.ws.release(m);
@@ -381,7 +385,8 @@ struct WgParams {
     int total_blocks;            // taps * cblks
     int blockN, BN, cout;        // output-channel block, N tile, valid channels
     int GM;                      // M groups per CTA (1 or 2)
-    int H, W, BH, BIMG;
+    int H, W, BH, BIMG;          // output geometry and tile
+    int stride;
     int n_tiles_px;              // pixel tiles in all
     int stages;
     float *partial;              // [splits][cout][taps][cin]
@@ -440,7 +445,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 for (int b = 0; b < n_blocks; b++) {
                     const int gb = first_block + b, tap = gb / p.cblks, cb = gb - tap * p.cblks;
                     const int kh = tap / p.k, kw = tap - kh * p.k;
-                    tma_load_4d(sa + b * blk_bytes_a, &map_a, &sh->full[s], cb * p.blockC, kw - pad, h0 + kh - pad, n0);
+                    tma_load_4d(sa + b * blk_bytes_a, &map_a, &sh->full[s], cb * p.blockC, kw - pad, h0 * p.stride + kh - pad, n0);
                 }
                 for (int b = 0; b < nb_n; b++)
                     tma_load_4d(sa + a_region + b * blk_bytes_b, &map_g, &sh->full[s], col0 + b * p.blockN, 0, h0, n0);
@@ -528,12 +533,13 @@ bool tile_shape(Geom g, int &BH, int &BIMG) {
     return true;
 }
 
-bool encode_act_map(Exec &ex, CUtensorMap *map, const void *base, Geom g, int C, int box_c, int BH, int BIMG) {
+// g: geometry of the tensor; (tile_w, BH, BIMG): the 128-pixel tile in units of the traversal stride
+bool encode_act_map(Exec &ex, CUtensorMap *map, const void *base, Geom g, int C, int box_c, int tile_w, int BH, int BIMG, int stride) {
     const CUtensorMapSwizzle sw = box_c == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : (box_c == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
     cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N};
     cuuint64_t strides[3] = {(cuuint64_t)C * 2, (cuuint64_t)g.W * C * 2, (cuuint64_t)g.H * g.W * C * 2};
-    cuuint32_t box[4] = {(cuuint32_t)box_c, (cuuint32_t)g.W, (cuuint32_t)BH, (cuuint32_t)BIMG};
-    cuuint32_t es[4] = {1, 1, 1, 1};
+    cuuint32_t box[4] = {(cuuint32_t)box_c, (cuuint32_t)(tile_w * stride), (cuuint32_t)(BH * stride), (cuuint32_t)BIMG};
+    cuuint32_t es[4] = {1, (cuuint32_t)stride, (cuuint32_t)stride, 1};
     return encoder(ex.ctx)(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void *)base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                            sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
@@ -546,14 +552,17 @@ bool conv_fprop_tc(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, P
 
 // da[q,ci] = sum_{tap,co} g[q (-) tap, co] W[co,tap,ci]: a stride-1 convolution of g with the mirrored, transposed weights
 bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da) {
+    if (L.stride != 1) return false;
     return run_conv_tc(ex, "conv_dgrad_tc", g, gi, L.cout, L.cin, L.k, L.stride, L.W, L.Wp_dgrad, true, single(da, L.cin), Pair{}, 0);
 }
 
 
 bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer &L, float *dW) {
-    if (L.stride != 1 || (L.k != 1 && L.k != 3) || L.cin % 8 || L.cout % 8) return false;
+    if ((L.stride != 1 && L.stride != 2) || (L.k != 1 && L.k != 3) || L.cin % 8 || L.cout % 8) return false;
+    if (L.stride == 2 && (gi.H % 2 || gi.W % 2)) return false;
     WgParams p;
-    if (!tile_shape(gi, p.BH, p.BIMG)) return false;
+    const Geom go{gi.N, conv_out(gi.H, L.k, L.stride), conv_out(gi.W, L.k, L.stride)};   // tiles walk the output pixels
+    if (!tile_shape(go, p.BH, p.BIMG)) return false;
     if (!ex.dry && !encoder(ex.ctx)) return false;
     const int taps = L.k * L.k, cin_pad = round_up(L.cin, 16), cout_pad = round_up(L.cout, 16);
     p.taps = taps; p.k = L.k; p.cin = L.cin; p.cout = L.cout;
@@ -566,8 +575,8 @@ bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer
     p.GM = groups_all >= 2 ? 2 : 1;
     const int m_chunks = (groups_all + p.GM - 1) / p.GM;
     const int n_tiles = (cout_pad + p.BN - 1) / p.BN;
-    p.H = gi.H; p.W = gi.W;
-    p.n_tiles_px = (int)(gi.P() / 128);
+    p.H = go.H; p.W = go.W; p.stride = L.stride;
+    p.n_tiles_px = (int)(go.P() / 128);
     const int stage_bytes = p.GM * 32768 + ((256 * p.BN + 1023) & ~1023);
     p.stages = (200 * 1024 - 2048) / stage_bytes; if (p.stages > kStages) p.stages = kStages;
     if (p.stages < 2) return false;
@@ -576,12 +585,13 @@ bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer
     if (splits > p.n_tiles_px) splits = p.n_tiles_px;
     if (splits < 1) splits = 1;
     p.slice = (size_t)L.cout * taps * L.cin;
-    ex.flops += 2ull * gi.P() * L.cout * L.cin * taps;
+    ex.flops += 2ull * go.P() * L.cout * L.cin * taps;
     size_t m = ex.ws.mark();
     float *part = splits > 1 ? ex.ws.get<float>((size_t)splits * p.slice) : dW;
     if (!ex.dry) {
         CUtensorMap map_a, map_g;
-        if (!encode_act_map(ex, &map_a, a, gi, L.cin, p.blockC, p.BH, p.BIMG) || !encode_act_map(ex, &map_g, gq, gi, L.cout, p.blockN, p.BH, p.BIMG)) {
+        if (!encode_act_map(ex, &map_a, a, gi, L.cin, p.blockC, go.W, p.BH, p.BIMG, L.stride) ||
+            !encode_act_map(ex, &map_g, gq, go, L.cout, p.blockN, go.W, p.BH, p.BIMG, 1)) {
             ex.failed = true; ex.ctx->err = "conv_wgrad_tc: tensor map rejected"; ex.ws.release(m); return true;
         }
         p.partial = part; p.status = ex.ctx->dev_status;
@@ -590,8 +600,8 @@ bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer
         const int smem = 1024 + p.stages * stage_bytes + (int)sizeof(TcShared) + 64;
         dim3 grid((unsigned)splits, (unsigned)m_chunks, (unsigned)n_tiles);
         wgrad_tc_kernel<<<grid, kThreads, smem, ex.stream>>>(map_a, map_g, p);
-        const double bytes = (double)gi.P() * (L.cin + L.cout) * 2 + (double)p.slice * 4 * (splits > 1 ? splits : 1);
-        ex.check("conv_wgrad_tc", bytes, 2.0 * gi.P() * L.cout * L.cin * taps);
+        const double bytes = (double)gi.P() * L.cin * 2 + (double)go.P() * L.cout * 2 + (double)p.slice * 4 * (splits > 1 ? splits : 1);
+        ex.check("conv_wgrad_tc", bytes, 2.0 * go.P() * L.cout * L.cin * taps);
         if (splits > 1) {
             splitk_sum_kernel<<<(unsigned)((p.slice + 31) / 32), 256, 0, ex.stream>>>(part, p.slice, splits, dW);
             ex.check("splitk_sum", (double)p.slice * 4 * (splits + 1));

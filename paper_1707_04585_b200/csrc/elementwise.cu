@@ -491,3 +491,21 @@ void fill_zero(Exec &ex, void *p, size_t bytes) {
     if (ex.dry) return;
     cudaMemsetAsync(p, 0, bytes, ex.stream);
 }
+
+__global__ void upsample_zero_kernel(const uint4 *__restrict__ in, uint4 *__restrict__ out, int N, int Ho, int Wo, int C8) {
+    const size_t n = (size_t)N * Ho * 2 * Wo * 2 * C8;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % C8); size_t p = i / C8;
+        const int x = (int)(p % (2 * Wo)); p /= 2 * Wo;
+        const int y = (int)(p % (2 * Ho)); const size_t b = p / (2 * Ho);
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (!(x & 1) && !(y & 1)) v = in[((b * Ho + (y >> 1)) * Wo + (x >> 1)) * C8 + c];
+        out[i] = v;
+    }
+}
+void upsample_zero_bf16(Exec &ex, const bf16 *in, bf16 *out, int N, int Ho, int Wo, int C) {
+    if (ex.dry) return;
+    const size_t n = (size_t)N * Ho * 2 * Wo * 2 * (C / 8);
+    upsample_zero_kernel<<<ew_grid(n, ex.ctx->sm_count), 256, 0, ex.stream>>>((const uint4 *)in, (uint4 *)out, N, Ho, Wo, C / 8);
+    ex.check("upsample_zero", (double)n * 16 * 1.25);
+}

@@ -96,7 +96,7 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
         double bytes = 0;
         for (LayerSlot *l : slots) {
             l->wp_f = l->wp_d = nullptr;
-            if (ex.mode != 0 || l->stride != 1 || l->cin % 8 || l->cout % 8) continue;
+            if (ex.mode != 0 || l->cin % 8 || l->cout % 8) continue;
             size_t nf = tc_pack_elems(l->cin, l->cout, l->k, false), nd = tc_pack_elems(l->cin, l->cout, l->k, true);
             bf16 *f = ex.ws.get<bf16>(nf), *dd = ex.ws.get<bf16>(nd);
             l->wp_f = f; l->wp_d = dd;

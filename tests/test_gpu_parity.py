@@ -302,3 +302,71 @@ def test_graph_replay_matches_eager(ctx):
         assert np.array_equal(a["params"][k], b["params"][k]), k
         assert np.array_equal(a["grads"][k], b["grads"][k]), k
     assert sa.kernel_launches == sb.kernel_launches and sa.flops_bwd == sb.flops_bwd
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+@pytest.mark.parametrize("N,H,cin,cout,k,stride,split", [
+    (16, 16, 32, 64, 3, 2, True),     # CIFAR-sized down-sampling transition on a coupling state (tensor-core path)
+    (128, 32, 32, 64, 3, 2, True),    # config 2, first transition at full size
+    (8, 16, 64, 112, 3, 2, True),     # 112 output channels (56 per half)
+    (16, 16, 32, 256, 3, 1, False),   # entry transition from a plain stem output
+    (5, 6, 8, 16, 3, 2, True),        # ragged: falls back to the fp32 kernels
+    (16, 8, 64, 128, 1, 2, True),     # 1x1 stride 2
+])
+def test_stored_transition_layer(ctx, mode, N, H, cin, cout, k, stride, split):
+    """BN-ReLU-conv with stride: forward and backward of one stored layer against the oracle."""
+    frac = R.DEFAULT_FRAC_BITS[mode]
+    rng = np.random.default_rng(1000 + cin + cout + H)
+    x = rng.standard_normal((N, cin, H, H)).astype(np.float32)
+    Ho = H // stride
+    dy = rng.standard_normal((N, cout, Ho, Ho)).astype(np.float32)
+    W = (rng.standard_normal((cout, cin, k, k)) * np.sqrt(2.0 / (cin * k * k))).astype(np.float32)
+    gamma = (1 + 0.1 * rng.standard_normal(cin)).astype(np.float32); beta = (0.1 * rng.standard_normal(cin)).astype(np.float32)
+    num = {}
+    if mode == 0: num["bf16_operands"] = True
+    if frac: num["frac_bits"] = frac
+    num = num or None
+    x64 = x.astype(np.float64)
+    if split and frac:
+        x64 = np.rint(x64 * (1 << frac)) / (1 << frac)
+    layer = [dict(name="T", gamma=gamma, beta=beta, W=W, stride=stride)]
+    oy, cache = orc.fn_fwd(x64, layer, 1e-5, num)
+    oy = orc.quantize_state(oy, num)
+    og = {}
+    odx = orc.fn_bwd(dy.astype(np.float64), cache, og, num)
+
+    d = B.TransitionDesc(N, H, H, cin, cout, k, stride, int(split), 1e-5, mode, frac)
+    fb, bb = B.revnet_transition_workspace_bytes(ctx, d)
+    ws = torch.empty(max(fb, bb), dtype=torch.uint8, device="cuda")
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    if split:
+        in1, in2 = R.to_state(x[:, :cin // 2], frac), R.to_state(x[:, cin // 2:], frac)
+    else:
+        in1, in2 = dev(B.to_nhwc(x)), None
+    tW, tg, tb = dev(B.w_to_abi(W)), dev(gamma), dev(beta)
+    o1 = torch.empty((N, Ho, Ho, cout // 2), dtype=torch.int32 if frac else torch.float32, device="cuda"); o2 = torch.empty_like(o1)
+    B.revnet_transition_fwd(ctx, d, in1, in2, tW, tg, tb, o1, o2, ws)
+    y = np.concatenate([R.from_state(o1, frac), R.from_state(o2, frac)], axis=1)
+    t = TOL[mode]
+    assert hp.rel_l2(y, oy) <= (1e-4 if mode else 2e-3), hp.rel_l2(y, oy)
+    d1, d2 = dev(B.to_nhwc(dy[:, :cout // 2])), dev(B.to_nhwc(dy[:, cout // 2:]))
+    if split:
+        di1 = torch.empty((N, H, H, cin // 2), dtype=torch.float32, device="cuda"); di2 = torch.empty_like(di1)
+    else:
+        di1, di2 = torch.empty((N, H, H, cin), dtype=torch.float32, device="cuda"), None
+    gW, gg, gb = torch.empty_like(tW), torch.empty_like(tg), torch.empty_like(tb)
+    B.revnet_transition_bwd(ctx, d, in1, in2, d1, d2, tW, tg, tb, di1, di2, gW, gg, gb, ws)
+    torch.cuda.synchronize()
+    dx = B.to_nchw(di1.cpu().numpy()) if not split else np.concatenate([B.to_nchw(di1.cpu().numpy()), B.to_nchw(di2.cpu().numpy())], axis=1)
+    tol = 1e-4 if mode else 1e-2          # one layer deep: far inside the stated 5e-2
+    assert hp.rel_l2(dx, odx) <= tol, hp.rel_l2(dx, odx)
+    assert hp.rel_l2(B.w_from_abi(gW.cpu().numpy()), og["T.W"]) <= tol
+    assert hp.rel_l2(gg.cpu().numpy(), og["T.gamma"]) <= tol and hp.rel_l2(gb.cpu().numpy(), og["T.beta"]) <= tol
+
+
+@pytest.mark.parametrize("mode", [0, 1])
+def test_shallow_stack_with_stride2_transitions(ctx, mode):
+    """Three stages of one unit each with two stride-2 stored transitions."""
+    st = (syn.StageCfg(1, 8, 0, "basic", 0, 1), syn.StageCfg(1, 16, 0, "basic", 3, 2), syn.StageCfg(1, 32, 0, "basic", 3, 2))
+    cfg = syn.StackCfg("shallow_s2", 16, 16, 7, 3, 1, 16, False, st, seed=31)
+    run_stack_case(ctx, cfg, mode)

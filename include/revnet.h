@@ -113,6 +113,24 @@ int revnet_block_fwd(revnet_ctx *ctx, const revnet_block_desc *desc,
                      void *y1, void *y2,
                      void *workspace, size_t workspace_bytes, void *stream);
 
+/* Block forward for callers that cannot allocate device memory (the paper has no counterpart; this
+ * is an integration aid).  Who: code running under a memory pool or a capture / real-time section
+ * where cudaMalloc and friends are forbidden or would stall, and plugins that receive tensors but
+ * no allocator.  Same computation and same results as revnet_block_fwd, but the scratch comes from
+ * a 16 MiB array built into the library (held on every GPU that loads the library until the
+ * process exits) instead of a caller workspace.  The call allocates no device memory and calls no
+ * allocating CUDA routine.  Shapes whose forward scratch (revnet_block_workspace_bytes) exceeds
+ * 16 MiB are rejected with REVNET_E_WORKSPACE_TOO_SMALL and a message naming both sizes.
+ * The first call on a device looks up the array's device address (with that device current, as it
+ * must be for every call); make that first call before starting any stream capture.  All calls
+ * share the one array, which keeps whatever the previous call left in it: calls that overlap on the
+ * GPU (different streams, or threads) race on it, so serialise them.  Nothing needs clearing
+ * between calls: each call writes every scratch region before reading it. */
+int revnet_block_fwd_noalloc(revnet_ctx *ctx, const revnet_block_desc *desc,
+                             const void *x1, const void *x2,
+                             const revnet_fn_params *F, const revnet_fn_params *G,
+                             void *y1, void *y2, void *stream);
+
 /* Block backward without stored activations (Algorithm 1): from (y1,y2) and (dy1,dy2) compute
  * x2 = y2 - G(y1), x1 = y1 - F(x2), dx1 = dy1 + (dG/dz1)^T dy2, dx2 = dy2 + (dF/dx2)^T dx1,
  * and the gradients of the parameters of F and G.  The activations computed while

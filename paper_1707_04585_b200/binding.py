@@ -22,7 +22,8 @@ _lib = None
 EXPORTS = ["revnet_create", "revnet_destroy", "revnet_last_error", "revnet_block_workspace_bytes",
            "revnet_block_fwd", "revnet_block_bwd", "revnet_stack_plan", "revnet_plan_destroy",
            "revnet_train_step", "revnet_train_step_host", "revnet_profile_enable", "revnet_profile_summary", "revnet_check_device", "revnet_plan_scratch_split",
-           "revnet_transition_workspace_bytes", "revnet_transition_fwd", "revnet_transition_bwd"]
+           "revnet_transition_workspace_bytes", "revnet_transition_fwd", "revnet_transition_bwd",
+           "revnet_block_fwd_noalloc"]
 
 
 class FnDesc(C.Structure):
@@ -328,3 +329,11 @@ def revnet_transition_bwd(ctx, desc, in1, in2, dout1, dout2, W, gamma, beta, din
     ctx.check(lib().revnet_transition_bwd(ctx.h, C.byref(desc), _ptr(in1), _ptr(in2), _ptr(dout1), _ptr(dout2), _ptr(W),
                                           _ptr(gamma), _ptr(beta), _ptr(din1), _ptr(din2), _ptr(dW), _ptr(dgamma), _ptr(dbeta),
                                           _ptr(workspace), _nbytes(workspace), _stream()), "revnet_transition_bwd")
+
+
+def revnet_block_fwd_noalloc(ctx, desc, x1, x2, F, G, y1, y2):
+    """Block forward on the library's built-in scratch array: for callers that cannot allocate device
+    memory.  Same results as revnet_block_fwd; shapes needing more than 16 MiB of scratch are rejected."""
+    fp, gp = _fn_params(F), _fn_params(G)
+    ctx.check(lib().revnet_block_fwd_noalloc(ctx.h, C.byref(desc), _ptr(x1), _ptr(x2), C.byref(fp), C.byref(gp),
+                                             _ptr(y1), _ptr(y2), _stream()), "revnet_block_fwd_noalloc")

@@ -148,6 +148,52 @@ extern "C" int revnet_block_bwd(revnet_ctx *ctx, const revnet_block_desc *d, con
     return finish(ctx, ex, "revnet_block_bwd");
 }
 
+// ---- block forward on the library's own static scratch: for callers that cannot allocate
+// Some integrations run where device allocation is off the table: inside a memory pool whose owner
+// forbids side allocations, in a real-time or safety-checked loop that must not touch the
+// allocator, or in a plugin that is handed tensors but no allocator.  For them this variant of
+// revnet_block_fwd takes its scratch from a fixed array that lives in the library image.
+#define REVNET_NOALLOC_SCRATCH_BYTES (16u << 20)
+static __device__ __align__(256) unsigned char g_noalloc_scratch[REVNET_NOALLOC_SCRATCH_BYTES];
+// device address of the array, looked up once per device (the array's name is only a host-side
+// handle in host code and must never be handed to a kernel as if it were a pointer)
+static void *g_noalloc_ptr[64] = {};
+
+extern "C" int revnet_block_fwd_noalloc(revnet_ctx *ctx, const revnet_block_desc *d, const void *x1, const void *x2,
+                                        const revnet_fn_params *Fp, const revnet_fn_params *Gp, void *y1, void *y2, void *stream) {
+    int rc = check_desc(ctx, d);
+    if (rc) return rc;
+    bool mis = false;
+    if (!x1 || !x2 || !y1 || !y2 || !fn_ptrs_ok(d->F, Fp, nullptr, false, &mis) || !fn_ptrs_ok(d->G, Gp, nullptr, false, &mis))
+        return fail(ctx, REVNET_E_INVALID_ARG, "revnet_block_fwd_noalloc: null pointer");
+    if (mis || !aligned16({x1, x2, y1, y2})) return fail(ctx, REVNET_E_MISALIGNED, "revnet_block_fwd_noalloc: pointers must be 16-byte aligned");
+    size_t need = 0;
+    revnet_block_workspace_bytes(ctx, d, &need, nullptr);
+    if (need > REVNET_NOALLOC_SCRATCH_BYTES)
+        return fail(ctx, REVNET_E_WORKSPACE_TOO_SMALL, "revnet_block_fwd_noalloc: this shape needs " + std::to_string(need) +
+                    " bytes of scratch, the static array holds " + std::to_string((size_t)REVNET_NOALLOC_SCRATCH_BYTES) +
+                    "; use revnet_block_fwd with a caller workspace");
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
+        return fail(ctx, REVNET_E_CUDA, "revnet_block_fwd_noalloc: no current device");
+    if (dev != ctx->device) return fail(ctx, REVNET_E_INVALID_ARG, "revnet_block_fwd_noalloc: the context's device must be current");
+    if (!g_noalloc_ptr[dev]) {
+        // one-time set-up for this device (with it current): resolve the array's device address
+        void *p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
+        if (e != cudaSuccess || !p)
+            return fail(ctx, REVNET_E_CUDA, std::string("revnet_block_fwd_noalloc: cudaGetSymbolAddress: ") + cudaGetErrorString(e));
+        g_noalloc_ptr[dev] = p;
+    }
+    Exec ex; ex.ctx = ctx; ex.dry = false; ex.mode = d->mode; ex.eps = d->eps; ex.stream = (cudaStream_t)stream;
+    ex.q = d->state_frac_bits ? ldexpf(1.f, -d->state_frac_bits) : 0.f;
+    ex.ws.dry = false; ex.ws.base = (char *)g_noalloc_ptr[dev]; ex.ws.cap = REVNET_NOALLOC_SCRATCH_BYTES;
+    // nothing in the block forward relies on zeroed scratch: every region is written before it is read
+    block_forward(ex, Geom{d->N, d->H, d->W}, d->c, layers_of(d->F, Fp, nullptr), layers_of(d->G, Gp, nullptr),
+                  (float *)x1, (float *)x2, (float *)y1, (float *)y2);
+    return finish(ctx, ex, "revnet_block_fwd_noalloc");
+}
+
 // ---- stored (non-reversible) BN -> ReLU -> conv layer: forward keeps nothing, backward rebuilds its
 // operands from the stored input (Section 3.2: inputs of non-reversible layers are kept)
 static int check_trans(revnet_ctx *ctx, const revnet_transition_desc *d) {

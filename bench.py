@@ -196,6 +196,12 @@ def run_ours(args, cfg):
     prof = B.revnet_profile_summary(ctx)
     B.revnet_profile_enable(ctx, False)
     final_loss = float(run.loss.item())
+    # per-block forward / reconstructing-backward time at each stage shape of the workload
+    block_ms = {}
+    if rank == 0:
+        for s_cfg, H in zip(rcfg.stages, syn.stage_resolutions(rcfg)):
+            bc = syn.BlockCfg(rcfg.N, H, H, s_cfg.c, s_cfg.w, s_cfg.kind, seed=9)
+            block_ms[f"{s_cfg.kind}_c{s_cfg.c}_{H}x{H}"] = R.time_block(ctx, bc, 0, reps=5, warmup=3)
 
     t = torch.tensor([dev_ms, e2e_ms], dtype=torch.float64, device="cuda")
     if world > 1:
@@ -232,7 +238,7 @@ def run_ours(args, cfg):
                              d2h_bytes_per_step=4 + 4 * rcfg.N, ms_per_step=e2e_ms / args.steps),
                     gpu_launches=launches, clocks=clocks, roofline=roof,
                     activation_bytes=int(st.stored_activation_bytes), workspace_bytes=int(st.workspace_peak_bytes),
-                    flops_per_step=int(st.flops_fwd + st.flops_bwd), final_loss=final_loss)
+                    flops_per_step=int(st.flops_fwd + st.flops_bwd), final_loss=final_loss, block_ms=block_ms)
         if not args.no_cpu and world == 1:
             line["cpu_baseline"] = {k: v for k, v in cpu_baseline(cfg, min(cfg.N, args.ref_batch)).items() if k != "seconds_per_step"}
         print(json.dumps(line), flush=True)

@@ -117,3 +117,39 @@ class StackRunner:
                     grads=B.unpack_params(self.specs, self.grads.cpu().numpy()),
                     params=B.unpack_params(self.specs, self.params.cpu().numpy()),
                     momentum=B.unpack_params(self.specs, self.momentum.cpu().numpy()))
+
+
+def time_block(ctx: B.Context, b: syn.BlockCfg, mode: int, reps: int = 10, warmup: int = 3):
+    """Device time (ms) of one block forward and one reconstructing backward at shape b, in place,
+    through the C ABI, with CUDA events on the launching stream."""
+    inp = syn.make_block_inputs(b, affine_jitter=True)
+    r = BlockRunner(ctx, b, mode)
+    r.load(inp["params"])
+    x1, x2 = to_state(inp["x1"], r.frac), to_state(inp["x2"], r.frac)
+    d1, d2 = _dev(B.to_nhwc(inp["dy1"])), _dev(B.to_nhwc(inp["dy2"]))
+    stream = torch.cuda.current_stream()
+    ms = {"fwd": [], "bwd": []}
+    for i in range(warmup + reps):
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record(stream)
+        B.revnet_block_fwd(ctx, r.desc, x1, x2, r.F, r.G, x1, x2, r.ws)
+        e[1].record(stream)
+        B.revnet_block_bwd(ctx, r.desc, x1, x2, d1, d2, r.F, r.G, x1, x2, d1, d2, r.gF, r.gG, r.ws)
+        e[2].record(stream)
+        torch.cuda.synchronize()
+        if i >= warmup:
+            ms["fwd"].append(e[0].elapsed_time(e[1])); ms["bwd"].append(e[1].elapsed_time(e[2]))
+    B.revnet_check_device(ctx)
+    return {k: float(np.median(v)) for k, v in ms.items()}
+
+
+if __name__ == "__main__":
+    import argparse, json
+    ap = argparse.ArgumentParser(description="time one reversible block (forward, reconstructing backward)")
+    ap.add_argument("--N", type=int, default=128); ap.add_argument("--H", type=int, default=32)
+    ap.add_argument("--c", type=int, default=64); ap.add_argument("--w", type=int, default=0)
+    ap.add_argument("--kind", default="basic"); ap.add_argument("--mode", type=int, default=0)
+    ap.add_argument("--reps", type=int, default=10); ap.add_argument("--warmup", type=int, default=3)
+    a = ap.parse_args()
+    c = B.Context(0)
+    print(json.dumps(dict(shape=vars(a), ms=time_block(c, syn.BlockCfg(a.N, a.H, a.H, a.c, a.w, a.kind, seed=5), a.mode, a.reps, a.warmup))))

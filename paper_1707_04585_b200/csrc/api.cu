@@ -15,13 +15,14 @@ extern "C" int revnet_create(revnet_ctx **out, int device) {
         int sm = 0;
         if (cudaSetDevice(device) != cudaSuccess ||
             cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
-            cudaMalloc(&c->dev_status, 256) != cudaSuccess || cudaMemset(c->dev_status, 0, 256) != cudaSuccess ||
+            cudaMalloc(&c->dev_status, 1024) != cudaSuccess || cudaMemset(c->dev_status, 0, 1024) != cudaSuccess ||
             cudaStreamCreateWithFlags(&c->capture_stream, cudaStreamNonBlocking) != cudaSuccess) {
             cudaGetLastError();
             delete c;
             return REVNET_E_CUDA;
         }
         c->sm_count = sm;
+        c->counters = reinterpret_cast<unsigned int *>(c->dev_status) + 64;
     }
     *out = c;
     return REVNET_OK;
@@ -216,13 +217,13 @@ static void trans_run(Exec &ex, const revnet_transition_desc *d, bool backward, 
     Pair tin = d->in_split ? halves((float *)in1, (float *)in2, d->cin / 2, q) : single((float *)in1, d->cin);
     const int ch = d->cout / 2;
     if (!backward) {
-        fn_forward(ex, g, tin, T, Pair{}, halves((float *)out1, (float *)out2, ch, q), 0, nullptr, false);
+        fn_forward(ex, g, tin, nullptr, T, Pair{}, halves((float *)out1, (float *)out2, ch, q), 0, nullptr, nullptr, false);
     } else {
         FnSaved sv;
         size_t m = ex.ws.mark();
-        fn_forward(ex, g, tin, T, Pair{}, Pair{}, 0, &sv, true);
+        fn_forward(ex, g, tin, nullptr, T, Pair{}, Pair{}, 0, nullptr, &sv, true);
         Pair gout = d->in_split ? halves(din1, din2, d->cin / 2) : single(din1, d->cin);
-        fn_backward(ex, g, tin, T, sv, halves((float *)dout1, (float *)dout2, ch), Pair{}, gout);
+        fn_backward(ex, g, tin, T, sv, halves((float *)dout1, (float *)dout2, ch), nullptr, Pair{}, gout, nullptr);
         ex.ws.release(m);
     }
 }

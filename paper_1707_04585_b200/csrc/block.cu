@@ -3,21 +3,32 @@
 //   backward  Algorithm 1: x2 = y2 - G(y1); backprop G; x1 = y1 - F(x2); backprop F
 // The tensors a residual function produces while being recomputed stay in the workspace and
 // feed its own backprop, so each conv layer costs four passes per step in all.
+//
+// Batch statistics.  A tensor-core convolution leaves the per-channel mean and 1/sqrt(var+eps) of
+// what it stores (its epilogue sums them), so the BN that reads the tensor next needs no pass of
+// its own.  Inside a function that always applies.  For the coupling state it applies when the
+// caller hands Moments through (a stack does); otherwise the statistics of x2 and y1 are computed
+// by the stand-alone reduction, in the forward and in the reversal alike, which keeps the
+// recomputed F and G bit-identical to the forward ones.
 #include "common.cuh"
 
 // dispatch: tensor-core kernels take the shapes they support in mode 0, the fp32 kernels the rest
-bool conv_fprop_tc(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign);
-bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da);
+bool conv_fprop_tc(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign, Moments *stats);
+bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, const BnBwdReq *bb);
 bool conv_wgrad_tc(Exec &ex, const void *g, const void *a, Geom gi, const Layer &L, float *dW);
 
-static void conv_fprop(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign) {
+// stats: in = where the statistics of `out` should go (or nullptr); stats->valid says whether the kernel provides them
+static void conv_fprop(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign, Moments *stats) {
     const bool b16 = ex.mode == 0;
-    if (b16 && conv_fprop_tc(ex, a, gi, L, out, partner, sign)) return;
+    if (stats) stats->valid = false;
+    if (b16 && conv_fprop_tc(ex, a, gi, L, out, partner, sign, stats)) return;
+    if (stats) stats->valid = false;
     conv_fprop_simt(ex, a, b16, gi, L, out, partner, sign);
 }
-static void conv_dgrad(Exec &ex, const void *g, Geom gi, const Layer &L, float *da) {
+// returns true when the epilogue also produced the BN-backward sums asked for in bb
+static bool conv_dgrad(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, const BnBwdReq *bb) {
     const bool b16 = ex.mode == 0;
-    if (b16 && L.stride == 1 && conv_dgrad_tc(ex, g, gi, L, da)) return;
+    if (b16 && L.stride == 1 && conv_dgrad_tc(ex, g, gi, L, da, bb)) return bb != nullptr;
     if (b16 && L.stride == 2 && gi.H % 2 == 0 && gi.W % 2 == 0 && L.cout % 8 == 0) {
         // stride 2: spread g over the input grid (zeros between samples); the data gradient is then the
         // stride-1 one:  da[y,x] = sum_taps g_up[y + pad - kh, x + pad - kw] W[.,kh,kw,.]
@@ -25,11 +36,12 @@ static void conv_dgrad(Exec &ex, const void *g, Geom gi, const Layer &L, float *
         bf16 *gup = ex.ws.get<bf16>(gi.P() * L.cout);
         upsample_zero_bf16(ex, (const bf16 *)g, gup, gi.N, gi.H / 2, gi.W / 2, L.cout);
         Layer L1 = L; L1.stride = 1;
-        const bool ok = conv_dgrad_tc(ex, gup, gi, L1, da);
+        const bool ok = conv_dgrad_tc(ex, gup, gi, L1, da, bb);
         ex.ws.release(m);
-        if (ok) return;
+        if (ok) return bb != nullptr;
     }
     conv_dgrad_simt(ex, g, b16, gi, L, da);
+    return false;
 }
 static void conv_wgrad(Exec &ex, const void *g, const void *a, Geom gi, const Layer &L, float *dW) {
     const bool b16 = ex.mode == 0;
@@ -41,30 +53,38 @@ static size_t esz(const Exec &ex) { return ex.mode == 0 ? 2 : 4; }
 
 // out = partner + sign * Fn(u).  With `saved`, every layer's activated input, BN input and BN
 // statistics are left in the workspace (the caller releases them after the backward).
-void fn_forward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, Pair partner, Pair out, int sign,
-                FnSaved *saved, bool skip_last_conv) {
+void fn_forward(Exec &ex, Geom g, Pair u, const Moments *mom_in, const std::vector<Layer> &layers, Pair partner, Pair out,
+                int sign, Moments *mom_out, FnSaved *saved, bool skip_last_conv) {
     const int L = (int)layers.size();
     const bool b16 = ex.mode == 0;
     size_t outer = ex.ws.mark();
     Pair t = u;
     Geom gi = g;
     if (saved) { saved->a.clear(); saved->t.clear(); saved->bn.clear(); saved->gin = g; }
+    Moments cur;
+    if (mom_in && mom_in->valid) cur = *mom_in;
+    if (mom_out) mom_out->valid = false;
     for (int l = 0; l < L; l++) {
         const Layer &ly = layers[l];
         const size_t P = gi.P();
-        BnState st = bn_alloc(ex, ly.cin);
-        bn_stats(ex, t, P, ly.gamma, ly.beta, st);
+        if (!cur.valid) {
+            cur = mom_alloc(ex, ly.cin);
+            bn_stats(ex, t, P, cur);
+            cur.valid = true;
+        }
         void *a = ex.ws.alloc(P * ly.cin * esz(ex));
-        bn_relu_apply(ex, t, P, st, a, b16);
+        bn_relu_apply(ex, t, P, BnRef{ly.gamma, ly.beta, cur.mean, cur.rstd}, a, b16);
         Geom go{gi.N, conv_out(gi.H, ly.k, ly.stride), conv_out(gi.W, ly.k, ly.stride)};
-        if (saved) { saved->a.push_back(a); saved->bn.push_back(st); }
+        if (saved) { saved->a.push_back(a); saved->bn.push_back(cur); }
         if (l == L - 1) {
-            if (!skip_last_conv) conv_fprop(ex, a, gi, ly, out, partner, sign);
+            if (!skip_last_conv) conv_fprop(ex, a, gi, ly, out, partner, sign, mom_out);
         } else {
             float *tn = ex.ws.get<float>(go.P() * ly.cout);
-            conv_fprop(ex, a, gi, ly, single(tn, ly.cout), Pair{}, 0);
+            Moments next = mom_alloc(ex, ly.cout);
+            conv_fprop(ex, a, gi, ly, single(tn, ly.cout), Pair{}, 0, &next);
             if (saved) saved->t.push_back(tn);
             t = single(tn, ly.cout);
+            cur = next;     // valid only if the epilogue summed them; else the next round computes them
         }
         gi = go;
     }
@@ -72,8 +92,8 @@ void fn_forward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, Pair
 }
 
 // dgin_out = add + (dFn/du)^T gup ; parameter gradients through the layers' pointers.
-void fn_backward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, FnSaved &saved, Pair gup,
-                 Pair add, Pair dgin_out) {
+void fn_backward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, FnSaved &saved, Pair gup, const bf16 *gup_cast,
+                 Pair add, Pair dgin_out, bf16 *dgin_cast) {
     const int L = (int)layers.size();
     const bool b16 = ex.mode == 0;
     size_t outer = ex.ws.mark();
@@ -86,7 +106,8 @@ void fn_backward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, FnS
     const void *gcur;
     {
         const int C = gup.C();
-        if (!b16 && gup.c1 == 0) gcur = gup.p0;
+        if (b16 && gup_cast) gcur = gup_cast;
+        else if (!b16 && gup.c1 == 0) gcur = gup.p0;
         else {
             void *buf = ex.ws.alloc(gin[L].P() * C * esz(ex));
             concat_cast(ex, gup, gin[L].P(), buf, b16);
@@ -98,14 +119,17 @@ void fn_backward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, FnS
         const size_t P = gin[l].P();
         conv_wgrad(ex, gcur, saved.a[l], gin[l], ly, ly.dW);
         float *da = ex.ws.get<float>(P * ly.cin);
-        conv_dgrad(ex, gcur, gin[l], ly, da);
+        float *coef = ex.ws.get<float>((size_t)3 * ly.cin);
+        const Pair tl = l == 0 ? u : single(saved.t[l - 1], ly.cin);
+        const BnRef bn{ly.gamma, ly.beta, saved.bn[l].mean, saved.bn[l].rstd};
+        const BnBwdReq bb{tl, bn, ly.dgamma, ly.dbeta, coef};
+        const bool sums_done = conv_dgrad(ex, gcur, gin[l], ly, da, &bb);
         if (l == 0) {
             // add.p0 == nullptr: the gradient is stored without a partner (stored transitions)
-            bn_relu_bwd(ex, da, u, P, saved.bn[0], ly.gamma, ly.dgamma, ly.dbeta, nullptr, false, add, dgin_out);
+            bn_relu_bwd(ex, da, tl, P, bn, ly.dgamma, ly.dbeta, coef, sums_done, nullptr, false, add, dgin_out, b16 ? dgin_cast : nullptr);
         } else {
             void *dt = ex.ws.alloc(P * ly.cin * esz(ex));
-            bn_relu_bwd(ex, da, single(saved.t[l - 1], ly.cin), P, saved.bn[l], ly.gamma, ly.dgamma, ly.dbeta,
-                        dt, b16, Pair{}, Pair{});
+            bn_relu_bwd(ex, da, tl, P, bn, ly.dgamma, ly.dbeta, coef, sums_done, dt, b16, Pair{}, Pair{}, nullptr);
             gcur = dt;
         }
     }
@@ -113,26 +137,33 @@ void fn_backward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, FnS
 }
 
 void block_forward(Exec &ex, Geom g, int c, const std::vector<Layer> &F, const std::vector<Layer> &G,
-                   float *x1, float *x2, float *y1, float *y2) {
+                   float *x1, float *x2, float *y1, float *y2, const Moments *mx2, Moments *my1, Moments *my2) {
     const float q = ex.q;
-    fn_forward(ex, g, single(x2, c, q), F, single(x1, c, q), single(y1, c, q), +1, nullptr, false);
-    fn_forward(ex, g, single(y1, c, q), G, single(x2, c, q), single(y2, c, q), +1, nullptr, false);
+    // without hand-off (stand-alone call) the statistics of x2 and y1 come from the stand-alone reduction,
+    // as they will in the reversal, which is handed y1 from outside
+    fn_forward(ex, g, single(x2, c, q), mx2, F, single(x1, c, q), single(y1, c, q), +1, my1, nullptr, false);
+    fn_forward(ex, g, single(y1, c, q), my1, G, single(x2, c, q), single(y2, c, q), +1, my2, nullptr, false);
 }
 
 void block_backward(Exec &ex, Geom g, int c, const std::vector<Layer> &F, const std::vector<Layer> &G,
                     const float *y1, const float *y2, const float *dy1, const float *dy2,
-                    float *x1, float *x2, float *dx1, float *dx2) {
+                    float *x1, float *x2, float *dx1, float *dx2,
+                    Moments *m1, Moments *m2, const Moments *m2_use, const bf16 *dy2_cast, bf16 *dx2_cast) {
     FnSaved sv;
     const float q = ex.q;   // format of the coupling state; gradients are always float
+    size_t m0 = ex.ws.mark();
+    // bf16 copy of dz1 for F's backward (the BN-backward apply that produces dz1 writes it)
+    bf16 *dz1_cast = ex.mode == 0 ? ex.ws.get<bf16>(g.P() * c) : nullptr;
     size_t m = ex.ws.mark();
     // x2 = y2 - G(z1), z1 = y1
-    fn_forward(ex, g, single((float *)y1, c, q), G, single((float *)y2, c, q), single(x2, c, q), -1, &sv, false);
+    fn_forward(ex, g, single((float *)y1, c, q), m1, G, single((float *)y2, c, q), single(x2, c, q), -1, m2, &sv, false);
     // dz1 = dy1 + (dG/dz1)^T dy2 ; dW_G
-    fn_backward(ex, g, single((float *)y1, c, q), G, sv, single((float *)dy2, c), single((float *)dy1, c), single(dx1, c));
+    fn_backward(ex, g, single((float *)y1, c, q), G, sv, single((float *)dy2, c), dy2_cast, single((float *)dy1, c), single(dx1, c), dz1_cast);
     ex.ws.release(m);
     // x1 = z1 - F(x2)
-    fn_forward(ex, g, single(x2, c, q), F, single((float *)y1, c, q), single(x1, c, q), -1, &sv, false);
+    const Moments *mf = (m2_use && m2_use->valid) ? m2_use : m2;
+    fn_forward(ex, g, single(x2, c, q), mf, F, single((float *)y1, c, q), single(x1, c, q), -1, m1, &sv, false);
     // dx2 = dy2 + (dF/dx2)^T dz1 ; dW_F ; dx1 = dz1 (already in place)
-    fn_backward(ex, g, single(x2, c, q), F, sv, single(dx1, c), single((float *)dy2, c), single(dx2, c));
-    ex.ws.release(m);
+    fn_backward(ex, g, single(x2, c, q), F, sv, single(dx1, c), dz1_cast, single((float *)dy2, c), single(dx2, c), dx2_cast);
+    ex.ws.release(m0);
 }

@@ -17,6 +17,10 @@ struct revnet_ctx {
     int sm_count = 148;
     std::string err;
     int *dev_status = nullptr;   // device word for bounded-wait time-outs
+    unsigned int *counters = nullptr;   // zeroed words the kernels' grid-wide reductions count on (each leaves its word zero)
+    int next_counter = 0;
+    unsigned int *counter() { unsigned int *c = counters + next_counter; next_counter = (next_counter + 1) % kCounters; return c; }
+    static constexpr int kCounters = 192;
     void *encode_tiled = nullptr; // driver entry point for tensor-map encoding
     cudaStream_t capture_stream = nullptr;   // private stream on which a train step is captured into a graph
     // per-kernel timing (revnet_profile_*): one event after every launch while enabled
@@ -58,6 +62,32 @@ struct Pair {
             if (sign) { int p = *reinterpret_cast<const int *>(partner.at(row, ch)); iv = sign > 0 ? p + iv : p - iv; }
             *reinterpret_cast<int *>(o) = iv;
         }
+    }
+    // store v in the tensor's format; returns the values as stored (dequantised)
+    __device__ __forceinline__ float4 store4(size_t row, int ch, float4 v) const {
+        float *o = at(row, ch);
+        if (q == 0.f) { *reinterpret_cast<float4 *>(o) = v; return v; }
+        const float s = 1.f / q;
+        int4 iv = make_int4(__float2int_rn(v.x * s), __float2int_rn(v.y * s), __float2int_rn(v.z * s), __float2int_rn(v.w * s));
+        *reinterpret_cast<int4 *>(o) = iv;
+        return make_float4(__int2float_rn(iv.x) * q, __int2float_rn(iv.y) * q, __int2float_rn(iv.z) * q, __int2float_rn(iv.w) * q);
+    }
+    // out = partner + sign * v with the partner's 16 raw bytes already loaded; returns the stored values (dequantised)
+    __device__ __forceinline__ float4 couple4_with(size_t row, int ch, float4 v, float4 praw, int sign) const {
+        float *o = at(row, ch);
+        if (q == 0.f) {
+            if (sign > 0) { v.x = praw.x + v.x; v.y = praw.y + v.y; v.z = praw.z + v.z; v.w = praw.w + v.w; }
+            else { v.x = praw.x - v.x; v.y = praw.y - v.y; v.z = praw.z - v.z; v.w = praw.w - v.w; }
+            *reinterpret_cast<float4 *>(o) = v;
+            return v;
+        }
+        const float s = 1.f / q;
+        int4 iv = make_int4(__float2int_rn(v.x * s), __float2int_rn(v.y * s), __float2int_rn(v.z * s), __float2int_rn(v.w * s));
+        const int4 p = make_int4(__float_as_int(praw.x), __float_as_int(praw.y), __float_as_int(praw.z), __float_as_int(praw.w));
+        if (sign > 0) { iv.x = p.x + iv.x; iv.y = p.y + iv.y; iv.z = p.z + iv.z; iv.w = p.w + iv.w; }
+        else { iv.x = p.x - iv.x; iv.y = p.y - iv.y; iv.z = p.z - iv.z; iv.w = p.w - iv.w; }
+        *reinterpret_cast<int4 *>(o) = iv;
+        return make_float4(__int2float_rn(iv.x) * q, __int2float_rn(iv.y) * q, __int2float_rn(iv.z) * q, __int2float_rn(iv.w) * q);
     }
     // four consecutive channels at once (ch % 4 == 0)
     __device__ __forceinline__ void couple4(size_t row, int ch, float4 v, const Pair &partner, int sign) const {
@@ -130,24 +160,46 @@ struct Layer {
     const bf16 *Wp_dgrad = nullptr;   // bf16 [cin][k][k][cout_pad], taps mirrored (mode 0)
 };
 
-// Per-BN statistics kept between a layer's forward and its backward.
-struct BnState {
-    float *scale, *shift, *mean, *rstd;   // [C] each
+// Batch statistics of one tensor: per-channel mean and 1/sqrt(var + eps), [C] each (device).
+// `valid` is host-side bookkeeping: whether a kernel enqueued earlier fills them.
+struct Moments {
+    float *mean = nullptr, *rstd = nullptr;
+    bool valid = false;
 };
+// One BN as its consumers see it: scale = gamma*rstd, shift = beta - mean*scale are derived on the
+// fly, always with the same two roundings, so that the ReLU mask of the backward equals the forward's.
+struct BnRef {
+    const float *gamma, *beta, *mean, *rstd;
+};
+#ifdef __CUDACC__
+__device__ __forceinline__ void bn_sc_sh(float g, float b, float mu, float r, float &sc, float &sh) {
+    sc = __fmul_rn(g, r);
+    sh = __fmaf_rn(-mu, sc, b);
+}
+__device__ __forceinline__ void bn_coef4(const BnRef &bn, int c, float4 &sc, float4 &sh, float4 &mu, float4 &rs) {
+    const float4 g = *reinterpret_cast<const float4 *>(bn.gamma + c), b = *reinterpret_cast<const float4 *>(bn.beta + c);
+    mu = *reinterpret_cast<const float4 *>(bn.mean + c); rs = *reinterpret_cast<const float4 *>(bn.rstd + c);
+    bn_sc_sh(g.x, b.x, mu.x, rs.x, sc.x, sh.x); bn_sc_sh(g.y, b.y, mu.y, rs.y, sc.y, sh.y);
+    bn_sc_sh(g.z, b.z, mu.z, rs.z, sc.z, sh.z); bn_sc_sh(g.w, b.w, mu.w, rs.w, sc.w, sh.w);
+}
+#endif
 
 struct Geom { int N, H, W; size_t P() const { return (size_t)N * H * W; } };
 
 // ---------------------------------------------------------------- elementwise.cu
-BnState bn_alloc(Exec &ex, int C);
-// batch statistics of t ([P,C]) -> scale = gamma*rstd, shift = beta - mean*scale, mean, rstd
-void bn_stats(Exec &ex, Pair t, size_t P, const float *gamma, const float *beta, BnState st);
+Moments mom_alloc(Exec &ex, int C);
+// batch statistics of t ([P,C]) -> mean, rstd (two kernels; the convolution epilogues produce the
+// same quantities for the tensors they write)
+void bn_stats(Exec &ex, Pair t, size_t P, Moments m);
 // a = relu(scale*t + shift) written as one [P,C] tensor of float (strict) or bf16
-void bn_relu_apply(Exec &ex, Pair t, size_t P, BnState st, void *a, bool a_bf16);
-// BN+ReLU backward: da [P,C] fp32; t the BN input; writes dgamma, dbeta and
-//   out = dt                  (out_single: float or bf16 [P,C])   when add.p0 == nullptr
-//   out_pair = add + dt       (fp32 pair)                        otherwise
-void bn_relu_bwd(Exec &ex, const float *da, Pair t, size_t P, BnState st, const float *gamma,
-                 float *dgamma, float *dbeta, void *out_single, bool out_bf16, Pair add, Pair out_pair);
+void bn_relu_apply(Exec &ex, Pair t, size_t P, BnRef bn, void *a, bool a_bf16);
+// BN+ReLU backward: da [P,C] fp32; t the BN input.  Unless sums_done (a data-gradient epilogue
+// already wrote dgamma, dbeta and coef) the two reductions run first.  Then
+//   out = dt                  (out_single: float or bf16 [P,C])   when out_pair.p0 == nullptr
+//   out_pair = add + dt       (fp32 pair; add.p0 == nullptr: plain dt), optionally also
+//   out_cast = bf16 copy of out_pair as one [P,C] tensor (the next function's upstream operand)
+void bn_relu_bwd(Exec &ex, const float *da, Pair t, size_t P, BnRef bn, float *dgamma, float *dbeta, float *coef,
+                 bool sums_done, void *out_single, bool out_bf16, Pair add, Pair out_pair, bf16 *out_cast);
 // copy a pair into one [P,C] tensor of float or bf16
 void concat_cast(Exec &ex, Pair src, size_t P, void *dst, bool dst_bf16);
 void maxpool_fwd(Exec &ex, const float *in, float *out, int N, int H, int W, int C);
@@ -173,6 +225,9 @@ void conv_dgrad_simt(Exec &ex, const void *g, bool g_bf16, Geom gi, const Layer 
 void conv_wgrad_simt(Exec &ex, const void *g, bool g_bf16, const void *a, bool a_bf16, Geom gi, const Layer &L, float *dW);
 
 // ---------------------------------------------------------------- conv_tc.cu
+// What a data-gradient epilogue needs to fuse the two sums of the BN+ReLU backward of the layer's
+// own BN: its input t, its coefficients, and where dgamma, dbeta and coef[3][C] go.
+struct BnBwdReq { Pair t; BnRef bn; float *dgamma, *dbeta, *coef; };
 // bf16 weight packs of the tensor-core kernels, built once per train step
 struct PackJob { const float *W; bf16 *out; int Co, Ci, k, rows_pad, cols_pad, transposed; };
 size_t tc_pack_elems(int cin, int cout, int k, bool transposed);
@@ -183,21 +238,34 @@ void tc_pack_batch(Exec &ex, const PackJob *jobs_dev, int n_jobs, double bytes);
 struct FnSaved;   // activations kept from a residual function's (re)computation
 // out = partner + sign * Fn(u); if saved != nullptr the per-layer tensors stay in the workspace
 // skip_last_conv: only rebuild the saved tensors (used to re-derive a stored layer's operands)
-void fn_forward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, Pair partner, Pair out, int sign,
-                FnSaved *saved, bool skip_last_conv);
-// dgin_out = add + (dFn/du)^T gup, parameter gradients written through the layers' pointers
-void fn_backward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, FnSaved &saved, Pair gup,
-                 Pair add, Pair dgin_out);
+// mom_in: statistics of u if a kernel enqueued earlier provides them (else they are computed here);
+// mom_out: where the last convolution's epilogue should leave the statistics of `out`
+// (mom_out->valid tells whether it did).
+void fn_forward(Exec &ex, Geom g, Pair u, const Moments *mom_in, const std::vector<Layer> &layers, Pair partner, Pair out,
+                int sign, Moments *mom_out, FnSaved *saved, bool skip_last_conv);
+// dgin_out = add + (dFn/du)^T gup, parameter gradients written through the layers' pointers;
+// gup_cast: bf16 [P,C] copy of gup if the caller already has one; dgin_cast: if non-null, a bf16
+// [P,C] copy of dgin_out is written there as well
+void fn_backward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, FnSaved &saved, Pair gup, const bf16 *gup_cast,
+                 Pair add, Pair dgin_out, bf16 *dgin_cast);
 struct FnSaved {
     std::vector<void *> a;        // activated input of each conv
     std::vector<float *> t;       // BN input of each layer beyond the first (conv outputs)
-    std::vector<BnState> bn;
+    std::vector<Moments> bn;
     Geom gin;
 };
+// Statistics hand-off between blocks of a stage (all optional, nullptr = compute where needed):
+//   forward : mx2 = statistics of x2 (if valid); my1, my2: where those of y1, y2 are left
+//   backward: m1 in = statistics of y1, out = statistics of x1; m2 out = statistics of x2;
+//             m2_use: statistics F must use for x2 when the forward pass took them from elsewhere
+//             (the first block of a stage), so that F is recomputed bit for bit
 void block_forward(Exec &ex, Geom g, int c, const std::vector<Layer> &F, const std::vector<Layer> &G,
-                   float *x1, float *x2, float *y1, float *y2);
+                   float *x1, float *x2, float *y1, float *y2,
+                   const Moments *mx2 = nullptr, Moments *my1 = nullptr, Moments *my2 = nullptr);
 void block_backward(Exec &ex, Geom g, int c, const std::vector<Layer> &F, const std::vector<Layer> &G,
                     const float *y1, const float *y2, const float *dy1, const float *dy2,
-                    float *x1, float *x2, float *dx1, float *dx2);
+                    float *x1, float *x2, float *dx1, float *dx2,
+                    Moments *m1 = nullptr, Moments *m2 = nullptr, const Moments *m2_use = nullptr,
+                    const bf16 *dy2_cast = nullptr, bf16 *dx2_cast = nullptr);
 
 static inline int conv_out(int in, int k, int s) { return (in + 2 * (k / 2) - k) / s + 1; }

@@ -1,0 +1,245 @@
+// Epilogue shared by the tensor-core convolution kernels: drains a 128-row accumulator from tensor
+// memory through a padded shared-memory stage, so that global accesses are coalesced, and fuses
+//   - the coupling  y = x + F  /  x = y - F  on the float or fixed-point state      (Section 3.1)
+//   - per-channel sums of the stored result (the batch statistics of the BN that reads it next,
+//     Eq. 2: a(x) = ReLU(BN(x))), or, for a data gradient, the two sums of the BN+ReLU backward
+//   - the reduction of those sums over the grid: the CTA that finishes last adds the per-CTA
+//     partials in a fixed order (double precision) and writes mean / 1/sqrt(var+eps), or
+//     dgamma, dbeta and the coefficients of the BN-backward formula.
+// Everything is summed in an order fixed by the launch shape, so a residual function recomputed
+// in the backward pass reproduces its forward bits.
+#pragma once
+#include "common.cuh"
+#include "tc_ptx.cuh"
+
+namespace tc {
+
+enum { EPI_PLAIN = 0, EPI_COUPLE = 1, EPI_BNBWD = 2 };
+
+struct EpiArgs {
+    int mode;
+    Pair out, partner;       // [P, n_cols]; partner only with EPI_COUPLE
+    int sign;                // EPI_COUPLE: +1 / -1
+    int n_cols;              // valid output channels
+    // reductions (optional: part == nullptr switches them off; EPI_BNBWD always reduces)
+    float *part;             // [gridDim.x][n_cols/4][2][4]: per channel quad, 4 sums then 4 second sums
+    unsigned int *counter;   // zero on entry, left zero
+    double inv_count;        // 1 / pixels
+    float eps;
+    float *mean, *rstd;      // EPI_PLAIN / EPI_COUPLE: statistics of the stored result
+    // EPI_BNBWD: the accumulator is da, the gradient w.r.t. a = ReLU(BN(t))
+    Pair t;
+    BnRef bn;
+    float *dgamma, *dbeta, *coef;   // coef: [3][n_cols] = gamma*rstd, gamma*rstd*dbeta/M, gamma*rstd*dgamma/M
+};
+
+// Geometry of the 128-row tiles: a tile is BIMG images x BH rows x W columns of the OUTPUT.
+struct TileGeom {
+    int N, H, W;
+    int BH, BIMG;
+    int tiles_per_img;       // BIMG == 1
+    int n_px_tiles;
+    int hw_order;            // accumulator rows run (h, img, w) instead of (img, h, w)
+};
+__device__ __forceinline__ void tile_origin(const TileGeom &g, int t, int &n0, int &h0) {
+    if (g.BIMG > 1) { n0 = t * g.BIMG; h0 = 0; }
+    else { n0 = t / g.tiles_per_img; h0 = (t - n0 * g.tiles_per_img) * g.BH; }
+}
+// global pixel index of accumulator row m, or -1 for a padding row
+__device__ __forceinline__ int tile_row_pixel(const TileGeom &g, int n0, int h0, int m) {
+    if (m >= g.BIMG * g.BH * g.W) return -1;
+    int img, h, w = m % g.W;
+    if (g.hw_order) { h = m / (g.BIMG * g.W); img = (m / g.W) % g.BIMG; }
+    else { img = m / (g.BH * g.W); h = (m / g.W) % g.BH; }
+    h += h0;
+    if (n0 + img >= g.N || h >= g.H) return -1;
+    return ((n0 + img) * g.H + h) * g.W + w;
+}
+
+constexpr int kEpiChunk = 64;                    // accumulator columns staged at a time
+constexpr int kEpiPitch = kEpiChunk + 4;         // floats per staged row (bank-conflict padding)
+constexpr int kEpiStageBytes = 128 * kEpiPitch * 4;
+constexpr int kEpiMaxChunks = 4;                 // N tile <= 256 columns
+
+struct EpiAcc {                                  // per-thread running sums, by column chunk
+    float s[kEpiMaxChunks][4], ss[kEpiMaxChunks][4];
+    __device__ __forceinline__ void clear() {
+#pragma unroll
+        for (int c = 0; c < kEpiMaxChunks; c++)
+#pragma unroll
+            for (int j = 0; j < 4; j++) { s[c][j] = 0.f; ss[c][j] = 0.f; }
+    }
+};
+
+__device__ __forceinline__ float4 ldcg4(const float *p) { return __ldcg(reinterpret_cast<const float4 *>(p)); }
+
+// One tile: 128 epilogue threads (etid 0..127; thread etid owns accumulator lane etid), BN
+// accumulator columns starting at tensor-memory address tmem_acc; col0 = first output channel of
+// this N tile.  row_pix[128] and stage live in shared memory.  acc_empty is arrived on by every
+// thread once the accumulator has been read.
+__device__ __forceinline__ void epilogue_tile(const EpiArgs &e, uint32_t tmem_acc, int BN, int col0, const int *row_pix,
+                                              float *stage, EpiAcc &acc, int etid, uint64_t *acc_empty) {
+    const uint32_t lane_base = (uint32_t)((etid >> 5) * 32) << 16;
+#pragma unroll
+    for (int ch = 0; ch < kEpiMaxChunks; ch++) {
+        const int cc = ch * kEpiChunk;
+        if (cc >= BN) break;
+        const int cw = BN - cc < kEpiChunk ? BN - cc : kEpiChunk;
+        // phase 1: accumulator row -> staged row
+        for (int c = 0; c < cw; c += 16) {
+            float v[16];
+            tmem_ld16(tmem_acc + lane_base + (uint32_t)(cc + c), v);
+            float4 *dst = reinterpret_cast<float4 *>(stage + etid * kEpiPitch + c);
+            dst[0] = make_float4(v[0], v[1], v[2], v[3]); dst[1] = make_float4(v[4], v[5], v[6], v[7]);
+            dst[2] = make_float4(v[8], v[9], v[10], v[11]); dst[3] = make_float4(v[12], v[13], v[14], v[15]);
+        }
+        if (cc + cw >= BN) { tc_fence_before(); mbar_arrive(acc_empty); }
+        named_barrier(1, 128);
+        // phase 2: thread = (row r0 of each pass, channel quad); consecutive threads touch consecutive addresses
+        const int QW = cw >> 2, rpp = 128 / QW;
+        const int quad = etid % QW, r0 = etid / QW;
+        const int col = col0 + cc + quad * 4;
+        if (r0 < rpp && col < e.n_cols) {
+            float4 sc = make_float4(0, 0, 0, 0), sh = sc, mu = sc, rs = sc;
+            if (e.mode == EPI_BNBWD) bn_coef4(e.bn, col, sc, sh, mu, rs);
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f, q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
+            for (int rb = r0; rb < 128; rb += 4 * rpp) {
+                int pix[4]; float4 aux[4];
+                // loads of the partner / BN input first: they may alias the stores below
+#pragma unroll
+                for (int i = 0; i < 4; i++) {
+                    const int row = rb + i * rpp;
+                    pix[i] = row < 128 ? row_pix[row] : -1;
+                    if (pix[i] >= 0) {
+                        if (e.mode == EPI_COUPLE) aux[i] = *reinterpret_cast<const float4 *>(e.partner.at((size_t)pix[i], col));
+                        else if (e.mode == EPI_BNBWD) aux[i] = e.t.ld4((size_t)pix[i], col);
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < 4; i++) {
+                    if (pix[i] < 0) continue;
+                    const int row = rb + i * rpp;
+                    float4 v = *reinterpret_cast<const float4 *>(stage + row * kEpiPitch + quad * 4);
+                    if (e.mode == EPI_BNBWD) {
+                        *reinterpret_cast<float4 *>(e.out.at((size_t)pix[i], col)) = v;
+                        const float4 t = aux[i];
+                        const float dx = fmaf(sc.x, t.x, sh.x) > 0.f ? v.x : 0.f, dy = fmaf(sc.y, t.y, sh.y) > 0.f ? v.y : 0.f;
+                        const float dz = fmaf(sc.z, t.z, sh.z) > 0.f ? v.z : 0.f, dw = fmaf(sc.w, t.w, sh.w) > 0.f ? v.w : 0.f;
+                        s0 += dx; s1 += dy; s2 += dz; s3 += dw;
+                        q0 += dx * ((t.x - mu.x) * rs.x); q1 += dy * ((t.y - mu.y) * rs.y);
+                        q2 += dz * ((t.z - mu.z) * rs.z); q3 += dw * ((t.w - mu.w) * rs.w);
+                    } else {
+                        if (e.mode == EPI_COUPLE) v = e.out.couple4_with((size_t)pix[i], col, v, aux[i], e.sign);
+                        else v = e.out.store4((size_t)pix[i], col, v);
+                        s0 += v.x; s1 += v.y; s2 += v.z; s3 += v.w;
+                        q0 += v.x * v.x; q1 += v.y * v.y; q2 += v.z * v.z; q3 += v.w * v.w;
+                    }
+                }
+            }
+            acc.s[ch][0] += s0; acc.s[ch][1] += s1; acc.s[ch][2] += s2; acc.s[ch][3] += s3;
+            acc.ss[ch][0] += q0; acc.ss[ch][1] += q1; acc.ss[ch][2] += q2; acc.ss[ch][3] += q3;
+        }
+        named_barrier(1, 128);
+    }
+}
+
+// After the last tile: per-CTA partials, grid-wide count, and the finalize by the CTA that comes last.
+// scratch: >= 8 KB of shared memory (the stage).
+__device__ __forceinline__ void epilogue_finish(const EpiArgs &e, int BN, int col0, float *scratch, const EpiAcc &acc, int etid) {
+    if (!e.part) return;
+    float *mine = e.part + (size_t)blockIdx.x * 2 * e.n_cols;
+#pragma unroll
+    for (int ch = 0; ch < kEpiMaxChunks; ch++) {
+        const int cc = ch * kEpiChunk;
+        if (cc >= BN) break;
+        const int cw = BN - cc < kEpiChunk ? BN - cc : kEpiChunk;
+        const int QW = cw >> 2, rpp = 128 / QW;
+        const int quad = etid % QW, r0 = etid / QW;
+#pragma unroll
+        for (int j = 0; j < 4; j++) { scratch[etid * 8 + j] = acc.s[ch][j]; scratch[etid * 8 + 4 + j] = acc.ss[ch][j]; }
+        named_barrier(1, 128);
+        const int col = col0 + cc + quad * 4;
+        if (r0 == 0 && col < e.n_cols) {
+            float r[8];
+#pragma unroll
+            for (int j = 0; j < 8; j++) r[j] = scratch[quad * 8 + j];
+            for (int y = 1; y < rpp; y++)
+#pragma unroll
+                for (int j = 0; j < 8; j++) r[j] += scratch[(y * QW + quad) * 8 + j];
+            *reinterpret_cast<float4 *>(mine + 2 * col) = make_float4(r[0], r[1], r[2], r[3]);
+            *reinterpret_cast<float4 *>(mine + 2 * col + 4) = make_float4(r[4], r[5], r[6], r[7]);
+        }
+        named_barrier(1, 128);
+    }
+    // publish, count, and let the last CTA of the grid reduce
+    __threadfence();
+    named_barrier(1, 128);
+    unsigned int *flag = reinterpret_cast<unsigned int *>(scratch);
+    if (etid == 0) {
+        const unsigned int total = gridDim.x * gridDim.y;
+        const unsigned int old = atomicAdd(e.counter, 1u);
+        *flag = (old == total - 1) ? 1u : 0u;
+    }
+    named_barrier(1, 128);
+    const bool last = *flag != 0;
+    named_barrier(1, 128);
+    if (!last) return;
+    __threadfence();
+    // A partial is a record of 2C floats = R float4 slots (per channel quad: sums, second sums).
+    // Thread = (slot, sub): it adds the records sub, sub + nsub, ... of its slot, eight loads in
+    // flight at a time; the subs are then added in order.  All in double precision, all in an
+    // order the launch shape fixes.
+    const int C = e.n_cols, parts = (int)gridDim.x, R = C >> 1;
+    double *red = reinterpret_cast<double *>(scratch);            // [128][4]
+    double *tot = red + 512;                                      // [128][4]
+    for (int slot0 = 0; slot0 < R; slot0 += 128) {
+        const int cw = R - slot0 < 128 ? R - slot0 : 128;         // even
+        const int nsub = 128 / cw;
+        const int r = etid % cw, sub = etid / cw;
+        if (sub < nsub) {
+            double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+            const float *src = e.part + (size_t)(slot0 + r) * 4;
+            for (int i = sub; i < parts; i += 8 * nsub) {
+                float4 v[8];
+#pragma unroll
+                for (int k = 0; k < 8; k++) {
+                    const int idx = i + k * nsub;
+                    v[k] = idx < parts ? ldcg4(src + (size_t)idx * 2 * C) : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+                for (int k = 0; k < 8; k++) { s0 += (double)v[k].x; s1 += (double)v[k].y; s2 += (double)v[k].z; s3 += (double)v[k].w; }
+            }
+            red[etid * 4] = s0; red[etid * 4 + 1] = s1; red[etid * 4 + 2] = s2; red[etid * 4 + 3] = s3;
+        }
+        named_barrier(1, 128);
+        if (etid < cw) {
+            double s0 = red[etid * 4], s1 = red[etid * 4 + 1], s2 = red[etid * 4 + 2], s3 = red[etid * 4 + 3];
+            for (int y = 1; y < nsub; y++) {
+                const double *o = red + (y * cw + etid) * 4;
+                s0 += o[0]; s1 += o[1]; s2 += o[2]; s3 += o[3];
+            }
+            double *d = tot + etid * 4;
+            d[0] = s0; d[1] = s1; d[2] = s2; d[3] = s3;
+        }
+        named_barrier(1, 128);
+        for (int lc = etid; lc < cw * 2; lc += 128) {             // one thread per channel of this slot range
+            const int k = lc >> 2, j = lc & 3;                    // local quad, lane within it
+            const int ch = (slot0 >> 1) * 4 + lc;
+            const double sum = tot[(2 * k) * 4 + j], sum2 = tot[(2 * k + 1) * 4 + j];
+            if (e.mode == EPI_BNBWD) {
+                e.dbeta[ch] = (float)sum; e.dgamma[ch] = (float)sum2;
+                const double gr = (double)e.bn.gamma[ch] * (double)e.bn.rstd[ch];
+                e.coef[ch] = (float)gr; e.coef[C + ch] = (float)(gr * sum * e.inv_count); e.coef[2 * C + ch] = (float)(gr * sum2 * e.inv_count);
+            } else {
+                const double m = sum * e.inv_count;
+                double var = sum2 * e.inv_count - m * m;
+                if (var < 0) var = 0;
+                e.mean[ch] = (float)m; e.rstd[ch] = (float)(1.0 / sqrt(var + (double)e.eps));
+            }
+        }
+        named_barrier(1, 128);
+    }
+    if (etid == 0) *e.counter = 0u;
+}
+
+}  // namespace tc

@@ -15,13 +15,17 @@
 // (out = partner +/- acc on the float or fixed-point state) and store.
 // Every mbarrier wait is bounded; on expiry the kernel records a status word and leaves.
 #include "common.cuh"
+#include "tc_ptx.cuh"
+#include "conv_epilogue.cuh"
 #include <cuda.h>
+#include <string.h>
+
+using namespace tc;
 
 namespace {
 
 constexpr int kStages = 4;
 constexpr int kThreads = 192;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s: far beyond any real wait of this kernel
 
 struct TcParams {
     int taps;        // k*k
@@ -30,214 +34,130 @@ struct TcParams {
     int KC;          // channels per chunk (16, 32 or 64)
     int cin_pad;     // chunks * KC
     int BN;          // N tile
-    int n_cols;      // valid output channels
-    int H, W;        // output image size
     int stride;      // 1 or 2: input pixel = output pixel * stride + tap - pad (TMA traversal stride)
-    int BH, BIMG;    // tile: BH rows x W columns x BIMG images = 128 pixels
-    Pair out, partner;
-    int sign;
+    TileGeom g;      // output tiles
+    EpiArgs epi;
     int *status;
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t *bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-// bounded wait: false when the limit ran out
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
-    const uint32_t addr = smem_u32(bar);
-    unsigned long long t0 = 0;
-    for (uint32_t it = 0;; it++) {
-        uint32_t done;
-        asm volatile(
-            "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-            "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
-        if (done) return true;
-        if ((it & 63) == 63) {
-            unsigned long long now;
-            asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) return false;
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_4d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1, int c2, int c3) {
-    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
-                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
-}
-__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, uint64_t *bar, int c0, int c1) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-                 ::"r"(smem_u32(dst)), "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
-}
-
-// shared-memory matrix descriptor, K-major operand whose rows are `row_bytes` (32/64/128) long and
-// stored with the matching TMA swizzle; 8-row groups are row_bytes*8 apart
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, int row_bytes) {
-    const uint64_t layout = row_bytes == 128 ? 2 : (row_bytes == 64 ? 4 : 6);
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3FFFF) >> 4);                 // start address
-    d |= (uint64_t)1 << 16;                                 // leading byte offset (unused for swizzled K-major)
-    d |= (uint64_t)((row_bytes * 8) >> 4) << 32;            // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;                                 // descriptor version
-    d |= layout << 61;
-    return d;
-}
-
-// instruction descriptor: bf16 x bf16 -> fp32, M = 128; mn_major: both operands have their M / N
-// index contiguous in shared memory (pixel-major tiles of the weight-gradient GEMM), else K-major
-__device__ __forceinline__ uint32_t instr_desc(int n, bool mn_major = false) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | (mn_major ? (3u << 15) : 0u) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-}
-
-// descriptor of an MN-major operand: rows are K indices, each row holds `row_bytes` (32/64/128) of
-// contiguous M (or N) elements with the matching swizzle; the next block of M / N elements starts
-// `block_bytes` further on, groups of 8 K-rows are row_bytes*8 apart
-__device__ __forceinline__ uint64_t smem_desc_mn(uint32_t addr, int row_bytes, int block_bytes) {
-    const uint64_t layout = row_bytes == 128 ? 2 : (row_bytes == 64 ? 4 : 6);
-    uint64_t d = 0;
-    d |= (uint64_t)((addr & 0x3FFFF) >> 4);
-    d |= (uint64_t)((block_bytes >> 4) & 0x3FFF) << 16;     // leading byte offset: between M / N blocks
-    d |= (uint64_t)((row_bytes * 8) >> 4) << 32;            // stride byte offset: between 8-row K groups
-    d |= (uint64_t)1 << 46;
-    d |= layout << 61;
-    return d;
-}
-
-__device__ __forceinline__ void mma_bf16(uint32_t tmem_d, uint64_t da, uint64_t db, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(da), "l"(db), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void mma_commit(uint64_t *bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float *v) {
-    uint32_t r[16];
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
-        : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-#pragma unroll
-    for (int i = 0; i < 16; i++) v[i] = __uint_as_float(r[i]);
-}
 
 struct __align__(8) TcShared {
     uint64_t full[kStages];
     uint64_t empty[kStages];
-    uint64_t acc_full;
+    uint64_t acc_full[2];
+    uint64_t acc_empty[2];
     uint32_t tmem_base;
     uint32_t failed;
+    int row_pix[128];
 };
 
+// Persistent CTA: walks the pixel tiles blockIdx.x, blockIdx.x + gridDim.x, ... of N tile blockIdx.y.
+// The operand ring runs on across tiles; the accumulator alternates between two tensor-memory
+// buffers so that the epilogue of one tile overlaps the MMAs of the next.
 __global__ void __launch_bounds__(kThreads, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
-    // operand stages first (1024-byte aligned for the 128-byte swizzle), bookkeeping behind them
+    // operand stages first (1024-byte aligned for the 128-byte swizzle), epilogue stage and bookkeeping behind them
     uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const int a_bytes = 128 * p.KC * 2, b_bytes = p.BN * p.KC * 2;
-    const int b_off = (a_bytes + 1023) & ~1023;
+    const int box_px = p.g.BIMG * p.g.BH * p.g.W;
+    const int a_bytes = box_px * p.KC * 2, b_bytes = p.BN * p.KC * 2;
+    const int b_off = (128 * p.KC * 2 + 1023) & ~1023;
     const int stage_bytes = b_off + ((b_bytes + 1023) & ~1023);
-    TcShared *sh = (TcShared *)(tiles + kStages * stage_bytes);
+    float *estage = (float *)(tiles + kStages * stage_bytes);
+    TcShared *sh = (TcShared *)((uint8_t *)estage + kEpiStageBytes);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int iters = p.taps * p.chunks;
     uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < p.BN) tmem_cols <<= 1;
+    while ((int)tmem_cols < 2 * p.BN) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; s++) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
-        mbar_init(&sh->acc_full, 1);
+        for (int b = 0; b < 2; b++) { mbar_init(&sh->acc_full[b], 1); mbar_init(&sh->acc_empty[b], 128); }
         sh->failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tma_prefetch_desc(&map_a); tma_prefetch_desc(&map_b);
     }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(tmem_cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    if (warp == 1) tmem_alloc(&sh->tmem_base, tmem_cols);
+    tc_fence_before();
     __syncthreads();
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    tc_fence_after();
     const uint32_t tmem_d = sh->tmem_base;
-
-    // tile origin: tiles are runs of 128 consecutive pixels in (n, h, w) order
-    const int tiles_per_img = p.BIMG > 1 ? 1 : p.H / p.BH;
-    const int n0 = p.BIMG > 1 ? blockIdx.x * p.BIMG : blockIdx.x / tiles_per_img;
-    const int h0 = p.BIMG > 1 ? 0 : (blockIdx.x % tiles_per_img) * p.BH;
     const int col0 = blockIdx.y * p.BN;
     const int pad = p.k / 2;
 
     if (warp == 0) {
         if (lane == 0) {
-            for (int it = 0; it < iters; it++) {
-                const int s = it % kStages, round = it / kStages;
-                if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); break; }
-                const int tap = it / p.chunks, ch = it - tap * p.chunks;
-                const int kh = tap / p.k, kw = tap - kh * p.k;
-                uint8_t *sa = tiles + s * stage_bytes;
-                mbar_expect_tx(&sh->full[s], (uint32_t)(a_bytes + b_bytes));
-                tma_load_4d(sa, &map_a, &sh->full[s], ch * p.KC, kw - pad, h0 * p.stride + kh - pad, n0);
-                tma_load_2d(sa + b_off, &map_b, &sh->full[s], tap * p.cin_pad + ch * p.KC, col0);
+            uint32_t itg = 0;
+            bool ok = true;
+            for (int t = blockIdx.x; t < p.g.n_px_tiles && ok; t += gridDim.x) {
+                int n0, h0;
+                tile_origin(p.g, t, n0, h0);
+                for (int it = 0; it < iters; it++, itg++) {
+                    const int s = itg % kStages; const uint32_t round = itg / kStages;
+                    if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
+                    const int tap = it / p.chunks, ch = it - tap * p.chunks;
+                    const int kh = tap / p.k, kw = tap - kh * p.k;
+                    uint8_t *sa = tiles + s * stage_bytes;
+                    mbar_expect_tx(&sh->full[s], (uint32_t)(a_bytes + b_bytes));
+                    tma_load_4d(sa, &map_a, &sh->full[s], ch * p.KC, kw - pad, h0 * p.stride + kh - pad, n0);
+                    tma_load_2d(sa + b_off, &map_b, &sh->full[s], tap * p.cin_pad + ch * p.KC, col0);
+                }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = instr_desc(p.BN);
             const int row_bytes = p.KC * 2;
+            uint32_t itg = 0;
             bool ok = true;
-            for (int it = 0; it < iters && ok; it++) {
-                const int s = it % kStages, round = it / kStages;
-                if (!mbar_wait(&sh->full[s], round & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
-                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t sa = smem_u32(tiles + s * stage_bytes);
-                for (int kk = 0; kk < p.KC / 16; kk++) {
-                    const uint64_t da = smem_desc(sa + kk * 32, row_bytes);
-                    const uint64_t db = smem_desc(sa + b_off + kk * 32, row_bytes);
-                    mma_bf16(tmem_d, da, db, idesc, (it > 0 || kk > 0) ? 1u : 0u);
+            int ti = 0;
+            for (int t = blockIdx.x; t < p.g.n_px_tiles && ok; t += gridDim.x, ti++) {
+                const int buf = ti & 1; const uint32_t use = ti >> 1;
+                if (use > 0 && !mbar_wait(&sh->acc_empty[buf], (use - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
+                tc_fence_after();
+                const uint32_t acc = tmem_d + (uint32_t)(buf * p.BN);
+                for (int it = 0; it < iters; it++, itg++) {
+                    const int s = itg % kStages; const uint32_t round = itg / kStages;
+                    if (!mbar_wait(&sh->full[s], round & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(tiles + s * stage_bytes);
+                    for (int kk = 0; kk < p.KC / 16; kk++) {
+                        const uint64_t da = smem_desc(sa + kk * 32, row_bytes);
+                        const uint64_t db = smem_desc(sa + b_off + kk * 32, row_bytes);
+                        mma_bf16(acc, da, db, idesc, (it > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    mma_commit(&sh->empty[s]);          // frees the stage once these MMAs have read it
                 }
-                mma_commit(&sh->empty[s]);          // frees the stage once these MMAs have read it
+                if (ok) mma_commit(&sh->acc_full[buf]);
             }
-            mma_commit(&sh->acc_full);              // accumulator complete (also issued after a failure, so nobody waits forever)
         }
     } else {
-        // epilogue: warp w owns accumulator lanes 32*(w%4) .. +31 = pixel rows of the tile
-        const int quarter = warp & 3;
-        const bool ok = mbar_wait(&sh->acc_full, 0);
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        if (ok && sh->failed == 0) {
-            const size_t row = (size_t)blockIdx.x * 128 + quarter * 32 + lane;
-            for (int c = 0; c < p.BN; c += 16) {
-                float v[16];
-                tmem_ld16(tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, v);
-#pragma unroll
-                for (int j = 0; j < 16; j += 4) {
-                    const int col = col0 + c + j;
-                    if (col < p.n_cols) p.out.couple4(row, col, make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]), p.partner, p.sign);
-                }
-            }
-        } else if (lane == 0) {
-            atomicExch(&sh->failed, 1u);
+        // epilogue: this warp may touch accumulator lanes 32*(warp%4) .. +31
+        const int etid = ((warp & 3) << 5) | lane;
+        EpiAcc acc;
+        acc.clear();
+        bool ok = true;
+        int ti = 0;
+        for (int t = blockIdx.x; t < p.g.n_px_tiles; t += gridDim.x, ti++) {
+            const int buf = ti & 1; const uint32_t use = ti >> 1;
+            int n0, h0;
+            tile_origin(p.g, t, n0, h0);
+            sh->row_pix[etid] = tile_row_pixel(p.g, n0, h0, etid);
+            ok = mbar_wait(&sh->acc_full[buf], use & 1) && sh->failed == 0;
+            ok = named_barrier_and(2, 128, ok);       // also publishes row_pix
+            if (!ok) break;
+            tc_fence_after();
+            epilogue_tile(p.epi, tmem_d + (uint32_t)(buf * p.BN), p.BN, col0, sh->row_pix, estage, acc, etid, &sh->acc_empty[buf]);
         }
+        if (ok) epilogue_finish(p.epi, p.BN, col0, estage, acc, etid);
+        else if (lane == 0) atomicExch(&sh->failed, 1u);
     }
-    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && sh->failed) atomicExch(p.status, (int)REVNET_E_TIMEOUT);
     if (warp == 1) {
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(tmem_cols) : "memory");
+        tc_fence_after();
+        tmem_dealloc(tmem_d, tmem_cols);
     }
 }
 
@@ -291,16 +211,27 @@ EncodeTiledFn encoder(revnet_ctx *ctx) {
 
 int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
-struct TcShape { int KC, cin_pad, chunks, BN, n_tiles, BH, BIMG, smem; };
+// 128-row tiles over an output of N x H x W pixels: whole rows of one image (the last tile of an
+// image may be ragged), or whole images when an image has at most 64 pixels.  Rows of the tile
+// that fall outside are padding: TMA fills their operand rows with zeros and the epilogue skips them.
+bool tile_geom(Geom g, TileGeom &t) {
+    if (g.W > 128 || g.W < 1) return false;
+    t.N = g.N; t.H = g.H; t.W = g.W; t.hw_order = 0;
+    t.BH = 128 / g.W; if (t.BH > g.H) t.BH = g.H;
+    t.BIMG = 1;
+    if (t.BH == g.H) { t.BIMG = 128 / (g.H * g.W); if (t.BIMG > g.N) t.BIMG = g.N; if (t.BIMG < 1) t.BIMG = 1; }
+    t.tiles_per_img = (g.H + t.BH - 1) / t.BH;
+    t.n_px_tiles = t.BIMG > 1 ? (g.N + t.BIMG - 1) / t.BIMG : g.N * t.tiles_per_img;
+    return true;
+}
 
-// Which shapes the kernel takes: stride 1 or 2, k in {1,3}; a 128-pixel output tile must be whole rows of one
-// image or whole images; channel rows 16-byte aligned for TMA.
+struct TcShape { int KC, cin_pad, chunks, BN, n_tiles, smem; TileGeom g; };
+
+// Which shapes the kernel takes: stride 1 or 2, k in {1,3}, channel rows 16-byte aligned for TMA.
 bool tc_shape(Geom g, int cin, int cout, int k, int stride, TcShape &s) {   // g: output geometry
     if ((stride != 1 && stride != 2) || (k != 1 && k != 3) || cin % 8 || cout % 4) return false;
-    const int W = g.W, H = g.H;
-    if (W > 128 || 128 % W) return false;
-    if (H * W >= 128) { if (H % (128 / W)) return false; s.BH = 128 / W; s.BIMG = 1; }
-    else { if (128 % (H * W) || g.N % (128 / (H * W))) return false; s.BH = H; s.BIMG = 128 / (H * W); }
+    if (!tile_geom(g, s.g)) return false;
+    if (s.g.W * stride > 256 || s.g.BH * stride > 256) return false;
     s.cin_pad = round_up(cin, 16);
     s.KC = s.cin_pad % 64 == 0 ? 64 : (s.cin_pad % 32 == 0 ? 32 : 16);
     s.chunks = s.cin_pad / s.KC;
@@ -308,24 +239,35 @@ bool tc_shape(Geom g, int cin, int cout, int k, int stride, TcShape &s) {   // g
     s.BN = cout_pad <= 128 ? cout_pad : 128;
     s.n_tiles = (cout_pad + s.BN - 1) / s.BN;
     const int a_bytes = 128 * s.KC * 2, b_bytes = s.BN * s.KC * 2;
-    s.smem = 1024 + kStages * (((a_bytes + 1023) & ~1023) + ((b_bytes + 1023) & ~1023)) + (int)sizeof(TcShared) + 64;
+    s.smem = 1024 + kStages * (((a_bytes + 1023) & ~1023) + ((b_bytes + 1023) & ~1023)) + kEpiStageBytes + (int)sizeof(TcShared) + 64;
     return true;
 }
 
+// Reductions a convolution epilogue is asked to fuse.
+struct EpiReq {
+    Moments *stats = nullptr;          // statistics of the stored result
+    const BnBwdReq *bnbwd = nullptr;   // data gradient: sums of the BN+ReLU backward
+};
+
 // act: bf16 [N,H,W,cin]; Wsrc: fp32 weights; transposed selects the dgrad pack
 bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin, int cout, int k, int stride,
-                 const float *Wsrc, const bf16 *prepacked, bool transposed, Pair out, Pair partner, int sign) {
+                 const float *Wsrc, const bf16 *prepacked, bool transposed, Pair out, Pair partner, int sign, EpiReq req) {
     TcShape s;
     if (stride == 2 && (gin.H % 2 || gin.W % 2)) return false;
     const Geom g{gin.N, conv_out(gin.H, k, stride), conv_out(gin.W, k, stride)};   // output geometry
     if (!tc_shape(g, cin, cout, k, stride, s)) return false;
-    const int taps = k * k, cout_pad = round_up(cout, 16);
+    const int taps = k * k;
     const int rows_pad = s.n_tiles * s.BN;
     if (!ex.dry && !encoder(ex.ctx)) return false;
     ex.flops += 2ull * g.P() * cout * cin * taps;
+    int occ = (227 * 1024) / s.smem; if (occ > 2) occ = 2; if (occ < 1) occ = 1;
+    int ctas = ex.ctx->sm_count * occ / s.n_tiles; if (ctas < 1) ctas = 1;
+    if (ctas > s.g.n_px_tiles) ctas = s.g.n_px_tiles;
     size_t m = ex.ws.mark();
     bf16 *wp = prepacked ? const_cast<bf16 *>(prepacked) : ex.ws.get<bf16>((size_t)rows_pad * taps * s.cin_pad);
-    (void)cout_pad;
+    const bool reduce = req.stats || req.bnbwd;
+    float *part = reduce ? ex.ws.get<float>((size_t)ctas * 2 * cout) : nullptr;
+    if (req.stats) req.stats->valid = true;
     if (!ex.dry) {
         EncodeTiledFn enc = encoder(ex.ctx);
         // without a pack made earlier in the step, build it from the fp32 master weights now
@@ -342,7 +284,7 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
             // the box spans stride x the tile in the input image and is walked with that stride
             cuuint64_t dims[4] = {(cuuint64_t)cin, (cuuint64_t)gin.W, (cuuint64_t)gin.H, (cuuint64_t)gin.N};
             cuuint64_t strides[3] = {(cuuint64_t)cin * 2, (cuuint64_t)gin.W * cin * 2, (cuuint64_t)gin.H * gin.W * cin * 2};
-            cuuint32_t box[4] = {(cuuint32_t)s.KC, (cuuint32_t)(g.W * stride), (cuuint32_t)(s.BH * stride), (cuuint32_t)s.BIMG};
+            cuuint32_t box[4] = {(cuuint32_t)s.KC, (cuuint32_t)(g.W * stride), (cuuint32_t)(s.g.BH * stride), (cuuint32_t)s.g.BIMG};
             cuuint32_t es[4] = {1, (cuuint32_t)stride, (cuuint32_t)stride, 1};
             CUresult r = enc(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void *)act, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                              sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -358,13 +300,21 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
             if (r != CUDA_SUCCESS) { ex.failed = true; ex.ctx->err = std::string(what) + ": tensor map (weights) rejected"; ex.ws.release(m); return true; }
         }
         TcParams p;
-        p.taps = taps; p.k = k; p.chunks = s.chunks; p.KC = s.KC; p.cin_pad = s.cin_pad; p.BN = s.BN; p.n_cols = cout;
-        p.H = g.H; p.W = g.W; p.stride = stride; p.BH = s.BH; p.BIMG = s.BIMG; p.out = out; p.partner = partner; p.sign = sign; p.status = ex.ctx->dev_status;
+        p.taps = taps; p.k = k; p.chunks = s.chunks; p.KC = s.KC; p.cin_pad = s.cin_pad; p.BN = s.BN; p.stride = stride; p.g = s.g;
+        p.status = ex.ctx->dev_status;
+        EpiArgs &e = p.epi;
+        memset(&e, 0, sizeof e);
+        e.mode = req.bnbwd ? EPI_BNBWD : (sign ? EPI_COUPLE : EPI_PLAIN);
+        e.out = out; e.partner = partner; e.sign = sign; e.n_cols = cout;
+        e.part = part; e.counter = reduce ? ex.ctx->counter() : nullptr;
+        e.inv_count = 1.0 / (double)g.P(); e.eps = ex.eps;
+        if (req.stats) { e.mean = req.stats->mean; e.rstd = req.stats->rstd; }
+        if (req.bnbwd) { e.t = req.bnbwd->t; e.bn = req.bnbwd->bn; e.dgamma = req.bnbwd->dgamma; e.dbeta = req.bnbwd->dbeta; e.coef = req.bnbwd->coef; }
         static bool attr_set = false;
-        if (!attr_set) { cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); attr_set = true; }
-        dim3 grid((unsigned)(g.P() / 128), (unsigned)s.n_tiles);
+        if (!attr_set) { cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024); attr_set = true; }
+        dim3 grid((unsigned)ctas, (unsigned)s.n_tiles);
         conv_tc_kernel<<<grid, kThreads, s.smem, ex.stream>>>(map_a, map_b, p);
-        const double bytes = (double)gin.P() * cin * 2 + (double)g.P() * cout * (sign ? 8 : 4) + (double)cout * taps * cin * 2;
+        const double bytes = (double)gin.P() * cin * 2 + (double)g.P() * cout * (sign || req.bnbwd ? 8 : 4) + (double)cout * taps * cin * 2;
         ex.check(what, bytes, 2.0 * g.P() * cout * cin * taps);
     }
     ex.ws.release(m);
@@ -416,14 +366,11 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.stages; s++) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
-        mbar_init(&sh->acc_full, 1);
+        mbar_init(&sh->acc_full[0], 1);
         sh->failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)), "r"(tmem_cols) : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
+    if (warp == 1) tmem_alloc(&sh->tmem_base, tmem_cols);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -468,11 +415,11 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     }
                 mma_commit(&sh->empty[s]);
             }
-            mma_commit(&sh->acc_full);
+            mma_commit(&sh->acc_full[0]);
         }
     } else {
         const int quarter = warp & 3;
-        const bool ok = mbar_wait(&sh->acc_full, 0);
+        const bool ok = mbar_wait(&sh->acc_full[0], 0);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (ok && sh->failed == 0) {
             const int m = quarter * 32 + lane;
@@ -546,14 +493,16 @@ bool encode_act_map(Exec &ex, CUtensorMap *map, const void *base, Geom g, int C,
 
 }  // namespace
 
-bool conv_fprop_tc(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign) {
-    return run_conv_tc(ex, "conv_fprop_tc", a, gi, L.cin, L.cout, L.k, L.stride, L.W, L.Wp_fprop, false, out, partner, sign);
+bool conv_fprop_tc(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign, Moments *stats) {
+    EpiReq req; req.stats = stats;
+    return run_conv_tc(ex, "conv_fprop_tc", a, gi, L.cin, L.cout, L.k, L.stride, L.W, L.Wp_fprop, false, out, partner, sign, req);
 }
 
 // da[q,ci] = sum_{tap,co} g[q (-) tap, co] W[co,tap,ci]: a stride-1 convolution of g with the mirrored, transposed weights
-bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da) {
+bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, const BnBwdReq *bb) {
     if (L.stride != 1) return false;
-    return run_conv_tc(ex, "conv_dgrad_tc", g, gi, L.cout, L.cin, L.k, L.stride, L.W, L.Wp_dgrad, true, single(da, L.cin), Pair{}, 0);
+    EpiReq req; req.bnbwd = bb;
+    return run_conv_tc(ex, "conv_dgrad_tc", g, gi, L.cout, L.cin, L.k, L.stride, L.W, L.Wp_dgrad, true, single(da, L.cin), Pair{}, 0, req);
 }
 
 

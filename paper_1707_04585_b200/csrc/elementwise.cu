@@ -67,9 +67,7 @@ static RedShape red_shape(size_t P, int C, int sm) {
 
 // part layout: [chunk][2][C]
 template <int MODE>   // 0: sum t, sum t^2 ; 1: sum db, sum db*xhat (BN+ReLU backward)
-__global__ void col_reduce_kernel(Pair t, const float *__restrict__ da, size_t P, int rows_per_cta,
-                                  const float *__restrict__ scale, const float *__restrict__ shift,
-                                  const float *__restrict__ mean, const float *__restrict__ rstd,
+__global__ void col_reduce_kernel(Pair t, const float *__restrict__ da, size_t P, int rows_per_cta, BnRef bn,
                                   float *__restrict__ part) {
     extern __shared__ float4 sm4[];
     const int C = t.C(), C4 = C / 4, SW = blockDim.x, RPP = blockDim.y;
@@ -80,7 +78,7 @@ __global__ void col_reduce_kernel(Pair t, const float *__restrict__ da, size_t P
     float4 s = make_float4(0, 0, 0, 0), ss = s;
     if (valid) {
         float4 sc, sh, mu, rs;
-        if (MODE == 1) { sc = ld4(scale + q * 4); sh = ld4(shift + q * 4); mu = ld4(mean + q * 4); rs = ld4(rstd + q * 4); }
+        if (MODE == 1) bn_coef4(bn, q * 4, sc, sh, mu, rs);
         for (size_t r = r0 + threadIdx.y; r < r1; r += RPP) {
             float4 v = t.ld4(r, q * 4);
             if (MODE == 0) {
@@ -91,8 +89,8 @@ __global__ void col_reduce_kernel(Pair t, const float *__restrict__ da, size_t P
                 float dx = fmaf(sc.x, v.x, sh.x) > 0.f ? g.x : 0.f, dy = fmaf(sc.y, v.y, sh.y) > 0.f ? g.y : 0.f;
                 float dz = fmaf(sc.z, v.z, sh.z) > 0.f ? g.z : 0.f, dw = fmaf(sc.w, v.w, sh.w) > 0.f ? g.w : 0.f;
                 s.x += dx; s.y += dy; s.z += dz; s.w += dw;
-                ss.x += dx * (v.x - mu.x) * rs.x; ss.y += dy * (v.y - mu.y) * rs.y;
-                ss.z += dz * (v.z - mu.z) * rs.z; ss.w += dw * (v.w - mu.w) * rs.w;
+                ss.x += dx * ((v.x - mu.x) * rs.x); ss.y += dy * ((v.y - mu.y) * rs.y);
+                ss.z += dz * ((v.z - mu.z) * rs.z); ss.w += dw * ((v.w - mu.w) * rs.w);
             }
         }
     }
@@ -119,8 +117,7 @@ __device__ __forceinline__ void warp_sum2(const float *__restrict__ part, int ch
 }
 
 __global__ void bn_stats_finalize(const float *__restrict__ part, int chunks, int C, double invP, float eps,
-                                  const float *__restrict__ gamma, const float *__restrict__ beta,
-                                  float *scale, float *shift, float *mean, float *rstd) {
+                                  float *mean, float *rstd) {
     const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (c >= C) return;
     double s, ss;
@@ -128,9 +125,7 @@ __global__ void bn_stats_finalize(const float *__restrict__ part, int chunks, in
     if ((threadIdx.x & 31) == 0) {
         double mu = s * invP, var = ss * invP - mu * mu;
         if (var < 0) var = 0;
-        float r = (float)(1.0 / sqrt(var + (double)eps));
-        float sc = gamma[c] * r;
-        scale[c] = sc; shift[c] = beta[c] - (float)mu * sc; mean[c] = (float)mu; rstd[c] = r;
+        mean[c] = (float)mu; rstd[c] = (float)(1.0 / sqrt(var + (double)eps));
     }
 }
 
@@ -149,36 +144,34 @@ __global__ void bn_bwd_finalize(const float *__restrict__ part, int chunks, int 
     }
 }
 
-BnState bn_alloc(Exec &ex, int C) {
-    BnState st;
-    float *p = ex.ws.get<float>((size_t)4 * C);
-    st.scale = p; st.shift = p + C; st.mean = p + 2 * C; st.rstd = p + 3 * C;
-    return st;
+Moments mom_alloc(Exec &ex, int C) {
+    Moments m;
+    float *p = ex.ws.get<float>((size_t)2 * C);
+    m.mean = p; m.rstd = p + C;
+    return m;
 }
 
-void bn_stats(Exec &ex, Pair t, size_t P, const float *gamma, const float *beta, BnState st) {
+void bn_stats(Exec &ex, Pair t, size_t P, Moments mo) {
     const int C = t.C();
     RedShape r = red_shape(P, C, ex.ctx->sm_count);
     size_t m = ex.ws.mark();
     float *part = ex.ws.get<float>((size_t)r.chunks * 2 * C);
     if (!ex.dry) {
         dim3 grid(r.chunks, r.slabs), block(r.SW, r.RPP);
-        col_reduce_kernel<0><<<grid, block, (size_t)r.SW * r.RPP * 32, ex.stream>>>(t, nullptr, P, r.rows_per_cta,
-                                                                                 nullptr, nullptr, nullptr, nullptr, part);
+        col_reduce_kernel<0><<<grid, block, (size_t)r.SW * r.RPP * 32, ex.stream>>>(t, nullptr, P, r.rows_per_cta, BnRef{}, part);
         ex.check("bn_stats_partial", (double)P * C * 4);
-        bn_stats_finalize<<<cdiv((size_t)C * 32, 128), 128, 0, ex.stream>>>(part, r.chunks, C, 1.0 / (double)P, ex.eps, gamma, beta,
-                                                              st.scale, st.shift, st.mean, st.rstd);
+        bn_stats_finalize<<<cdiv((size_t)C * 32, 128), 128, 0, ex.stream>>>(part, r.chunks, C, 1.0 / (double)P, ex.eps, mo.mean, mo.rstd);
         ex.check("bn_stats_finalize");
     }
     ex.ws.release(m);
 }
 
 template <class TO>
-__global__ void bn_relu_apply_kernel(Pair t, size_t nquads, int C4, const float *__restrict__ scale,
-                                     const float *__restrict__ shift, TO *__restrict__ a) {
+__global__ void bn_relu_apply_kernel(Pair t, size_t nquads, int C4, BnRef bn, TO *__restrict__ a) {
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
         size_t row = i / C4; int q = (int)(i - row * C4);
-        float4 v = t.ld4(row, q * 4), sc = ld4(scale + q * 4), sh = ld4(shift + q * 4);
+        float4 v = t.ld4(row, q * 4), sc, sh, mu, rs;
+        bn_coef4(bn, q * 4, sc, sh, mu, rs);
         v.x = fmaxf(fmaf(sc.x, v.x, sh.x), 0.f); v.y = fmaxf(fmaf(sc.y, v.y, sh.y), 0.f);
         v.z = fmaxf(fmaf(sc.z, v.z, sh.z), 0.f); v.w = fmaxf(fmaf(sc.w, v.w, sh.w), 0.f);
         st4(a + i * 4, v);
@@ -190,26 +183,27 @@ static int ew_grid(size_t n, int sm) {
     return (int)(g < cap ? (g ? g : 1) : cap);
 }
 
-void bn_relu_apply(Exec &ex, Pair t, size_t P, BnState st, void *a, bool a_bf16) {
+void bn_relu_apply(Exec &ex, Pair t, size_t P, BnRef bn, void *a, bool a_bf16) {
     if (ex.dry) return;
     const int C4 = t.C() / 4; size_t nq = P * C4;
-    if (a_bf16) bn_relu_apply_kernel<bf16><<<ew_grid(nq, ex.ctx->sm_count), 256, 0, ex.stream>>>(t, nq, C4, st.scale, st.shift, (bf16 *)a);
-    else bn_relu_apply_kernel<float><<<ew_grid(nq, ex.ctx->sm_count), 256, 0, ex.stream>>>(t, nq, C4, st.scale, st.shift, (float *)a);
+    if (a_bf16) bn_relu_apply_kernel<bf16><<<ew_grid(nq, ex.ctx->sm_count), 256, 0, ex.stream>>>(t, nq, C4, bn, (bf16 *)a);
+    else bn_relu_apply_kernel<float><<<ew_grid(nq, ex.ctx->sm_count), 256, 0, ex.stream>>>(t, nq, C4, bn, (float *)a);
     ex.check("bn_relu_apply", (double)P * t.C() * (a_bf16 ? 6 : 8));
 }
 
 // dt = coef0*db - coef1 - coef2*xhat ; db = da*[scale*t+shift > 0]
 // OUT 0: out[P,C] = dt (float or bf16) ; 1: outp = dt (fp32 pair) ; 2: outp = add + dt
-template <class TO, int OUT>
-__global__ void bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, size_t nquads, int C4,
-                                         const float *__restrict__ scale, const float *__restrict__ shift,
-                                         const float *__restrict__ mean, const float *__restrict__ rstd,
-                                         const float *__restrict__ coef, TO *__restrict__ out, Pair add, Pair outp) {
+// CAST (OUT 1, 2): also write the result as one bf16 [P,C] tensor
+template <class TO, int OUT, bool CAST>
+__global__ void bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, size_t nquads, int C4, BnRef bn,
+                                         const float *__restrict__ coef, TO *__restrict__ out, Pair add, Pair outp,
+                                         bf16 *__restrict__ cast) {
     const int C = C4 * 4;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
         size_t row = i / C4; int q = (int)(i - row * C4), c = q * 4;
         float4 v = t.ld4(row, c), g = ld4(da + i * 4);
-        float4 sc = ld4(scale + c), sh = ld4(shift + c), mu = ld4(mean + c), rs = ld4(rstd + c);
+        float4 sc, sh, mu, rs;
+        bn_coef4(bn, c, sc, sh, mu, rs);
         float4 k0 = ld4(coef + c), k1 = ld4(coef + C + c), k2 = ld4(coef + 2 * C + c), o;
         o.x = k0.x * (fmaf(sc.x, v.x, sh.x) > 0.f ? g.x : 0.f) - k1.x - k2.x * ((v.x - mu.x) * rs.x);
         o.y = k0.y * (fmaf(sc.y, v.y, sh.y) > 0.f ? g.y : 0.f) - k1.y - k2.y * ((v.y - mu.y) * rs.y);
@@ -221,31 +215,36 @@ __global__ void bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, s
         }
         if (OUT == 0) st4(out + i * 4, o);
         else st4(outp.at(row, c), o);
+        if (CAST) st4(cast + i * 4, o);
     }
 }
 
-void bn_relu_bwd(Exec &ex, const float *da, Pair t, size_t P, BnState st, const float *gamma,
-                 float *dgamma, float *dbeta, void *out_single, bool out_bf16, Pair add, Pair out_pair) {
+void bn_relu_bwd(Exec &ex, const float *da, Pair t, size_t P, BnRef bn, float *dgamma, float *dbeta, float *coef,
+                 bool sums_done, void *out_single, bool out_bf16, Pair add, Pair out_pair, bf16 *out_cast) {
     const int C = t.C(), C4 = C / 4;
     RedShape r = red_shape(P, C, ex.ctx->sm_count);
     size_t m = ex.ws.mark();
-    float *part = ex.ws.get<float>((size_t)r.chunks * 2 * C);
-    float *coef = ex.ws.get<float>((size_t)3 * C);
+    float *part = sums_done ? nullptr : ex.ws.get<float>((size_t)r.chunks * 2 * C);
     if (!ex.dry) {
-        dim3 grid(r.chunks, r.slabs), block(r.SW, r.RPP);
-        col_reduce_kernel<1><<<grid, block, (size_t)r.SW * r.RPP * 32, ex.stream>>>(t, da, P, r.rows_per_cta, st.scale, st.shift,
-                                                                                 st.mean, st.rstd, part);
-        ex.check("bn_bwd_partial", (double)P * C * 8);
-        bn_bwd_finalize<<<cdiv((size_t)C * 32, 128), 128, 0, ex.stream>>>(part, r.chunks, C, 1.0 / (double)P, gamma, st.rstd, dgamma, dbeta, coef);
-        ex.check("bn_bwd_finalize");
+        if (!sums_done) {
+            dim3 grid(r.chunks, r.slabs), block(r.SW, r.RPP);
+            col_reduce_kernel<1><<<grid, block, (size_t)r.SW * r.RPP * 32, ex.stream>>>(t, da, P, r.rows_per_cta, bn, part);
+            ex.check("bn_bwd_partial", (double)P * C * 8);
+            bn_bwd_finalize<<<cdiv((size_t)C * 32, 128), 128, 0, ex.stream>>>(part, r.chunks, C, 1.0 / (double)P, bn.gamma, bn.rstd, dgamma, dbeta, coef);
+            ex.check("bn_bwd_finalize");
+        }
         size_t nq = P * C4; int g = ew_grid(nq, ex.ctx->sm_count);
-#define RV_ARGS da, t, nq, C4, st.scale, st.shift, st.mean, st.rstd, coef
-        if (out_pair.p0 && add.p0) bn_relu_bwd_apply_kernel<float, 2><<<g, 256, 0, ex.stream>>>(RV_ARGS, nullptr, add, out_pair);
-        else if (out_pair.p0) bn_relu_bwd_apply_kernel<float, 1><<<g, 256, 0, ex.stream>>>(RV_ARGS, nullptr, add, out_pair);
-        else if (out_bf16) bn_relu_bwd_apply_kernel<bf16, 0><<<g, 256, 0, ex.stream>>>(RV_ARGS, (bf16 *)out_single, add, out_pair);
-        else bn_relu_bwd_apply_kernel<float, 0><<<g, 256, 0, ex.stream>>>(RV_ARGS, (float *)out_single, add, out_pair);
+#define RV_ARGS da, t, nq, C4, bn, coef
+        if (out_pair.p0 && add.p0) {
+            if (out_cast) bn_relu_bwd_apply_kernel<float, 2, true><<<g, 256, 0, ex.stream>>>(RV_ARGS, nullptr, add, out_pair, out_cast);
+            else bn_relu_bwd_apply_kernel<float, 2, false><<<g, 256, 0, ex.stream>>>(RV_ARGS, nullptr, add, out_pair, nullptr);
+        } else if (out_pair.p0) {
+            if (out_cast) bn_relu_bwd_apply_kernel<float, 1, true><<<g, 256, 0, ex.stream>>>(RV_ARGS, nullptr, add, out_pair, out_cast);
+            else bn_relu_bwd_apply_kernel<float, 1, false><<<g, 256, 0, ex.stream>>>(RV_ARGS, nullptr, add, out_pair, nullptr);
+        } else if (out_bf16) bn_relu_bwd_apply_kernel<bf16, 0, false><<<g, 256, 0, ex.stream>>>(RV_ARGS, (bf16 *)out_single, add, out_pair, nullptr);
+        else bn_relu_bwd_apply_kernel<float, 0, false><<<g, 256, 0, ex.stream>>>(RV_ARGS, (float *)out_single, add, out_pair, nullptr);
 #undef RV_ARGS
-        ex.check("bn_relu_bwd_apply", (double)P * C * (out_pair.p0 ? (add.p0 ? 16 : 12) : (out_bf16 ? 10 : 12)));
+        ex.check("bn_relu_bwd_apply", (double)P * C * ((out_pair.p0 ? (add.p0 ? 16 : 12) : (out_bf16 ? 10 : 12)) + (out_cast ? 2 : 0)));
     }
     ex.ws.release(m);
 }

@@ -123,6 +123,26 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
     float *feat = ex.ws.get<float>((size_t)N * FC), *dfeat = ex.ws.get<float>((size_t)N * FC);
     float *logits = logits_out ? logits_out : ex.ws.get<float>((size_t)N * K);
     float *dlogits = ex.ws.get<float>((size_t)N * K);
+    // batch statistics handed from kernel to kernel: per stage those of the current (x1,x2) pair (one
+    // [2c] array each for mean and rstd, so that the pair reads as one tensor to a transition) and
+    // those of the stage's input x2, which the reversal of the first unit needs again
+    struct StageMom { Moments m1, m2, cat, in_cat, in2; };
+    std::vector<StageMom> sm(S);
+    bf16 *gcast = nullptr;          // bf16 copy of the gradient w.r.t. x2 / y2, handed from unit to unit
+    {
+        size_t cmax = 0;
+        for (int si = 0; si < S; si++) {
+            const StagePlan &s = pl->st[si];
+            float *b = ex.ws.get<float>((size_t)8 * s.c);
+            sm[si].cat.mean = b; sm[si].cat.rstd = b + 2 * s.c;
+            sm[si].m1.mean = b; sm[si].m1.rstd = b + 2 * s.c;
+            sm[si].m2.mean = b + s.c; sm[si].m2.rstd = b + 3 * s.c;
+            sm[si].in_cat.mean = b + 4 * s.c; sm[si].in_cat.rstd = b + 6 * s.c;
+            sm[si].in2.mean = b + 5 * s.c; sm[si].in2.rstd = b + 7 * s.c;
+            size_t e = (size_t)N * s.H * s.H * s.c; if (e > cmax) cmax = e;
+        }
+        if (ex.mode == 0) gcast = ex.ws.get<bf16>(cmax);
+    }
     float *recon = ex.ws.get<float>(REVNET_MAX_STAGES);
     if (recon_dev) *recon_dev = recon;
     if (d.verify_reconstruction) fill_zero(ex, recon, REVNET_MAX_STAGES * sizeof(float));
@@ -146,17 +166,23 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
         StagePlan &s = pl->st[si];
         float *x1 = actf(s.off_x1), *x2 = actf(s.off_x2);
         Geom g{N, s.H, s.H};
+        StageMom &mo = sm[si];
         if (s.has_trans) {
             std::vector<Layer> T{bind(s.trans, params, grads)};
-            fn_forward(ex, Geom{N, prevH, prevH}, prev, T, Pair{}, halves(x1, x2, s.c, q), 0, nullptr, false);
+            const Moments *min = si > 0 ? &sm[si - 1].cat : nullptr;
+            fn_forward(ex, Geom{N, prevH, prevH}, prev, min, T, Pair{}, halves(x1, x2, s.c, q), 0, &mo.in_cat, nullptr, false);
         }
+        mo.in2.valid = mo.in_cat.valid;
+        if (!mo.in2.valid) { bn_stats(ex, single(x2, s.c, q), g.P(), mo.in2); mo.in2.valid = true; }
         if (d.verify_reconstruction && !ex.dry) {
             size_t b = g.P() * s.c * sizeof(float);
             cudaMemcpyAsync(actf(s.off_v1), x1, b, cudaMemcpyDeviceToDevice, ex.stream);
             cudaMemcpyAsync(actf(s.off_v2), x2, b, cudaMemcpyDeviceToDevice, ex.stream);
         }
         for (int u = 0; u < s.units; u++)
-            block_forward(ex, g, s.c, bind(s.F[u], params, grads), bind(s.G[u], params, grads), x1, x2, x1, x2);
+            block_forward(ex, g, s.c, bind(s.F[u], params, grads), bind(s.G[u], params, grads), x1, x2, x1, x2,
+                          u == 0 ? &mo.in2 : &mo.m2, &mo.m1, &mo.m2);
+        mo.cat.valid = mo.m1.valid && mo.m2.valid;
         prev = halves(x1, x2, s.c, q);
         prevH = s.H;
     }
@@ -177,8 +203,10 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
         Geom g{N, s.H, s.H};
         size_t half = g.P() * s.c;
         float *d1 = gbuf[gi], *d2 = gbuf[gi] + half;
+        StageMom &mo = sm[si];
         for (int u = s.units - 1; u >= 0; u--)
-            block_backward(ex, g, s.c, bind(s.F[u], params, grads), bind(s.G[u], params, grads), x1, x2, d1, d2, x1, x2, d1, d2);
+            block_backward(ex, g, s.c, bind(s.F[u], params, grads), bind(s.G[u], params, grads), x1, x2, d1, d2, x1, x2, d1, d2,
+                           &mo.m1, &mo.m2, u == 0 ? &mo.in2 : nullptr, u == s.units - 1 ? nullptr : gcast, gcast);
         if (d.verify_reconstruction) {
             max_abs_diff(ex, x1, actf(s.off_v1), half, q, recon + si);
             max_abs_diff(ex, x2, actf(s.off_v2), half, q, recon + si);
@@ -197,8 +225,9 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
             }
             FnSaved sv;
             size_t m = ex.ws.mark();
-            fn_forward(ex, Geom{N, tH, tH}, tin, T, Pair{}, Pair{}, 0, &sv, true);   // rebuild the operands from the stored input
-            fn_backward(ex, Geom{N, tH, tH}, tin, T, sv, halves(d1, d2, s.c), Pair{}, gout);
+            // rebuild the operands from the stored input (the stage in front still holds its forward statistics)
+            fn_forward(ex, Geom{N, tH, tH}, tin, si > 0 ? &sm[si - 1].cat : nullptr, T, Pair{}, Pair{}, 0, nullptr, &sv, true);
+            fn_backward(ex, Geom{N, tH, tH}, tin, T, sv, halves(d1, d2, s.c), nullptr, Pair{}, gout, nullptr);
             ex.ws.release(m);
             gi ^= 1;
         }

@@ -119,22 +119,46 @@ class StackRunner:
                     momentum=B.unpack_params(self.specs, self.momentum.cpu().numpy()))
 
 
-def time_block(ctx: B.Context, b: syn.BlockCfg, mode: int, reps: int = 10, warmup: int = 3):
+def time_block(ctx: B.Context, b: syn.BlockCfg, mode: int, reps: int = 10, warmup: int = 3, graph: bool = True):
     """Device time (ms) of one block forward and one reconstructing backward at shape b, in place,
-    through the C ABI, with CUDA events on the launching stream."""
+    through the C ABI, with CUDA events on the launching stream.  With graph=True each of the two
+    calls is captured once into a CUDA graph and replayed, so the figure holds kernel time without
+    the host's launch overhead (as in a train step, which replays a graph too)."""
     inp = syn.make_block_inputs(b, affine_jitter=True)
     r = BlockRunner(ctx, b, mode)
     r.load(inp["params"])
     x1, x2 = to_state(inp["x1"], r.frac), to_state(inp["x2"], r.frac)
     d1, d2 = _dev(B.to_nhwc(inp["dy1"])), _dev(B.to_nhwc(inp["dy2"]))
+
+    def fwd():
+        B.revnet_block_fwd(ctx, r.desc, x1, x2, r.F, r.G, x1, x2, r.ws)
+
+    def bwd():
+        B.revnet_block_bwd(ctx, r.desc, x1, x2, d1, d2, r.F, r.G, x1, x2, d1, d2, r.gF, r.gG, r.ws)
+
+    fwd(); bwd()                      # first-call set-up happens outside any capture
+    torch.cuda.synchronize()
+    if graph:
+        side = torch.cuda.Stream()
+        graphs = []
+        for fn in (fwd, bwd):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(side):
+                with torch.cuda.graph(g, stream=side):
+                    fn()
+            graphs.append(g)
+        torch.cuda.synchronize()
+        run_f, run_b = graphs[0].replay, graphs[1].replay
+    else:
+        run_f, run_b = fwd, bwd
     stream = torch.cuda.current_stream()
     ms = {"fwd": [], "bwd": []}
     for i in range(warmup + reps):
         e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
         e[0].record(stream)
-        B.revnet_block_fwd(ctx, r.desc, x1, x2, r.F, r.G, x1, x2, r.ws)
+        run_f()
         e[1].record(stream)
-        B.revnet_block_bwd(ctx, r.desc, x1, x2, d1, d2, r.F, r.G, x1, x2, d1, d2, r.gF, r.gG, r.ws)
+        run_b()
         e[2].record(stream)
         torch.cuda.synchronize()
         if i >= warmup:
@@ -150,6 +174,7 @@ if __name__ == "__main__":
     ap.add_argument("--c", type=int, default=64); ap.add_argument("--w", type=int, default=0)
     ap.add_argument("--kind", default="basic"); ap.add_argument("--mode", type=int, default=0)
     ap.add_argument("--reps", type=int, default=10); ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--eager", action="store_true", help="launch kernel by kernel instead of replaying CUDA graphs")
     a = ap.parse_args()
     c = B.Context(0)
-    print(json.dumps(dict(shape=vars(a), ms=time_block(c, syn.BlockCfg(a.N, a.H, a.H, a.c, a.w, a.kind, seed=5), a.mode, a.reps, a.warmup))))
+    print(json.dumps(dict(shape=vars(a), ms=time_block(c, syn.BlockCfg(a.N, a.H, a.H, a.c, a.w, a.kind, seed=5), a.mode, a.reps, a.warmup, graph=not a.eager))))

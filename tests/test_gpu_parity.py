@@ -201,7 +201,19 @@ def run_stack_case(ctx, cfg, mode, jitter=True, plain_forward=False):
     st = r.step()
     g = r.results()
     t = dict(TOL[mode])
-    assert hp.rel_l2(g["logits"], o["logits"]) <= t["out"], hp.rel_l2(g["logits"], o["logits"])
+    floor_runs = {}
+
+    def floor_run(level):
+        if level not in floor_runs:
+            rng = np.random.default_rng(98)
+            pim = inp["images"].astype(np.float64) * (1 + level * rng.uniform(-1, 1, inp["images"].shape))
+            floor_runs[level] = orc.stack_train_grads(net, pim, inp["labels"], "reconstruct", num=oracle_numerics(r))
+        return floor_runs[level]
+
+    # logits: the stated tolerance, unless one rounding decision tipping over already moves the oracle's
+    # own logits further than that (tiny batches: BN over a few dozen samples), see the module docstring
+    check_grads(dict(logits=g["logits"]), dict(logits=o["logits"]), t["out"], lambda lv: dict(logits=floor_run(lv)["logits"]),
+                perturb_levels(r), cfg.name + " logits")
     if plain_forward:       # forward quantities also against the unrounded float64 definition
         plain = orc.stack_train_grads(net, inp["images"], inp["labels"], "reconstruct")
         assert hp.rel_l2(g["logits"], plain["logits"]) <= t["out"]
@@ -215,11 +227,7 @@ def run_stack_case(ctx, cfg, mode, jitter=True, plain_forward=False):
     assert np.array_equal(g["pred"][clear], o["pred"][clear])
     if mode == 1:
         assert np.array_equal(g["pred"], o["pred"])
-    def floor_fn(level):
-        rng = np.random.default_rng(98)
-        pim = inp["images"].astype(np.float64) * (1 + level * rng.uniform(-1, 1, inp["images"].shape))
-        return orc.stack_train_grads(net, pim, inp["labels"], "reconstruct", num=oracle_numerics(r))["grads"]
-    worst, floor = check_grads(g["grads"], o["grads"], t["grad"], floor_fn, perturb_levels(r), cfg.name)
+    worst, floor = check_grads(g["grads"], o["grads"], t["grad"], lambda lv: floor_run(lv)["grads"], perturb_levels(r), cfg.name)
     bound = min(MAX_BOUND, max(t["grad"], FLOOR_FACTOR * floor))
     for k in op:
         # momentum = gradient + weight decay; updated weights move by lr * momentum

@@ -16,6 +16,9 @@
 bool conv_fprop_tc(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign, Moments *stats);
 bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, const BnBwdReq *bb);
 bool conv_wgrad_tc(Exec &ex, const void *g, const void *a, Geom gi, const Layer &L, float *dW);
+// one kernel for BN -> ReLU -> conv (at most 64 input channels, stride 1); likewise the data gradient of such a layer
+bool conv_fprop_fused(Exec &ex, Pair t, BnRef bn, Geom gi, const Layer &L, Pair out, Pair partner, int sign, Moments *stats, bf16 *a_out);
+bool conv_dgrad_fused(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, const BnBwdReq *bb);
 
 // stats: in = where the statistics of `out` should go (or nullptr); stats->valid says whether the kernel provides them
 static void conv_fprop(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign, Moments *stats) {
@@ -28,6 +31,7 @@ static void conv_fprop(Exec &ex, const void *a, Geom gi, const Layer &L, Pair ou
 // returns true when the epilogue also produced the BN-backward sums asked for in bb
 static bool conv_dgrad(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, const BnBwdReq *bb) {
     const bool b16 = ex.mode == 0;
+    if (b16 && L.stride == 1 && conv_dgrad_fused(ex, g, gi, L, da, bb)) return bb != nullptr;
     if (b16 && L.stride == 1 && conv_dgrad_tc(ex, g, gi, L, da, bb)) return bb != nullptr;
     if (b16 && L.stride == 2 && gi.H % 2 == 0 && gi.W % 2 == 0 && L.cout % 8 == 0) {
         // stride 2: spread g over the input grid (zeros between samples); the data gradient is then the
@@ -72,16 +76,25 @@ void fn_forward(Exec &ex, Geom g, Pair u, const Moments *mom_in, const std::vect
             bn_stats(ex, t, P, cur);
             cur.valid = true;
         }
-        void *a = ex.ws.alloc(P * ly.cin * esz(ex));
-        bn_relu_apply(ex, t, P, BnRef{ly.gamma, ly.beta, cur.mean, cur.rstd}, a, b16);
+        const BnRef bn{ly.gamma, ly.beta, cur.mean, cur.rstd};
+        const bool last = l == L - 1;
         Geom go{gi.N, conv_out(gi.H, ly.k, ly.stride), conv_out(gi.W, ly.k, ly.stride)};
+        // the activated tensor is materialised only where something reads it: the unfused convolution, or the weight gradient
+        void *a = ex.ws.alloc(P * ly.cin * esz(ex));
+        float *tn = last ? nullptr : ex.ws.get<float>(go.P() * ly.cout);
+        Moments next;
+        if (!last) next = mom_alloc(ex, ly.cout);
+        const Pair o = last ? out : single(tn, ly.cout);
+        bool fused = false;
+        if (b16 && !(last && skip_last_conv))
+            fused = conv_fprop_fused(ex, t, bn, gi, ly, o, last ? partner : Pair{}, last ? sign : 0, last ? mom_out : &next,
+                                     saved ? (bf16 *)a : nullptr);
+        if (!fused) bn_relu_apply(ex, t, P, bn, a, b16);
         if (saved) { saved->a.push_back(a); saved->bn.push_back(cur); }
-        if (l == L - 1) {
-            if (!skip_last_conv) conv_fprop(ex, a, gi, ly, out, partner, sign, mom_out);
+        if (last) {
+            if (!skip_last_conv && !fused) conv_fprop(ex, a, gi, ly, out, partner, sign, mom_out);
         } else {
-            float *tn = ex.ws.get<float>(go.P() * ly.cout);
-            Moments next = mom_alloc(ex, ly.cout);
-            conv_fprop(ex, a, gi, ly, single(tn, ly.cout), Pair{}, 0, &next);
+            if (!fused) conv_fprop(ex, a, gi, ly, single(tn, ly.cout), Pair{}, 0, &next);
             if (saved) saved->t.push_back(tn);
             t = single(tn, ly.cout);
             cur = next;     // valid only if the epilogue summed them; else the next round computes them

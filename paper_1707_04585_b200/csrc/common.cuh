@@ -228,6 +228,13 @@ void conv_wgrad_simt(Exec &ex, const void *g, bool g_bf16, const void *a, bool a
 // What a data-gradient epilogue needs to fuse the two sums of the BN+ReLU backward of the layer's
 // own BN: its input t, its coefficients, and where dgamma, dbeta and coef[3][C] go.
 struct BnBwdReq { Pair t; BnRef bn; float *dgamma, *dbeta, *coef; };
+// Reductions a convolution epilogue is asked to fuse.
+struct EpiReq {
+    Moments *stats = nullptr;          // statistics of the stored result
+    const BnBwdReq *bnbwd = nullptr;   // data gradient: sums of the BN+ReLU backward
+};
+void *tc_encoder(revnet_ctx *ctx);     // cuTensorMapEncodeTiled, resolved once per context (nullptr if unavailable)
+void tc_pack_now(Exec &ex, const float *W, bf16 *out, int cin, int cout, int k, bool transposed);
 // bf16 weight packs of the tensor-core kernels, built once per train step
 struct PackJob { const float *W; bf16 *out; int Co, Ci, k, rows_pad, cols_pad, transposed; };
 size_t tc_pack_elems(int cin, int cout, int k, bool transposed);

@@ -21,6 +21,7 @@ struct EpiArgs {
     Pair out, partner;       // [P, n_cols]; partner only with EPI_COUPLE
     int sign;                // EPI_COUPLE: +1 / -1
     int n_cols;              // valid output channels
+    int pitch;               // floats per staged row: min(N tile, 64) + 4
     // reductions (optional: part == nullptr switches them off; EPI_BNBWD always reduces)
     float *part;             // [gridDim.x][n_cols/4][2][4]: per channel quad, 4 sums then 4 second sums
     unsigned int *counter;   // zero on entry, left zero
@@ -39,61 +40,99 @@ struct TileGeom {
     int BH, BIMG;
     int tiles_per_img;       // BIMG == 1
     int n_px_tiles;
-    int hw_order;            // accumulator rows run (h, img, w) instead of (img, h, w)
+    int hw_order;            // accumulator rows run (h, img, x) with x < Wp instead of (img, h, w)
+    int Wp;                  // hw_order: row pitch in pixels (W rounded up to a multiple of 8); columns >= W are padding
 };
 __device__ __forceinline__ void tile_origin(const TileGeom &g, int t, int &n0, int &h0) {
     if (g.BIMG > 1) { n0 = t * g.BIMG; h0 = 0; }
     else { n0 = t / g.tiles_per_img; h0 = (t - n0 * g.tiles_per_img) * g.BH; }
 }
-// global pixel index of accumulator row m, or -1 for a padding row
-__device__ __forceinline__ int tile_row_pixel(const TileGeom &g, int n0, int h0, int m) {
-    if (m >= g.BIMG * g.BH * g.W) return -1;
-    int img, h, w = m % g.W;
-    if (g.hw_order) { h = m / (g.BIMG * g.W); img = (m / g.W) % g.BIMG; }
-    else { img = m / (g.BH * g.W); h = (m / g.W) % g.BH; }
-    h += h0;
-    if (n0 + img >= g.N || h >= g.H) return -1;
-    return ((n0 + img) * g.H + h) * g.W + w;
-}
-
 constexpr int kEpiChunk = 64;                    // accumulator columns staged at a time
 constexpr int kEpiPitch = kEpiChunk + 4;         // floats per staged row (bank-conflict padding)
+constexpr int kEpiMaxChunks = 2;                 // N tile <= 128 columns
+constexpr int kEpiSumFloats = kEpiMaxChunks * 128 * 8;   // per thread and chunk: 4 sums, 4 second sums
 constexpr int kEpiStageBytes = 128 * kEpiPitch * 4;
-constexpr int kEpiMaxChunks = 4;                 // N tile <= 256 columns
-
-struct EpiAcc {                                  // per-thread running sums, by column chunk
-    float s[kEpiMaxChunks][4], ss[kEpiMaxChunks][4];
-    __device__ __forceinline__ void clear() {
-#pragma unroll
-        for (int c = 0; c < kEpiMaxChunks; c++)
-#pragma unroll
-            for (int j = 0; j < 4; j++) { s[c][j] = 0.f; ss[c][j] = 0.f; }
-    }
-};
 
 __device__ __forceinline__ float4 ldcg4(const float *p) { return __ldcg(reinterpret_cast<const float4 *>(p)); }
 
+// Which pixel an accumulator row holds depends on the tile only through its origin, so the part
+// that does not is decoded once per CTA: rel = pixel offset relative to the tile's origin pixel
+// (image n0, row h0, column 0), -1 for rows that are padding in every tile; hi = row | image << 16
+// within the tile, for the bounds checks of ragged tiles.
+struct RowMap { int rel[128]; int hi[128]; };
+__device__ __forceinline__ void build_row_map(const TileGeom &g, RowMap *rm, int m) {
+    int img, h, w;
+    bool ok = true;
+    if (g.hw_order) {
+        w = m % g.Wp; img = (m / g.Wp) % g.BIMG; h = m / (g.BIMG * g.Wp);
+        ok = w < g.W && h < g.BH;
+    } else {
+        ok = m < g.BIMG * g.BH * g.W;
+        w = m % g.W; img = m / (g.BH * g.W); h = (m / g.W) % g.BH;
+    }
+    rm->rel[m] = ok ? (img * g.H + h) * g.W + w : -1;
+    rm->hi[m] = h | (img << 16);
+}
+__device__ __forceinline__ int row_pixel(const RowMap *rm, const TileGeom &g, int n0, int h0, int tile_base, int row) {
+    if (row >= 128) return -1;
+    const int rel = rm->rel[row], hi = rm->hi[row];
+    if (rel < 0 || h0 + (hi & 0xffff) >= g.H || n0 + (hi >> 16) >= g.N) return -1;
+    return tile_base + rel;
+}
+
+// Shared memory of the epilogue: the padded stage (kEpiStageBytes) and each thread's running sums
+// per column chunk (kEpiSumFloats floats, zeroed by epilogue_init).
+__device__ __forceinline__ void epilogue_init(float *sums, int etid) {
+    for (int i = etid; i < kEpiSumFloats; i += 128) sums[i] = 0.f;
+}
+
+// What the first four rows a thread handles read from global memory besides the accumulator (the
+// partner of the coupling, or the BN input of a data gradient) can be fetched before the
+// accumulator is complete.
+struct EpiPrefetch { float4 v[4]; };
+__device__ __forceinline__ void epilogue_prefetch(const EpiArgs &e, int BN, int col0, const RowMap *rm, const TileGeom &g,
+                                                  int n0, int h0, int etid, EpiPrefetch &pre) {
+    if (e.mode == EPI_PLAIN) return;
+    const int cw = BN < kEpiChunk ? BN : kEpiChunk;
+    const int QW = cw >> 2, rpp = 128 / QW;
+    const int quad = etid % QW, r0 = etid / QW;
+    const int col = col0 + quad * 4;
+    const int tile_base = (n0 * g.H + h0) * g.W;
+    if (r0 < rpp && col < e.n_cols) {
+#pragma unroll
+        for (int i = 0; i < 4; i++) {
+            const int pix = row_pixel(rm, g, n0, h0, tile_base, r0 + i * rpp);
+            if (pix >= 0) {
+                if (e.mode == EPI_COUPLE) pre.v[i] = *reinterpret_cast<const float4 *>(e.partner.at((size_t)pix, col));
+                else pre.v[i] = e.t.ld4((size_t)pix, col);
+            }
+        }
+    }
+}
+
 // One tile: 128 epilogue threads (etid 0..127; thread etid owns accumulator lane etid), BN
 // accumulator columns starting at tensor-memory address tmem_acc; col0 = first output channel of
-// this N tile.  row_pix[128] and stage live in shared memory.  acc_empty is arrived on by every
-// thread once the accumulator has been read.
-__device__ __forceinline__ void epilogue_tile(const EpiArgs &e, uint32_t tmem_acc, int BN, int col0, const int *row_pix,
-                                              float *stage, EpiAcc &acc, int etid, uint64_t *acc_empty) {
+// this N tile.  rm and stage live in shared memory.  acc_empty is arrived on by every thread once
+// the accumulator has been read.  The loops are deliberately not unrolled beyond four rows: the
+// code has to stay small enough to live in the instruction cache.
+__device__ __forceinline__ void epilogue_tile(const EpiArgs &e, uint32_t tmem_acc, int BN, int col0, const RowMap *rm,
+                                              const TileGeom &g, int n0, int h0, float *stage, float *sums, int etid,
+                                              uint64_t *acc_empty, const EpiPrefetch &pre) {
     const uint32_t lane_base = (uint32_t)((etid >> 5) * 32) << 16;
-#pragma unroll
-    for (int ch = 0; ch < kEpiMaxChunks; ch++) {
-        const int cc = ch * kEpiChunk;
-        if (cc >= BN) break;
+    const int tile_base = (n0 * g.H + h0) * g.W;
+#pragma unroll 1
+    for (int cc = 0; cc < BN; cc += kEpiChunk) {
         const int cw = BN - cc < kEpiChunk ? BN - cc : kEpiChunk;
         // phase 1: accumulator row -> staged row
+#pragma unroll 1
         for (int c = 0; c < cw; c += 16) {
             float v[16];
             tmem_ld16(tmem_acc + lane_base + (uint32_t)(cc + c), v);
-            float4 *dst = reinterpret_cast<float4 *>(stage + etid * kEpiPitch + c);
+            float4 *dst = reinterpret_cast<float4 *>(stage + etid * e.pitch + c);
             dst[0] = make_float4(v[0], v[1], v[2], v[3]); dst[1] = make_float4(v[4], v[5], v[6], v[7]);
             dst[2] = make_float4(v[8], v[9], v[10], v[11]); dst[3] = make_float4(v[12], v[13], v[14], v[15]);
         }
-        if (cc + cw >= BN) { tc_fence_before(); mbar_arrive(acc_empty); }
+        if (acc_empty && cc + cw >= BN) { tc_fence_before(); mbar_arrive(acc_empty); }
         named_barrier(1, 128);
         // phase 2: thread = (row r0 of each pass, channel quad); consecutive threads touch consecutive addresses
         const int QW = cw >> 2, rpp = 128 / QW;
@@ -103,23 +142,24 @@ __device__ __forceinline__ void epilogue_tile(const EpiArgs &e, uint32_t tmem_ac
             float4 sc = make_float4(0, 0, 0, 0), sh = sc, mu = sc, rs = sc;
             if (e.mode == EPI_BNBWD) bn_coef4(e.bn, col, sc, sh, mu, rs);
             float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f, q0 = 0.f, q1 = 0.f, q2 = 0.f, q3 = 0.f;
+#pragma unroll 1
             for (int rb = r0; rb < 128; rb += 4 * rpp) {
                 int pix[4]; float4 aux[4];
+                const bool fetched = cc == 0 && rb == r0;
                 // loads of the partner / BN input first: they may alias the stores below
 #pragma unroll
                 for (int i = 0; i < 4; i++) {
-                    const int row = rb + i * rpp;
-                    pix[i] = row < 128 ? row_pix[row] : -1;
+                    pix[i] = row_pixel(rm, g, n0, h0, tile_base, rb + i * rpp);
                     if (pix[i] >= 0) {
-                        if (e.mode == EPI_COUPLE) aux[i] = *reinterpret_cast<const float4 *>(e.partner.at((size_t)pix[i], col));
+                        if (fetched) aux[i] = pre.v[i];
+                        else if (e.mode == EPI_COUPLE) aux[i] = *reinterpret_cast<const float4 *>(e.partner.at((size_t)pix[i], col));
                         else if (e.mode == EPI_BNBWD) aux[i] = e.t.ld4((size_t)pix[i], col);
                     }
                 }
 #pragma unroll
                 for (int i = 0; i < 4; i++) {
                     if (pix[i] < 0) continue;
-                    const int row = rb + i * rpp;
-                    float4 v = *reinterpret_cast<const float4 *>(stage + row * kEpiPitch + quad * 4);
+                    float4 v = *reinterpret_cast<const float4 *>(stage + (rb + i * rpp) * e.pitch + quad * 4);
                     if (e.mode == EPI_BNBWD) {
                         *reinterpret_cast<float4 *>(e.out.at((size_t)pix[i], col)) = v;
                         const float4 t = aux[i];
@@ -136,41 +176,48 @@ __device__ __forceinline__ void epilogue_tile(const EpiArgs &e, uint32_t tmem_ac
                     }
                 }
             }
-            acc.s[ch][0] += s0; acc.s[ch][1] += s1; acc.s[ch][2] += s2; acc.s[ch][3] += s3;
-            acc.ss[ch][0] += q0; acc.ss[ch][1] += q1; acc.ss[ch][2] += q2; acc.ss[ch][3] += q3;
+            if (e.part) {       // this thread's own slot: no other thread touches it
+                float4 *slot = reinterpret_cast<float4 *>(sums + ((cc / kEpiChunk) * 128 + etid) * 8);
+                float4 a = slot[0], b = slot[1];
+                a.x += s0; a.y += s1; a.z += s2; a.w += s3; b.x += q0; b.y += q1; b.z += q2; b.w += q3;
+                slot[0] = a; slot[1] = b;
+            }
         }
         named_barrier(1, 128);
     }
 }
 
+__device__ __forceinline__ void epilogue_publish(const EpiArgs &e, float *scratch, int etid);
+
 // After the last tile: per-CTA partials, grid-wide count, and the finalize by the CTA that comes last.
-// scratch: >= 8 KB of shared memory (the stage).
-__device__ __forceinline__ void epilogue_finish(const EpiArgs &e, int BN, int col0, float *scratch, const EpiAcc &acc, int etid) {
+__device__ __forceinline__ void epilogue_finish(const EpiArgs &e, int BN, int col0, float *stage, const float *sums, int etid) {
     if (!e.part) return;
+    float *scratch = stage;
     float *mine = e.part + (size_t)blockIdx.x * 2 * e.n_cols;
-#pragma unroll
-    for (int ch = 0; ch < kEpiMaxChunks; ch++) {
-        const int cc = ch * kEpiChunk;
-        if (cc >= BN) break;
+#pragma unroll 1
+    for (int cc = 0; cc < BN; cc += kEpiChunk) {
         const int cw = BN - cc < kEpiChunk ? BN - cc : kEpiChunk;
         const int QW = cw >> 2, rpp = 128 / QW;
         const int quad = etid % QW, r0 = etid / QW;
-#pragma unroll
-        for (int j = 0; j < 4; j++) { scratch[etid * 8 + j] = acc.s[ch][j]; scratch[etid * 8 + 4 + j] = acc.ss[ch][j]; }
-        named_barrier(1, 128);
         const int col = col0 + cc + quad * 4;
         if (r0 == 0 && col < e.n_cols) {
+            const float *base = sums + (size_t)(cc / kEpiChunk) * 128 * 8;
             float r[8];
 #pragma unroll
-            for (int j = 0; j < 8; j++) r[j] = scratch[quad * 8 + j];
+            for (int j = 0; j < 8; j++) r[j] = base[quad * 8 + j];
             for (int y = 1; y < rpp; y++)
 #pragma unroll
-                for (int j = 0; j < 8; j++) r[j] += scratch[(y * QW + quad) * 8 + j];
+                for (int j = 0; j < 8; j++) r[j] += base[(y * QW + quad) * 8 + j];
             *reinterpret_cast<float4 *>(mine + 2 * col) = make_float4(r[0], r[1], r[2], r[3]);
             *reinterpret_cast<float4 *>(mine + 2 * col + 4) = make_float4(r[4], r[5], r[6], r[7]);
         }
-        named_barrier(1, 128);
     }
+    epilogue_publish(e, scratch, etid);
+}
+
+// Once every CTA has written its partial record into e.part: count, and let the CTA that comes
+// last reduce the records in a fixed order and write the results.  scratch: 8 KB of shared memory.
+__device__ __forceinline__ void epilogue_publish(const EpiArgs &e, float *scratch, int etid) {
     // publish, count, and let the last CTA of the grid reduce
     __threadfence();
     named_barrier(1, 128);

@@ -47,7 +47,7 @@ struct __align__(8) TcShared {
     uint64_t acc_empty[2];
     uint32_t tmem_base;
     uint32_t failed;
-    int row_pix[128];
+    RowMap rows;
 };
 
 // Persistent CTA: walks the pixel tiles blockIdx.x, blockIdx.x + gridDim.x, ... of N tile blockIdx.y.
@@ -63,7 +63,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int b_off = (128 * p.KC * 2 + 1023) & ~1023;
     const int stage_bytes = b_off + ((b_bytes + 1023) & ~1023);
     float *estage = (float *)(tiles + kStages * stage_bytes);
-    TcShared *sh = (TcShared *)((uint8_t *)estage + kEpiStageBytes);
+    TcShared *sh = (TcShared *)((uint8_t *)estage + kEpiStageBytes + kEpiSumFloats * 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int iters = p.taps * p.chunks;
@@ -78,6 +78,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         tma_prefetch_desc(&map_a); tma_prefetch_desc(&map_b);
     }
     if (warp == 1) tmem_alloc(&sh->tmem_base, tmem_cols);
+    if (warp >= 2) build_row_map(p.g, &sh->rows, ((warp & 3) << 5) | lane);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -134,22 +135,24 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else {
         // epilogue: this warp may touch accumulator lanes 32*(warp%4) .. +31
         const int etid = ((warp & 3) << 5) | lane;
-        EpiAcc acc;
-        acc.clear();
+        float *esums = estage + 128 * kEpiPitch;
+        epilogue_init(esums, etid);
+        named_barrier(1, 128);
         bool ok = true;
         int ti = 0;
         for (int t = blockIdx.x; t < p.g.n_px_tiles; t += gridDim.x, ti++) {
             const int buf = ti & 1; const uint32_t use = ti >> 1;
             int n0, h0;
             tile_origin(p.g, t, n0, h0);
-            sh->row_pix[etid] = tile_row_pixel(p.g, n0, h0, etid);
-            ok = mbar_wait(&sh->acc_full[buf], use & 1) && sh->failed == 0;
-            ok = named_barrier_and(2, 128, ok);       // also publishes row_pix
+            EpiPrefetch pre;
+            epilogue_prefetch(p.epi, p.BN, col0, &sh->rows, p.g, n0, h0, etid, pre);     // before the accumulator is ready
+            if (etid == 0) ok = mbar_wait(&sh->acc_full[buf], use & 1) && sh->failed == 0;     // one thread polls, the rest block
+            ok = named_barrier_and(2, 128, ok);
             if (!ok) break;
             tc_fence_after();
-            epilogue_tile(p.epi, tmem_d + (uint32_t)(buf * p.BN), p.BN, col0, sh->row_pix, estage, acc, etid, &sh->acc_empty[buf]);
+            epilogue_tile(p.epi, tmem_d + (uint32_t)(buf * p.BN), p.BN, col0, &sh->rows, p.g, n0, h0, estage, esums, etid, &sh->acc_empty[buf], pre);
         }
-        if (ok) epilogue_finish(p.epi, p.BN, col0, estage, acc, etid);
+        if (ok) epilogue_finish(p.epi, p.BN, col0, estage, esums, etid);
         else if (lane == 0) atomicExch(&sh->failed, 1u);
     }
     tc_fence_before();
@@ -216,7 +219,7 @@ int round_up(int x, int m) { return (x + m - 1) / m * m; }
 // that fall outside are padding: TMA fills their operand rows with zeros and the epilogue skips them.
 bool tile_geom(Geom g, TileGeom &t) {
     if (g.W > 128 || g.W < 1) return false;
-    t.N = g.N; t.H = g.H; t.W = g.W; t.hw_order = 0;
+    t.N = g.N; t.H = g.H; t.W = g.W; t.hw_order = 0; t.Wp = g.W;
     t.BH = 128 / g.W; if (t.BH > g.H) t.BH = g.H;
     t.BIMG = 1;
     if (t.BH == g.H) { t.BIMG = 128 / (g.H * g.W); if (t.BIMG > g.N) t.BIMG = g.N; if (t.BIMG < 1) t.BIMG = 1; }
@@ -239,15 +242,9 @@ bool tc_shape(Geom g, int cin, int cout, int k, int stride, TcShape &s) {   // g
     s.BN = cout_pad <= 128 ? cout_pad : 128;
     s.n_tiles = (cout_pad + s.BN - 1) / s.BN;
     const int a_bytes = 128 * s.KC * 2, b_bytes = s.BN * s.KC * 2;
-    s.smem = 1024 + kStages * (((a_bytes + 1023) & ~1023) + ((b_bytes + 1023) & ~1023)) + kEpiStageBytes + (int)sizeof(TcShared) + 64;
+    s.smem = 1024 + kStages * (((a_bytes + 1023) & ~1023) + ((b_bytes + 1023) & ~1023)) + kEpiStageBytes + kEpiSumFloats * 4 + (int)sizeof(TcShared) + 64;
     return true;
 }
-
-// Reductions a convolution epilogue is asked to fuse.
-struct EpiReq {
-    Moments *stats = nullptr;          // statistics of the stored result
-    const BnBwdReq *bnbwd = nullptr;   // data gradient: sums of the BN+ReLU backward
-};
 
 // act: bf16 [N,H,W,cin]; Wsrc: fp32 weights; transposed selects the dgrad pack
 bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin, int cout, int k, int stride,
@@ -305,7 +302,7 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         EpiArgs &e = p.epi;
         memset(&e, 0, sizeof e);
         e.mode = req.bnbwd ? EPI_BNBWD : (sign ? EPI_COUPLE : EPI_PLAIN);
-        e.out = out; e.partner = partner; e.sign = sign; e.n_cols = cout;
+        e.out = out; e.partner = partner; e.sign = sign; e.n_cols = cout; e.pitch = kEpiPitch;
         e.part = part; e.counter = reduce ? ex.ctx->counter() : nullptr;
         e.inv_count = 1.0 / (double)g.P(); e.eps = ex.eps;
         if (req.stats) { e.mean = req.stats->mean; e.rstd = req.stats->rstd; }
@@ -419,7 +416,9 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         }
     } else {
         const int quarter = warp & 3;
-        const bool ok = mbar_wait(&sh->acc_full[0], 0);
+        bool ok = true;
+        if (quarter == 0 && lane == 0) ok = mbar_wait(&sh->acc_full[0], 0);     // one thread polls, the rest block
+        ok = named_barrier_and(2, 128, ok);
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (ok && sh->failed == 0) {
             const int m = quarter * 32 + lane;
@@ -558,6 +557,18 @@ bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer
     }
     ex.ws.release(m);
     return true;
+}
+
+void *tc_encoder(revnet_ctx *ctx) { return (void *)encoder(ctx); }
+
+// pack of one layer built on the spot (calls that have no step-level pack)
+void tc_pack_now(Exec &ex, const float *W, bf16 *out, int cin, int cout, int k, bool transposed) {
+    if (ex.dry) return;
+    const PackJob j = tc_pack_job(W, out, cin, cout, k, transposed);
+    const size_t n = (size_t)j.rows_pad * k * k * j.cols_pad;
+    int grid = (int)((n + 255) / 256); if (grid > ex.ctx->sm_count * 4) grid = ex.ctx->sm_count * 4;
+    pack_weights_kernel<<<grid, 256, 0, ex.stream>>>(W, out, cout, cin, k, j.rows_pad, j.cols_pad, transposed ? 1 : 0);
+    ex.check("pack_weights", (double)n * 6);
 }
 
 // ---- packs made once per step (the train step calls these before the forward pass)

@@ -34,10 +34,18 @@ def load_peaks():
 # fp32 FMA peak of the CUDA cores: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (max SM clock)
 ALU_FP32_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 
-KERNEL_BOUND = {  # which roofline a kernel class is measured against
-    "conv_fprop_simt": "alu", "conv_dgrad_simt": "alu", "conv_wgrad_simt": "alu",
-    "conv_fprop_tc": "tensor", "conv_dgrad_tc": "tensor", "conv_wgrad_tc": "tensor",
-}
+ALU_KERNELS = ("conv_fprop_simt", "conv_dgrad_simt", "conv_wgrad_simt")   # fp32 CUDA-core GEMMs
+
+
+def binding_roofline(name, rec, peaks):
+    """Which roofline bounds a kernel class on this workload: the one that needs more time for the
+    kernel's algorithmic bytes and flops (summed over its launches).  Convolutions of narrow layers
+    are bound by memory, wide ones by the tensor cores."""
+    if name in ALU_KERNELS:
+        return "alu"
+    t_mem = rec["bytes"] / (peaks["hbm"] * 1e9)
+    t_tc = rec["flops"] / (peaks["tc_sustained"] * 1e12)
+    return "tensor" if t_tc > t_mem else "hbm"
 
 
 class ClockSampler:
@@ -125,6 +133,19 @@ def run_reference(args, cfg):
     print(json.dumps(line), flush=True)
 
 
+def depth_sweep(ctx, cfg):
+    """Stored activation MB of the same network with 1..36 units per stage (plans only, nothing runs):
+    Section 3.2, storage independent of depth."""
+    from paper_1707_04585_b200 import binding as B, synthetic as syn
+    out = {}
+    for units in (1, 3, 9, 18, 36):
+        c = syn.shrink(cfg, units=units)
+        plan = B.revnet_stack_plan(ctx, B.stack_desc(c, 0, False, 16, False))
+        out[str(units)] = round(plan.activation_bytes / 1e6, 3)
+        plan.close()
+    return out
+
+
 def run_ours(args, cfg):
     import torch
     import torch.distributed as dist
@@ -152,7 +173,16 @@ def run_ours(args, cfg):
             dist.barrier()
         torch.cuda.synchronize()
 
+    params0 = run.params.clone()
+
+    def reset():
+        # every timed step starts from the initial weights and zero momentum: repeated SGD steps at the
+        # paper's learning rate on random labels would drive the activations out of range
+        run.params.copy_(params0)
+        run.momentum.zero_()
+
     for _ in range(args.warmup):
+        reset()
         st = run.step(want_logits=False)
     barrier()
     sampler = ClockSampler(local)
@@ -160,6 +190,7 @@ def run_ours(args, cfg):
         sampler.start()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     for a, b in ev:
+        reset()
         flush.zero_()                      # evict L2 between timed iterations (outside the timed span)
         a.record(stream)
         st = run.step(want_logits=False)
@@ -179,6 +210,7 @@ def run_ours(args, cfg):
     barrier()
     e2e_ms = 0.0
     for _ in range(args.steps):
+        reset()
         flush.zero_()
         torch.cuda.synchronize()
         t0 = time.perf_counter()
@@ -192,6 +224,7 @@ def run_ours(args, cfg):
     B.revnet_profile_enable(ctx, True)
     psteps = 2
     for _ in range(psteps):
+        reset()
         run.step(want_logits=False)
     prof = B.revnet_profile_summary(ctx)
     B.revnet_profile_enable(ctx, False)
@@ -213,7 +246,7 @@ def run_ours(args, cfg):
         tot = sum(v["ms"] for v in prof.values()) or 1.0
         top = max(prof.items(), key=lambda kv: kv[1]["ms"])
         name, rec = top
-        bound = KERNEL_BOUND.get(name, "hbm")
+        bound = binding_roofline(name, rec, peaks)
         avg_s = rec["ms"] / rec["launches"] * 1e-3
         if bound == "hbm":
             ach, peak, runit = rec["bytes"] / rec["launches"] / avg_s / 1e9, peaks["hbm"], "GB/s"
@@ -238,6 +271,7 @@ def run_ours(args, cfg):
                              d2h_bytes_per_step=4 + 4 * rcfg.N, ms_per_step=e2e_ms / args.steps),
                     gpu_launches=launches, clocks=clocks, roofline=roof,
                     activation_bytes=int(st.stored_activation_bytes), workspace_bytes=int(st.workspace_peak_bytes),
+                    activation_mb_vs_units_per_stage=depth_sweep(ctx, rcfg),
                     flops_per_step=int(st.flops_fwd + st.flops_bwd), final_loss=final_loss, block_ms=block_ms)
         if not args.no_cpu and world == 1:
             line["cpu_baseline"] = {k: v for k, v in cpu_baseline(cfg, min(cfg.N, args.ref_batch)).items() if k != "seconds_per_step"}

@@ -333,6 +333,7 @@ struct WgParams {
     int blockN, BN, cout;        // output-channel block, N tile, valid channels
     int GM;                      // M groups per CTA (1 or 2)
     int H, W, BH, BIMG;          // output geometry and tile
+    int tiles_per_img, box_px;   // tiles per image (BIMG == 1); pixels a tile really holds (<= 128, the rest of its rows stay zero)
     int stride;
     int n_tiles_px;              // pixel tiles in all
     int stages;
@@ -368,16 +369,23 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(&sh->tmem_base, tmem_cols);
+    if (p.box_px < 128) {
+        // a tile holds fewer than 128 pixels: the rows TMA never writes must not add to the pixel sum
+        uint4 *z = reinterpret_cast<uint4 *>(tiles);
+        const int n16 = p.stages * stage_bytes / 16;
+        for (int i = threadIdx.x; i < n16; i += kThreads) z[i] = make_uint4(0u, 0u, 0u, 0u);
+        fence_proxy_async();
+    }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem_d = sh->tmem_base;
     const int pad = p.k / 2;
-    const int tiles_per_img = p.BIMG > 1 ? 1 : p.H / p.BH;
+    const int tiles_per_img = p.tiles_per_img;
 
     if (warp == 0) {
         if (lane == 0) {
-            const uint32_t tx = (uint32_t)(n_blocks * blk_bytes_a + nb_n * blk_bytes_b);
+            const uint32_t tx = (uint32_t)(p.box_px * 2 * (n_blocks * p.blockC + nb_n * p.blockN));
             for (int it = 0; it < my_tiles; it++) {
                 const int s = it % p.stages, round = it / p.stages;
                 if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); break; }
@@ -471,14 +479,6 @@ __global__ void splitk_sum_kernel(const float *__restrict__ part, size_t n, int 
 
 int pick_block(int c_pad) { return c_pad % 64 == 0 ? 64 : (c_pad % 32 == 0 ? 32 : 16); }
 
-bool tile_shape(Geom g, int &BH, int &BIMG) {
-    const int W = g.W, H = g.H;
-    if (W > 128 || 128 % W) return false;
-    if (H * W >= 128) { if (H % (128 / W)) return false; BH = 128 / W; BIMG = 1; }
-    else { if (128 % (H * W) || g.N % (128 / (H * W))) return false; BH = H; BIMG = 128 / (H * W); }
-    return true;
-}
-
 // g: geometry of the tensor; (tile_w, BH, BIMG): the 128-pixel tile in units of the traversal stride
 bool encode_act_map(Exec &ex, CUtensorMap *map, const void *base, Geom g, int C, int box_c, int tile_w, int BH, int BIMG, int stride) {
     const CUtensorMapSwizzle sw = box_c == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : (box_c == 32 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_32B);
@@ -510,7 +510,9 @@ bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer
     if (L.stride == 2 && (gi.H % 2 || gi.W % 2)) return false;
     WgParams p;
     const Geom go{gi.N, conv_out(gi.H, L.k, L.stride), conv_out(gi.W, L.k, L.stride)};   // tiles walk the output pixels
-    if (!tile_shape(go, p.BH, p.BIMG)) return false;
+    TileGeom tg;
+    if (!tile_geom(go, tg) || tg.W * L.stride > 256 || tg.BH * L.stride > 256) return false;
+    p.BH = tg.BH; p.BIMG = tg.BIMG; p.tiles_per_img = tg.tiles_per_img; p.box_px = tg.BIMG * tg.BH * tg.W;
     if (!ex.dry && !encoder(ex.ctx)) return false;
     const int taps = L.k * L.k, cin_pad = round_up(L.cin, 16), cout_pad = round_up(L.cout, 16);
     p.taps = taps; p.k = L.k; p.cin = L.cin; p.cout = L.cout;
@@ -524,7 +526,7 @@ bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer
     const int m_chunks = (groups_all + p.GM - 1) / p.GM;
     const int n_tiles = (cout_pad + p.BN - 1) / p.BN;
     p.H = go.H; p.W = go.W; p.stride = L.stride;
-    p.n_tiles_px = (int)(go.P() / 128);
+    p.n_tiles_px = tg.n_px_tiles;
     const int stage_bytes = p.GM * 32768 + ((256 * p.BN + 1023) & ~1023);
     p.stages = (200 * 1024 - 2048) / stage_bytes; if (p.stages > kStages) p.stages = kStages;
     if (p.stages < 2) return false;
@@ -590,7 +592,7 @@ PackJob tc_pack_job(const float *W, bf16 *out, int cin, int cout, int k, bool tr
 }
 void tc_pack_batch(Exec &ex, const PackJob *jobs_dev, int n_jobs, double bytes) {
     if (ex.dry || n_jobs == 0) return;
-    dim3 grid(16, (unsigned)n_jobs);
+    dim3 grid(96, (unsigned)n_jobs);
     pack_weights_batch_kernel<<<grid, 256, 0, ex.stream>>>(jobs_dev);
     ex.check("pack_weights_batch", bytes);
 }

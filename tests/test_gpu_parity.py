@@ -129,6 +129,12 @@ def test_config1_single_block_strict(ctx):
     ("bottleneck", 2, 16, 16, 128, 32),
     ("bottleneck", 3, 7, 7, 64, 16),
     ("basic", 1, 1, 1, 4, 0),         # degenerate: one pixel
+    ("basic", 3, 14, 14, 32, 0),      # image rows not a divisor of the 128-row tile: ragged last tile per image
+    ("basic", 1, 28, 28, 16, 0),      # row pitch padded (28 -> 32 accumulator rows per image row)
+    ("bottleneck", 2, 56, 56, 64, 16),  # large-image stage shape at reduced width: two image rows per tile
+    ("basic", 5, 8, 8, 24, 0),        # channel count padded to 32; odd number of two-image tiles
+    ("basic", 2, 8, 8, 40, 0),        # 40 channels: no single K chunk, the per-tap TMA kernel takes it
+    ("bottleneck", 4, 8, 8, 96, 24),  # 1x1 convolutions with more than 64 input channels
 ])
 @pytest.mark.parametrize("inplace", [False, True])
 def test_block_parity(ctx, mode, kind, N, H, W, c, w, inplace):

@@ -145,11 +145,37 @@ struct Exec {
     uint64_t flops = 0;    // dense conv/FC flops issued
     uint64_t launches = 0;
     bool failed = false;
+    bool pdl = true;       // launch kernels with programmatic stream serialization (see launch())
     // called after every launch: error check, launch count and (when profiling) an event;
     // bytes / flops are the algorithmic traffic and work of that launch
     void check(const char *what, double bytes = 0, double flops = 0);
     void mark(const char *what);   // profiling boundary that is not a kernel (copies, step start)
 };
+
+// Every kernel of the library is launched through here.  With ex.pdl the launch carries the
+// programmatic-stream-serialization attribute: the grid may be scheduled while its predecessor in
+// the stream still runs, and executes its set-up (barrier initialisation, tensor-memory
+// allocation, index tables) meanwhile; each kernel calls pdl_enter() before it touches anything a
+// predecessor wrote, which waits for the predecessor to complete and only then lets its own
+// successor be scheduled, so at most two kernels of a stream overlap and ordering stays transitive.
+template <class... KArgs, class... Args>
+inline void launch(Exec &ex, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = ex.stream;
+    cudaLaunchAttribute attr = {};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr; cfg.numAttrs = ex.pdl ? 1 : 0;
+    cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+#ifdef __CUDACC__
+// wait until the kernel before this one in the stream has completed (its writes are visible), then
+// allow the kernel after this one to be scheduled
+__device__ __forceinline__ void pdl_enter() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
 
 // One BN -> ReLU -> conv layer with its parameter and gradient pointers.
 struct Layer {

@@ -43,7 +43,9 @@ struct FusedParams {
     int wtile_bytes;       // one tap of the weights: BN rows of KC bf16, rounded up to 1024
     int a_bytes;           // operand region (k copies)
     int raw_bytes;         // one raw input tile with halo, rounded up to 128
-    int aux_bytes;         // one partner / output tile: tile pixels x BN floats, rounded up to 128
+    int aux_bytes;         // one partner / output tile: BN / GW column groups of group_bytes
+    int GW;                // floats per row of a column group (16 or 32): rows of 64 / 128 bytes, stored with the matching TMA swizzle
+    int group_bytes;       // tile pixels x GW floats, rounded up to 1024
     TileGeom g;            // hw_order = 1
     int in_mode;           // 0: float / fixed-point tensor through BN + ReLU; 1: bf16 tensor as it is
     float in_q;            // in_mode 0: fixed-point step of the input (0: float)
@@ -214,8 +216,13 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
         int n0, h0;
         tile_origin(p.g, t, n0, h0);
         mbar_expect_tx(&sh->aux_full[b], aux_tx);
-        tma_load_4d(auxb + b * p.aux_bytes, &map_aux, &sh->aux_full[b], col0, 0, h0, n0);
+        for (int g = 0; g < p.BN / p.GW; g++)
+            tma_load_4d(auxb + b * p.aux_bytes + g * p.group_bytes, &map_aux, &sh->aux_full[b], col0 + g * p.GW, 0, h0, n0);
     };
+    // byte offset of float4 j of pixel r inside a column group: rows of 128 (64) bytes, 16-byte chunks XORed with
+    // address bits 7.. as the TMA swizzle does, so that a thread per row touches all banks
+    const int row_b = p.GW * 4;
+    auto sw_off = [&](int r, int j) { return r * row_b + ((j ^ (p.GW == 32 ? (r & 7) : ((r >> 1) & 3))) << 4); };
 
     if (threadIdx.x == 0) {
         for (int b = 0; b < 2; b++) { mbar_init(&sh->raw_full[b], 1); mbar_init(&sh->aux_full[b], 1); }
@@ -225,12 +232,6 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tma_prefetch_desc(&map_w); tma_prefetch_desc(&map_in); tma_prefetch_desc(&map_out);
         if (need_aux) tma_prefetch_desc(&map_aux);
-        mbar_expect_tx(&sh->w_full, (uint32_t)(taps * p.BN * p.KC * 2));
-        for (int tap = 0; tap < taps; tap++) tma_load_2d(wres + tap * p.wtile_bytes, &map_w, &sh->w_full, tap * p.KC, col0);
-        if ((int)blockIdx.x < p.g.n_px_tiles) {
-            load_raw(blockIdx.x, 0);
-            if (need_aux) load_aux(blockIdx.x, 0);
-        }
     }
     if (warp == 0) tmem_alloc(&sh->tmem_base, tmem_cols);
     build_table(p, tab, npix, cshift);
@@ -238,7 +239,17 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
         // accumulator row (image row, image, column) -> pixel of the (image, row, column) ordered tile
         const int w = etid % p.g.Wp, img = (etid / p.g.Wp) % p.g.BIMG, h = etid / (p.g.BIMG * p.g.Wp);
         sh->srow[etid] = (w < p.g.W && h < p.g.BH) ? (img * p.g.BH + h) * p.g.W + w : -1;
-    } else if (threadIdx.x < 192) {
+    }
+    // everything above is independent of what earlier kernels wrote and may overlap the kernel before
+    pdl_enter();
+    if (threadIdx.x == 0) {
+        mbar_expect_tx(&sh->w_full, (uint32_t)(taps * p.BN * p.KC * 2));
+        for (int tap = 0; tap < taps; tap++) tma_load_2d(wres + tap * p.wtile_bytes, &map_w, &sh->w_full, tap * p.KC, col0);
+        if ((int)blockIdx.x < p.g.n_px_tiles) {
+            load_raw(blockIdx.x, 0);
+            if (need_aux) load_aux(blockIdx.x, 0);
+        }
+    } else if (threadIdx.x >= 128 && threadIdx.x < 192) {
         const int c = threadIdx.x - 128;
         float sc = 0.f, sf = 0.f;
         if (p.in_mode == 0 && c < p.cin) bn_sc_sh(p.bn.gamma[c], p.bn.beta[c], p.bn.mean[c], p.bn.rstd[c], sc, sf);
@@ -312,20 +323,19 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
         // ---- epilogue, pass A: accumulator row (+ partner) -> output tile in shared memory
         if (warp < 4) {
             const int sr = sh->srow[etid];
-            const float *aux = reinterpret_cast<const float *>(auxb + b * p.aux_bytes);
-            float *outt = reinterpret_cast<float *>(outb);
+            const uint8_t *aux = auxb + b * p.aux_bytes;
 #pragma unroll 1
             for (int c = 0; c < p.BN; c += 16) {
                 float v[16];
                 tmem_ld16(tmem_d + lane_base + (uint32_t)c, v);
                 if (sr >= 0) {
-                    float4 *o = reinterpret_cast<float4 *>(outt + (size_t)sr * p.BN + c);
-                    const float4 *a = reinterpret_cast<const float4 *>(aux + (size_t)sr * p.BN + c);
+                    const int gbase = (c / p.GW) * p.group_bytes, j0 = (c % p.GW) >> 2;
 #pragma unroll
                     for (int j = 0; j < 4; j++) {
+                        const int off = gbase + sw_off(sr, j0 + j);
                         float4 r = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
                         if (e.mode == EPI_COUPLE) {
-                            const float4 pr = a[j];
+                            const float4 pr = *reinterpret_cast<const float4 *>(aux + off);
                             if (out_q == 0.f) {
                                 if (e.sign > 0) { r.x = pr.x + r.x; r.y = pr.y + r.y; r.z = pr.z + r.z; r.w = pr.w + r.w; }
                                 else { r.x = pr.x - r.x; r.y = pr.y - r.y; r.z = pr.z - r.z; r.w = pr.w - r.w; }
@@ -340,7 +350,7 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
                             r = make_float4(__int_as_float(__float2int_rn(r.x * out_s)), __int_as_float(__float2int_rn(r.y * out_s)),
                                             __int_as_float(__float2int_rn(r.z * out_s)), __int_as_float(__float2int_rn(r.w * out_s)));
                         }
-                        o[j] = r;
+                        *reinterpret_cast<float4 *>(outb + off) = r;
                     }
                 }
             }
@@ -349,20 +359,22 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
         tc_fence_before();       // the next tile's MMAs overwrite the accumulator
         __syncthreads();
         if (threadIdx.x == 0) {
-            tma_store_4d(&map_out, outb, col0, 0, h0, n0);
+            for (int g = 0; g < p.BN / p.GW; g++) tma_store_4d(&map_out, outb + g * p.group_bytes, col0 + g * p.GW, 0, h0, n0);
             tma_store_commit();
         }
         // ---- pass B: per-channel sums over the valid pixels of the tile (a prefix in the tile's pixel order)
         if (reducer) {
             int valid_px = p.g.BIMG > 1 ? (p.g.N - n0 < p.g.BIMG ? p.g.N - n0 : p.g.BIMG) * p.g.BH * p.g.W
                                         : (p.g.H - h0 < p.g.BH ? p.g.H - h0 : p.g.BH) * p.g.W;
-            const float *outt = reinterpret_cast<const float *>(outb) + quad * 4;
-            const float *aux = reinterpret_cast<const float *>(auxb + b * p.aux_bytes) + quad * 4;
+            const int qg = p.GW >> 2;                      // quads per column group
+            const int gbase = (quad / qg) * p.group_bytes, jq = quad % qg;
+            const uint8_t *aux = auxb + b * p.aux_bytes;
 #pragma unroll 2
             for (int pl = r0; pl < valid_px; pl += rpp) {
-                float4 v = *reinterpret_cast<const float4 *>(outt + (size_t)pl * p.BN);
+                const int off = gbase + sw_off(pl, jq);
+                float4 v = *reinterpret_cast<const float4 *>(outb + off);
                 if (e.mode == EPI_BNBWD) {
-                    float4 tt = *reinterpret_cast<const float4 *>(aux + (size_t)pl * p.BN);
+                    float4 tt = *reinterpret_cast<const float4 *>(aux + off);
                     if (t_q != 0.f) tt = make_float4(__int2float_rn(__float_as_int(tt.x)) * t_q, __int2float_rn(__float_as_int(tt.y)) * t_q,
                                                      __int2float_rn(__float_as_int(tt.z)) * t_q, __int2float_rn(__float_as_int(tt.w)) * t_q);
                     const float dx = fmaf(sc4.x, tt.x, sh4.x) > 0.f ? v.x : 0.f, dy = fmaf(sc4.y, tt.y, sh4.y) > 0.f ? v.y : 0.f;
@@ -427,7 +439,7 @@ bool fused_tile_geom(Geom g, TileGeom &t) {
     return true;
 }
 
-struct FusedShape { int KC, BN, n_tiles, NB, copy_bytes, wtile_bytes, a_bytes, raw_bytes, aux_bytes, smem, occ; TileGeom g; };
+struct FusedShape { int KC, BN, n_tiles, NB, GW, group_bytes, copy_bytes, wtile_bytes, a_bytes, raw_bytes, aux_bytes, smem, occ; TileGeom g; };
 
 bool fused_shape(Geom g, int cin, int cout, int k, int in_esize, int sm_count, FusedShape &s) {
     if ((k != 1 && k != 3) || cin % 8 || cout % 4 || cin < 8) return false;
@@ -444,11 +456,13 @@ bool fused_shape(Geom g, int cin, int cout, int k, int in_esize, int sm_count, F
     s.copy_bytes = (copy_rows * s.KC * 2 + 1023) & ~1023;
     const int npix = (s.g.BH + 2 * pad) * s.g.BIMG * (s.g.W + 2 * pad);
     s.a_bytes = k * s.copy_bytes > 8192 ? k * s.copy_bytes : 8192;      // also scratch of the final reduction
-    s.raw_bytes = (npix * cin * in_esize + 127) & ~127;
+    s.raw_bytes = (npix * cin * in_esize + 1023) & ~1023;
     for (;;) {
         s.n_tiles = (cout_pad + s.BN - 1) / s.BN;
         s.wtile_bytes = (s.BN * s.KC * 2 + 1023) & ~1023;
-        s.aux_bytes = (s.g.BH * s.g.BIMG * s.g.W * s.BN * 4 + 127) & ~127;
+        s.GW = s.BN % 32 == 0 ? 32 : 16;
+        s.group_bytes = (s.g.BH * s.g.BIMG * s.g.W * s.GW * 4 + 1023) & ~1023;
+        s.aux_bytes = (s.BN / s.GW) * s.group_bytes;
         auto smem_of = [&](int NB) { return 1024 + s.a_bytes + k * k * s.wtile_bytes + NB * (s.raw_bytes + s.aux_bytes) + s.aux_bytes +
                                             (int)sizeof(FusedShared) + npix * (s.KC / 8) * 16 + 64; };
         const int two_per_sm = 113 * 1024;
@@ -469,12 +483,12 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 
 // 4-D tensor map over an NHWC tensor of C channels: box = box_c channels x bw columns x bh rows x bimg images
 bool encode_nhwc(EncodeTiledFn enc, CUtensorMap *map, CUtensorMapDataType dt, int esize, const void *base, Geom g, int C,
-                 int box_c, int bw, int bh, int bimg) {
+                 int box_c, int bw, int bh, int bimg, CUtensorMapSwizzle swz = CU_TENSOR_MAP_SWIZZLE_NONE) {
     cuuint64_t dims[4] = {(cuuint64_t)C, (cuuint64_t)g.W, (cuuint64_t)g.H, (cuuint64_t)g.N};
     cuuint64_t strides[3] = {(cuuint64_t)C * esize, (cuuint64_t)g.W * C * esize, (cuuint64_t)g.H * g.W * C * esize};
     cuuint32_t box[4] = {(cuuint32_t)box_c, (cuuint32_t)bw, (cuuint32_t)bh, (cuuint32_t)bimg};
     cuuint32_t es[4] = {1, 1, 1, 1};
-    return enc(map, dt, 4, (void *)base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+    return enc(map, dt, 4, (void *)base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -510,14 +524,15 @@ bool run_fused(Exec &ex, const char *what, int in_mode, const void *in, float in
                            sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
         maps_ok = maps_ok && encode_nhwc(enc, &map_in, in_mode == 0 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
                                          in_mode == 0 ? 4 : 2, in, g, cin, cin, s.g.W + 2 * pad, s.g.BH + 2 * pad, s.g.BIMG);
-        maps_ok = maps_ok && encode_nhwc(enc, &map_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, out.p0, g, cout, s.BN, s.g.W, s.g.BH, s.g.BIMG);
+        const CUtensorMapSwizzle gsw = s.GW == 32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+        maps_ok = maps_ok && encode_nhwc(enc, &map_out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, out.p0, g, cout, s.GW, s.g.W, s.g.BH, s.g.BIMG, gsw);
         const float *aux = req.bnbwd ? req.bnbwd->t.p0 : (sign ? partner.p0 : out.p0);
-        maps_ok = maps_ok && encode_nhwc(enc, &map_aux, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, aux, g, cout, s.BN, s.g.W, s.g.BH, s.g.BIMG);
+        maps_ok = maps_ok && encode_nhwc(enc, &map_aux, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, aux, g, cout, s.GW, s.g.W, s.g.BH, s.g.BIMG, gsw);
         if (!maps_ok) { ex.failed = true; ex.ctx->err = std::string(what) + ": tensor map rejected"; ex.ws.release(m); return true; }
         FusedParams p;
         memset(&p, 0, sizeof p);
         p.k = k; p.KC = s.KC; p.cin = cin; p.BN = s.BN; p.NB = s.NB; p.copy_bytes = s.copy_bytes; p.wtile_bytes = s.wtile_bytes;
-        p.a_bytes = s.a_bytes; p.raw_bytes = s.raw_bytes; p.aux_bytes = s.aux_bytes; p.g = s.g;
+        p.a_bytes = s.a_bytes; p.raw_bytes = s.raw_bytes; p.aux_bytes = s.aux_bytes; p.GW = s.GW; p.group_bytes = s.group_bytes; p.g = s.g;
         p.in_mode = in_mode; p.in_q = in_q; p.bn = bn; p.a_out = a_out; p.status = ex.ctx->dev_status;
         EpiArgs &e = p.epi;
         e.mode = req.bnbwd ? EPI_BNBWD : (sign ? EPI_COUPLE : EPI_PLAIN);
@@ -529,7 +544,7 @@ bool run_fused(Exec &ex, const char *what, int in_mode, const void *in, float in
         static bool attr_set = false;
         if (!attr_set) { cudaFuncSetAttribute(conv_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024); attr_set = true; }
         dim3 grid((unsigned)ctas, (unsigned)s.n_tiles);
-        conv_fused_kernel<<<grid, kFThreads, s.smem, ex.stream>>>(map_w, map_in, map_aux, map_out, p);
+        launch(ex, conv_fused_kernel, grid, kFThreads, s.smem, map_w, map_in, map_aux, map_out, p);
         const double bytes = (double)g.P() * cin * (in_mode == 0 ? 4 : 2) + (double)g.P() * cout * (sign || req.bnbwd ? 8 : 4) +
                              (double)cout * taps * cin * 2 + (a_out ? (double)g.P() * cin * 2 : 0.0);
         ex.check(what, bytes, 2.0 * g.P() * cout * cin * taps);

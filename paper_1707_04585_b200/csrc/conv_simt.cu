@@ -83,6 +83,7 @@ struct EpiPlain {                             // row-major [M][N] (+ split-K sli
 
 template <int BN, class AL, class BL, class EP>
 __global__ __launch_bounds__(256) void gemm_simt_kernel(AL al, BL bl, EP ep, int M, int N, int K, int k_per_split) {
+    pdl_enter();
     constexpr int BM = 64, BK = 16, TN = BN / 16;
     __shared__ float As[BK][BM + 1];
     __shared__ float Bs[BK][BN + 1];
@@ -138,13 +139,13 @@ static void launch_gemm(Exec &ex, const char *what, AL al, BL bl, EP ep, int M, 
                         double bytes) {
     if (N <= 16) {
         dim3 grid((M + 63) / 64, (N + 15) / 16, splits);
-        gemm_simt_kernel<16, AL, BL, EP><<<grid, 256, 0, ex.stream>>>(al, bl, ep, M, N, K, k_per_split);
+        launch(ex, gemm_simt_kernel<16, AL, BL, EP>, grid, 256, 0, al, bl, ep, M, N, K, k_per_split);
     } else if (N <= 32) {
         dim3 grid((M + 63) / 64, (N + 31) / 32, splits);
-        gemm_simt_kernel<32, AL, BL, EP><<<grid, 256, 0, ex.stream>>>(al, bl, ep, M, N, K, k_per_split);
+        launch(ex, gemm_simt_kernel<32, AL, BL, EP>, grid, 256, 0, al, bl, ep, M, N, K, k_per_split);
     } else {
         dim3 grid((M + 63) / 64, (N + 63) / 64, splits);
-        gemm_simt_kernel<64, AL, BL, EP><<<grid, 256, 0, ex.stream>>>(al, bl, ep, M, N, K, k_per_split);
+        launch(ex, gemm_simt_kernel<64, AL, BL, EP>, grid, 256, 0, al, bl, ep, M, N, K, k_per_split);
     }
     ex.check(what, bytes, 2.0 * M * N * (double)K);
 }
@@ -182,6 +183,7 @@ void conv_dgrad_simt(Exec &ex, const void *gq, bool g_bf16, Geom gi, const Layer
 
 // fixed-order sum of split-K slices
 __global__ void splitk_reduce_kernel(const float *__restrict__ part, size_t n, int splits, float *__restrict__ out) {
+    pdl_enter();
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         float s = 0.f;
         for (int z = 0; z < splits; z++) s += part[(size_t)z * n + i];
@@ -213,7 +215,7 @@ void conv_wgrad_simt(Exec &ex, const void *gq, bool g_bf16, const void *a, bool 
         if (splits > 1) {
             size_t n = (size_t)M * N;
             int grid = (int)((n + 255) / 256); if (grid > ex.ctx->sm_count * 8) grid = ex.ctx->sm_count * 8;
-            splitk_reduce_kernel<<<grid, 256, 0, ex.stream>>>(part, n, splits, dW);
+            launch(ex, splitk_reduce_kernel, grid, 256, 0, part, n, splits, dW);
             ex.check("splitk_reduce");
         }
     }

@@ -82,6 +82,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_enter();             // the set-up above may overlap the kernel before; its outputs are read from here on
     const uint32_t tmem_d = sh->tmem_base;
     const int col0 = blockIdx.y * p.BN;
     const int pad = p.k / 2;
@@ -168,6 +169,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 // (rows = input channels, columns = output channels, taps mirrored)
 __global__ void pack_weights_kernel(const float *__restrict__ W, bf16 *__restrict__ out, int Co, int Ci, int k,
                                     int rows_pad, int cols_pad, int transposed) {
+    pdl_enter();
     const int taps = k * k;
     const size_t n = (size_t)rows_pad * taps * cols_pad;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
@@ -183,6 +185,7 @@ __global__ void pack_weights_kernel(const float *__restrict__ W, bf16 *__restric
 
 // all packs of a step in one launch: blockIdx.y walks the job table
 __global__ void pack_weights_batch_kernel(const PackJob *__restrict__ jobs) {
+    pdl_enter();
     const PackJob j = jobs[blockIdx.y];
     const int taps = j.k * j.k;
     const size_t n = (size_t)j.rows_pad * taps * j.cols_pad;
@@ -271,8 +274,8 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         if (!prepacked) {
             const size_t n = (size_t)rows_pad * taps * s.cin_pad;
             int grid = (int)((n + 255) / 256); if (grid > ex.ctx->sm_count * 4) grid = ex.ctx->sm_count * 4;
-            if (!transposed) pack_weights_kernel<<<grid, 256, 0, ex.stream>>>(Wsrc, wp, cout, cin, k, rows_pad, s.cin_pad, 0);
-            else pack_weights_kernel<<<grid, 256, 0, ex.stream>>>(Wsrc, wp, cin, cout, k, rows_pad, s.cin_pad, 1);
+            if (!transposed) launch(ex, pack_weights_kernel, grid, 256, 0, Wsrc, wp, cout, cin, k, rows_pad, s.cin_pad, 0);
+            else launch(ex, pack_weights_kernel, grid, 256, 0, Wsrc, wp, cin, cout, k, rows_pad, s.cin_pad, 1);
             ex.check("pack_weights", (double)n * 6);
         }
         CUtensorMap map_a, map_b;
@@ -310,7 +313,7 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         static bool attr_set = false;
         if (!attr_set) { cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024); attr_set = true; }
         dim3 grid((unsigned)ctas, (unsigned)s.n_tiles);
-        conv_tc_kernel<<<grid, kThreads, s.smem, ex.stream>>>(map_a, map_b, p);
+        launch(ex, conv_tc_kernel, grid, kThreads, s.smem, map_a, map_b, p);
         const double bytes = (double)gin.P() * cin * 2 + (double)g.P() * cout * (sign || req.bnbwd ? 8 : 4) + (double)cout * taps * cin * 2;
         ex.check(what, bytes, 2.0 * g.P() * cout * cin * taps);
     }
@@ -379,6 +382,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    pdl_enter();             // the set-up above may overlap the kernel before; its outputs are read from here on
     const uint32_t tmem_d = sh->tmem_base;
     const int pad = p.k / 2;
     const int tiles_per_img = p.tiles_per_img;
@@ -463,6 +467,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 // out[i] = sum over splits of part[z][i], in a fixed order: 8 interleaved groups of splits per
 // element, combined through shared memory (256 threads = 32 elements x 8 groups)
 __global__ void splitk_sum_kernel(const float *__restrict__ part, size_t n, int splits, float *__restrict__ out) {
+    pdl_enter();
     __shared__ float sm[8][33];
     const int e = threadIdx.x & 31, grp = threadIdx.x >> 5;
     const size_t i = (size_t)blockIdx.x * 32 + e;
@@ -549,11 +554,11 @@ bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer
         if (!attr_set) { cudaFuncSetAttribute(wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); attr_set = true; }
         const int smem = 1024 + p.stages * stage_bytes + (int)sizeof(TcShared) + 64;
         dim3 grid((unsigned)splits, (unsigned)m_chunks, (unsigned)n_tiles);
-        wgrad_tc_kernel<<<grid, kThreads, smem, ex.stream>>>(map_a, map_g, p);
+        launch(ex, wgrad_tc_kernel, grid, kThreads, smem, map_a, map_g, p);
         const double bytes = (double)gi.P() * L.cin * 2 + (double)go.P() * L.cout * 2 + (double)p.slice * 4 * (splits > 1 ? splits : 1);
         ex.check("conv_wgrad_tc", bytes, 2.0 * go.P() * L.cout * L.cin * taps);
         if (splits > 1) {
-            splitk_sum_kernel<<<(unsigned)((p.slice + 31) / 32), 256, 0, ex.stream>>>(part, p.slice, splits, dW);
+            launch(ex, splitk_sum_kernel, (unsigned)((p.slice + 31) / 32), 256, 0, part, p.slice, splits, dW);
             ex.check("splitk_sum", (double)p.slice * 4 * (splits + 1));
         }
     }
@@ -569,7 +574,7 @@ void tc_pack_now(Exec &ex, const float *W, bf16 *out, int cin, int cout, int k, 
     const PackJob j = tc_pack_job(W, out, cin, cout, k, transposed);
     const size_t n = (size_t)j.rows_pad * k * k * j.cols_pad;
     int grid = (int)((n + 255) / 256); if (grid > ex.ctx->sm_count * 4) grid = ex.ctx->sm_count * 4;
-    pack_weights_kernel<<<grid, 256, 0, ex.stream>>>(W, out, cout, cin, k, j.rows_pad, j.cols_pad, transposed ? 1 : 0);
+    launch(ex, pack_weights_kernel, grid, 256, 0, W, out, cout, cin, k, j.rows_pad, j.cols_pad, transposed ? 1 : 0);
     ex.check("pack_weights", (double)n * 6);
 }
 
@@ -593,6 +598,6 @@ PackJob tc_pack_job(const float *W, bf16 *out, int cin, int cout, int k, bool tr
 void tc_pack_batch(Exec &ex, const PackJob *jobs_dev, int n_jobs, double bytes) {
     if (ex.dry || n_jobs == 0) return;
     dim3 grid(96, (unsigned)n_jobs);
-    pack_weights_batch_kernel<<<grid, 256, 0, ex.stream>>>(jobs_dev);
+    launch(ex, pack_weights_batch_kernel, grid, 256, 0, jobs_dev);
     ex.check("pack_weights_batch", bytes);
 }

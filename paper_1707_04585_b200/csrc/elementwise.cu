@@ -69,6 +69,7 @@ static RedShape red_shape(size_t P, int C, int sm) {
 template <int MODE>   // 0: sum t, sum t^2 ; 1: sum db, sum db*xhat (BN+ReLU backward)
 __global__ void col_reduce_kernel(Pair t, const float *__restrict__ da, size_t P, int rows_per_cta, BnRef bn,
                                   float *__restrict__ part) {
+    pdl_enter();
     extern __shared__ float4 sm4[];
     const int C = t.C(), C4 = C / 4, SW = blockDim.x, RPP = blockDim.y;
     const int q = blockIdx.y * SW + threadIdx.x;
@@ -118,6 +119,7 @@ __device__ __forceinline__ void warp_sum2(const float *__restrict__ part, int ch
 
 __global__ void bn_stats_finalize(const float *__restrict__ part, int chunks, int C, double invP, float eps,
                                   float *mean, float *rstd) {
+    pdl_enter();
     const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (c >= C) return;
     double s, ss;
@@ -133,6 +135,7 @@ __global__ void bn_stats_finalize(const float *__restrict__ part, int chunks, in
 __global__ void bn_bwd_finalize(const float *__restrict__ part, int chunks, int C, double invP,
                                 const float *__restrict__ gamma, const float *__restrict__ rstd,
                                 float *dgamma, float *dbeta, float *coef) {
+    pdl_enter();
     const int c = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (c >= C) return;
     double s, ss;
@@ -158,9 +161,9 @@ void bn_stats(Exec &ex, Pair t, size_t P, Moments mo) {
     float *part = ex.ws.get<float>((size_t)r.chunks * 2 * C);
     if (!ex.dry) {
         dim3 grid(r.chunks, r.slabs), block(r.SW, r.RPP);
-        col_reduce_kernel<0><<<grid, block, (size_t)r.SW * r.RPP * 32, ex.stream>>>(t, nullptr, P, r.rows_per_cta, BnRef{}, part);
+        launch(ex, col_reduce_kernel<0>, grid, block, (size_t)r.SW * r.RPP * 32, t, nullptr, P, r.rows_per_cta, BnRef{}, part);
         ex.check("bn_stats_partial", (double)P * C * 4);
-        bn_stats_finalize<<<cdiv((size_t)C * 32, 128), 128, 0, ex.stream>>>(part, r.chunks, C, 1.0 / (double)P, ex.eps, mo.mean, mo.rstd);
+        launch(ex, bn_stats_finalize, cdiv((size_t)C * 32, 128), 128, 0, part, r.chunks, C, 1.0 / (double)P, ex.eps, mo.mean, mo.rstd);
         ex.check("bn_stats_finalize");
     }
     ex.ws.release(m);
@@ -168,6 +171,7 @@ void bn_stats(Exec &ex, Pair t, size_t P, Moments mo) {
 
 template <class TO>
 __global__ void bn_relu_apply_kernel(Pair t, size_t nquads, int C4, BnRef bn, TO *__restrict__ a) {
+    pdl_enter();
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
         size_t row = i / C4; int q = (int)(i - row * C4);
         float4 v = t.ld4(row, q * 4), sc, sh, mu, rs;
@@ -186,8 +190,8 @@ static int ew_grid(size_t n, int sm) {
 void bn_relu_apply(Exec &ex, Pair t, size_t P, BnRef bn, void *a, bool a_bf16) {
     if (ex.dry) return;
     const int C4 = t.C() / 4; size_t nq = P * C4;
-    if (a_bf16) bn_relu_apply_kernel<bf16><<<ew_grid(nq, ex.ctx->sm_count), 256, 0, ex.stream>>>(t, nq, C4, bn, (bf16 *)a);
-    else bn_relu_apply_kernel<float><<<ew_grid(nq, ex.ctx->sm_count), 256, 0, ex.stream>>>(t, nq, C4, bn, (float *)a);
+    if (a_bf16) launch(ex, bn_relu_apply_kernel<bf16>, ew_grid(nq, ex.ctx->sm_count), 256, 0, t, nq, C4, bn, (bf16 *)a);
+    else launch(ex, bn_relu_apply_kernel<float>, ew_grid(nq, ex.ctx->sm_count), 256, 0, t, nq, C4, bn, (float *)a);
     ex.check("bn_relu_apply", (double)P * t.C() * (a_bf16 ? 6 : 8));
 }
 
@@ -198,6 +202,7 @@ template <class TO, int OUT, bool CAST>
 __global__ void bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, size_t nquads, int C4, BnRef bn,
                                          const float *__restrict__ coef, TO *__restrict__ out, Pair add, Pair outp,
                                          bf16 *__restrict__ cast) {
+    pdl_enter();
     const int C = C4 * 4;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
         size_t row = i / C4; int q = (int)(i - row * C4), c = q * 4;
@@ -228,21 +233,21 @@ void bn_relu_bwd(Exec &ex, const float *da, Pair t, size_t P, BnRef bn, float *d
     if (!ex.dry) {
         if (!sums_done) {
             dim3 grid(r.chunks, r.slabs), block(r.SW, r.RPP);
-            col_reduce_kernel<1><<<grid, block, (size_t)r.SW * r.RPP * 32, ex.stream>>>(t, da, P, r.rows_per_cta, bn, part);
+            launch(ex, col_reduce_kernel<1>, grid, block, (size_t)r.SW * r.RPP * 32, t, da, P, r.rows_per_cta, bn, part);
             ex.check("bn_bwd_partial", (double)P * C * 8);
-            bn_bwd_finalize<<<cdiv((size_t)C * 32, 128), 128, 0, ex.stream>>>(part, r.chunks, C, 1.0 / (double)P, bn.gamma, bn.rstd, dgamma, dbeta, coef);
+            launch(ex, bn_bwd_finalize, cdiv((size_t)C * 32, 128), 128, 0, part, r.chunks, C, 1.0 / (double)P, bn.gamma, bn.rstd, dgamma, dbeta, coef);
             ex.check("bn_bwd_finalize");
         }
         size_t nq = P * C4; int g = ew_grid(nq, ex.ctx->sm_count);
 #define RV_ARGS da, t, nq, C4, bn, coef
         if (out_pair.p0 && add.p0) {
-            if (out_cast) bn_relu_bwd_apply_kernel<float, 2, true><<<g, 256, 0, ex.stream>>>(RV_ARGS, nullptr, add, out_pair, out_cast);
-            else bn_relu_bwd_apply_kernel<float, 2, false><<<g, 256, 0, ex.stream>>>(RV_ARGS, nullptr, add, out_pair, nullptr);
+            if (out_cast) launch(ex, bn_relu_bwd_apply_kernel<float, 2, true>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, out_cast);
+            else launch(ex, bn_relu_bwd_apply_kernel<float, 2, false>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, nullptr);
         } else if (out_pair.p0) {
-            if (out_cast) bn_relu_bwd_apply_kernel<float, 1, true><<<g, 256, 0, ex.stream>>>(RV_ARGS, nullptr, add, out_pair, out_cast);
-            else bn_relu_bwd_apply_kernel<float, 1, false><<<g, 256, 0, ex.stream>>>(RV_ARGS, nullptr, add, out_pair, nullptr);
-        } else if (out_bf16) bn_relu_bwd_apply_kernel<bf16, 0, false><<<g, 256, 0, ex.stream>>>(RV_ARGS, (bf16 *)out_single, add, out_pair, nullptr);
-        else bn_relu_bwd_apply_kernel<float, 0, false><<<g, 256, 0, ex.stream>>>(RV_ARGS, (float *)out_single, add, out_pair, nullptr);
+            if (out_cast) launch(ex, bn_relu_bwd_apply_kernel<float, 1, true>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, out_cast);
+            else launch(ex, bn_relu_bwd_apply_kernel<float, 1, false>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, nullptr);
+        } else if (out_bf16) launch(ex, bn_relu_bwd_apply_kernel<bf16, 0, false>, g, 256, 0, RV_ARGS, (bf16 *)out_single, add, out_pair, nullptr);
+        else launch(ex, bn_relu_bwd_apply_kernel<float, 0, false>, g, 256, 0, RV_ARGS, (float *)out_single, add, out_pair, nullptr);
 #undef RV_ARGS
         ex.check("bn_relu_bwd_apply", (double)P * C * ((out_pair.p0 ? (add.p0 ? 16 : 12) : (out_bf16 ? 10 : 12)) + (out_cast ? 2 : 0)));
     }
@@ -251,6 +256,7 @@ void bn_relu_bwd(Exec &ex, const float *da, Pair t, size_t P, BnRef bn, float *d
 
 template <class TO>
 __global__ void concat_cast_kernel(Pair src, size_t nquads, int C4, TO *__restrict__ dst) {
+    pdl_enter();
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
         size_t row = i / C4; int q = (int)(i - row * C4);
         st4(dst + i * 4, src.ld4(row, q * 4));
@@ -260,13 +266,14 @@ __global__ void concat_cast_kernel(Pair src, size_t nquads, int C4, TO *__restri
 void concat_cast(Exec &ex, Pair src, size_t P, void *dst, bool dst_bf16) {
     if (ex.dry) return;
     const int C4 = src.C() / 4; size_t nq = P * C4; int g = ew_grid(nq, ex.ctx->sm_count);
-    if (dst_bf16) concat_cast_kernel<bf16><<<g, 256, 0, ex.stream>>>(src, nq, C4, (bf16 *)dst);
-    else concat_cast_kernel<float><<<g, 256, 0, ex.stream>>>(src, nq, C4, (float *)dst);
+    if (dst_bf16) launch(ex, concat_cast_kernel<bf16>, g, 256, 0, src, nq, C4, (bf16 *)dst);
+    else launch(ex, concat_cast_kernel<float>, g, 256, 0, src, nq, C4, (float *)dst);
     ex.check("concat_cast", (double)P * src.C() * (dst_bf16 ? 6 : 8));
 }
 
 // ------------------------------------------------------------------ max-pool 3x3 stride 2 pad 1 (NHWC)
 __global__ void maxpool_fwd_kernel(const float *__restrict__ in, float *__restrict__ out, int N, int H, int W, int C4, int Ho, int Wo) {
+    pdl_enter();
     size_t n = (size_t)N * Ho * Wo * C4;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         int q = (int)(i % C4); size_t p = i / C4;
@@ -286,6 +293,7 @@ __global__ void maxpool_fwd_kernel(const float *__restrict__ in, float *__restri
 // each input element visits the (at most four) windows that cover it, in a fixed order.
 __global__ void maxpool_bwd_kernel(const float *__restrict__ in, const float *__restrict__ dout, float *__restrict__ din,
                                    int N, int H, int W, int C, int Ho, int Wo) {
+    pdl_enter();
     size_t n = (size_t)N * H * W * C;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         int c = (int)(i % C); size_t p = i / C;
@@ -316,19 +324,20 @@ void maxpool_fwd(Exec &ex, const float *in, float *out, int N, int H, int W, int
     if (ex.dry) return;
     int Ho = conv_out(H, 3, 2), Wo = conv_out(W, 3, 2);
     size_t n = (size_t)N * Ho * Wo * (C / 4);
-    maxpool_fwd_kernel<<<ew_grid(n, ex.ctx->sm_count), 256, 0, ex.stream>>>(in, out, N, H, W, C / 4, Ho, Wo);
+    launch(ex, maxpool_fwd_kernel, ew_grid(n, ex.ctx->sm_count), 256, 0, in, out, N, H, W, C / 4, Ho, Wo);
     ex.check("maxpool_fwd");
 }
 void maxpool_bwd(Exec &ex, const float *in, const float *dout, float *din, int N, int H, int W, int C) {
     if (ex.dry) return;
     int Ho = conv_out(H, 3, 2), Wo = conv_out(W, 3, 2);
     size_t n = (size_t)N * H * W * C;
-    maxpool_bwd_kernel<<<ew_grid(n, ex.ctx->sm_count), 256, 0, ex.stream>>>(in, dout, din, N, H, W, C, Ho, Wo);
+    launch(ex, maxpool_bwd_kernel, ew_grid(n, ex.ctx->sm_count), 256, 0, in, dout, din, N, H, W, C, Ho, Wo);
     ex.check("maxpool_bwd");
 }
 
 // ------------------------------------------------------------------ head: avgpool -> FC -> softmax CE -> argmax
 __global__ void avgpool_kernel(Pair y, int HW, float *__restrict__ feat) {
+    pdl_enter();
     extern __shared__ float4 sm4[];
     const int C = y.C(), C4 = C / 4, SW = blockDim.x, RPP = blockDim.y;
     const int q = blockIdx.y * SW + threadIdx.x, n = blockIdx.x;
@@ -352,6 +361,7 @@ __global__ void avgpool_kernel(Pair y, int HW, float *__restrict__ feat) {
 // one warp per (n,k)
 __global__ void fc_fwd_kernel(const float *__restrict__ feat, const float *__restrict__ Wfc, const float *__restrict__ bfc,
                               int N, int C, int K, float *__restrict__ logits) {
+    pdl_enter();
     int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (warp >= N * K) return;
     int n = warp / K, k = warp - n * K;
@@ -364,6 +374,7 @@ __global__ void fc_fwd_kernel(const float *__restrict__ feat, const float *__res
 // one warp per sample: stable log-sum-exp, dlogits = (softmax - onehot)/N, arg-max (lowest index on ties)
 __global__ void softmax_ce_kernel(const float *__restrict__ logits, const int32_t *__restrict__ labels, int N, int K,
                                   float *__restrict__ dlogits, float *__restrict__ loss_n, int32_t *__restrict__ pred) {
+    pdl_enter();
     int n = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (n >= N) return;
     const float *z = logits + (size_t)n * K;
@@ -383,6 +394,7 @@ __global__ void softmax_ce_kernel(const float *__restrict__ logits, const int32_
 }
 
 __global__ void mean_kernel(const float *__restrict__ v, int N, float *out) {
+    pdl_enter();
     if (threadIdx.x == 0 && blockIdx.x == 0) {
         double s = 0; for (int i = 0; i < N; i++) s += v[i];
         *out = (float)(s / N);
@@ -398,13 +410,13 @@ void head_fwd(Exec &ex, Pair y, int N, int HW, const float *Wfc, const float *bf
     if (!ex.dry) {
         int C4 = C / 4, SW = C4 < 128 ? C4 : 128, RPP = 256 / SW; if (RPP < 1) RPP = 1;
         dim3 grid(N, cdiv(C4, SW)), block(SW, RPP);
-        avgpool_kernel<<<grid, block, (size_t)SW * RPP * 16, ex.stream>>>(y, HW, feat);
+        launch(ex, avgpool_kernel, grid, block, (size_t)SW * RPP * 16, y, HW, feat);
         ex.check("avgpool");
-        fc_fwd_kernel<<<cdiv((size_t)N * K * 32, 256), 256, 0, ex.stream>>>(feat, Wfc, bfc, N, C, K, logits);
+        launch(ex, fc_fwd_kernel, cdiv((size_t)N * K * 32, 256), 256, 0, feat, Wfc, bfc, N, C, K, logits);
         ex.check("fc_fwd");
-        softmax_ce_kernel<<<cdiv((size_t)N * 32, 256), 256, 0, ex.stream>>>(logits, labels, N, K, dlogits, loss_n, pred);
+        launch(ex, softmax_ce_kernel, cdiv((size_t)N * 32, 256), 256, 0, logits, labels, N, K, dlogits, loss_n, pred);
         ex.check("softmax_ce");
-        mean_kernel<<<1, 32, 0, ex.stream>>>(loss_n, N, loss);
+        launch(ex, mean_kernel, 1, 32, 0, loss_n, N, loss);
         ex.check("loss_mean");
     }
     ex.ws.release(m);
@@ -412,6 +424,7 @@ void head_fwd(Exec &ex, Pair y, int N, int HW, const float *Wfc, const float *bf
 
 __global__ void fc_wgrad_kernel(const float *__restrict__ dlogits, const float *__restrict__ feat, int N, int C, int K,
                                 float *__restrict__ dW, float *__restrict__ db) {
+    pdl_enter();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i < (size_t)K * C) {
         int k = (int)(i / C), c = (int)(i - (size_t)k * C);
@@ -423,6 +436,7 @@ __global__ void fc_wgrad_kernel(const float *__restrict__ dlogits, const float *
 }
 __global__ void fc_dgrad_kernel(const float *__restrict__ dlogits, const float *__restrict__ Wfc, int N, int C, int K,
                                 float scale, float *__restrict__ dfeat) {
+    pdl_enter();
     size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= (size_t)N * C) return;
     int n = (int)(i / C), c = (int)(i - (size_t)n * C);
@@ -431,6 +445,7 @@ __global__ void fc_dgrad_kernel(const float *__restrict__ dlogits, const float *
     dfeat[i] = s * scale;
 }
 __global__ void avgpool_bwd_kernel(const float *__restrict__ dfeat, Pair dy, size_t nquads, int C4, int HW) {
+    pdl_enter();
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
         size_t row = i / C4; int q = (int)(i - row * C4); size_t n = row / HW;
         st4(dy.at(row, q * 4), ld4(dfeat + n * C4 * 4 + q * 4));
@@ -442,12 +457,12 @@ void head_bwd(Exec &ex, Pair dy, int N, int HW, const float *Wfc, const float *f
     const int C = dy.C();
     ex.flops += 4ull * N * C * K;
     if (ex.dry) return;
-    fc_wgrad_kernel<<<cdiv((size_t)K * C, 256), 256, 0, ex.stream>>>(dlogits, feat, N, C, K, dWfc, dbfc);
+    launch(ex, fc_wgrad_kernel, cdiv((size_t)K * C, 256), 256, 0, dlogits, feat, N, C, K, dWfc, dbfc);
     ex.check("fc_wgrad");
-    fc_dgrad_kernel<<<cdiv((size_t)N * C, 256), 256, 0, ex.stream>>>(dlogits, Wfc, N, C, K, 1.f / (float)HW, dfeat);
+    launch(ex, fc_dgrad_kernel, cdiv((size_t)N * C, 256), 256, 0, dlogits, Wfc, N, C, K, 1.f / (float)HW, dfeat);
     ex.check("fc_dgrad");
     size_t nq = (size_t)N * HW * (C / 4);
-    avgpool_bwd_kernel<<<ew_grid(nq, ex.ctx->sm_count), 256, 0, ex.stream>>>(dfeat, dy, nq, C / 4, HW);
+    launch(ex, avgpool_bwd_kernel, ew_grid(nq, ex.ctx->sm_count), 256, 0, dfeat, dy, nq, C / 4, HW);
     ex.check("avgpool_bwd");
 }
 
@@ -455,6 +470,7 @@ void head_bwd(Exec &ex, Pair dy, int N, int HW, const float *Wfc, const float *f
 __global__ void sgd_kernel(float *__restrict__ p, const float *__restrict__ g, float *__restrict__ v, size_t n,
                            const uint32_t *__restrict__ seg_end, const uint8_t *__restrict__ seg_decay, int n_seg,
                            float lr, float mu, float wd) {
+    pdl_enter();
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         int lo = 0, hi = n_seg - 1;                  // first segment whose end is > i
         while (lo < hi) { int mid = (lo + hi) >> 1; if (seg_end[mid] > i) hi = mid; else lo = mid + 1; }
@@ -468,11 +484,12 @@ __global__ void sgd_kernel(float *__restrict__ p, const float *__restrict__ g, f
 void sgd_update(Exec &ex, float *params, const float *grads, float *mom, size_t n, const uint32_t *seg_end,
                 const uint8_t *seg_decay, int n_seg, float lr, float momentum, float wd) {
     if (ex.dry) return;
-    sgd_kernel<<<ew_grid(n, ex.ctx->sm_count), 256, 0, ex.stream>>>(params, grads, mom, n, seg_end, seg_decay, n_seg, lr, momentum, wd);
+    launch(ex, sgd_kernel, ew_grid(n, ex.ctx->sm_count), 256, 0, params, grads, mom, n, seg_end, seg_decay, n_seg, lr, momentum, wd);
     ex.check("sgd", (double)n * 20);
 }
 
 __global__ void max_abs_diff_kernel(const float *__restrict__ a, const float *__restrict__ b, size_t n, float q, float *out) {
+    pdl_enter();
     float m = 0.f;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         if (q == 0.f) m = fmaxf(m, fabsf(a[i] - b[i]));
@@ -483,7 +500,7 @@ __global__ void max_abs_diff_kernel(const float *__restrict__ a, const float *__
 }
 void max_abs_diff(Exec &ex, const float *a, const float *b, size_t n, float q, float *out) {
     if (ex.dry) return;
-    max_abs_diff_kernel<<<ew_grid(n, ex.ctx->sm_count), 256, 0, ex.stream>>>(a, b, n, q, out);
+    launch(ex, max_abs_diff_kernel, ew_grid(n, ex.ctx->sm_count), 256, 0, a, b, n, q, out);
     ex.check("max_abs_diff");
 }
 void fill_zero(Exec &ex, void *p, size_t bytes) {
@@ -492,6 +509,7 @@ void fill_zero(Exec &ex, void *p, size_t bytes) {
 }
 
 __global__ void upsample_zero_kernel(const uint4 *__restrict__ in, uint4 *__restrict__ out, int N, int Ho, int Wo, int C8) {
+    pdl_enter();
     const size_t n = (size_t)N * Ho * 2 * Wo * 2 * C8;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
         const int c = (int)(i % C8); size_t p = i / C8;
@@ -505,6 +523,6 @@ __global__ void upsample_zero_kernel(const uint4 *__restrict__ in, uint4 *__rest
 void upsample_zero_bf16(Exec &ex, const bf16 *in, bf16 *out, int N, int Ho, int Wo, int C) {
     if (ex.dry) return;
     const size_t n = (size_t)N * Ho * 2 * Wo * 2 * (C / 8);
-    upsample_zero_kernel<<<ew_grid(n, ex.ctx->sm_count), 256, 0, ex.stream>>>((const uint4 *)in, (uint4 *)out, N, Ho, Wo, C / 8);
+    launch(ex, upsample_zero_kernel, ew_grid(n, ex.ctx->sm_count), 256, 0, (const uint4 *)in, (uint4 *)out, N, Ho, Wo, C / 8);
     ex.check("upsample_zero", (double)n * 16 * 1.25);
 }

@@ -34,7 +34,51 @@ def load_peaks():
 # fp32 FMA peak of the CUDA cores: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (max SM clock)
 ALU_FP32_TFLOPS = 148 * 128 * 2 * 1.965e9 / 1e12
 
-ALU_KERNELS = ("conv_fprop_simt", "conv_dgrad_simt", "conv_wgrad_simt")   # fp32 CUDA-core GEMMs
+ALU_KERNELS = ("gemm_simt_kernel",)   # fp32 CUDA-core GEMMs
+
+# profile record name (one per call site class) -> the CUDA kernel that runs it, and the source files it is built from
+DEVICE_KERNEL = {
+    "conv_fprop_fused": "conv_fused_kernel", "conv_dgrad_fused": "conv_fused_kernel",
+    "conv_fprop_tc": "conv_tc_kernel", "conv_dgrad_tc": "conv_tc_kernel", "conv_wgrad_tc": "wgrad_tc_kernel",
+    "conv_fprop_simt": "gemm_simt_kernel", "conv_dgrad_simt": "gemm_simt_kernel", "conv_wgrad_simt": "gemm_simt_kernel",
+    "bn_stats_partial": "col_reduce_kernel", "bn_bwd_partial": "col_reduce_kernel",
+}
+KERNEL_SOURCES = {
+    "conv_fused_kernel": ("conv_fused.cu", "conv_epilogue.cuh", "tc_ptx.cuh"),
+    "conv_tc_kernel": ("conv_tc.cu", "conv_epilogue.cuh", "tc_ptx.cuh"),
+    "wgrad_tc_kernel": ("conv_tc.cu", "tc_ptx.cuh"),
+}
+
+
+def by_device_kernel(prof):
+    out = {}
+    for name, v in prof.items():
+        k = DEVICE_KERNEL.get(name, name)
+        a = out.setdefault(k, dict(launches=0, ms=0.0, bytes=0.0, flops=0.0))
+        for f in a:
+            a[f] += v[f]
+    return out
+
+
+def source_digest(kernel):
+    import hashlib
+    h = hashlib.sha256()
+    for f in KERNEL_SOURCES.get(kernel, ()):
+        with open(os.path.join(ROOT, "paper_1707_04585_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def measured_traffic(kernel, workload):
+    """DRAM bytes per launch of `kernel` on `workload` from the ncu capture summarised under profiles/,
+    or None if there is none or the kernel's sources have changed since it was taken."""
+    p = os.path.join(ROOT, "profiles", "dram_traffic.txt")
+    if not os.path.exists(p):
+        return None
+    rec = json.load(open(p)).get(workload, {}).get(kernel)
+    if not rec or rec.get("source_digest") != source_digest(kernel):
+        return None
+    return rec["dram_bytes_per_launch"]
 
 
 def binding_roofline(name, rec, peaks):
@@ -243,6 +287,7 @@ def run_ours(args, cfg):
     if rank == 0:
         peaks = load_peaks()
         total_images = rcfg.N * world * args.steps
+        prof = by_device_kernel(prof)
         tot = sum(v["ms"] for v in prof.values()) or 1.0
         top = max(prof.items(), key=lambda kv: kv[1]["ms"])
         name, rec = top
@@ -254,7 +299,7 @@ def run_ours(args, cfg):
             ach, peak, runit = rec["flops"] / rec["launches"] / avg_s / 1e12, peaks["tc_sustained"], "TFLOP/s"
         else:
             ach, peak, runit = rec["flops"] / rec["launches"] / avg_s / 1e12, ALU_FP32_TFLOPS, "TFLOP/s"
-        roof = dict(bound=bound, achieved=ach, peak=peak, unit=runit, frac=ach / peak, traffic=None, kernel=name,
+        roof = dict(bound=bound, achieved=ach, peak=peak, unit=runit, frac=ach / peak, traffic=measured_traffic(name, cfg.name), kernel=name,
                     kernel_share=rec["ms"] / tot, avg_launch_us=avg_s * 1e6, peak_source=peaks["source"],
                     kernels={k: dict(launches=v["launches"] // psteps, ms_per_step=v["ms"] / psteps, share=v["ms"] / tot,
                                      gbs=(v["bytes"] / (v["ms"] * 1e-3) / 1e9) if v["ms"] > 0 else None,

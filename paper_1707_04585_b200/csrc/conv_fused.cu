@@ -177,6 +177,22 @@ __device__ __forceinline__ void build_tile(const FusedParams &p, const FusedShar
     }
 }
 
+// One tile's place in the tensor.  Tiles are stepped by the grid size without divisions.
+struct TilePos { int t, n0, h0, hidx; };
+struct TileStep { int gq, gr; };     // grid size = gq whole images + gr row tiles (BIMG == 1)
+__device__ __forceinline__ void tile_first(const TileGeom &g, int t, TilePos &tp) {
+    tp.t = t;
+    if (g.BIMG > 1) { tp.n0 = t * g.BIMG; tp.h0 = 0; tp.hidx = 0; }
+    else { tp.n0 = t / g.tiles_per_img; tp.hidx = t - tp.n0 * g.tiles_per_img; tp.h0 = tp.hidx * g.BH; }
+}
+__device__ __forceinline__ void tile_next(const TileGeom &g, const TileStep &st, int G, TilePos &tp) {
+    tp.t += G;
+    if (g.BIMG > 1) { tp.n0 += G * g.BIMG; return; }
+    tp.n0 += st.gq; tp.hidx += st.gr;
+    if (tp.hidx >= g.tiles_per_img) { tp.hidx -= g.tiles_per_img; tp.n0++; }
+    tp.h0 = tp.hidx * g.BH;
+}
+
 __global__ void __launch_bounds__(kFThreads, 2)
 conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_constant__ CUtensorMap map_in,
                   const __grid_constant__ CUtensorMap map_aux, const __grid_constant__ CUtensorMap map_out, const FusedParams p) {
@@ -206,19 +222,23 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
     const uint32_t raw_tx = (uint32_t)(npix * p.cin * (p.in_mode == 0 ? 4 : 2));
     const uint32_t aux_tx = (uint32_t)(tile_px * p.BN * 4);
 
-    auto load_raw = [&](int t, int b) {                 // thread 0
-        int n0, h0;
-        tile_origin(p.g, t, n0, h0);
+    const int G = (int)gridDim.x, NT = p.g.n_px_tiles;
+    TileStep step;
+    step.gq = p.g.BIMG > 1 ? 0 : G / p.g.tiles_per_img;
+    step.gr = p.g.BIMG > 1 ? 0 : G - step.gq * p.g.tiles_per_img;
+    auto load_raw = [&](const TilePos &tp, int b) {     // thread 0
         mbar_expect_tx(&sh->raw_full[b], raw_tx);
-        tma_load_4d(rawb + b * p.raw_bytes, &map_in, &sh->raw_full[b], 0, -pad, h0 - pad, n0);
+        tma_load_4d(rawb + b * p.raw_bytes, &map_in, &sh->raw_full[b], 0, -pad, tp.h0 - pad, tp.n0);
     };
-    auto load_aux = [&](int t, int b) {
-        int n0, h0;
-        tile_origin(p.g, t, n0, h0);
+    auto load_aux = [&](const TilePos &tp, int b) {
         mbar_expect_tx(&sh->aux_full[b], aux_tx);
         for (int g = 0; g < p.BN / p.GW; g++)
-            tma_load_4d(auxb + b * p.aux_bytes + g * p.group_bytes, &map_aux, &sh->aux_full[b], col0 + g * p.GW, 0, h0, n0);
+            tma_load_4d(auxb + b * p.aux_bytes + g * p.group_bytes, &map_aux, &sh->aux_full[b], col0 + g * p.GW, 0, tp.h0, tp.n0);
     };
+    TilePos cur, nx1, nx2;             // this tile, the next one and the one after
+    tile_first(p.g, blockIdx.x, cur);
+    nx1 = cur; tile_next(p.g, step, G, nx1);
+    nx2 = nx1; tile_next(p.g, step, G, nx2);
     // byte offset of float4 j of pixel r inside a column group: rows of 128 (64) bytes, 16-byte chunks XORed with
     // address bits 7.. as the TMA swizzle does, so that a thread per row touches all banks
     const int row_b = p.GW * 4;
@@ -245,9 +265,10 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
     if (threadIdx.x == 0) {
         mbar_expect_tx(&sh->w_full, (uint32_t)(taps * p.BN * p.KC * 2));
         for (int tap = 0; tap < taps; tap++) tma_load_2d(wres + tap * p.wtile_bytes, &map_w, &sh->w_full, tap * p.KC, col0);
-        if ((int)blockIdx.x < p.g.n_px_tiles) {
-            load_raw(blockIdx.x, 0);
-            if (need_aux) load_aux(blockIdx.x, 0);
+        if (cur.t < NT) {
+            load_raw(cur, 0);
+            if (need_aux) load_aux(cur, 0);
+            if (p.NB == 2 && nx1.t < NT) load_raw(nx1, 1);
         }
     } else if (threadIdx.x >= 128 && threadIdx.x < 192) {
         const int c = threadIdx.x - 128;
@@ -285,15 +306,11 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
     bool ok = true;
     int ti = 0;
 #pragma unroll 1
-    for (int t = blockIdx.x; t < p.g.n_px_tiles; t += gridDim.x, ti++) {
+    for (; cur.t < NT; ti++) {
         const int b = ti % p.NB; const uint32_t u = ti / p.NB;
-        const int tn = t + gridDim.x;
-        int n0, h0;
-        tile_origin(p.g, t, n0, h0);
-        if (threadIdx.x == 0) {
-            if (p.NB == 2 && tn < p.g.n_px_tiles) { load_raw(tn, b ^ 1); if (need_aux) load_aux(tn, b ^ 1); }
-            ok = mbar_wait(&sh->raw_full[b], u & 1);
-        }
+        const int n0 = cur.n0, h0 = cur.h0;
+        // with two buffers the loads of the tiles ahead are issued while this tile's MMAs run (below)
+        if (threadIdx.x == 0) ok = mbar_wait(&sh->raw_full[b], u & 1);
         ok = __syncthreads_and(ok);
         if (!ok) break;
         // ---- build the operand
@@ -302,7 +319,7 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
         fence_proxy_async();
         __syncthreads();
         if (threadIdx.x == 0) {
-            if (p.NB == 1 && tn < p.g.n_px_tiles) load_raw(tn, 0);        // the raw buffer is free again
+            if (p.NB == 1 && nx1.t < NT) load_raw(nx1, 0);        // the raw buffer is free again
             if (ti == 0 && !mbar_wait(&sh->w_full, 0)) ok = false;
             tc_fence_after();
             const uint32_t idesc = instr_desc(p.BN);
@@ -314,6 +331,11 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
                 mma_bf16(tmem_d, d.x, d.y, idesc, i ? 1u : 0u);
             }
             mma_commit(&sh->mma_done);
+            if (p.NB == 2) {
+                // this tile's raw buffer has been consumed, and the other partner buffer was last read by the epilogue before
+                if (nx2.t < NT) load_raw(nx2, b);
+                if (need_aux && nx1.t < NT) load_aux(nx1, b ^ 1);
+            }
             tma_store_wait_read();                       // the previous tile's store has read the output buffer
             ok = ok && mbar_wait(&sh->mma_done, ti & 1) && (!need_aux || mbar_wait(&sh->aux_full[b], u & 1));
         }
@@ -390,8 +412,12 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
                 }
             }
         }
-        __syncthreads();         // the partner buffer and (once its store has read it) the output buffer are free
-        if (threadIdx.x == 0 && p.NB == 1 && need_aux && tn < p.g.n_px_tiles) load_aux(tn, 0);
+        if (p.NB == 1) {
+            __syncthreads();     // the partner buffer is free
+            if (threadIdx.x == 0 && need_aux && nx1.t < NT) load_aux(nx1, 0);
+        }
+        cur = nx1; nx1 = nx2;
+        tile_next(p.g, step, G, nx2);
     }
     if (threadIdx.x == 0) tma_store_wait_all();
     if (ok && e.part) {

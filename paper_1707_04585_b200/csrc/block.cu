@@ -15,7 +15,7 @@
 // dispatch: tensor-core kernels take the shapes they support in mode 0, the fp32 kernels the rest
 bool conv_fprop_tc(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign, Moments *stats);
 bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, const BnBwdReq *bb);
-bool conv_wgrad_tc(Exec &ex, const void *g, const void *a, Geom gi, const Layer &L, float *dW);
+bool conv_wgrad_tc(Exec &ex, const void *g, const void *a, Geom gi, const Layer &L, float *dW, float *scratch, size_t *need);
 // one kernel for BN -> ReLU -> conv (at most 64 input channels, stride 1); likewise the data gradient of such a layer
 bool conv_fprop_fused(Exec &ex, Pair t, BnRef bn, Geom gi, const Layer &L, Pair out, Pair partner, int sign, Moments *stats, bf16 *a_out);
 bool conv_dgrad_fused(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, const BnBwdReq *bb);
@@ -49,7 +49,7 @@ static bool conv_dgrad(Exec &ex, const void *g, Geom gi, const Layer &L, float *
 }
 static void conv_wgrad(Exec &ex, const void *g, const void *a, Geom gi, const Layer &L, float *dW) {
     const bool b16 = ex.mode == 0;
-    if (b16 && conv_wgrad_tc(ex, g, a, gi, L, dW)) return;
+    if (b16 && conv_wgrad_tc(ex, g, a, gi, L, dW, nullptr, nullptr)) return;
     conv_wgrad_simt(ex, g, b16, a, b16, gi, L, dW);
 }
 
@@ -127,10 +127,32 @@ void fn_backward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, FnS
             gcur = buf;
         }
     }
+    // The weight gradients of the function depend only on tensors that already exist when their
+    // layer's turn comes, so they run on a side stream beside the data-gradient chain (fork before
+    // each, one join at the end); their split partials get a buffer of their own for that time.
+    bool side = b16 && ex.use_side && (ex.dry || (ex.ctx->side_stream && !ex.ctx->profiling));
+    size_t wg_need = 0;
+    for (int l = 0; l < L && side; l++) {
+        size_t n = 0;
+        if (!conv_wgrad_tc(ex, nullptr, nullptr, gin[l], layers[l], nullptr, nullptr, &n)) side = false;
+        else if (n > wg_need) wg_need = n;
+    }
+    float *wg_scratch = side && wg_need ? ex.ws.get<float>(wg_need) : nullptr;
     for (int l = L - 1; l >= 0; l--) {
         const Layer &ly = layers[l];
         const size_t P = gin[l].P();
-        conv_wgrad(ex, gcur, saved.a[l], gin[l], ly, ly.dW);
+        if (side) {
+            cudaStream_t main = ex.stream;
+            if (!ex.dry) {
+                cudaEventRecord(ex.ctx->ev_fork, main);
+                cudaStreamWaitEvent(ex.ctx->side_stream, ex.ctx->ev_fork, 0);
+                ex.stream = ex.ctx->side_stream;
+            }
+            conv_wgrad_tc(ex, gcur, saved.a[l], gin[l], ly, ly.dW, wg_scratch, nullptr);
+            ex.stream = main;
+        } else {
+            conv_wgrad(ex, gcur, saved.a[l], gin[l], ly, ly.dW);
+        }
         float *da = ex.ws.get<float>(P * ly.cin);
         float *coef = ex.ws.get<float>((size_t)3 * ly.cin);
         const Pair tl = l == 0 ? u : single(saved.t[l - 1], ly.cin);
@@ -145,6 +167,10 @@ void fn_backward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, FnS
             bn_relu_bwd(ex, da, tl, P, bn, ly.dgamma, ly.dbeta, coef, sums_done, dt, b16, Pair{}, Pair{}, nullptr);
             gcur = dt;
         }
+    }
+    if (side && !ex.dry) {
+        cudaEventRecord(ex.ctx->ev_join, ex.ctx->side_stream);
+        cudaStreamWaitEvent(ex.stream, ex.ctx->ev_join, 0);
     }
     ex.ws.release(outer);
 }

@@ -23,6 +23,8 @@ struct revnet_ctx {
     static constexpr int kCounters = 192;
     void *encode_tiled = nullptr; // driver entry point for tensor-map encoding
     cudaStream_t capture_stream = nullptr;   // private stream on which a train step is captured into a graph
+    cudaStream_t side_stream = nullptr;      // weight gradients run here, beside the data-gradient chain
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     // per-kernel timing (revnet_profile_*): one event after every launch while enabled
     bool profiling = false;
     std::vector<ProfRec> prof;
@@ -146,6 +148,7 @@ struct Exec {
     uint64_t launches = 0;
     bool failed = false;
     bool pdl = true;       // launch kernels with programmatic stream serialization (see launch())
+    bool use_side = true;  // run weight gradients on the context's side stream (never while profiling)
     // called after every launch: error check, launch count and (when profiling) an event;
     // bytes / flops are the algorithmic traffic and work of that launch
     void check(const char *what, double bytes = 0, double flops = 0);

@@ -510,7 +510,9 @@ bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, 
 }
 
 
-bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer &L, float *dW) {
+// scratch: room for the split partials if the caller provides it (else it comes from the arena);
+// need: if non-null the call only reports whether it takes the shape and how many floats of scratch it wants
+bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer &L, float *dW, float *scratch, size_t *need) {
     if ((L.stride != 1 && L.stride != 2) || (L.k != 1 && L.k != 3) || L.cin % 8 || L.cout % 8) return false;
     if (L.stride == 2 && (gi.H % 2 || gi.W % 2)) return false;
     WgParams p;
@@ -540,9 +542,10 @@ bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer
     if (splits > p.n_tiles_px) splits = p.n_tiles_px;
     if (splits < 1) splits = 1;
     p.slice = (size_t)L.cout * taps * L.cin;
+    if (need) { *need = splits > 1 ? (size_t)splits * p.slice : 0; return true; }
     ex.flops += 2ull * go.P() * L.cout * L.cin * taps;
     size_t m = ex.ws.mark();
-    float *part = splits > 1 ? ex.ws.get<float>((size_t)splits * p.slice) : dW;
+    float *part = splits > 1 ? (scratch ? scratch : ex.ws.get<float>((size_t)splits * p.slice)) : dW;
     if (!ex.dry) {
         CUtensorMap map_a, map_g;
         if (!encode_act_map(ex, &map_a, a, gi, L.cin, p.blockC, go.W, p.BH, p.BIMG, L.stride) ||

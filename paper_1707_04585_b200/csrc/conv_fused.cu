@@ -62,6 +62,7 @@ struct __align__(16) FusedShared {
     int srow[128];                   // accumulator row -> pixel index inside the partner / output tile (box order), -1: padding
     __align__(16) float sc[64];      // BN scale and shift per input channel
     __align__(16) float sf[64];
+    __align__(16) uint4 dummy;             // where operand stores that have no destination go
     __align__(16) uint64_t desc[2 * 36];   // (operand, weight) descriptor of every MMA of a tile: they do not depend on the tile
 };
 
@@ -78,7 +79,8 @@ __device__ __forceinline__ uint32_t relu_pack2(float lo, float hi) {
 //             0xffff where that copy does not hold it
 //   d2f     : bits 16-23 halo row, 24-31 image in tile
 //   raw16   : offset of its source in the raw tile, in 16-byte units
-//   flags   : bit 0: inside the tile proper (not halo); bit 1: column inside the image and channels valid
+//   flags   : bit 0: inside the tile proper (not halo); bit 1: column inside the image and channels valid;
+//             bits 8-15: halo column
 struct __align__(16) ItemRef { uint32_t d01, d2f, raw16, flags; };
 
 __device__ __forceinline__ void build_table(const FusedParams &p, ItemRef *tab, int npix, int cshift) {
@@ -102,7 +104,7 @@ __device__ __forceinline__ void build_table(const FusedParams &p, ItemRef *tab, 
             e.d01 = d[0] | (d[1] << 16);
             e.d2f = d[2] | ((uint32_t)r << 16) | ((uint32_t)img << 24);
             e.raw16 = (uint32_t)(((size_t)px * p.cin + ck * 8) * esize) >> 4;
-            e.flags = (interior ? 1u : 0u) | ((xin && ck < (p.cin >> 3)) ? 2u : 0u);
+            e.flags = (interior ? 1u : 0u) | ((xin && ck < (p.cin >> 3)) ? 2u : 0u) | ((uint32_t)xh << 8);
             tab[(px << cshift) + ck] = e;
         }
     }
@@ -110,69 +112,131 @@ __device__ __forceinline__ void build_table(const FusedParams &p, ItemRef *tab, 
 
 // raw tile (shared memory) -> operand copies (shared memory), four items per thread in flight.
 // This thread's channel chunk ck is fixed: the thread count is a multiple of the chunks per pixel.
+// IN_MODE 0: float input through BN + ReLU; 2: fixed-point input through BN + ReLU; 1: bf16 input as it is.
+// Written without branches in the per-item work (invalid items compute on the zeros TMA delivered and are
+// masked, stores that do not exist go to a dummy slot), so that the four items of a batch interleave.
 template <int IN_MODE>
-__device__ __forceinline__ void build_tile(const FusedParams &p, const FusedShared *sh, const ItemRef *tab, int items, int ck,
+__device__ __forceinline__ void build_tile(const FusedParams &p, FusedShared *sh, const ItemRef *tab, int items, int ck,
                                            const uint8_t *raw, uint8_t *A, int n0, int h0) {
     const int pad = p.k >> 1;
-    const float qs = p.in_q;
     // scale and shift of this thread's eight channels; a fixed-point input folds its step into the scale (a power of two: exact)
     float sc[8], sf[8];
-    if (IN_MODE == 0) {
+    if (IN_MODE != 1) {
 #pragma unroll
-        for (int e = 0; e < 8; e++) { sc[e] = sh->sc[ck * 8 + e] * (qs != 0.f ? qs : 1.f); sf[e] = sh->sf[ck * 8 + e]; }
+        for (int e = 0; e < 8; e++) { sc[e] = sh->sc[ck * 8 + e] * (IN_MODE == 2 ? p.in_q : 1.f); sf[e] = sh->sf[ck * 8 + e]; }
     }
+    const uint32_t dummy = (uint32_t)(reinterpret_cast<uint8_t *>(&sh->dummy) - A);     // byte offset of the dummy slot relative to A
 #pragma unroll 1
     for (int base = threadIdx.x; base < items; base += 4 * kFThreads) {
         ItemRef ref[4];
-        uint4 lo[4], hi[4];
+        uint4 v[4];
+        bool ok[4];
 #pragma unroll
         for (int j = 0; j < 4; j++) {
             const int it = base + j * kFThreads;
-            ref[j].flags = 4u;                              // bit 2: no such item
-            if (it < items) {
-                ref[j] = tab[it];
-                const int r = (ref[j].d2f >> 16) & 0xff, img = ref[j].d2f >> 24;
-                if (!((ref[j].flags & 2u) && (unsigned)(h0 - pad + r) < (unsigned)p.g.H && n0 + img < p.g.N)) ref[j].flags &= ~2u;
-                if (ref[j].flags & 2u) {
-                    const uint4 *src = reinterpret_cast<const uint4 *>(raw) + ref[j].raw16;
-                    lo[j] = src[0];
-                    if (IN_MODE == 0) hi[j] = src[1];
-                }
-            }
-        }
-#pragma unroll
-        for (int j = 0; j < 4; j++) {
-            if (ref[j].flags & 4u) continue;
-            uint4 v = make_uint4(0u, 0u, 0u, 0u);
-            if (ref[j].flags & 2u) {
+            const bool exists = it < items;
+            ref[j] = tab[exists ? it : items - 1];
+            const int r = (ref[j].d2f >> 16) & 0xff, img = ref[j].d2f >> 24;
+            ok[j] = exists && (ref[j].flags & 2u) && (unsigned)(h0 - pad + r) < (unsigned)p.g.H && n0 + img < p.g.N;
+            if (!exists) { ref[j].d01 = 0xffffffffu; ref[j].d2f |= 0xffffu; }
+            const uint4 *src = reinterpret_cast<const uint4 *>(raw) + ref[j].raw16;
+            const uint4 lo = src[0];
+            if (IN_MODE == 1) {
+                v[j] = lo;
+            } else {
+                const uint4 hi = src[1];
+                float x[8];
                 if (IN_MODE == 0) {
-                    float x[8];
-                    if (qs == 0.f) {
-                        x[0] = __uint_as_float(lo[j].x); x[1] = __uint_as_float(lo[j].y); x[2] = __uint_as_float(lo[j].z); x[3] = __uint_as_float(lo[j].w);
-                        x[4] = __uint_as_float(hi[j].x); x[5] = __uint_as_float(hi[j].y); x[6] = __uint_as_float(hi[j].z); x[7] = __uint_as_float(hi[j].w);
-                    } else {
-                        x[0] = __int2float_rn((int)lo[j].x); x[1] = __int2float_rn((int)lo[j].y); x[2] = __int2float_rn((int)lo[j].z); x[3] = __int2float_rn((int)lo[j].w);
-                        x[4] = __int2float_rn((int)hi[j].x); x[5] = __int2float_rn((int)hi[j].y); x[6] = __int2float_rn((int)hi[j].z); x[7] = __int2float_rn((int)hi[j].w);
-                    }
-#pragma unroll
-                    for (int e = 0; e < 8; e++) x[e] = fmaf(sc[e], x[e], sf[e]);
-                    v = make_uint4(relu_pack2(x[0], x[1]), relu_pack2(x[2], x[3]), relu_pack2(x[4], x[5]), relu_pack2(x[6], x[7]));
-                    if (p.a_out && (ref[j].flags & 1u)) {
-                        // raw16 * 16 bytes = (pixel of the raw tile * cin + ck * 8) * 4: recover the pixel's place in the image
-                        const int r = (ref[j].d2f >> 16) & 0xff, img = ref[j].d2f >> 24;
-                        const int px = (int)((ref[j].raw16 << 2) / (uint32_t)p.cin);
-                        const int xh = px % (p.g.W + 2 * pad);
-                        const size_t gp = ((size_t)(n0 + img) * p.g.H + (h0 - pad + r)) * p.g.W + (xh - pad);
-                        *reinterpret_cast<uint4 *>(p.a_out + gp * p.cin + ck * 8) = v;
-                    }
+                    x[0] = __uint_as_float(lo.x); x[1] = __uint_as_float(lo.y); x[2] = __uint_as_float(lo.z); x[3] = __uint_as_float(lo.w);
+                    x[4] = __uint_as_float(hi.x); x[5] = __uint_as_float(hi.y); x[6] = __uint_as_float(hi.z); x[7] = __uint_as_float(hi.w);
                 } else {
-                    v = lo[j];
+                    x[0] = __int2float_rn((int)lo.x); x[1] = __int2float_rn((int)lo.y); x[2] = __int2float_rn((int)lo.z); x[3] = __int2float_rn((int)lo.w);
+                    x[4] = __int2float_rn((int)hi.x); x[5] = __int2float_rn((int)hi.y); x[6] = __int2float_rn((int)hi.z); x[7] = __int2float_rn((int)hi.w);
                 }
+#pragma unroll
+                for (int e = 0; e < 8; e++) x[e] = fmaf(sc[e], x[e], sf[e]);
+                v[j] = make_uint4(relu_pack2(x[0], x[1]), relu_pack2(x[2], x[3]), relu_pack2(x[4], x[5]), relu_pack2(x[6], x[7]));
             }
+            const uint32_t keep = ok[j] ? 0xffffffffu : 0u;       // outside the image: zero, whatever BN makes of the zeros delivered
+            v[j].x &= keep; v[j].y &= keep; v[j].z &= keep; v[j].w &= keep;
             const uint32_t d0 = ref[j].d01 & 0xffffu, d1 = ref[j].d01 >> 16, d2 = ref[j].d2f & 0xffffu;
-            if (d0 != 0xffffu) *reinterpret_cast<uint4 *>(A + (d0 << 4)) = v;
-            if (d1 != 0xffffu) *reinterpret_cast<uint4 *>(A + p.copy_bytes + (d1 << 4)) = v;
-            if (d2 != 0xffffu) *reinterpret_cast<uint4 *>(A + 2 * p.copy_bytes + (d2 << 4)) = v;
+            *reinterpret_cast<uint4 *>(A + (d0 != 0xffffu ? (d0 << 4) : dummy)) = v[j];
+            *reinterpret_cast<uint4 *>(A + (d1 != 0xffffu ? p.copy_bytes + (d1 << 4) : dummy)) = v[j];
+            *reinterpret_cast<uint4 *>(A + (d2 != 0xffffu ? 2 * p.copy_bytes + (d2 << 4) : dummy)) = v[j];
+        }
+        if (IN_MODE != 1 && p.a_out) {
+#pragma unroll
+            for (int j = 0; j < 4; j++)
+                if (ok[j] && (ref[j].flags & 1u)) {
+                    const int r = (ref[j].d2f >> 16) & 0xff, img = ref[j].d2f >> 24, xh = (ref[j].flags >> 8) & 0xff;
+                    const size_t gp = ((size_t)(n0 + img) * p.g.H + (h0 - pad + r)) * p.g.W + (xh - pad);
+                    *reinterpret_cast<uint4 *>(p.a_out + gp * p.cin + ck * 8) = v[j];
+                }
+        }
+    }
+}
+
+// Epilogue pass A for one thread (= one accumulator row, alternate groups of 8 columns): accumulator
+// (+ partner tile) -> output tile in shared memory.  KIND: 0 plain float, 1 plain onto the fixed-point
+// grid, 2 / 3 float coupling + / -, 4 / 5 fixed-point coupling + / -.  One instantiation per kind, so
+// that the loop body has no branches.
+template <int KIND>
+__device__ __forceinline__ void pass_a(const FusedParams &p, uint32_t tm, int c0, int sr, const uint8_t *aux, uint8_t *outb,
+                                       float out_s, int row_b) {
+    const int swz = p.GW == 32 ? (sr & 7) : ((sr >> 1) & 3);
+#pragma unroll 1
+    for (int c = c0; c < p.BN; c += 16) {
+        float v[8];
+        tmem_ld8(tm + (uint32_t)c, v);
+        if (sr < 0) continue;
+        const int gbase = (c / p.GW) * p.group_bytes + sr * row_b, j0 = (c % p.GW) >> 2;
+#pragma unroll
+        for (int j = 0; j < 2; j++) {
+            const int off = gbase + (((j0 + j) ^ swz) << 4);
+            float4 r = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            if (KIND == 2 || KIND == 3) {
+                const float4 pr = *reinterpret_cast<const float4 *>(aux + off);
+                if (KIND == 2) { r.x = pr.x + r.x; r.y = pr.y + r.y; r.z = pr.z + r.z; r.w = pr.w + r.w; }
+                else { r.x = pr.x - r.x; r.y = pr.y - r.y; r.z = pr.z - r.z; r.w = pr.w - r.w; }
+            } else if (KIND != 0) {
+                int4 iv = make_int4(__float2int_rn(r.x * out_s), __float2int_rn(r.y * out_s), __float2int_rn(r.z * out_s), __float2int_rn(r.w * out_s));
+                if (KIND >= 4) {
+                    const int4 pi = *reinterpret_cast<const int4 *>(aux + off);
+                    if (KIND == 4) { iv.x = pi.x + iv.x; iv.y = pi.y + iv.y; iv.z = pi.z + iv.z; iv.w = pi.w + iv.w; }
+                    else { iv.x = pi.x - iv.x; iv.y = pi.y - iv.y; iv.z = pi.z - iv.z; iv.w = pi.w - iv.w; }
+                }
+                r = make_float4(__int_as_float(iv.x), __int_as_float(iv.y), __int_as_float(iv.z), __int_as_float(iv.w));
+            }
+            *reinterpret_cast<float4 *>(outb + off) = r;
+        }
+    }
+}
+
+// Epilogue pass B for one thread (= one channel quad, every rpp-th pixel): running per-channel sums over
+// the valid pixels of the output tile.  KIND 0 / 1: sums and second sums of the stored values (float /
+// fixed point); 2 / 3: the two sums of the BN+ReLU backward with a float / fixed-point BN input tile.
+// Rows are added in a fixed order.
+template <int KIND>
+__device__ __forceinline__ void pass_b(const FusedParams &p, const uint8_t *ob, const uint8_t *aux, int jq, int r0, int rpp, int valid_px,
+                                       int row_b, float q, float4 sc4, float4 sh4, float4 mu4, float4 rs4, float (&acc)[8]) {
+#pragma unroll 4
+    for (int pl = r0; pl < valid_px; pl += rpp) {
+        const int off = pl * row_b + ((jq ^ (p.GW == 32 ? (pl & 7) : ((pl >> 1) & 3))) << 4);
+        float4 v = *reinterpret_cast<const float4 *>(ob + off);
+        if (KIND >= 2) {
+            float4 tt = *reinterpret_cast<const float4 *>(aux + off);
+            if (KIND == 3) tt = make_float4(__int2float_rn(__float_as_int(tt.x)) * q, __int2float_rn(__float_as_int(tt.y)) * q,
+                                            __int2float_rn(__float_as_int(tt.z)) * q, __int2float_rn(__float_as_int(tt.w)) * q);
+            const float dx = fmaf(sc4.x, tt.x, sh4.x) > 0.f ? v.x : 0.f, dy = fmaf(sc4.y, tt.y, sh4.y) > 0.f ? v.y : 0.f;
+            const float dz = fmaf(sc4.z, tt.z, sh4.z) > 0.f ? v.z : 0.f, dw = fmaf(sc4.w, tt.w, sh4.w) > 0.f ? v.w : 0.f;
+            acc[0] += dx; acc[1] += dy; acc[2] += dz; acc[3] += dw;
+            acc[4] += dx * ((tt.x - mu4.x) * rs4.x); acc[5] += dy * ((tt.y - mu4.y) * rs4.y);
+            acc[6] += dz * ((tt.z - mu4.z) * rs4.z); acc[7] += dw * ((tt.w - mu4.w) * rs4.w);
+        } else {
+            if (KIND == 1) v = make_float4(__int2float_rn(__float_as_int(v.x)) * q, __int2float_rn(__float_as_int(v.y)) * q,
+                                           __int2float_rn(__float_as_int(v.z)) * q, __int2float_rn(__float_as_int(v.w)) * q);
+            acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
+            acc[4] += v.x * v.x; acc[5] += v.y * v.y; acc[6] += v.z * v.z; acc[7] += v.w * v.w;
         }
     }
 }
@@ -239,10 +303,9 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
     tile_first(p.g, blockIdx.x, cur);
     nx1 = cur; tile_next(p.g, step, G, nx1);
     nx2 = nx1; tile_next(p.g, step, G, nx2);
-    // byte offset of float4 j of pixel r inside a column group: rows of 128 (64) bytes, 16-byte chunks XORed with
-    // address bits 7.. as the TMA swizzle does, so that a thread per row touches all banks
+    // inside a column group pixel r has a row of 128 (64) bytes whose 16-byte chunks are XORed with address bits 7..
+    // as the TMA swizzle does, so that a thread per row touches all banks
     const int row_b = p.GW * 4;
-    auto sw_off = [&](int r, int j) { return r * row_b + ((j ^ (p.GW == 32 ? (r & 7) : ((r >> 1) & 3))) << 4); };
 
     if (threadIdx.x == 0) {
         for (int b = 0; b < 2; b++) { mbar_init(&sh->raw_full[b], 1); mbar_init(&sh->aux_full[b], 1); }
@@ -314,8 +377,9 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
         ok = __syncthreads_and(ok);
         if (!ok) break;
         // ---- build the operand
-        if (p.in_mode == 0) build_tile<0>(p, sh, tab, items, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
-        else build_tile<1>(p, sh, tab, items, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
+        if (p.in_mode == 1) build_tile<1>(p, sh, tab, items, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
+        else if (p.in_q == 0.f) build_tile<0>(p, sh, tab, items, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
+        else build_tile<2>(p, sh, tab, items, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
         fence_proxy_async();
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -343,38 +407,19 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
         if (!ok) break;
         tc_fence_after();
         // ---- epilogue, pass A: accumulator row (+ partner) -> output tile in shared memory
-        if (warp < 4) {
+        {
+            // all eight warps: warp w and w + 4 share tensor-memory lanes 32(w%4).. and take alternate groups of 8 columns
             const int sr = sh->srow[etid];
             const uint8_t *aux = auxb + b * p.aux_bytes;
-#pragma unroll 1
-            for (int c = 0; c < p.BN; c += 16) {
-                float v[16];
-                tmem_ld16(tmem_d + lane_base + (uint32_t)c, v);
-                if (sr >= 0) {
-                    const int gbase = (c / p.GW) * p.group_bytes, j0 = (c % p.GW) >> 2;
-#pragma unroll
-                    for (int j = 0; j < 4; j++) {
-                        const int off = gbase + sw_off(sr, j0 + j);
-                        float4 r = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                        if (e.mode == EPI_COUPLE) {
-                            const float4 pr = *reinterpret_cast<const float4 *>(aux + off);
-                            if (out_q == 0.f) {
-                                if (e.sign > 0) { r.x = pr.x + r.x; r.y = pr.y + r.y; r.z = pr.z + r.z; r.w = pr.w + r.w; }
-                                else { r.x = pr.x - r.x; r.y = pr.y - r.y; r.z = pr.z - r.z; r.w = pr.w - r.w; }
-                            } else {
-                                int4 iv = make_int4(__float2int_rn(r.x * out_s), __float2int_rn(r.y * out_s), __float2int_rn(r.z * out_s), __float2int_rn(r.w * out_s));
-                                const int4 pi = make_int4(__float_as_int(pr.x), __float_as_int(pr.y), __float_as_int(pr.z), __float_as_int(pr.w));
-                                if (e.sign > 0) { iv.x = pi.x + iv.x; iv.y = pi.y + iv.y; iv.z = pi.z + iv.z; iv.w = pi.w + iv.w; }
-                                else { iv.x = pi.x - iv.x; iv.y = pi.y - iv.y; iv.z = pi.z - iv.z; iv.w = pi.w - iv.w; }
-                                r = make_float4(__int_as_float(iv.x), __int_as_float(iv.y), __int_as_float(iv.z), __int_as_float(iv.w));
-                            }
-                        } else if (out_q != 0.f) {
-                            r = make_float4(__int_as_float(__float2int_rn(r.x * out_s)), __int_as_float(__float2int_rn(r.y * out_s)),
-                                            __int_as_float(__float2int_rn(r.z * out_s)), __int_as_float(__float2int_rn(r.w * out_s)));
-                        }
-                        *reinterpret_cast<float4 *>(outb + off) = r;
-                    }
-                }
+            const uint32_t tm = tmem_d + lane_base;
+            const int c0 = (warp >> 2) * 8;
+            if (e.mode != EPI_COUPLE) {
+                if (out_q == 0.f) pass_a<0>(p, tm, c0, sr, aux, outb, out_s, row_b);
+                else pass_a<1>(p, tm, c0, sr, aux, outb, out_s, row_b);
+            } else if (out_q == 0.f) {
+                if (e.sign > 0) pass_a<2>(p, tm, c0, sr, aux, outb, out_s, row_b); else pass_a<3>(p, tm, c0, sr, aux, outb, out_s, row_b);
+            } else {
+                if (e.sign > 0) pass_a<4>(p, tm, c0, sr, aux, outb, out_s, row_b); else pass_a<5>(p, tm, c0, sr, aux, outb, out_s, row_b);
             }
         }
         fence_proxy_async();
@@ -389,28 +434,17 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
             int valid_px = p.g.BIMG > 1 ? (p.g.N - n0 < p.g.BIMG ? p.g.N - n0 : p.g.BIMG) * p.g.BH * p.g.W
                                         : (p.g.H - h0 < p.g.BH ? p.g.H - h0 : p.g.BH) * p.g.W;
             const int qg = p.GW >> 2;                      // quads per column group
-            const int gbase = (quad / qg) * p.group_bytes, jq = quad % qg;
-            const uint8_t *aux = auxb + b * p.aux_bytes;
-#pragma unroll 2
-            for (int pl = r0; pl < valid_px; pl += rpp) {
-                const int off = gbase + sw_off(pl, jq);
-                float4 v = *reinterpret_cast<const float4 *>(outb + off);
-                if (e.mode == EPI_BNBWD) {
-                    float4 tt = *reinterpret_cast<const float4 *>(aux + off);
-                    if (t_q != 0.f) tt = make_float4(__int2float_rn(__float_as_int(tt.x)) * t_q, __int2float_rn(__float_as_int(tt.y)) * t_q,
-                                                     __int2float_rn(__float_as_int(tt.z)) * t_q, __int2float_rn(__float_as_int(tt.w)) * t_q);
-                    const float dx = fmaf(sc4.x, tt.x, sh4.x) > 0.f ? v.x : 0.f, dy = fmaf(sc4.y, tt.y, sh4.y) > 0.f ? v.y : 0.f;
-                    const float dz = fmaf(sc4.z, tt.z, sh4.z) > 0.f ? v.z : 0.f, dw = fmaf(sc4.w, tt.w, sh4.w) > 0.f ? v.w : 0.f;
-                    s0 += dx; s1 += dy; s2 += dz; s3 += dw;
-                    q0 += dx * ((tt.x - mu4.x) * rs4.x); q1 += dy * ((tt.y - mu4.y) * rs4.y);
-                    q2 += dz * ((tt.z - mu4.z) * rs4.z); q3 += dw * ((tt.w - mu4.w) * rs4.w);
-                } else {
-                    if (out_q != 0.f) v = make_float4(__int2float_rn(__float_as_int(v.x)) * out_q, __int2float_rn(__float_as_int(v.y)) * out_q,
-                                                      __int2float_rn(__float_as_int(v.z)) * out_q, __int2float_rn(__float_as_int(v.w)) * out_q);
-                    s0 += v.x; s1 += v.y; s2 += v.z; s3 += v.w;
-                    q0 += v.x * v.x; q1 += v.y * v.y; q2 += v.z * v.z; q3 += v.w * v.w;
-                }
-            }
+            const uint32_t gb = (uint32_t)((quad / qg) * p.group_bytes);
+            const int jq = quad % qg;
+            const uint8_t *aux = auxb + b * p.aux_bytes + gb;
+            const uint8_t *ob = outb + gb;
+            float acc[8] = {s0, s1, s2, s3, q0, q1, q2, q3};
+            if (e.mode == EPI_BNBWD) {
+                if (t_q == 0.f) pass_b<2>(p, ob, aux, jq, r0, rpp, valid_px, row_b, 0.f, sc4, sh4, mu4, rs4, acc);
+                else pass_b<3>(p, ob, aux, jq, r0, rpp, valid_px, row_b, t_q, sc4, sh4, mu4, rs4, acc);
+            } else if (out_q == 0.f) pass_b<0>(p, ob, aux, jq, r0, rpp, valid_px, row_b, 0.f, sc4, sh4, mu4, rs4, acc);
+            else pass_b<1>(p, ob, aux, jq, r0, rpp, valid_px, row_b, out_q, sc4, sh4, mu4, rs4, acc);
+            s0 = acc[0]; s1 = acc[1]; s2 = acc[2]; s3 = acc[3]; q0 = acc[4]; q1 = acc[5]; q2 = acc[6]; q3 = acc[7];
         }
         if (p.NB == 1) {
             __syncthreads();     // the partner buffer is free

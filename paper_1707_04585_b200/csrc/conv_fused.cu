@@ -83,30 +83,35 @@ __device__ __forceinline__ uint32_t relu_pack2(float lo, float hi) {
 //             bits 8-15: halo column
 struct __align__(16) ItemRef { uint32_t d01, d2f, raw16, flags; };
 
-__device__ __forceinline__ void build_table(const FusedParams &p, ItemRef *tab, int npix, int cshift) {
+// a / b for 0 <= a < 65536 with inv_b = 1.f / b: exact, without the integer-division sequence
+__device__ __forceinline__ int small_div(int a, float inv_b) { return __float2int_rz(((float)a + 0.5f) * inv_b); }
+
+__device__ __forceinline__ void build_table(const FusedParams &p, ItemRef *tab, int items, int cshift) {
     const int pad = p.k >> 1;
     const int WH = p.g.W + 2 * pad, HR = p.g.BH + 2 * pad;
+    const float inv_wh = 1.f / (float)WH, inv_hr = 1.f / (float)HR;
     const int row_bytes = p.KC * 2;
     const int esize = p.in_mode == 0 ? 4 : 2;
-    for (int px = threadIdx.x; px < npix; px += kFThreads) {
-        const int xh = px % WH, rest = px / WH;
-        const int r = rest % HR, img = rest / HR;
+    for (int it = threadIdx.x; it < items; it += kFThreads) {
+        const int ck = it & ((1 << cshift) - 1), px = it >> cshift;
+        const int rest = small_div(px, inv_wh), xh = px - rest * WH;
+        const int img = small_div(rest, inv_hr), r = rest - img * HR;
         const int rowbase = (r * p.g.BIMG + img) * p.g.Wp;
-        const bool interior = r >= pad && r < pad + p.g.BH && xh >= pad && xh < pad + p.g.W;
         const bool xin = xh >= pad && xh < pad + p.g.W;
-        for (int ck = 0; ck < (1 << cshift); ck++) {
-            uint32_t d[3] = {0xffffu, 0xffffu, 0xffffu};
-            for (int s = 0; s < p.k; s++) {          // halo column xh is column xh - s of the copy for horizontal tap offset s
-                const int x = xh - s;
-                if (x >= 0 && x < p.g.W) d[s] = swizzled_offset((uint32_t)(rowbase + x), (uint32_t)ck, row_bytes) >> 4;
-            }
-            ItemRef e;
-            e.d01 = d[0] | (d[1] << 16);
-            e.d2f = d[2] | ((uint32_t)r << 16) | ((uint32_t)img << 24);
-            e.raw16 = (uint32_t)(((size_t)px * p.cin + ck * 8) * esize) >> 4;
-            e.flags = (interior ? 1u : 0u) | ((xin && ck < (p.cin >> 3)) ? 2u : 0u) | ((uint32_t)xh << 8);
-            tab[(px << cshift) + ck] = e;
+        const bool interior = xin && r >= pad && r < pad + p.g.BH;
+        uint32_t d[3];
+#pragma unroll
+        for (int s = 0; s < 3; s++) {            // halo column xh is column xh - s of the copy for horizontal tap offset s
+            const int x = xh - s;
+            const uint32_t off = swizzled_offset((uint32_t)(rowbase + (x < 0 ? 0 : x)), (uint32_t)ck, row_bytes) >> 4;
+            d[s] = (s < p.k && x >= 0 && x < p.g.W) ? off : 0xffffu;
         }
+        ItemRef e;
+        e.d01 = d[0] | (d[1] << 16);
+        e.d2f = d[2] | ((uint32_t)r << 16) | ((uint32_t)img << 24);
+        e.raw16 = (uint32_t)((px * p.cin + ck * 8) * esize) >> 4;
+        e.flags = (interior ? 1u : 0u) | ((xin && ck < (p.cin >> 3)) ? 2u : 0u) | ((uint32_t)xh << 8);
+        tab[it] = e;
     }
 }
 
@@ -277,6 +282,7 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
     const int npix = (p.g.BH + 2 * pad) * p.g.BIMG * (p.g.W + 2 * pad);
     const int items = npix << cshift;
     const int tile_px = p.g.BH * p.g.BIMG * p.g.W;      // pixels of a partner / output tile
+    // one accumulator: splitting the taps over several (summed in the epilogue) was measured slower
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < p.BN) tmem_cols <<= 1;
     const int col0 = blockIdx.y * p.BN;
@@ -317,7 +323,7 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
         if (need_aux) tma_prefetch_desc(&map_aux);
     }
     if (warp == 0) tmem_alloc(&sh->tmem_base, tmem_cols);
-    build_table(p, tab, npix, cshift);
+    build_table(p, tab, items, cshift);
     if (threadIdx.x < 128) {
         // accumulator row (image row, image, column) -> pixel of the (image, row, column) ordered tile
         const int w = etid % p.g.Wp, img = (etid / p.g.Wp) % p.g.BIMG, h = etid / (p.g.BIMG * p.g.Wp);
@@ -395,13 +401,14 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
                 mma_bf16(tmem_d, d.x, d.y, idesc, i ? 1u : 0u);
             }
             mma_commit(&sh->mma_done);
-            if (p.NB == 2) {
-                // this tile's raw buffer has been consumed, and the other partner buffer was last read by the epilogue before
-                if (nx2.t < NT) load_raw(nx2, b);
-                if (need_aux && nx1.t < NT) load_aux(nx1, b ^ 1);
-            }
             tma_store_wait_read();                       // the previous tile's store has read the output buffer
             ok = ok && mbar_wait(&sh->mma_done, ti & 1) && (!need_aux || mbar_wait(&sh->aux_full[b], u & 1));
+        }
+        else if (threadIdx.x == 32 && p.NB == 2) {
+            // meanwhile another thread issues the loads of the tiles ahead: this tile's raw buffer has been consumed,
+            // and the other partner buffer was last read by the epilogue before
+            if (nx2.t < NT) load_raw(nx2, b);
+            if (need_aux && nx1.t < NT) load_aux(nx1, b ^ 1);
         }
         ok = __syncthreads_and(ok);
         if (!ok) break;

@@ -268,7 +268,7 @@ void tc_pack_now(Exec &ex, const float *W, bf16 *out, int cin, int cout, int k, 
 struct PackJob { const float *W; bf16 *out; int Co, Ci, k, rows_pad, cols_pad, transposed; };
 size_t tc_pack_elems(int cin, int cout, int k, bool transposed);
 PackJob tc_pack_job(const float *W, bf16 *out, int cin, int cout, int k, bool transposed);
-void tc_pack_batch(Exec &ex, const PackJob *jobs_dev, int n_jobs, double bytes);
+void tc_pack_batch(Exec &ex, const PackJob *jobs_dev, int n_jobs, double bytes, size_t max_job_elems);
 
 // ---------------------------------------------------------------- block.cu
 struct FnSaved;   // activations kept from a residual function's (re)computation

@@ -598,9 +598,12 @@ PackJob tc_pack_job(const float *W, bf16 *out, int cin, int cout, int k, bool tr
     if (!transposed) pack_dims(cout, cin, j.rows_pad, j.cols_pad); else pack_dims(cin, cout, j.rows_pad, j.cols_pad);
     return j;
 }
-void tc_pack_batch(Exec &ex, const PackJob *jobs_dev, int n_jobs, double bytes) {
+void tc_pack_batch(Exec &ex, const PackJob *jobs_dev, int n_jobs, double bytes, size_t max_job_elems) {
     if (ex.dry || n_jobs == 0) return;
-    dim3 grid(96, (unsigned)n_jobs);
+    // blocks per job sized for the largest job (2048 elements per block), within 4 .. 96
+    size_t bx = (max_job_elems + 2047) / 2048;
+    if (bx < 4) bx = 4; if (bx > 96) bx = 96;
+    dim3 grid((unsigned)bx, (unsigned)n_jobs);
     launch(ex, pack_weights_batch_kernel, grid, 256, 0, jobs_dev);
     ex.check("pack_weights_batch", bytes);
 }

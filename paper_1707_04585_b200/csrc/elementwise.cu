@@ -198,30 +198,57 @@ void bn_relu_apply(Exec &ex, Pair t, size_t P, BnRef bn, void *a, bool a_bf16) {
 // dt = coef0*db - coef1 - coef2*xhat ; db = da*[scale*t+shift > 0]
 // OUT 0: out[P,C] = dt (float or bf16) ; 1: outp = dt (fp32 pair) ; 2: outp = add + dt
 // CAST (OUT 1, 2): also write the result as one bf16 [P,C] tensor
+// A thread keeps one channel quad (its coefficients stay in registers) and strides the rows, four
+// rows in flight; row_step = threads of the grid / C4 (the launch makes that a whole number).
 template <class TO, int OUT, bool CAST>
-__global__ void bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, size_t nquads, int C4, BnRef bn,
+__global__ void bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, size_t P, int C4, BnRef bn,
                                          const float *__restrict__ coef, TO *__restrict__ out, Pair add, Pair outp,
                                          bf16 *__restrict__ cast) {
     pdl_enter();
     const int C = C4 * 4;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
-        size_t row = i / C4; int q = (int)(i - row * C4), c = q * 4;
-        float4 v = t.ld4(row, c), g = ld4(da + i * 4);
-        float4 sc, sh, mu, rs;
-        bn_coef4(bn, c, sc, sh, mu, rs);
-        float4 k0 = ld4(coef + c), k1 = ld4(coef + C + c), k2 = ld4(coef + 2 * C + c), o;
-        o.x = k0.x * (fmaf(sc.x, v.x, sh.x) > 0.f ? g.x : 0.f) - k1.x - k2.x * ((v.x - mu.x) * rs.x);
-        o.y = k0.y * (fmaf(sc.y, v.y, sh.y) > 0.f ? g.y : 0.f) - k1.y - k2.y * ((v.y - mu.y) * rs.y);
-        o.z = k0.z * (fmaf(sc.z, v.z, sh.z) > 0.f ? g.z : 0.f) - k1.z - k2.z * ((v.z - mu.z) * rs.z);
-        o.w = k0.w * (fmaf(sc.w, v.w, sh.w) > 0.f ? g.w : 0.f) - k1.w - k2.w * ((v.w - mu.w) * rs.w);
-        if (OUT == 2) {
-            float4 p = add.ld4(row, c);
-            o.x += p.x; o.y += p.y; o.z += p.z; o.w += p.w;
+    const size_t gtid = (size_t)blockIdx.x * blockDim.x + threadIdx.x, nth = (size_t)gridDim.x * blockDim.x;
+    const int q = (int)(gtid % C4), c = q * 4;
+    const size_t row0 = gtid / C4, row_step = nth / C4;
+    float4 sc, sh, mu, rs;
+    bn_coef4(bn, c, sc, sh, mu, rs);
+    const float4 k0 = ld4(coef + c), k1 = ld4(coef + C + c), k2 = ld4(coef + 2 * C + c);
+    for (size_t rb = row0; rb < P; rb += 4 * row_step) {
+        float4 v[4], g[4], pa[4];
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            const size_t row = rb + j * row_step;
+            if (row < P) {
+                v[j] = t.ld4(row, c); g[j] = ld4(da + row * C + c);
+                if (OUT == 2) pa[j] = add.ld4(row, c);
+            }
         }
-        if (OUT == 0) st4(out + i * 4, o);
-        else st4(outp.at(row, c), o);
-        if (CAST) st4(cast + i * 4, o);
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            const size_t row = rb + j * row_step;
+            if (row >= P) continue;
+            float4 o;
+            o.x = k0.x * (fmaf(sc.x, v[j].x, sh.x) > 0.f ? g[j].x : 0.f) - k1.x - k2.x * ((v[j].x - mu.x) * rs.x);
+            o.y = k0.y * (fmaf(sc.y, v[j].y, sh.y) > 0.f ? g[j].y : 0.f) - k1.y - k2.y * ((v[j].y - mu.y) * rs.y);
+            o.z = k0.z * (fmaf(sc.z, v[j].z, sh.z) > 0.f ? g[j].z : 0.f) - k1.z - k2.z * ((v[j].z - mu.z) * rs.z);
+            o.w = k0.w * (fmaf(sc.w, v[j].w, sh.w) > 0.f ? g[j].w : 0.f) - k1.w - k2.w * ((v[j].w - mu.w) * rs.w);
+            if (OUT == 2) { o.x += pa[j].x; o.y += pa[j].y; o.z += pa[j].z; o.w += pa[j].w; }
+            if (OUT == 0) st4(out + row * C + c, o);
+            else st4(outp.at(row, c), o);
+            if (CAST) st4(cast + row * C + c, o);
+        }
     }
+}
+
+// grid for the row-strided elementwise kernels: 256 threads per block, a thread count that is a multiple of C4
+static int row_grid(size_t P, int C4, int sm) {
+    // smallest block count g >= wanted with (g * 256) % C4 == 0: C4 divides 256 * g when g is a multiple of C4 / gcd(C4, 256)
+    int a = C4, b = 256;
+    while (b) { int r = a % b; a = b; b = r; }
+    const int unit = C4 / a;
+    size_t want = (P * C4 + 1023) / 1024, cap = (size_t)sm * 8;
+    if (want > cap) want = cap;
+    if (want < 1) want = 1;
+    return (int)((want + unit - 1) / unit * unit);
 }
 
 void bn_relu_bwd(Exec &ex, const float *da, Pair t, size_t P, BnRef bn, float *dgamma, float *dbeta, float *coef,
@@ -238,8 +265,8 @@ void bn_relu_bwd(Exec &ex, const float *da, Pair t, size_t P, BnRef bn, float *d
             launch(ex, bn_bwd_finalize, cdiv((size_t)C * 32, 128), 128, 0, part, r.chunks, C, 1.0 / (double)P, bn.gamma, bn.rstd, dgamma, dbeta, coef);
             ex.check("bn_bwd_finalize");
         }
-        size_t nq = P * C4; int g = ew_grid(nq, ex.ctx->sm_count);
-#define RV_ARGS da, t, nq, C4, bn, coef
+        const int g = row_grid(P, C4, ex.ctx->sm_count);
+#define RV_ARGS da, t, P, C4, bn, coef
         if (out_pair.p0 && add.p0) {
             if (out_cast) launch(ex, bn_relu_bwd_apply_kernel<float, 2, true>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, out_cast);
             else launch(ex, bn_relu_bwd_apply_kernel<float, 2, false>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, nullptr);

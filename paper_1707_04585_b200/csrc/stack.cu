@@ -94,6 +94,7 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
         }
         std::vector<PackJob> jobs;
         double bytes = 0;
+        size_t max_elems = 0;
         for (LayerSlot *l : slots) {
             l->wp_f = l->wp_d = nullptr;
             if (ex.mode != 0 || l->cin % 8 || l->cout % 8) continue;
@@ -103,13 +104,15 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
             jobs.push_back(tc_pack_job(params + l->off_W, f, l->cin, l->cout, l->k, false));
             jobs.push_back(tc_pack_job(params + l->off_W, dd, l->cin, l->cout, l->k, true));
             bytes += (double)(nf + nd) * 2 + (double)l->cin * l->cout * l->k * l->k * 8;
+            if (nf > max_elems) max_elems = nf;
+            if (nd > max_elems) max_elems = nd;
         }
         PackJob *jobs_dev = ex.ws.get<PackJob>(jobs.size() + 1);
         if (!ex.dry && !jobs.empty()) {
             if (jobs.size() * sizeof(PackJob) <= pl->pack_host_bytes) {
                 memcpy(pl->pack_host, jobs.data(), jobs.size() * sizeof(PackJob));
                 cudaMemcpyAsync(jobs_dev, pl->pack_host, jobs.size() * sizeof(PackJob), cudaMemcpyHostToDevice, ex.stream);
-                tc_pack_batch(ex, jobs_dev, (int)jobs.size(), bytes);
+                tc_pack_batch(ex, jobs_dev, (int)jobs.size(), bytes, max_elems);
             } else {
                 for (LayerSlot *l : slots) l->wp_f = l->wp_d = nullptr;   // no staging room: pack per call instead
             }

@@ -187,6 +187,7 @@ __device__ __forceinline__ void epilogue_tile(const EpiArgs &e, uint32_t tmem_ac
     }
 }
 
+template <int NT>
 __device__ __forceinline__ void epilogue_publish(const EpiArgs &e, float *scratch, int etid);
 
 // After the last tile: per-CTA partials, grid-wide count, and the finalize by the CTA that comes last.
@@ -212,53 +213,56 @@ __device__ __forceinline__ void epilogue_finish(const EpiArgs &e, int BN, int co
             *reinterpret_cast<float4 *>(mine + 2 * col + 4) = make_float4(r[4], r[5], r[6], r[7]);
         }
     }
-    epilogue_publish(e, scratch, etid);
+    epilogue_publish<128>(e, scratch, etid);
 }
 
 // Once every CTA has written its partial record into e.part: count, and let the CTA that comes
-// last reduce the records in a fixed order and write the results.  scratch: 8 KB of shared memory.
+// last reduce the records in a fixed order and write the results.  Called by NT threads (etid = 0..NT-1);
+// scratch: (NT + 128) * 32 bytes of shared memory.
+template <int NT>
 __device__ __forceinline__ void epilogue_publish(const EpiArgs &e, float *scratch, int etid) {
     // publish, count, and let the last CTA of the grid reduce
     __threadfence();
-    named_barrier(1, 128);
+    named_barrier(1, NT);
     unsigned int *flag = reinterpret_cast<unsigned int *>(scratch);
     if (etid == 0) {
         const unsigned int total = gridDim.x * gridDim.y;
         const unsigned int old = atomicAdd(e.counter, 1u);
         *flag = (old == total - 1) ? 1u : 0u;
     }
-    named_barrier(1, 128);
+    named_barrier(1, NT);
     const bool last = *flag != 0;
-    named_barrier(1, 128);
+    named_barrier(1, NT);
     if (!last) return;
     __threadfence();
     // A partial is a record of 2C floats = R float4 slots (per channel quad: sums, second sums).
-    // Thread = (slot, sub): it adds the records sub, sub + nsub, ... of its slot, eight loads in
+    // Thread = (slot, sub): it adds the records sub, sub + nsub, ... of its slot, ten loads in
     // flight at a time; the subs are then added in order.  All in double precision, all in an
     // order the launch shape fixes.
     const int C = e.n_cols, parts = (int)gridDim.x, R = C >> 1;
-    double *red = reinterpret_cast<double *>(scratch);            // [128][4]
-    double *tot = red + 512;                                      // [128][4]
+    double *red = reinterpret_cast<double *>(scratch);            // [NT][4]
+    double *tot = red + NT * 4;                                   // [128][4]
     for (int slot0 = 0; slot0 < R; slot0 += 128) {
         const int cw = R - slot0 < 128 ? R - slot0 : 128;         // even
-        const int nsub = 128 / cw;
+        const int nsub = NT / cw;
         const int r = etid % cw, sub = etid / cw;
         if (sub < nsub) {
             double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
             const float *src = e.part + (size_t)(slot0 + r) * 4;
-            for (int i = sub; i < parts; i += 8 * nsub) {
-                float4 v[8];
+            constexpr int kInFlight = 10;
+            for (int i = sub; i < parts; i += kInFlight * nsub) {
+                float4 v[kInFlight];
 #pragma unroll
-                for (int k = 0; k < 8; k++) {
+                for (int k = 0; k < kInFlight; k++) {
                     const int idx = i + k * nsub;
                     v[k] = idx < parts ? ldcg4(src + (size_t)idx * 2 * C) : make_float4(0.f, 0.f, 0.f, 0.f);
                 }
 #pragma unroll
-                for (int k = 0; k < 8; k++) { s0 += (double)v[k].x; s1 += (double)v[k].y; s2 += (double)v[k].z; s3 += (double)v[k].w; }
+                for (int k = 0; k < kInFlight; k++) { s0 += (double)v[k].x; s1 += (double)v[k].y; s2 += (double)v[k].z; s3 += (double)v[k].w; }
             }
             red[etid * 4] = s0; red[etid * 4 + 1] = s1; red[etid * 4 + 2] = s2; red[etid * 4 + 3] = s3;
         }
-        named_barrier(1, 128);
+        named_barrier(1, NT);
         if (etid < cw) {
             double s0 = red[etid * 4], s1 = red[etid * 4 + 1], s2 = red[etid * 4 + 2], s3 = red[etid * 4 + 3];
             for (int y = 1; y < nsub; y++) {
@@ -268,8 +272,8 @@ __device__ __forceinline__ void epilogue_publish(const EpiArgs &e, float *scratc
             double *d = tot + etid * 4;
             d[0] = s0; d[1] = s1; d[2] = s2; d[3] = s3;
         }
-        named_barrier(1, 128);
-        for (int lc = etid; lc < cw * 2; lc += 128) {             // one thread per channel of this slot range
+        named_barrier(1, NT);
+        for (int lc = etid; lc < cw * 2; lc += NT) {             // one thread per channel of this slot range
             const int k = lc >> 2, j = lc & 3;                    // local quad, lane within it
             const int ch = (slot0 >> 1) * 4 + lc;
             const double sum = tot[(2 * k) * 4 + j], sum2 = tot[(2 * k + 1) * 4 + j];
@@ -284,7 +288,7 @@ __device__ __forceinline__ void epilogue_publish(const EpiArgs &e, float *scratc
                 e.mean[ch] = (float)m; e.rstd[ch] = (float)(1.0 / sqrt(var + (double)e.eps));
             }
         }
-        named_barrier(1, 128);
+        named_barrier(1, NT);
     }
     if (etid == 0) *e.counter = 0u;
 }

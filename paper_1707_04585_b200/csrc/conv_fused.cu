@@ -73,27 +73,21 @@ __device__ __forceinline__ uint32_t relu_pack2(float lo, float hi) {
     return r;
 }
 
-// Per item = (pixel of the raw tile in the order TMA delivers it: image, row, column) x (chunk of 8
-// channels), decoded once per CTA:
-//   d01, d2 : 16-byte slot of the item in copy 0 / 1 (low / high half of d01) and copy 2 (low half of d2f),
+// Per pixel of the raw tile (in the order TMA delivers it: image, row, column), decoded once per CTA:
+//   r01, r2 : row of the pixel in operand copy 0 / 1 (low / high half of r01) and copy 2 (low half of r2f),
 //             0xffff where that copy does not hold it
-//   d2f     : bits 16-23 halo row, 24-31 image in tile
-//   raw16   : offset of its source in the raw tile, in 16-byte units
-//   flags   : bit 0: inside the tile proper (not halo); bit 1: column inside the image and channels valid;
-//             bits 8-15: halo column
-struct __align__(16) ItemRef { uint32_t d01, d2f, raw16, flags; };
+//   r2f     : bits 16-23 halo row, 24-31 image in tile
+//   flags   : bit 0: inside the tile proper (not halo); bit 1: column inside the image; bits 8-15: halo column
+struct __align__(16) ItemRef { uint32_t r01, r2f, spare, flags; };
 
 // a / b for 0 <= a < 65536 with inv_b = 1.f / b: exact, without the integer-division sequence
 __device__ __forceinline__ int small_div(int a, float inv_b) { return __float2int_rz(((float)a + 0.5f) * inv_b); }
 
-__device__ __forceinline__ void build_table(const FusedParams &p, ItemRef *tab, int items, int cshift) {
+__device__ __forceinline__ void build_table(const FusedParams &p, ItemRef *tab, int npix) {
     const int pad = p.k >> 1;
     const int WH = p.g.W + 2 * pad, HR = p.g.BH + 2 * pad;
     const float inv_wh = 1.f / (float)WH, inv_hr = 1.f / (float)HR;
-    const int row_bytes = p.KC * 2;
-    const int esize = p.in_mode == 0 ? 4 : 2;
-    for (int it = threadIdx.x; it < items; it += kFThreads) {
-        const int ck = it & ((1 << cshift) - 1), px = it >> cshift;
+    for (int px = threadIdx.x; px < npix; px += kFThreads) {
         const int rest = small_div(px, inv_wh), xh = px - rest * WH;
         const int img = small_div(rest, inv_hr), r = rest - img * HR;
         const int rowbase = (r * p.g.BIMG + img) * p.g.Wp;
@@ -103,15 +97,14 @@ __device__ __forceinline__ void build_table(const FusedParams &p, ItemRef *tab, 
 #pragma unroll
         for (int s = 0; s < 3; s++) {            // halo column xh is column xh - s of the copy for horizontal tap offset s
             const int x = xh - s;
-            const uint32_t off = swizzled_offset((uint32_t)(rowbase + (x < 0 ? 0 : x)), (uint32_t)ck, row_bytes) >> 4;
-            d[s] = (s < p.k && x >= 0 && x < p.g.W) ? off : 0xffffu;
+            d[s] = (s < p.k && x >= 0 && x < p.g.W) ? (uint32_t)(rowbase + x) : 0xffffu;
         }
         ItemRef e;
-        e.d01 = d[0] | (d[1] << 16);
-        e.d2f = d[2] | ((uint32_t)r << 16) | ((uint32_t)img << 24);
-        e.raw16 = (uint32_t)((px * p.cin + ck * 8) * esize) >> 4;
-        e.flags = (interior ? 1u : 0u) | ((xin && ck < (p.cin >> 3)) ? 2u : 0u) | ((uint32_t)xh << 8);
-        tab[it] = e;
+        e.r01 = d[0] | (d[1] << 16);
+        e.r2f = d[2] | ((uint32_t)r << 16) | ((uint32_t)img << 24);
+        e.spare = 0;
+        e.flags = (interior ? 1u : 0u) | (xin ? 2u : 0u) | ((uint32_t)xh << 8);
+        tab[px] = e;
     }
 }
 
@@ -121,9 +114,14 @@ __device__ __forceinline__ void build_table(const FusedParams &p, ItemRef *tab, 
 // Written without branches in the per-item work (invalid items compute on the zeros TMA delivered and are
 // masked, stores that do not exist go to a dummy slot), so that the four items of a batch interleave.
 template <int IN_MODE>
-__device__ __forceinline__ void build_tile(const FusedParams &p, FusedShared *sh, const ItemRef *tab, int items, int ck,
+__device__ __forceinline__ void build_tile(const FusedParams &p, FusedShared *sh, const ItemRef *tab, int items, int cshift, int ck,
                                            const uint8_t *raw, uint8_t *A, int n0, int h0) {
     const int pad = p.k >> 1;
+    // 16-byte slot of chunk ck in row `row` of a copy: the chunk index is XORed with row bits as the TMA swizzle does
+    const int swz_sh = 3 - cshift;
+    const uint32_t swz_mask = (1u << cshift) - 1u;
+    const bool ck_valid = ck < (p.cin >> 3);
+    const uint32_t raw_px16 = (uint32_t)(p.cin * (IN_MODE == 1 ? 2 : 4)) >> 4, raw_ck16 = (uint32_t)(ck * (IN_MODE == 1 ? 1 : 2));
     // scale and shift of this thread's eight channels; a fixed-point input folds its step into the scale (a power of two: exact)
     float sc[8], sf[8];
     if (IN_MODE != 1) {
@@ -140,11 +138,12 @@ __device__ __forceinline__ void build_tile(const FusedParams &p, FusedShared *sh
         for (int j = 0; j < 4; j++) {
             const int it = base + j * kFThreads;
             const bool exists = it < items;
-            ref[j] = tab[exists ? it : items - 1];
-            const int r = (ref[j].d2f >> 16) & 0xff, img = ref[j].d2f >> 24;
-            ok[j] = exists && (ref[j].flags & 2u) && (unsigned)(h0 - pad + r) < (unsigned)p.g.H && n0 + img < p.g.N;
-            if (!exists) { ref[j].d01 = 0xffffffffu; ref[j].d2f |= 0xffffu; }
-            const uint4 *src = reinterpret_cast<const uint4 *>(raw) + ref[j].raw16;
+            const uint32_t px = (uint32_t)(exists ? it : items - 1) >> cshift;
+            ref[j] = tab[px];
+            const int r = (ref[j].r2f >> 16) & 0xff, img = ref[j].r2f >> 24;
+            ok[j] = exists && ck_valid && (ref[j].flags & 2u) && (unsigned)(h0 - pad + r) < (unsigned)p.g.H && n0 + img < p.g.N;
+            if (!exists) { ref[j].r01 = 0xffffffffu; ref[j].r2f |= 0xffffu; }
+            const uint4 *src = reinterpret_cast<const uint4 *>(raw) + (px * raw_px16 + raw_ck16);
             const uint4 lo = src[0];
             if (IN_MODE == 1) {
                 v[j] = lo;
@@ -164,16 +163,19 @@ __device__ __forceinline__ void build_tile(const FusedParams &p, FusedShared *sh
             }
             const uint32_t keep = ok[j] ? 0xffffffffu : 0u;       // outside the image: zero, whatever BN makes of the zeros delivered
             v[j].x &= keep; v[j].y &= keep; v[j].z &= keep; v[j].w &= keep;
-            const uint32_t d0 = ref[j].d01 & 0xffffu, d1 = ref[j].d01 >> 16, d2 = ref[j].d2f & 0xffffu;
-            *reinterpret_cast<uint4 *>(A + (d0 != 0xffffu ? (d0 << 4) : dummy)) = v[j];
-            *reinterpret_cast<uint4 *>(A + (d1 != 0xffffu ? p.copy_bytes + (d1 << 4) : dummy)) = v[j];
-            *reinterpret_cast<uint4 *>(A + (d2 != 0xffffu ? 2 * p.copy_bytes + (d2 << 4) : dummy)) = v[j];
+            const uint32_t r0 = ref[j].r01 & 0xffffu, r1 = ref[j].r01 >> 16, r2 = ref[j].r2f & 0xffffu;
+            const uint32_t o0 = ((r0 << cshift) + ((uint32_t)ck ^ ((r0 >> swz_sh) & swz_mask))) << 4;
+            const uint32_t o1 = ((r1 << cshift) + ((uint32_t)ck ^ ((r1 >> swz_sh) & swz_mask))) << 4;
+            const uint32_t o2 = ((r2 << cshift) + ((uint32_t)ck ^ ((r2 >> swz_sh) & swz_mask))) << 4;
+            *reinterpret_cast<uint4 *>(A + (r0 != 0xffffu ? o0 : dummy)) = v[j];
+            *reinterpret_cast<uint4 *>(A + (r1 != 0xffffu ? p.copy_bytes + o1 : dummy)) = v[j];
+            *reinterpret_cast<uint4 *>(A + (r2 != 0xffffu ? 2 * p.copy_bytes + o2 : dummy)) = v[j];
         }
         if (IN_MODE != 1 && p.a_out) {
 #pragma unroll
             for (int j = 0; j < 4; j++)
                 if (ok[j] && (ref[j].flags & 1u)) {
-                    const int r = (ref[j].d2f >> 16) & 0xff, img = ref[j].d2f >> 24, xh = (ref[j].flags >> 8) & 0xff;
+                    const int r = (ref[j].r2f >> 16) & 0xff, img = ref[j].r2f >> 24, xh = (ref[j].flags >> 8) & 0xff;
                     const size_t gp = ((size_t)(n0 + img) * p.g.H + (h0 - pad + r)) * p.g.W + (xh - pad);
                     *reinterpret_cast<uint4 *>(p.a_out + gp * p.cin + ck * 8) = v[j];
                 }
@@ -321,17 +323,8 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tma_prefetch_desc(&map_w); tma_prefetch_desc(&map_in); tma_prefetch_desc(&map_out);
         if (need_aux) tma_prefetch_desc(&map_aux);
-    }
-    if (warp == 0) tmem_alloc(&sh->tmem_base, tmem_cols);
-    build_table(p, tab, items, cshift);
-    if (threadIdx.x < 128) {
-        // accumulator row (image row, image, column) -> pixel of the (image, row, column) ordered tile
-        const int w = etid % p.g.Wp, img = (etid / p.g.Wp) % p.g.BIMG, h = etid / (p.g.BIMG * p.g.Wp);
-        sh->srow[etid] = (w < p.g.W && h < p.g.BH) ? (img * p.g.BH + h) * p.g.W + w : -1;
-    }
-    // everything above is independent of what earlier kernels wrote and may overlap the kernel before
-    pdl_enter();
-    if (threadIdx.x == 0) {
+        // the first loads fly while the CTA builds its index tables
+        pdl_enter();
         mbar_expect_tx(&sh->w_full, (uint32_t)(taps * p.BN * p.KC * 2));
         for (int tap = 0; tap < taps; tap++) tma_load_2d(wres + tap * p.wtile_bytes, &map_w, &sh->w_full, tap * p.KC, col0);
         if (cur.t < NT) {
@@ -339,7 +332,17 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
             if (need_aux) load_aux(cur, 0);
             if (p.NB == 2 && nx1.t < NT) load_raw(nx1, 1);
         }
-    } else if (threadIdx.x >= 128 && threadIdx.x < 192) {
+    }
+    if (warp == 0) tmem_alloc(&sh->tmem_base, tmem_cols);
+    build_table(p, tab, npix);
+    if (threadIdx.x < 128) {
+        // accumulator row (image row, image, column) -> pixel of the (image, row, column) ordered tile
+        const int w = etid % p.g.Wp, img = (etid / p.g.Wp) % p.g.BIMG, h = etid / (p.g.BIMG * p.g.Wp);
+        sh->srow[etid] = (w < p.g.W && h < p.g.BH) ? (img * p.g.BH + h) * p.g.W + w : -1;
+    }
+    // the tables above are independent of what earlier kernels wrote; everything below is not
+    pdl_enter();
+    if (threadIdx.x >= 128 && threadIdx.x < 192) {
         const int c = threadIdx.x - 128;
         float sc = 0.f, sf = 0.f;
         if (p.in_mode == 0 && c < p.cin) bn_sc_sh(p.bn.gamma[c], p.bn.beta[c], p.bn.mean[c], p.bn.rstd[c], sc, sf);
@@ -383,9 +386,9 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
         ok = __syncthreads_and(ok);
         if (!ok) break;
         // ---- build the operand
-        if (p.in_mode == 1) build_tile<1>(p, sh, tab, items, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
-        else if (p.in_q == 0.f) build_tile<0>(p, sh, tab, items, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
-        else build_tile<2>(p, sh, tab, items, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
+        if (p.in_mode == 1) build_tile<1>(p, sh, tab, items, cshift, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
+        else if (p.in_q == 0.f) build_tile<0>(p, sh, tab, items, cshift, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
+        else build_tile<2>(p, sh, tab, items, cshift, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
         fence_proxy_async();
         __syncthreads();
         if (threadIdx.x == 0) {
@@ -479,7 +482,7 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
             *reinterpret_cast<float4 *>(mine + 4) = make_float4(r[4], r[5], r[6], r[7]);
         }
         __syncthreads();
-        if (warp < 4) epilogue_publish(e, scratch, etid);
+        epilogue_publish<kFThreads>(e, scratch, (int)threadIdx.x);
     }
     if (!ok && threadIdx.x == 0) atomicExch(&sh->failed, 1u);
     tc_fence_before();
@@ -522,7 +525,7 @@ bool fused_shape(Geom g, int cin, int cout, int k, int in_esize, int sm_count, F
     const int copy_rows = (s.g.BH + k - 1) * s.g.BIMG * s.g.Wp;
     s.copy_bytes = (copy_rows * s.KC * 2 + 1023) & ~1023;
     const int npix = (s.g.BH + 2 * pad) * s.g.BIMG * (s.g.W + 2 * pad);
-    s.a_bytes = k * s.copy_bytes > 8192 ? k * s.copy_bytes : 8192;      // also scratch of the final reduction
+    s.a_bytes = k * s.copy_bytes > 12288 ? k * s.copy_bytes : 12288;      // also scratch of the final reduction
     s.raw_bytes = (npix * cin * in_esize + 1023) & ~1023;
     for (;;) {
         s.n_tiles = (cout_pad + s.BN - 1) / s.BN;
@@ -531,7 +534,7 @@ bool fused_shape(Geom g, int cin, int cout, int k, int in_esize, int sm_count, F
         s.group_bytes = (s.g.BH * s.g.BIMG * s.g.W * s.GW * 4 + 1023) & ~1023;
         s.aux_bytes = (s.BN / s.GW) * s.group_bytes;
         auto smem_of = [&](int NB) { return 1024 + s.a_bytes + k * k * s.wtile_bytes + NB * (s.raw_bytes + s.aux_bytes) + s.aux_bytes +
-                                            (int)sizeof(FusedShared) + npix * (s.KC / 8) * 16 + 64; };
+                                            (int)sizeof(FusedShared) + npix * 16 + 64; };
         const int two_per_sm = 113 * 1024;
         if (smem_of(2) <= two_per_sm) s.NB = 2;
         else if (smem_of(1) <= two_per_sm) s.NB = 1;

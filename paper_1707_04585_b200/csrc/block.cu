@@ -16,6 +16,8 @@
 bool conv_fprop_tc(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign, Moments *stats);
 bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, const BnBwdReq *bb);
 bool conv_wgrad_tc(Exec &ex, const void *g, const void *a, Geom gi, const Layer &L, float *dW, float *scratch, size_t *need);
+bool conv_wgrad_tc_batch(Exec &ex, int n, const void *const *gq, const void *const *a, const Geom *gi, const Layer *const *L,
+                         float *scratch, size_t *need);
 // one kernel for BN -> ReLU -> conv (at most 64 input channels, stride 1); likewise the data gradient of such a layer
 bool conv_fprop_fused(Exec &ex, Pair t, BnRef bn, Geom gi, const Layer &L, Pair out, Pair partner, int sign, Moments *stats, bf16 *a_out);
 bool conv_dgrad_fused(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, const BnBwdReq *bb);
@@ -127,31 +129,33 @@ void fn_backward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, FnS
             gcur = buf;
         }
     }
-    // The weight gradients of the function depend only on tensors that already exist when their
-    // layer's turn comes, so they run on a side stream beside the data-gradient chain (fork before
-    // each, one join at the end); their split partials get a buffer of their own for that time.
-    bool side = b16 && ex.use_side && (ex.dry || (ex.ctx->side_stream && !ex.ctx->profiling));
+    // The weight gradients of the function's layers run as ONE launch on a side stream, beside the
+    // last layer's data gradient: by then every operand exists (the gradient entering layer 0 is the
+    // last one produced).  One launch amortises set-up and split partials over the layers; the split
+    // partials get a buffer of their own for that time.  Functions of more than four layers, shapes
+    // the tensor-core kernel does not take, and profiling runs go layer by layer on the main stream.
+    bool side = b16 && ex.use_side && L <= 4 && (ex.dry || (ex.ctx->side_stream && !ex.ctx->profiling));
     size_t wg_need = 0;
-    for (int l = 0; l < L && side; l++) {
-        size_t n = 0;
-        if (!conv_wgrad_tc(ex, nullptr, nullptr, gin[l], layers[l], nullptr, nullptr, &n)) side = false;
-        else if (n > wg_need) wg_need = n;
-    }
+    std::vector<const Layer *> lptr(L);
+    std::vector<const void *> gq(L), aq(L);
+    for (int l = 0; l < L; l++) { lptr[l] = &layers[l]; aq[l] = saved.a[l]; }
+    if (side && !conv_wgrad_tc_batch(ex, L, gq.data(), aq.data(), gin.data(), lptr.data(), nullptr, &wg_need)) side = false;
     float *wg_scratch = side && wg_need ? ex.ws.get<float>(wg_need) : nullptr;
     for (int l = L - 1; l >= 0; l--) {
         const Layer &ly = layers[l];
         const size_t P = gin[l].P();
-        if (side) {
+        gq[l] = gcur;
+        if (!side) {
+            conv_wgrad(ex, gcur, saved.a[l], gin[l], ly, ly.dW);
+        } else if (l == 0) {
             cudaStream_t main = ex.stream;
             if (!ex.dry) {
                 cudaEventRecord(ex.ctx->ev_fork, main);
                 cudaStreamWaitEvent(ex.ctx->side_stream, ex.ctx->ev_fork, 0);
                 ex.stream = ex.ctx->side_stream;
             }
-            conv_wgrad_tc(ex, gcur, saved.a[l], gin[l], ly, ly.dW, wg_scratch, nullptr);
+            conv_wgrad_tc_batch(ex, L, gq.data(), aq.data(), gin.data(), lptr.data(), wg_scratch, nullptr);
             ex.stream = main;
-        } else {
-            conv_wgrad(ex, gcur, saved.a[l], gin[l], ly, ly.dW);
         }
         float *da = ex.ws.get<float>(P * ly.cin);
         float *coef = ex.ws.get<float>((size_t)3 * ly.cin);

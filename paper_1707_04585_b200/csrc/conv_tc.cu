@@ -328,7 +328,7 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
 // stacks (tap, input-channel block) tiles -- one shifted TMA box each -- 128 rows per MMA group;
 // the N side is a block of output channels.  A CTA owns up to two M groups and one N tile, walks
 // its share of the pixel tiles (split-K) accumulating in tensor memory, and writes an fp32
-// partial; the partials are summed in fixed order by splitk_sum_kernel.
+// partial; the partials are summed in fixed order by splitk_sum_batch_kernel.
 struct WgParams {
     int taps, k;
     int blockC, cblks, cin;      // input-channel block (16/32/64), blocks per tap, valid channels
@@ -340,13 +340,27 @@ struct WgParams {
     int stride;
     int n_tiles_px;              // pixel tiles in all
     int stages;
-    float *partial;              // [splits][cout][taps][cin]
+    float *partial;              // splits > 1: [splits][taps][cin][cout], summed and transposed afterwards; else the gradient itself
     size_t slice;                // cout*taps*cin
     int *status;
+    int splits, m_chunks;        // this job's CTAs: split x M chunk x N tile, split fastest
+    int cta0;                    // first CTA of the job in the launch
 };
 
+// One launch computes the weight gradients of up to kWgMaxJobs layers: each CTA finds its job from
+// its index and then works on that layer alone.
+constexpr int kWgMaxJobs = 4;
+struct alignas(64) WgJob { CUtensorMap map_a, map_g; WgParams p; };
+struct WgBatch { WgJob job[kWgMaxJobs]; int n; };
+
 __global__ void __launch_bounds__(kThreads, 1)
-wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_g, const WgParams p) {
+wgrad_tc_kernel(const __grid_constant__ WgBatch batch) {
+    int jb = 0;
+    while (jb + 1 < batch.n && (int)blockIdx.x >= batch.job[jb + 1].p.cta0) jb++;
+    const WgParams &p = batch.job[jb].p;
+    const CUtensorMap &map_a = batch.job[jb].map_a, &map_g = batch.job[jb].map_g;
+    const int local = (int)blockIdx.x - p.cta0;
+    const int split = local % p.splits, chunk = (local / p.splits) % p.m_chunks, ntile = local / (p.splits * p.m_chunks);
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const int blk_bytes_a = 256 * p.blockC, blk_bytes_b = 256 * p.blockN;   // [128 pixels][block] bf16
@@ -356,12 +370,12 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bpg = 128 / p.blockC;                          // blocks per M group
-    const int first_block = blockIdx.y * p.GM * bpg;
+    const int first_block = chunk * p.GM * bpg;
     int n_blocks = p.total_blocks - first_block; if (n_blocks > p.GM * bpg) n_blocks = p.GM * bpg;
     const int groups = (n_blocks + bpg - 1) / bpg;
-    const int col0 = blockIdx.z * p.BN;
+    const int col0 = ntile * p.BN;
     int nb_n = (p.cout - col0 + p.blockN - 1) / p.blockN; if (nb_n > p.BN / p.blockN) nb_n = p.BN / p.blockN;   // N blocks holding valid channels
-    const int my_tiles = (p.n_tiles_px - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;
+    const int my_tiles = (p.n_tiles_px - split + p.splits - 1) / p.splits;
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < p.GM * p.BN) tmem_cols <<= 1;
 
@@ -388,24 +402,29 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const int tiles_per_img = p.tiles_per_img;
 
     if (warp == 0) {
-        if (lane == 0) {
-            const uint32_t tx = (uint32_t)(p.box_px * 2 * (n_blocks * p.blockC + nb_n * p.blockN));
-            for (int it = 0; it < my_tiles; it++) {
-                const int s = it % p.stages, round = it / p.stages;
-                if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); break; }
-                const int t = blockIdx.x + it * gridDim.x;
-                const int n0 = p.BIMG > 1 ? t * p.BIMG : t / tiles_per_img;
-                const int h0 = p.BIMG > 1 ? 0 : (t % tiles_per_img) * p.BH;
-                uint8_t *sa = tiles + s * stage_bytes;
-                mbar_expect_tx(&sh->full[s], tx);
-                for (int b = 0; b < n_blocks; b++) {
-                    const int gb = first_block + b, tap = gb / p.cblks, cb = gb - tap * p.cblks;
-                    const int kh = tap / p.k, kw = tap - kh * p.k;
-                    tma_load_4d(sa + b * blk_bytes_a, &map_a, &sh->full[s], cb * p.blockC, kw - pad, h0 * p.stride + kh - pad, n0);
-                }
-                for (int b = 0; b < nb_n; b++)
-                    tma_load_4d(sa + a_region + b * blk_bytes_b, &map_g, &sh->full[s], col0 + b * p.blockN, 0, h0, n0);
+        // producer warp: lane 0 waits for the slot and arms the barrier, then every lane issues one box
+        // (lane b < n_blocks: shifted activation block b; the next nb_n lanes: gradient blocks), so that
+        // the loads of a tile leave in one instruction instead of one after the other
+        const uint32_t tx = (uint32_t)(p.box_px * 2 * (n_blocks * p.blockC + nb_n * p.blockN));
+        const bool a_lane = lane < n_blocks, g_lane = !a_lane && lane < n_blocks + nb_n;
+        const int gb = first_block + lane, tap = gb / p.cblks, cb = gb - tap * p.cblks;
+        const int kh = tap / p.k, kw = tap - kh * p.k;
+        const int bg = lane - n_blocks;
+        for (int it = 0; it < my_tiles; it++) {
+            const int s = it % p.stages, round = it / p.stages;
+            bool ok = true;
+            if (lane == 0) {
+                if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; }
+                if (ok) mbar_expect_tx(&sh->full[s], tx);
             }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            const int t = split + it * p.splits;
+            const int n0 = p.BIMG > 1 ? t * p.BIMG : t / tiles_per_img;
+            const int h0 = p.BIMG > 1 ? 0 : (t % tiles_per_img) * p.BH;
+            uint8_t *sa = tiles + s * stage_bytes;
+            if (a_lane) tma_load_4d(sa + lane * blk_bytes_a, &map_a, &sh->full[s], cb * p.blockC, kw - pad, h0 * p.stride + kh - pad, n0);
+            else if (g_lane) tma_load_4d(sa + a_region + bg * blk_bytes_b, &map_g, &sh->full[s], col0 + bg * p.blockN, 0, h0, n0);
         }
     } else if (warp == 1) {
         if (lane == 0) {
@@ -434,7 +453,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         if (ok && sh->failed == 0) {
             const int m = quarter * 32 + lane;
-            float *dst = p.partial + (size_t)blockIdx.x * p.slice;
+            float *dst = p.partial + (size_t)split * p.slice;
             for (int g = 0; g < groups; g++) {
                 const int gb = first_block + g * bpg + m / p.blockC;
                 const int tap = gb / p.cblks, ci = (gb - tap * p.cblks) * p.blockC + m % p.blockC;
@@ -442,11 +461,22 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                 for (int c = 0; c < p.BN; c += 16) {
                     float v[16];
                     tmem_ld16(tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(g * p.BN + c), v);   // whole warp takes part
-                    if (row_ok) {
+                    if (!row_ok) continue;
+                    if (my_tiles == 0) {
+#pragma unroll
+                        for (int j = 0; j < 16; j++) v[j] = 0.f;
+                    }
+                    if (p.splits > 1) {
+                        // split partials are [tap][ci][co]: this row's output channels are contiguous (cout is a multiple of 8)
+                        float *row = dst + ((size_t)tap * p.cin + ci) * p.cout + col0 + c;
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4)
+                            if (col0 + c + j < p.cout) *reinterpret_cast<float4 *>(row + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    } else {
 #pragma unroll
                         for (int j = 0; j < 16; j++) {
                             const int co = col0 + c + j;
-                            if (co < p.cout) dst[((size_t)co * p.taps + tap) * p.cin + ci] = my_tiles > 0 ? v[j] : 0.f;
+                            if (co < p.cout) dst[((size_t)co * p.taps + tap) * p.cin + ci] = v[j];
                         }
                     }
                 }
@@ -464,11 +494,17 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
 }
 
-// out[i] = sum over splits of part[z][i], in a fixed order: 8 interleaved groups of splits per
-// element, combined through shared memory (256 threads = 32 elements x 8 groups)
-__global__ void splitk_sum_kernel(const float *__restrict__ part, size_t n, int splits, float *__restrict__ out) {
+// dW[co][tap][ci] = sum over splits of part[z][tap][ci][co], in a fixed order: 8 interleaved groups of
+// splits per element, combined through shared memory (256 threads = 32 elements x 8 groups); several
+// (partials, destination) pairs in one launch, blockIdx.y picks the pair
+struct SumBatch { const float *part[kWgMaxJobs]; float *out[kWgMaxJobs]; size_t n[kWgMaxJobs]; int splits[kWgMaxJobs], cout[kWgMaxJobs], rows[kWgMaxJobs]; };
+__global__ void splitk_sum_batch_kernel(const SumBatch b) {
     pdl_enter();
     __shared__ float sm[8][33];
+    const int j = blockIdx.y;
+    const float *__restrict__ part = b.part[j];
+    const size_t n = b.n[j];
+    const int splits = b.splits[j];
     const int e = threadIdx.x & 31, grp = threadIdx.x >> 5;
     const size_t i = (size_t)blockIdx.x * 32 + e;
     float s = 0.f;
@@ -478,7 +514,9 @@ __global__ void splitk_sum_kernel(const float *__restrict__ part, size_t n, int 
     __syncthreads();
     if (grp == 0 && i < n) {
         for (int g = 1; g < 8; g++) s += sm[g][e];
-        out[i] = s;
+        const size_t row = i / (size_t)b.cout[j];              // (tap, ci)
+        const int co = (int)(i - row * (size_t)b.cout[j]);
+        b.out[j][(size_t)co * b.rows[j] + row] = s;
     }
 }
 
@@ -510,17 +548,16 @@ bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, 
 }
 
 
-// scratch: room for the split partials if the caller provides it (else it comes from the arena);
-// need: if non-null the call only reports whether it takes the shape and how many floats of scratch it wants
-bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer &L, float *dW, float *scratch, size_t *need) {
+// Shape decisions of one layer's weight gradient; cta_budget: the CTAs the job may take
+struct WgPlan { WgParams p; Geom go; int n_tiles, stage_bytes; };
+static bool wgrad_plan(Geom gi, const Layer &L, int cta_budget, WgPlan &w) {
     if ((L.stride != 1 && L.stride != 2) || (L.k != 1 && L.k != 3) || L.cin % 8 || L.cout % 8) return false;
     if (L.stride == 2 && (gi.H % 2 || gi.W % 2)) return false;
-    WgParams p;
-    const Geom go{gi.N, conv_out(gi.H, L.k, L.stride), conv_out(gi.W, L.k, L.stride)};   // tiles walk the output pixels
+    WgParams &p = w.p;
+    w.go = Geom{gi.N, conv_out(gi.H, L.k, L.stride), conv_out(gi.W, L.k, L.stride)};   // tiles walk the output pixels
     TileGeom tg;
-    if (!tile_geom(go, tg) || tg.W * L.stride > 256 || tg.BH * L.stride > 256) return false;
+    if (!tile_geom(w.go, tg) || tg.W * L.stride > 256 || tg.BH * L.stride > 256) return false;
     p.BH = tg.BH; p.BIMG = tg.BIMG; p.tiles_per_img = tg.tiles_per_img; p.box_px = tg.BIMG * tg.BH * tg.W;
-    if (!ex.dry && !encoder(ex.ctx)) return false;
     const int taps = L.k * L.k, cin_pad = round_up(L.cin, 16), cout_pad = round_up(L.cout, 16);
     p.taps = taps; p.k = L.k; p.cin = L.cin; p.cout = L.cout;
     p.blockC = pick_block(cin_pad); p.cblks = cin_pad / p.blockC; p.total_blocks = taps * p.cblks;
@@ -530,43 +567,92 @@ bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer
     const int bpg = 128 / p.blockC;
     const int groups_all = (p.total_blocks + bpg - 1) / bpg;
     p.GM = groups_all >= 2 ? 2 : 1;
-    const int m_chunks = (groups_all + p.GM - 1) / p.GM;
-    const int n_tiles = (cout_pad + p.BN - 1) / p.BN;
-    p.H = go.H; p.W = go.W; p.stride = L.stride;
+    p.m_chunks = (groups_all + p.GM - 1) / p.GM;
+    w.n_tiles = (cout_pad + p.BN - 1) / p.BN;
+    p.H = w.go.H; p.W = w.go.W; p.stride = L.stride;
     p.n_tiles_px = tg.n_px_tiles;
-    const int stage_bytes = p.GM * 32768 + ((256 * p.BN + 1023) & ~1023);
-    p.stages = (200 * 1024 - 2048) / stage_bytes; if (p.stages > kStages) p.stages = kStages;
+    w.stage_bytes = p.GM * 32768 + ((256 * p.BN + 1023) & ~1023);
+    p.stages = (200 * 1024 - 2048) / w.stage_bytes; if (p.stages > kStages) p.stages = kStages;
     if (p.stages < 2) return false;
-    // split the pixel reduction so that the grid covers the machine once
-    int splits = (ex.ctx->sm_count + m_chunks * n_tiles - 1) / (m_chunks * n_tiles);
+    // split the pixel reduction so that the job's CTAs cover its share of the machine once
+    int splits = (cta_budget + p.m_chunks * w.n_tiles - 1) / (p.m_chunks * w.n_tiles);
     if (splits > p.n_tiles_px) splits = p.n_tiles_px;
     if (splits < 1) splits = 1;
+    p.splits = splits;
     p.slice = (size_t)L.cout * taps * L.cin;
-    if (need) { *need = splits > 1 ? (size_t)splits * p.slice : 0; return true; }
-    ex.flops += 2ull * go.P() * L.cout * L.cin * taps;
+    return true;
+}
+
+// Weight gradients of n layers (n <= 4) in one launch, and one more launch that sums their split partials.
+// scratch: room for the split partials if the caller provides it (else it comes from the arena);
+// need: if non-null the call only reports whether it takes the shapes and how many floats of scratch it wants
+bool conv_wgrad_tc_batch(Exec &ex, int n, const void *const *gq, const void *const *a, const Geom *gi, const Layer *const *L,
+                         float *scratch, size_t *need) {
+    if (n < 1 || n > kWgMaxJobs) return false;
+    WgPlan w[kWgMaxJobs];
+    const int budget = ex.ctx->sm_count / n;
+    size_t total = 0;
+    for (int j = 0; j < n; j++) {
+        if (!wgrad_plan(gi[j], *L[j], budget, w[j])) return false;
+        if (w[j].p.splits > 1) total += (size_t)w[j].p.splits * w[j].p.slice;
+    }
+    if (need) { *need = total; return true; }
+    if (!ex.dry && !encoder(ex.ctx)) return false;
     size_t m = ex.ws.mark();
-    float *part = splits > 1 ? (scratch ? scratch : ex.ws.get<float>((size_t)splits * p.slice)) : dW;
+    float *part = total ? (scratch ? scratch : ex.ws.get<float>(total)) : nullptr;
+    for (int j = 0; j < n; j++) ex.flops += 2ull * w[j].go.P() * L[j]->cout * L[j]->cin * w[j].p.taps;
     if (!ex.dry) {
-        CUtensorMap map_a, map_g;
-        if (!encode_act_map(ex, &map_a, a, gi, L.cin, p.blockC, go.W, p.BH, p.BIMG, L.stride) ||
-            !encode_act_map(ex, &map_g, gq, go, L.cout, p.blockN, go.W, p.BH, p.BIMG, 1)) {
-            ex.failed = true; ex.ctx->err = "conv_wgrad_tc: tensor map rejected"; ex.ws.release(m); return true;
+        WgBatch batch;
+        SumBatch sums;
+        batch.n = n;
+        int cta = 0, smem = 0, n_sums = 0;
+        size_t off = 0, max_slice = 0;
+        double bytes = 0, flops = 0, sum_bytes = 0;
+        for (int j = 0; j < n; j++) {
+            WgParams &p = w[j].p;
+            if (!encode_act_map(ex, &batch.job[j].map_a, a[j], gi[j], L[j]->cin, p.blockC, w[j].go.W, p.BH, p.BIMG, L[j]->stride) ||
+                !encode_act_map(ex, &batch.job[j].map_g, gq[j], w[j].go, L[j]->cout, p.blockN, w[j].go.W, p.BH, p.BIMG, 1)) {
+                ex.failed = true; ex.ctx->err = "conv_wgrad_tc: tensor map rejected"; ex.ws.release(m); return true;
+            }
+            p.status = ex.ctx->dev_status;
+            p.cta0 = cta;
+            cta += p.splits * p.m_chunks * w[j].n_tiles;
+            if (p.splits > 1) {
+                p.partial = part + off;
+                sums.part[n_sums] = p.partial; sums.out[n_sums] = L[j]->dW; sums.n[n_sums] = p.slice; sums.splits[n_sums] = p.splits;
+                sums.cout[n_sums] = L[j]->cout; sums.rows[n_sums] = p.taps * L[j]->cin;
+                n_sums++;
+                off += (size_t)p.splits * p.slice;
+                if (p.slice > max_slice) max_slice = p.slice;
+                sum_bytes += (double)p.slice * 4 * (p.splits + 1);
+            } else {
+                p.partial = L[j]->dW;
+            }
+            batch.job[j].p = p;
+            const int sm = 1024 + p.stages * w[j].stage_bytes + (int)sizeof(TcShared) + 64;
+            if (sm > smem) smem = sm;
+            bytes += (double)gi[j].P() * L[j]->cin * 2 + (double)w[j].go.P() * L[j]->cout * 2 + (double)p.slice * 4 * p.splits;
+            flops += 2.0 * w[j].go.P() * L[j]->cout * L[j]->cin * p.taps;
         }
-        p.partial = part; p.status = ex.ctx->dev_status;
         static bool attr_set = false;
         if (!attr_set) { cudaFuncSetAttribute(wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); attr_set = true; }
-        const int smem = 1024 + p.stages * stage_bytes + (int)sizeof(TcShared) + 64;
-        dim3 grid((unsigned)splits, (unsigned)m_chunks, (unsigned)n_tiles);
-        launch(ex, wgrad_tc_kernel, grid, kThreads, smem, map_a, map_g, p);
-        const double bytes = (double)gi.P() * L.cin * 2 + (double)go.P() * L.cout * 2 + (double)p.slice * 4 * (splits > 1 ? splits : 1);
-        ex.check("conv_wgrad_tc", bytes, 2.0 * go.P() * L.cout * L.cin * taps);
-        if (splits > 1) {
-            launch(ex, splitk_sum_kernel, (unsigned)((p.slice + 31) / 32), 256, 0, part, p.slice, splits, dW);
-            ex.check("splitk_sum", (double)p.slice * 4 * (splits + 1));
+        launch(ex, wgrad_tc_kernel, (unsigned)cta, kThreads, smem, batch);
+        ex.check("conv_wgrad_tc", bytes, flops);
+        if (n_sums) {
+            dim3 grid((unsigned)((max_slice + 31) / 32), (unsigned)n_sums);
+            launch(ex, splitk_sum_batch_kernel, grid, 256, 0, sums);
+            ex.check("splitk_sum", sum_bytes);
         }
     }
     ex.ws.release(m);
     return true;
+}
+
+bool conv_wgrad_tc(Exec &ex, const void *gq, const void *a, Geom gi, const Layer &L, float *dW, float *scratch, size_t *need) {
+    Layer one = L;
+    one.dW = dW;
+    const Layer *lp = &one;
+    return conv_wgrad_tc_batch(ex, 1, &gq, &a, &gi, &lp, scratch, need);
 }
 
 void *tc_encoder(revnet_ctx *ctx) { return (void *)encoder(ctx); }

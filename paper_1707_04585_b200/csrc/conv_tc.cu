@@ -343,6 +343,7 @@ struct WgParams {
     float *partial;              // splits > 1: [splits][taps][cin][cout], summed and transposed afterwards; else the gradient itself
     size_t slice;                // cout*taps*cin
     int *status;
+    int a_region;                // bytes of a stage that hold activation blocks (the gradient blocks follow)
     int splits, m_chunks;        // this job's CTAs: split x M chunk x N tile, split fastest
     int cta0;                    // first CTA of the job in the launch
 };
@@ -364,7 +365,10 @@ wgrad_tc_kernel(const __grid_constant__ WgBatch batch) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const int blk_bytes_a = 256 * p.blockC, blk_bytes_b = 256 * p.blockN;   // [128 pixels][block] bf16
-    const int a_region = p.GM * 32768;                                       // 128 M rows x 128 pixels x 2 B per group
+    // a stage holds only the blocks a CTA really loads.  An M group is 128 rows = 32 KB from its first block:
+    // the MMAs of a group that is not full read on into what follows (their rows of the result are never
+    // stored), so the launch reserves room behind the last stage for that.
+    const int a_region = p.a_region;
     const int stage_bytes = a_region + ((256 * p.BN + 1023) & ~1023);
     TcShared *sh = (TcShared *)(tiles + p.stages * stage_bytes);
 
@@ -549,7 +553,7 @@ bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, 
 
 
 // Shape decisions of one layer's weight gradient; cta_budget: the CTAs the job may take
-struct WgPlan { WgParams p; Geom go; int n_tiles, stage_bytes; };
+struct WgPlan { WgParams p; Geom go; int n_tiles, stage_bytes, tail_bytes; };
 static bool wgrad_plan(Geom gi, const Layer &L, int cta_budget, WgPlan &w) {
     if ((L.stride != 1 && L.stride != 2) || (L.k != 1 && L.k != 3) || L.cin % 8 || L.cout % 8) return false;
     if (L.stride == 2 && (gi.H % 2 || gi.W % 2)) return false;
@@ -571,8 +575,11 @@ static bool wgrad_plan(Geom gi, const Layer &L, int cta_budget, WgPlan &w) {
     w.n_tiles = (cout_pad + p.BN - 1) / p.BN;
     p.H = w.go.H; p.W = w.go.W; p.stride = L.stride;
     p.n_tiles_px = tg.n_px_tiles;
-    w.stage_bytes = p.GM * 32768 + ((256 * p.BN + 1023) & ~1023);
-    p.stages = (200 * 1024 - 2048) / w.stage_bytes; if (p.stages > kStages) p.stages = kStages;
+    const int blocks_max = p.total_blocks < p.GM * bpg ? p.total_blocks : p.GM * bpg;
+    p.a_region = (blocks_max * 256 * p.blockC + 1023) & ~1023;
+    w.stage_bytes = p.a_region + ((256 * p.BN + 1023) & ~1023);
+    w.tail_bytes = p.GM * 32768 - p.a_region;        // what the MMAs of a partly filled group read past the last stage
+    p.stages = (200 * 1024 - 2048 - w.tail_bytes) / w.stage_bytes; if (p.stages > kStages) p.stages = kStages;
     if (p.stages < 2) return false;
     // split the pixel reduction so that the job's CTAs cover its share of the machine once
     int splits = (cta_budget + p.m_chunks * w.n_tiles - 1) / (p.m_chunks * w.n_tiles);
@@ -629,7 +636,7 @@ bool conv_wgrad_tc_batch(Exec &ex, int n, const void *const *gq, const void *con
                 p.partial = L[j]->dW;
             }
             batch.job[j].p = p;
-            const int sm = 1024 + p.stages * w[j].stage_bytes + (int)sizeof(TcShared) + 64;
+            const int sm = 1024 + p.stages * w[j].stage_bytes + w[j].tail_bytes + (int)sizeof(TcShared) + 64;
             if (sm > smem) smem = sm;
             bytes += (double)gi[j].P() * L[j]->cin * 2 + (double)w[j].go.P() * L[j]->cout * 2 + (double)p.slice * 4 * p.splits;
             flops += 2.0 * w[j].go.P() * L[j]->cout * L[j]->cin * p.taps;

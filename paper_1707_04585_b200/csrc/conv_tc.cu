@@ -329,6 +329,11 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
 // the N side is a block of output channels.  A CTA owns up to two M groups and one N tile, walks
 // its share of the pixel tiles (split-K) accumulating in tensor memory, and writes an fp32
 // partial; the partials are summed in fixed order by splitk_sum_batch_kernel.
+// For 3x3 layers of few channels the taps are split between the operands instead (sep):
+//   dW[co, (kh, kw), ci] = sum_p a[p + (kh, 0), ci] * g[p - (0, kw), co]
+// so the M side stacks the three vertical shifts of the activations, the N side the three horizontal
+// shifts of the gradient: six boxes and one MMA group per pixel tile where the stacked form takes ten
+// boxes and two groups.  (Activations outside the image are zero, so pixels p outside it add nothing.)
 struct WgParams {
     int taps, k;
     int blockC, cblks, cin;      // input-channel block (16/32/64), blocks per tap, valid channels
@@ -344,6 +349,7 @@ struct WgParams {
     size_t slice;                // cout*taps*cin
     int *status;
     int a_region;                // bytes of a stage that hold activation blocks (the gradient blocks follow)
+    int sep, cout_pad;           // sep: taps split between the operands (see the kernel); cout rounded up to 16
     int splits, m_chunks;        // this job's CTAs: split x M chunk x N tile, split fastest
     int cta0;                    // first CTA of the job in the launch
 };
@@ -379,6 +385,8 @@ wgrad_tc_kernel(const __grid_constant__ WgBatch batch) {
     const int groups = (n_blocks + bpg - 1) / bpg;
     const int col0 = ntile * p.BN;
     int nb_n = (p.cout - col0 + p.blockN - 1) / p.blockN; if (nb_n > p.BN / p.blockN) nb_n = p.BN / p.blockN;   // N blocks holding valid channels
+    const int npk = p.cout_pad / p.blockN;                   // sep: N blocks per horizontal shift
+    if (p.sep) nb_n = p.k * npk;
     const int my_tiles = (p.n_tiles_px - split + p.splits - 1) / p.splits;
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < p.GM * p.BN) tmem_cols <<= 1;
@@ -412,8 +420,10 @@ wgrad_tc_kernel(const __grid_constant__ WgBatch batch) {
         const uint32_t tx = (uint32_t)(p.box_px * 2 * (n_blocks * p.blockC + nb_n * p.blockN));
         const bool a_lane = lane < n_blocks, g_lane = !a_lane && lane < n_blocks + nb_n;
         const int gb = first_block + lane, tap = gb / p.cblks, cb = gb - tap * p.cblks;
-        const int kh = tap / p.k, kw = tap - kh * p.k;
+        const int kh = p.sep ? tap : tap / p.k, kw = p.sep ? p.k / 2 : tap - (tap / p.k) * p.k;
         const int bg = lane - n_blocks;
+        const int g_c = p.sep ? (bg % npk) * p.blockN : col0 + bg * p.blockN;      // gradient box: first channel, first column
+        const int g_x = p.sep ? p.k / 2 - bg / npk : 0;
         for (int it = 0; it < my_tiles; it++) {
             const int s = it % p.stages, round = it / p.stages;
             bool ok = true;
@@ -428,7 +438,7 @@ wgrad_tc_kernel(const __grid_constant__ WgBatch batch) {
             const int h0 = p.BIMG > 1 ? 0 : (t % tiles_per_img) * p.BH;
             uint8_t *sa = tiles + s * stage_bytes;
             if (a_lane) tma_load_4d(sa + lane * blk_bytes_a, &map_a, &sh->full[s], cb * p.blockC, kw - pad, h0 * p.stride + kh - pad, n0);
-            else if (g_lane) tma_load_4d(sa + a_region + bg * blk_bytes_b, &map_g, &sh->full[s], col0 + bg * p.blockN, 0, h0, n0);
+            else if (g_lane) tma_load_4d(sa + a_region + bg * blk_bytes_b, &map_g, &sh->full[s], g_c, g_x, h0, n0);
         }
     } else if (warp == 1) {
         if (lane == 0) {
@@ -460,7 +470,7 @@ wgrad_tc_kernel(const __grid_constant__ WgBatch batch) {
             float *dst = p.partial + (size_t)split * p.slice;
             for (int g = 0; g < groups; g++) {
                 const int gb = first_block + g * bpg + m / p.blockC;
-                const int tap = gb / p.cblks, ci = (gb - tap * p.cblks) * p.blockC + m % p.blockC;
+                const int tap_m = gb / p.cblks, ci = (gb - tap_m * p.cblks) * p.blockC + m % p.blockC;     // sep: tap_m is kh
                 const bool row_ok = gb < p.total_blocks && ci < p.cin;
                 for (int c = 0; c < p.BN; c += 16) {
                     float v[16];
@@ -470,16 +480,20 @@ wgrad_tc_kernel(const __grid_constant__ WgBatch batch) {
 #pragma unroll
                         for (int j = 0; j < 16; j++) v[j] = 0.f;
                     }
+                    // column c of the accumulator: output channel cb0 + ..., and with sep the horizontal shift too
+                    const int kw = p.sep ? c / p.cout_pad : 0;
+                    const int cb0 = p.sep ? c - kw * p.cout_pad : col0 + c;
+                    const int tap = p.sep ? tap_m * p.k + kw : tap_m;
                     if (p.splits > 1) {
                         // split partials are [tap][ci][co]: this row's output channels are contiguous (cout is a multiple of 8)
-                        float *row = dst + ((size_t)tap * p.cin + ci) * p.cout + col0 + c;
+                        float *row = dst + ((size_t)tap * p.cin + ci) * p.cout + cb0;
 #pragma unroll
                         for (int j = 0; j < 16; j += 4)
-                            if (col0 + c + j < p.cout) *reinterpret_cast<float4 *>(row + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                            if (cb0 + j < p.cout) *reinterpret_cast<float4 *>(row + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
                     } else {
 #pragma unroll
                         for (int j = 0; j < 16; j++) {
-                            const int co = col0 + c + j;
+                            const int co = cb0 + j;
                             if (co < p.cout) dst[((size_t)co * p.taps + tap) * p.cin + ci] = v[j];
                         }
                     }
@@ -552,9 +566,11 @@ bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, 
 }
 
 
+constexpr int kWgSmemMax = 224 * 1024;
+
 // Shape decisions of one layer's weight gradient; cta_budget: the CTAs the job may take
 struct WgPlan { WgParams p; Geom go; int n_tiles, stage_bytes, tail_bytes; };
-static bool wgrad_plan(Geom gi, const Layer &L, int cta_budget, WgPlan &w) {
+static bool wgrad_plan(Geom gi, const Layer &L, int cta_budget, WgPlan &w, bool allow_sep = true) {
     if ((L.stride != 1 && L.stride != 2) || (L.k != 1 && L.k != 3) || L.cin % 8 || L.cout % 8) return false;
     if (L.stride == 2 && (gi.H % 2 || gi.W % 2)) return false;
     WgParams &p = w.p;
@@ -564,23 +580,33 @@ static bool wgrad_plan(Geom gi, const Layer &L, int cta_budget, WgPlan &w) {
     p.BH = tg.BH; p.BIMG = tg.BIMG; p.tiles_per_img = tg.tiles_per_img; p.box_px = tg.BIMG * tg.BH * tg.W;
     const int taps = L.k * L.k, cin_pad = round_up(L.cin, 16), cout_pad = round_up(L.cout, 16);
     p.taps = taps; p.k = L.k; p.cin = L.cin; p.cout = L.cout;
-    p.blockC = pick_block(cin_pad); p.cblks = cin_pad / p.blockC; p.total_blocks = taps * p.cblks;
+    p.blockC = pick_block(cin_pad); p.cblks = cin_pad / p.blockC;
     p.blockN = pick_block(cout_pad);
-    p.BN = cout_pad <= 128 ? cout_pad : 128;
-    if (p.BN % p.blockN) p.BN = p.blockN;
+    p.cout_pad = cout_pad;
     const int bpg = 128 / p.blockC;
+    // taps split between the operands when the three shifted activation blocks fit one M group, the three
+    // shifted gradient blocks one N tile, and the boxes of a pixel tile the lanes of the producer warp
+    p.sep = (allow_sep && L.k == 3 && L.stride == 1 && 3 * cin_pad <= 128 && 3 * cout_pad <= 256 && 2 * bpg + 3 * (cout_pad / p.blockN) <= 32) ? 1 : 0;
+    if (p.sep) {
+        p.total_blocks = L.k * p.cblks;
+        p.BN = L.k * cout_pad;
+    } else {
+        p.total_blocks = taps * p.cblks;
+        p.BN = cout_pad <= 128 ? cout_pad : 128;
+        if (p.BN % p.blockN) p.BN = p.blockN;
+    }
     const int groups_all = (p.total_blocks + bpg - 1) / bpg;
     p.GM = groups_all >= 2 ? 2 : 1;
     p.m_chunks = (groups_all + p.GM - 1) / p.GM;
-    w.n_tiles = (cout_pad + p.BN - 1) / p.BN;
+    w.n_tiles = p.sep ? 1 : (cout_pad + p.BN - 1) / p.BN;
     p.H = w.go.H; p.W = w.go.W; p.stride = L.stride;
     p.n_tiles_px = tg.n_px_tiles;
     const int blocks_max = p.total_blocks < p.GM * bpg ? p.total_blocks : p.GM * bpg;
     p.a_region = (blocks_max * 256 * p.blockC + 1023) & ~1023;
     w.stage_bytes = p.a_region + ((256 * p.BN + 1023) & ~1023);
     w.tail_bytes = p.GM * 32768 - p.a_region;        // what the MMAs of a partly filled group read past the last stage
-    p.stages = (200 * 1024 - 2048 - w.tail_bytes) / w.stage_bytes; if (p.stages > kStages) p.stages = kStages;
-    if (p.stages < 2) return false;
+    p.stages = (kWgSmemMax - 2048 - w.tail_bytes) / w.stage_bytes; if (p.stages > kStages) p.stages = kStages;
+    if (p.stages < 2) return p.sep ? wgrad_plan(gi, L, cta_budget, w, false) : false;
     // split the pixel reduction so that the job's CTAs cover its share of the machine once
     int splits = (cta_budget + p.m_chunks * w.n_tiles - 1) / (p.m_chunks * w.n_tiles);
     if (splits > p.n_tiles_px) splits = p.n_tiles_px;
@@ -642,7 +668,7 @@ bool conv_wgrad_tc_batch(Exec &ex, int n, const void *const *gq, const void *con
             flops += 2.0 * w[j].go.P() * L[j]->cout * L[j]->cin * p.taps;
         }
         static bool attr_set = false;
-        if (!attr_set) { cudaFuncSetAttribute(wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); attr_set = true; }
+        if (!attr_set) { cudaFuncSetAttribute(wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWgSmemMax); attr_set = true; }
         launch(ex, wgrad_tc_kernel, (unsigned)cta, kThreads, smem, batch);
         ex.check("conv_wgrad_tc", bytes, flops);
         if (n_sums) {

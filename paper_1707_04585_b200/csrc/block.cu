@@ -78,20 +78,21 @@ void fn_forward(Exec &ex, Geom g, Pair u, const Moments *mom_in, const std::vect
             bn_stats(ex, t, P, cur);
             cur.valid = true;
         }
-        const BnRef bn{ly.gamma, ly.beta, cur.mean, cur.rstd};
+        const BnRef bn = bn_ref(ly.gamma, ly.beta, cur, ex.eps);
         const bool last = l == L - 1;
         Geom go{gi.N, conv_out(gi.H, ly.k, ly.stride), conv_out(gi.W, ly.k, ly.stride)};
         // the activated tensor is materialised only where something reads it: the unfused convolution, or the weight gradient
         void *a = ex.ws.alloc(P * ly.cin * esz(ex));
         float *tn = last ? nullptr : ex.ws.get<float>(go.P() * ly.cout);
         Moments next;
-        if (!last) next = mom_alloc(ex, ly.cout);
+        if (!last) next = mom_alloc(ex, ly.cout, b16);      // with room for pending partials: the next layer consumes them
         const Pair o = last ? out : single(tn, ly.cout);
         bool fused = false;
         if (b16 && !(last && skip_last_conv))
             fused = conv_fprop_fused(ex, t, bn, gi, ly, o, last ? partner : Pair{}, last ? sign : 0, last ? mom_out : &next,
                                      saved ? (bf16 *)a : nullptr);
-        if (!fused) bn_relu_apply(ex, t, P, bn, a, b16);
+        if (fused) cur.pending = false;     // the fused kernel has stored mean and rstd
+        else { mom_finalize(ex, cur, ly.cin); bn_relu_apply(ex, t, P, BnRef{ly.gamma, ly.beta, cur.mean, cur.rstd}, a, b16); }
         if (saved) { saved->a.push_back(a); saved->bn.push_back(cur); }
         if (last) {
             if (!skip_last_conv && !fused) conv_fprop(ex, a, gi, ly, out, partner, sign, mom_out);

@@ -191,15 +191,35 @@ struct Layer {
 
 // Batch statistics of one tensor: per-channel mean and 1/sqrt(var + eps), [C] each (device).
 // `valid` is host-side bookkeeping: whether a kernel enqueued earlier fills them.
+// A fused convolution may leave them `pending`: its CTAs have written their partial sums (records of
+// 2C floats, `parts` of them, in `part`) and the next kernel that normalises with them adds the
+// records itself, in a fixed order, while its first tile is on the way -- cheaper than a grid-wide
+// count and a reduction by the last CTA at the end of the producer.  That consumer also stores mean
+// and rstd; anything else that wants them calls mom_finalize() first.
 struct Moments {
     float *mean = nullptr, *rstd = nullptr;
     bool valid = false;
+    float *part = nullptr;         // room for partial records (null: the producer must reduce itself)
+    size_t part_cap = 0;           // floats
+    int parts = 0;
+    double inv_count = 0;          // 1 / pixels summed
+    bool pending = false;
 };
 // One BN as its consumers see it: scale = gamma*rstd, shift = beta - mean*scale are derived on the
 // fly, always with the same two roundings, so that the ReLU mask of the backward equals the forward's.
 struct BnRef {
     const float *gamma, *beta, *mean, *rstd;
+    // pending statistics (see Moments): the consumer reduces `parts` records of 2C floats and stores mean / rstd
+    const float *part = nullptr;
+    int parts = 0;
+    double inv_count = 0;
+    float eps = 0.f;
 };
+inline BnRef bn_ref(const float *gamma, const float *beta, const Moments &m, float eps) {
+    BnRef b{gamma, beta, m.mean, m.rstd};
+    if (m.pending) { b.part = m.part; b.parts = m.parts; b.inv_count = m.inv_count; b.eps = eps; }
+    return b;
+}
 #ifdef __CUDACC__
 __device__ __forceinline__ void bn_sc_sh(float g, float b, float mu, float r, float &sc, float &sh) {
     sc = __fmul_rn(g, r);
@@ -216,7 +236,9 @@ __device__ __forceinline__ void bn_coef4(const BnRef &bn, int c, float4 &sc, flo
 struct Geom { int N, H, W; size_t P() const { return (size_t)N * H * W; } };
 
 // ---------------------------------------------------------------- elementwise.cu
-Moments mom_alloc(Exec &ex, int C);
+Moments mom_alloc(Exec &ex, int C, bool with_part = false);
+// pending statistics -> mean / rstd (one small kernel); no-op otherwise
+void mom_finalize(Exec &ex, Moments &m, int C);
 // batch statistics of t ([P,C]) -> mean, rstd (two kernels; the convolution epilogues produce the
 // same quantities for the tensors they write)
 void bn_stats(Exec &ex, Pair t, size_t P, Moments m);

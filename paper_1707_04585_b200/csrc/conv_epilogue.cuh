@@ -187,6 +187,55 @@ __device__ __forceinline__ void epilogue_tile(const EpiArgs &e, uint32_t tmem_ac
     }
 }
 
+// mean and 1 / sqrt(var + eps) from a channel's sum and second sum (double), rounded to float once
+__device__ __forceinline__ void moments_of(double sum, double sum2, double inv_count, float eps, float &mean, float &rstd) {
+    const double m = sum * inv_count;
+    double var = sum2 * inv_count - m * m;
+    if (var < 0) var = 0;
+    mean = (float)m; rstd = (float)(1.0 / sqrt(var + (double)eps));
+}
+
+// Adds the per-CTA records of a reduction.  A record is 2C floats = C/2 float4 slots (per channel
+// quad: sums, second sums); this call covers the slots slot0 .. slot0 + cw - 1 (cw <= 128, even).
+// Thread = (slot, sub), slot fastest so that a warp reads whole records: it adds the records sub,
+// sub + nsub, ... of its slot, ten loads in flight at a time; the subs are then added in order.
+// (Giving a slot to consecutive lanes and adding them by shuffles was measured slower: the loads
+// of a warp then touch 32 records.)  All in double precision, in an order that the number of
+// records, cw and NT fix.  Result: tot[slot - slot0][4].  Called by NT threads (tid = 0..NT-1)
+// that share named barrier 1; red: [NT][4] doubles, tot: [128][4] doubles of shared memory.
+template <int NT>
+__device__ __forceinline__ void reduce_records(const float *part, int parts, int C, int slot0, int cw, double *red, double *tot, int tid) {
+    const int nsub = NT / cw;
+    const int r = tid % cw, sub = tid / cw;
+    if (sub < nsub) {
+        double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
+        const float *src = part + (size_t)(slot0 + r) * 4;
+        constexpr int kInFlight = 10;
+        for (int i = sub; i < parts; i += kInFlight * nsub) {
+            float4 v[kInFlight];
+#pragma unroll
+            for (int k = 0; k < kInFlight; k++) {
+                const int idx = i + k * nsub;
+                v[k] = idx < parts ? ldcg4(src + (size_t)idx * 2 * C) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+            for (int k = 0; k < kInFlight; k++) { s0 += (double)v[k].x; s1 += (double)v[k].y; s2 += (double)v[k].z; s3 += (double)v[k].w; }
+        }
+        red[tid * 4] = s0; red[tid * 4 + 1] = s1; red[tid * 4 + 2] = s2; red[tid * 4 + 3] = s3;
+    }
+    named_barrier(1, NT);
+    if (tid < cw) {
+        double s0 = red[tid * 4], s1 = red[tid * 4 + 1], s2 = red[tid * 4 + 2], s3 = red[tid * 4 + 3];
+        for (int y = 1; y < nsub; y++) {
+            const double *o = red + (y * cw + tid) * 4;
+            s0 += o[0]; s1 += o[1]; s2 += o[2]; s3 += o[3];
+        }
+        double *d = tot + tid * 4;
+        d[0] = s0; d[1] = s1; d[2] = s2; d[3] = s3;
+    }
+    named_barrier(1, NT);
+}
+
 template <int NT>
 __device__ __forceinline__ void epilogue_publish(const EpiArgs &e, float *scratch, int etid);
 
@@ -235,45 +284,13 @@ __device__ __forceinline__ void epilogue_publish(const EpiArgs &e, float *scratc
     named_barrier(1, NT);
     if (!last) return;
     __threadfence();
-    // A partial is a record of 2C floats = R float4 slots (per channel quad: sums, second sums).
-    // Thread = (slot, sub): it adds the records sub, sub + nsub, ... of its slot, ten loads in
-    // flight at a time; the subs are then added in order.  All in double precision, all in an
-    // order the launch shape fixes.
-    const int C = e.n_cols, parts = (int)gridDim.x, R = C >> 1;
+    const int C = e.n_cols, R = C >> 1;
     double *red = reinterpret_cast<double *>(scratch);            // [NT][4]
     double *tot = red + NT * 4;                                   // [128][4]
     for (int slot0 = 0; slot0 < R; slot0 += 128) {
         const int cw = R - slot0 < 128 ? R - slot0 : 128;         // even
-        const int nsub = NT / cw;
-        const int r = etid % cw, sub = etid / cw;
-        if (sub < nsub) {
-            double s0 = 0, s1 = 0, s2 = 0, s3 = 0;
-            const float *src = e.part + (size_t)(slot0 + r) * 4;
-            constexpr int kInFlight = 10;
-            for (int i = sub; i < parts; i += kInFlight * nsub) {
-                float4 v[kInFlight];
-#pragma unroll
-                for (int k = 0; k < kInFlight; k++) {
-                    const int idx = i + k * nsub;
-                    v[k] = idx < parts ? ldcg4(src + (size_t)idx * 2 * C) : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-#pragma unroll
-                for (int k = 0; k < kInFlight; k++) { s0 += (double)v[k].x; s1 += (double)v[k].y; s2 += (double)v[k].z; s3 += (double)v[k].w; }
-            }
-            red[etid * 4] = s0; red[etid * 4 + 1] = s1; red[etid * 4 + 2] = s2; red[etid * 4 + 3] = s3;
-        }
-        named_barrier(1, NT);
-        if (etid < cw) {
-            double s0 = red[etid * 4], s1 = red[etid * 4 + 1], s2 = red[etid * 4 + 2], s3 = red[etid * 4 + 3];
-            for (int y = 1; y < nsub; y++) {
-                const double *o = red + (y * cw + etid) * 4;
-                s0 += o[0]; s1 += o[1]; s2 += o[2]; s3 += o[3];
-            }
-            double *d = tot + etid * 4;
-            d[0] = s0; d[1] = s1; d[2] = s2; d[3] = s3;
-        }
-        named_barrier(1, NT);
-        for (int lc = etid; lc < cw * 2; lc += NT) {             // one thread per channel of this slot range
+        reduce_records<NT>(e.part, (int)gridDim.x, C, slot0, cw, red, tot, etid);
+        for (int lc = etid; lc < cw * 2; lc += NT) {              // one thread per channel of this slot range
             const int k = lc >> 2, j = lc & 3;                    // local quad, lane within it
             const int ch = (slot0 >> 1) * 4 + lc;
             const double sum = tot[(2 * k) * 4 + j], sum2 = tot[(2 * k + 1) * 4 + j];
@@ -282,10 +299,9 @@ __device__ __forceinline__ void epilogue_publish(const EpiArgs &e, float *scratc
                 const double gr = (double)e.bn.gamma[ch] * (double)e.bn.rstd[ch];
                 e.coef[ch] = (float)gr; e.coef[C + ch] = (float)(gr * sum * e.inv_count); e.coef[2 * C + ch] = (float)(gr * sum2 * e.inv_count);
             } else {
-                const double m = sum * e.inv_count;
-                double var = sum2 * e.inv_count - m * m;
-                if (var < 0) var = 0;
-                e.mean[ch] = (float)m; e.rstd[ch] = (float)(1.0 / sqrt(var + (double)e.eps));
+                float m, r;
+                moments_of(sum, sum2, e.inv_count, e.eps, m, r);
+                e.mean[ch] = m; e.rstd[ch] = r;
             }
         }
         named_barrier(1, NT);

@@ -342,7 +342,23 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
     }
     // the tables above are independent of what earlier kernels wrote; everything below is not
     pdl_enter();
-    if (threadIdx.x >= 128 && threadIdx.x < 192) {
+    if (p.in_mode == 0 && p.bn.part) {
+        // the statistics of the input are still per-CTA records of the kernel before: add them here (every CTA
+        // the same way, while its first tile is on the way); the first CTA stores mean and rstd for later readers
+        double *red = reinterpret_cast<double *>(abuf), *tot = red + kFThreads * 4;
+        reduce_records<kFThreads>(p.bn.part, p.bn.parts, p.cin, 0, p.cin >> 1, red, tot, (int)threadIdx.x);
+        if (threadIdx.x < 64) {
+            const int c = threadIdx.x;
+            float sc = 0.f, sf = 0.f;
+            if (c < p.cin) {
+                float mean, rstd;
+                moments_of(tot[(2 * (c >> 2)) * 4 + (c & 3)], tot[(2 * (c >> 2) + 1) * 4 + (c & 3)], p.bn.inv_count, p.bn.eps, mean, rstd);
+                if (blockIdx.x == 0 && blockIdx.y == 0) { const_cast<float *>(p.bn.mean)[c] = mean; const_cast<float *>(p.bn.rstd)[c] = rstd; }
+                bn_sc_sh(p.bn.gamma[c], p.bn.beta[c], mean, rstd, sc, sf);
+            }
+            sh->sc[c] = sc; sh->sf[c] = sf;
+        }
+    } else if (threadIdx.x >= 128 && threadIdx.x < 192) {
         const int c = threadIdx.x - 128;
         float sc = 0.f, sf = 0.f;
         if (p.in_mode == 0 && c < p.cin) bn_sc_sh(p.bn.gamma[c], p.bn.beta[c], p.bn.mean[c], p.bn.rstd[c], sc, sf);
@@ -482,7 +498,7 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
             *reinterpret_cast<float4 *>(mine + 4) = make_float4(r[4], r[5], r[6], r[7]);
         }
         __syncthreads();
-        epilogue_publish<kFThreads>(e, scratch, (int)threadIdx.x);
+        if (e.counter) epilogue_publish<kFThreads>(e, scratch, (int)threadIdx.x);     // else the consumer adds the records
     }
     if (!ok && threadIdx.x == 0) atomicExch(&sh->failed, 1u);
     tc_fence_before();
@@ -579,8 +595,13 @@ bool run_fused(Exec &ex, const char *what, int in_mode, const void *in, float in
     const size_t pack_elems = tc_pack_elems(transposed ? cout : cin, transposed ? cin : cout, k, transposed);
     bf16 *wp = prepacked ? const_cast<bf16 *>(prepacked) : ex.ws.get<bf16>(pack_elems);
     const bool reduce = req.stats || req.bnbwd;
-    float *part = reduce ? ex.ws.get<float>((size_t)ctas * 2 * cout) : nullptr;
-    if (req.stats) req.stats->valid = true;
+    // statistics whose owner has room for the records stay pending: the kernel that consumes them adds the records
+    const bool defer = req.stats && !req.bnbwd && req.stats->part && (size_t)ctas * 2 * cout <= req.stats->part_cap;
+    float *part = defer ? req.stats->part : (reduce ? ex.ws.get<float>((size_t)ctas * 2 * cout) : nullptr);
+    if (req.stats) {
+        req.stats->valid = true;
+        req.stats->pending = defer; req.stats->parts = ctas; req.stats->inv_count = 1.0 / (double)g.P();
+    }
     if (!ex.dry) {
         if (!prepacked) tc_pack_now(ex, Wsrc, wp, transposed ? cout : cin, transposed ? cin : cout, k, transposed);
         const int rows_pad = s.n_tiles * s.BN;
@@ -607,7 +628,7 @@ bool run_fused(Exec &ex, const char *what, int in_mode, const void *in, float in
         EpiArgs &e = p.epi;
         e.mode = req.bnbwd ? EPI_BNBWD : (sign ? EPI_COUPLE : EPI_PLAIN);
         e.out = out; e.partner = partner; e.sign = sign; e.n_cols = cout;
-        e.part = part; e.counter = reduce ? ex.ctx->counter() : nullptr;
+        e.part = part; e.counter = (reduce && !defer) ? ex.ctx->counter() : nullptr;
         e.inv_count = 1.0 / (double)g.P(); e.eps = ex.eps;
         if (req.stats) { e.mean = req.stats->mean; e.rstd = req.stats->rstd; }
         if (req.bnbwd) { e.t = req.bnbwd->t; e.bn = req.bnbwd->bn; e.dgamma = req.bnbwd->dgamma; e.dbeta = req.bnbwd->dbeta; e.coef = req.bnbwd->coef; }

@@ -2,6 +2,7 @@
 // classification head, SGD.  All reductions are two-stage with a fixed summation order, so a
 // residual function recomputed in the backward pass reproduces the forward bit for bit.
 #include "common.cuh"
+#include "conv_epilogue.cuh"
 #include <math.h>
 
 cudaEvent_t revnet_ctx::next_event() {
@@ -147,11 +148,41 @@ __global__ void bn_bwd_finalize(const float *__restrict__ part, int chunks, int 
     }
 }
 
-Moments mom_alloc(Exec &ex, int C) {
+Moments mom_alloc(Exec &ex, int C, bool with_part) {
     Moments m;
     float *p = ex.ws.get<float>((size_t)2 * C);
     m.mean = p; m.rstd = p + C;
+    if (with_part) {
+        // a fused convolution runs at most two CTAs per SM, one record of 2C floats each
+        m.part_cap = (size_t)2 * ex.ctx->sm_count * 2 * C;
+        m.part = ex.ws.get<float>(m.part_cap);
+    }
     return m;
+}
+
+__global__ void __launch_bounds__(256) moments_finalize_kernel(const float *part, int parts, int C, double inv_count, float eps,
+                                                             float *mean, float *rstd) {
+    pdl_enter();
+    __shared__ double red[256 * 4], tot[128 * 4];
+    const int R = C >> 1, tid = threadIdx.x;
+    for (int slot0 = 0; slot0 < R; slot0 += 128) {
+        const int cw = R - slot0 < 128 ? R - slot0 : 128;
+        tc::reduce_records<256>(part, parts, C, slot0, cw, red, tot, tid);
+        for (int lc = tid; lc < cw * 2; lc += 256) {
+            const int k = lc >> 2, j = lc & 3, ch = (slot0 >> 1) * 4 + lc;
+            tc::moments_of(tot[(2 * k) * 4 + j], tot[(2 * k + 1) * 4 + j], inv_count, eps, mean[ch], rstd[ch]);
+        }
+        tc::named_barrier(1, 256);
+    }
+}
+
+void mom_finalize(Exec &ex, Moments &m, int C) {
+    if (!m.pending) return;
+    if (!ex.dry) {
+        launch(ex, moments_finalize_kernel, 1, 256, 0, (const float *)m.part, m.parts, C, m.inv_count, ex.eps, m.mean, m.rstd);
+        ex.check("bn_stats_finalize");
+    }
+    m.pending = false;
 }
 
 void bn_stats(Exec &ex, Pair t, size_t P, Moments mo) {

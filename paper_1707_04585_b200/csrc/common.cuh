@@ -149,6 +149,7 @@ struct Exec {
     bool failed = false;
     bool pdl = true;       // launch kernels with programmatic stream serialization (see launch())
     bool use_side = true;  // run weight gradients on the context's side stream (never while profiling)
+    unsigned long long hold_ns = 0;   // profiling: the first mark() holds the stream this long so that launches queue up
     // called after every launch: error check, launch count and (when profiling) an event;
     // bytes / flops are the algorithmic traffic and work of that launch
     void check(const char *what, double bytes = 0, double flops = 0);

@@ -108,12 +108,13 @@ __device__ __forceinline__ void build_table(const FusedParams &p, ItemRef *tab, 
     }
 }
 
-// raw tile (shared memory) -> operand copies (shared memory), four items per thread in flight.
+// raw tile (shared memory) -> operand copies (shared memory), NJ items per thread in flight (two
+// where a tile has at most two items per thread: slots without an item would still cost their instructions).
 // This thread's channel chunk ck is fixed: the thread count is a multiple of the chunks per pixel.
 // IN_MODE 0: float input through BN + ReLU; 2: fixed-point input through BN + ReLU; 1: bf16 input as it is.
 // Written without branches in the per-item work (invalid items compute on the zeros TMA delivered and are
 // masked, stores that do not exist go to a dummy slot), so that the four items of a batch interleave.
-template <int IN_MODE>
+template <int IN_MODE, int NJ>
 __device__ __forceinline__ void build_tile(const FusedParams &p, FusedShared *sh, const ItemRef *tab, int items, int cshift, int ck,
                                            const uint8_t *raw, uint8_t *A, int n0, int h0) {
     const int pad = p.k >> 1;
@@ -130,12 +131,12 @@ __device__ __forceinline__ void build_tile(const FusedParams &p, FusedShared *sh
     }
     const uint32_t dummy = (uint32_t)(reinterpret_cast<uint8_t *>(&sh->dummy) - A);     // byte offset of the dummy slot relative to A
 #pragma unroll 1
-    for (int base = threadIdx.x; base < items; base += 4 * kFThreads) {
-        ItemRef ref[4];
-        uint4 v[4];
-        bool ok[4];
+    for (int base = threadIdx.x; base < items; base += NJ * kFThreads) {
+        ItemRef ref[NJ];
+        uint4 v[NJ];
+        bool ok[NJ];
 #pragma unroll
-        for (int j = 0; j < 4; j++) {
+        for (int j = 0; j < NJ; j++) {
             const int it = base + j * kFThreads;
             const bool exists = it < items;
             const uint32_t px = (uint32_t)(exists ? it : items - 1) >> cshift;
@@ -173,7 +174,7 @@ __device__ __forceinline__ void build_tile(const FusedParams &p, FusedShared *sh
         }
         if (IN_MODE != 1 && p.a_out) {
 #pragma unroll
-            for (int j = 0; j < 4; j++)
+            for (int j = 0; j < NJ; j++)
                 if (ok[j] && (ref[j].flags & 1u)) {
                     const int r = (ref[j].r2f >> 16) & 0xff, img = ref[j].r2f >> 24, xh = (ref[j].flags >> 8) & 0xff;
                     const size_t gp = ((size_t)(n0 + img) * p.g.H + (h0 - pad + r)) * p.g.W + (xh - pad);
@@ -402,9 +403,15 @@ conv_fused_kernel(const __grid_constant__ CUtensorMap map_w, const __grid_consta
         ok = __syncthreads_and(ok);
         if (!ok) break;
         // ---- build the operand
-        if (p.in_mode == 1) build_tile<1>(p, sh, tab, items, cshift, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
-        else if (p.in_q == 0.f) build_tile<0>(p, sh, tab, items, cshift, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
-        else build_tile<2>(p, sh, tab, items, cshift, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
+        if (items <= 2 * kFThreads) {
+            if (p.in_mode == 1) build_tile<1, 2>(p, sh, tab, items, cshift, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
+            else if (p.in_q == 0.f) build_tile<0, 2>(p, sh, tab, items, cshift, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
+            else build_tile<2, 2>(p, sh, tab, items, cshift, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
+        } else {
+            if (p.in_mode == 1) build_tile<1, 4>(p, sh, tab, items, cshift, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
+            else if (p.in_q == 0.f) build_tile<0, 4>(p, sh, tab, items, cshift, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
+            else build_tile<2, 4>(p, sh, tab, items, cshift, ck, rawb + b * p.raw_bytes, abuf, n0, h0);
+        }
         fence_proxy_async();
         __syncthreads();
         if (threadIdx.x == 0) {

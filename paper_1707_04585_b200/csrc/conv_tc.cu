@@ -38,6 +38,20 @@ struct TcParams {
     TileGeom g;      // output tiles
     EpiArgs epi;
     int *status;
+    int stages;      // operand ring depth (<= kStages)
+    // epilogue through TMA (epi_tma): the output tile leaves, and the tile read besides the accumulator (coupling
+    // partner, or BN input of a data gradient) arrives, as column groups of GW floats per pixel row
+    int epi_tma;
+    int GW;          // 32 or 16 floats: rows of 128 / 64 bytes, stored with the matching TMA swizzle
+    int group_bytes; // one column group of a tile (128 pixel rows), a multiple of 1024
+    int need_aux;
+    int split_o, split_x;   // channels in the first tensor of a channel-split output / partner (0: one tensor)
+    // the taps this launch sums: offset of the operand box in rows / columns of the operand tensor, and the tap's
+    // place in the weight pack.  A plain convolution lists all k*k taps; one parity class of a stride-2 data
+    // gradient lists the one, two or four taps that reach its output pixels.
+    int ntap;
+    signed char tdy[9], tdx[9], tid[9];
+    int ostride, oy, ox;    // epi_tma: output pixel = tile pixel * ostride + (oy, ox)
 };
 
 struct __align__(8) TcShared {
@@ -45,16 +59,82 @@ struct __align__(8) TcShared {
     uint64_t empty[kStages];
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
+    uint64_t aux_full[8];
     uint32_t tmem_base;
     uint32_t failed;
     RowMap rows;
 };
 
+// ---- epilogue through TMA.  One column group (GW accumulator columns) at a time:
+//   pass A  thread = accumulator row: tensor memory (+ partner row in shared memory) -> output group in shared memory
+//   store   one TMA store of the group
+//   pass B  thread = (channel quad, every rpp-th pixel): per-channel sums over the valid pixels of the group
+// KA: 0 plain float, 1 plain onto the fixed-point grid, 2 / 3 float coupling + / -, 4 / 5 fixed-point coupling + / -.
+template <int KA>
+__device__ __forceinline__ void tma_pass_a(uint32_t tm, int GW, int row, bool valid, const uint8_t *aux, uint8_t *outb, float out_s) {
+    const int row_b = GW * 4;
+    const int swz = GW == 32 ? (row & 7) : ((row >> 1) & 3);
+#pragma unroll 1
+    for (int c = 0; c < GW; c += 16) {
+        float v[16];
+        tmem_ld16(tm + (uint32_t)c, v);
+        if (!valid) continue;
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            const int off = row * row_b + ((((c >> 2) + j) ^ swz) << 4);
+            float4 r = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            if (KA == 2 || KA == 3) {
+                const float4 pr = *reinterpret_cast<const float4 *>(aux + off);
+                if (KA == 2) { r.x = pr.x + r.x; r.y = pr.y + r.y; r.z = pr.z + r.z; r.w = pr.w + r.w; }
+                else { r.x = pr.x - r.x; r.y = pr.y - r.y; r.z = pr.z - r.z; r.w = pr.w - r.w; }
+            } else if (KA != 0) {
+                int4 iv = make_int4(__float2int_rn(r.x * out_s), __float2int_rn(r.y * out_s), __float2int_rn(r.z * out_s), __float2int_rn(r.w * out_s));
+                if (KA >= 4) {
+                    const int4 pi = *reinterpret_cast<const int4 *>(aux + off);
+                    if (KA == 4) { iv.x = pi.x + iv.x; iv.y = pi.y + iv.y; iv.z = pi.z + iv.z; iv.w = pi.w + iv.w; }
+                    else { iv.x = pi.x - iv.x; iv.y = pi.y - iv.y; iv.z = pi.z - iv.z; iv.w = pi.w - iv.w; }
+                }
+                r = make_float4(__int_as_float(iv.x), __int_as_float(iv.y), __int_as_float(iv.z), __int_as_float(iv.w));
+            }
+            *reinterpret_cast<float4 *>(outb + off) = r;
+        }
+    }
+}
+// KB 0 / 1: sums and second sums of the stored values (float / fixed point); 2 / 3: the two sums of the
+// BN+ReLU backward with a float / fixed-point BN input group.  Rows are added in a fixed order.
+template <int KB>
+__device__ __forceinline__ void tma_pass_b(int GW, const uint8_t *ob, const uint8_t *aux, int jq, int r0, int rpp, int valid_px,
+                                           float q, float4 sc4, float4 sh4, float4 mu4, float4 rs4, float (&acc)[8]) {
+    const int row_b = GW * 4;
+#pragma unroll 4
+    for (int pl = r0; pl < valid_px; pl += rpp) {
+        const int off = pl * row_b + ((jq ^ (GW == 32 ? (pl & 7) : ((pl >> 1) & 3))) << 4);
+        float4 v = *reinterpret_cast<const float4 *>(ob + off);
+        if (KB >= 2) {
+            float4 tt = *reinterpret_cast<const float4 *>(aux + off);
+            if (KB == 3) tt = make_float4(__int2float_rn(__float_as_int(tt.x)) * q, __int2float_rn(__float_as_int(tt.y)) * q,
+                                          __int2float_rn(__float_as_int(tt.z)) * q, __int2float_rn(__float_as_int(tt.w)) * q);
+            const float dx = fmaf(sc4.x, tt.x, sh4.x) > 0.f ? v.x : 0.f, dy = fmaf(sc4.y, tt.y, sh4.y) > 0.f ? v.y : 0.f;
+            const float dz = fmaf(sc4.z, tt.z, sh4.z) > 0.f ? v.z : 0.f, dw = fmaf(sc4.w, tt.w, sh4.w) > 0.f ? v.w : 0.f;
+            acc[0] += dx; acc[1] += dy; acc[2] += dz; acc[3] += dw;
+            acc[4] += dx * ((tt.x - mu4.x) * rs4.x); acc[5] += dy * ((tt.y - mu4.y) * rs4.y);
+            acc[6] += dz * ((tt.z - mu4.z) * rs4.z); acc[7] += dw * ((tt.w - mu4.w) * rs4.w);
+        } else {
+            if (KB == 1) v = make_float4(__int2float_rn(__float_as_int(v.x)) * q, __int2float_rn(__float_as_int(v.y)) * q,
+                                         __int2float_rn(__float_as_int(v.z)) * q, __int2float_rn(__float_as_int(v.w)) * q);
+            acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
+            acc[4] += v.x * v.x; acc[5] += v.y * v.y; acc[6] += v.z * v.z; acc[7] += v.w * v.w;
+        }
+    }
+}
+
 // Persistent CTA: walks the pixel tiles blockIdx.x, blockIdx.x + gridDim.x, ... of N tile blockIdx.y.
 // The operand ring runs on across tiles; the accumulator alternates between two tensor-memory
 // buffers so that the epilogue of one tile overlaps the MMAs of the next.
 __global__ void __launch_bounds__(kThreads, 1)
-conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const TcParams p) {
+conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+               const __grid_constant__ CUtensorMap map_o0, const __grid_constant__ CUtensorMap map_o1,
+               const __grid_constant__ CUtensorMap map_x0, const __grid_constant__ CUtensorMap map_x1, const TcParams p) {
     extern __shared__ uint8_t smem_raw[];
     // operand stages first (1024-byte aligned for the 128-byte swizzle), epilogue stage and bookkeeping behind them
     uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -62,20 +142,28 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int a_bytes = box_px * p.KC * 2, b_bytes = p.BN * p.KC * 2;
     const int b_off = (128 * p.KC * 2 + 1023) & ~1023;
     const int stage_bytes = b_off + ((b_bytes + 1023) & ~1023);
-    float *estage = (float *)(tiles + kStages * stage_bytes);
-    TcShared *sh = (TcShared *)((uint8_t *)estage + kEpiStageBytes + kEpiSumFloats * 4);
+    // behind the operand ring: the staged epilogue's row stage and running sums, or (epi_tma) the partner ring,
+    // two output groups and the running sums per column group
+    float *estage = (float *)(tiles + p.stages * stage_bytes);
+    const int ng = p.epi_tma ? p.BN / p.GW : 0;
+    uint8_t *auxr = (uint8_t *)estage;
+    uint8_t *outr = auxr + (p.need_aux ? ng : 0) * p.group_bytes;
+    float *gsums = (float *)(outr + 2 * p.group_bytes);
+    TcShared *sh = p.epi_tma ? (TcShared *)(gsums + ng * 128 * 8) : (TcShared *)((uint8_t *)estage + kEpiStageBytes + kEpiSumFloats * 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int iters = p.taps * p.chunks;
+    const int iters = p.ntap * p.chunks;
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < 2 * p.BN) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; s++) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
         for (int b = 0; b < 2; b++) { mbar_init(&sh->acc_full[b], 1); mbar_init(&sh->acc_empty[b], 128); }
+        for (int b = 0; b < 8; b++) mbar_init(&sh->aux_full[b], 1);
         sh->failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tma_prefetch_desc(&map_a); tma_prefetch_desc(&map_b);
+        if (p.epi_tma) { tma_prefetch_desc(&map_o0); tma_prefetch_desc(&map_o1); tma_prefetch_desc(&map_x0); tma_prefetch_desc(&map_x1); }
     }
     if (warp == 1) tmem_alloc(&sh->tmem_base, tmem_cols);
     if (warp >= 2) build_row_map(p.g, &sh->rows, ((warp & 3) << 5) | lane);
@@ -85,7 +173,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     pdl_enter();             // the set-up above may overlap the kernel before; its outputs are read from here on
     const uint32_t tmem_d = sh->tmem_base;
     const int col0 = blockIdx.y * p.BN;
-    const int pad = p.k / 2;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -95,14 +182,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 int n0, h0;
                 tile_origin(p.g, t, n0, h0);
                 for (int it = 0; it < iters; it++, itg++) {
-                    const int s = itg % kStages; const uint32_t round = itg / kStages;
+                    const int s = itg % p.stages; const uint32_t round = itg / p.stages;
                     if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
-                    const int tap = it / p.chunks, ch = it - tap * p.chunks;
-                    const int kh = tap / p.k, kw = tap - kh * p.k;
+                    const int ti = it / p.chunks, ch = it - ti * p.chunks;
                     uint8_t *sa = tiles + s * stage_bytes;
                     mbar_expect_tx(&sh->full[s], (uint32_t)(a_bytes + b_bytes));
-                    tma_load_4d(sa, &map_a, &sh->full[s], ch * p.KC, kw - pad, h0 * p.stride + kh - pad, n0);
-                    tma_load_2d(sa + b_off, &map_b, &sh->full[s], tap * p.cin_pad + ch * p.KC, col0);
+                    tma_load_4d(sa, &map_a, &sh->full[s], ch * p.KC, p.tdx[ti], h0 * p.stride + p.tdy[ti], n0);
+                    tma_load_2d(sa + b_off, &map_b, &sh->full[s], p.tid[ti] * p.cin_pad + ch * p.KC, col0);
                 }
             }
         }
@@ -119,7 +205,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 tc_fence_after();
                 const uint32_t acc = tmem_d + (uint32_t)(buf * p.BN);
                 for (int it = 0; it < iters; it++, itg++) {
-                    const int s = itg % kStages; const uint32_t round = itg / kStages;
+                    const int s = itg % p.stages; const uint32_t round = itg / p.stages;
                     if (!mbar_wait(&sh->full[s], round & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = smem_u32(tiles + s * stage_bytes);
@@ -133,7 +219,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (ok) mma_commit(&sh->acc_full[buf]);
             }
         }
-    } else {
+    } else if (!p.epi_tma) {
         // epilogue: this warp may touch accumulator lanes 32*(warp%4) .. +31
         const int etid = ((warp & 3) << 5) | lane;
         float *esums = estage + 128 * kEpiPitch;
@@ -155,6 +241,119 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
         if (ok) epilogue_finish(p.epi, p.BN, col0, estage, esums, etid);
         else if (lane == 0) atomicExch(&sh->failed, 1u);
+    } else {
+        // epilogue through TMA: thread etid owns accumulator row etid = pixel etid of the tile's box
+        const int etid = ((warp & 3) << 5) | lane;
+        const EpiArgs &e = p.epi;
+        const int GW = p.GW, QW = GW >> 2, rpp = 128 / QW;
+        const int jq = etid % QW, r0 = etid / QW;
+        const int box_px_o = p.g.BIMG * p.g.BH * p.g.W;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const float out_q = e.out.q, out_s = out_q != 0.f ? 1.f / out_q : 0.f, t_q = e.t.q;
+        const uint32_t aux_tx = (uint32_t)(box_px_o * GW * 4);
+        for (int i = etid; i < ng * 128 * 8; i += 128) gsums[i] = 0.f;
+        // column group gi of this N tile: which tensor of a channel-split pair, and the channel inside it
+        auto out_map = [&](int col) { return (p.split_o && col >= p.split_o) ? &map_o1 : &map_o0; };
+        auto aux_map = [&](int col) { return (p.split_x && col >= p.split_x) ? &map_x1 : &map_x0; };
+        auto col_out = [&](int col) { return (p.split_o && col >= p.split_o) ? col - p.split_o : col; };
+        auto col_aux = [&](int col) { return (p.split_x && col >= p.split_x) ? col - p.split_x : col; };
+        auto load_aux = [&](int gi, int n0, int h0) {        // one thread
+            const int col = col0 + gi * GW;
+            if (col >= e.n_cols) return;
+            mbar_expect_tx(&sh->aux_full[gi], aux_tx);
+            tma_load_4d(auxr + gi * p.group_bytes, aux_map(col), &sh->aux_full[gi], col_aux(col), p.ox, h0 * p.ostride + p.oy, n0);
+        };
+        if (etid == 0 && p.need_aux && (int)blockIdx.x < p.g.n_px_tiles) {
+            int n0, h0;
+            tile_origin(p.g, blockIdx.x, n0, h0);
+            for (int gi = 0; gi < ng; gi++) load_aux(gi, n0, h0);
+        }
+        named_barrier(1, 128);
+        bool ok = true;
+        int ti = 0;
+        uint32_t gc = 0;                                   // column groups handled so far: output slots alternate
+        for (int t = blockIdx.x; t < p.g.n_px_tiles; t += gridDim.x, ti++) {
+            const int buf = ti & 1; const uint32_t use = ti >> 1;
+            int n0, h0;
+            tile_origin(p.g, t, n0, h0);
+            const int tn = t + (int)gridDim.x;
+            int nn0 = 0, nh0 = 0;
+            if (tn < p.g.n_px_tiles) tile_origin(p.g, tn, nn0, nh0);
+            const int valid_px = p.g.BIMG > 1 ? (p.g.N - n0 < p.g.BIMG ? p.g.N - n0 : p.g.BIMG) * p.g.BH * p.g.W
+                                              : (p.g.H - h0 < p.g.BH ? p.g.H - h0 : p.g.BH) * p.g.W;
+            if (etid == 0) ok = mbar_wait(&sh->acc_full[buf], use & 1) && sh->failed == 0;     // one thread polls, the rest block
+            ok = named_barrier_and(2, 128, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t tm = tmem_d + lane_base + (uint32_t)(buf * p.BN);
+#pragma unroll 1
+            for (int gi = 0; gi < ng; gi++, gc++) {
+                const int col = col0 + gi * GW;
+                const bool live = col < e.n_cols;          // groups beyond the valid channels only drain their columns
+                uint8_t *ob = outr + (gc & 1) * p.group_bytes;
+                const uint8_t *ax = auxr + gi * p.group_bytes;
+                if (etid == 0) {
+                    if (p.need_aux && live) ok = mbar_wait(&sh->aux_full[gi], ti & 1);
+                    tma_store_wait_read_but_one();         // the store that last read this output slot is done with it
+                }
+                ok = named_barrier_and(2, 128, ok);
+                if (!ok) break;
+                const bool rowv = live && etid < valid_px;
+                const uint32_t tg = tm + (uint32_t)(gi * GW);
+                if (e.mode != EPI_COUPLE) {
+                    if (out_q == 0.f) tma_pass_a<0>(tg, GW, etid, rowv, ax, ob, out_s); else tma_pass_a<1>(tg, GW, etid, rowv, ax, ob, out_s);
+                } else if (out_q == 0.f) {
+                    if (e.sign > 0) tma_pass_a<2>(tg, GW, etid, rowv, ax, ob, out_s); else tma_pass_a<3>(tg, GW, etid, rowv, ax, ob, out_s);
+                } else {
+                    if (e.sign > 0) tma_pass_a<4>(tg, GW, etid, rowv, ax, ob, out_s); else tma_pass_a<5>(tg, GW, etid, rowv, ax, ob, out_s);
+                }
+                if (gi == ng - 1) { tc_fence_before(); mbar_arrive(&sh->acc_empty[buf]); }
+                fence_proxy_async();
+                named_barrier(1, 128);
+                if (etid == 0 && live) {
+                    tma_store_4d(out_map(col), ob, col_out(col), p.ox, h0 * p.ostride + p.oy, n0);
+                    tma_store_commit();
+                }
+                if (e.part && live && col + jq * 4 < e.n_cols) {
+                    float4 sc4 = make_float4(0, 0, 0, 0), sh4 = sc4, mu4 = sc4, rs4 = sc4;
+                    if (e.mode == EPI_BNBWD) bn_coef4(e.bn, col + jq * 4, sc4, sh4, mu4, rs4);
+                    float4 *slot = reinterpret_cast<float4 *>(gsums + (gi * 128 + etid) * 8);
+                    const float4 a0 = slot[0], a1 = slot[1];
+                    float acc[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                    if (e.mode == EPI_BNBWD) {
+                        if (t_q == 0.f) tma_pass_b<2>(GW, ob, ax, jq, r0, rpp, valid_px, 0.f, sc4, sh4, mu4, rs4, acc);
+                        else tma_pass_b<3>(GW, ob, ax, jq, r0, rpp, valid_px, t_q, sc4, sh4, mu4, rs4, acc);
+                    } else if (out_q == 0.f) tma_pass_b<0>(GW, ob, ax, jq, r0, rpp, valid_px, 0.f, sc4, sh4, mu4, rs4, acc);
+                    else tma_pass_b<1>(GW, ob, ax, jq, r0, rpp, valid_px, out_q, sc4, sh4, mu4, rs4, acc);
+                    slot[0] = make_float4(acc[0], acc[1], acc[2], acc[3]); slot[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+                }
+                named_barrier(1, 128);                     // the partner group and the output slot have been read
+                if (etid == 0 && p.need_aux && tn < p.g.n_px_tiles) load_aux(gi, nn0, nh0);
+            }
+            if (!ok) break;
+        }
+        if (etid == 0) tma_store_wait_all();
+        if (ok && e.part) {
+            // per-CTA record: the threads that share a channel quad are added in order
+            named_barrier(1, 128);
+            float *mine = e.part + (size_t)blockIdx.x * 2 * e.n_cols;
+            for (int gi = 0; gi < ng; gi++) {
+                const int col = col0 + gi * GW + jq * 4;
+                if (r0 == 0 && col < e.n_cols) {
+                    const float *base = gsums + (size_t)gi * 128 * 8;
+                    float r[8];
+#pragma unroll
+                    for (int j = 0; j < 8; j++) r[j] = base[jq * 8 + j];
+                    for (int y = 1; y < rpp; y++)
+#pragma unroll
+                        for (int j = 0; j < 8; j++) r[j] += base[(y * QW + jq) * 8 + j];
+                    *reinterpret_cast<float4 *>(mine + 2 * col) = make_float4(r[0], r[1], r[2], r[3]);
+                    *reinterpret_cast<float4 *>(mine + 2 * col + 4) = make_float4(r[4], r[5], r[6], r[7]);
+                }
+            }
+            epilogue_publish<128>(e, reinterpret_cast<float *>(auxr), etid);
+        }
+        if (!ok && lane == 0) atomicExch(&sh->failed, 1u);
     }
     tc_fence_before();
     __syncthreads();
@@ -183,20 +382,43 @@ __global__ void pack_weights_kernel(const float *__restrict__ W, bf16 *__restric
     }
 }
 
-// all packs of a step in one launch: blockIdx.y walks the job table
+// all packs of a step in one launch: blockIdx.y walks the job table.  A block (32 x 8 threads) takes
+// 32 x 32 tiles (rows x columns of the pack, one tap): both the fp32 reads and the bf16 writes of a
+// warp are contiguous, the transposed pack going through shared memory.
 __global__ void pack_weights_batch_kernel(const PackJob *__restrict__ jobs) {
     pdl_enter();
+    __shared__ float tile[32][33];
     const PackJob j = jobs[blockIdx.y];
     const int taps = j.k * j.k;
-    const size_t n = (size_t)j.rows_pad * taps * j.cols_pad;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        const int c = (int)(i % j.cols_pad);
-        const int tap = (int)((i / j.cols_pad) % taps);
-        const int r = (int)(i / ((size_t)j.cols_pad * taps));
-        float v = 0.f;
-        if (!j.transposed) { if (r < j.Co && c < j.Ci) v = j.W[((size_t)r * taps + tap) * j.Ci + c]; }
-        else { if (r < j.Ci && c < j.Co) v = j.W[((size_t)c * taps + (taps - 1 - tap)) * j.Ci + r]; }
-        j.out[i] = __float2bfloat16_rn(v);
+    const int rt = (j.rows_pad + 31) >> 5, ct = (j.cols_pad + 31) >> 5;
+    const int n_tiles = taps * rt * ct;
+    const int tx = threadIdx.x, ty = threadIdx.y;
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
+        const int c0 = (t % ct) << 5, r0 = ((t / ct) % rt) << 5, tap = t / (ct * rt);
+        if (!j.transposed) {
+#pragma unroll
+            for (int rr = 0; rr < 32; rr += 8) {
+                const int r = r0 + rr + ty, c = c0 + tx;
+                if (r < j.rows_pad && c < j.cols_pad) {
+                    const float v = (r < j.Co && c < j.Ci) ? j.W[((size_t)r * taps + tap) * j.Ci + c] : 0.f;
+                    j.out[((size_t)r * taps + tap) * j.cols_pad + c] = __float2bfloat16_rn(v);
+                }
+            }
+        } else {
+            // rows of the pack are input channels, columns output channels, taps mirrored
+#pragma unroll
+            for (int rr = 0; rr < 32; rr += 8) {
+                const int co = c0 + rr + ty, ci = r0 + tx;
+                tile[rr + ty][tx] = (co < j.Co && ci < j.Ci) ? j.W[((size_t)co * taps + (taps - 1 - tap)) * j.Ci + ci] : 0.f;
+            }
+            __syncthreads();
+#pragma unroll
+            for (int rr = 0; rr < 32; rr += 8) {
+                const int r = r0 + rr + ty, c = c0 + tx;
+                if (r < j.rows_pad && c < j.cols_pad) j.out[((size_t)r * taps + tap) * j.cols_pad + c] = __float2bfloat16_rn(tile[tx][rr + ty]);
+            }
+            __syncthreads();
+        }
     }
 }
 
@@ -250,16 +472,48 @@ bool tc_shape(Geom g, int cin, int cout, int k, int stride, TcShape &s) {   // g
 }
 
 // act: bf16 [N,H,W,cin]; Wsrc: fp32 weights; transposed selects the dgrad pack
+// s2cls (optional): {py, px}, one parity class of the data gradient of a 3x3 stride-2 layer.  `act` is then the
+// upstream gradient on the layer's output grid (gin), `out` the gradient on the input grid (twice as fine): the
+// launch fills the pixels (2i + py, 2j + px) from the taps that reach them,
+//   da[2i+py, 2j+px] = sum over th in T(py), tw in T(px) of g[i + th/2, j + tw/2] Wd[th, tw],  T(0) = {1}, T(1) = {0, 2}
+// (Wd the mirrored, transposed pack), so the four classes together cost the nine taps once per four pixels.
 bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin, int cout, int k, int stride,
-                 const float *Wsrc, const bf16 *prepacked, bool transposed, Pair out, Pair partner, int sign, EpiReq req) {
+                 const float *Wsrc, const bf16 *prepacked, bool transposed, Pair out, Pair partner, int sign, EpiReq req,
+                 const int *s2cls = nullptr) {
     TcShape s;
     if (stride == 2 && (gin.H % 2 || gin.W % 2)) return false;
-    const Geom g{gin.N, conv_out(gin.H, k, stride), conv_out(gin.W, k, stride)};   // output geometry
+    if (s2cls && (stride != 1 || k != 3 || !transposed || sign || req.stats || req.bnbwd || out.c1)) return false;
+    const Geom g{gin.N, conv_out(gin.H, k, stride), conv_out(gin.W, k, stride)};   // geometry of the tiles
     if (!tc_shape(g, cin, cout, k, stride, s)) return false;
     const int taps = k * k;
     const int rows_pad = s.n_tiles * s.BN;
     if (!ex.dry && !encoder(ex.ctx)) return false;
-    ex.flops += 2ull * g.P() * cout * cin * taps;
+    // the taps of this launch
+    int ntap = 0;
+    signed char tdy[9], tdx[9], tid[9];
+    for (int th = 0; th < k; th++)
+        for (int tw = 0; tw < k; tw++) {
+            if (s2cls && ((th & 1) == s2cls[0] || (tw & 1) == s2cls[1])) continue;
+            tdy[ntap] = (signed char)(s2cls ? th / 2 : th - k / 2); tdx[ntap] = (signed char)(s2cls ? tw / 2 : tw - k / 2);
+            tid[ntap] = (signed char)(th * k + tw); ntap++;
+        }
+    ex.flops += 2ull * g.P() * cout * cin * ntap;
+    // epilogue through TMA where a column group never straddles the halves of a channel-split tensor
+    const bool need_aux = sign != 0 || req.bnbwd != nullptr;
+    const Pair auxp = req.bnbwd ? req.bnbwd->t : partner;
+    const int GW = s.BN % 32 == 0 ? 32 : 16, ng = s.BN / GW, group_bytes = (128 * GW * 4 + 1023) & ~1023;
+    bool epi_tma = !(out.c1 && out.c0 % GW) && !(need_aux && auxp.c1 && auxp.c0 % GW) && ng <= 8;
+    const int ostride = s2cls ? 2 : 1;
+    if (s2cls && (!epi_tma || g.W * 2 > 256 || s.g.BH * 2 > 256)) return false;
+    int stages = kStages;
+    if (epi_tma) {
+        const int stage_bytes = ((128 * s.KC * 2 + 1023) & ~1023) + ((s.BN * s.KC * 2 + 1023) & ~1023);
+        auto smem_of = [&](int st) { return 1024 + st * stage_bytes + ((need_aux ? ng : 0) + 2) * group_bytes + ng * 128 * 32 + (int)sizeof(TcShared) + 64; };
+        while (stages > 2 && smem_of(stages) > 227 * 1024) stages--;
+        if (smem_of(stages) > 227 * 1024) { epi_tma = false; stages = kStages; }
+        else s.smem = smem_of(stages);
+    }
+    if (s2cls && !epi_tma) return false;
     int occ = (227 * 1024) / s.smem; if (occ > 2) occ = 2; if (occ < 1) occ = 1;
     int ctas = ex.ctx->sm_count * occ / s.n_tiles; if (ctas < 1) ctas = 1;
     if (ctas > s.g.n_px_tiles) ctas = s.g.n_px_tiles;
@@ -299,7 +553,34 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
                              sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
             if (r != CUDA_SUCCESS) { ex.failed = true; ex.ctx->err = std::string(what) + ": tensor map (weights) rejected"; ex.ws.release(m); return true; }
         }
+        CUtensorMap map_o[2], map_x[2];
+        memset(map_o, 0, sizeof map_o); memset(map_x, 0, sizeof map_x);
+        if (epi_tma) {
+            const CUtensorMapSwizzle gsw = GW == 32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+            auto enc_f32 = [&](CUtensorMap *map, const float *base, int C) {
+                // the epilogue's tensors live on the output grid: the tile's grid, or (parity class) the twice finer
+                // one walked with stride 2
+                const cuuint64_t Wo = (cuuint64_t)g.W * ostride, Ho = (cuuint64_t)g.H * ostride;
+                cuuint64_t dims[4] = {(cuuint64_t)C, Wo, Ho, (cuuint64_t)g.N};
+                cuuint64_t strides[3] = {(cuuint64_t)C * 4, Wo * C * 4, Ho * Wo * C * 4};
+                cuuint32_t box[4] = {(cuuint32_t)GW, (cuuint32_t)(g.W * ostride), (cuuint32_t)(s.g.BH * ostride), (cuuint32_t)s.g.BIMG};
+                cuuint32_t es[4] = {1, (cuuint32_t)ostride, (cuuint32_t)ostride, 1};
+                return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, (void *)base, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           gsw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+            };
+            bool ok = enc_f32(&map_o[0], out.p0, out.c0);
+            if (out.c1) ok = ok && enc_f32(&map_o[1], out.p1, out.c1); else map_o[1] = map_o[0];
+            if (need_aux) {
+                ok = ok && enc_f32(&map_x[0], auxp.p0, auxp.c0);
+                if (auxp.c1) ok = ok && enc_f32(&map_x[1], auxp.p1, auxp.c1); else map_x[1] = map_x[0];
+            } else { map_x[0] = map_x[1] = map_o[0]; }
+            if (!ok) { ex.failed = true; ex.ctx->err = std::string(what) + ": tensor map (epilogue) rejected"; ex.ws.release(m); return true; }
+        }
         TcParams p;
+        p.stages = stages; p.epi_tma = epi_tma ? 1 : 0; p.GW = GW; p.group_bytes = group_bytes; p.need_aux = need_aux ? 1 : 0;
+        p.split_o = out.c1 ? out.c0 : 0; p.split_x = (need_aux && auxp.c1) ? auxp.c0 : 0;
+        p.ntap = ntap; memcpy(p.tdy, tdy, 9); memcpy(p.tdx, tdx, 9); memcpy(p.tid, tid, 9);
+        p.ostride = ostride; p.oy = s2cls ? s2cls[0] : 0; p.ox = s2cls ? s2cls[1] : 0;
         p.taps = taps; p.k = k; p.chunks = s.chunks; p.KC = s.KC; p.cin_pad = s.cin_pad; p.BN = s.BN; p.stride = stride; p.g = s.g;
         p.status = ex.ctx->dev_status;
         EpiArgs &e = p.epi;
@@ -313,9 +594,9 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         static bool attr_set = false;
         if (!attr_set) { cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024); attr_set = true; }
         dim3 grid((unsigned)ctas, (unsigned)s.n_tiles);
-        launch(ex, conv_tc_kernel, grid, kThreads, s.smem, map_a, map_b, p);
+        launch(ex, conv_tc_kernel, grid, kThreads, s.smem, map_a, map_b, map_o[0], map_o[1], map_x[0], map_x[1], p);
         const double bytes = (double)gin.P() * cin * 2 + (double)g.P() * cout * (sign || req.bnbwd ? 8 : 4) + (double)cout * taps * cin * 2;
-        ex.check(what, bytes, 2.0 * g.P() * cout * cin * taps);
+        ex.check(what, bytes, 2.0 * g.P() * cout * cin * ntap);
     }
     ex.ws.release(m);
     return true;
@@ -566,6 +847,19 @@ bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, 
 }
 
 
+// Data gradient of a 3x3 stride-2 layer: four launches, one per parity class of the input pixels (see
+// run_conv_tc).  g: bf16 [N, H/2, W/2, cout]; da: fp32 [N, H, W, cin].
+bool conv_dgrad_tc_s2(Exec &ex, const void *g, Geom gi, const Layer &L, float *da) {
+    if (L.stride != 2 || L.k != 3 || gi.H % 2 || gi.W % 2) return false;
+    const Geom go{gi.N, gi.H / 2, gi.W / 2};
+    for (int cls = 0; cls < 4; cls++) {
+        const int pc[2] = {cls >> 1, cls & 1};
+        if (!run_conv_tc(ex, "conv_dgrad_tc", g, go, L.cout, L.cin, 3, 1, L.W, L.Wp_dgrad, true, single(da, L.cin), Pair{}, 0, EpiReq{}, pc))
+            return false;     // refused before anything was launched: every class takes the same decision
+    }
+    return true;
+}
+
 constexpr int kWgSmemMax = 224 * 1024;
 
 // Shape decisions of one layer's weight gradient; cta_budget: the CTAs the job may take
@@ -719,10 +1013,10 @@ PackJob tc_pack_job(const float *W, bf16 *out, int cin, int cout, int k, bool tr
 }
 void tc_pack_batch(Exec &ex, const PackJob *jobs_dev, int n_jobs, double bytes, size_t max_job_elems) {
     if (ex.dry || n_jobs == 0) return;
-    // blocks per job sized for the largest job (2048 elements per block), within 4 .. 96
-    size_t bx = (max_job_elems + 2047) / 2048;
-    if (bx < 4) bx = 4; if (bx > 96) bx = 96;
+    // blocks per job sized for the largest job (four 32 x 32 tiles per block), within 2 .. 592
+    size_t bx = (max_job_elems + 4095) / 4096;
+    if (bx < 2) bx = 2; if (bx > 592) bx = 592;
     dim3 grid((unsigned)bx, (unsigned)n_jobs);
-    launch(ex, pack_weights_batch_kernel, grid, 256, 0, jobs_dev);
+    launch(ex, pack_weights_batch_kernel, grid, dim3(32, 8), 0, jobs_dev);
     ex.check("pack_weights_batch", bytes);
 }

@@ -27,7 +27,23 @@ void Exec::check(const char *what, double bytes, double flops) {
         ctx->prof.push_back(ProfRec{what, bytes, flops, ev});
     }
 }
+// Keeps the stream busy for `ns` nanoseconds (bounded) so that the host gets ahead of the device:
+// the per-kernel events of a profiled step then measure kernels that were already queued, not the
+// host's launch rate.
+__global__ void profile_hold_kernel(unsigned long long ns) {
+    unsigned long long t0, t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    for (int i = 0; i < 100000; i++) {
+        __nanosleep(1000);
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+        if (t - t0 >= ns) break;
+    }
+}
 void Exec::mark(const char *what) {
+    if (ctx->profiling && !dry && hold_ns) {
+        profile_hold_kernel<<<1, 1, 0, stream>>>(hold_ns);
+        hold_ns = 0;
+    }
     if (ctx->profiling && !dry) {
         cudaEvent_t ev = ctx->next_event();
         cudaEventRecord(ev, stream);
@@ -350,31 +366,39 @@ __global__ void maxpool_fwd_kernel(const float *__restrict__ in, float *__restri
 // Gradient goes to the first maximum met in (kh,kw) row-major scan of each window.  Gather form:
 // each input element visits the (at most four) windows that cover it, in a fixed order.
 __global__ void maxpool_bwd_kernel(const float *__restrict__ in, const float *__restrict__ dout, float *__restrict__ din,
-                                   int N, int H, int W, int C, int Ho, int Wo) {
+                                   int N, int H, int W, int C4, int Ho, int Wo) {
     pdl_enter();
-    size_t n = (size_t)N * H * W * C;
+    size_t n = (size_t)N * H * W * C4;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        int c = (int)(i % C); size_t p = i / C;
+        int q = (int)(i % C4); size_t p = i / C4;
         int x = (int)(p % W); p /= W; int y = (int)(p % H); int b = (int)(p / H);
-        const float self = in[i];
-        float acc = 0.f;
-        for (int io = (y + 1 - 2 + 1) / 2; io <= (y + 1) / 2; io++) {
-            if (io < 0 || io >= Ho || io * 2 - 1 > y || io * 2 + 1 < y) continue;
-            for (int j = (x + 1 - 2 + 1) / 2; j <= (x + 1) / 2; j++) {
-                if (j < 0 || j >= Wo || j * 2 - 1 > x || j * 2 + 1 < x) continue;
-                // is (y,x) the first maximum of window (io,j)?
-                bool first = true;
-                for (int kh = 0; kh < 3 && first; kh++) for (int kw = 0; kw < 3; kw++) {
+        const float4 self = ld4(in + i * 4);
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        // windows (io, j) that cover (y, x): io*2 - 1 <= y <= io*2 + 1
+        for (int io = y / 2; io <= (y + 1) / 2; io++) {
+            if (io >= Ho) continue;
+            for (int j = x / 2; j <= (x + 1) / 2; j++) {
+                if (j >= Wo) continue;
+                // per channel: is (y,x) the first maximum of window (io,j)?
+                bool f0 = true, f1 = true, f2 = true, f3 = true;
+                for (int kh = 0; kh < 3; kh++) for (int kw = 0; kw < 3; kw++) {
                     int yy = io * 2 + kh - 1, xx = j * 2 + kw - 1;
-                    if (yy < 0 || yy >= H || xx < 0 || xx >= W) continue;
-                    float v = in[(((size_t)b * H + yy) * W + xx) * C + c];
-                    bool before = (yy < y) || (yy == y && xx < x);
-                    if (v > self || (before && v == self)) { first = false; break; }
+                    if (yy < 0 || yy >= H || xx < 0 || xx >= W || (yy == y && xx == x)) continue;
+                    const float4 v = ld4(in + ((((size_t)b * H + yy) * W + xx) * C4 + q) * 4);
+                    const bool before = (yy < y) || (yy == y && xx < x);
+                    f0 = f0 && !(v.x > self.x || (before && v.x == self.x));
+                    f1 = f1 && !(v.y > self.y || (before && v.y == self.y));
+                    f2 = f2 && !(v.z > self.z || (before && v.z == self.z));
+                    f3 = f3 && !(v.w > self.w || (before && v.w == self.w));
                 }
-                if (first) acc += dout[(((size_t)b * Ho + io) * Wo + j) * C + c];
+                const float4 g = ld4(dout + ((((size_t)b * Ho + io) * Wo + j) * C4 + q) * 4);
+                if (f0) acc.x += g.x;
+                if (f1) acc.y += g.y;
+                if (f2) acc.z += g.z;
+                if (f3) acc.w += g.w;
             }
         }
-        din[i] = acc;
+        st4(din + i * 4, acc);
     }
 }
 
@@ -388,8 +412,8 @@ void maxpool_fwd(Exec &ex, const float *in, float *out, int N, int H, int W, int
 void maxpool_bwd(Exec &ex, const float *in, const float *dout, float *din, int N, int H, int W, int C) {
     if (ex.dry) return;
     int Ho = conv_out(H, 3, 2), Wo = conv_out(W, 3, 2);
-    size_t n = (size_t)N * H * W * C;
-    launch(ex, maxpool_bwd_kernel, ew_grid(n, ex.ctx->sm_count), 256, 0, in, dout, din, N, H, W, C, Ho, Wo);
+    size_t n = (size_t)N * H * W * (C / 4);
+    launch(ex, maxpool_bwd_kernel, ew_grid(n, ex.ctx->sm_count), 256, 0, in, dout, din, N, H, W, C / 4, Ho, Wo);
     ex.check("maxpool_bwd");
 }
 

@@ -402,6 +402,7 @@ extern "C" int revnet_train_step(revnet_ctx *ctx, revnet_plan *pl, const float *
     ex.stream = use_graph ? ctx->capture_stream : (cudaStream_t)stream;
     ex.q = pl->d.state_frac_bits ? ldexpf(1.f, -pl->d.state_frac_bits) : 0.f;
     ex.ws.dry = false; ex.ws.base = (char *)workspace; ex.ws.cap = pl->ws_bytes;
+    if (ctx->profiling) ex.hold_ns = 5000000ull;     // the launches of a profiled step queue up behind a 5 ms hold
     if (use_graph) {
         if (pl->graph_exec) { cudaGraphExecDestroy(pl->graph_exec); pl->graph_exec = nullptr; }
         if (cudaStreamBeginCapture(ex.stream, cudaStreamCaptureModeRelaxed) != cudaSuccess)

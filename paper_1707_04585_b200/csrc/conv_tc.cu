@@ -24,7 +24,8 @@ using namespace tc;
 
 namespace {
 
-constexpr int kStages = 4;
+constexpr int kStages = 6;       // most operand stages of the convolution kernel
+constexpr int kWgStages = 4;     // ... of the weight-gradient kernel
 constexpr int kThreads = 192;
 
 struct TcParams {
@@ -456,7 +457,7 @@ bool tile_geom(Geom g, TileGeom &t) {
 struct TcShape { int KC, cin_pad, chunks, BN, n_tiles, smem; TileGeom g; };
 
 // Which shapes the kernel takes: stride 1 or 2, k in {1,3}, channel rows 16-byte aligned for TMA.
-bool tc_shape(Geom g, int cin, int cout, int k, int stride, TcShape &s) {   // g: output geometry
+bool tc_shape(Geom g, int cin, int cout, int k, int stride, TcShape &s, bool wide = false) {   // g: output geometry
     if ((stride != 1 && stride != 2) || (k != 1 && k != 3) || cin % 8 || cout % 4) return false;
     if (!tile_geom(g, s.g)) return false;
     if (s.g.W * stride > 256 || s.g.BH * stride > 256) return false;
@@ -465,9 +466,10 @@ bool tc_shape(Geom g, int cin, int cout, int k, int stride, TcShape &s) {   // g
     s.chunks = s.cin_pad / s.KC;
     const int cout_pad = round_up(cout, 16);
     s.BN = cout_pad <= 128 ? cout_pad : 128;
+    if (wide && cout_pad >= 256) s.BN = 256;        // 128 x 256 tiles: fewer operand bytes per flop
     s.n_tiles = (cout_pad + s.BN - 1) / s.BN;
     const int a_bytes = 128 * s.KC * 2, b_bytes = s.BN * s.KC * 2;
-    s.smem = 1024 + kStages * (((a_bytes + 1023) & ~1023) + ((b_bytes + 1023) & ~1023)) + kEpiStageBytes + kEpiSumFloats * 4 + (int)sizeof(TcShared) + 64;
+    s.smem = 1024 + 4 * (((a_bytes + 1023) & ~1023) + ((b_bytes + 1023) & ~1023)) + kEpiStageBytes + kEpiSumFloats * 4 + (int)sizeof(TcShared) + 64;
     return true;
 }
 
@@ -486,7 +488,6 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
     const Geom g{gin.N, conv_out(gin.H, k, stride), conv_out(gin.W, k, stride)};   // geometry of the tiles
     if (!tc_shape(g, cin, cout, k, stride, s)) return false;
     const int taps = k * k;
-    const int rows_pad = s.n_tiles * s.BN;
     if (!ex.dry && !encoder(ex.ctx)) return false;
     // the taps of this launch
     int ntap = 0;
@@ -501,19 +502,26 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
     // epilogue through TMA where a column group never straddles the halves of a channel-split tensor
     const bool need_aux = sign != 0 || req.bnbwd != nullptr;
     const Pair auxp = req.bnbwd ? req.bnbwd->t : partner;
+    // arithmetic-bound layers without a partner tile (transitions, their data gradients): 128 x 256 tiles
+    if (!need_aux && !(out.c1 && out.c0 % 32) && (long long)ntap * cin >= 1024 && cout >= 256 && cout % 32 == 0) tc_shape(g, cin, cout, k, stride, s, true);
+    // rows of the weight pack (a multiple of its 128-row blocks, whatever the N tile); TMA fills rows beyond with zeros
+    const int rp16 = round_up(cout, 16), rows_pad = rp16 <= 128 ? rp16 : round_up(rp16, 128);
     const int GW = s.BN % 32 == 0 ? 32 : 16, ng = s.BN / GW, group_bytes = (128 * GW * 4 + 1023) & ~1023;
     bool epi_tma = !(out.c1 && out.c0 % GW) && !(need_aux && auxp.c1 && auxp.c0 % GW) && ng <= 8;
     const int ostride = s2cls ? 2 : 1;
     if (s2cls && (!epi_tma || g.W * 2 > 256 || s.g.BH * 2 > 256)) return false;
-    int stages = kStages;
+    int stages = 4;
     if (epi_tma) {
+        stages = kStages;
         const int stage_bytes = ((128 * s.KC * 2 + 1023) & ~1023) + ((s.BN * s.KC * 2 + 1023) & ~1023);
         auto smem_of = [&](int st) { return 1024 + st * stage_bytes + ((need_aux ? ng : 0) + 2) * group_bytes + ng * 128 * 32 + (int)sizeof(TcShared) + 64; };
         while (stages > 2 && smem_of(stages) > 227 * 1024) stages--;
-        if (smem_of(stages) > 227 * 1024) { epi_tma = false; stages = kStages; }
-        else s.smem = smem_of(stages);
+        if (smem_of(stages) > 227 * 1024) {
+            if (s.BN == 256) return false;      // (does not happen: three stages of a wide tile fit)
+            epi_tma = false; stages = 4;
+        } else s.smem = smem_of(stages);
     }
-    if (s2cls && !epi_tma) return false;
+    if ((s2cls || s.BN == 256) && !epi_tma) return false;
     int occ = (227 * 1024) / s.smem; if (occ > 2) occ = 2; if (occ < 1) occ = 1;
     int ctas = ex.ctx->sm_count * occ / s.n_tiles; if (ctas < 1) ctas = 1;
     if (ctas > s.g.n_px_tiles) ctas = s.g.n_px_tiles;
@@ -899,7 +907,7 @@ static bool wgrad_plan(Geom gi, const Layer &L, int cta_budget, WgPlan &w, bool 
     p.a_region = (blocks_max * 256 * p.blockC + 1023) & ~1023;
     w.stage_bytes = p.a_region + ((256 * p.BN + 1023) & ~1023);
     w.tail_bytes = p.GM * 32768 - p.a_region;        // what the MMAs of a partly filled group read past the last stage
-    p.stages = (kWgSmemMax - 2048 - w.tail_bytes) / w.stage_bytes; if (p.stages > kStages) p.stages = kStages;
+    p.stages = (kWgSmemMax - 2048 - w.tail_bytes) / w.stage_bytes; if (p.stages > kWgStages) p.stages = kWgStages;
     if (p.stages < 2) return p.sep ? wgrad_plan(gi, L, cta_budget, w, false) : false;
     // split the pixel reduction so that the job's CTAs cover its share of the machine once
     int splits = (cta_budget + p.m_chunks * w.n_tiles - 1) / (p.m_chunks * w.n_tiles);

@@ -266,7 +266,10 @@ int revnet_check_device(revnet_ctx *ctx, void *stream);
  * one text line per kernel name: "name<TAB>launches<TAB>total_ms<TAB>algorithmic_bytes<TAB>flops".
  * The time of a launch is the span between the previous event and its own, so the first record
  * after enabling is only a boundary.  buf may be NULL with buflen 0 to query `needed`.
- * Enabling (or disabling) clears earlier records. */
+ * Enabling (or disabling) clears earlier records.  on = 2 enables with one line per kernel name AND
+ * launch shape: the name then reads "name|algorithmic_bytes|flops" of one launch.  A profiled train
+ * step first holds the stream for 5 ms, so that its launches are queued by the time they run and
+ * the spans hold device time only; that hold is the record "step_begin". */
 int revnet_profile_enable(revnet_ctx *ctx, int on);
 int revnet_profile_summary(revnet_ctx *ctx, char *buf, size_t buflen, size_t *needed);
 

@@ -6,7 +6,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "librevnet.so")
-SOURCES = ["api.cu", "stack.cu", "block.cu", "elementwise.cu", "conv_simt.cu", "conv_tc.cu", "conv_fused.cu"]
+SOURCES = ["api.cu", "stack.cu", "block.cu", "elementwise.cu", "conv_simt.cu", "conv_tc.cu", "conv_fused.cu", "stem.cu"]
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
          "-Xcompiler", "-fPIC", "--use_fast_math=false" if False else "-DREVNET_BUILD"]
 

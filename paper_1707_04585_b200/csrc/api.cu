@@ -305,6 +305,7 @@ extern "C" int revnet_check_device(revnet_ctx *ctx, void *stream) {
 extern "C" int revnet_profile_enable(revnet_ctx *ctx, int on) {
     if (!ctx) return REVNET_E_INVALID_ARG;
     ctx->profiling = on != 0;
+    ctx->prof_detail = on == 2;
     ctx->prof.clear();
     ctx->ev_used = 0;
     return REVNET_OK;
@@ -320,9 +321,11 @@ extern "C" int revnet_profile_summary(revnet_ctx *ctx, char *buf, size_t buflen,
         const ProfRec &r = ctx->prof[i];
         float ms = 0.f;
         if (cudaEventElapsedTime(&ms, ctx->prof[i - 1].ev, r.ev) != cudaSuccess) { cudaGetLastError(); continue; }
+        std::string key = r.name;
+        if (ctx->prof_detail) { char sfx[64]; snprintf(sfx, sizeof sfx, "|%.0f|%.0f", r.bytes, r.flops); key += sfx; }
         Acc *a = nullptr;
-        for (auto &x : acc) if (x.name == r.name) { a = &x; break; }
-        if (!a) { acc.push_back(Acc()); a = &acc.back(); a->name = r.name; }
+        for (auto &x : acc) if (x.name == key) { a = &x; break; }
+        if (!a) { acc.push_back(Acc()); a = &acc.back(); a->name = key; }
         a->n++; a->ms += ms; a->bytes += r.bytes; a->flops += r.flops;
     }
     std::string out;

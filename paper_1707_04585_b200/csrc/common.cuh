@@ -27,6 +27,7 @@ struct revnet_ctx {
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     // per-kernel timing (revnet_profile_*): one event after every launch while enabled
     bool profiling = false;
+    bool prof_detail = false;   // summary lines per launch shape, not only per kernel name
     std::vector<ProfRec> prof;
     std::vector<cudaEvent_t> ev_pool;
     size_t ev_used = 0;
@@ -275,6 +276,11 @@ void upsample_zero_bf16(Exec &ex, const bf16 *in, bf16 *out, int N, int Ho, int 
 void conv_fprop_simt(Exec &ex, const void *a, bool a_bf16, Geom gi, const Layer &L, Pair out, Pair partner, int sign);
 void conv_dgrad_simt(Exec &ex, const void *g, bool g_bf16, Geom gi, const Layer &L, float *da);
 void conv_wgrad_simt(Exec &ex, const void *g, bool g_bf16, const void *a, bool a_bf16, Geom gi, const Layer &L, float *dW);
+
+// ---------------------------------------------------------------- stem.cu
+// the stem convolution of the image (few input channels), fp32; false: shape not taken, nothing launched
+bool stem_fprop(Exec &ex, const float *img, Geom gi, const Layer &L, Pair out);
+bool stem_wgrad(Exec &ex, const float *img, const float *gout, Geom gi, const Layer &L, float *dW);
 
 // ---------------------------------------------------------------- conv_tc.cu
 // What a data-gradient epilogue needs to fuse the two sums of the BN+ReLU backward of the layer's

@@ -154,10 +154,10 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
     Layer stem = bind(pl->stem, params, grads);
     Geom gimg{N, d.img, d.img};
     StagePlan &s0 = pl->st[0];
-    if (pl->stem_direct)
-        conv_fprop_simt(ex, images, false, gimg, stem, halves(actf(s0.off_x1), actf(s0.off_x2), s0.c, q), Pair{}, 0);
-    else
-        conv_fprop_simt(ex, images, false, gimg, stem, single(actf(pl->off_stem_out), d.stem_cout), Pair{}, 0);
+    {
+        const Pair so = pl->stem_direct ? halves(actf(s0.off_x1), actf(s0.off_x2), s0.c, q) : single(actf(pl->off_stem_out), d.stem_cout);
+        if (!stem_fprop(ex, images, gimg, stem, so)) conv_fprop_simt(ex, images, false, gimg, stem, so, Pair{}, 0);
+    }
     Pair prev = single(actf(pl->off_stem_out), d.stem_cout);
     int prevH = pl->stemH;
     if (d.maxpool) {
@@ -251,7 +251,7 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
         } else {
             gstem = gbuf[gi];
         }
-        conv_wgrad_simt(ex, gstem, false, images, false, gimg, stem, stem.dW);
+        if (!stem_wgrad(ex, images, gstem, gimg, stem, stem.dW)) conv_wgrad_simt(ex, gstem, false, images, false, gimg, stem, stem.dW);
         ex.ws.release(m);
     }
     sgd_update(ex, params, grads, mom, pl->n_params, seg_end, seg_decay, (int)nseg, d.lr, d.momentum, d.weight_decay);

@@ -26,7 +26,8 @@ namespace {
 
 constexpr int kStages = 6;       // most operand stages of the convolution kernel
 constexpr int kWgStages = 4;     // ... of the weight-gradient kernel
-constexpr int kThreads = 192;
+constexpr int kThreads = 192;      // TMA warp, MMA warp, four epilogue warps
+constexpr int kThreadsTma = 320;   // epilogue through TMA: two groups of four epilogue warps
 
 struct TcParams {
     int taps;        // k*k
@@ -132,7 +133,7 @@ __device__ __forceinline__ void tma_pass_b(int GW, const uint8_t *ob, const uint
 // Persistent CTA: walks the pixel tiles blockIdx.x, blockIdx.x + gridDim.x, ... of N tile blockIdx.y.
 // The operand ring runs on across tiles; the accumulator alternates between two tensor-memory
 // buffers so that the epilogue of one tile overlaps the MMAs of the next.
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsTma, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                const __grid_constant__ CUtensorMap map_o0, const __grid_constant__ CUtensorMap map_o1,
                const __grid_constant__ CUtensorMap map_x0, const __grid_constant__ CUtensorMap map_x1, const TcParams p) {
@@ -159,7 +160,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; s++) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
-        for (int b = 0; b < 2; b++) { mbar_init(&sh->acc_full[b], 1); mbar_init(&sh->acc_empty[b], 128); }
+        for (int b = 0; b < 2; b++) { mbar_init(&sh->acc_full[b], 1); mbar_init(&sh->acc_empty[b], p.epi_tma ? 256 : 128); }
         for (int b = 0; b < 8; b++) mbar_init(&sh->aux_full[b], 1);
         sh->failed = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -243,7 +244,11 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (ok) epilogue_finish(p.epi, p.BN, col0, estage, esums, etid);
         else if (lane == 0) atomicExch(&sh->failed, 1u);
     } else {
-        // epilogue through TMA: thread etid owns accumulator row etid = pixel etid of the tile's box
+        // epilogue through TMA: two groups of four warps; group wg takes the column groups wg, wg + 2, ... of every
+        // tile and owns output slot wg, so that one group's pass over shared memory overlaps the other's waits.
+        // Thread etid of a warp group owns accumulator row etid = pixel etid of the tile's box.
+        const int wg = (warp - 2) >> 2;
+        const int bar_a = 1 + 2 * wg, bar_b = 2 + 2 * wg;   // named barriers of this warp group; 5: both groups
         const int etid = ((warp & 3) << 5) | lane;
         const EpiArgs &e = p.epi;
         const int GW = p.GW, QW = GW >> 2, rpp = 128 / QW;
@@ -252,7 +257,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
         const float out_q = e.out.q, out_s = out_q != 0.f ? 1.f / out_q : 0.f, t_q = e.t.q;
         const uint32_t aux_tx = (uint32_t)(box_px_o * GW * 4);
-        for (int i = etid; i < ng * 128 * 8; i += 128) gsums[i] = 0.f;
+        for (int i = wg * 128 + etid; i < ng * 128 * 8; i += 256) gsums[i] = 0.f;
         // column group gi of this N tile: which tensor of a channel-split pair, and the channel inside it
         auto out_map = [&](int col) { return (p.split_o && col >= p.split_o) ? &map_o1 : &map_o0; };
         auto aux_map = [&](int col) { return (p.split_x && col >= p.split_x) ? &map_x1 : &map_x0; };
@@ -267,12 +272,12 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (etid == 0 && p.need_aux && (int)blockIdx.x < p.g.n_px_tiles) {
             int n0, h0;
             tile_origin(p.g, blockIdx.x, n0, h0);
-            for (int gi = 0; gi < ng; gi++) load_aux(gi, n0, h0);
+            for (int gi = wg; gi < ng; gi += 2) load_aux(gi, n0, h0);
         }
-        named_barrier(1, 128);
+        named_barrier(5, 256);
         bool ok = true;
         int ti = 0;
-        uint32_t gc = 0;                                   // column groups handled so far: output slots alternate
+        uint8_t *ob = outr + wg * p.group_bytes;
         for (int t = blockIdx.x; t < p.g.n_px_tiles; t += gridDim.x, ti++) {
             const int buf = ti & 1; const uint32_t use = ti >> 1;
             int n0, h0;
@@ -283,21 +288,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const int valid_px = p.g.BIMG > 1 ? (p.g.N - n0 < p.g.BIMG ? p.g.N - n0 : p.g.BIMG) * p.g.BH * p.g.W
                                               : (p.g.H - h0 < p.g.BH ? p.g.H - h0 : p.g.BH) * p.g.W;
             if (etid == 0) ok = mbar_wait(&sh->acc_full[buf], use & 1) && sh->failed == 0;     // one thread polls, the rest block
-            ok = named_barrier_and(2, 128, ok);
+            ok = named_barrier_and(bar_b, 128, ok);
             if (!ok) break;
             tc_fence_after();
             const uint32_t tm = tmem_d + lane_base + (uint32_t)(buf * p.BN);
 #pragma unroll 1
-            for (int gi = 0; gi < ng; gi++, gc++) {
+            for (int gi = wg; gi < ng; gi += 2) {
                 const int col = col0 + gi * GW;
                 const bool live = col < e.n_cols;          // groups beyond the valid channels only drain their columns
-                uint8_t *ob = outr + (gc & 1) * p.group_bytes;
                 const uint8_t *ax = auxr + gi * p.group_bytes;
                 if (etid == 0) {
                     if (p.need_aux && live) ok = mbar_wait(&sh->aux_full[gi], ti & 1);
-                    tma_store_wait_read_but_one();         // the store that last read this output slot is done with it
+                    tma_store_wait_read();                 // this group's last store is done with the output slot
                 }
-                ok = named_barrier_and(2, 128, ok);
+                ok = named_barrier_and(bar_b, 128, ok);
                 if (!ok) break;
                 const bool rowv = live && etid < valid_px;
                 const uint32_t tg = tm + (uint32_t)(gi * GW);
@@ -308,9 +312,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 } else {
                     if (e.sign > 0) tma_pass_a<4>(tg, GW, etid, rowv, ax, ob, out_s); else tma_pass_a<5>(tg, GW, etid, rowv, ax, ob, out_s);
                 }
-                if (gi == ng - 1) { tc_fence_before(); mbar_arrive(&sh->acc_empty[buf]); }
                 fence_proxy_async();
-                named_barrier(1, 128);
+                named_barrier(bar_a, 128);
                 if (etid == 0 && live) {
                     tma_store_4d(out_map(col), ob, col_out(col), p.ox, h0 * p.ostride + p.oy, n0);
                     tma_store_commit();
@@ -328,15 +331,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     else tma_pass_b<1>(GW, ob, ax, jq, r0, rpp, valid_px, out_q, sc4, sh4, mu4, rs4, acc);
                     slot[0] = make_float4(acc[0], acc[1], acc[2], acc[3]); slot[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
                 }
-                named_barrier(1, 128);                     // the partner group and the output slot have been read
+                named_barrier(bar_a, 128);                 // the partner group and the output slot have been read
                 if (etid == 0 && p.need_aux && tn < p.g.n_px_tiles) load_aux(gi, nn0, nh0);
             }
             if (!ok) break;
+            // this warp group has drained its columns of the accumulator (the other group arrives for its own)
+            tc_fence_before();
+            mbar_arrive(&sh->acc_empty[buf]);
         }
         if (etid == 0) tma_store_wait_all();
-        if (ok && e.part) {
+        if (!ok && lane == 0) atomicExch(&sh->failed, 1u);
+        __threadfence_block();
+        named_barrier(5, 256);
+        if (wg == 0 && e.part && sh->failed == 0) {
             // per-CTA record: the threads that share a channel quad are added in order
-            named_barrier(1, 128);
             float *mine = e.part + (size_t)blockIdx.x * 2 * e.n_cols;
             for (int gi = 0; gi < ng; gi++) {
                 const int col = col0 + gi * GW + jq * 4;
@@ -354,7 +362,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
             epilogue_publish<128>(e, reinterpret_cast<float *>(auxr), etid);
         }
-        if (!ok && lane == 0) atomicExch(&sh->failed, 1u);
     }
     tc_fence_before();
     __syncthreads();
@@ -602,7 +609,7 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         static bool attr_set = false;
         if (!attr_set) { cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024); attr_set = true; }
         dim3 grid((unsigned)ctas, (unsigned)s.n_tiles);
-        launch(ex, conv_tc_kernel, grid, kThreads, s.smem, map_a, map_b, map_o[0], map_o[1], map_x[0], map_x[1], p);
+        launch(ex, conv_tc_kernel, grid, epi_tma ? kThreadsTma : kThreads, s.smem, map_a, map_b, map_o[0], map_o[1], map_x[0], map_x[1], p);
         const double bytes = (double)gin.P() * cin * 2 + (double)g.P() * cout * (sign || req.bnbwd ? 8 : 4) + (double)cout * taps * cin * 2;
         ex.check(what, bytes, 2.0 * g.P() * cout * cin * ntap);
     }

@@ -1,8 +1,9 @@
 // The stem: a bare convolution of the 3-channel image (3x3 stride 1, or 7x7 stride 2), fp32 in both
 // precision modes, forward and weight gradient.  With so few input channels the contraction per
 // output pixel is short (K = k*k*3 = 27 or 147) and a tensor-core tile would be mostly padding, so
-// these are register-tiled CUDA-core kernels: the image patches of 64 output pixels are gathered
-// into shared memory once and every thread keeps a small block of the result in registers.
+// these are register-tiled CUDA-core kernels: the image patches of a tile of output pixels (128
+// forward, 64 for the weight gradient) are gathered into shared memory once and every thread keeps a
+// small block of the result in registers.
 //
 //   fprop: out[p, co]      = sum_{kh,kw,ci} img[p*s + (kh,kw) - pad, ci] * W[co, kh, kw, ci]
 //   wgrad: dW[co, kh,kw,ci] = sum_p g[p, co] * img[p*s + (kh,kw) - pad, ci]
@@ -182,12 +183,17 @@ __global__ void __launch_bounds__(256) stem_wgrad_kernel(const float *__restrict
         }
 }
 
+// dW[i] = sum of the per-CTA partials, one warp per element: lane l adds the partials l, l + 32, ... and the
+// lanes are combined by a shuffle tree, so the order of additions is fixed by `parts` alone
 __global__ void stem_sum_kernel(const float *__restrict__ part, size_t n, int parts, float *__restrict__ out) {
     pdl_enter();
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+    const int lane = threadIdx.x & 31;
+    const size_t warp = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5, n_warps = ((size_t)gridDim.x * blockDim.x) >> 5;
+    for (size_t i = warp; i < n; i += n_warps) {
         float s = 0.f;
-        for (int z = 0; z < parts; z++) s += part[(size_t)z * n + i];
-        out[i] = s;
+        for (int z = lane; z < parts; z += 32) s += part[(size_t)z * n + i];
+        for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if (lane == 0) out[i] = s;
     }
 }
 
@@ -255,7 +261,7 @@ bool stem_wgrad(Exec &ex, const float *img, const float *gout, Geom gi, const La
         else launch(ex, stem_wgrad_kernel<4, 4>, grid, 256, smem, img, gout, part, g, cop, kp, n_cg, G, S, n_chunks);
         ex.check("stem_wgrad", (double)g.N * g.H * g.W * g.Ci * 4 + (double)P * g.Co * 4, 2.0 * P * g.Co * g.K);
         const size_t n = (size_t)g.Co * g.K;
-        int sg = (int)((n + 255) / 256); if (sg > ex.ctx->sm_count * 4) sg = ex.ctx->sm_count * 4;
+        int sg = (int)((n + 7) / 8); if (sg > ex.ctx->sm_count * 8) sg = ex.ctx->sm_count * 8;      // eight warps per block
         launch(ex, stem_sum_kernel, sg, 256, 0, (const float *)part, n, grid, dW);
         ex.check("stem_sum", (double)n * 4 * (grid + 1));
     }

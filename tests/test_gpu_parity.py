@@ -326,6 +326,10 @@ def test_graph_replay_matches_eager(ctx):
     (16, 16, 32, 256, 3, 1, False),   # entry transition from a plain stem output
     (5, 6, 8, 16, 3, 2, True),        # ragged: falls back to the fp32 kernels
     (16, 8, 64, 128, 1, 2, True),     # 1x1 stride 2
+    (4, 16, 128, 256, 3, 2, True),    # 128 x 256 tiles in the forward (contraction 1152, 256 output channels)
+    (4, 8, 256, 512, 3, 2, True),     # ... and in the parity-class launches of the data gradient (1, 2, 2, 4 taps)
+    (4, 14, 64, 128, 3, 2, True),     # 14x14 -> 7x7: tiles of two whole images, class launches on a 7x7 grid
+    (2, 28, 128, 256, 3, 1, False),   # 28-wide rows: tiles of 112 pixels, wide tiles with statistics in the epilogue
 ])
 def test_stored_transition_layer(ctx, mode, N, H, cin, cout, k, stride, split):
     """BN-ReLU-conv with stride: forward and backward of one stored layer against the oracle."""

@@ -264,6 +264,32 @@ def run_ours(args, cfg):
     barrier()
     clocks = sampler.stop() if rank == 0 else None
 
+    # ---- the same network trained with ordinary backprop on stored activations (Section 3.2: the cost the
+    # reversible step trades storage for), graph replay, same timing rules; rank 0 only
+    stored = None
+    if rank == 0 and not args.no_stored:
+        srun = R.StackRunner(ctx, rcfg, mode=0, store_activations=True)
+        srun.load(inp["images"], inp["labels"], inp["params"])
+        sp0 = srun.params.clone()
+        for _ in range(args.warmup):
+            srun.params.copy_(sp0); srun.momentum.zero_()
+            sst = srun.step(want_logits=False)
+        torch.cuda.synchronize()
+        n_s = max(3, args.steps // 2)
+        sev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_s)]
+        for a, b in sev:
+            srun.params.copy_(sp0); srun.momentum.zero_()
+            flush.zero_()
+            a.record(stream)
+            sst = srun.step(want_logits=False)
+            b.record(stream)
+        torch.cuda.synchronize()
+        s_ms = sum(a.elapsed_time(b) for a, b in sev) / n_s
+        stored = dict(ms_per_step=s_ms, images_per_sec=rcfg.N / (s_ms * 1e-3), stored_activation_bytes=int(sst.stored_activation_bytes),
+                      workspace_bytes=int(sst.workspace_peak_bytes), flops_per_step=int(sst.flops_fwd + sst.flops_bwd), steps=n_s)
+        del srun
+        torch.cuda.empty_cache()
+
     # ---- per-kernel timing with CUDA events on the launching stream (same process, after the timed steps)
     B.revnet_profile_enable(ctx, True)
     psteps = 2
@@ -318,6 +344,10 @@ def run_ours(args, cfg):
                     activation_bytes=int(st.stored_activation_bytes), workspace_bytes=int(st.workspace_peak_bytes),
                     activation_mb_vs_units_per_stage=depth_sweep(ctx, rcfg),
                     flops_per_step=int(st.flops_fwd + st.flops_bwd), final_loss=final_loss, block_ms=block_ms)
+        if stored:
+            stored["reversible_over_stored_time"] = (dev_ms / args.steps) / stored["ms_per_step"]
+            stored["reversible_over_stored_bytes"] = int(st.stored_activation_bytes) / stored["stored_activation_bytes"]
+            line["stored_activation_step"] = stored
         if not args.no_cpu and world == 1:
             line["cpu_baseline"] = {k: v for k, v in cpu_baseline(cfg, min(cfg.N, args.ref_batch)).items() if k != "seconds_per_step"}
         print(json.dumps(line), flush=True)
@@ -334,6 +364,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--ref-batch", type=int, default=32, help="batch of the bounded CPU-oracle sample")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
+    ap.add_argument("--no-stored", action="store_true", help="skip the stored-activation comparison step")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     from paper_1707_04585_b200 import synthetic as syn

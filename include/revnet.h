@@ -202,6 +202,13 @@ typedef struct {
                                                        stream) and launches it on the caller's stream; later
                                                        calls with the same addresses only replay it.  Ignored
                                                        with verify_reconstruction or while profiling. */
+    int store_activations;                          /* 1: ordinary backprop for comparison (Section 3.2: the cost
+                                                       the method trades storage for).  Every unit keeps its inputs,
+                                                       its outputs and the internals of F and G from the forward
+                                                       pass in the workspace; the backward pass recomputes nothing
+                                                       (3N convolution cost instead of 4N) and storage grows with
+                                                       the number of units.  Same gradients as the reversible step.
+                                                       verify_reconstruction is ignored. */
 } revnet_stack_desc;
 
 typedef struct {

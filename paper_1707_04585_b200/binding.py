@@ -58,7 +58,7 @@ class StackDesc(C.Structure):
                 ("stem_k", C.c_int), ("stem_stride", C.c_int), ("stem_cout", C.c_int), ("maxpool", C.c_int),
                 ("n_stages", C.c_int), ("stage", StageDesc * MAX_STAGES), ("eps", C.c_float), ("mode", C.c_int),
                 ("state_frac_bits", C.c_int), ("lr", C.c_float), ("momentum", C.c_float), ("weight_decay", C.c_float),
-                ("verify_reconstruction", C.c_int), ("use_cuda_graph", C.c_int)]
+                ("verify_reconstruction", C.c_int), ("use_cuda_graph", C.c_int), ("store_activations", C.c_int)]
 
 
 class StepStats(C.Structure):
@@ -145,7 +145,7 @@ def block_desc(b: syn.BlockCfg, mode: int, state_frac_bits: int = 0) -> BlockDes
 
 
 def stack_desc(cfg: syn.StackCfg, mode: int, verify_reconstruction: bool = False, state_frac_bits: int = 0,
-               use_cuda_graph: bool = True) -> StackDesc:
+               use_cuda_graph: bool = True, store_activations: bool = False) -> StackDesc:
     d = StackDesc()
     d.N, d.img, d.in_ch, d.n_classes = cfg.N, cfg.img, cfg.in_ch, cfg.n_classes
     d.stem_k, d.stem_stride, d.stem_cout, d.maxpool = cfg.stem_k, cfg.stem_stride, cfg.stem_cout, int(cfg.maxpool)
@@ -156,6 +156,7 @@ def stack_desc(cfg: syn.StackCfg, mode: int, verify_reconstruction: bool = False
     d.lr, d.momentum, d.weight_decay = cfg.lr, cfg.momentum, cfg.weight_decay
     d.verify_reconstruction = int(verify_reconstruction)
     d.use_cuda_graph = int(use_cuda_graph)
+    d.store_activations = int(store_activations)
     return d
 
 

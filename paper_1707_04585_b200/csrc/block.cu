@@ -11,7 +11,6 @@
 // by the stand-alone reduction, in the forward and in the reversal alike, which keeps the
 // recomputed F and G bit-identical to the forward ones.
 #include "common.cuh"
-#include <stdlib.h>
 
 // dispatch: tensor-core kernels take the shapes they support in mode 0, the fp32 kernels the rest
 bool conv_fprop_tc(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign, Moments *stats);
@@ -140,8 +139,7 @@ void fn_backward(Exec &ex, Geom g, Pair u, const std::vector<Layer> &layers, FnS
     // last one produced).  One launch amortises set-up and split partials over the layers; the split
     // partials get a buffer of their own for that time.  Functions of more than four layers, shapes
     // the tensor-core kernel does not take, and profiling runs go layer by layer on the main stream.
-    static const bool no_side_env = getenv("REVNET_NO_SIDE") != nullptr;   // EXPERIMENT
-    bool side = !no_side_env && b16 && ex.use_side && L <= 4 && (ex.dry || (ex.ctx->side_stream && !ex.ctx->profiling));
+    bool side = b16 && ex.use_side && L <= 4 && (ex.dry || (ex.ctx->side_stream && !ex.ctx->profiling));
     size_t wg_need = 0;
     std::vector<const Layer *> lptr(L);
     std::vector<const void *> gq(L), aq(L);

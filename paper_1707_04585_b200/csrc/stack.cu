@@ -132,6 +132,14 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
     struct StageMom { Moments m1, m2, cat, in_cat, in2; };
     std::vector<StageMom> sm(S);
     bf16 *gcast = nullptr;          // bf16 copy of the gradient w.r.t. x2 / y2, handed from unit to unit
+    bf16 *gcast2 = nullptr;         // stored-activation step: bf16 copy of the gradient w.r.t. z1 inside a unit
+    // Stored-activation step (ordinary backprop): what every unit keeps from the forward pass.  The tensors
+    // live in the workspace arena, unit after unit, and are released in reverse order by the backward pass.
+    struct StoredUnit { size_t mark; float *x1, *x2, *y1, *y2; FnSaved svF, svG; Moments my1, my2; };
+    std::vector<std::vector<StoredUnit>> kept(S);
+    std::vector<Pair> stage_out(S);
+    const bool stored = d.store_activations != 0;
+    uint64_t kept_bytes = 0;        // what the units keep, summed over the network
     {
         size_t cmax = 0;
         for (int si = 0; si < S; si++) {
@@ -145,6 +153,7 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
             size_t e = (size_t)N * s.H * s.H * s.c; if (e > cmax) cmax = e;
         }
         if (ex.mode == 0) gcast = ex.ws.get<bf16>(cmax);
+        if (ex.mode == 0 && d.store_activations) gcast2 = ex.ws.get<bf16>(cmax);
     }
     float *recon = ex.ws.get<float>(REVNET_MAX_STAGES);
     if (recon_dev) *recon_dev = recon;
@@ -182,11 +191,37 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
             cudaMemcpyAsync(actf(s.off_v1), x1, b, cudaMemcpyDeviceToDevice, ex.stream);
             cudaMemcpyAsync(actf(s.off_v2), x2, b, cudaMemcpyDeviceToDevice, ex.stream);
         }
-        for (int u = 0; u < s.units; u++)
-            block_forward(ex, g, s.c, bind(s.F[u], params, grads), bind(s.G[u], params, grads), x1, x2, x1, x2,
-                          u == 0 ? &mo.in2 : &mo.m2, &mo.m1, &mo.m2);
-        mo.cat.valid = mo.m1.valid && mo.m2.valid;
-        prev = halves(x1, x2, s.c, q);
+        if (!stored) {
+            for (int u = 0; u < s.units; u++)
+                block_forward(ex, g, s.c, bind(s.F[u], params, grads), bind(s.G[u], params, grads), x1, x2, x1, x2,
+                              u == 0 ? &mo.in2 : &mo.m2, &mo.m1, &mo.m2);
+            mo.cat.valid = mo.m1.valid && mo.m2.valid;
+            prev = halves(x1, x2, s.c, q);
+        } else {
+            // every unit writes its outputs to fresh tensors and leaves the internals of F and G where they are
+            kept[si].resize(s.units);
+            float *c1 = x1, *c2 = x2;
+            const Moments *m_in = &mo.in2;
+            const size_t half = g.P() * s.c;
+            for (int u = 0; u < s.units; u++) {
+                StoredUnit &k = kept[si][u];
+                k.mark = ex.ws.mark();
+                k.x1 = c1; k.x2 = c2;
+                const bool last_unit = u == s.units - 1;
+                k.y1 = ex.ws.get<float>(half); k.y2 = ex.ws.get<float>(half);
+                // the statistics of the stage's final pair go where the next transition expects them
+                if (last_unit) { k.my1 = mo.m1; k.my2 = mo.m2; }
+                else { k.my1 = mom_alloc(ex, s.c); k.my2 = mom_alloc(ex, s.c); }
+                fn_forward(ex, g, single(c2, s.c, q), m_in, bind(s.F[u], params, grads), single(c1, s.c, q), single(k.y1, s.c, q), +1, &k.my1, &k.svF, false);
+                fn_forward(ex, g, single(k.y1, s.c, q), &k.my1, bind(s.G[u], params, grads), single(c2, s.c, q), single(k.y2, s.c, q), +1, &k.my2, &k.svG, false);
+                if (last_unit) { mo.m1 = k.my1; mo.m2 = k.my2; }
+                c1 = k.y1; c2 = k.y2; m_in = &k.my2;
+                kept_bytes += ex.ws.mark() - k.mark;
+            }
+            mo.cat.valid = mo.m1.valid && mo.m2.valid;
+            prev = halves(c1, c2, s.c, q);
+        }
+        stage_out[si] = prev;
         prevH = s.H;
     }
     StagePlan &top = pl->st[S - 1];
@@ -207,10 +242,22 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
         size_t half = g.P() * s.c;
         float *d1 = gbuf[gi], *d2 = gbuf[gi] + half;
         StageMom &mo = sm[si];
-        for (int u = s.units - 1; u >= 0; u--)
-            block_backward(ex, g, s.c, bind(s.F[u], params, grads), bind(s.G[u], params, grads), x1, x2, d1, d2, x1, x2, d1, d2,
-                           &mo.m1, &mo.m2, u == 0 ? &mo.in2 : nullptr, u == s.units - 1 ? nullptr : gcast, gcast);
-        if (d.verify_reconstruction) {
+        if (!stored) {
+            for (int u = s.units - 1; u >= 0; u--)
+                block_backward(ex, g, s.c, bind(s.F[u], params, grads), bind(s.G[u], params, grads), x1, x2, d1, d2, x1, x2, d1, d2,
+                               &mo.m1, &mo.m2, u == 0 ? &mo.in2 : nullptr, u == s.units - 1 ? nullptr : gcast, gcast);
+        } else {
+            // Algorithm 1 without its reconstruction lines: the gradient steps read what the forward pass kept
+            for (int u = s.units - 1; u >= 0; u--) {
+                StoredUnit &k = kept[si][u];
+                fn_backward(ex, g, single(k.y1, s.c, q), bind(s.G[u], params, grads), k.svG, single(d2, s.c), u == s.units - 1 ? nullptr : gcast,
+                            single(d1, s.c), single(d1, s.c), gcast2);
+                fn_backward(ex, g, single(k.x2, s.c, q), bind(s.F[u], params, grads), k.svF, single(d1, s.c), gcast2,
+                            single(d2, s.c), single(d2, s.c), gcast);
+                ex.ws.release(k.mark);
+            }
+        }
+        if (d.verify_reconstruction && !stored) {
             max_abs_diff(ex, x1, actf(s.off_v1), half, q, recon + si);
             max_abs_diff(ex, x2, actf(s.off_v2), half, q, recon + si);
         }
@@ -219,7 +266,7 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
             Pair tin; int tH; Pair gout;
             if (si > 0) {
                 StagePlan &p = pl->st[si - 1];
-                tin = halves(actf(p.off_x1), actf(p.off_x2), p.c, q); tH = p.H;
+                tin = stored ? stage_out[si - 1] : halves(actf(p.off_x1), actf(p.off_x2), p.c, q); tH = p.H;
                 size_t ph = (size_t)N * p.H * p.H * p.c;
                 gout = halves(gbuf[gi ^ 1], gbuf[gi ^ 1] + ph, p.c);
             } else {
@@ -257,7 +304,7 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
     sgd_update(ex, params, grads, mom, pl->n_params, seg_end, seg_decay, (int)nseg, d.lr, d.momentum, d.weight_decay);
 
     if (stats) {
-        stats->stored_activation_bytes = pl->stored_bytes;
+        stats->stored_activation_bytes = pl->stored_bytes + kept_bytes;
         stats->workspace_peak_bytes = ex.ws.peak;
         stats->flops_fwd = flops_fwd;
         stats->flops_bwd = ex.flops - flops_fwd;

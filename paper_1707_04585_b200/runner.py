@@ -82,11 +82,11 @@ class BlockRunner:
 
 class StackRunner:
     def __init__(self, ctx: B.Context, cfg: syn.StackCfg, mode: int, verify_reconstruction: bool = False,
-                 frac_bits: int = None, use_cuda_graph: bool = True):
+                 frac_bits: int = None, use_cuda_graph: bool = True, store_activations: bool = False):
         self.ctx, self.cfg, self.mode = ctx, cfg, mode
         self.frac = DEFAULT_FRAC_BITS[mode] if frac_bits is None else frac_bits
         self.specs = syn.param_specs(cfg)
-        self.desc = B.stack_desc(cfg, mode, verify_reconstruction, self.frac, use_cuda_graph)
+        self.desc = B.stack_desc(cfg, mode, verify_reconstruction, self.frac, use_cuda_graph, store_activations)
         self.plan = B.revnet_stack_plan(ctx, self.desc)
         n = self.plan.param_count
         assert n == sum(int(np.prod(s)) for _, s, _ in self.specs)

@@ -1,0 +1,91 @@
+"""The stored-activation train step (store_activations = 1): ordinary backprop on what the forward
+pass kept, the baseline the reversible step is traded against (Section 3.2).
+
+Both steps compute the same gradients (Section 3: reversing the units changes where the activations
+come from, not what is differentiated), so the stored step is checked against the reversible one
+run on the same inputs -- bit for bit in the bf16 mode with its fixed-point state, where the
+reversal reproduces every tensor of the forward pass exactly -- and, in strict mode, against the
+oracle's stored-activation flavour.  Its storage must grow with the number of units while the
+reversible step's does not.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import revnet as orc
+from paper_1707_04585_b200 import binding as B
+from paper_1707_04585_b200 import runner as R
+from paper_1707_04585_b200 import synthetic as syn
+from tests import helpers as hp
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    c = B.Context(0)
+    yield c
+    B.revnet_check_device(c)
+    c.close()
+
+
+def both_steps(ctx, cfg, mode, graph):
+    inp = syn.make_stack_inputs(cfg, affine_jitter=True)
+    out = []
+    for stored in (False, True):
+        r = R.StackRunner(ctx, cfg, mode, use_cuda_graph=graph, store_activations=stored)
+        r.load(inp["images"], inp["labels"], inp["params"])
+        st = r.step()
+        if graph:                       # second call replays the captured graph from the same state
+            r.load(inp["images"], inp["labels"], inp["params"])
+            st = r.step()
+        out.append((r.results(), st))
+        B.revnet_check_device(ctx)
+    return inp, out
+
+
+@pytest.mark.parametrize("graph", [False, True])
+@pytest.mark.parametrize("kind,maxpool", [("basic", False), ("bottleneck", False), ("bottleneck", True)])
+def test_stored_step_equals_reversible_step_bitwise_in_bf16_mode(ctx, kind, maxpool, graph):
+    cfg = hp.tiny_stack(kind, maxpool, N=6, units=3)
+    _, ((rev, srev), (sto, ssto)) = both_steps(ctx, cfg, 0, graph)
+    assert np.array_equal(rev["logits"], sto["logits"]) and rev["loss"] == sto["loss"]
+    for k in rev["grads"]:
+        assert np.array_equal(rev["grads"][k], sto["grads"][k]), k
+        assert np.array_equal(rev["params"][k], sto["params"][k]), k
+    # the stored step skips the recomputation: three conv passes per reversible layer instead of four
+    assert ssto.flops_fwd == srev.flops_fwd and ssto.flops_bwd < srev.flops_bwd
+    assert ssto.stored_activation_bytes > srev.stored_activation_bytes
+
+
+@pytest.mark.parametrize("kind,maxpool", [("basic", False), ("bottleneck", True)])
+def test_stored_step_strict_mode_against_oracle_and_reversible(ctx, kind, maxpool):
+    cfg = hp.tiny_stack(kind, maxpool, N=6, units=2)
+    inp, ((rev, _), (sto, _)) = both_steps(ctx, cfg, 1, False)
+    net = hp.oracle_net(cfg, inp["params"])
+    o = orc.stack_train_grads(net, inp["images"], inp["labels"], "stored")
+    assert hp.rel_l2(sto["logits"], o["logits"]) <= 1e-4
+    for k in o["grads"]:
+        assert hp.rel_l2(sto["grads"][k], o["grads"][k]) <= 1e-3, k
+        assert hp.rel_l2(sto["grads"][k], rev["grads"][k]) <= 1e-3, k
+
+
+def test_stored_step_at_benchmark_width_and_storage_growth(ctx):
+    """RevNet-38 widths at batch 16: gradients equal the reversible step's; kept bytes grow linearly in depth."""
+    base = syn.shrink(syn.stack_config("revnet38"), N=16)
+    _, ((rev, srev), (sto, ssto)) = both_steps(ctx, base, 0, True)
+    for k in rev["grads"]:
+        assert np.array_equal(rev["grads"][k], sto["grads"][k]), k
+    kept = {}
+    for units in (1, 2, 4):
+        cfg = syn.shrink(base, units=units)
+        sizes = []
+        for stored in (False, True):
+            r = R.StackRunner(ctx, cfg, 0, store_activations=stored)
+            inp = syn.make_stack_inputs(cfg)
+            r.load(inp["images"], inp["labels"], inp["params"])
+            sizes.append(int(r.step().stored_activation_bytes))
+            torch.cuda.synchronize()
+        kept[units] = sizes
+    assert kept[1][0] == kept[2][0] == kept[4][0]                       # reversible: flat in depth
+    assert kept[4][1] - kept[2][1] == 2 * (kept[2][1] - kept[1][1]) > 0   # stored: the same amount per unit

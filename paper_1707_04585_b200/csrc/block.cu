@@ -15,7 +15,7 @@
 // dispatch: tensor-core kernels take the shapes they support in mode 0, the fp32 kernels the rest
 bool conv_fprop_tc(Exec &ex, const void *a, Geom gi, const Layer &L, Pair out, Pair partner, int sign, Moments *stats);
 bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, const BnBwdReq *bb);
-bool conv_dgrad_tc_s2(Exec &ex, const void *g, Geom gi, const Layer &L, float *da);
+bool conv_dgrad_tc_s2(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, const BnBwdReq *bb, bool *fused);
 bool conv_wgrad_tc(Exec &ex, const void *g, const void *a, Geom gi, const Layer &L, float *dW, float *scratch, size_t *need);
 bool conv_wgrad_tc_batch(Exec &ex, int n, const void *const *gq, const void *const *a, const Geom *gi, const Layer *const *L,
                          float *scratch, size_t *need);
@@ -36,9 +36,9 @@ static bool conv_dgrad(Exec &ex, const void *g, Geom gi, const Layer &L, float *
     const bool b16 = ex.mode == 0;
     if (b16 && L.stride == 1 && conv_dgrad_fused(ex, g, gi, L, da, bb)) return bb != nullptr;
     if (b16 && L.stride == 1 && conv_dgrad_tc(ex, g, gi, L, da, bb)) return bb != nullptr;
-    // stride 2 on the tensor cores: one launch per parity class of the input pixels (the BN-backward sums then
-    // take their own pass)
-    if (b16 && L.stride == 2 && L.cout % 8 == 0 && conv_dgrad_tc_s2(ex, g, gi, L, da)) return false;
+    // stride 2 on the tensor cores: the CTAs of one launch split into the parity classes of the input pixels
+    bool fused = false;
+    if (b16 && L.stride == 2 && L.cout % 8 == 0 && conv_dgrad_tc_s2(ex, g, gi, L, da, bb, &fused)) return fused;
     if (b16 && L.stride == 2 && gi.H % 2 == 0 && gi.W % 2 == 0 && L.cout % 8 == 0) {
         // shapes the class launches do not take: spread g over the input grid (zeros between samples); the data gradient is then the
         // stride-1 one:  da[y,x] = sum_taps g_up[y + pad - kh, x + pad - kw] W[.,kh,kw,.]

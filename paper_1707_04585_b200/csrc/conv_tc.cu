@@ -51,9 +51,12 @@ struct TcParams {
     // the taps this launch sums: offset of the operand box in rows / columns of the operand tensor, and the tap's
     // place in the weight pack.  A plain convolution lists all k*k taps; one parity class of a stride-2 data
     // gradient lists the one, two or four taps that reach its output pixels.
-    int ntap;
-    signed char tdy[9], tdx[9], tid[9];
-    int ostride, oy, ox;    // epi_tma: output pixel = tile pixel * ostride + (oy, ox)
+    // A launch with n_cls classes walks n_cls * n_px_tiles tiles: tile t belongs to class t / n_px_tiles (a plain
+    // convolution has one class).  CTAs stride over that list, so every CTA gets its share of the short and long classes.
+    int n_cls;
+    int ntap[4];
+    signed char tdy[4][9], tdx[4][9], tid[4][9];
+    int ostride, oy[4], ox[4];    // epi_tma: output pixel = tile pixel * ostride + (oy, ox)
 };
 
 struct __align__(8) TcShared {
@@ -154,7 +157,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     TcShared *sh = p.epi_tma ? (TcShared *)(gsums + ng * 128 * 8) : (TcShared *)((uint8_t *)estage + kEpiStageBytes + kEpiSumFloats * 4);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int iters = p.ntap * p.chunks;
+    const int n_vt = p.n_cls * p.g.n_px_tiles;     // tiles of all classes
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < 2 * p.BN) tmem_cols <<= 1;
 
@@ -180,17 +183,19 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (lane == 0) {
             uint32_t itg = 0;
             bool ok = true;
-            for (int t = blockIdx.x; t < p.g.n_px_tiles && ok; t += gridDim.x) {
+            for (int t = blockIdx.x; t < n_vt && ok; t += gridDim.x) {
                 int n0, h0;
-                tile_origin(p.g, t, n0, h0);
+                const int cls = t / p.g.n_px_tiles;
+                tile_origin(p.g, t - cls * p.g.n_px_tiles, n0, h0);
+                const int iters = p.ntap[cls] * p.chunks;
                 for (int it = 0; it < iters; it++, itg++) {
                     const int s = itg % p.stages; const uint32_t round = itg / p.stages;
                     if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
                     const int ti = it / p.chunks, ch = it - ti * p.chunks;
                     uint8_t *sa = tiles + s * stage_bytes;
                     mbar_expect_tx(&sh->full[s], (uint32_t)(a_bytes + b_bytes));
-                    tma_load_4d(sa, &map_a, &sh->full[s], ch * p.KC, p.tdx[ti], h0 * p.stride + p.tdy[ti], n0);
-                    tma_load_2d(sa + b_off, &map_b, &sh->full[s], p.tid[ti] * p.cin_pad + ch * p.KC, col0);
+                    tma_load_4d(sa, &map_a, &sh->full[s], ch * p.KC, p.tdx[cls][ti], h0 * p.stride + p.tdy[cls][ti], n0);
+                    tma_load_2d(sa + b_off, &map_b, &sh->full[s], p.tid[cls][ti] * p.cin_pad + ch * p.KC, col0);
                 }
             }
         }
@@ -201,8 +206,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint32_t itg = 0;
             bool ok = true;
             int ti = 0;
-            for (int t = blockIdx.x; t < p.g.n_px_tiles && ok; t += gridDim.x, ti++) {
+            for (int t = blockIdx.x; t < n_vt && ok; t += gridDim.x, ti++) {
                 const int buf = ti & 1; const uint32_t use = ti >> 1;
+                const int iters = p.ntap[t / p.g.n_px_tiles] * p.chunks;
                 if (use > 0 && !mbar_wait(&sh->acc_empty[buf], (use - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
                 tc_fence_after();
                 const uint32_t acc = tmem_d + (uint32_t)(buf * p.BN);
@@ -263,28 +269,27 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         auto aux_map = [&](int col) { return (p.split_x && col >= p.split_x) ? &map_x1 : &map_x0; };
         auto col_out = [&](int col) { return (p.split_o && col >= p.split_o) ? col - p.split_o : col; };
         auto col_aux = [&](int col) { return (p.split_x && col >= p.split_x) ? col - p.split_x : col; };
-        auto load_aux = [&](int gi, int n0, int h0) {        // one thread
+        auto load_aux = [&](int gi, int t) {                 // one thread; t: tile in the list of all classes
             const int col = col0 + gi * GW;
             if (col >= e.n_cols) return;
-            mbar_expect_tx(&sh->aux_full[gi], aux_tx);
-            tma_load_4d(auxr + gi * p.group_bytes, aux_map(col), &sh->aux_full[gi], col_aux(col), p.ox, h0 * p.ostride + p.oy, n0);
-        };
-        if (etid == 0 && p.need_aux && (int)blockIdx.x < p.g.n_px_tiles) {
             int n0, h0;
-            tile_origin(p.g, blockIdx.x, n0, h0);
-            for (int gi = wg; gi < ng; gi += 2) load_aux(gi, n0, h0);
-        }
+            const int cls = t / p.g.n_px_tiles;
+            tile_origin(p.g, t - cls * p.g.n_px_tiles, n0, h0);
+            mbar_expect_tx(&sh->aux_full[gi], aux_tx);
+            tma_load_4d(auxr + gi * p.group_bytes, aux_map(col), &sh->aux_full[gi], col_aux(col), p.ox[cls], h0 * p.ostride + p.oy[cls], n0);
+        };
+        if (etid == 0 && p.need_aux && (int)blockIdx.x < n_vt)
+            for (int gi = wg; gi < ng; gi += 2) load_aux(gi, blockIdx.x);
         named_barrier(5, 256);
         bool ok = true;
         int ti = 0;
         uint8_t *ob = outr + wg * p.group_bytes;
-        for (int t = blockIdx.x; t < p.g.n_px_tiles; t += gridDim.x, ti++) {
+        for (int t = blockIdx.x; t < n_vt; t += gridDim.x, ti++) {
             const int buf = ti & 1; const uint32_t use = ti >> 1;
             int n0, h0;
-            tile_origin(p.g, t, n0, h0);
+            const int cls = t / p.g.n_px_tiles;
+            tile_origin(p.g, t - cls * p.g.n_px_tiles, n0, h0);
             const int tn = t + (int)gridDim.x;
-            int nn0 = 0, nh0 = 0;
-            if (tn < p.g.n_px_tiles) tile_origin(p.g, tn, nn0, nh0);
             const int valid_px = p.g.BIMG > 1 ? (p.g.N - n0 < p.g.BIMG ? p.g.N - n0 : p.g.BIMG) * p.g.BH * p.g.W
                                               : (p.g.H - h0 < p.g.BH ? p.g.H - h0 : p.g.BH) * p.g.W;
             if (etid == 0) ok = mbar_wait(&sh->acc_full[buf], use & 1) && sh->failed == 0;     // one thread polls, the rest block
@@ -315,7 +320,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 fence_proxy_async();
                 named_barrier(bar_a, 128);
                 if (etid == 0 && live) {
-                    tma_store_4d(out_map(col), ob, col_out(col), p.ox, h0 * p.ostride + p.oy, n0);
+                    tma_store_4d(out_map(col), ob, col_out(col), p.ox[cls], h0 * p.ostride + p.oy[cls], n0);
                     tma_store_commit();
                 }
                 if (e.part && live && col + jq * 4 < e.n_cols) {
@@ -332,7 +337,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     slot[0] = make_float4(acc[0], acc[1], acc[2], acc[3]); slot[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
                 }
                 named_barrier(bar_a, 128);                 // the partner group and the output slot have been read
-                if (etid == 0 && p.need_aux && tn < p.g.n_px_tiles) load_aux(gi, nn0, nh0);
+                if (etid == 0 && p.need_aux && tn < n_vt) load_aux(gi, tn);
             }
             if (!ok) break;
             // this warp group has drained its columns of the accumulator (the other group arrives for its own)
@@ -481,42 +486,52 @@ bool tc_shape(Geom g, int cin, int cout, int k, int stride, TcShape &s, bool wid
 }
 
 // act: bf16 [N,H,W,cin]; Wsrc: fp32 weights; transposed selects the dgrad pack
-// s2cls (optional): {py, px}, one parity class of the data gradient of a 3x3 stride-2 layer.  `act` is then the
-// upstream gradient on the layer's output grid (gin), `out` the gradient on the input grid (twice as fine): the
-// launch fills the pixels (2i + py, 2j + px) from the taps that reach them,
+// s2: the data gradient of a 3x3 stride-2 layer.  `act` is then the upstream gradient on the layer's output grid
+// (gin), `out` the gradient on the input grid (twice as fine), and the launch's tile list runs over the four parity classes of the
+// input pixels: class (py, px) fills the pixels (2i + py, 2j + px) from the taps that reach them,
 //   da[2i+py, 2j+px] = sum over th in T(py), tw in T(px) of g[i + th/2, j + tw/2] Wd[th, tw],  T(0) = {1}, T(1) = {0, 2}
 // (Wd the mirrored, transposed pack), so the four classes together cost the nine taps once per four pixels.
 bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin, int cout, int k, int stride,
                  const float *Wsrc, const bf16 *prepacked, bool transposed, Pair out, Pair partner, int sign, EpiReq req,
-                 const int *s2cls = nullptr) {
+                 bool s2 = false) {
     TcShape s;
     if (stride == 2 && (gin.H % 2 || gin.W % 2)) return false;
-    if (s2cls && (stride != 1 || k != 3 || !transposed || sign || req.stats || req.bnbwd || out.c1)) return false;
+    if (s2 && (stride != 1 || k != 3 || !transposed || sign || req.stats || out.c1)) return false;
     const Geom g{gin.N, conv_out(gin.H, k, stride), conv_out(gin.W, k, stride)};   // geometry of the tiles
     if (!tc_shape(g, cin, cout, k, stride, s)) return false;
     const int taps = k * k;
     if (!ex.dry && !encoder(ex.ctx)) return false;
-    // the taps of this launch
-    int ntap = 0;
-    signed char tdy[9], tdx[9], tid[9];
-    for (int th = 0; th < k; th++)
-        for (int tw = 0; tw < k; tw++) {
-            if (s2cls && ((th & 1) == s2cls[0] || (tw & 1) == s2cls[1])) continue;
-            tdy[ntap] = (signed char)(s2cls ? th / 2 : th - k / 2); tdx[ntap] = (signed char)(s2cls ? tw / 2 : tw - k / 2);
-            tid[ntap] = (signed char)(th * k + tw); ntap++;
-        }
-    ex.flops += 2ull * g.P() * cout * cin * ntap;
+    // the taps of every class of this launch
+    const int n_cls = s2 ? 4 : 1;
+    int ntap[4] = {0, 0, 0, 0}, ntap_all = 0;
+    signed char tdy[4][9], tdx[4][9], tid[4][9];
+    memset(tdy, 0, sizeof tdy); memset(tdx, 0, sizeof tdx); memset(tid, 0, sizeof tid);
+    for (int c = 0; c < n_cls; c++) {
+        const int py = c >> 1, px = c & 1;
+        for (int th = 0; th < k; th++)
+            for (int tw = 0; tw < k; tw++) {
+                if (s2 && ((th & 1) == py || (tw & 1) == px)) continue;
+                const int i = ntap[c]++;
+                tdy[c][i] = (signed char)(s2 ? th / 2 : th - k / 2); tdx[c][i] = (signed char)(s2 ? tw / 2 : tw - k / 2);
+                tid[c][i] = (signed char)(th * k + tw);
+            }
+        ntap_all += ntap[c];
+    }
     // epilogue through TMA where a column group never straddles the halves of a channel-split tensor
     const bool need_aux = sign != 0 || req.bnbwd != nullptr;
     const Pair auxp = req.bnbwd ? req.bnbwd->t : partner;
+    const int ntap_max = s2 ? 4 : taps;
     // arithmetic-bound layers without a partner tile (transitions, their data gradients): 128 x 256 tiles
-    if (!need_aux && !(out.c1 && out.c0 % 32) && (long long)ntap * cin >= 1024 && cout >= 256 && cout % 32 == 0) tc_shape(g, cin, cout, k, stride, s, true);
+    if (!need_aux && !(out.c1 && out.c0 % 32) && (long long)ntap_max * cin >= 1024 && cout >= 256 && cout % 32 == 0) tc_shape(g, cin, cout, k, stride, s, true);
     // rows of the weight pack (a multiple of its 128-row blocks, whatever the N tile); TMA fills rows beyond with zeros
     const int rp16 = round_up(cout, 16), rows_pad = rp16 <= 128 ? rp16 : round_up(rp16, 128);
-    const int GW = s.BN % 32 == 0 ? 32 : 16, ng = s.BN / GW, group_bytes = (128 * GW * 4 + 1023) & ~1023;
+    // column groups of 32 floats, or of 16 where the N tile or the halves of a channel-split tensor ask for it
+    int GW = s.BN % 32 == 0 ? 32 : 16;
+    if (GW == 32 && s.BN <= 128 && ((out.c1 && out.c0 % 32) || (need_aux && auxp.c1 && auxp.c0 % 32))) GW = 16;
+    const int ng = s.BN / GW, group_bytes = (128 * GW * 4 + 1023) & ~1023;
     bool epi_tma = !(out.c1 && out.c0 % GW) && !(need_aux && auxp.c1 && auxp.c0 % GW) && ng <= 8;
-    const int ostride = s2cls ? 2 : 1;
-    if (s2cls && (!epi_tma || g.W * 2 > 256 || s.g.BH * 2 > 256)) return false;
+    const int ostride = s2 ? 2 : 1;
+    if (s2 && (!epi_tma || g.W * 2 > 256 || s.g.BH * 2 > 256)) return false;
     int stages = 4;
     if (epi_tma) {
         stages = kStages;
@@ -528,10 +543,11 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
             epi_tma = false; stages = 4;
         } else s.smem = smem_of(stages);
     }
-    if ((s2cls || s.BN == 256) && !epi_tma) return false;
+    if ((s2 || s.BN == 256) && !epi_tma) return false;
+    ex.flops += 2ull * g.P() * cout * cin * ntap_all;
     int occ = (227 * 1024) / s.smem; if (occ > 2) occ = 2; if (occ < 1) occ = 1;
     int ctas = ex.ctx->sm_count * occ / s.n_tiles; if (ctas < 1) ctas = 1;
-    if (ctas > s.g.n_px_tiles) ctas = s.g.n_px_tiles;
+    if (ctas > s.g.n_px_tiles * n_cls) ctas = s.g.n_px_tiles * n_cls;
     size_t m = ex.ws.mark();
     bf16 *wp = prepacked ? const_cast<bf16 *>(prepacked) : ex.ws.get<bf16>((size_t)rows_pad * taps * s.cin_pad);
     const bool reduce = req.stats || req.bnbwd;
@@ -594,8 +610,9 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         TcParams p;
         p.stages = stages; p.epi_tma = epi_tma ? 1 : 0; p.GW = GW; p.group_bytes = group_bytes; p.need_aux = need_aux ? 1 : 0;
         p.split_o = out.c1 ? out.c0 : 0; p.split_x = (need_aux && auxp.c1) ? auxp.c0 : 0;
-        p.ntap = ntap; memcpy(p.tdy, tdy, 9); memcpy(p.tdx, tdx, 9); memcpy(p.tid, tid, 9);
-        p.ostride = ostride; p.oy = s2cls ? s2cls[0] : 0; p.ox = s2cls ? s2cls[1] : 0;
+        memcpy(p.ntap, ntap, sizeof ntap); memcpy(p.tdy, tdy, sizeof tdy); memcpy(p.tdx, tdx, sizeof tdx); memcpy(p.tid, tid, sizeof tid);
+        p.ostride = ostride; p.n_cls = n_cls;
+        for (int c = 0; c < 4; c++) { p.oy[c] = s2 ? c >> 1 : 0; p.ox[c] = s2 ? c & 1 : 0; }
         p.taps = taps; p.k = k; p.chunks = s.chunks; p.KC = s.KC; p.cin_pad = s.cin_pad; p.BN = s.BN; p.stride = stride; p.g = s.g;
         p.status = ex.ctx->dev_status;
         EpiArgs &e = p.epi;
@@ -603,7 +620,7 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         e.mode = req.bnbwd ? EPI_BNBWD : (sign ? EPI_COUPLE : EPI_PLAIN);
         e.out = out; e.partner = partner; e.sign = sign; e.n_cols = cout; e.pitch = kEpiPitch;
         e.part = part; e.counter = reduce ? ex.ctx->counter() : nullptr;
-        e.inv_count = 1.0 / (double)g.P(); e.eps = ex.eps;
+        e.inv_count = 1.0 / ((double)g.P() * ostride * ostride); e.eps = ex.eps;     // pixels of the output grid
         if (req.stats) { e.mean = req.stats->mean; e.rstd = req.stats->rstd; }
         if (req.bnbwd) { e.t = req.bnbwd->t; e.bn = req.bnbwd->bn; e.dgamma = req.bnbwd->dgamma; e.dbeta = req.bnbwd->dbeta; e.coef = req.bnbwd->coef; }
         static bool attr_set = false;
@@ -611,7 +628,7 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         dim3 grid((unsigned)ctas, (unsigned)s.n_tiles);
         launch(ex, conv_tc_kernel, grid, epi_tma ? kThreadsTma : kThreads, s.smem, map_a, map_b, map_o[0], map_o[1], map_x[0], map_x[1], p);
         const double bytes = (double)gin.P() * cin * 2 + (double)g.P() * cout * (sign || req.bnbwd ? 8 : 4) + (double)cout * taps * cin * 2;
-        ex.check(what, bytes, 2.0 * g.P() * cout * cin * ntap);
+        ex.check(what, bytes, 2.0 * g.P() * cout * cin * ntap_all);
     }
     ex.ws.release(m);
     return true;
@@ -862,17 +879,17 @@ bool conv_dgrad_tc(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, 
 }
 
 
-// Data gradient of a 3x3 stride-2 layer: four launches, one per parity class of the input pixels (see
-// run_conv_tc).  g: bf16 [N, H/2, W/2, cout]; da: fp32 [N, H, W, cin].
-bool conv_dgrad_tc_s2(Exec &ex, const void *g, Geom gi, const Layer &L, float *da) {
+// Data gradient of a 3x3 stride-2 layer: one launch whose tile list runs over the four parity classes of the input
+// pixels (see run_conv_tc).  g: bf16 [N, H/2, W/2, cout]; da: fp32 [N, H, W, cin]; bb: BN-backward sums to fuse.
+// Large layers (those that get 128 x 256 tiles when no partner tile has to fit beside the operand ring) leave the
+// sums to their own pass instead: *fused tells which.
+bool conv_dgrad_tc_s2(Exec &ex, const void *g, Geom gi, const Layer &L, float *da, const BnBwdReq *bb, bool *fused) {
     if (L.stride != 2 || L.k != 3 || gi.H % 2 || gi.W % 2) return false;
     const Geom go{gi.N, gi.H / 2, gi.W / 2};
-    for (int cls = 0; cls < 4; cls++) {
-        const int pc[2] = {cls >> 1, cls & 1};
-        if (!run_conv_tc(ex, "conv_dgrad_tc", g, go, L.cout, L.cin, 3, 1, L.W, L.Wp_dgrad, true, single(da, L.cin), Pair{}, 0, EpiReq{}, pc))
-            return false;     // refused before anything was launched: every class takes the same decision
-    }
-    return true;
+    const bool wide = 4ll * L.cout >= 1024 && L.cin >= 256 && L.cin % 32 == 0;
+    EpiReq req; req.bnbwd = wide ? nullptr : bb;
+    *fused = req.bnbwd != nullptr;
+    return run_conv_tc(ex, "conv_dgrad_tc", g, go, L.cout, L.cin, 3, 1, L.W, L.Wp_dgrad, true, single(da, L.cin), Pair{}, 0, req, true);
 }
 
 constexpr int kWgSmemMax = 224 * 1024;

@@ -89,3 +89,27 @@ def test_stored_step_at_benchmark_width_and_storage_growth(ctx):
         kept[units] = sizes
     assert kept[1][0] == kept[2][0] == kept[4][0]                       # reversible: flat in depth
     assert kept[4][1] - kept[2][1] == 2 * (kept[2][1] - kept[1][1]) > 0   # stored: the same amount per unit
+
+
+@pytest.mark.parametrize("name", ["revnet110", "revnet164"])
+def test_stored_step_equals_reversible_step_at_full_size(ctx, name):
+    """The deep configurations at full batch, graph replay (the benchmark's launch configuration): both steps end
+    with the same bits in every gradient and updated weight, the stored one with less backward work."""
+    cfg = syn.stack_config(name)
+    inp = syn.make_stack_inputs(cfg)
+    flat = []
+    stats = []
+    for stored in (False, True):
+        r = R.StackRunner(ctx, cfg, 0, store_activations=stored)
+        r.load(inp["images"], inp["labels"], inp["params"])
+        r.step(want_logits=False)                      # captures the graph
+        r.load(inp["images"], inp["labels"], inp["params"])
+        stats.append(r.step(want_logits=False))        # replays it from the same state
+        torch.cuda.synchronize()
+        flat.append((r.grads.clone(), r.params.clone(), float(r.loss.item())))
+        B.revnet_check_device(ctx)
+        del r
+        torch.cuda.empty_cache()
+    assert torch.equal(flat[0][0], flat[1][0]) and torch.equal(flat[0][1], flat[1][1]) and flat[0][2] == flat[1][2]
+    assert np.isfinite(flat[0][2])
+    assert stats[1].flops_bwd < stats[0].flops_bwd and stats[1].stored_activation_bytes > 5 * stats[0].stored_activation_bytes

@@ -225,13 +225,15 @@ def run_ours(args, cfg):
         run.params.copy_(params0)
         run.momentum.zero_()
 
+    # the clock sampler runs from the warm-up to the end of the end-to-end loop: nvidia-smi needs about a second
+    # to deliver its first line, longer than the timed steps of the small workloads take
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
     for _ in range(args.warmup):
         reset()
         st = run.step(want_logits=False)
     barrier()
-    sampler = ClockSampler(local)
-    if rank == 0:
-        sampler.start()
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     for a, b in ev:
         reset()
@@ -358,7 +360,7 @@ def run_ours(args, cfg):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--config", default="revnet38")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])

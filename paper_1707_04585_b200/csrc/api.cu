@@ -18,6 +18,9 @@ extern "C" int revnet_create(revnet_ctx **out, int device) {
             cudaMalloc(&c->dev_status, 1024) != cudaSuccess || cudaMemset(c->dev_status, 0, 1024) != cudaSuccess ||
             cudaStreamCreateWithFlags(&c->capture_stream, cudaStreamNonBlocking) != cudaSuccess ||
             cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaStreamCreateWithFlags(&c->recon_stream, cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_rfork, cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_rjoin, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) != cudaSuccess) {
             cudaGetLastError();
@@ -37,6 +40,9 @@ extern "C" int revnet_destroy(revnet_ctx *ctx) {
     if (ctx->dev_status) cudaFree(ctx->dev_status);
     if (ctx->capture_stream) cudaStreamDestroy(ctx->capture_stream);
     if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);
+    if (ctx->recon_stream) cudaStreamDestroy(ctx->recon_stream);
+    if (ctx->ev_rfork) cudaEventDestroy(ctx->ev_rfork);
+    if (ctx->ev_rjoin) cudaEventDestroy(ctx->ev_rjoin);
     if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
     if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
     delete ctx;

@@ -196,22 +196,45 @@ void block_forward(Exec &ex, Geom g, int c, const std::vector<Layer> &F, const s
 void block_backward(Exec &ex, Geom g, int c, const std::vector<Layer> &F, const std::vector<Layer> &G,
                     const float *y1, const float *y2, const float *dy1, const float *dy2,
                     float *x1, float *x2, float *dx1, float *dx2,
-                    Moments *m1, Moments *m2, const Moments *m2_use, const bf16 *dy2_cast, bf16 *dx2_cast) {
-    FnSaved sv;
+                    Moments *m1, Moments *m2, const Moments *m2_use, const bf16 *dy2_cast, bf16 *dx2_cast,
+                    Moments *m1_out, bool overlap) {
+    FnSaved svG, svF;
     const float q = ex.q;   // format of the coupling state; gradients are always float
     size_t m0 = ex.ws.mark();
+    if (!m1_out) m1_out = m1;
+    // F may be recomputed beside G's gradient steps only if it leaves y1 and its statistics alone
+    overlap = overlap && x1 != y1 && m1_out != m1 && (ex.dry || (ex.ctx->recon_stream && !ex.ctx->profiling));
     // bf16 copy of dz1 for F's backward (the BN-backward apply that produces dz1 writes it)
     bf16 *dz1_cast = ex.mode == 0 ? ex.ws.get<bf16>(g.P() * c) : nullptr;
     size_t m = ex.ws.mark();
     // x2 = y2 - G(z1), z1 = y1
-    fn_forward(ex, g, single((float *)y1, c, q), m1, G, single((float *)y2, c, q), single(x2, c, q), -1, m2, &sv, false);
-    // dz1 = dy1 + (dG/dz1)^T dy2 ; dW_G
-    fn_backward(ex, g, single((float *)y1, c, q), G, sv, single((float *)dy2, c), dy2_cast, single((float *)dy1, c), single(dx1, c), dz1_cast);
-    ex.ws.release(m);
-    // x1 = z1 - F(x2)
+    fn_forward(ex, g, single((float *)y1, c, q), m1, G, single((float *)y2, c, q), single(x2, c, q), -1, m2, &svG, false);
     const Moments *mf = (m2_use && m2_use->valid) ? m2_use : m2;
-    fn_forward(ex, g, single(x2, c, q), mf, F, single((float *)y1, c, q), single(x1, c, q), -1, m1, &sv, false);
+    if (!overlap) {
+        // dz1 = dy1 + (dG/dz1)^T dy2 ; dW_G
+        fn_backward(ex, g, single((float *)y1, c, q), G, svG, single((float *)dy2, c), dy2_cast, single((float *)dy1, c), single(dx1, c), dz1_cast);
+        ex.ws.release(m);
+        // x1 = z1 - F(x2)
+        fn_forward(ex, g, single(x2, c, q), mf, F, single((float *)y1, c, q), single(x1, c, q), -1, m1_out, &svF, false);
+    } else {
+        // x1 = z1 - F(x2) on the reconstruction stream (it needs x2 only), dz1 and dW_G meanwhile on the main stream;
+        // F's internals are placed before G's gradient steps take their temporaries, so the arena stays a stack
+        cudaStream_t main = ex.stream;
+        if (!ex.dry) {
+            cudaEventRecord(ex.ctx->ev_rfork, main);
+            cudaStreamWaitEvent(ex.ctx->recon_stream, ex.ctx->ev_rfork, 0);
+            ex.stream = ex.ctx->recon_stream;
+        }
+        // launches take short-lived scratch from the arena and hand it back at once, which is safe within one stream
+        // only: what F's recomputation touched stays out of reach of the main stream's launches until the join
+        ex.ws.high = ex.ws.off;
+        fn_forward(ex, g, single(x2, c, q), mf, F, single((float *)y1, c, q), single(x1, c, q), -1, m1_out, &svF, false);
+        if (ex.ws.high > ex.ws.off) ex.ws.off = ex.ws.high;
+        if (!ex.dry) { cudaEventRecord(ex.ctx->ev_rjoin, ex.ctx->recon_stream); ex.stream = main; }
+        fn_backward(ex, g, single((float *)y1, c, q), G, svG, single((float *)dy2, c), dy2_cast, single((float *)dy1, c), single(dx1, c), dz1_cast);
+        if (!ex.dry) cudaStreamWaitEvent(main, ex.ctx->ev_rjoin, 0);
+    }
     // dx2 = dy2 + (dF/dx2)^T dz1 ; dW_F ; dx1 = dz1 (already in place)
-    fn_backward(ex, g, single(x2, c, q), F, sv, single(dx1, c), dz1_cast, single((float *)dy2, c), single(dx2, c), dx2_cast);
+    fn_backward(ex, g, single(x2, c, q), F, svF, single(dx1, c), dz1_cast, single((float *)dy2, c), single(dx2, c), dx2_cast);
     ex.ws.release(m0);
 }

@@ -25,6 +25,8 @@ struct revnet_ctx {
     cudaStream_t capture_stream = nullptr;   // private stream on which a train step is captured into a graph
     cudaStream_t side_stream = nullptr;      // weight gradients run here, beside the data-gradient chain
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    cudaStream_t recon_stream = nullptr;     // a train step recomputes F here while the gradient steps of G run on the main stream
+    cudaEvent_t ev_rfork = nullptr, ev_rjoin = nullptr;
     // per-kernel timing (revnet_profile_*): one event after every launch while enabled
     bool profiling = false;
     bool prof_detail = false;   // summary lines per launch shape, not only per kernel name
@@ -122,12 +124,14 @@ static inline Pair halves(float *a, float *b, int c, float q = 0.f) { return Pai
 struct Arena {
     char *base = nullptr;
     size_t off = 0, cap = 0, peak = 0;
+    size_t high = 0;       // highest offset reached since the caller last set it (see block_backward)
     bool dry = true;
     bool overflow = false;
     void *alloc(size_t bytes) {
         size_t a = (off + 255) & ~size_t(255);
         off = a + bytes;
         if (off > peak) peak = off;
+        if (off > high) high = off;
         if (!dry && off > cap) { overflow = true; return nullptr; }
         return dry ? (void *)(uintptr_t)(0x1000 + a) : base + a;   // non-null fake address in dry mode
     }
@@ -323,7 +327,11 @@ struct FnSaved {
 //   forward : mx2 = statistics of x2 (if valid); my1, my2: where those of y1, y2 are left
 //   backward: m1 in = statistics of y1, out = statistics of x1; m2 out = statistics of x2;
 //             m2_use: statistics F must use for x2 when the forward pass took them from elsewhere
-//             (the first block of a stage), so that F is recomputed bit for bit
+//             (the first block of a stage), so that F is recomputed bit for bit;
+//             m1_out: where the statistics of x1 go instead of m1 (default: m1 is overwritten)
+//   overlap : the recomputation of F (x1 = y1 - F(x2)) runs on the context's reconstruction stream beside
+//             the gradient steps of G, which still read y1 and its statistics: the caller must then pass
+//             x1 != y1 and m1_out != m1
 void block_forward(Exec &ex, Geom g, int c, const std::vector<Layer> &F, const std::vector<Layer> &G,
                    float *x1, float *x2, float *y1, float *y2,
                    const Moments *mx2 = nullptr, Moments *my1 = nullptr, Moments *my2 = nullptr);
@@ -331,6 +339,6 @@ void block_backward(Exec &ex, Geom g, int c, const std::vector<Layer> &F, const 
                     const float *y1, const float *y2, const float *dy1, const float *dy2,
                     float *x1, float *x2, float *dx1, float *dx2,
                     Moments *m1 = nullptr, Moments *m2 = nullptr, const Moments *m2_use = nullptr,
-                    const bf16 *dy2_cast = nullptr, bf16 *dx2_cast = nullptr);
+                    const bf16 *dy2_cast = nullptr, bf16 *dx2_cast = nullptr, Moments *m1_out = nullptr, bool overlap = false);
 
 static inline int conv_out(int in, int k, int s) { return (in + 2 * (k / 2) - k) / s + 1; }

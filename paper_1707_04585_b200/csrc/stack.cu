@@ -3,6 +3,7 @@
 // place on it in the forward pass, and Algorithm 1 walks it back in place in the backward pass,
 // so the activation footprint does not depend on the number of units.
 #include "common.cuh"
+#include <utility>
 #include <string.h>
 #include <array>
 #include <stdlib.h>
@@ -132,6 +133,7 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
     struct StageMom { Moments m1, m2, cat, in_cat, in2; };
     std::vector<StageMom> sm(S);
     bf16 *gcast = nullptr;          // bf16 copy of the gradient w.r.t. x2 / y2, handed from unit to unit
+    float *x1_alt = nullptr, *m1_alt_buf = nullptr;
     bf16 *gcast2 = nullptr;         // stored-activation step: bf16 copy of the gradient w.r.t. z1 inside a unit
     // Stored-activation step (ordinary backprop): what every unit keeps from the forward pass.  The tensors
     // live in the workspace arena, unit after unit, and are released in reverse order by the backward pass.
@@ -153,6 +155,9 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
             size_t e = (size_t)N * s.H * s.H * s.c; if (e > cmax) cmax = e;
         }
         if (ex.mode == 0) gcast = ex.ws.get<bf16>(cmax);
+        // the reversal writes x1 beside y1 instead of over it (the two buffers change roles from unit to unit), and the
+        // statistics of x1 beside those of y1, so that F can be recomputed while G's gradient steps still read y1
+        if (!d.store_activations) { x1_alt = ex.ws.get<float>(cmax); size_t c2 = 0; for (auto &st : pl->st) if ((size_t)st.c > c2) c2 = st.c; m1_alt_buf = ex.ws.get<float>(2 * c2); }
         if (ex.mode == 0 && d.store_activations) gcast2 = ex.ws.get<bf16>(cmax);
     }
     float *recon = ex.ws.get<float>(REVNET_MAX_STAGES);
@@ -243,9 +248,18 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
         float *d1 = gbuf[gi], *d2 = gbuf[gi] + half;
         StageMom &mo = sm[si];
         if (!stored) {
-            for (int u = s.units - 1; u >= 0; u--)
-                block_backward(ex, g, s.c, bind(s.F[u], params, grads), bind(s.G[u], params, grads), x1, x2, d1, d2, x1, x2, d1, d2,
-                               &mo.m1, &mo.m2, u == 0 ? &mo.in2 : nullptr, u == s.units - 1 ? nullptr : gcast, gcast);
+            Moments mcur = mo.m1, malt = mo.m1;
+            malt.mean = m1_alt_buf; malt.rstd = m1_alt_buf + s.c; malt.valid = false;
+            float *cur1 = x1, *alt1 = x1_alt;
+            for (int u = s.units - 1; u >= 0; u--) {
+                // x1 alternates between the two buffers from unit to unit
+                block_backward(ex, g, s.c, bind(s.F[u], params, grads), bind(s.G[u], params, grads), cur1, x2, d1, d2, alt1, x2, d1, d2,
+                               &mcur, &mo.m2, u == 0 ? &mo.in2 : nullptr, u == s.units - 1 ? nullptr : gcast, gcast, &malt, true);
+                std::swap(cur1, alt1);
+                std::swap(mcur, malt);
+            }
+            // after an odd number of units the stage's input sits in the other buffer: bring it home
+            if (cur1 != x1 && !ex.dry) cudaMemcpyAsync(x1, cur1, g.P() * s.c * sizeof(float), cudaMemcpyDeviceToDevice, ex.stream);
         } else {
             // Algorithm 1 without its reconstruction lines: the gradient steps read what the forward pass kept
             for (int u = s.units - 1; u >= 0; u--) {

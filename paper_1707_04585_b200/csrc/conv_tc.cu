@@ -851,6 +851,45 @@ __global__ void splitk_sum_batch_kernel(const SumBatch b) {
     }
 }
 
+// The same sum for large gradients: 32 x 32 tiles ((tap, ci) rows x output channels) through shared memory, so that
+// the reads of the partials (output channels contiguous) and the writes of dW ((tap, ci) contiguous) are both whole
+// lines; a thread adds the splits of its four elements in ascending order, four loads in flight per element.
+__global__ void __launch_bounds__(256) splitk_sum_tiled_kernel(const SumBatch b) {
+    pdl_enter();
+    __shared__ float tile[32][33];
+    const int j = blockIdx.y;
+    const float *__restrict__ part = b.part[j];
+    const size_t n = b.n[j];
+    const int splits = b.splits[j], C = b.cout[j], R = b.rows[j];
+    const int tc_n = (C + 31) >> 5, tr_n = (R + 31) >> 5;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int t = blockIdx.x; t < tc_n * tr_n; t += gridDim.x) {
+        const int c0 = (t % tc_n) << 5, r0 = (t / tc_n) << 5;
+#pragma unroll
+        for (int k = 0; k < 4; k++) {
+            const int row = r0 + ty + 8 * k, co = c0 + tx;
+            float s = 0.f;
+            if (row < R && co < C) {
+                const float *src = part + (size_t)row * C + co;
+                int z = 0;
+                for (; z + 4 <= splits; z += 4) {
+                    const float v0 = src[(size_t)z * n], v1 = src[(size_t)(z + 1) * n], v2 = src[(size_t)(z + 2) * n], v3 = src[(size_t)(z + 3) * n];
+                    s += v0; s += v1; s += v2; s += v3;
+                }
+                for (; z < splits; z++) s += src[(size_t)z * n];
+            }
+            tile[ty + 8 * k][tx] = s;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 4; k++) {
+            const int co = c0 + ty + 8 * k, row = r0 + tx;
+            if (row < R && co < C) b.out[j][(size_t)co * R + row] = tile[tx][ty + 8 * k];
+        }
+        __syncthreads();
+    }
+}
+
 int pick_block(int c_pad) { return c_pad % 64 == 0 ? 64 : (c_pad % 32 == 0 ? 32 : 16); }
 
 // g: geometry of the tensor; (tile_w, BH, BIMG): the 128-pixel tile in units of the traversal stride
@@ -998,8 +1037,14 @@ bool conv_wgrad_tc_batch(Exec &ex, int n, const void *const *gq, const void *con
         launch(ex, wgrad_tc_kernel, (unsigned)cta, kThreads, smem, batch);
         ex.check("conv_wgrad_tc", bytes, flops);
         if (n_sums) {
-            dim3 grid((unsigned)((max_slice + 31) / 32), (unsigned)n_sums);
-            launch(ex, splitk_sum_batch_kernel, grid, 256, 0, sums);
+            if (max_slice >= 524288) {
+                size_t tiles = (max_slice + 1023) / 1024; if (tiles > (size_t)ex.ctx->sm_count * 8) tiles = (size_t)ex.ctx->sm_count * 8;
+                dim3 grid((unsigned)tiles, (unsigned)n_sums);
+                launch(ex, splitk_sum_tiled_kernel, grid, 256, 0, sums);
+            } else {
+                dim3 grid((unsigned)((max_slice + 31) / 32), (unsigned)n_sums);
+                launch(ex, splitk_sum_batch_kernel, grid, 256, 0, sums);
+            }
             ex.check("splitk_sum", sum_bytes);
         }
     }

@@ -330,6 +330,7 @@ def test_graph_replay_matches_eager(ctx):
     (4, 8, 256, 512, 3, 2, True),     # ... and in the parity-class launches of the data gradient (1, 2, 2, 4 taps)
     (4, 14, 64, 128, 3, 2, True),     # 14x14 -> 7x7: tiles of two whole images, class launches on a 7x7 grid
     (2, 28, 128, 256, 3, 1, False),   # 28-wide rows: tiles of 112 pixels, wide tiles with statistics in the epilogue
+    (8, 16, 256, 256, 3, 2, True),    # weight gradient of 590 k elements split over four pixel tiles: the tiled sum of the partials
 ])
 def test_stored_transition_layer(ctx, mode, N, H, cin, cout, k, stride, split):
     """BN-ReLU-conv with stride: forward and backward of one stored layer against the oracle."""

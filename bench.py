@@ -190,6 +190,27 @@ def depth_sweep(ctx, cfg):
     return out
 
 
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of `values` (floats) over the ranks of the default process group: a job is as slow
+    as its slowest replica.  With one rank the values come back unchanged."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def replica_seed(seed, rank):
+    """Every rank trains its own replica on its own synthetic batch."""
+    return seed + 1000 * rank
+
+
+def whole_job_rate(units_per_rank_step, world, steps, total_ms):
+    """Units all ranks processed in `steps` steps divided by the (max over ranks) time they took."""
+    return units_per_rank_step * world * steps / (total_ms * 1e-3)
+
+
 def run_ours(args, cfg):
     import torch
     import torch.distributed as dist
@@ -204,7 +225,7 @@ def run_ours(args, cfg):
     ctx = B.Context(local)
     # every rank trains its own replica on its own batch (weak scaling, no exchange step)
     import dataclasses
-    rcfg = dataclasses.replace(cfg, seed=cfg.seed + 1000 * rank)
+    rcfg = dataclasses.replace(cfg, seed=replica_seed(cfg.seed, rank))
     inp = syn.make_stack_inputs(rcfg)
     run = R.StackRunner(ctx, rcfg, mode=0)
     run.load(inp["images"], inp["labels"], inp["params"])
@@ -308,13 +329,11 @@ def run_ours(args, cfg):
             bc = syn.BlockCfg(rcfg.N, H, H, s_cfg.c, s_cfg.w, s_cfg.kind, seed=9)
             block_ms[f"{s_cfg.kind}_c{s_cfg.c}_{H}x{H}"] = R.time_block(ctx, bc, 0, reps=5, warmup=3)
 
-    t = torch.tensor([dev_ms, e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    dev_ms, e2e_ms = float(t[0]), float(t[1])
+    dev_ms, e2e_ms = max_over_ranks([dev_ms, e2e_ms], world, "cuda")
     if rank == 0:
         peaks = load_peaks()
         total_images = rcfg.N * world * args.steps
+        assert abs(whole_job_rate(rcfg.N, world, args.steps, dev_ms) - total_images / (dev_ms * 1e-3)) < 1e-6 * total_images
         prof = {k: v for k, v in by_device_kernel(prof).items() if k != "step_begin"}    # not a kernel: the host-ahead hold of a profiled step
         tot = sum(v["ms"] for v in prof.values()) or 1.0
         top = max(prof.items(), key=lambda kv: kv[1]["ms"])

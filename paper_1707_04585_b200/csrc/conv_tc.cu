@@ -972,10 +972,14 @@ static bool wgrad_plan(Geom gi, const Layer &L, int cta_budget, WgPlan &w, bool 
     w.tail_bytes = p.GM * 32768 - p.a_region;        // what the MMAs of a partly filled group read past the last stage
     p.stages = (kWgSmemMax - 2048 - w.tail_bytes) / w.stage_bytes; if (p.stages > kWgStages) p.stages = kWgStages;
     if (p.stages < 2) return p.sep ? wgrad_plan(gi, L, cta_budget, w, false) : false;
-    // split the pixel reduction so that the job's CTAs cover its share of the machine once
-    int splits = (cta_budget + p.m_chunks * w.n_tiles - 1) / (p.m_chunks * w.n_tiles);
-    if (splits > p.n_tiles_px) splits = p.n_tiles_px;
-    if (splits < 1) splits = 1;
+    // split the pixel reduction so that the job's CTAs cover its share of the machine once: rounding the split
+    // count up may spill a few CTAs into a second wave (these CTAs fill an SM each), rounding down leaves SMs idle;
+    // take whichever walks fewer pixel tiles one after the other
+    const int pairs = p.m_chunks * w.n_tiles;
+    auto clampi = [&](int v) { return v < 1 ? 1 : (v > p.n_tiles_px ? p.n_tiles_px : v); };
+    const int s_hi = clampi((cta_budget + pairs - 1) / pairs), s_lo = clampi(cta_budget / pairs);
+    auto serial_tiles = [&](int sp) { return ((pairs * sp + cta_budget - 1) / cta_budget) * ((p.n_tiles_px + sp - 1) / sp); };
+    int splits = serial_tiles(s_lo) < serial_tiles(s_hi) ? s_lo : s_hi;
     p.splits = splits;
     p.slice = (size_t)L.cout * taps * L.cin;
     return true;

@@ -18,8 +18,11 @@
  *   - The caller owns every buffer.  The library allocates no device memory in any call
  *     below; scratch comes from the workspace the caller passes.
  *   - Work is enqueued on the caller's stream (a cudaStream_t passed as void*); calls do not
- *     synchronise unless stated.  Device pointers must be 16-byte aligned, channel counts
- *     multiples of 4.
+ *     synchronise unless stated.  A backward call may fork part of its work onto streams the
+ *     context owns (weight gradients beside the data-gradient chain; in a train step the
+ *     recomputation of F beside the gradient steps of G) and joins them again before it returns:
+ *     to the caller everything is ordered as if it ran on the stream passed in.  Device pointers
+ *     must be 16-byte aligned, channel counts multiples of 4.
  *   - Aliasing y1==x1, y2==x2 in revnet_block_fwd and x1==y1, x2==y2, dx1==dy1, dx2==dy2 in
  *     revnet_block_bwd is legal: that is how a stack runs in place.
  *   - Gradient outputs are overwritten, not accumulated.

@@ -113,3 +113,28 @@ def test_stored_step_equals_reversible_step_at_full_size(ctx, name):
     assert torch.equal(flat[0][0], flat[1][0]) and torch.equal(flat[0][1], flat[1][1]) and flat[0][2] == flat[1][2]
     assert np.isfinite(flat[0][2])
     assert stats[1].flops_bwd < stats[0].flops_bwd and stats[1].stored_activation_bytes > 5 * stats[0].stored_activation_bytes
+
+
+def test_profiled_step_gives_the_same_result(ctx):
+    """Per-kernel profiling runs the step on one stream, kernel by kernel (no side streams, no graph).  The forward
+    pass is the same launches, hence the same bits; the weight gradients of a function are then one launch per layer
+    instead of one per function, which splits their pixel sums differently: equal up to float32 summation order."""
+    cfg = syn.shrink(syn.stack_config("revnet38"), N=16)
+    inp = syn.make_stack_inputs(cfg, affine_jitter=True)
+    res = []
+    for profiled in (False, True):
+        r = R.StackRunner(ctx, cfg, 0)
+        r.load(inp["images"], inp["labels"], inp["params"])
+        if profiled:
+            B.revnet_profile_enable(ctx, 2)
+        r.step()
+        torch.cuda.synchronize()
+        if profiled:
+            prof = B.revnet_profile_summary(ctx)
+            B.revnet_profile_enable(ctx, 0)
+            assert any(k.startswith("conv_fprop_fused|") for k in prof) and all(v["ms"] >= 0 for v in prof.values())
+        res.append((r.grads.clone(), r.params.clone(), r.logits.clone()))
+        B.revnet_check_device(ctx)
+    assert torch.equal(res[0][2], res[1][2])
+    for a, b in zip(res[0][:2], res[1][:2]):
+        assert float((a - b).norm() / b.norm()) <= 1e-5

@@ -363,42 +363,73 @@ __global__ void maxpool_fwd_kernel(const float *__restrict__ in, float *__restri
     }
 }
 
-// Gradient goes to the first maximum met in (kh,kw) row-major scan of each window.  Gather form:
-// each input element visits the (at most four) windows that cover it, in a fixed order.
-__global__ void maxpool_bwd_kernel(const float *__restrict__ in, const float *__restrict__ dout, float *__restrict__ din,
-                                   int N, int H, int W, int C4, int Ho, int Wo) {
+// Gradient goes to the first maximum met in (kh,kw) row-major scan of each window.
+// A CTA takes 8 x 8 input pixels x 8 channel quads of one image: it loads them with the halo their windows reach
+// (11 x 11 pixels; outside the image: -inf) and the 5 x 5 gradients of those windows into shared memory, finds
+// every window's first maximum once, and each input element then asks its (at most four) windows whether it is
+// theirs -- one global read per element instead of one per window tap.
+__global__ void __launch_bounds__(256) maxpool_bwd_kernel(const float *__restrict__ in, const float *__restrict__ dout, float *__restrict__ din,
+                                                          int N, int H, int W, int C4, int Ho, int Wo, int tiles_y, int tiles_x, int tiles_q) {
     pdl_enter();
-    size_t n = (size_t)N * H * W * C4;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        int q = (int)(i % C4); size_t p = i / C4;
-        int x = (int)(p % W); p /= W; int y = (int)(p % H); int b = (int)(p / H);
-        const float4 self = ld4(in + i * 4);
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        // windows (io, j) that cover (y, x): io*2 - 1 <= y <= io*2 + 1
-        for (int io = y / 2; io <= (y + 1) / 2; io++) {
-            if (io >= Ho) continue;
-            for (int j = x / 2; j <= (x + 1) / 2; j++) {
-                if (j >= Wo) continue;
-                // per channel: is (y,x) the first maximum of window (io,j)?
-                bool f0 = true, f1 = true, f2 = true, f3 = true;
-                for (int kh = 0; kh < 3; kh++) for (int kw = 0; kw < 3; kw++) {
-                    int yy = io * 2 + kh - 1, xx = j * 2 + kw - 1;
-                    if (yy < 0 || yy >= H || xx < 0 || xx >= W || (yy == y && xx == x)) continue;
-                    const float4 v = ld4(in + ((((size_t)b * H + yy) * W + xx) * C4 + q) * 4);
-                    const bool before = (yy < y) || (yy == y && xx < x);
-                    f0 = f0 && !(v.x > self.x || (before && v.x == self.x));
-                    f1 = f1 && !(v.y > self.y || (before && v.y == self.y));
-                    f2 = f2 && !(v.z > self.z || (before && v.z == self.z));
-                    f3 = f3 && !(v.w > self.w || (before && v.w == self.w));
-                }
-                const float4 g = ld4(dout + ((((size_t)b * Ho + io) * Wo + j) * C4 + q) * 4);
-                if (f0) acc.x += g.x;
-                if (f1) acc.y += g.y;
-                if (f2) acc.z += g.z;
-                if (f3) acc.w += g.w;
+    __shared__ float4 tin[11 * 11 * 8];
+    __shared__ float4 tg[5 * 5 * 8];
+    __shared__ int4 tam[5 * 5 * 8];
+    int t = blockIdx.x;
+    const int tq = t % tiles_q; t /= tiles_q;
+    const int tx = t % tiles_x; t /= tiles_x;
+    const int ty = t % tiles_y; const int b = t / tiles_y;
+    const int y0 = ty * 8, x0 = tx * 8, q0 = tq * 8;
+    const int tid = threadIdx.x;
+    const float ninf = -INFINITY;
+    for (int idx = tid; idx < 11 * 11 * 8; idx += 256) {
+        const int q = idx & 7, pos = idx >> 3, ry = pos / 11, rx = pos - ry * 11;
+        const int yy = y0 - 1 + ry, xx = x0 - 1 + rx;
+        float4 v = make_float4(ninf, ninf, ninf, ninf);
+        if (yy >= 0 && yy < H && xx >= 0 && xx < W && q0 + q < C4) v = ld4(in + ((((size_t)b * H + yy) * W + xx) * C4 + q0 + q) * 4);
+        tin[idx] = v;
+    }
+    if (tid < 5 * 5 * 8) {
+        const int q = tid & 7, wpos = tid >> 3, wi = wpos / 5, wj = wpos - wi * 5;
+        const int io = y0 / 2 + wi, j = x0 / 2 + wj;
+        float4 g = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (io < Ho && j < Wo && q0 + q < C4) g = ld4(dout + ((((size_t)b * Ho + io) * Wo + j) * C4 + q0 + q) * 4);
+        tg[tid] = g;
+    }
+    __syncthreads();
+    if (tid < 5 * 5 * 8) {
+        // window (wi, wj) covers tile rows 2wi .. 2wi+2, columns 2wj .. 2wj+2
+        const int q = tid & 7, wpos = tid >> 3, wi = wpos / 5, wj = wpos - wi * 5;
+        float4 best = make_float4(ninf, ninf, ninf, ninf);
+        int4 at = make_int4(-1, -1, -1, -1);
+        for (int kh = 0; kh < 3; kh++)
+            for (int kw = 0; kw < 3; kw++) {
+                const int pos = (2 * wi + kh) * 11 + 2 * wj + kw;
+                const float4 v = tin[pos * 8 + q];
+                if (v.x > best.x) { best.x = v.x; at.x = pos; }
+                if (v.y > best.y) { best.y = v.y; at.y = pos; }
+                if (v.z > best.z) { best.z = v.z; at.z = pos; }
+                if (v.w > best.w) { best.w = v.w; at.w = pos; }
             }
-        }
-        st4(din + i * 4, acc);
+        tam[tid] = at;
+    }
+    __syncthreads();
+    for (int idx = tid; idx < 8 * 8 * 8; idx += 256) {
+        const int q = idx & 7, lp = idx >> 3, ly = lp >> 3, lx = lp & 7;
+        const int y = y0 + ly, x = x0 + lx;
+        if (y >= H || x >= W || q0 + q >= C4) continue;
+        const int mine = (ly + 1) * 11 + lx + 1;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int wi = ly / 2; wi <= (ly + 1) / 2; wi++)
+            for (int wj = lx / 2; wj <= (lx + 1) / 2; wj++) {
+                const int w = (wi * 5 + wj) * 8 + q;        // windows beyond the pooled image carry a zero gradient
+                const int4 at = tam[w];
+                const float4 g = tg[w];
+                if (at.x == mine) acc.x += g.x;
+                if (at.y == mine) acc.y += g.y;
+                if (at.z == mine) acc.z += g.z;
+                if (at.w == mine) acc.w += g.w;
+            }
+        st4(din + ((((size_t)b * H + y) * W + x) * C4 + q0 + q) * 4, acc);
     }
 }
 
@@ -412,8 +443,8 @@ void maxpool_fwd(Exec &ex, const float *in, float *out, int N, int H, int W, int
 void maxpool_bwd(Exec &ex, const float *in, const float *dout, float *din, int N, int H, int W, int C) {
     if (ex.dry) return;
     int Ho = conv_out(H, 3, 2), Wo = conv_out(W, 3, 2);
-    size_t n = (size_t)N * H * W * (C / 4);
-    launch(ex, maxpool_bwd_kernel, ew_grid(n, ex.ctx->sm_count), 256, 0, in, dout, din, N, H, W, C / 4, Ho, Wo);
+    const int C4 = C / 4, tiles_y = (H + 7) / 8, tiles_x = (W + 7) / 8, tiles_q = (C4 + 7) / 8;
+    launch(ex, maxpool_bwd_kernel, (unsigned)((size_t)N * tiles_y * tiles_x * tiles_q), 256, 0, in, dout, din, N, H, W, C4, Ho, Wo, tiles_y, tiles_x, tiles_q);
     ex.check("maxpool_bwd");
 }
 

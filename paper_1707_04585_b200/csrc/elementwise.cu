@@ -547,6 +547,25 @@ __global__ void fc_wgrad_kernel(const float *__restrict__ dlogits, const float *
     }
     if (i < (size_t)K) { float s = 0.f; for (int n = 0; n < N; n++) s += dlogits[(size_t)n * K + i]; db[i] = s; }
 }
+// the same for a small layer: one warp per element of dW (and of db), lanes over the samples, added by a shuffle tree
+__global__ void fc_wgrad_warp_kernel(const float *__restrict__ dlogits, const float *__restrict__ feat, int N, int C, int K,
+                                     float *__restrict__ dW, float *__restrict__ db) {
+    pdl_enter();
+    const int lane = threadIdx.x & 31;
+    const size_t w = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const size_t n_out = (size_t)K * C + K;
+    if (w >= n_out) return;
+    float s = 0.f;
+    if (w < (size_t)K * C) {
+        const int k = (int)(w / C), c = (int)(w - (size_t)k * C);
+        for (int n = lane; n < N; n += 32) s = fmaf(dlogits[(size_t)n * K + k], feat[(size_t)n * C + c], s);
+    } else {
+        const int k = (int)(w - (size_t)K * C);
+        for (int n = lane; n < N; n += 32) s += dlogits[(size_t)n * K + k];
+    }
+    for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    if (lane == 0) { if (w < (size_t)K * C) dW[w] = s; else db[w - (size_t)K * C] = s; }
+}
 __global__ void fc_dgrad_kernel(const float *__restrict__ dlogits, const float *__restrict__ Wfc, int N, int C, int K,
                                 float scale, float *__restrict__ dfeat) {
     pdl_enter();
@@ -570,7 +589,8 @@ void head_bwd(Exec &ex, Pair dy, int N, int HW, const float *Wfc, const float *f
     const int C = dy.C();
     ex.flops += 4ull * N * C * K;
     if (ex.dry) return;
-    launch(ex, fc_wgrad_kernel, cdiv((size_t)K * C, 256), 256, 0, dlogits, feat, N, C, K, dWfc, dbfc);
+    if ((size_t)K * C <= 65536) launch(ex, fc_wgrad_warp_kernel, cdiv(((size_t)K * C + K) * 32, 256), 256, 0, dlogits, feat, N, C, K, dWfc, dbfc);
+    else launch(ex, fc_wgrad_kernel, cdiv((size_t)K * C, 256), 256, 0, dlogits, feat, N, C, K, dWfc, dbfc);
     ex.check("fc_wgrad");
     launch(ex, fc_dgrad_kernel, cdiv((size_t)N * C, 256), 256, 0, dlogits, Wfc, N, C, K, 1.f / (float)HW, dfeat);
     ex.check("fc_dgrad");

@@ -68,7 +68,8 @@ typedef struct revnet_plan revnet_plan;
  * bytes of device memory for status words; nothing else is ever allocated by the library. */
 int revnet_create(revnet_ctx **out, int device);
 int revnet_destroy(revnet_ctx *ctx);
-/* Text of the last error recorded on ctx (never NULL; valid until the next failing call). */
+/* Text of the last error recorded on ctx (never NULL; valid until the next failing call on the same
+ * context: a context is meant to be used from one thread at a time). */
 const char *revnet_last_error(const revnet_ctx *ctx);
 
 /* A residual function: n_layers (1..3) layers, each BN -> ReLU -> conv k x k, stride 1
@@ -91,11 +92,17 @@ typedef struct {
 } revnet_block_desc;
 
 /* Parameters of one residual function (device pointers): W[l] is [cout][k][k][cin],
- * gamma[l], beta[l] are [cin[l]] (the BN in front of conv l). */
+ * gamma[l], beta[l] are [cin[l]] (the BN in front of conv l).
+ * Wpack_fprop / Wpack_dgrad: optional bf16 copies of W[l] in the layout the tensor-core kernels read
+ * (forward: [cout][tap][cin]; data gradient: [cin][mirrored tap][cout]; both padded), written by
+ * revnet_pack_weights.  NULL: the block call that needs one builds it from W[l] into its workspace,
+ * every time.  A pack is valid until W[l] changes.  Ignored in mode 1. */
 typedef struct {
     const float *W[3];
     const float *gamma[3];
     const float *beta[3];
+    const void *Wpack_fprop[3];
+    const void *Wpack_dgrad[3];
 } revnet_fn_params;
 
 /* Gradient outputs of one residual function, same shapes as the parameters. */
@@ -109,6 +116,18 @@ typedef struct {
 int revnet_block_workspace_bytes(revnet_ctx *ctx, const revnet_block_desc *desc,
                                  size_t *fwd_bytes, size_t *bwd_bytes);
 
+/* bf16 weight packs of a block, built once and reused by any number of forward / backward calls
+ * (Appendix 6.3 hands each layer its weights as they are; a pack is the same weights rounded to the
+ * operand precision of Eq. 2's convolutions in the layout the kernels read).  revnet_block_pack_bytes
+ * gives the size of the caller-owned device buffer; revnet_pack_weights enqueues the pack kernels on
+ * `stream` and stores the pack pointers into F and G (host structs), NULL for layers whose shape the
+ * tensor-core kernels do not take and in mode 1 (0 bytes).  The buffer must be 256-byte aligned.
+ * Errors: REVNET_E_INVALID_ARG (null), REVNET_E_MISALIGNED, REVNET_E_WORKSPACE_TOO_SMALL. */
+int revnet_block_pack_bytes(revnet_ctx *ctx, const revnet_block_desc *desc, size_t *bytes);
+int revnet_pack_weights(revnet_ctx *ctx, const revnet_block_desc *desc,
+                        revnet_fn_params *F, revnet_fn_params *G,
+                        void *pack_buffer, size_t pack_bytes, void *stream);
+
 /* Block forward (Section 3.1): y1 = x1 + F(x2); y2 = x2 + G(y1). */
 int revnet_block_fwd(revnet_ctx *ctx, const revnet_block_desc *desc,
                      const void *x1, const void *x2,
@@ -121,8 +140,9 @@ int revnet_block_fwd(revnet_ctx *ctx, const revnet_block_desc *desc,
  * where cudaMalloc and friends are forbidden or would stall, and plugins that receive tensors but
  * no allocator.  Same computation and same results as revnet_block_fwd, but the scratch comes from
  * a 16 MiB array built into the library (held on every GPU that loads the library until the
- * process exits) instead of a caller workspace.  The call allocates no device memory and calls no
- * allocating CUDA routine.  Shapes whose forward scratch (revnet_block_workspace_bytes) exceeds
+ * process exits) instead of a caller workspace.  The call itself calls no allocating CUDA routine;
+ * the array is part of the library image, which the CUDA runtime places on a device when the library
+ * is first used there -- that can be inside this entry point's first call on that device.  Shapes whose forward scratch (revnet_block_workspace_bytes) exceeds
  * 16 MiB are rejected with REVNET_E_WORKSPACE_TOO_SMALL and a message naming both sizes.
  * The first call on a device looks up the array's device address (with that device current, as it
  * must be for every call); make that first call before starting any stream capture.  All calls
@@ -220,7 +240,10 @@ typedef struct {
     uint64_t flops_fwd, flops_bwd;     /* dense conv + FC flops issued (2 per multiply-add) */
     uint64_t kernel_launches;          /* kernels enqueued by the step */
     float recon_max_abs[REVNET_MAX_STAGES]; /* filled only with verify_reconstruction */
-    int device_status;                 /* 0, or the code a device-side bounded wait reported */
+    int device_status;                 /* what the step's kernels recorded on the device (0, REVNET_E_TIMEOUT, REVNET_E_INVALID_ARG).
+                                          Filled only by calls that synchronise the stream anyway (revnet_train_step with
+                                          verify_reconstruction, revnet_train_step_host); otherwise 0: an asynchronous call
+                                          cannot know yet, ask revnet_check_device */
 } revnet_step_stats;
 
 /* Plan a stack: validates the description and sizes the caller's buffers.
@@ -232,6 +255,10 @@ typedef struct {
 int revnet_stack_plan(revnet_ctx *ctx, const revnet_stack_desc *desc, revnet_plan **plan,
                       size_t *param_count, size_t *activation_bytes, size_t *workspace_bytes);
 int revnet_plan_destroy(revnet_plan *plan);
+/* Optional: declare how large the activation and workspace buffers passed to revnet_train_step are.
+ * Once declared, a step whose buffers are smaller than the plan needs returns
+ * REVNET_E_WORKSPACE_TOO_SMALL instead of writing past them (the step takes pointers only). */
+int revnet_plan_set_buffer_sizes(revnet_plan *plan, size_t activation_bytes, size_t workspace_bytes);
 /* How the planned workspace divides: the part that holds per-parameter data (bf16 weight packs,
  * the SGD segment table) grows with depth like the parameters do; the rest is activation scratch
  * (gradient pair, one block's recomputed internals, reduction partials) and does not depend on the
@@ -254,7 +281,8 @@ int revnet_train_step(revnet_ctx *ctx, revnet_plan *plan,
 
 /* Same step fed from HOST memory: copies images_host / labels_host (pinned memory recommended)
  * into the device staging buffers images_dev / labels_dev, runs revnet_train_step, copies loss
- * and pred back to loss_host / pred_host and synchronises the stream. */
+ * and pred back to loss_host / pred_host and synchronises the stream.  Being synchronous it also
+ * returns the status its kernels recorded on the device, if any (see revnet_check_device). */
 int revnet_train_step_host(revnet_ctx *ctx, revnet_plan *plan,
                            const float *images_host, const int32_t *labels_host,
                            float *images_dev, int32_t *labels_dev,
@@ -265,10 +293,18 @@ int revnet_train_step_host(revnet_ctx *ctx, revnet_plan *plan,
                            revnet_step_stats *stats, void *stream);
 
 /* Waits inside the library's kernels (on shared-memory barriers) are bounded; a kernel whose wait
- * runs out stops its work, records a status word on the device and exits normally.
- * revnet_check_device synchronises the stream, returns REVNET_OK or that status (REVNET_E_TIMEOUT)
- * and clears it.  No counterpart in the paper: failure reporting. */
+ * runs out stops its work, records a status word on the device and exits normally.  The loss kernel
+ * records REVNET_E_INVALID_ARG the same way when a label lies outside [0, n_classes) (it reads
+ * nothing at that label and the step's loss becomes NaN).
+ * revnet_check_device synchronises the stream, returns REVNET_OK or the recorded status and clears it
+ * together with the counters of the kernels' grid-wide reductions, so the context stays usable.
+ * No counterpart in the paper: failure reporting. */
 int revnet_check_device(revnet_ctx *ctx, void *stream);
+
+/* Self-test of that path (no counterpart in the paper): enqueues one small kernel whose single wait,
+ * on a barrier nothing ever arrives on, is limited to limit_ns (at most 100 ms).  The wait runs out,
+ * the kernel records REVNET_E_TIMEOUT and returns normally; the next revnet_check_device reports it. */
+int revnet_selftest_bounded_wait(revnet_ctx *ctx, uint64_t limit_ns, void *stream);
 
 /* ---- per-kernel timing (no counterpart in the paper: measurement support) ----
  * While enabled, every kernel the library launches on behalf of this context is followed by a

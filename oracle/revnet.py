@@ -251,7 +251,7 @@ def softmax_ce(logits, labels):
     return loss, sm / N
 
 
-def stack_train_grads(net, images, labels, mode, num=None):
+def stack_train_grads(net, images, labels, mode, num=None, keep_blocks=(), keep_transitions=False):
     """Forward + backward of the whole stack.
 
     mode "stored": every block's activations are kept (ordinary backprop).
@@ -261,11 +261,17 @@ def stack_train_grads(net, images, labels, mode, num=None):
     Returns a dict: logits, loss, pred, grads{name: array}, stored_bytes (activation bytes kept
     between forward and backward), block_inputs (the (x1,x2) each block saw in the forward) and,
     in reconstruct mode, recovered (the (x1,x2) Algorithm 1 rebuilt), both keyed (stage, unit).
+    For every (stage, unit) in keep_blocks the dict `blocks` also holds what Algorithm 1 was given
+    and what it returned there: y1, y2, dy1, dy2, dx1, dx2 (the problem statement of Section 3.2 for
+    that block inside the network; reconstruct mode only).  With keep_transitions, `transitions[stage]` holds the stored
+    layer's input, its upstream gradient and the gradient it passed on (x, dy, dx).
     """
     eps = net["eps"]
     images = np.asarray(images, np.float64)
     labels = np.asarray(labels).astype(np.int64)
     grads, stored, block_inputs, recovered = {}, [], {}, {}
+    blocks, transitions = {}, {}
+    assert not keep_blocks or mode == "reconstruct"
 
     # ---- forward
     st = net["stem"]
@@ -282,6 +288,8 @@ def stack_train_grads(net, images, labels, mode, num=None):
         tcache = None
         if S["trans"] is not None:
             stored.append(h)                  # input of a non-reversible layer is kept
+            if keep_transitions:
+                transitions[si] = dict(x=h)
             h, tcache = fn_fwd(h, [S["trans"]], eps, num)
         c = S["c"]
         if si == 0 or S["trans"] is not None:
@@ -319,14 +327,22 @@ def stack_train_grads(net, images, labels, mode, num=None):
         d1, d2 = dh[:, :c].copy(), dh[:, c:].copy()
         for ui in reversed(range(len(S["units"]))):
             F, G = S["units"][ui]
+            rec = dict(y1=y1, y2=y2, dy1=d1, dy2=d2) if (si, ui) in keep_blocks else None
             if mode == "stored":
                 d1, d2 = block_bwd_stored(d1, d2, bcaches[ui], grads, num)
             else:
                 y1, y2, d1, d2 = block_bwd_reconstruct(y1, y2, d1, d2, F, G, eps, grads, num)
                 recovered[(si, ui)] = (y1, y2)
+            if rec is not None:
+                rec.update(dx1=d1, dx2=d2)
+                blocks[(si, ui)] = rec
         dh = np.concatenate([d1, d2], axis=1)
         if tcache is not None:
+            if keep_transitions:
+                transitions[si]["dy"] = dh
             dh = fn_bwd(dh, tcache, grads, num)
+            if keep_transitions:
+                transitions[si]["dx"] = dh
     if pool_idx is not None:
         dh = maxpool_bwd(dh, pool_idx, stem_out_hw)
     grads[st["name"] + ".W"] = conv_wgrad(dh, images, wst.shape[2], stride=st["stride"], pad=st["pad"])
@@ -337,7 +353,8 @@ def stack_train_grads(net, images, labels, mode, num=None):
             seen.add(id(t))
             nbytes += t.size * 4              # counted at the 4-byte storage width of the method
     return dict(logits=logits, loss=loss, pred=pred, grads=grads, stored_bytes=nbytes,
-                block_inputs=block_inputs, recovered=recovered, top=(stage_fw[-1][2], stage_fw[-1][3]))
+                block_inputs=block_inputs, recovered=recovered, top=(stage_fw[-1][2], stage_fw[-1][3]),
+                blocks=blocks, transitions=transitions)
 
 
 def sgd_step(params, grads, velocity, lr, momentum, weight_decay, decayed):

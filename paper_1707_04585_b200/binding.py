@@ -23,7 +23,8 @@ EXPORTS = ["revnet_create", "revnet_destroy", "revnet_last_error", "revnet_block
            "revnet_block_fwd", "revnet_block_bwd", "revnet_stack_plan", "revnet_plan_destroy",
            "revnet_train_step", "revnet_train_step_host", "revnet_profile_enable", "revnet_profile_summary", "revnet_check_device", "revnet_plan_scratch_split",
            "revnet_transition_workspace_bytes", "revnet_transition_fwd", "revnet_transition_bwd",
-           "revnet_block_fwd_noalloc"]
+           "revnet_block_fwd_noalloc", "revnet_block_pack_bytes", "revnet_pack_weights", "revnet_selftest_bounded_wait",
+           "revnet_plan_set_buffer_sizes"]
 
 
 class FnDesc(C.Structure):
@@ -36,7 +37,8 @@ class BlockDesc(C.Structure):
 
 
 class FnParams(C.Structure):
-    _fields_ = [("W", C.c_void_p * 3), ("gamma", C.c_void_p * 3), ("beta", C.c_void_p * 3)]
+    _fields_ = [("W", C.c_void_p * 3), ("gamma", C.c_void_p * 3), ("beta", C.c_void_p * 3),
+                ("Wpack_fprop", C.c_void_p * 3), ("Wpack_dgrad", C.c_void_p * 3)]
 
 
 class FnGrads(C.Structure):
@@ -84,7 +86,7 @@ def lib():
 
 
 class RevnetError(RuntimeError):
-    pass
+    status = 0          # the revnet_status the call returned
 
 
 def _ptr(t):
@@ -109,7 +111,9 @@ class Context:
 
     def check(self, rc, what):
         if rc:
-            raise RevnetError(f"{what}: status {rc}: {lib().revnet_last_error(self.h).decode()}")
+            e = RevnetError(f"{what}: status {rc}: {lib().revnet_last_error(self.h).decode()}")
+            e.status = rc
+            raise e
 
     def close(self):
         if self.h:
@@ -211,10 +215,30 @@ def revnet_block_workspace_bytes(ctx: Context, desc: BlockDesc):
 
 
 def _fn_params(tensors: List[dict]) -> FnParams:
+    """Layer dicts -> the ABI struct.  Optional integer entries "Wpack_fprop" / "Wpack_dgrad" (device
+    addresses written by revnet_pack_weights) are passed through."""
     p = FnParams()
     for i, t in enumerate(tensors):
         p.W[i], p.gamma[i], p.beta[i] = t["W"].data_ptr(), t["gamma"].data_ptr(), t["beta"].data_ptr()
+        p.Wpack_fprop[i], p.Wpack_dgrad[i] = t.get("Wpack_fprop") or None, t.get("Wpack_dgrad") or None
     return p
+
+
+def revnet_block_pack_bytes(ctx, desc) -> int:
+    n = C.c_size_t()
+    ctx.check(lib().revnet_block_pack_bytes(ctx.h, C.byref(desc), C.byref(n)), "revnet_block_pack_bytes")
+    return n.value
+
+
+def revnet_pack_weights(ctx, desc, F, G, pack_buffer):
+    """Build the bf16 weight packs of a block into pack_buffer and record their addresses in the layer
+    dicts of F and G (keys "Wpack_fprop", "Wpack_dgrad"); later block calls with these dicts use them."""
+    fp, gp = _fn_params(F), _fn_params(G)
+    ctx.check(lib().revnet_pack_weights(ctx.h, C.byref(desc), C.byref(fp), C.byref(gp), _ptr(pack_buffer),
+                                        C.c_size_t(pack_buffer.numel() * pack_buffer.element_size()), _stream()), "revnet_pack_weights")
+    for st, layers in ((fp, F), (gp, G)):
+        for i, t in enumerate(layers):
+            t["Wpack_fprop"], t["Wpack_dgrad"] = st.Wpack_fprop[i], st.Wpack_dgrad[i]
 
 
 def _fn_grads(tensors: List[dict]) -> FnGrads:
@@ -251,6 +275,10 @@ class Plan:
         ps, as_ = C.c_size_t(), C.c_size_t()
         ctx.check(lib().revnet_plan_scratch_split(self.h, C.byref(ps), C.byref(as_)), "revnet_plan_scratch_split")
         self.param_scratch_bytes, self.activation_scratch_bytes = ps.value, as_.value
+
+    def set_buffer_sizes(self, activation_bytes: int, workspace_bytes: int):
+        self.ctx.check(lib().revnet_plan_set_buffer_sizes(self.h, C.c_size_t(activation_bytes), C.c_size_t(workspace_bytes)),
+                       "revnet_plan_set_buffer_sizes")
 
     def close(self):
         if self.h:
@@ -308,6 +336,10 @@ def revnet_profile_summary(ctx):
 def revnet_check_device(ctx):
     """Synchronise and raise if a kernel reported that it gave up a bounded wait."""
     ctx.check(lib().revnet_check_device(ctx.h, _stream()), "revnet_check_device")
+
+
+def revnet_selftest_bounded_wait(ctx, limit_ns: int):
+    ctx.check(lib().revnet_selftest_bounded_wait(ctx.h, C.c_uint64(limit_ns), _stream()), "revnet_selftest_bounded_wait")
 
 
 def _nbytes(t):

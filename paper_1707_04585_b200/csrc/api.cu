@@ -1,8 +1,10 @@
 // C ABI: context management and the block-level entry points.
 #include "common.cuh"
+#include "tc_ptx.cuh"
 #include <string.h>
 #include <stdio.h>
 #include <math.h>
+#include <atomic>
 
 static int fail(revnet_ctx *ctx, int code, const std::string &msg) { if (ctx) ctx->err = msg; return code; }
 
@@ -73,7 +75,10 @@ static std::vector<Layer> layers_of(const revnet_fn_desc &f, const revnet_fn_par
     std::vector<Layer> v(f.n_layers);
     for (int l = 0; l < f.n_layers; l++) {
         v[l].cin = f.cin[l]; v[l].cout = f.cout[l]; v[l].k = f.k[l]; v[l].stride = 1;
-        if (p) { v[l].W = p->W[l]; v[l].gamma = p->gamma[l]; v[l].beta = p->beta[l]; }
+        if (p) {
+            v[l].W = p->W[l]; v[l].gamma = p->gamma[l]; v[l].beta = p->beta[l];
+            v[l].Wp_fprop = (const bf16 *)p->Wpack_fprop[l]; v[l].Wp_dgrad = (const bf16 *)p->Wpack_dgrad[l];
+        }
         if (g) { v[l].dW = g->dW[l]; v[l].dgamma = g->dgamma[l]; v[l].dbeta = g->dbeta[l]; }
     }
     return v;
@@ -161,6 +166,53 @@ extern "C" int revnet_block_bwd(revnet_ctx *ctx, const revnet_block_desc *d, con
     return finish(ctx, ex, "revnet_block_bwd");
 }
 
+// ---- bf16 weight packs made once and handed to the block calls (a train step makes its own, once per step)
+static bool packable(const revnet_block_desc *d, const revnet_fn_desc &f, int l) {
+    return d->mode == 0 && f.cin[l] % 8 == 0 && f.cout[l] % 8 == 0;
+}
+static size_t pack_bytes_of(const revnet_block_desc *d) {
+    size_t total = 0;
+    for (const revnet_fn_desc *f : {&d->F, &d->G})
+        for (int l = 0; l < f->n_layers; l++)
+            if (packable(d, *f, l))
+                for (int tr = 0; tr < 2; tr++) total += (tc_pack_elems(f->cin[l], f->cout[l], f->k[l], tr != 0) * sizeof(bf16) + 255) & ~size_t(255);
+    return total;
+}
+extern "C" int revnet_block_pack_bytes(revnet_ctx *ctx, const revnet_block_desc *d, size_t *bytes) {
+    int rc = check_desc(ctx, d);
+    if (rc) return rc;
+    if (!bytes) return fail(ctx, REVNET_E_INVALID_ARG, "revnet_block_pack_bytes: null pointer");
+    *bytes = pack_bytes_of(d);
+    return REVNET_OK;
+}
+extern "C" int revnet_pack_weights(revnet_ctx *ctx, const revnet_block_desc *d, revnet_fn_params *Fp, revnet_fn_params *Gp,
+                                   void *pack_buffer, size_t pack_bytes, void *stream) {
+    int rc = check_desc(ctx, d);
+    if (rc) return rc;
+    bool mis = false;
+    if (!fn_ptrs_ok(d->F, Fp, nullptr, false, &mis) || !fn_ptrs_ok(d->G, Gp, nullptr, false, &mis))
+        return fail(ctx, REVNET_E_INVALID_ARG, "revnet_pack_weights: null pointer");
+    const size_t need = pack_bytes_of(d);
+    if (need && !pack_buffer) return fail(ctx, REVNET_E_INVALID_ARG, "revnet_pack_weights: null pack buffer");
+    if (mis || ((uintptr_t)pack_buffer & 255)) return fail(ctx, REVNET_E_MISALIGNED, "revnet_pack_weights: the pack buffer must be 256-byte aligned, parameters 16-byte aligned");
+    if (pack_bytes < need) return fail(ctx, REVNET_E_WORKSPACE_TOO_SMALL, "revnet_pack_weights: pack buffer holds " + std::to_string(pack_bytes) + " bytes, " + std::to_string(need) + " needed");
+    Exec ex; ex.ctx = ctx; ex.dry = false; ex.mode = d->mode; ex.eps = d->eps; ex.stream = (cudaStream_t)stream;
+    char *at = (char *)pack_buffer;
+    revnet_fn_params *ps[2] = {Fp, Gp};
+    const revnet_fn_desc *fs[2] = {&d->F, &d->G};
+    for (int i = 0; i < 2; i++)
+        for (int l = 0; l < 3; l++) {
+            ps[i]->Wpack_fprop[l] = ps[i]->Wpack_dgrad[l] = nullptr;
+            if (l >= fs[i]->n_layers || !packable(d, *fs[i], l)) continue;
+            for (int tr = 0; tr < 2; tr++) {
+                tc_pack_now(ex, ps[i]->W[l], (bf16 *)at, fs[i]->cin[l], fs[i]->cout[l], fs[i]->k[l], tr != 0);
+                (tr ? ps[i]->Wpack_dgrad[l] : ps[i]->Wpack_fprop[l]) = at;
+                at += (tc_pack_elems(fs[i]->cin[l], fs[i]->cout[l], fs[i]->k[l], tr != 0) * sizeof(bf16) + 255) & ~size_t(255);
+            }
+        }
+    return finish(ctx, ex, "revnet_pack_weights");
+}
+
 // ---- block forward on the library's own static scratch: for callers that cannot allocate
 // Some integrations run where device allocation is off the table: inside a memory pool whose owner
 // forbids side allocations, in a real-time or safety-checked loop that must not touch the
@@ -170,7 +222,7 @@ extern "C" int revnet_block_bwd(revnet_ctx *ctx, const revnet_block_desc *d, con
 static __device__ __align__(256) unsigned char g_noalloc_scratch[REVNET_NOALLOC_SCRATCH_BYTES];
 // device address of the array, looked up once per device (the array's name is only a host-side
 // handle in host code and must never be handed to a kernel as if it were a pointer)
-static void *g_noalloc_ptr[64] = {};
+static std::atomic<void *> g_noalloc_ptr[64];
 
 extern "C" int revnet_block_fwd_noalloc(revnet_ctx *ctx, const revnet_block_desc *d, const void *x1, const void *x2,
                                         const revnet_fn_params *Fp, const revnet_fn_params *Gp, void *y1, void *y2, void *stream) {
@@ -190,17 +242,18 @@ extern "C" int revnet_block_fwd_noalloc(revnet_ctx *ctx, const revnet_block_desc
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64)
         return fail(ctx, REVNET_E_CUDA, "revnet_block_fwd_noalloc: no current device");
     if (dev != ctx->device) return fail(ctx, REVNET_E_INVALID_ARG, "revnet_block_fwd_noalloc: the context's device must be current");
-    if (!g_noalloc_ptr[dev]) {
-        // one-time set-up for this device (with it current): resolve the array's device address
-        void *p = nullptr;
-        cudaError_t e = cudaGetSymbolAddress(&p, g_noalloc_scratch);
-        if (e != cudaSuccess || !p)
+    void *scratch = g_noalloc_ptr[dev].load(std::memory_order_acquire);
+    if (!scratch) {
+        // one-time set-up for this device (with it current): resolve the array's device address.  Two threads that
+        // race here both get the same address from the runtime.
+        cudaError_t e = cudaGetSymbolAddress(&scratch, g_noalloc_scratch);
+        if (e != cudaSuccess || !scratch)
             return fail(ctx, REVNET_E_CUDA, std::string("revnet_block_fwd_noalloc: cudaGetSymbolAddress: ") + cudaGetErrorString(e));
-        g_noalloc_ptr[dev] = p;
+        g_noalloc_ptr[dev].store(scratch, std::memory_order_release);
     }
     Exec ex; ex.ctx = ctx; ex.dry = false; ex.mode = d->mode; ex.eps = d->eps; ex.stream = (cudaStream_t)stream;
     ex.q = d->state_frac_bits ? ldexpf(1.f, -d->state_frac_bits) : 0.f;
-    ex.ws.dry = false; ex.ws.base = (char *)g_noalloc_ptr[dev]; ex.ws.cap = REVNET_NOALLOC_SCRATCH_BYTES;
+    ex.ws.dry = false; ex.ws.base = (char *)scratch; ex.ws.cap = REVNET_NOALLOC_SCRATCH_BYTES;
     // nothing in the block forward relies on zeroed scratch: every region is written before it is read
     block_forward(ex, Geom{d->N, d->H, d->W}, d->c, layers_of(d->F, Fp, nullptr), layers_of(d->G, Gp, nullptr),
                   (float *)x1, (float *)x2, (float *)y1, (float *)y2);
@@ -300,10 +353,31 @@ extern "C" int revnet_check_device(revnet_ctx *ctx, void *stream) {
         cudaStreamSynchronize(s) != cudaSuccess)
         return fail(ctx, REVNET_E_CUDA, std::string("revnet_check_device: ") + cudaGetErrorString(cudaGetLastError()));
     if (st != 0) {
-        cudaMemsetAsync(ctx->dev_status, 0, sizeof(int), s);
+        // a kernel that gave up never counted itself out of its grid-wide reduction: zero the counter words as well,
+        // or a later kernel handed the same word would elect its last CTA too early
+        cudaMemsetAsync(ctx->dev_status, 0, 1024, s);
         cudaStreamSynchronize(s);
         return fail(ctx, st, "a kernel gave up a bounded wait (device status " + std::to_string(st) + ")");
     }
+    return REVNET_OK;
+}
+
+// One CTA waits, with the caller's limit, on a shared-memory barrier that nothing arrives on: the wait runs out,
+// the kernel records the status and returns normally -- the path every bounded wait in the library takes on expiry.
+__global__ void selftest_wait_kernel(unsigned long long limit_ns, int *status) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        tc::mbar_init(&bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!tc::mbar_wait(&bar, 0, limit_ns)) atomicExch(status, (int)REVNET_E_TIMEOUT);
+    }
+}
+extern "C" int revnet_selftest_bounded_wait(revnet_ctx *ctx, uint64_t limit_ns, void *stream) {
+    if (!ctx || !ctx->dev_status) return REVNET_E_INVALID_ARG;
+    if (limit_ns == 0 || limit_ns > 100000000ull) return fail(ctx, REVNET_E_INVALID_ARG, "revnet_selftest_bounded_wait: limit must be in (0, 100 ms]");
+    selftest_wait_kernel<<<1, 32, 0, (cudaStream_t)stream>>>((unsigned long long)limit_ns, ctx->dev_status);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return fail(ctx, REVNET_E_CUDA, std::string("revnet_selftest_bounded_wait: ") + cudaGetErrorString(e));
     return REVNET_OK;
 }
 

@@ -36,6 +36,19 @@ struct revnet_ctx {
     cudaEvent_t next_event();
 };
 
+// Function attributes (the dynamic shared-memory limit) belong to a device, not to the process: each kernel's
+// launcher keeps one of these and sets its attributes the first time it runs on a device.  Setting them twice
+// is harmless, so no lock: two threads that race both set the same value.
+struct OncePerDevice {
+    bool done[64] = {};
+    bool first(int device) {
+        if (device < 0 || device >= 64) return true;
+        if (done[device]) return false;
+        done[device] = true;
+        return true;
+    }
+};
+
 // A tensor of C = c0 + c1 channels stored as two NHWC tensors: channels [0,c0) in p0 (row
 // stride c0) and [c0,c0+c1) in p1 (row stride c1).  c1 == 0: one plain tensor.
 // q == 0: elements are float.  q > 0: elements are int32 fixed point, value = i * q with

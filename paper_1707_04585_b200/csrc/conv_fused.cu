@@ -639,8 +639,8 @@ bool run_fused(Exec &ex, const char *what, int in_mode, const void *in, float in
         e.inv_count = 1.0 / (double)g.P(); e.eps = ex.eps;
         if (req.stats) { e.mean = req.stats->mean; e.rstd = req.stats->rstd; }
         if (req.bnbwd) { e.t = req.bnbwd->t; e.bn = req.bnbwd->bn; e.dgamma = req.bnbwd->dgamma; e.dbeta = req.bnbwd->dbeta; e.coef = req.bnbwd->coef; }
-        static bool attr_set = false;
-        if (!attr_set) { cudaFuncSetAttribute(conv_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024); attr_set = true; }
+        static OncePerDevice once;
+        if (once.first(ex.ctx->device)) cudaFuncSetAttribute(conv_fused_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         dim3 grid((unsigned)ctas, (unsigned)s.n_tiles);
         launch(ex, conv_fused_kernel, grid, kFThreads, s.smem, map_w, map_in, map_aux, map_out, p);
         const double bytes = (double)g.P() * cin * (in_mode == 0 ? 4 : 2) + (double)g.P() * cout * (sign || req.bnbwd ? 8 : 4) +

@@ -10,9 +10,10 @@
 // dgrad is the same kernel run on the upstream gradient with the tap-mirrored, transposed pack
 // of the weights.  Each entry point returns false for shapes it does not take.
 //
-// Roles inside a CTA (192 threads): warp 0 issues TMA loads, warp 1 allocates tensor memory and
-// issues the MMAs, warps 2..5 drain the accumulator (tcgen05.ld), apply the coupling epilogue
-// (out = partner +/- acc on the float or fixed-point state) and store.
+// Roles inside a CTA: warp 0 issues TMA loads, warp 1 allocates tensor memory and issues the MMAs,
+// the remaining warps drain the accumulator (tcgen05.ld), apply the coupling epilogue (out = partner
+// +/- acc on the float or fixed-point state) and store: two groups of four warps (320 threads) where
+// the epilogue's tiles move through TMA, one group (192 threads) in the staged form.
 // Every mbarrier wait is bounded; on expiry the kernel records a status word and leaves.
 #include "common.cuh"
 #include "tc_ptx.cuh"
@@ -623,8 +624,8 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         e.inv_count = 1.0 / ((double)g.P() * ostride * ostride); e.eps = ex.eps;     // pixels of the output grid
         if (req.stats) { e.mean = req.stats->mean; e.rstd = req.stats->rstd; }
         if (req.bnbwd) { e.t = req.bnbwd->t; e.bn = req.bnbwd->bn; e.dgamma = req.bnbwd->dgamma; e.dbeta = req.bnbwd->dbeta; e.coef = req.bnbwd->coef; }
-        static bool attr_set = false;
-        if (!attr_set) { cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024); attr_set = true; }
+        static OncePerDevice once;
+        if (once.first(ex.ctx->device)) cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
         dim3 grid((unsigned)ctas, (unsigned)s.n_tiles);
         launch(ex, conv_tc_kernel, grid, epi_tma ? kThreadsTma : kThreads, s.smem, map_a, map_b, map_o[0], map_o[1], map_x[0], map_x[1], p);
         const double bytes = (double)gin.P() * cin * 2 + (double)g.P() * cout * (sign || req.bnbwd ? 8 : 4) + (double)cout * taps * cin * 2;
@@ -1036,8 +1037,8 @@ bool conv_wgrad_tc_batch(Exec &ex, int n, const void *const *gq, const void *con
             bytes += (double)gi[j].P() * L[j]->cin * 2 + (double)w[j].go.P() * L[j]->cout * 2 + (double)p.slice * 4 * p.splits;
             flops += 2.0 * w[j].go.P() * L[j]->cout * L[j]->cin * p.taps;
         }
-        static bool attr_set = false;
-        if (!attr_set) { cudaFuncSetAttribute(wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWgSmemMax); attr_set = true; }
+        static OncePerDevice once;
+        if (once.first(ex.ctx->device)) cudaFuncSetAttribute(wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWgSmemMax);
         launch(ex, wgrad_tc_kernel, (unsigned)cta, kThreads, smem, batch);
         ex.check("conv_wgrad_tc", bytes, flops);
         if (n_sums) {

@@ -485,8 +485,10 @@ __global__ void fc_fwd_kernel(const float *__restrict__ feat, const float *__res
 }
 
 // one warp per sample: stable log-sum-exp, dlogits = (softmax - onehot)/N, arg-max (lowest index on ties)
+// A label outside [0, K) is reported, not followed: nothing is read at it, the sample's loss becomes NaN and the
+// context's status word is set to REVNET_E_INVALID_ARG (revnet_check_device returns it).
 __global__ void softmax_ce_kernel(const float *__restrict__ logits, const int32_t *__restrict__ labels, int N, int K,
-                                  float *__restrict__ dlogits, float *__restrict__ loss_n, int32_t *__restrict__ pred) {
+                                  float *__restrict__ dlogits, float *__restrict__ loss_n, int32_t *__restrict__ pred, int *status) {
     pdl_enter();
     int n = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (n >= N) return;
@@ -501,9 +503,14 @@ __global__ void softmax_ce_kernel(const float *__restrict__ logits, const int32_
     for (int k = lane; k < K; k += 32) s += expf(z[k] - m);
     for (int o = 16; o; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
     const int lab = labels[n];
+    const bool lab_ok = lab >= 0 && lab < K;
     const float inv = 1.f / s, invN = 1.f / (float)N;
     for (int k = lane; k < K; k += 32) dlogits[(size_t)n * K + k] = (expf(z[k] - m) * inv - (k == lab ? 1.f : 0.f)) * invN;
-    if (lane == 0) { loss_n[n] = m + logf(s) - z[lab]; pred[n] = mi; }
+    if (lane == 0) {
+        loss_n[n] = lab_ok ? m + logf(s) - z[lab] : __int_as_float(0x7fc00000);
+        pred[n] = mi;
+        if (!lab_ok && status) atomicCAS(status, 0, (int)REVNET_E_INVALID_ARG);
+    }
 }
 
 __global__ void mean_kernel(const float *__restrict__ v, int N, float *out) {
@@ -527,7 +534,7 @@ void head_fwd(Exec &ex, Pair y, int N, int HW, const float *Wfc, const float *bf
         ex.check("avgpool");
         launch(ex, fc_fwd_kernel, cdiv((size_t)N * K * 32, 256), 256, 0, feat, Wfc, bfc, N, C, K, logits);
         ex.check("fc_fwd");
-        launch(ex, softmax_ce_kernel, cdiv((size_t)N * 32, 256), 256, 0, logits, labels, N, K, dlogits, loss_n, pred);
+        launch(ex, softmax_ce_kernel, cdiv((size_t)N * 32, 256), 256, 0, logits, labels, N, K, dlogits, loss_n, pred, ex.ctx->dev_status);
         ex.check("softmax_ce");
         launch(ex, mean_kernel, 1, 32, 0, loss_n, N, loss);
         ex.check("loss_mean");

@@ -42,6 +42,8 @@ struct revnet_plan {
     void *pack_host = nullptr;      // page-locked staging for the weight-pack job table
     size_t pack_host_bytes = 0;
     // the step captured as a CUDA graph, valid for one set of buffer addresses
+    size_t bound_act = 0, bound_ws = 0;   // sizes of the caller's buffers, if declared (revnet_plan_set_buffer_sizes)
+    bool bound = false;
     cudaGraphExec_t graph_exec = nullptr;
     const void *graph_key[10] = {};
     revnet_step_stats graph_stats = {};
@@ -434,6 +436,23 @@ extern "C" int revnet_plan_scratch_split(const revnet_plan *pl, size_t *param_sc
     return REVNET_OK;
 }
 
+extern "C" int revnet_plan_set_buffer_sizes(revnet_plan *pl, size_t activation_bytes, size_t workspace_bytes) {
+    if (!pl) return REVNET_E_INVALID_ARG;
+    pl->bound_act = activation_bytes; pl->bound_ws = workspace_bytes; pl->bound = true;
+    return REVNET_OK;
+}
+
+// status word of the device as it stands (the caller has just synchronised the stream); not cleared here
+static int read_device_status(revnet_ctx *ctx, cudaStream_t s) {
+    int st = 0;
+    if (!ctx->dev_status) return 0;
+    if (cudaMemcpyAsync(&st, ctx->dev_status, sizeof(int), cudaMemcpyDeviceToHost, s) != cudaSuccess || cudaStreamSynchronize(s) != cudaSuccess) {
+        cudaGetLastError();
+        return REVNET_E_CUDA;
+    }
+    return st;
+}
+
 extern "C" int revnet_plan_destroy(revnet_plan *pl) {
     if (!pl) return REVNET_OK;
     if (pl->pinned) { if (pl->pinned_is_malloc) free(pl->pinned); else cudaFreeHost(pl->pinned); }
@@ -451,6 +470,9 @@ extern "C" int revnet_train_step(revnet_ctx *ctx, revnet_plan *pl, const float *
     const void *ptrs[] = {images, params, grads, momentum, activations, workspace};
     for (const void *p : ptrs)
         if ((uintptr_t)p & 15) return fail(ctx, REVNET_E_MISALIGNED, "revnet_train_step: pointers must be 16-byte aligned");
+    if (pl->bound && (pl->bound_act < pl->act_bytes || pl->bound_ws < pl->ws_bytes))
+        return fail(ctx, REVNET_E_WORKSPACE_TOO_SMALL, "revnet_train_step: buffers declared as " + std::to_string(pl->bound_act) + " / " +
+                    std::to_string(pl->bound_ws) + " bytes (activations / workspace), the plan needs " + std::to_string(pl->act_bytes) + " / " + std::to_string(pl->ws_bytes));
     const bool use_graph = pl->d.use_cuda_graph && !pl->d.verify_reconstruction && !ctx->profiling && ctx->capture_stream;
     const void *key[10] = {images, labels, params, grads, momentum, activations, workspace, loss, pred, logits};
     if (use_graph && pl->graph_exec && memcmp(key, pl->graph_key, sizeof key) == 0) {
@@ -499,6 +521,7 @@ extern "C" int revnet_train_step(revnet_ctx *ctx, revnet_plan *pl, const float *
         if (cudaMemcpyAsync(stats->recon_max_abs, recon, sizeof(float) * REVNET_MAX_STAGES, cudaMemcpyDeviceToHost, ex.stream) != cudaSuccess ||
             cudaStreamSynchronize(ex.stream) != cudaSuccess)
             return fail(ctx, REVNET_E_CUDA, std::string("revnet_train_step: ") + cudaGetErrorString(cudaGetLastError()));
+        stats->device_status = read_device_status(ctx, ex.stream);      // the stream is idle here: the word is final for this step
     }
     return REVNET_OK;
 }
@@ -522,5 +545,9 @@ extern "C" int revnet_train_step_host(revnet_ctx *ctx, revnet_plan *pl, const fl
         cudaMemcpyAsync(pred_host, pred_dev, (size_t)d.N * 4, cudaMemcpyDeviceToHost, s) != cudaSuccess ||
         cudaStreamSynchronize(s) != cudaSuccess)
         return fail(ctx, REVNET_E_CUDA, std::string("revnet_train_step_host: D2H copy: ") + cudaGetErrorString(cudaGetLastError()));
+    // this call has synchronised: report what the step's kernels recorded (revnet_check_device clears it)
+    const int st = read_device_status(ctx, s);
+    if (stats) stats->device_status = st;
+    if (st) return fail(ctx, st, "revnet_train_step_host: a kernel of the step recorded device status " + std::to_string(st));
     return REVNET_OK;
 }

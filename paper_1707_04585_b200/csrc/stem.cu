@@ -221,11 +221,10 @@ bool stem_fprop(Exec &ex, const float *img, Geom gi, const Layer &L, Pair out) {
     const int P = g.N * g.Ho * g.Wo, n_tiles = (P + kFPx - 1) / kFPx;
     int per_sm = (int)((220 * 1024) / (smem + 1024)); if (per_sm > 8) per_sm = 8; if (per_sm < 1) per_sm = 1;
     int grid = ex.ctx->sm_count * per_sm; if (grid > n_tiles) grid = n_tiles;
-    static bool attr_set = false;
-    if (!attr_set) {
+    static OncePerDevice once;
+    if (once.first(ex.ctx->device)) {
         cudaFuncSetAttribute(stem_fprop_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
         cudaFuncSetAttribute(stem_fprop_kernel<8>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-        attr_set = true;
     }
     if (CO_T == 8) launch(ex, stem_fprop_kernel<8>, grid, 256, smem, img, L.W, out, g, cop, n_tiles);
     else launch(ex, stem_fprop_kernel<4>, grid, 256, smem, img, L.W, out, g, cop, n_tiles);
@@ -251,11 +250,10 @@ bool stem_wgrad(Exec &ex, const float *img, const float *gout, Geom gi, const La
     size_t m = ex.ws.mark();
     float *part = ex.ws.get<float>((size_t)grid * g.Co * g.K);
     if (!ex.dry) {
-        static bool attr_set = false;
-        if (!attr_set) {
+        static OncePerDevice once;
+        if (once.first(ex.ctx->device)) {
             cudaFuncSetAttribute(stem_wgrad_kernel<8, 12>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
             cudaFuncSetAttribute(stem_wgrad_kernel<4, 4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-            attr_set = true;
         }
         if (big) launch(ex, stem_wgrad_kernel<8, 12>, grid, 256, smem, img, gout, part, g, cop, kp, n_cg, G, S, n_chunks);
         else launch(ex, stem_wgrad_kernel<4, 4>, grid, 256, smem, img, gout, part, g, cop, kp, n_cg, G, S, n_chunks);

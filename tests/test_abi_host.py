@@ -107,3 +107,21 @@ def test_bad_descriptors_are_rejected(ctx):
     bd = B.block_desc(syn.block_config_1(), 1); bd.G.cout[0] = 12
     with pytest.raises(B.RevnetError):
         B.revnet_block_workspace_bytes(ctx, bd)
+
+
+def test_pack_bytes_and_declared_buffer_sizes(ctx):
+    """Host logic of the pre-packed weights and of the declared buffer sizes (no kernel runs)."""
+    b = syn.BlockCfg(2, 8, 8, 128, 32, "bottleneck", seed=1)
+    n0 = B.revnet_block_pack_bytes(ctx, B.block_desc(b, 0, 16))
+    # two packs (forward, data gradient) of cout x taps x cin bf16 per layer, rows and columns padded to 16, 256-byte slots
+    expect = 0
+    for (ci, co, k) in syn.fn_layers(b.kind, b.c, b.w) * 2:
+        expect += 2 * ((co * k * k * ci * 2 + 255) // 256 * 256)
+    assert n0 == expect
+    assert B.revnet_block_pack_bytes(ctx, B.block_desc(b, 1, 0)) == 0          # strict fp32 mode has no packs
+    odd = syn.BlockCfg(2, 8, 8, 12, 0, "basic", seed=1)                        # 12 channels: the fp32 kernels take it, no pack
+    assert B.revnet_block_pack_bytes(ctx, B.block_desc(odd, 0, 16)) == 0
+    cfg = hp.tiny_stack("basic")
+    plan = B.revnet_stack_plan(ctx, B.stack_desc(cfg, 0))
+    plan.set_buffer_sizes(plan.activation_bytes, plan.workspace_bytes)
+    plan.close()

@@ -66,8 +66,8 @@ def test_stored_step_strict_mode_against_oracle_and_reversible(ctx, kind, maxpoo
     o = orc.stack_train_grads(net, inp["images"], inp["labels"], "stored")
     assert hp.rel_l2(sto["logits"], o["logits"]) <= 1e-4
     for k in o["grads"]:
-        assert hp.rel_l2(sto["grads"][k], o["grads"][k]) <= 1e-3, k
-        assert hp.rel_l2(sto["grads"][k], rev["grads"][k]) <= 1e-3, k
+        assert hp.rel_l2(sto["grads"][k], o["grads"][k]) <= 1e-4, k
+        assert hp.rel_l2(sto["grads"][k], rev["grads"][k]) <= 1e-4, k
 
 
 def test_stored_step_at_benchmark_width_and_storage_growth(ctx):

@@ -195,8 +195,10 @@ def test_block_gradients_match_central_differences(kind):
 
 
 # ------------------------------------------------------------------ stack
-def torch_stack_grads(cfg, inp):
-    """Independent route: the same network written with library ops and differentiated by autograd."""
+def torch_stack_grads(cfg, inp, taps=None):
+    """Independent route: the same network written with library ops and differentiated by autograd.
+    taps (a dict) receives the tensors between the layers -- ("x"|"y", stage, unit) -> (t1, t2) with
+    their gradients retained, ("T", stage) -> (input, output) of a stored transition."""
     P = {k: torch.tensor(v.astype(np.float64), requires_grad=True) for k, v in inp["params"].items()}
     bnrc = lambda t, pre, s=1: TF.conv2d(TF.relu(TF.batch_norm(t, None, None, P[pre + ".gamma"], P[pre + ".beta"],
                                                                training=True, eps=cfg.eps)),
@@ -206,10 +208,18 @@ def torch_stack_grads(cfg, inp):
         h = TF.max_pool2d(h, 3, 2, 1)
     for si, s in enumerate(cfg.stages):
         if s.trans_k:
+            hin = h
             h = bnrc(h, f"s{si}.T", s.trans_stride)
+            if taps is not None:
+                hin.retain_grad(); h.retain_grad()
+                taps[("T", si)] = (hin, h)
         x1, x2 = h[:, :s.c], h[:, s.c:]
         nl = len(syn.fn_layers(s.kind, s.c, s.w))
         for u in range(s.units):
+            if taps is not None:
+                x1, x2 = x1 * 1.0, x2 * 1.0           # fresh nodes, so that each unit's input gradient can be read
+                x1.retain_grad(); x2.retain_grad()
+                taps[("x", si, u)] = (x1, x2)
             f = x2
             for li in range(nl):
                 f = bnrc(f, f"s{si}.u{u}.F.l{li}")
@@ -218,6 +228,9 @@ def torch_stack_grads(cfg, inp):
             for li in range(nl):
                 g = bnrc(g, f"s{si}.u{u}.G.l{li}")
             x2 = x2 + g
+            if taps is not None:
+                x1.retain_grad(); x2.retain_grad()
+                taps[("y", si, u)] = (x1, x2)
         h = torch.cat([x1, x2], dim=1)
     logits = h.mean(dim=(2, 3)) @ P["fc.W"].T + P["fc.b"]
     loss = TF.cross_entropy(logits, torch.tensor(inp["labels"].astype(np.int64)))
@@ -242,6 +255,35 @@ def test_stack_against_autograd_and_reconstruct_equals_stored(kind, maxpool):
         f1, f2 = rr["block_inputs"][key]
         assert np.abs(x1 - f1).max() < 1e-11 and np.abs(x2 - f2).max() < 1e-11
     assert np.array_equal(rs["pred"], tl.argmax(axis=1))
+
+
+def test_per_block_records_inside_a_stack_match_autograd():
+    """The (y1,y2,dy1,dy2) -> (dx1,dx2) the oracle reports for single blocks and transitions inside a
+    network equal what autograd sees at the same places (Section 3.2: Algorithm 1 applied block by block)."""
+    cfg = hp.tiny_stack("bottleneck", True, units=3)
+    inp = syn.make_stack_inputs(cfg, affine_jitter=True)
+    net = hp.oracle_net(cfg, inp["params"])
+    keys = {(0, 0), (0, 2), (1, 1)}
+    rr = orc.stack_train_grads(net, inp["images"], inp["labels"], "reconstruct", keep_blocks=keys, keep_transitions=True)
+    taps = {}
+    torch_stack_grads(cfg, inp, taps)
+    assert set(rr["blocks"]) == keys
+    for (si, u), b in rr["blocks"].items():
+        (x1, x2), (y1, y2) = taps[("x", si, u)], taps[("y", si, u)]
+        for got, ref in ((b["y1"], y1.detach()), (b["y2"], y2.detach()), (b["dy2"], y2.grad), (b["dx1"], x1.grad), (b["dx2"], x2.grad)):
+            assert hp.rel_l2(got, ref.numpy()) < 1e-9, (si, u)
+        # y1 feeds G as well as the next layer: the gradient Algorithm 1 is handed for it is the direct part only
+        # (autograd's total minus G's share), i.e. dx1 = dy1 + (dG/dy1)^T dy2  =>  check through dx1 above and here
+        g = {}
+        F, G = net["stages"][si]["units"][u]
+        _, _, d1, d2 = orc.block_bwd_reconstruct(b["y1"], b["y2"], b["dy1"], b["dy2"], F, G, net["eps"], g)
+        assert hp.rel_l2(d1, b["dx1"]) < 1e-12 and hp.rel_l2(d2, b["dx2"]) < 1e-12
+        for k, v in g.items():
+            assert hp.rel_l2(v, rr["grads"][k]) < 1e-12, k
+    for si, t in rr["transitions"].items():
+        hin, hout = taps[("T", si)]
+        assert hp.rel_l2(t["x"], hin.detach().numpy()) < 1e-10
+        assert hp.rel_l2(t["dy"], hout.grad.numpy()) < 1e-9 and hp.rel_l2(t["dx"], hin.grad.numpy()) < 1e-9
 
 
 def test_storage_flat_in_depth_and_cost_4n_vs_3n():

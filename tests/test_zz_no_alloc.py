@@ -27,10 +27,16 @@ def test_noalloc_block_forward_matches_workspace_version_twice(mode):
         ref1, ref2 = torch.empty_like(x1), torch.empty_like(x2)
         B.revnet_block_fwd(ctx, r.desc, x1, x2, r.F, r.G, ref1, ref2, r.ws)
         y1, y2 = torch.empty_like(x1), torch.empty_like(x2)
-        before = torch.cuda.memory_allocated()
+        torch.cuda.synchronize()
+        # free device memory as the driver sees it (torch's own counters cannot see what a library allocates)
+        free_before = torch.cuda.mem_get_info()[0]
         B.revnet_block_fwd_noalloc(ctx, r.desc, x1, x2, r.F, r.G, y1, y2)
         torch.cuda.synchronize()
-        assert torch.cuda.memory_allocated() == before
+        free_after = torch.cuda.mem_get_info()[0]
+        if call == 1:
+            # the first call on a device may make the runtime place the library's image (with the array) there;
+            # from the second call on nothing on the device may change hands
+            assert free_after == free_before, (free_before, free_after)
         # same kernels, same order, same inputs: identical bits (well inside the parity tolerances)
         assert torch.equal(y1, ref1) and torch.equal(y2, ref2)
         assert not torch.equal(y1, x1)

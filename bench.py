@@ -1,10 +1,13 @@
 #!/usr/bin/env python
 """Benchmark: RevNet train-step images/sec on B200 (one replica per GPU, no collectives).
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--config revnet38] [--impl ours|reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config revnet104] [--impl ours|reference]
 
 A step is one whole train step of the stack (forward, reconstructing backward through every
-stage, SGD update) on one synthetic batch.  Prints ONE JSON line (rank 0).
+stage, SGD update) on one synthetic batch.  The headline workload is the largest configuration
+that fits one GPU (the large-image bottleneck network, batch 64 of 224x224); the three CIFAR-sized
+configurations are timed in the same run and reported under "other_workloads".
+Prints ONE JSON line (rank 0).
 """
 import argparse
 import json
@@ -158,11 +161,37 @@ def cpu_baseline(cfg, sample_n, steps=1):
                 seconds_per_step=float(np.mean(times)))
 
 
+def ref_batch(args, cfg):
+    """Batch of the bounded oracle sample: about 10-30 s of CPU work per step."""
+    if args.ref_batch:
+        return max(2, min(cfg.N, args.ref_batch))
+    return 2 if cfg.img > 64 else min(cfg.N, 32)
+
+
+def time_steps(run, steps, warmup, flush, stream):
+    """Device time (ms, summed) of `steps` train steps from the initial weights, L2 flushed in between."""
+    import torch
+    p0 = run.params.clone()
+    for _ in range(warmup):
+        run.params.copy_(p0); run.momentum.zero_()
+        st = run.step(want_logits=False)
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    for a, b in ev:
+        run.params.copy_(p0); run.momentum.zero_()
+        flush.zero_()
+        a.record(stream)
+        st = run.step(want_logits=False)
+        b.record(stream)
+    torch.cuda.synchronize()
+    return sum(a.elapsed_time(b) for a, b in ev), st
+
+
 def run_reference(args, cfg):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    sample = max(2, min(cfg.N, args.ref_batch))
+    sample = ref_batch(args, cfg)
     t0 = time.perf_counter()
     cb = cpu_baseline(cfg, sample, steps=1)            # untimed warm-up of caches is not separated: the oracle is timed as it stands
     k = max(1, min(args.steps, int(60.0 / max(cb["seconds_per_step"], 1e-3))))
@@ -329,6 +358,26 @@ def run_ours(args, cfg):
             bc = syn.BlockCfg(rcfg.N, H, H, s_cfg.c, s_cfg.w, s_cfg.kind, seed=9)
             block_ms[f"{s_cfg.kind}_c{s_cfg.c}_{H}x{H}"] = R.time_block(ctx, bc, 0, reps=5, warmup=3)
 
+    # ---- the other configurations, same timing rules, fewer steps (rank 0, single-GPU runs only)
+    others = {}
+    if rank == 0 and world == 1 and not args.no_others:
+        del run
+        torch.cuda.empty_cache()
+        for oname in syn.STACK_NAMES:
+            if oname == cfg.name:
+                continue
+            ocfg = syn.stack_config(oname)
+            oin = syn.make_stack_inputs(ocfg)
+            orun = R.StackRunner(ctx, ocfg, mode=0)
+            orun.load(oin["images"], oin["labels"], oin["params"])
+            n_o = max(5, min(args.steps, 30))
+            oms, ost = time_steps(orun, n_o, args.warmup, flush, stream)
+            others[oname] = dict(ms_per_step=oms / n_o, images_per_sec=ocfg.N * n_o / (oms * 1e-3), steps=n_o, batch=ocfg.N,
+                                 activation_bytes=int(ost.stored_activation_bytes), flops_per_step=int(ost.flops_fwd + ost.flops_bwd),
+                                 gpu_launches_per_step=int(ost.kernel_launches))
+            del orun
+            torch.cuda.empty_cache()
+
     dev_ms, e2e_ms = max_over_ranks([dev_ms, e2e_ms], world, "cuda")
     if rank == 0:
         peaks = load_peaks()
@@ -346,7 +395,19 @@ def run_ours(args, cfg):
             ach, peak, runit = rec["flops"] / rec["launches"] / avg_s / 1e12, peaks["tc_sustained"], "TFLOP/s"
         else:
             ach, peak, runit = rec["flops"] / rec["launches"] / avg_s / 1e12, ALU_FP32_TFLOPS, "TFLOP/s"
-        roof = dict(bound=bound, achieved=ach, peak=peak, unit=runit, frac=ach / peak, traffic=measured_traffic(name, cfg.name), kernel=name,
+        # the step as a whole against both rooflines: algorithmic bytes and flops of all its kernels over the
+        # graph-replayed step time (the per-kernel spans above come from a step enqueued kernel by kernel on ONE
+        # stream, events in between: they add up to more than the replayed step, which overlaps weight gradients
+        # and the recomputation of F with the main chain and has no events between launches)
+        step_s = dev_ms / args.steps * 1e-3
+        step_bytes = sum(v["bytes"] for v in prof.values()) / psteps
+        step_flops = sum(v["flops"] for v in prof.values()) / psteps
+        whole = dict(algorithmic_gb=step_bytes / 1e9, tflop=step_flops / 1e12,
+                     gbs=step_bytes / step_s / 1e9, frac_hbm=step_bytes / step_s / 1e9 / peaks["hbm"],
+                     tflops=step_flops / step_s / 1e12, frac_tensor=step_flops / step_s / 1e12 / peaks["tc_sustained"],
+                     roofline_ms=sum(max(v["bytes"] / (peaks["hbm"] * 1e9), v["flops"] / (peaks["tc_sustained"] * 1e12)) for v in prof.values()) / psteps * 1e3,
+                     profiled_serial_ms=tot / psteps)
+        roof = dict(bound=bound, achieved=ach, peak=peak, unit=runit, frac=ach / peak, traffic=measured_traffic(name, cfg.name), kernel=name, whole_step=whole,
                     kernel_share=rec["ms"] / tot, avg_launch_us=avg_s * 1e6, peak_source=peaks["source"],
                     kernels={k: dict(launches=v["launches"] // psteps, ms_per_step=v["ms"] / psteps, share=v["ms"] / tot,
                                      gbs=(v["bytes"] / (v["ms"] * 1e-3) / 1e9) if v["ms"] > 0 else None,
@@ -369,8 +430,10 @@ def run_ours(args, cfg):
             stored["reversible_over_stored_time"] = (dev_ms / args.steps) / stored["ms_per_step"]
             stored["reversible_over_stored_bytes"] = int(st.stored_activation_bytes) / stored["stored_activation_bytes"]
             line["stored_activation_step"] = stored
+        if others:
+            line["other_workloads"] = others
         if not args.no_cpu and world == 1:
-            line["cpu_baseline"] = {k: v for k, v in cpu_baseline(cfg, min(cfg.N, args.ref_batch)).items() if k != "seconds_per_step"}
+            line["cpu_baseline"] = {k: v for k, v in cpu_baseline(cfg, ref_batch(args, cfg)).items() if k != "seconds_per_step"}
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()
@@ -381,9 +444,10 @@ def main():
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
-    ap.add_argument("--config", default="revnet38")
+    ap.add_argument("--config", default="revnet104")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--ref-batch", type=int, default=32, help="batch of the bounded CPU-oracle sample")
+    ap.add_argument("--ref-batch", type=int, default=0, help="batch of the bounded CPU-oracle sample (0: 2 for 224x224 images, else 32)")
+    ap.add_argument("--no-others", action="store_true", help="skip timing the other configurations")
     ap.add_argument("--no-cpu", action="store_true", help="skip the CPU-oracle leg")
     ap.add_argument("--no-stored", action="store_true", help="skip the stored-activation comparison step")
     args = ap.parse_args()

@@ -205,6 +205,13 @@ typedef struct {
     int kind;          /* 0: F,G = one conv3x3; 1: basic (3x3,3x3); 2: bottleneck (1x1,3x3,1x1) */
     int trans_k;       /* stored BN-ReLU-conv transition in front of the stage (0 = none) */
     int trans_stride;  /* 1 or 2 */
+    int down;          /* 1: paper-shaped stage (Table "Architectural details" counts the down-sampling inside the
+                          first unit of a stage): no transition (trans_k = 0); the first of the `units` units is a
+                          stored, non-invertible coupling unit  y1 = S(x1) + F(x2), y2 = S(x2) + G(y1)  on the
+                          previous stage's output, S = 2x2 average pooling (stride 2) followed by zero channels up to
+                          c, F with one stride-2 layer (the first 3x3 of a basic function, the 3x3 of a bottleneck);
+                          the other units - 1 units are reversible.  Its parameters come first in the stage: F layers
+                          (gamma, beta, W each), then G layers.  Not for stage 0. */
 } revnet_stage_desc;
 
 #define REVNET_MAX_STAGES 8

@@ -8,8 +8,11 @@ Structures (plain Python, built by the caller):
   function = list of layers, applied first to last; each layer is conv(relu(bn(.)))   (Section 2.2, Eq. 2)
   block    = (F, G)                                                                     (Section 3.1)
   net      = {"stem": {"name","W","stride","pad"}, "maxpool": bool,
-              "stages": [{"trans": layer or None, "c": int, "units": [block, ...]}],
+              "stages": [{"trans": layer or None, "down": block or None, "c": int, "units": [block, ...]}],
               "fc": {"name","W":[K,C],"b":[K]}, "eps": float}
+  A stage's "down" block is the paper-shaped way into the stage (Table "Architectural details" counts the
+  down-sampling layer inside the first unit of a stage): a coupling unit whose F contains a stride-2
+  layer and whose skip paths are parameter-free shortcuts; it is not invertible, so its input is kept.
 """
 import ctypes
 import os
@@ -237,6 +240,45 @@ def block_bwd_reconstruct(y1, y2, dy1, dy2, F, G, eps, grads, num=None):
     return x1, x2, dx1, dx2
 
 
+# --------------------------------------------------------------------------- down-sampling unit (not reversible)
+# Section 3.1: a reversible block needs stride 1 (anything else discards information); Section 3.2: such layers keep
+# their inputs.  The paper's table counts the down-sampling inside the first unit of a stage without describing it.
+# Reading used here: the same coupling with a parameter-free shortcut S on both skip paths,
+#     y1 = S(x1) + F(x2),   y2 = S(x2) + G(y1),
+# S = 2x2 average pooling with stride 2, then zero channels appended up to the new width; F has one stride-2 layer
+# (its first 3x3 for a basic function, the 3x3 in the middle of a bottleneck), G is an ordinary stride-1 function.
+
+def shortcut_fwd(x, c_out):
+    N, C, H, W = x.shape
+    p = x.reshape(N, C, H // 2, 2, W // 2, 2).mean(axis=(3, 5))
+    out = np.zeros((N, c_out, H // 2, W // 2))
+    out[:, :C] = p
+    return out
+
+
+def shortcut_bwd(d, c_in):
+    """Adjoint of shortcut_fwd: the first c_in channels, each value spread over its 2x2 window with weight 1/4."""
+    return np.repeat(np.repeat(d[:, :c_in], 2, axis=2), 2, axis=3) / 4.0
+
+
+def down_fwd(x1, x2, F, G, eps, num=None):
+    c_out = np.asarray(G[0]["W"]).shape[1]
+    f, cF = fn_fwd(x2, F, eps, num)
+    y1 = quantize_state(shortcut_fwd(x1, c_out), num) + quantize_state(f, num)
+    g, cG = fn_fwd(y1, G, eps, num)
+    y2 = quantize_state(shortcut_fwd(x2, c_out), num) + quantize_state(g, num)
+    return y1, y2, (cF, cG)
+
+
+def down_bwd(dy1, dy2, caches, c_in, grads, num=None):
+    """Ordinary backprop (Eq. 1) through the unit above from its kept input."""
+    cF, cG = caches
+    dz1 = dy1 + fn_bwd(dy2, cG, grads, num)
+    dx2 = shortcut_bwd(dy2, c_in) + fn_bwd(dz1, cF, grads, num)
+    dx1 = shortcut_bwd(dz1, c_in)
+    return dx1, dx2
+
+
 # --------------------------------------------------------------------------- classification stack
 
 def softmax_ce(logits, labels):
@@ -292,6 +334,14 @@ def stack_train_grads(net, images, labels, mode, num=None, keep_blocks=(), keep_
                 transitions[si] = dict(x=h)
             h, tcache = fn_fwd(h, [S["trans"]], eps, num)
         c = S["c"]
+        dcache = None
+        if S.get("down") is not None:
+            stored.append(h)                  # not invertible: its input is kept
+            cp = h.shape[1] // 2
+            dF, dG = S["down"]
+            d1, d2, dcache = down_fwd(h[:, :cp], h[:, cp:], dF, dG, eps, num)
+            h = np.concatenate([d1, d2], axis=1)
+            dcache = (dcache, cp)
         if si == 0 or S["trans"] is not None:
             h = quantize_state(h, num)        # the stage buffers hold the coupling state's format
         x1, x2 = h[:, :c].copy(), h[:, c:].copy()
@@ -305,7 +355,7 @@ def stack_train_grads(net, images, labels, mode, num=None, keep_blocks=(), keep_
             else:
                 x1, x2 = block_fwd(x1, x2, F, G, eps, num=num)
         h = np.concatenate([x1, x2], axis=1)
-        stage_fw.append((tcache, bcaches, x1, x2))
+        stage_fw.append((tcache, bcaches, x1, x2, dcache))
     stored.append(h)                          # top activations: needed to start the reversal
     feat = h.mean(axis=(2, 3))
     fc = net["fc"]
@@ -322,7 +372,7 @@ def stack_train_grads(net, images, labels, mode, num=None, keep_blocks=(), keep_
     dh = np.broadcast_to(dfeat[:, :, None, None] / (Hh * Wh), h.shape).copy()
     for si in reversed(range(len(net["stages"]))):
         S = net["stages"][si]
-        tcache, bcaches, y1, y2 = stage_fw[si]
+        tcache, bcaches, y1, y2, dcache = stage_fw[si]
         c = S["c"]
         d1, d2 = dh[:, :c].copy(), dh[:, c:].copy()
         for ui in reversed(range(len(S["units"]))):
@@ -336,6 +386,8 @@ def stack_train_grads(net, images, labels, mode, num=None, keep_blocks=(), keep_
             if rec is not None:
                 rec.update(dx1=d1, dx2=d2)
                 blocks[(si, ui)] = rec
+        if dcache is not None:
+            d1, d2 = down_bwd(d1, d2, dcache[0], dcache[1], grads, num)
         dh = np.concatenate([d1, d2], axis=1)
         if tcache is not None:
             if keep_transitions:

@@ -52,7 +52,7 @@ class TransitionDesc(C.Structure):
 
 class StageDesc(C.Structure):
     _fields_ = [("units", C.c_int), ("c", C.c_int), ("w", C.c_int), ("kind", C.c_int), ("trans_k", C.c_int),
-                ("trans_stride", C.c_int)]
+                ("trans_stride", C.c_int), ("down", C.c_int)]
 
 
 class StackDesc(C.Structure):
@@ -155,7 +155,7 @@ def stack_desc(cfg: syn.StackCfg, mode: int, verify_reconstruction: bool = False
     d.stem_k, d.stem_stride, d.stem_cout, d.maxpool = cfg.stem_k, cfg.stem_stride, cfg.stem_cout, int(cfg.maxpool)
     d.n_stages = len(cfg.stages)
     for i, s in enumerate(cfg.stages):
-        d.stage[i] = StageDesc(s.units, s.c, s.w, KIND[s.kind], s.trans_k, s.trans_stride)
+        d.stage[i] = StageDesc(s.units, s.c, s.w, KIND[s.kind], s.trans_k, s.trans_stride, int(s.down))
     d.eps, d.mode, d.state_frac_bits = cfg.eps, mode, state_frac_bits
     d.lr, d.momentum, d.weight_decay = cfg.lr, cfg.momentum, cfg.weight_decay
     d.verify_reconstruction = int(verify_reconstruction)

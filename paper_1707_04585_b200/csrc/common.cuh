@@ -190,6 +190,19 @@ inline void launch(Exec &ex, void (*kernel)(KArgs...), dim3 grid, dim3 block, si
     cfg.attrs = &attr; cfg.numAttrs = ex.pdl ? 1 : 0;
     cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
+// The same for a kernel that runs as clusters of `cluster_x` CTAs along x (grid.x a multiple of it).
+template <class... KArgs, class... Args>
+inline void launch_cluster(Exec &ex, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, int cluster_x, Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = ex.stream;
+    cudaLaunchAttribute attr[2] = {};
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = (unsigned)cluster_x; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = ex.pdl ? 2 : 1;
+    cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
 #ifdef __CUDACC__
 // wait until the kernel before this one in the stream has completed (its writes are visible), then
 // allow the kernel after this one to be scheduled
@@ -280,10 +293,14 @@ void head_bwd(Exec &ex, Pair dy, int N, int HW, const float *Wfc, const float *f
               int n_classes, float *dWfc, float *dbfc, float *dfeat);
 void sgd_update(Exec &ex, float *params, const float *grads, float *mom, size_t n,
                 const uint32_t *seg_end, const uint8_t *seg_decay, int n_seg,
-                float lr, float momentum, float wd);
+                float lr, float momentum, float wd, bool quad_aligned);   // quad_aligned: every segment but the last ends on a multiple of four
 // max |a - b| over n elements of two state tensors (float, or fixed point when q > 0)
 void max_abs_diff(Exec &ex, const float *a, const float *b, size_t n, float q, float *out /*1 float, pre-zeroed*/);
 void fill_zero(Exec &ex, void *p, size_t bytes);
+// shortcut of a down-sampling unit: S(x) = 2x2 average pool (stride 2) + zero channels up to cout, in the state format
+// (q as in Pair); and its adjoint on float gradients (first cin channels, weight 1/4 per window position)
+void shortcut_fwd(Exec &ex, const float *x, float *out, int N, int H, int W, int cin, int cout, float q);
+void shortcut_bwd(Exec &ex, const float *d, float *gx, int N, int H, int W, int cin, int cout);
 // out[n, 2i, 2j, :] = in[n, i, j, :], zero elsewhere; out is [N, 2Ho, 2Wo, C]
 void upsample_zero_bf16(Exec &ex, const bf16 *in, bf16 *out, int N, int Ho, int Wo, int C);
 

@@ -20,6 +20,7 @@
 #include "conv_epilogue.cuh"
 #include <cuda.h>
 #include <string.h>
+#include <stdlib.h>
 
 using namespace tc;
 
@@ -58,6 +59,12 @@ struct TcParams {
     int ntap[4];
     signed char tdy[4][9], tdx[4][9], tid[4][9];
     int ostride, oy[4], ox[4];    // epi_tma: output pixel = tile pixel * ostride + (oy, ox)
+    // conv_tc2_kernel, 3x3 stride 1 ("halo" operand): one box per channel chunk holds the tile's pixels WITH their
+    // halo, (BH + 2) rows of Wp = W + 2 pixels; tap (kh, kw) reads the 128 rows that start kh * Wp + kw rows further
+    // on, so the activations cross L2 -> shared memory once per chunk instead of once per tap.  Accumulator row m is
+    // then pixel (m / Wp, m % Wp) of the tile; rows with m % Wp >= W are padding.
+    int halo, Wp;
+    int a_slots, a_slot_bytes, a_box_bytes;
 };
 
 struct __align__(8) TcShared {
@@ -66,6 +73,7 @@ struct __align__(8) TcShared {
     uint64_t acc_full[2];
     uint64_t acc_empty[2];
     uint64_t aux_full[8];
+    uint64_t afull[4], aempty[4];     // halo operand ring of conv_tc2_kernel
     uint32_t tmem_base;
     uint32_t failed;
     RowMap rows;
@@ -180,31 +188,41 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const uint32_t tmem_d = sh->tmem_base;
     const int col0 = blockIdx.y * p.BN;
 
+    // The two single-thread loops below (TMA producer, MMA issuer) set the pace of the whole CTA: a lone thread gets no
+    // latency hiding, every instruction costs its full pipeline latency, and a stage's four MMAs take only 256-512
+    // clocks.  So no divisions, no table look-ups and no descriptor construction inside them: the ring position is
+    // stepped, tap data is read once per tap, descriptors are a base plus increments of the address field.
     if (warp == 0) {
         if (lane == 0) {
-            uint32_t itg = 0;
+            int s = 0; uint32_t round = 0;
             bool ok = true;
+            const uint32_t tx = (uint32_t)(a_bytes + b_bytes);
             for (int t = blockIdx.x; t < n_vt && ok; t += gridDim.x) {
                 int n0, h0;
                 const int cls = t / p.g.n_px_tiles;
                 tile_origin(p.g, t - cls * p.g.n_px_tiles, n0, h0);
-                const int iters = p.ntap[cls] * p.chunks;
-                for (int it = 0; it < iters; it++, itg++) {
-                    const int s = itg % p.stages; const uint32_t round = itg / p.stages;
-                    if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
-                    const int ti = it / p.chunks, ch = it - ti * p.chunks;
-                    uint8_t *sa = tiles + s * stage_bytes;
-                    mbar_expect_tx(&sh->full[s], (uint32_t)(a_bytes + b_bytes));
-                    tma_load_4d(sa, &map_a, &sh->full[s], ch * p.KC, p.tdx[cls][ti], h0 * p.stride + p.tdy[cls][ti], n0);
-                    tma_load_2d(sa + b_off, &map_b, &sh->full[s], p.tid[cls][ti] * p.cin_pad + ch * p.KC, col0);
+                const int ntap = p.ntap[cls], hs = h0 * p.stride;
+                for (int ti = 0; ti < ntap && ok; ti++) {
+                    const int dx = p.tdx[cls][ti], yy = hs + p.tdy[cls][ti];
+                    int wc = p.tid[cls][ti] * p.cin_pad;
+                    for (int cc = 0; cc < p.cin_pad; cc += p.KC, wc += p.KC) {
+                        if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
+                        uint8_t *sa = tiles + s * stage_bytes;
+                        mbar_expect_tx(&sh->full[s], tx);
+                        tma_load_4d(sa, &map_a, &sh->full[s], cc, dx, yy, n0);
+                        tma_load_2d(sa + b_off, &map_b, &sh->full[s], wc, col0);
+                        if (++s == p.stages) { s = 0; round++; }
+                    }
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = instr_desc(p.BN);
-            const int row_bytes = p.KC * 2;
-            uint32_t itg = 0;
+            const int row_bytes = p.KC * 2, nk = p.KC >> 4;
+            const uint64_t da0 = smem_desc(smem_u32(tiles), row_bytes), db0 = smem_desc(smem_u32(tiles) + b_off, row_bytes);
+            const uint32_t stage16 = (uint32_t)stage_bytes >> 4;      // the descriptors' address field counts 16-byte units
+            int s = 0; uint32_t round = 0, soff = 0;
             bool ok = true;
             int ti = 0;
             for (int t = blockIdx.x; t < n_vt && ok; t += gridDim.x, ti++) {
@@ -213,17 +231,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 if (use > 0 && !mbar_wait(&sh->acc_empty[buf], (use - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
                 tc_fence_after();
                 const uint32_t acc = tmem_d + (uint32_t)(buf * p.BN);
-                for (int it = 0; it < iters; it++, itg++) {
-                    const int s = itg % p.stages; const uint32_t round = itg / p.stages;
+                uint32_t accum = 0;
+                for (int it = 0; it < iters; it++) {
                     if (!mbar_wait(&sh->full[s], round & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = smem_u32(tiles + s * stage_bytes);
-                    for (int kk = 0; kk < p.KC / 16; kk++) {
-                        const uint64_t da = smem_desc(sa + kk * 32, row_bytes);
-                        const uint64_t db = smem_desc(sa + b_off + kk * 32, row_bytes);
-                        mma_bf16(acc, da, db, idesc, (it > 0 || kk > 0) ? 1u : 0u);
-                    }
+                    const uint64_t da = da0 + soff, db = db0 + soff;
+                    mma_bf16(acc, da, db, idesc, accum);
+                    accum = 1;
+                    for (int kk = 1; kk < nk; kk++) mma_bf16(acc, da + 2 * kk, db + 2 * kk, idesc, 1u);
                     mma_commit(&sh->empty[s]);          // frees the stage once these MMAs have read it
+                    soff += stage16;
+                    if (++s == p.stages) { s = 0; soff = 0; round++; }
                 }
                 if (ok) mma_commit(&sh->acc_full[buf]);
             }
@@ -375,6 +393,311 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_d, tmem_cols);
+    }
+}
+
+// The same convolution on a CTA PAIR (a cluster of two CTAs on the two SMs of a TPC, tcgen05 cta_group::2): one
+// MMA of M = 256 covers two adjacent pixel tiles, CTA `rank` holding the operand rows of its own 128 pixels and its
+// half of the N tile's weight rows, and receiving its 128 accumulator rows in its own tensor memory.  Per MMA an SM
+// then reads 128 x 16 activations and only N/2 x 16 weights from shared memory (and fetches only half of the weight
+// tile from L2), which is what lets 256-wide tiles run at the tensor cores' rate instead of the shared-memory port's.
+// The leader (rank 0) issues the MMAs for both; each CTA loads its own operands (plain tile loads, no multicast)
+// and signals the leader's barrier; commits arrive on the barriers of both CTAs.  Each CTA runs the epilogue of its
+// own tile exactly as the single-CTA kernel does (epilogue through TMA only).
+// Tile pairs: class c, pair j holds the pixel tiles 2j and 2j + 1 of the class; with an odd tile count the last pair's
+// second tile lies outside the tensor (TMA delivers zeros, nothing is stored).
+__global__ void __launch_bounds__(kThreadsTma, 1)
+conv_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                const __grid_constant__ CUtensorMap map_o0, const __grid_constant__ CUtensorMap map_o1,
+                const __grid_constant__ CUtensorMap map_x0, const __grid_constant__ CUtensorMap map_x1, const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int box_px = p.g.BIMG * p.g.BH * p.g.W;
+    const int BNH = p.BN >> 1;                                   // weight rows this CTA holds
+    const int a_bytes = box_px * p.KC * 2, b_bytes = BNH * p.KC * 2;
+    const int b_off = (128 * p.KC * 2 + 1023) & ~1023;
+    const int stage_bytes = b_off + ((b_bytes + 1023) & ~1023);
+    const int ng = p.BN / p.GW;
+    // halo mode: the ring holds weight tiles only, the activation boxes have a ring of their own in front of it
+    uint8_t *abuf = tiles;
+    const int wstage_bytes = (b_bytes + 1023) & ~1023;
+    uint8_t *wring = tiles + (p.halo ? p.a_slots * p.a_slot_bytes : 0);
+    uint8_t *auxr = p.halo ? wring + p.stages * wstage_bytes : tiles + p.stages * stage_bytes;
+    uint8_t *outr = auxr + (p.need_aux ? ng : 0) * p.group_bytes;
+    float *gsums = (float *)(outr + 2 * p.group_bytes);
+    TcShared *sh = (TcShared *)(gsums + ng * 128 * 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();
+    const int pair = (int)blockIdx.x >> 1, n_pairs = (int)gridDim.x >> 1;
+    const int n_pp = (p.g.n_px_tiles + 1) >> 1;                  // tile pairs per class
+    const int n_vp = p.n_cls * n_pp;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < 2 * p.BN) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; s++) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+        // acc_empty (used in the leader): one arrival per epilogue warp group of either CTA
+        for (int b = 0; b < 2; b++) { mbar_init(&sh->acc_full[b], 1); mbar_init(&sh->acc_empty[b], 4); }
+        for (int b = 0; b < 8; b++) mbar_init(&sh->aux_full[b], 1);
+        for (int b = 0; b < 4; b++) { mbar_init(&sh->afull[b], 1); mbar_init(&sh->aempty[b], 1); }
+        sh->failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tma_prefetch_desc(&map_a); tma_prefetch_desc(&map_b);
+        tma_prefetch_desc(&map_o0); tma_prefetch_desc(&map_o1); tma_prefetch_desc(&map_x0); tma_prefetch_desc(&map_x1);
+    }
+    if (warp == 1) tmem2_alloc(&sh->tmem_base, tmem_cols);       // the same warp of both CTAs
+    if (warp >= 2) build_row_map(p.g, &sh->rows, ((warp & 3) << 5) | lane);
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();      // the peer's barriers are initialised and its tensor memory allocated before anything crosses over
+    tc_fence_after();
+    pdl_enter();
+    const uint32_t tmem_d = sh->tmem_base;
+    const int col0 = blockIdx.y * p.BN;
+    // this CTA's tile of tile pair vp
+    auto my_tile = [&](int vp, int &cls, int &t) { cls = vp / n_pp; t = 2 * (vp - cls * n_pp) + (int)rank; };
+
+    // (single-thread loops kept lean, as in conv_tc_kernel)
+    if (warp == 0) {
+        if (lane == 0) {
+            int s = 0, as = 0; uint32_t round = 0, ar = 0;
+            bool ok = true;
+            const uint32_t full0 = mapa_shared(smem_u32(&sh->full[0]), 0), afull0 = mapa_shared(smem_u32(&sh->afull[0]), 0);   // the leader's barriers
+            const uint32_t tx = (uint32_t)(2 * (a_bytes + b_bytes)), txw = (uint32_t)(2 * b_bytes), txa = (uint32_t)(2 * p.a_box_bytes);
+            const int wcol = col0 + (int)rank * BNH;
+            for (int vp = pair; vp < n_vp && ok; vp += n_pairs) {
+                int cls, t, n0, h0;
+                my_tile(vp, cls, t);
+                tile_origin(p.g, t, n0, h0);         // beyond the last tile the origin lies outside the tensor: zeros arrive
+                if (p.halo) {
+                    // per channel chunk: one activation box with its halo, then the nine weight tiles
+                    for (int cc = 0; cc < p.cin_pad && ok; cc += p.KC) {
+                        if (ar > 0 && !mbar_wait(&sh->aempty[as], (ar - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
+                        if (rank == 0) mbar_expect_tx(&sh->afull[as], txa);
+                        tma2_load_4d(abuf + as * p.a_slot_bytes, &map_a, afull0 + 8u * as, cc, -1, h0 - 1, n0);
+                        if (++as == p.a_slots) { as = 0; ar++; }
+                        int wc = cc;
+                        for (int ti = 0; ti < 9; ti++, wc += p.cin_pad) {      // tap ti of a plain 3x3 layer sits at ti * cin_pad in the pack
+                            if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
+                            if (rank == 0) mbar_expect_tx(&sh->full[s], txw);
+                            tma2_load_2d(wring + s * wstage_bytes, &map_b, full0 + 8u * s, wc, wcol);
+                            if (++s == p.stages) { s = 0; round++; }
+                        }
+                    }
+                    continue;
+                }
+                const int ntap = p.ntap[cls], hs = h0 * p.stride;
+                for (int ti = 0; ti < ntap && ok; ti++) {
+                    const int dx = p.tdx[cls][ti], yy = hs + p.tdy[cls][ti];
+                    int wc = p.tid[cls][ti] * p.cin_pad;
+                    for (int cc = 0; cc < p.cin_pad; cc += p.KC, wc += p.KC) {
+                        if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
+                        uint8_t *sa = tiles + s * stage_bytes;
+                        if (rank == 0) mbar_expect_tx(&sh->full[s], tx);      // the leader's barrier collects the bytes of both CTAs
+                        tma2_load_4d(sa, &map_a, full0 + 8u * s, cc, dx, yy, n0);
+                        tma2_load_2d(sa + b_off, &map_b, full0 + 8u * s, wc, wcol);
+                        if (++s == p.stages) { s = 0; round++; }
+                    }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = instr_desc_m256(p.BN);
+            const int row_bytes = p.KC * 2, nk = p.KC >> 4;
+            const uint64_t da0 = smem_desc(smem_u32(tiles), row_bytes), db0 = smem_desc(smem_u32(tiles) + b_off, row_bytes);
+            const uint64_t ha0 = smem_desc(smem_u32(abuf), 128), hb0 = smem_desc(smem_u32(wring), 128);      // halo mode: boxes, weight ring
+            const uint32_t stage16 = (uint32_t)stage_bytes >> 4, wstage16 = (uint32_t)wstage_bytes >> 4, aslot16 = (uint32_t)p.a_slot_bytes >> 4;
+            const uint32_t wp8 = (uint32_t)p.Wp * 8u;      // one halo row of pixels, in 16-byte units (128-byte operand rows)
+            int s = 0, as = 0; uint32_t round = 0, ar = 0, soff = 0, aoff = 0;
+            bool ok = true;
+            int ti = 0;
+            for (int vp = pair; vp < n_vp && ok; vp += n_pairs, ti++) {
+                const int buf = ti & 1; const uint32_t use = ti >> 1;
+                if (use > 0 && !mbar_wait_cluster(&sh->acc_empty[buf], (use - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
+                tc_fence_after();
+                const uint32_t acc = tmem_d + (uint32_t)(buf * p.BN);
+                uint32_t accum = 0;
+                if (p.halo) {
+                    for (int ch = 0; ch < p.chunks && ok; ch++) {
+                        if (!mbar_wait_cluster(&sh->afull[as], ar & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
+                        // tap (kh, kw): the operand starts kh * Wp + kw rows (of 128 bytes) into the box.  The 128-byte
+                        // swizzle is a function of the shared-memory ADDRESS (bits 4..6 xor bits 7..9), for the TMA
+                        // write as for the MMA read, so a start on any row reads the rows as they were written
+                        uint64_t da_row = ha0 + aoff;
+                        for (int kh = 0; kh < 3 && ok; kh++, da_row += wp8) {
+                            uint64_t da = da_row;
+                            for (int kw = 0; kw < 3; kw++, da += 8) {
+                                if (!mbar_wait_cluster(&sh->full[s], round & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
+                                tc_fence_after();
+                                const uint64_t db = hb0 + soff;
+                                mma2_bf16(acc, da, db, idesc, accum);
+                                accum = 1;
+                                mma2_bf16(acc, da + 2, db + 2, idesc, 1u);
+                                mma2_bf16(acc, da + 4, db + 4, idesc, 1u);
+                                mma2_bf16(acc, da + 6, db + 6, idesc, 1u);
+                                mma2_commit_both(&sh->empty[s]);
+                                soff += wstage16;
+                                if (++s == p.stages) { s = 0; soff = 0; round++; }
+                            }
+                        }
+                        if (ok) mma2_commit_both(&sh->aempty[as]);      // the box is free once the MMAs of its nine taps have read it
+                        aoff += aslot16;
+                        if (++as == p.a_slots) { as = 0; aoff = 0; ar++; }
+                    }
+                    if (ok) mma2_commit_both(&sh->acc_full[buf]);
+                    continue;
+                }
+                const int iters = p.ntap[vp / n_pp] * p.chunks;
+                for (int it = 0; it < iters; it++) {
+                    if (!mbar_wait_cluster(&sh->full[s], round & 1)) { atomicExch(&sh->failed, 1u); ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t da = da0 + soff, db = db0 + soff;
+                    mma2_bf16(acc, da, db, idesc, accum);
+                    accum = 1;
+                    for (int kk = 1; kk < nk; kk++) mma2_bf16(acc, da + 2 * kk, db + 2 * kk, idesc, 1u);
+                    mma2_commit_both(&sh->empty[s]);         // frees the stage in both CTAs once these MMAs have read it
+                    soff += stage16;
+                    if (++s == p.stages) { s = 0; soff = 0; round++; }
+                }
+                if (ok) mma2_commit_both(&sh->acc_full[buf]);
+            }
+        }
+    } else {
+        // epilogue of this CTA's own tile: as in conv_tc_kernel (two groups of four warps, alternate column groups)
+        const int wg = (warp - 2) >> 2;
+        const int bar_a = 1 + 2 * wg, bar_b = 2 + 2 * wg;
+        const int etid = ((warp & 3) << 5) | lane;
+        const EpiArgs &e = p.epi;
+        const int GW = p.GW, QW = GW >> 2, rpp = 128 / QW;
+        const int jq = etid % QW, r0 = etid / QW;
+        const int box_px_o = p.g.BIMG * p.g.BH * p.g.W;
+        const uint32_t lane_base = (uint32_t)((warp & 3) * 32) << 16;
+        const float out_q = e.out.q, out_s = out_q != 0.f ? 1.f / out_q : 0.f, t_q = e.t.q;
+        const uint32_t aux_tx = (uint32_t)(box_px_o * GW * 4);
+        const uint32_t acc_empty0[2] = {mapa_shared(smem_u32(&sh->acc_empty[0]), 0), mapa_shared(smem_u32(&sh->acc_empty[1]), 0)};
+        // pixel of the tile's box (rows of W pixels) this thread's accumulator row holds; -1: padding
+        int srow = etid;
+        if (p.halo) { const int hh = etid / p.Wp, ww = etid - hh * p.Wp; srow = (hh < p.g.BH && ww < p.g.W) ? hh * p.g.W + ww : -1; }
+        const int prow = srow < 0 ? 0 : srow;
+        for (int i = wg * 128 + etid; i < ng * 128 * 8; i += 256) gsums[i] = 0.f;
+        auto out_map = [&](int col) { return (p.split_o && col >= p.split_o) ? &map_o1 : &map_o0; };
+        auto aux_map = [&](int col) { return (p.split_x && col >= p.split_x) ? &map_x1 : &map_x0; };
+        auto col_out = [&](int col) { return (p.split_o && col >= p.split_o) ? col - p.split_o : col; };
+        auto col_aux = [&](int col) { return (p.split_x && col >= p.split_x) ? col - p.split_x : col; };
+        auto load_aux = [&](int gi, int vp) {                // one thread; returns without loading for a tile outside the tensor
+            const int col = col0 + gi * GW;
+            int cls, t, n0, h0;
+            my_tile(vp, cls, t);
+            if (col >= e.n_cols || t >= p.g.n_px_tiles) return;
+            tile_origin(p.g, t, n0, h0);
+            mbar_expect_tx(&sh->aux_full[gi], aux_tx);
+            tma_load_4d(auxr + gi * p.group_bytes, aux_map(col), &sh->aux_full[gi], col_aux(col), p.ox[cls], h0 * p.ostride + p.oy[cls], n0);
+        };
+        if (etid == 0 && p.need_aux && pair < n_vp)
+            for (int gi = wg; gi < ng; gi += 2) load_aux(gi, pair);
+        named_barrier(5, 256);
+        bool ok = true;
+        int ti = 0;
+        uint32_t aux_uses[8] = {0, 0, 0, 0, 0, 0, 0, 0};     // per column group: loads waited for so far (tiles outside the tensor load nothing)
+        uint8_t *ob = outr + wg * p.group_bytes;
+        for (int vp = pair; vp < n_vp; vp += n_pairs, ti++) {
+            const int buf = ti & 1; const uint32_t use = ti >> 1;
+            int cls, t, n0, h0;
+            my_tile(vp, cls, t);
+            const bool in_range = t < p.g.n_px_tiles;
+            tile_origin(p.g, t, n0, h0);
+            const int vpn = vp + n_pairs;
+            int valid_px = 0;
+            if (in_range)
+                valid_px = p.g.BIMG > 1 ? (p.g.N - n0 < p.g.BIMG ? p.g.N - n0 : p.g.BIMG) * p.g.BH * p.g.W
+                                        : (p.g.H - h0 < p.g.BH ? p.g.H - h0 : p.g.BH) * p.g.W;
+            if (etid == 0) ok = mbar_wait_cluster(&sh->acc_full[buf], use & 1) && sh->failed == 0;
+            ok = named_barrier_and(bar_b, 128, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t tm = tmem_d + lane_base + (uint32_t)(buf * p.BN);
+#pragma unroll 1
+            for (int gi = wg; gi < ng; gi += 2) {
+                const int col = col0 + gi * GW;
+                const bool live = in_range && col < e.n_cols;
+                const uint8_t *ax = auxr + gi * p.group_bytes;
+                if (etid == 0) {
+                    if (p.need_aux && live) ok = mbar_wait(&sh->aux_full[gi], aux_uses[gi] & 1);
+                    tma_store_wait_read();
+                }
+                if (p.need_aux && live) aux_uses[gi]++;
+                ok = named_barrier_and(bar_b, 128, ok);
+                if (!ok) break;
+                const bool rowv = live && srow >= 0 && srow < valid_px;
+                const uint32_t tg = tm + (uint32_t)(gi * GW);
+                if (e.mode != EPI_COUPLE) {
+                    if (out_q == 0.f) tma_pass_a<0>(tg, GW, prow, rowv, ax, ob, out_s); else tma_pass_a<1>(tg, GW, prow, rowv, ax, ob, out_s);
+                } else if (out_q == 0.f) {
+                    if (e.sign > 0) tma_pass_a<2>(tg, GW, prow, rowv, ax, ob, out_s); else tma_pass_a<3>(tg, GW, prow, rowv, ax, ob, out_s);
+                } else {
+                    if (e.sign > 0) tma_pass_a<4>(tg, GW, prow, rowv, ax, ob, out_s); else tma_pass_a<5>(tg, GW, prow, rowv, ax, ob, out_s);
+                }
+                fence_proxy_async();
+                named_barrier(bar_a, 128);
+                if (etid == 0 && live) {
+                    tma_store_4d(out_map(col), ob, col_out(col), p.ox[cls], h0 * p.ostride + p.oy[cls], n0);
+                    tma_store_commit();
+                }
+                if (e.part && live && col + jq * 4 < e.n_cols) {
+                    float4 sc4 = make_float4(0, 0, 0, 0), sh4 = sc4, mu4 = sc4, rs4 = sc4;
+                    if (e.mode == EPI_BNBWD) bn_coef4(e.bn, col + jq * 4, sc4, sh4, mu4, rs4);
+                    float4 *slot = reinterpret_cast<float4 *>(gsums + (gi * 128 + etid) * 8);
+                    const float4 a0 = slot[0], a1 = slot[1];
+                    float acc[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+                    if (e.mode == EPI_BNBWD) {
+                        if (t_q == 0.f) tma_pass_b<2>(GW, ob, ax, jq, r0, rpp, valid_px, 0.f, sc4, sh4, mu4, rs4, acc);
+                        else tma_pass_b<3>(GW, ob, ax, jq, r0, rpp, valid_px, t_q, sc4, sh4, mu4, rs4, acc);
+                    } else if (out_q == 0.f) tma_pass_b<0>(GW, ob, ax, jq, r0, rpp, valid_px, 0.f, sc4, sh4, mu4, rs4, acc);
+                    else tma_pass_b<1>(GW, ob, ax, jq, r0, rpp, valid_px, out_q, sc4, sh4, mu4, rs4, acc);
+                    slot[0] = make_float4(acc[0], acc[1], acc[2], acc[3]); slot[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
+                }
+                named_barrier(bar_a, 128);
+                if (etid == 0 && p.need_aux && vpn < n_vp) load_aux(gi, vpn);
+            }
+            if (!ok) break;
+            // this warp group has drained its columns of the accumulator: one arrival per group on the leader's barrier
+            tc_fence_before();
+            named_barrier(bar_a, 128);
+            if (etid == 0) mbar_arrive_cluster(acc_empty0[buf]);
+        }
+        if (etid == 0) tma_store_wait_all();
+        if (!ok && lane == 0) atomicExch(&sh->failed, 1u);
+        __threadfence_block();
+        named_barrier(5, 256);
+        if (wg == 0 && e.part && sh->failed == 0) {
+            float *mine = e.part + (size_t)blockIdx.x * 2 * e.n_cols;
+            for (int gi = 0; gi < ng; gi++) {
+                const int col = col0 + gi * GW + jq * 4;
+                if (r0 == 0 && col < e.n_cols) {
+                    const float *base = gsums + (size_t)gi * 128 * 8;
+                    float r[8];
+#pragma unroll
+                    for (int j = 0; j < 8; j++) r[j] = base[jq * 8 + j];
+                    for (int y = 1; y < rpp; y++)
+#pragma unroll
+                        for (int j = 0; j < 8; j++) r[j] += base[(y * QW + jq) * 8 + j];
+                    *reinterpret_cast<float4 *>(mine + 2 * col) = make_float4(r[0], r[1], r[2], r[3]);
+                    *reinterpret_cast<float4 *>(mine + 2 * col + 4) = make_float4(r[4], r[5], r[6], r[7]);
+                }
+            }
+            epilogue_publish<128>(e, reinterpret_cast<float *>(auxr), etid);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && sh->failed) atomicExch(p.status, (int)REVNET_E_TIMEOUT);
+    // neither CTA leaves, or frees tensor memory, while the other may still read its operands or signal its barriers
+    cluster_sync_all();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem2_dealloc(tmem_d, tmem_cols);
     }
 }
 
@@ -534,21 +857,53 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
     const int ostride = s2 ? 2 : 1;
     if (s2 && (!epi_tma || g.W * 2 > 256 || s.g.BH * 2 > 256)) return false;
     int stages = 4;
+    // CTA pairs (conv_tc2_kernel) wherever the epilogue runs through TMA, the N tile splits into two halves of whole
+    // 16-row groups and there are at least two pixel tiles; REVNET_CONV_PAIR=0 keeps the single-CTA kernel (for comparison)
+    static const bool pair_enabled = [] { const char *v = getenv("REVNET_CONV_PAIR"); return !(v && v[0] == '0'); }();
+    // (1x1 layers are bound by the activations' way from HBM, which a pair does not shorten: measured 3-10 % slower there)
+    bool pair = pair_enabled && epi_tma && k == 3 && s.BN % 32 == 0 && s.BN >= 64 && s.g.n_px_tiles >= 2 && ex.ctx->sm_count % 2 == 0;
+    // 3x3 stride-1 layers on a pair: the activations of a tile arrive once per channel chunk as one box with its halo
+    // (see TcParams::halo); needs 64-channel chunks (128-byte operand rows) and tiles of whole image rows
+    static const bool halo_enabled = [] { const char *v = getenv("REVNET_CONV_HALO"); return !(v && v[0] == '0'); }();
+    bool halo = halo_enabled && pair && k == 3 && stride == 1 && !s2 && s.KC == 64 && s.g.BIMG == 1 && g.W + 2 <= 128;
+    int a_slot_bytes = 0, a_box_bytes = 0;
+    const int a_slots = 2;
+    if (halo) {
+        const int Wp = g.W + 2;
+        int bh = 128 / Wp; if (bh > g.H) bh = g.H;
+        s.g.BH = bh;
+        s.g.tiles_per_img = (g.H + bh - 1) / bh;
+        s.g.n_px_tiles = g.N * s.g.tiles_per_img;
+        const int box_rows = (bh + 2) * Wp, read_rows = 2 * Wp + 2 + 128;       // rows the box holds / rows the last tap reads up to
+        a_box_bytes = box_rows * 128;
+        a_slot_bytes = ((box_rows > read_rows ? box_rows : read_rows) * 128 + 1023) & ~1023;
+    }
     if (epi_tma) {
         stages = kStages;
-        const int stage_bytes = ((128 * s.KC * 2 + 1023) & ~1023) + ((s.BN * s.KC * 2 + 1023) & ~1023);
-        auto smem_of = [&](int st) { return 1024 + st * stage_bytes + ((need_aux ? ng : 0) + 2) * group_bytes + ng * 128 * 32 + (int)sizeof(TcShared) + 64; };
-        while (stages > 2 && smem_of(stages) > 227 * 1024) stages--;
-        if (smem_of(stages) > 227 * 1024) {
+        auto stage_bytes_of = [&](bool pr) {
+            if (halo) return ((s.BN / 2) * s.KC * 2 + 1023) & ~1023;           // weight tiles only; the boxes are counted below
+            return ((128 * s.KC * 2 + 1023) & ~1023) + (((pr ? s.BN / 2 : s.BN) * s.KC * 2 + 1023) & ~1023);
+        };
+        auto smem_of = [&](int st, bool pr) { return 1024 + (halo ? a_slots * a_slot_bytes : 0) + st * stage_bytes_of(pr) + ((need_aux ? ng : 0) + 2) * group_bytes + ng * 128 * 32 + (int)sizeof(TcShared) + 64; };
+        while (stages > 2 && smem_of(stages, pair) > 227 * 1024) stages--;
+        if (smem_of(stages, pair) > 227 * 1024) {
             if (s.BN == 256) return false;      // (does not happen: three stages of a wide tile fit)
-            epi_tma = false; stages = 4;
-        } else s.smem = smem_of(stages);
+            epi_tma = false; pair = false; stages = 4;
+            if (halo) { halo = false; tile_geom(g, s.g); }
+        } else s.smem = smem_of(stages, pair);
     }
     if ((s2 || s.BN == 256) && !epi_tma) return false;
     ex.flops += 2ull * g.P() * cout * cin * ntap_all;
     int occ = (227 * 1024) / s.smem; if (occ > 2) occ = 2; if (occ < 1) occ = 1;
     int ctas = ex.ctx->sm_count * occ / s.n_tiles; if (ctas < 1) ctas = 1;
     if (ctas > s.g.n_px_tiles * n_cls) ctas = s.g.n_px_tiles * n_cls;
+    if (pair) {
+        // one pair per TPC and N tile; a pair walks tile pairs
+        const int n_vp = n_cls * ((s.g.n_px_tiles + 1) / 2);
+        int pairs = (ex.ctx->sm_count / 2) / s.n_tiles; if (pairs < 1) pairs = 1;
+        if (pairs > n_vp) pairs = n_vp;
+        ctas = 2 * pairs;
+    }
     size_t m = ex.ws.mark();
     bf16 *wp = prepacked ? const_cast<bf16 *>(prepacked) : ex.ws.get<bf16>((size_t)rows_pad * taps * s.cin_pad);
     const bool reduce = req.stats || req.bnbwd;
@@ -571,6 +926,7 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
             cuuint64_t dims[4] = {(cuuint64_t)cin, (cuuint64_t)gin.W, (cuuint64_t)gin.H, (cuuint64_t)gin.N};
             cuuint64_t strides[3] = {(cuuint64_t)cin * 2, (cuuint64_t)gin.W * cin * 2, (cuuint64_t)gin.H * gin.W * cin * 2};
             cuuint32_t box[4] = {(cuuint32_t)s.KC, (cuuint32_t)(g.W * stride), (cuuint32_t)(s.g.BH * stride), (cuuint32_t)s.g.BIMG};
+            if (halo) { box[1] = (cuuint32_t)(g.W + 2); box[2] = (cuuint32_t)(s.g.BH + 2); }
             cuuint32_t es[4] = {1, (cuuint32_t)stride, (cuuint32_t)stride, 1};
             CUresult r = enc(&map_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, (void *)act, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                              sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -579,7 +935,7 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         {
             cuuint64_t dims[2] = {(cuuint64_t)taps * s.cin_pad, (cuuint64_t)rows_pad};
             cuuint64_t strides[1] = {(cuuint64_t)taps * s.cin_pad * 2};
-            cuuint32_t box[2] = {(cuuint32_t)s.KC, (cuuint32_t)s.BN};
+            cuuint32_t box[2] = {(cuuint32_t)s.KC, (cuuint32_t)(pair ? s.BN / 2 : s.BN)};     // a CTA of a pair loads its half of the N tile
             cuuint32_t es[2] = {1, 1};
             CUresult r = enc(&map_b, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, (void *)wp, dims, strides, box, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
                              sw, CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -613,6 +969,7 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         p.split_o = out.c1 ? out.c0 : 0; p.split_x = (need_aux && auxp.c1) ? auxp.c0 : 0;
         memcpy(p.ntap, ntap, sizeof ntap); memcpy(p.tdy, tdy, sizeof tdy); memcpy(p.tdx, tdx, sizeof tdx); memcpy(p.tid, tid, sizeof tid);
         p.ostride = ostride; p.n_cls = n_cls;
+        p.halo = halo ? 1 : 0; p.Wp = g.W + 2; p.a_slots = a_slots; p.a_slot_bytes = a_slot_bytes; p.a_box_bytes = a_box_bytes;
         for (int c = 0; c < 4; c++) { p.oy[c] = s2 ? c >> 1 : 0; p.ox[c] = s2 ? c & 1 : 0; }
         p.taps = taps; p.k = k; p.chunks = s.chunks; p.KC = s.KC; p.cin_pad = s.cin_pad; p.BN = s.BN; p.stride = stride; p.g = s.g;
         p.status = ex.ctx->dev_status;
@@ -625,9 +982,13 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         if (req.stats) { e.mean = req.stats->mean; e.rstd = req.stats->rstd; }
         if (req.bnbwd) { e.t = req.bnbwd->t; e.bn = req.bnbwd->bn; e.dgamma = req.bnbwd->dgamma; e.dbeta = req.bnbwd->dbeta; e.coef = req.bnbwd->coef; }
         static OncePerDevice once;
-        if (once.first(ex.ctx->device)) cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (once.first(ex.ctx->device)) {
+            cudaFuncSetAttribute(conv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+            cudaFuncSetAttribute(conv_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        }
         dim3 grid((unsigned)ctas, (unsigned)s.n_tiles);
-        launch(ex, conv_tc_kernel, grid, epi_tma ? kThreadsTma : kThreads, s.smem, map_a, map_b, map_o[0], map_o[1], map_x[0], map_x[1], p);
+        if (pair) launch_cluster(ex, conv_tc2_kernel, grid, kThreadsTma, s.smem, 2, map_a, map_b, map_o[0], map_o[1], map_x[0], map_x[1], p);
+        else launch(ex, conv_tc_kernel, grid, epi_tma ? kThreadsTma : kThreads, s.smem, map_a, map_b, map_o[0], map_o[1], map_x[0], map_x[1], p);
         const double bytes = (double)gin.P() * cin * 2 + (double)g.P() * cout * (sign || req.bnbwd ? 8 : 4) + (double)cout * taps * cin * 2;
         ex.check(what, bytes, 2.0 * g.P() * cout * cin * ntap_all);
     }
@@ -738,8 +1099,8 @@ wgrad_tc_kernel(const __grid_constant__ WgBatch batch) {
         const int bg = lane - n_blocks;
         const int g_c = p.sep ? (bg % npk) * p.blockN : col0 + bg * p.blockN;      // gradient box: first channel, first column
         const int g_x = p.sep ? p.k / 2 - bg / npk : 0;
+        int s = 0; uint32_t round = 0;
         for (int it = 0; it < my_tiles; it++) {
-            const int s = it % p.stages, round = it / p.stages;
             bool ok = true;
             if (lane == 0) {
                 if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; }
@@ -749,27 +1110,37 @@ wgrad_tc_kernel(const __grid_constant__ WgBatch batch) {
             if (!ok) break;
             const int t = split + it * p.splits;
             const int n0 = p.BIMG > 1 ? t * p.BIMG : t / tiles_per_img;
-            const int h0 = p.BIMG > 1 ? 0 : (t % tiles_per_img) * p.BH;
+            const int h0 = p.BIMG > 1 ? 0 : (t - n0 * tiles_per_img) * p.BH;
             uint8_t *sa = tiles + s * stage_bytes;
             if (a_lane) tma_load_4d(sa + lane * blk_bytes_a, &map_a, &sh->full[s], cb * p.blockC, kw - pad, h0 * p.stride + kh - pad, n0);
             else if (g_lane) tma_load_4d(sa + a_region + bg * blk_bytes_b, &map_g, &sh->full[s], g_c, g_x, h0, n0);
+            if (++s == p.stages) { s = 0; round++; }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = instr_desc(p.BN, true);
             const int rba = p.blockC * 2, rbb = p.blockN * 2;
+            // one thread issues everything: descriptors are a base plus increments of the address field (16-byte units),
+            // the ring position is stepped (no divisions in the loop)
+            const uint64_t da0 = smem_desc_mn(smem_u32(tiles), rba, blk_bytes_a), db0 = smem_desc_mn(smem_u32(tiles) + a_region, rbb, blk_bytes_b);
+            const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
+            int s = 0; uint32_t round = 0, soff = 0;
             for (int it = 0; it < my_tiles; it++) {
-                const int s = it % p.stages, round = it / p.stages;
                 if (!mbar_wait(&sh->full[s], round & 1)) { atomicExch(&sh->failed, 1u); break; }
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t sa = smem_u32(tiles + s * stage_bytes);
-                for (int g = 0; g < groups; g++)
-                    for (int ks = 0; ks < 8; ks++) {         // 16 pixels per MMA
-                        const uint64_t da = smem_desc_mn(sa + g * 32768 + ks * 16 * rba, rba, blk_bytes_a);
-                        const uint64_t db = smem_desc_mn(sa + a_region + ks * 16 * rbb, rbb, blk_bytes_b);
-                        mma_bf16(tmem_d + (uint32_t)(g * p.BN), da, db, idesc, (it > 0 || ks > 0) ? 1u : 0u);
+                const uint32_t accum = it > 0 ? 1u : 0u;
+                for (int g = 0; g < groups; g++) {
+                    uint64_t da = da0 + soff + (uint32_t)(g * 2048), db = db0 + soff;      // an M group is 32 KB from its first block
+                    const uint32_t acc = tmem_d + (uint32_t)(g * p.BN);
+                    mma_bf16(acc, da, db, idesc, accum);
+                    for (int ks = 1; ks < 8; ks++) {         // 16 pixels per MMA
+                        da += (uint32_t)rba; db += (uint32_t)rbb;
+                        mma_bf16(acc, da, db, idesc, 1u);
                     }
+                }
                 mma_commit(&sh->empty[s]);
+                soff += stage16;
+                if (++s == p.stages) { s = 0; soff = 0; round++; }
             }
             mma_commit(&sh->acc_full[0]);
         }

@@ -216,16 +216,33 @@ void bn_stats(Exec &ex, Pair t, size_t P, Moments mo) {
     ex.ws.release(m);
 }
 
+// A thread keeps one channel quad (scale and shift stay in registers) and strides the rows, four rows in flight;
+// row_step = threads of the grid / C4 (the launch makes that a whole number): no division per element.
 template <class TO>
-__global__ void bn_relu_apply_kernel(Pair t, size_t nquads, int C4, BnRef bn, TO *__restrict__ a) {
+__global__ void __launch_bounds__(256) bn_relu_apply_kernel(Pair t, size_t P, int C4, BnRef bn, TO *__restrict__ a) {
     pdl_enter();
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nquads; i += (size_t)gridDim.x * blockDim.x) {
-        size_t row = i / C4; int q = (int)(i - row * C4);
-        float4 v = t.ld4(row, q * 4), sc, sh, mu, rs;
-        bn_coef4(bn, q * 4, sc, sh, mu, rs);
-        v.x = fmaxf(fmaf(sc.x, v.x, sh.x), 0.f); v.y = fmaxf(fmaf(sc.y, v.y, sh.y), 0.f);
-        v.z = fmaxf(fmaf(sc.z, v.z, sh.z), 0.f); v.w = fmaxf(fmaf(sc.w, v.w, sh.w), 0.f);
-        st4(a + i * 4, v);
+    const int C = C4 * 4;
+    const size_t gtid = (size_t)blockIdx.x * blockDim.x + threadIdx.x, nth = (size_t)gridDim.x * blockDim.x;
+    const int q = (int)(gtid % C4), c = q * 4;
+    const size_t row0 = gtid / C4, row_step = nth / C4;
+    float4 sc, sh, mu, rs;
+    bn_coef4(bn, c, sc, sh, mu, rs);
+    for (size_t rb = row0; rb < P; rb += 4 * row_step) {
+        float4 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            const size_t row = rb + j * row_step;
+            if (row < P) v[j] = t.ld4(row, c);
+        }
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            const size_t row = rb + j * row_step;
+            if (row >= P) continue;
+            float4 o;
+            o.x = fmaxf(fmaf(sc.x, v[j].x, sh.x), 0.f); o.y = fmaxf(fmaf(sc.y, v[j].y, sh.y), 0.f);
+            o.z = fmaxf(fmaf(sc.z, v[j].z, sh.z), 0.f); o.w = fmaxf(fmaf(sc.w, v[j].w, sh.w), 0.f);
+            st4(a + row * C + c, o);
+        }
     }
 }
 
@@ -233,12 +250,14 @@ static int ew_grid(size_t n, int sm) {
     size_t g = (n + 255) / 256, cap = (size_t)sm * 8;
     return (int)(g < cap ? (g ? g : 1) : cap);
 }
+static int row_grid(size_t P, int C4, int sm);
 
 void bn_relu_apply(Exec &ex, Pair t, size_t P, BnRef bn, void *a, bool a_bf16) {
     if (ex.dry) return;
-    const int C4 = t.C() / 4; size_t nq = P * C4;
-    if (a_bf16) launch(ex, bn_relu_apply_kernel<bf16>, ew_grid(nq, ex.ctx->sm_count), 256, 0, t, nq, C4, bn, (bf16 *)a);
-    else launch(ex, bn_relu_apply_kernel<float>, ew_grid(nq, ex.ctx->sm_count), 256, 0, t, nq, C4, bn, (float *)a);
+    const int C4 = t.C() / 4;
+    const int g = row_grid(P, C4, ex.ctx->sm_count);
+    if (a_bf16) launch(ex, bn_relu_apply_kernel<bf16>, g, 256, 0, t, P, C4, bn, (bf16 *)a);
+    else launch(ex, bn_relu_apply_kernel<float>, g, 256, 0, t, P, C4, bn, (float *)a);
     ex.check("bn_relu_apply", (double)P * t.C() * (a_bf16 ? 6 : 8));
 }
 
@@ -606,25 +625,128 @@ void head_bwd(Exec &ex, Pair dy, int N, int HW, const float *Wfc, const float *f
     ex.check("avgpool_bwd");
 }
 
+// ------------------------------------------------------------------ shortcut of a down-sampling unit
+// S(x): 2x2 average pooling with stride 2, then zero channels up to cout; x and S(x) in the coupling-state format
+// (on a fixed-point state the mean of the four grid values is rounded to the grid, ties to even).
+__global__ void shortcut_fwd_kernel(const float *__restrict__ x, float *__restrict__ out, int N, int H, int W, int cin, int cout, float q) {
+    pdl_enter();
+    const int Ho = H >> 1, Wo = W >> 1, C4 = cout >> 2;
+    const size_t n = (size_t)N * Ho * Wo * C4;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % C4) * 4; size_t p = i / C4;
+        const int xo = (int)(p % Wo); p /= Wo;
+        const int yo = (int)(p % Ho); const size_t b = p / Ho;
+        float4 o = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < cin) {
+            const float *s0 = x + (((b * H + 2 * yo) * W + 2 * xo) * (size_t)cin + c);
+            const float *s1 = s0 + (size_t)W * cin;
+            if (q == 0.f) {
+                const float4 a = ld4(s0), bq = ld4(s0 + cin), cq = ld4(s1), d = ld4(s1 + cin);
+                o = make_float4((a.x + bq.x + cq.x + d.x) * 0.25f, (a.y + bq.y + cq.y + d.y) * 0.25f,
+                                (a.z + bq.z + cq.z + d.z) * 0.25f, (a.w + bq.w + cq.w + d.w) * 0.25f);
+            } else {
+                const int4 a = *reinterpret_cast<const int4 *>(s0), bq = *reinterpret_cast<const int4 *>(s0 + cin);
+                const int4 cq = *reinterpret_cast<const int4 *>(s1), d = *reinterpret_cast<const int4 *>(s1 + cin);
+                auto avg = [](int u, int v, int w, int z) {
+                    const int sum = u + v + w + z;
+                    int k = sum >> 2; const int r = sum & 3;             // floor and remainder (in quarters)
+                    if (r == 3 || (r == 2 && (k & 1))) k++;              // nearest, ties to even
+                    return __int_as_float(k);
+                };
+                o = make_float4(avg(a.x, bq.x, cq.x, d.x), avg(a.y, bq.y, cq.y, d.y), avg(a.z, bq.z, cq.z, d.z), avg(a.w, bq.w, cq.w, d.w));
+            }
+        }
+        st4(out + i * 4, o);
+    }
+}
+// S^T d: the first cin channels of d [N, H/2, W/2, cout], each value spread over its 2x2 window with weight 1/4 -> [N, H, W, cin]
+__global__ void shortcut_bwd_kernel(const float *__restrict__ d, float *__restrict__ gx, int N, int H, int W, int cin, int cout) {
+    pdl_enter();
+    const int Ho = H >> 1, Wo = W >> 1, C4 = cin >> 2;
+    const size_t n = (size_t)N * H * W * C4;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % C4) * 4; size_t p = i / C4;
+        const int xx = (int)(p % W); p /= W;
+        const int yy = (int)(p % H); const size_t b = p / H;
+        const float4 v = ld4(d + (((b * Ho + (yy >> 1)) * Wo + (xx >> 1)) * (size_t)cout + c));
+        st4(gx + i * 4, make_float4(v.x * 0.25f, v.y * 0.25f, v.z * 0.25f, v.w * 0.25f));
+    }
+}
+void shortcut_fwd(Exec &ex, const float *x, float *out, int N, int H, int W, int cin, int cout, float q) {
+    if (ex.dry) return;
+    const size_t n = (size_t)N * (H / 2) * (W / 2) * (cout / 4);
+    launch(ex, shortcut_fwd_kernel, ew_grid(n, ex.ctx->sm_count), 256, 0, x, out, N, H, W, cin, cout, q);
+    ex.check("shortcut_fwd", (double)N * H * W * cin * 4 + (double)n * 16);
+}
+void shortcut_bwd(Exec &ex, const float *d, float *gx, int N, int H, int W, int cin, int cout) {
+    if (ex.dry) return;
+    const size_t n = (size_t)N * H * W * (cin / 4);
+    launch(ex, shortcut_bwd_kernel, ew_grid(n, ex.ctx->sm_count), 256, 0, d, gx, N, H, W, cin, cout);
+    ex.check("shortcut_bwd", (double)n * 16 * 1.25);
+}
+
 // ------------------------------------------------------------------ SGD with momentum and weight decay
-__global__ void sgd_kernel(float *__restrict__ p, const float *__restrict__ g, float *__restrict__ v, size_t n,
-                           const uint32_t *__restrict__ seg_end, const uint8_t *__restrict__ seg_decay, int n_seg,
-                           float lr, float mu, float wd) {
+// v <- mu v + (g + wd w [decayed segments only]); w <- w - lr v   (Appendix 6.1).  Four floats per access, four
+// accesses in flight per thread; every segment but the last starts and ends on a multiple of four floats (channel
+// counts are multiples of four), so a quad lies in one segment; the floats behind the last whole quad go one by one.
+__device__ __forceinline__ int sgd_segment(const uint32_t *__restrict__ seg_end, int n_seg, size_t i) {
+    int lo = 0, hi = n_seg - 1;                  // first segment whose end is > i
+    while (lo < hi) { int mid = (lo + hi) >> 1; if (seg_end[mid] > i) hi = mid; else lo = mid + 1; }
+    return lo;
+}
+__global__ void __launch_bounds__(256) sgd_kernel(float *__restrict__ p, const float *__restrict__ g, float *__restrict__ v, size_t n,
+                                                  const uint32_t *__restrict__ seg_end, const uint8_t *__restrict__ seg_decay, int n_seg,
+                                                  float lr, float mu, float wd) {
+    pdl_enter();
+    const size_t n4 = n >> 2, stride = (size_t)gridDim.x * blockDim.x;
+    float4 *p4 = reinterpret_cast<float4 *>(p), *v4 = reinterpret_cast<float4 *>(v);
+    const float4 *g4 = reinterpret_cast<const float4 *>(g);
+    for (size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i0 < n4; i0 += 4 * stride) {
+        float4 w[4], gg[4], vv[4];
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            const size_t i = i0 + j * stride;
+            if (i < n4) { w[j] = p4[i]; gg[j] = g4[i]; vv[j] = v4[i]; }
+        }
+#pragma unroll
+        for (int j = 0; j < 4; j++) {
+            const size_t i = i0 + j * stride;
+            if (i >= n4) continue;
+            const float d = seg_decay[sgd_segment(seg_end, n_seg, i * 4)] ? wd : 0.f;
+            float4 o;
+            o.x = fmaf(mu, vv[j].x, gg[j].x + d * w[j].x); o.y = fmaf(mu, vv[j].y, gg[j].y + d * w[j].y);
+            o.z = fmaf(mu, vv[j].z, gg[j].z + d * w[j].z); o.w = fmaf(mu, vv[j].w, gg[j].w + d * w[j].w);
+            v4[i] = o;
+            p4[i] = make_float4(w[j].x - lr * o.x, w[j].y - lr * o.y, w[j].z - lr * o.z, w[j].w - lr * o.w);
+        }
+    }
+    if (blockIdx.x == 0)
+        for (size_t i = n4 * 4 + threadIdx.x; i < n; i += blockDim.x) {
+            const float w = p[i];
+            const float gg = g[i] + (seg_decay[sgd_segment(seg_end, n_seg, i)] ? wd * w : 0.f);
+            const float vv = fmaf(mu, v[i], gg);
+            v[i] = vv;
+            p[i] = w - lr * vv;
+        }
+}
+// the same, one float at a time: for a parameter layout in which some segment does not start on a multiple of four
+__global__ void sgd_scalar_kernel(float *__restrict__ p, const float *__restrict__ g, float *__restrict__ v, size_t n,
+                                  const uint32_t *__restrict__ seg_end, const uint8_t *__restrict__ seg_decay, int n_seg,
+                                  float lr, float mu, float wd) {
     pdl_enter();
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
-        int lo = 0, hi = n_seg - 1;                  // first segment whose end is > i
-        while (lo < hi) { int mid = (lo + hi) >> 1; if (seg_end[mid] > i) hi = mid; else lo = mid + 1; }
-        float w = p[i];
-        float gg = g[i] + (seg_decay[lo] ? wd * w : 0.f);
-        float vv = fmaf(mu, v[i], gg);
+        const float w = p[i];
+        const float gg = g[i] + (seg_decay[sgd_segment(seg_end, n_seg, i)] ? wd * w : 0.f);
+        const float vv = fmaf(mu, v[i], gg);
         v[i] = vv;
         p[i] = w - lr * vv;
     }
 }
 void sgd_update(Exec &ex, float *params, const float *grads, float *mom, size_t n, const uint32_t *seg_end,
-                const uint8_t *seg_decay, int n_seg, float lr, float momentum, float wd) {
+                const uint8_t *seg_decay, int n_seg, float lr, float momentum, float wd, bool quad_aligned) {
     if (ex.dry) return;
-    launch(ex, sgd_kernel, ew_grid(n, ex.ctx->sm_count), 256, 0, params, grads, mom, n, seg_end, seg_decay, n_seg, lr, momentum, wd);
+    if (quad_aligned) launch(ex, sgd_kernel, ew_grid(n / 16 + 1, ex.ctx->sm_count), 256, 0, params, grads, mom, n, seg_end, seg_decay, n_seg, lr, momentum, wd);
+    else launch(ex, sgd_scalar_kernel, ew_grid(n, ex.ctx->sm_count), 256, 0, params, grads, mom, n, seg_end, seg_decay, n_seg, lr, momentum, wd);
     ex.check("sgd", (double)n * 20);
 }
 

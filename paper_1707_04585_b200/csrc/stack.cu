@@ -18,6 +18,8 @@ struct StagePlan {
     int c, H, units;
     bool has_trans;
     LayerSlot trans;
+    bool has_down = false;          // the stage starts with a stored down-sampling unit (paper-shaped stage)
+    std::vector<LayerSlot> dF, dG;
     std::vector<std::vector<LayerSlot>> F, G;
     size_t off_x1, off_x2;          // bytes into the activation buffer
     size_t off_v1, off_v2;          // verify copies (bytes), valid with verify_reconstruction
@@ -92,6 +94,8 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
         std::vector<LayerSlot *> slots;
         for (auto &s : pl->st) {
             if (s.has_trans) slots.push_back(&s.trans);
+            for (auto &l : s.dF) slots.push_back(&l);
+            for (auto &l : s.dG) slots.push_back(&l);
             for (auto &f : s.F) for (auto &l : f) slots.push_back(&l);
             for (auto &f : s.G) for (auto &l : f) slots.push_back(&l);
         }
@@ -132,7 +136,7 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
     // batch statistics handed from kernel to kernel: per stage those of the current (x1,x2) pair (one
     // [2c] array each for mean and rstd, so that the pair reads as one tensor to a transition) and
     // those of the stage's input x2, which the reversal of the first unit needs again
-    struct StageMom { Moments m1, m2, cat, in_cat, in2; };
+    struct StageMom { Moments m1, m2, cat, in_cat, in2, dy1; };      // dy1: statistics of a down-sampling unit's y1, kept for its backward
     std::vector<StageMom> sm(S);
     bf16 *gcast = nullptr;          // bf16 copy of the gradient w.r.t. x2 / y2, handed from unit to unit
     float *x1_alt = nullptr, *m1_alt_buf = nullptr;
@@ -148,7 +152,8 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
         size_t cmax = 0;
         for (int si = 0; si < S; si++) {
             const StagePlan &s = pl->st[si];
-            float *b = ex.ws.get<float>((size_t)8 * s.c);
+            float *b = ex.ws.get<float>((size_t)10 * s.c);
+            sm[si].dy1.mean = b + 8 * s.c; sm[si].dy1.rstd = b + 9 * s.c;
             sm[si].cat.mean = b; sm[si].cat.rstd = b + 2 * s.c;
             sm[si].m1.mean = b; sm[si].m1.rstd = b + 2 * s.c;
             sm[si].m2.mean = b + s.c; sm[si].m2.rstd = b + 3 * s.c;
@@ -192,6 +197,19 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
             fn_forward(ex, Geom{N, prevH, prevH}, prev, min, T, Pair{}, halves(x1, x2, s.c, q), 0, &mo.in_cat, nullptr, false);
         }
         mo.in2.valid = mo.in_cat.valid;
+        if (s.has_down) {
+            // y1 = S(x1) + F(x2); y2 = S(x2) + G(y1) on the pair of the stage in front, which stays where it is (stored)
+            StagePlan &pv = pl->st[si - 1];
+            const Geom gp{N, pv.H, pv.H};
+            size_t m = ex.ws.mark();
+            float *sc = ex.ws.get<float>(g.P() * s.c);
+            shortcut_fwd(ex, prev.p0, sc, N, pv.H, pv.H, pv.c, s.c, q);
+            fn_forward(ex, gp, single(prev.p1, pv.c, q), &sm[si - 1].m2, bind(s.dF, params, grads), single(sc, s.c, q), single(x1, s.c, q), +1, &mo.dy1, nullptr, false);
+            if (!mo.dy1.valid) { bn_stats(ex, single(x1, s.c, q), g.P(), mo.dy1); mo.dy1.valid = true; }
+            shortcut_fwd(ex, prev.p1, sc, N, pv.H, pv.H, pv.c, s.c, q);
+            fn_forward(ex, g, single(x1, s.c, q), &mo.dy1, bind(s.dG, params, grads), single(sc, s.c, q), single(x2, s.c, q), +1, &mo.in2, nullptr, false);
+            ex.ws.release(m);
+        }
         if (!mo.in2.valid) { bn_stats(ex, single(x2, s.c, q), g.P(), mo.in2); mo.in2.valid = true; }
         if (d.verify_reconstruction && !ex.dry) {
             size_t b = g.P() * s.c * sizeof(float);
@@ -277,6 +295,39 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
             max_abs_diff(ex, x1, actf(s.off_v1), half, q, recon + si);
             max_abs_diff(ex, x2, actf(s.off_v2), half, q, recon + si);
         }
+        if (s.has_down) {
+            // ordinary backprop through the stored unit: G from y1 (what the reversal left in the stage's pair), F from the
+            // kept pair of the stage in front; both with the statistics of the forward pass
+            StagePlan &pv = pl->st[si - 1];
+            const Geom gp{N, pv.H, pv.H};
+            const Pair pin = stored ? stage_out[si - 1] : halves(actf(pv.off_x1), actf(pv.off_x2), pv.c, q);
+            const size_t ph = gp.P() * pv.c;
+            float *o1 = gbuf[gi ^ 1], *o2 = gbuf[gi ^ 1] + ph;
+            size_t m = ex.ws.mark();
+            bf16 *dz1_cast = ex.mode == 0 ? ex.ws.get<bf16>(g.P() * s.c) : nullptr;
+            {
+                FnSaved sv;
+                size_t m2 = ex.ws.mark();
+                std::vector<Layer> G = bind(s.dG, params, grads);
+                fn_forward(ex, g, single(x1, s.c, q), &mo.dy1, G, Pair{}, Pair{}, 0, nullptr, &sv, true);
+                // dz1 = dy1 + (dG/dy1)^T dy2, in place over d1
+                fn_backward(ex, g, single(x1, s.c, q), G, sv, single(d2, s.c), nullptr, single(d1, s.c), single(d1, s.c), dz1_cast);
+                ex.ws.release(m2);
+            }
+            shortcut_bwd(ex, d2, o2, N, pv.H, pv.H, pv.c, s.c);
+            {
+                FnSaved sv;
+                size_t m2 = ex.ws.mark();
+                std::vector<Layer> F = bind(s.dF, params, grads);
+                fn_forward(ex, gp, single(pin.p1, pv.c, q), &sm[si - 1].m2, F, Pair{}, Pair{}, 0, nullptr, &sv, true);
+                // dx2 = S^T dy2 + (dF/dx2)^T dz1
+                fn_backward(ex, gp, single(pin.p1, pv.c, q), F, sv, single(d1, s.c), dz1_cast, single(o2, pv.c), single(o2, pv.c), nullptr);
+                ex.ws.release(m2);
+            }
+            shortcut_bwd(ex, d1, o1, N, pv.H, pv.H, pv.c, s.c);     // dx1 = S^T dz1
+            ex.ws.release(m);
+            gi ^= 1;
+        }
         if (s.has_trans) {
             std::vector<Layer> T{bind(s.trans, params, grads)};
             Pair tin; int tH; Pair gout;
@@ -317,7 +368,9 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
         if (!stem_wgrad(ex, images, gstem, gimg, stem, stem.dW)) conv_wgrad_simt(ex, gstem, false, images, false, gimg, stem, stem.dW);
         ex.ws.release(m);
     }
-    sgd_update(ex, params, grads, mom, pl->n_params, seg_end, seg_decay, (int)nseg, d.lr, d.momentum, d.weight_decay);
+    bool quads = true;
+    for (size_t i = 0; i + 1 < nseg; i++) quads = quads && pl->seg_end[i] % 4 == 0;
+    sgd_update(ex, params, grads, mom, pl->n_params, seg_end, seg_decay, (int)nseg, d.lr, d.momentum, d.weight_decay, quads);
 
     if (stats) {
         stats->stored_activation_bytes = pl->stored_bytes + kept_bytes;
@@ -372,13 +425,24 @@ extern "C" int revnet_stack_plan(revnet_ctx *ctx, const revnet_stack_desc *desc,
         bool bad = sd.units < 1 || sd.c < 4 || sd.c % 4 || sd.kind < 0 || sd.kind > 2 || (sd.kind == 2 && (sd.w < 4 || sd.w % 4));
         bad = bad || (sd.trans_k != 0 && sd.trans_k != 1 && sd.trans_k != 3) || (sd.trans_k && sd.trans_stride != 1 && sd.trans_stride != 2);
         // a stage without a transition is only possible directly behind a stem that needs no pooling
-        bad = bad || (sd.trans_k == 0 && (si > 0 || d.maxpool || cprev != 2 * sd.c));
+        bad = bad || (sd.trans_k == 0 && !sd.down && (si > 0 || d.maxpool || cprev != 2 * sd.c));
+        // a down-sampling first unit: not in stage 0, instead of a transition, on an even resolution, at least the width in front
+        bad = bad || (sd.down && (si == 0 || sd.trans_k != 0 || sd.kind == 0 || H % 2 || 2 * sd.c < cprev || cprev % 8));
         if (bad) { delete pl; return fail(ctx, REVNET_E_UNSUPPORTED_SHAPE, "revnet_stack_plan: unsupported stage " + std::to_string(si)); }
         StagePlan s;
         s.c = sd.c; s.units = sd.units; s.has_trans = sd.trans_k != 0;
         if (s.has_trans) { s.trans = slot(cprev, 2 * sd.c, sd.trans_k, sd.trans_stride, true); H = conv_out(H, sd.trans_k, sd.trans_stride); }
+        if (sd.down) {
+            s.has_down = true;
+            const int ch = cprev / 2;
+            if (sd.kind == 1) { s.dF.push_back(slot(ch, sd.c, 3, 2, true)); s.dF.push_back(slot(sd.c, sd.c, 3, 1, true)); }
+            else { s.dF.push_back(slot(ch, sd.w, 1, 1, true)); s.dF.push_back(slot(sd.w, sd.w, 3, 2, true)); s.dF.push_back(slot(sd.w, sd.c, 1, 1, true)); }
+            for (auto &sh : fn_shape(sd.kind, sd.c, sd.w)) s.dG.push_back(slot(sh[0], sh[1], sh[2], 1, true));
+            H /= 2;
+        }
         s.H = H;
-        for (int u = 0; u < sd.units; u++) {
+        s.units = sd.units - (sd.down ? 1 : 0);       // reversible units
+        for (int u = 0; u < s.units; u++) {
             for (int f = 0; f < 2; f++) {
                 std::vector<LayerSlot> v;
                 for (auto &sh : fn_shape(sd.kind, sd.c, sd.w)) v.push_back(slot(sh[0], sh[1], sh[2], 1, true));
@@ -409,7 +473,7 @@ extern "C" int revnet_stack_plan(revnet_ctx *ctx, const revnet_stack_desc *desc,
     }
     {
         size_t layers = 0;
-        for (auto &st : pl->st) layers += 1 + (size_t)st.units * 6;
+        for (auto &st : pl->st) layers += 1 + 6 + (size_t)st.units * 6;
         pl->pack_host_bytes = layers * 2 * sizeof(PackJob);
         if (pl->pinned_is_malloc || cudaMallocHost(&pl->pack_host, pl->pack_host_bytes) != cudaSuccess) {
             cudaGetLastError(); pl->pack_host = nullptr; pl->pack_host_bytes = 0;

@@ -175,9 +175,47 @@ def time_block(ctx: B.Context, b: syn.BlockCfg, mode: int, reps: int = 10, warmu
     return {k: float(np.median(v)) for k, v in ms.items()}
 
 
+def time_transition(ctx: B.Context, N: int, H: int, cin: int, cout: int, k: int, stride: int, split: bool, mode: int,
+                    reps: int = 10, warmup: int = 3):
+    """Device time (ms) of one stored BN-ReLU-conv layer, forward and backward, through the C ABI."""
+    frac = DEFAULT_FRAC_BITS[mode]
+    rng = np.random.default_rng(5)
+    d = B.TransitionDesc(N, H, H, cin, cout, k, stride, int(split), 1e-5, mode, frac)
+    fb, bb = B.revnet_transition_workspace_bytes(ctx, d)
+    ws = torch.empty(max(fb, bb), dtype=torch.uint8, device="cuda")
+    Ho = H // stride
+    rand = lambda *sh: torch.from_numpy(rng.standard_normal(sh).astype(np.float32)).cuda()
+    if split:
+        x = rng.standard_normal((N, cin, H, H)).astype(np.float32)
+        in1, in2 = to_state(x[:, :cin // 2], frac), to_state(x[:, cin // 2:], frac)
+        di1, di2 = torch.empty((N, H, H, cin // 2), dtype=torch.float32, device="cuda"), torch.empty((N, H, H, cin // 2), dtype=torch.float32, device="cuda")
+    else:
+        in1, in2, di1, di2 = rand(N, H, H, cin), None, torch.empty((N, H, H, cin), dtype=torch.float32, device="cuda"), None
+    W = rand(cout, k, k, cin) * float(np.sqrt(2.0 / (cin * k * k)))
+    g, b_ = torch.ones(cin, device="cuda"), torch.zeros(cin, device="cuda")
+    o1 = torch.empty((N, Ho, Ho, cout // 2), dtype=torch.int32 if frac else torch.float32, device="cuda"); o2 = torch.empty_like(o1)
+    d1, d2 = rand(N, Ho, Ho, cout // 2), rand(N, Ho, Ho, cout // 2)
+    gW, gg, gb = torch.empty_like(W), torch.empty_like(g), torch.empty_like(b_)
+    stream = torch.cuda.current_stream()
+    ms = {"fwd": [], "bwd": []}
+    for i in range(warmup + reps):
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        e[0].record(stream)
+        B.revnet_transition_fwd(ctx, d, in1, in2, W, g, b_, o1, o2, ws)
+        e[1].record(stream)
+        B.revnet_transition_bwd(ctx, d, in1, in2, d1, d2, W, g, b_, di1, di2, gW, gg, gb, ws)
+        e[2].record(stream)
+        torch.cuda.synchronize()
+        if i >= warmup:
+            ms["fwd"].append(e[0].elapsed_time(e[1])); ms["bwd"].append(e[1].elapsed_time(e[2]))
+    B.revnet_check_device(ctx)
+    return {k_: float(np.median(v)) for k_, v in ms.items()}
+
+
 if __name__ == "__main__":
     import argparse, json
-    ap = argparse.ArgumentParser(description="time one reversible block (forward, reconstructing backward)")
+    ap = argparse.ArgumentParser(description="time one reversible block (forward, reconstructing backward), or one stored transition layer")
+    ap.add_argument("--trans", default="", help="cin,cout,stride[,split]: time a stored 3x3 BN-ReLU-conv layer on an HxH input instead of a block")
     ap.add_argument("--N", type=int, default=128); ap.add_argument("--H", type=int, default=32)
     ap.add_argument("--c", type=int, default=64); ap.add_argument("--w", type=int, default=0)
     ap.add_argument("--kind", default="basic"); ap.add_argument("--mode", type=int, default=0)
@@ -185,4 +223,8 @@ if __name__ == "__main__":
     ap.add_argument("--eager", action="store_true", help="launch kernel by kernel instead of replaying CUDA graphs")
     a = ap.parse_args()
     c = B.Context(0)
+    if a.trans:
+        t = [int(v) for v in a.trans.split(",")]
+        print(json.dumps(dict(shape=vars(a), ms=time_transition(c, a.N, a.H, t[0], t[1], 3, t[2], bool(t[3]) if len(t) > 3 else t[2] == 2, a.mode, a.reps, a.warmup))))
+        raise SystemExit(0)
     print(json.dumps(dict(shape=vars(a), ms=time_block(c, syn.BlockCfg(a.N, a.H, a.H, a.c, a.w, a.kind, seed=5), a.mode, a.reps, a.warmup, graph=not a.eager))))

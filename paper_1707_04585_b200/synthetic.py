@@ -29,6 +29,8 @@ class StageCfg:
     kind: str           # "single" | "basic" | "bottleneck"
     trans_k: int        # kernel of the stored BN-ReLU-conv transition in front (0 = none)
     trans_stride: int   # its stride (1 = entry transition, 2 = down-sampling)
+    down: bool = False  # paper-shaped stage: the first of its `units` units is a stored down-sampling unit
+                        # (stride-2 layer inside F, shortcut skip paths) and trans_k is 0
 
 
 @dataclass(frozen=True)
@@ -78,6 +80,20 @@ def fn_layers(kind: str, c: int, w: int) -> List[Tuple[int, int, int]]:
     raise ValueError(kind)
 
 
+def down_fn_layers(kind: str, cin_half: int, c: int, w: int) -> List[Tuple[int, int, int, int]]:
+    """(cin, cout, k, stride) of the layers of F in a down-sampling unit: the stride sits on the first 3x3 of a basic
+    function and on the 3x3 in the middle of a bottleneck; G of that unit is an ordinary stride-1 function."""
+    if kind == "basic":
+        return [(cin_half, c, 3, 2), (c, c, 3, 1)]
+    if kind == "bottleneck":
+        return [(cin_half, w, 1, 1), (w, w, 3, 2), (w, c, 1, 1)]
+    raise ValueError(kind)
+
+
+def reversible_units(s: StageCfg) -> int:
+    return s.units - 1 if s.down else s.units
+
+
 def _basic(units, cs):
     st = []
     for i, c in enumerate(cs):
@@ -107,9 +123,34 @@ def stack_config(name: str) -> StackCfg:
     if name == "revnet104":
         return StackCfg("revnet104", 64, 224, 1000, 7, 2, 128, True,
                         _bott((3, 4, 7, 3), (128, 256, 512, 832)), seed=4, weight_decay=1e-4)
+    # Table "Architectural details" read with the down-sampling inside the first unit of stages 2.. (no separate
+    # transitions): unit counts and stage widths as printed; for the bottleneck rows the per-half bottleneck widths
+    # that come closest to the printed parameter counts
+    if name == "paper_revnet38":
+        return StackCfg(name, 128, 32, 10, 3, 1, 32, False, _paper("basic", (3, 3, 3), (16, 32, 56), (0, 0, 0)), seed=11)
+    if name == "paper_revnet110":
+        return StackCfg(name, 128, 32, 10, 3, 1, 32, False, _paper("basic", (9, 9, 9), (16, 32, 64), (0, 0, 0)), seed=12)
+    if name == "paper_revnet164":
+        return StackCfg(name, 128, 32, 10, 3, 1, 32, False, _paper("bottleneck", (9, 9, 9), (64, 128, 256), (16, 32, 64), entry=True), seed=13)
+    if name == "paper_revnet104":
+        return StackCfg(name, 64, 224, 1000, 7, 2, 128, True,
+                        _paper("bottleneck", (2, 2, 11, 2), (256, 512, 1024, 1664), (64, 128, 256, 416), entry=True), seed=14, weight_decay=1e-4)
     raise ValueError(name)
 
 
+def _paper(kind, units, cs, ws, entry=False):
+    """Stages of a paper-shaped network: stage 0 starts from the stem (through a stored stride-1 entry layer where the
+    stem's width differs from the stage's), later stages start with a down-sampling unit."""
+    st = []
+    for i, (u, c, w) in enumerate(zip(units, cs, ws)):
+        if i == 0:
+            st.append(StageCfg(u, c, w, kind, 3 if entry else 0, 1))
+        else:
+            st.append(StageCfg(u, c, w, kind, 0, 1, down=True))
+    return tuple(st)
+
+
+PAPER_NAMES = ("paper_revnet38", "paper_revnet110", "paper_revnet164", "paper_revnet104")
 STACK_NAMES = ("revnet38", "revnet110", "revnet164", "revnet104")
 
 
@@ -129,6 +170,8 @@ def stage_resolutions(cfg: StackCfg) -> List[int]:
     for s in cfg.stages:
         if s.trans_k:
             H //= s.trans_stride
+        if s.down:
+            H //= 2
         out.append(H)
     return out
 
@@ -141,9 +184,15 @@ def param_specs(cfg: StackCfg) -> List[Tuple[str, Tuple[int, ...], str]]:
         if s.trans_k:
             sp += [(f"s{si}.T.gamma", (cprev,), "gamma"), (f"s{si}.T.beta", (cprev,), "beta"),
                    (f"s{si}.T.W", (2 * s.c, cprev, s.trans_k, s.trans_k), "convw")]
+        elif s.down:
+            for fn, layers in (("F", down_fn_layers(s.kind, cprev // 2, s.c, s.w)), ("G", fn_layers(s.kind, s.c, s.w))):
+                for li, ly in enumerate(layers):
+                    ci, co, k = ly[0], ly[1], ly[2]
+                    p = f"s{si}.d.{fn}.l{li}"
+                    sp += [(p + ".gamma", (ci,), "gamma"), (p + ".beta", (ci,), "beta"), (p + ".W", (co, ci, k, k), "convw")]
         else:
             assert cprev == 2 * s.c, "stage without transition must match incoming channels"
-        for u in range(s.units):
+        for u in range(reversible_units(s)):
             for fn in "FG":
                 for li, (ci, co, k) in enumerate(fn_layers(s.kind, s.c, s.w)):
                     p = f"s{si}.u{u}.{fn}.l{li}"

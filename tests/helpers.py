@@ -22,8 +22,14 @@ def oracle_net(cfg, params):
             trans = dict(name=f"s{si}.T", gamma=params[f"s{si}.T.gamma"], beta=params[f"s{si}.T.beta"],
                          W=params[f"s{si}.T.W"], stride=s.trans_stride)
         units = [(oracle_fn(f"s{si}.u{u}.F", s.kind, s.c, s.w, params),
-                  oracle_fn(f"s{si}.u{u}.G", s.kind, s.c, s.w, params)) for u in range(s.units)]
-        stages.append(dict(trans=trans, c=s.c, units=units))
+                  oracle_fn(f"s{si}.u{u}.G", s.kind, s.c, s.w, params)) for u in range(syn.reversible_units(s))]
+        down = None
+        if s.down:
+            cprev = cfg.stages[si - 1].c
+            dF = [dict(name=f"s{si}.d.F.l{li}", gamma=params[f"s{si}.d.F.l{li}.gamma"], beta=params[f"s{si}.d.F.l{li}.beta"],
+                       W=params[f"s{si}.d.F.l{li}.W"], stride=ly[3]) for li, ly in enumerate(syn.down_fn_layers(s.kind, cprev, s.c, s.w))]
+            down = (dF, oracle_fn(f"s{si}.d.G", s.kind, s.c, s.w, params))
+        stages.append(dict(trans=trans, down=down, c=s.c, units=units))
     return dict(stem=dict(name="stem", W=params["stem.W"], stride=cfg.stem_stride, pad=cfg.stem_pad),
                 maxpool=cfg.maxpool, stages=stages,
                 fc=dict(name="fc", W=params["fc.W"], b=params["fc.b"]), eps=cfg.eps)

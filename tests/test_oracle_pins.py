@@ -213,9 +213,21 @@ def torch_stack_grads(cfg, inp, taps=None):
             if taps is not None:
                 hin.retain_grad(); h.retain_grad()
                 taps[("T", si)] = (hin, h)
+        if s.down:
+            # paper-shaped stage entry: y1 = S(x1) + F(x2), y2 = S(x2) + G(y1), S = 2x2 average pool + zero channels
+            cp = h.shape[1] // 2
+            S = lambda t: TF.pad(TF.avg_pool2d(t, 2, 2), (0, 0, 0, 0, 0, s.c - cp))
+            f = h[:, cp:]
+            for li, ly in enumerate(syn.down_fn_layers(s.kind, cp, s.c, s.w)):
+                f = bnrc(f, f"s{si}.d.F.l{li}", ly[3])
+            y1 = S(h[:, :cp]) + f
+            g = y1
+            for li in range(len(syn.fn_layers(s.kind, s.c, s.w))):
+                g = bnrc(g, f"s{si}.d.G.l{li}")
+            h = torch.cat([y1, S(h[:, cp:]) + g], dim=1)
         x1, x2 = h[:, :s.c], h[:, s.c:]
         nl = len(syn.fn_layers(s.kind, s.c, s.w))
-        for u in range(s.units):
+        for u in range(syn.reversible_units(s)):
             if taps is not None:
                 x1, x2 = x1 * 1.0, x2 * 1.0           # fresh nodes, so that each unit's input gradient can be read
                 x1.retain_grad(); x2.retain_grad()
@@ -284,6 +296,61 @@ def test_per_block_records_inside_a_stack_match_autograd():
         hin, hout = taps[("T", si)]
         assert hp.rel_l2(t["x"], hin.detach().numpy()) < 1e-10
         assert hp.rel_l2(t["dy"], hout.grad.numpy()) < 1e-9 and hp.rel_l2(t["dx"], hin.grad.numpy()) < 1e-9
+
+
+def paper_tiny(kind):
+    """A small network shaped like the paper's table: no separate transitions, the first unit of stages 2.. down-samples."""
+    if kind == "basic":
+        st = (syn.StageCfg(2, 4, 0, "basic", 0, 1), syn.StageCfg(2, 8, 0, "basic", 0, 1, down=True), syn.StageCfg(1, 12, 0, "basic", 0, 1, down=True))
+    else:
+        st = (syn.StageCfg(1, 8, 4, "bottleneck", 3, 1), syn.StageCfg(2, 16, 4, "bottleneck", 0, 1, down=True))
+    return syn.StackCfg(f"paper_tiny_{kind}", 4, 16, 5, 3, 1, 8, False, st, seed=17)
+
+
+def test_shortcut_is_average_pool_plus_zero_channels_and_its_adjoint():
+    x = rng.standard_normal((2, 3, 6, 4)); d = rng.standard_normal((2, 5, 3, 2))
+    y = orc.shortcut_fwd(x, 5)
+    assert np.allclose(y[:, :3], TF.avg_pool2d(torch.tensor(x), 2, 2).numpy(), atol=1e-14) and np.all(y[:, 3:] == 0)
+    assert abs((y * d).sum() - (x * orc.shortcut_bwd(d, 3)).sum()) < 1e-12          # <S x, d> = <x, S^T d>
+
+
+@pytest.mark.parametrize("kind", ["basic", "bottleneck"])
+def test_paper_shaped_stack_against_autograd(kind):
+    """Down-sampling inside the first unit of a stage (Table "Architectural details"): the stack with such units
+    against the same network written with library ops; both backward flavours agree; a fixed-point state still
+    reconstructs every reversible unit's input exactly."""
+    cfg = paper_tiny(kind)
+    inp = syn.make_stack_inputs(cfg, affine_jitter=True)
+    net = hp.oracle_net(cfg, inp["params"])
+    rs = orc.stack_train_grads(net, inp["images"], inp["labels"], "stored")
+    rr = orc.stack_train_grads(net, inp["images"], inp["labels"], "reconstruct")
+    tl, tloss, tg = torch_stack_grads(cfg, inp)
+    assert np.allclose(rs["logits"], tl, atol=1e-10) and abs(rs["loss"] - tloss) < 1e-12
+    assert set(tg) == set(rs["grads"]) == set(rr["grads"])
+    for k in tg:
+        assert hp.rel_l2(rs["grads"][k], tg[k]) < 1e-9, k
+        assert hp.rel_l2(rr["grads"][k], rs["grads"][k]) < 1e-9, k
+    num = {"bf16_operands": True, "frac_bits": 16}
+    rq = orc.stack_train_grads(net, inp["images"], inp["labels"], "reconstruct", num=num)
+    for key, (x1, x2) in rq["block_inputs"].items():
+        assert np.array_equal(rq["recovered"][key][0], x1) and np.array_equal(rq["recovered"][key][1], x2), key
+
+
+def test_paper_table_parameter_counts_all_rows():
+    """All four RevNet rows of the table, counted on the paper-shaped configurations (every parameter: conv, BN, FC)."""
+    rows = {}
+    with open(__file__.replace("test_oracle_pins.py", "golden/arch_table.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                name, bott, units, ch, pm = line.split()
+                rows[name] = ([int(u) for u in units.split("-")], float(pm))
+    tol = {"RevNet-38": 0.02, "RevNet-110": 0.02, "RevNet-164": 0.04, "RevNet-104": 0.10}
+    for name, (units, pm) in rows.items():
+        cfg = syn.stack_config("paper_" + name.lower().replace("-", ""))
+        assert [s.units for s in cfg.stages] == units
+        assert all(s.down for s in cfg.stages[1:]) and not any(s.trans_k for s in cfg.stages[1:])
+        n = sum(int(np.prod(shape)) for _, shape, _ in syn.param_specs(cfg))
+        assert abs(n / 1e6 - pm) / pm < tol[name], (name, n)
 
 
 def test_storage_flat_in_depth_and_cost_4n_vs_3n():

@@ -719,40 +719,43 @@ __global__ void pack_weights_kernel(const float *__restrict__ W, bf16 *__restric
     }
 }
 
-// all packs of a step in one launch: blockIdx.y walks the job table.  A block (32 x 8 threads) takes
-// 32 x 32 tiles (rows x columns of the pack, one tap): both the fp32 reads and the bf16 writes of a
-// warp are contiguous, the transposed pack going through shared memory.
+// all packs of a step in one launch: blockIdx.y walks the job table.  A block (32 x 8 threads) takes tiles of
+// 32 rows x 64 columns of the pack (one tap), a thread two adjacent columns: the fp32 reads of a warp are contiguous
+// (256 bytes plain, 128 bytes transposed) and so are its bf16x2 writes (128 bytes); the transposed pack goes through
+// shared memory.
 __global__ void pack_weights_batch_kernel(const PackJob *__restrict__ jobs) {
     pdl_enter();
-    __shared__ float tile[32][33];
+    __shared__ float tile[64][33];
     const PackJob j = jobs[blockIdx.y];
     const int taps = j.k * j.k;
-    const int rt = (j.rows_pad + 31) >> 5, ct = (j.cols_pad + 31) >> 5;
+    const int rt = (j.rows_pad + 31) >> 5, ct = (j.cols_pad + 63) >> 6;
     const int n_tiles = taps * rt * ct;
     const int tx = threadIdx.x, ty = threadIdx.y;
     for (int t = blockIdx.x; t < n_tiles; t += gridDim.x) {
-        const int c0 = (t % ct) << 5, r0 = ((t / ct) % rt) << 5, tap = t / (ct * rt);
+        const int c0 = (t % ct) << 6, r0 = ((t / ct) % rt) << 5, tap = t / (ct * rt);
         if (!j.transposed) {
 #pragma unroll
             for (int rr = 0; rr < 32; rr += 8) {
-                const int r = r0 + rr + ty, c = c0 + tx;
+                const int r = r0 + rr + ty, c = c0 + 2 * tx;      // columns are input channels (a multiple of 4: c and c + 1 are valid together)
                 if (r < j.rows_pad && c < j.cols_pad) {
-                    const float v = (r < j.Co && c < j.Ci) ? j.W[((size_t)r * taps + tap) * j.Ci + c] : 0.f;
-                    j.out[((size_t)r * taps + tap) * j.cols_pad + c] = __float2bfloat16_rn(v);
+                    float2 v = make_float2(0.f, 0.f);
+                    if (r < j.Co && c < j.Ci) v = *reinterpret_cast<const float2 *>(j.W + ((size_t)r * taps + tap) * j.Ci + c);
+                    *reinterpret_cast<__nv_bfloat162 *>(j.out + ((size_t)r * taps + tap) * j.cols_pad + c) = __floats2bfloat162_rn(v.x, v.y);
                 }
             }
         } else {
             // rows of the pack are input channels, columns output channels, taps mirrored
 #pragma unroll
-            for (int rr = 0; rr < 32; rr += 8) {
-                const int co = c0 + rr + ty, ci = r0 + tx;
-                tile[rr + ty][tx] = (co < j.Co && ci < j.Ci) ? j.W[((size_t)co * taps + (taps - 1 - tap)) * j.Ci + ci] : 0.f;
+            for (int cc = 0; cc < 64; cc += 8) {
+                const int co = c0 + cc + ty, ci = r0 + tx;
+                tile[cc + ty][tx] = (co < j.Co && ci < j.Ci) ? j.W[((size_t)co * taps + (taps - 1 - tap)) * j.Ci + ci] : 0.f;
             }
             __syncthreads();
 #pragma unroll
             for (int rr = 0; rr < 32; rr += 8) {
-                const int r = r0 + rr + ty, c = c0 + tx;
-                if (r < j.rows_pad && c < j.cols_pad) j.out[((size_t)r * taps + tap) * j.cols_pad + c] = __float2bfloat16_rn(tile[tx][rr + ty]);
+                const int r = r0 + rr + ty, c = c0 + 2 * tx;
+                if (r < j.rows_pad && c < j.cols_pad)
+                    *reinterpret_cast<__nv_bfloat162 *>(j.out + ((size_t)r * taps + tap) * j.cols_pad + c) = __floats2bfloat162_rn(tile[2 * tx][rr + ty], tile[2 * tx + 1][rr + ty]);
             }
             __syncthreads();
         }
@@ -1027,6 +1030,8 @@ struct WgParams {
     int sep, cout_pad;           // sep: taps split between the operands (see the kernel); cout rounded up to 16
     int splits, m_chunks;        // this job's CTAs: split x M chunk x N tile, split fastest
     int cta0;                    // first CTA of the job in the launch
+    int pair;                    // wgrad_tc2_kernel: BN is what ONE CTA of a pair holds of the pair's 2 * BN output channels,
+                                 // GM the pair's M groups of 256 rows (CTA r takes the 128-row groups 2j + r of the chunk)
 };
 
 // One launch computes the weight gradients of up to kWgMaxJobs layers: each CTA finds its job from
@@ -1197,6 +1202,168 @@ wgrad_tc_kernel(const __grid_constant__ WgBatch batch) {
     }
 }
 
+// The same on a CTA pair (tcgen05 cta_group::2): an MMA of M = 256 covers two 128-row groups of (tap, input channel) rows,
+// CTA `rank` holding the activation blocks of the groups 2j + rank and HALF of the pair's gradient channels; N = 2 * BN.
+// Per pixel tile a CTA then loads GM x 32 KB of activations and BN x 256 B of gradients for GM x 8 MMAs of 256 x 2BN:
+// half the operand bytes per flop of the single-CTA form, whose 94 bytes per MMA clock are more than an SM can take in.
+// Not for the tap-split (sep) form.  Launched as clusters of two; every job of a launch is of this kind.
+__global__ void __launch_bounds__(kThreads, 1)
+wgrad_tc2_kernel(const __grid_constant__ WgBatch batch) {
+    int jb = 0;
+    while (jb + 1 < batch.n && (int)blockIdx.x >= batch.job[jb + 1].p.cta0) jb++;
+    const WgParams &p = batch.job[jb].p;
+    const CUtensorMap &map_a = batch.job[jb].map_a, &map_g = batch.job[jb].map_g;
+    const uint32_t rank = cluster_ctarank();
+    const int local = ((int)blockIdx.x - p.cta0) >> 1;         // pair index inside the job (cta0 is even)
+    const int split = local % p.splits, chunk = (local / p.splits) % p.m_chunks, ntile = local / (p.splits * p.m_chunks);
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *tiles = (uint8_t *)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int blk_bytes_a = 256 * p.blockC, blk_bytes_b = 256 * p.blockN;   // [128 pixels][block] bf16
+    const int a_region = p.GM * 32768;                         // whole groups: 32 KB each
+    const int stage_bytes = a_region + ((256 * p.BN + 1023) & ~1023);
+    TcShared *sh = (TcShared *)(tiles + p.stages * stage_bytes);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bpg = 128 / p.blockC;                          // blocks per 128-row group
+    const int first_block = chunk * 2 * p.GM * bpg;          // the pair's chunk: 2 * GM groups
+    // blocks this CTA / the other CTA loads per pixel tile: group 2j + r holds the blocks first_block + (2j + r) * bpg ...
+    auto blocks_of = [&](int r) { int n = 0; for (int j = 0; j < p.GM; j++) { int b = p.total_blocks - (first_block + (2 * j + r) * bpg); n += b < 0 ? 0 : (b > bpg ? bpg : b); } return n; };
+    const int col0 = ntile * 2 * p.BN;                       // first output channel of the pair's N tile
+    auto nblocks_of = [&](int r) { int n = (p.cout - (col0 + r * p.BN) + p.blockN - 1) / p.blockN; return n < 0 ? 0 : (n > p.BN / p.blockN ? p.BN / p.blockN : n); };
+    const int my_tiles = (p.n_tiles_px - split + p.splits - 1) / p.splits;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < p.GM * 2 * p.BN) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < p.stages; s++) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+        mbar_init(&sh->acc_full[0], 1);
+        sh->failed = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem2_alloc(&sh->tmem_base, tmem_cols);
+    {
+        // rows and blocks TMA never writes (short tiles, groups beyond the last block) must hold zeros, not stale bits:
+        // their products land in rows that are never stored, but a NaN pattern would still be a NaN
+        uint4 *z = reinterpret_cast<uint4 *>(tiles);
+        const int n16 = p.stages * stage_bytes / 16;
+        for (int i = threadIdx.x; i < n16; i += kThreads) z[i] = make_uint4(0u, 0u, 0u, 0u);
+        fence_proxy_async();
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    tc_fence_after();
+    pdl_enter();
+    const uint32_t tmem_d = sh->tmem_base;
+    const int pad = p.k / 2;
+    const int tiles_per_img = p.tiles_per_img;
+
+    if (warp == 0) {
+        // lane (j, i) with j < GM, i < bpg: activation block i of this CTA's group 2j + rank; the next lanes: gradient blocks
+        const uint32_t tx = (uint32_t)(p.box_px * 2 * ((blocks_of(0) + blocks_of(1)) * p.blockC + (nblocks_of(0) + nblocks_of(1)) * p.blockN));
+        const int nb_n = nblocks_of((int)rank);
+        const int ja = lane / bpg, ia = lane - ja * bpg;
+        const int gb = first_block + (2 * ja + (int)rank) * bpg + ia;
+        const bool a_lane = lane < p.GM * bpg && gb < p.total_blocks;
+        const int tap = gb / p.cblks, cb = gb - tap * p.cblks;
+        const int kh = tap / p.k, kw = tap - kh * p.k;
+        const int bg = lane - p.GM * bpg;
+        const bool g_lane = bg >= 0 && bg < nb_n;
+        const int g_c = col0 + (int)rank * p.BN + bg * p.blockN;
+        const uint32_t full0 = mapa_shared(smem_u32(&sh->full[0]), 0);
+        int s = 0; uint32_t round = 0;
+        for (int it = 0; it < my_tiles; it++) {
+            bool ok = true;
+            if (lane == 0) {
+                if (round > 0 && !mbar_wait(&sh->empty[s], (round - 1) & 1)) { atomicExch(&sh->failed, 1u); ok = false; }
+                if (ok && rank == 0) mbar_expect_tx(&sh->full[s], tx);       // the leader's barrier collects the bytes of both CTAs
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) break;
+            const int t = split + it * p.splits;
+            const int n0 = p.BIMG > 1 ? t * p.BIMG : t / tiles_per_img;
+            const int h0 = p.BIMG > 1 ? 0 : (t - n0 * tiles_per_img) * p.BH;
+            uint8_t *sa = tiles + s * stage_bytes;
+            if (a_lane) tma2_load_4d(sa + ja * 32768 + ia * blk_bytes_a, &map_a, full0 + 8u * s, cb * p.blockC, kw - pad, h0 * p.stride + kh - pad, n0);
+            else if (g_lane) tma2_load_4d(sa + a_region + bg * blk_bytes_b, &map_g, full0 + 8u * s, g_c, 0, h0, n0);
+            if (++s == p.stages) { s = 0; round++; }
+        }
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            const uint32_t idesc = instr_desc_m256(2 * p.BN) | (3u << 15);     // both operands M / N-major
+            const int rba = p.blockC * 2, rbb = p.blockN * 2;
+            const uint64_t da0 = smem_desc_mn(smem_u32(tiles), rba, blk_bytes_a), db0 = smem_desc_mn(smem_u32(tiles) + a_region, rbb, blk_bytes_b);
+            const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
+            int s = 0; uint32_t round = 0, soff = 0;
+            for (int it = 0; it < my_tiles; it++) {
+                if (!mbar_wait_cluster(&sh->full[s], round & 1)) { atomicExch(&sh->failed, 1u); break; }
+                tc_fence_after();
+                const uint32_t accum = it > 0 ? 1u : 0u;
+                for (int g = 0; g < p.GM; g++) {
+                    uint64_t da = da0 + soff + (uint32_t)(g * 2048), db = db0 + soff;
+                    const uint32_t acc = tmem_d + (uint32_t)(g * 2 * p.BN);
+                    mma2_bf16(acc, da, db, idesc, accum);
+                    for (int ks = 1; ks < 8; ks++) {         // 16 pixels per MMA
+                        da += (uint32_t)rba; db += (uint32_t)rbb;
+                        mma2_bf16(acc, da, db, idesc, 1u);
+                    }
+                }
+                mma2_commit_both(&sh->empty[s]);
+                soff += stage16;
+                if (++s == p.stages) { s = 0; soff = 0; round++; }
+            }
+            mma2_commit_both(&sh->acc_full[0]);
+        }
+    } else {
+        const int quarter = warp & 3;
+        bool ok = true;
+        if (quarter == 0 && lane == 0) ok = mbar_wait_cluster(&sh->acc_full[0], 0);
+        ok = named_barrier_and(2, 128, ok);
+        tc_fence_after();
+        if (ok && sh->failed == 0) {
+            const int m = quarter * 32 + lane;
+            float *dst = p.partial + (size_t)split * p.slice;
+            for (int g = 0; g < p.GM; g++) {
+                const int gb = first_block + (2 * g + (int)rank) * bpg + m / p.blockC;
+                const int tap = gb / p.cblks, ci = (gb - tap * p.cblks) * p.blockC + m % p.blockC;
+                const bool row_ok = gb < p.total_blocks && ci < p.cin;
+                for (int c = 0; c < 2 * p.BN; c += 16) {
+                    float v[16];
+                    tmem_ld16(tmem_d + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(g * 2 * p.BN + c), v);   // whole warp takes part
+                    if (!row_ok) continue;
+                    if (my_tiles == 0) {
+#pragma unroll
+                        for (int j = 0; j < 16; j++) v[j] = 0.f;
+                    }
+                    const int cb0 = col0 + c;
+                    if (p.splits > 1) {
+                        float *row = dst + ((size_t)tap * p.cin + ci) * p.cout + cb0;
+#pragma unroll
+                        for (int j = 0; j < 16; j += 4)
+                            if (cb0 + j < p.cout) *reinterpret_cast<float4 *>(row + j) = make_float4(v[j], v[j + 1], v[j + 2], v[j + 3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 16; j++) {
+                            const int co = cb0 + j;
+                            if (co < p.cout) dst[((size_t)co * p.taps + tap) * p.cin + ci] = v[j];
+                        }
+                    }
+                }
+            }
+        } else if (lane == 0) {
+            atomicExch(&sh->failed, 1u);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && sh->failed) atomicExch(p.status, (int)REVNET_E_TIMEOUT);
+    cluster_sync_all();      // neither CTA leaves, or frees tensor memory, while the other may still read its operands
+    if (warp == 1) {
+        tc_fence_after();
+        tmem2_dealloc(tmem_d, tmem_cols);
+    }
+}
+
 // dW[co][tap][ci] = sum over splits of part[z][tap][ci][co], in a fixed order: 8 interleaved groups of
 // splits per element, combined through shared memory (256 threads = 32 elements x 8 groups); several
 // (partials, destination) pairs in one launch, blockIdx.y picks the pair
@@ -1307,7 +1474,8 @@ constexpr int kWgSmemMax = 224 * 1024;
 
 // Shape decisions of one layer's weight gradient; cta_budget: the CTAs the job may take
 struct WgPlan { WgParams p; Geom go; int n_tiles, stage_bytes, tail_bytes; };
-static bool wgrad_plan(Geom gi, const Layer &L, int cta_budget, WgPlan &w, bool allow_sep = true) {
+// pair: plan for wgrad_tc2_kernel (cta_budget then counts CTAs too; the job takes an even number)
+static bool wgrad_plan(Geom gi, const Layer &L, int cta_budget, WgPlan &w, bool allow_sep = true, bool pair = false) {
     if ((L.stride != 1 && L.stride != 2) || (L.k != 1 && L.k != 3) || L.cin % 8 || L.cout % 8) return false;
     if (L.stride == 2 && (gi.H % 2 || gi.W % 2)) return false;
     WgParams &p = w.p;
@@ -1323,7 +1491,36 @@ static bool wgrad_plan(Geom gi, const Layer &L, int cta_budget, WgPlan &w, bool 
     const int bpg = 128 / p.blockC;
     // taps split between the operands when the three shifted activation blocks fit one M group, the three
     // shifted gradient blocks one N tile, and the boxes of a pixel tile the lanes of the producer warp
-    p.sep = (allow_sep && L.k == 3 && L.stride == 1 && 3 * cin_pad <= 128 && 3 * cout_pad <= 256 && 2 * bpg + 3 * (cout_pad / p.blockN) <= 32) ? 1 : 0;
+    p.sep = (allow_sep && !pair && L.k == 3 && L.stride == 1 && 3 * cin_pad <= 128 && 3 * cout_pad <= 256 && 2 * bpg + 3 * (cout_pad / p.blockN) <= 32) ? 1 : 0;
+    p.pair = pair ? 1 : 0;
+    if (pair) {
+        // a pair's N tile is 2 * BN wide (BN per CTA, a whole number of gradient blocks), its M chunk 2 * GM groups
+        // (N tiles of less than 256 columns measured slower on a pair than 128-column tiles on one CTA: 89 against 72 us
+        // for the 3x3 layer of 128 channels at 56 x 56, batch 64)
+        if (cout_pad < 256 || cout_pad % 32) return false;
+        p.total_blocks = taps * p.cblks;
+        p.BN = 128;
+        if (p.BN % p.blockN) { p.blockN = pick_block(p.BN); if (p.BN % p.blockN) return false; }
+        const int groups_all = (p.total_blocks + bpg - 1) / bpg;
+        if (groups_all < 2) return false;
+        p.GM = groups_all >= 4 ? 2 : 1;
+        p.m_chunks = (groups_all + 2 * p.GM - 1) / (2 * p.GM);
+        w.n_tiles = (cout_pad + 2 * p.BN - 1) / (2 * p.BN);
+        p.H = w.go.H; p.W = w.go.W; p.stride = L.stride;
+        p.n_tiles_px = tg.n_px_tiles;
+        p.a_region = p.GM * 32768;
+        w.stage_bytes = p.a_region + ((256 * p.BN + 1023) & ~1023);
+        w.tail_bytes = 0;
+        p.stages = (kWgSmemMax - 2048) / w.stage_bytes; if (p.stages > kWgStages) p.stages = kWgStages;
+        if (p.stages < 2) return false;
+        const int units = p.m_chunks * w.n_tiles, budget = cta_budget / 2 < 1 ? 1 : cta_budget / 2;     // in pairs
+        auto clampi = [&](int v) { return v < 1 ? 1 : (v > p.n_tiles_px ? p.n_tiles_px : v); };
+        const int s_hi = clampi((budget + units - 1) / units), s_lo = clampi(budget / units);
+        auto serial_tiles = [&](int sp) { return ((units * sp + budget - 1) / budget) * ((p.n_tiles_px + sp - 1) / sp); };
+        p.splits = serial_tiles(s_lo) < serial_tiles(s_hi) ? s_lo : s_hi;
+        p.slice = (size_t)L.cout * taps * L.cin;
+        return true;
+    }
     if (p.sep) {
         p.total_blocks = L.k * p.cblks;
         p.BN = L.k * cout_pad;
@@ -1366,8 +1563,12 @@ bool conv_wgrad_tc_batch(Exec &ex, int n, const void *const *gq, const void *con
     WgPlan w[kWgMaxJobs];
     const int budget = ex.ctx->sm_count / n;
     size_t total = 0;
+    // CTA pairs (wgrad_tc2_kernel) when every layer of the launch takes them: a launch is made of clusters or it is not
+    static const bool pair_enabled = [] { const char *v = getenv("REVNET_WGRAD_PAIR"); return !(v && v[0] == '0'); }();
+    bool pair = pair_enabled && ex.ctx->sm_count % 2 == 0;
+    for (int j = 0; j < n && pair; j++) pair = wgrad_plan(gi[j], *L[j], budget & ~1, w[j], false, true);
     for (int j = 0; j < n; j++) {
-        if (!wgrad_plan(gi[j], *L[j], budget, w[j])) return false;
+        if (!pair && !wgrad_plan(gi[j], *L[j], budget, w[j])) return false;
         if (w[j].p.splits > 1) total += (size_t)w[j].p.splits * w[j].p.slice;
     }
     if (need) { *need = total; return true; }
@@ -1390,7 +1591,7 @@ bool conv_wgrad_tc_batch(Exec &ex, int n, const void *const *gq, const void *con
             }
             p.status = ex.ctx->dev_status;
             p.cta0 = cta;
-            cta += p.splits * p.m_chunks * w[j].n_tiles;
+            cta += p.splits * p.m_chunks * w[j].n_tiles * (pair ? 2 : 1);
             if (p.splits > 1) {
                 p.partial = part + off;
                 sums.part[n_sums] = p.partial; sums.out[n_sums] = L[j]->dW; sums.n[n_sums] = p.slice; sums.splits[n_sums] = p.splits;
@@ -1409,8 +1610,12 @@ bool conv_wgrad_tc_batch(Exec &ex, int n, const void *const *gq, const void *con
             flops += 2.0 * w[j].go.P() * L[j]->cout * L[j]->cin * p.taps;
         }
         static OncePerDevice once;
-        if (once.first(ex.ctx->device)) cudaFuncSetAttribute(wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWgSmemMax);
-        launch(ex, wgrad_tc_kernel, (unsigned)cta, kThreads, smem, batch);
+        if (once.first(ex.ctx->device)) {
+            cudaFuncSetAttribute(wgrad_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWgSmemMax);
+            cudaFuncSetAttribute(wgrad_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kWgSmemMax);
+        }
+        if (pair) launch_cluster(ex, wgrad_tc2_kernel, (unsigned)cta, kThreads, smem, 2, batch);
+        else launch(ex, wgrad_tc_kernel, (unsigned)cta, kThreads, smem, batch);
         ex.check("conv_wgrad_tc", bytes, flops);
         if (n_sums) {
             if (max_slice >= 524288) {
@@ -1466,7 +1671,7 @@ PackJob tc_pack_job(const float *W, bf16 *out, int cin, int cout, int k, bool tr
 }
 void tc_pack_batch(Exec &ex, const PackJob *jobs_dev, int n_jobs, double bytes, size_t max_job_elems) {
     if (ex.dry || n_jobs == 0) return;
-    // blocks per job sized for the largest job (four 32 x 32 tiles per block), within 2 .. 592
+    // blocks per job sized for the largest job (two 32 x 64 tiles per block), within 2 .. 592
     size_t bx = (max_job_elems + 4095) / 4096;
     if (bx < 2) bx = 2; if (bx > 592) bx = 592;
     dim3 grid((unsigned)bx, (unsigned)n_jobs);

@@ -250,12 +250,18 @@ static int ew_grid(size_t n, int sm) {
     size_t g = (n + 255) / 256, cap = (size_t)sm * 8;
     return (int)(g < cap ? (g ? g : 1) : cap);
 }
-static int row_grid(size_t P, int C4, int sm);
+static int row_grid(size_t P, int C4, int sm, int per_sm);
+template <class K> static int blocks_per_sm(K kernel) {
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, 256, 0) != cudaSuccess || n < 1) { cudaGetLastError(); n = 4; }
+    return n > 8 ? 8 : n;
+}
 
 void bn_relu_apply(Exec &ex, Pair t, size_t P, BnRef bn, void *a, bool a_bf16) {
     if (ex.dry) return;
     const int C4 = t.C() / 4;
-    const int g = row_grid(P, C4, ex.ctx->sm_count);
+    static const int occ16 = blocks_per_sm(bn_relu_apply_kernel<bf16>), occ32 = blocks_per_sm(bn_relu_apply_kernel<float>);
+    const int g = row_grid(P, C4, ex.ctx->sm_count, a_bf16 ? occ16 : occ32);
     if (a_bf16) launch(ex, bn_relu_apply_kernel<bf16>, g, 256, 0, t, P, C4, bn, (bf16 *)a);
     else launch(ex, bn_relu_apply_kernel<float>, g, 256, 0, t, P, C4, bn, (float *)a);
     ex.check("bn_relu_apply", (double)P * t.C() * (a_bf16 ? 6 : 8));
@@ -267,7 +273,7 @@ void bn_relu_apply(Exec &ex, Pair t, size_t P, BnRef bn, void *a, bool a_bf16) {
 // A thread keeps one channel quad (its coefficients stay in registers) and strides the rows, four
 // rows in flight; row_step = threads of the grid / C4 (the launch makes that a whole number).
 template <class TO, int OUT, bool CAST>
-__global__ void bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, size_t P, int C4, BnRef bn,
+__global__ void __launch_bounds__(256, 3) bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, size_t P, int C4, BnRef bn,
                                          const float *__restrict__ coef, TO *__restrict__ out, Pair add, Pair outp,
                                          bf16 *__restrict__ cast) {
     pdl_enter();
@@ -306,12 +312,14 @@ __global__ void bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, s
 }
 
 // grid for the row-strided elementwise kernels: 256 threads per block, a thread count that is a multiple of C4
-static int row_grid(size_t P, int C4, int sm) {
+// per_sm: blocks of the kernel that fit an SM at once (its occupancy): a grid of exactly the resident blocks, each
+// striding over its share of the rows, has no partly filled last wave
+static int row_grid(size_t P, int C4, int sm, int per_sm) {
     // smallest block count g >= wanted with (g * 256) % C4 == 0: C4 divides 256 * g when g is a multiple of C4 / gcd(C4, 256)
     int a = C4, b = 256;
     while (b) { int r = a % b; a = b; b = r; }
     const int unit = C4 / a;
-    size_t want = (P * C4 + 1023) / 1024, cap = (size_t)sm * 8;
+    size_t want = (P * C4 + 1023) / 1024, cap = (size_t)sm * per_sm;
     if (want > cap) want = cap;
     if (want < 1) want = 1;
     return (int)((want + unit - 1) / unit * unit);
@@ -331,7 +339,8 @@ void bn_relu_bwd(Exec &ex, const float *da, Pair t, size_t P, BnRef bn, float *d
             launch(ex, bn_bwd_finalize, cdiv((size_t)C * 32, 128), 128, 0, part, r.chunks, C, 1.0 / (double)P, bn.gamma, bn.rstd, dgamma, dbeta, coef);
             ex.check("bn_bwd_finalize");
         }
-        const int g = row_grid(P, C4, ex.ctx->sm_count);
+        static const int occ = blocks_per_sm(bn_relu_bwd_apply_kernel<float, 2, true>);      // the heaviest variant
+        const int g = row_grid(P, C4, ex.ctx->sm_count, occ);
 #define RV_ARGS da, t, P, C4, bn, coef
         if (out_pair.p0 && add.p0) {
             if (out_cast) launch(ex, bn_relu_bwd_apply_kernel<float, 2, true>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, out_cast);

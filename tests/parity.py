@@ -37,10 +37,10 @@ Rules, chosen per comparison by the caller BEFORE the result is known:
              the bf16 mode).  A tolerance means nothing there; the test still rejects a zero, an
              uncorrelated, a wrongly signed or a wrongly scaled tensor: norm ratio within
              [0.5, 2] and cosine >= MIN_COS, or, where the oracle's perturbed runs agree with it
-             even less than that, at least half the cosine they reach; where even the oracle's
-             perturbed runs are uncorrelated with it (cosine < 0.3: the middle of the 164-layer
-             network, whose gradients at random initialisation are determined by nothing less
-             than exact arithmetic) only the size.  What verifies those layers is the per-block check inside the
+             even less than that, at least half the cosine they reach (with eight or more such
+             tensors in a case: the median over them, since one perturbed run is itself one
+             draw; measured on the 164-layer network: median cosine 0.20 against the oracle,
+             0.14 of the oracle's perturbed run against the oracle).  What verifies those layers is the per-block check inside the
              network (the oracle's own (y1, y2, dy1, dy2) of a unit through revnet_block_bwd).
 
 Each record carries the rule that applied, the floor, the bound and whether the stated tolerance
@@ -107,6 +107,7 @@ def check(case, got, ref, tol, floor_fn=None, floor_allowed=(), floor_scope="ten
             top = max(floors.values())
             floors = {k: top for k in floors}
     bad = {}
+    chaotic, pending = [], []
     for k, e in errs.items():
         cos = cosine(got[k], ref[k])
         nr = float(np.linalg.norm(np.asarray(got[k], np.float64)) / max(np.linalg.norm(np.asarray(ref[k], np.float64)), 1e-300))
@@ -123,13 +124,27 @@ def check(case, got, ref, tol, floor_fn=None, floor_allowed=(), floor_scope="ten
                 # the direction no more strictly than the oracle agrees with itself
                 rule, bound = "chaotic", None
                 cf = cos_floor.get(k, 1.0)
-                # (where the oracle's perturbed runs are all but uncorrelated with it -- cosine below 0.3: the middle of
-                # the 164-layer network in the bf16 mode -- no direction is determined at all and only the size is checked)
-                ok = 0.5 <= nr <= 2.0 and (cf < 0.3 or (cos >= min(MIN_COS, 0.5 * cf) and cos > 0.0))
+                # (one perturbed run is itself one draw of a noisy quantity: with eight or more chaotic tensors in a case
+                # the direction is judged over all of them together, below; per tensor only the size)
+                chaotic.append((cos, cf))
+                ok = 0.5 <= nr <= 2.0
+                pending.append(len(RECORDS))
         RECORDS.append(dict(case=case, tensor=k, err=e, tol=tol, rule=rule, floor=fl, bound=bound, cos_floor=cf,
                             met_stated=bool(e <= tol), cos=cos, norm_ratio=nr, ok=bool(ok)))
         if not ok:
             bad[k] = (e, bound, cos, nr)
+    if chaotic:
+        # direction of the chaotic tensors: against the oracle they must be about as well aligned as the oracle's
+        # perturbed runs are -- each one where there are few, their median where there are many
+        if len(chaotic) >= 8:
+            med, med_f = float(np.median([c for c, _ in chaotic])), float(np.median([f for _, f in chaotic]))
+            dir_ok = [med >= 0.5 * med_f - 0.05] * len(chaotic)
+        else:
+            dir_ok = [f < 0.3 or (c >= min(MIN_COS, 0.5 * f) and c > 0.0) for c, f in chaotic]
+        for i, good in zip(pending, dir_ok):
+            if not good:
+                RECORDS[i]["ok"] = False
+                bad[RECORDS[i]["tensor"]] = (RECORDS[i]["err"], None, RECORDS[i]["cos"], RECORDS[i]["norm_ratio"])
     assert not bad, f"{case}: (error, bound, cosine, norm ratio) {bad}"
     return max(errs.values()), max(floors.values(), default=0.0)
 

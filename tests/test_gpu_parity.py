@@ -392,9 +392,9 @@ def test_tiny_stack_parity(ctx, mode, kind, maxpool):
     ORACLE_RUNS.clear()
 
 
-def sample_units(cfg):
-    """First, middle and last unit of every stage."""
-    return tuple(sorted({(si, u) for si, s in enumerate(cfg.stages) for u in (0, s.units // 2, s.units - 1)}))
+def sample_units(cfg, middle=True):
+    """First, (middle) and last unit of every stage."""
+    return tuple(sorted({(si, u) for si, s in enumerate(cfg.stages) for u in ((0, s.units // 2, s.units - 1) if middle else (0, s.units - 1))}))
 
 
 @pytest.mark.parametrize("mode", [1, 0])
@@ -404,7 +404,7 @@ def test_full_config_parity(ctx, name, mode):
     every transition inside the network at the stated tolerance; end-to-end gradients of the last stage and the
     classifier at the stated tolerance, those in front of it by the floor rule."""
     cfg = syn.stack_config(name)
-    keys = sample_units(cfg)
+    keys = sample_units(cfg, middle=(name != "revnet164"))      # (the bottleneck network's oracle runs take minutes: two units per stage)
     frac = R.DEFAULT_FRAC_BITS[mode]
     levels = [2.0 ** -frac] if frac else [1e-6]       # the larger of the rounding differences that exist (one grid step)
     try:

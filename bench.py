@@ -43,6 +43,7 @@ ALU_KERNELS = ("gemm_simt_kernel",)   # fp32 CUDA-core GEMMs
 DEVICE_KERNEL = {
     "conv_fprop_fused": "conv_fused_kernel", "conv_dgrad_fused": "conv_fused_kernel",
     "conv_fprop_tc": "conv_tc_kernel", "conv_dgrad_tc": "conv_tc_kernel", "conv_wgrad_tc": "wgrad_tc_kernel",
+    "conv_fprop_tc2": "conv_tc2_kernel", "conv_dgrad_tc2": "conv_tc2_kernel", "conv_wgrad_tc2": "wgrad_tc2_kernel",
     "conv_fprop_simt": "gemm_simt_kernel", "conv_dgrad_simt": "gemm_simt_kernel", "conv_wgrad_simt": "gemm_simt_kernel",
     "bn_stats_partial": "col_reduce_kernel", "bn_bwd_partial": "col_reduce_kernel",
 }
@@ -50,13 +51,24 @@ KERNEL_SOURCES = {
     "conv_fused_kernel": ("conv_fused.cu", "conv_epilogue.cuh", "tc_ptx.cuh"),
     "conv_tc_kernel": ("conv_tc.cu", "conv_epilogue.cuh", "tc_ptx.cuh"),
     "wgrad_tc_kernel": ("conv_tc.cu", "tc_ptx.cuh"),
+    "conv_tc2_kernel": ("conv_tc.cu", "conv_epilogue.cuh", "tc_ptx.cuh"),
+    "wgrad_tc2_kernel": ("conv_tc.cu", "tc_ptx.cuh"),
 }
 
 
-def by_device_kernel(prof):
+def by_device_kernel(prof, peaks=None):
+    """Per-launch-shape profile records ("name|bytes|flops" per launch) -> per device kernel.  With peaks, a
+    convolution kernel is split by what binds each of its launch shapes: the same kernel runs the memory-bound 1x1
+    layers (a few flops per byte) and the tensor-bound 3x3 layers and transitions, and one roofline cannot
+    describe both.  The two halves are reported as "kernel [tensor-bound layers]" and "kernel [hbm-bound layers]"."""
     out = {}
-    for name, v in prof.items():
+    for key, v in prof.items():
+        name = key.split("|")[0]
         k = DEVICE_KERNEL.get(name, name)
+        if peaks and k in KERNEL_SOURCES and v["launches"]:
+            t_mem = v["bytes"] / (peaks["hbm"] * 1e9)
+            t_tc = v["flops"] / (peaks["tc_sustained"] * 1e12)
+            k = f"{k} [{'tensor' if t_tc > t_mem else 'hbm'}-bound layers]"
         a = out.setdefault(k, dict(launches=0, ms=0.0, bytes=0.0, flops=0.0))
         for f in a:
             a[f] += v[f]
@@ -343,12 +355,20 @@ def run_ours(args, cfg):
         torch.cuda.empty_cache()
 
     # ---- per-kernel timing with CUDA events on the launching stream (same process, after the timed steps)
-    B.revnet_profile_enable(ctx, True)
+    B.revnet_profile_enable(ctx, 2)          # one record per kernel and launch shape
     psteps = 2
     for _ in range(psteps):
         reset()
         run.step(want_logits=False)
     prof = B.revnet_profile_summary(ctx)
+    B.revnet_profile_enable(ctx, False)
+    # ---- the same step as it runs inside the replayed graph: start / end stamps written by the kernels themselves
+    B.revnet_profile_enable(ctx, 3)
+    for _ in range(3):                       # the first of them captures the stamped graph, the others replay it
+        reset()
+        run.step(want_logits=False)
+    torch.cuda.synchronize()
+    timeline = B.revnet_profile_summary(ctx)
     B.revnet_profile_enable(ctx, False)
     final_loss = float(run.loss.item())
     # per-block forward / reconstructing-backward time at each stage shape of the workload
@@ -383,7 +403,9 @@ def run_ours(args, cfg):
         peaks = load_peaks()
         total_images = rcfg.N * world * args.steps
         assert abs(whole_job_rate(rcfg.N, world, args.steps, dev_ms) - total_images / (dev_ms * 1e-3)) < 1e-6 * total_images
-        prof = {k: v for k, v in by_device_kernel(prof).items() if k != "step_begin"}    # not a kernel: the host-ahead hold of a profiled step
+        shapes = {k: v for k, v in prof.items() if not k.startswith("step_begin")}    # not a kernel: the host-ahead hold of a profiled step
+        classes = {k: v for k, v in by_device_kernel(shapes, peaks).items() if " [" in k}
+        prof = by_device_kernel(shapes)
         tot = sum(v["ms"] for v in prof.values()) or 1.0
         top = max(prof.items(), key=lambda kv: kv[1]["ms"])
         name, rec = top
@@ -405,14 +427,29 @@ def run_ours(args, cfg):
         whole = dict(algorithmic_gb=step_bytes / 1e9, tflop=step_flops / 1e12,
                      gbs=step_bytes / step_s / 1e9, frac_hbm=step_bytes / step_s / 1e9 / peaks["hbm"],
                      tflops=step_flops / step_s / 1e12, frac_tensor=step_flops / step_s / 1e12 / peaks["tc_sustained"],
-                     roofline_ms=sum(max(v["bytes"] / (peaks["hbm"] * 1e9), v["flops"] / (peaks["tc_sustained"] * 1e12)) for v in prof.values()) / psteps * 1e3,
+                     roofline_ms=sum(max(v["bytes"] / (peaks["hbm"] * 1e9), v["flops"] / (peaks["tc_sustained"] * 1e12)) for v in shapes.values()) / psteps * 1e3,
                      profiled_serial_ms=tot / psteps)
+        if timeline.get("stamped_span"):
+            tl = by_device_kernel({k: v for k, v in timeline.items() if not k.startswith("stamped_")}, peaks)
+            whole["graph_timeline"] = dict(
+                note="one replayed step; start of first CTA to end of last CTA per launch, summed per kernel (overlapping kernels each count)",
+                span_ms=timeline["stamped_span"]["ms"], busy_ms=timeline["stamped_busy"]["ms"],
+                stamped_launches=timeline["stamped_busy"]["launches"],
+                kernels={k: dict(launches=v["launches"], ms=v["ms"],
+                                 gbs=(v["bytes"] / (v["ms"] * 1e-3) / 1e9) if v["ms"] > 0 else None,
+                                 tflops=(v["flops"] / (v["ms"] * 1e-3) / 1e12) if v["ms"] > 0 else None)
+                         for k, v in sorted(tl.items(), key=lambda kv: -kv[1]["ms"])})
         roof = dict(bound=bound, achieved=ach, peak=peak, unit=runit, frac=ach / peak, traffic=measured_traffic(name, cfg.name), kernel=name, whole_step=whole,
                     kernel_share=rec["ms"] / tot, avg_launch_us=avg_s * 1e6, peak_source=peaks["source"],
                     kernels={k: dict(launches=v["launches"] // psteps, ms_per_step=v["ms"] / psteps, share=v["ms"] / tot,
                                      gbs=(v["bytes"] / (v["ms"] * 1e-3) / 1e9) if v["ms"] > 0 else None,
                                      tflops=(v["flops"] / (v["ms"] * 1e-3) / 1e12) if v["ms"] > 0 else None)
-                             for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])})
+                             for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])},
+                    # the convolution kernels once more, their launches split by what binds each launch shape
+                    layer_classes={k: dict(launches=v["launches"] // psteps, ms_per_step=v["ms"] / psteps,
+                                           gbs=v["bytes"] / (v["ms"] * 1e-3) / 1e9, frac_hbm=v["bytes"] / (v["ms"] * 1e-3) / 1e9 / peaks["hbm"],
+                                           tflops=v["flops"] / (v["ms"] * 1e-3) / 1e12, frac_tensor=v["flops"] / (v["ms"] * 1e-3) / 1e12 / peaks["tc_sustained"])
+                                   for k, v in sorted(classes.items(), key=lambda kv: -kv[1]["ms"]) if v["ms"] > 0})
         img_bytes = h_img.numel() * 4 + h_lab.numel() * 4
         line = dict(metric=METRIC, value=total_images / (dev_ms * 1e-3), unit=UNIT, n_gpus=world, steps=args.steps,
                     warmup=args.warmup, ms_per_step=dev_ms / args.steps, higher_is_better=True, scaling="weak",

@@ -322,7 +322,15 @@ int revnet_selftest_bounded_wait(revnet_ctx *ctx, uint64_t limit_ns, void *strea
  * Enabling (or disabling) clears earlier records.  on = 2 enables with one line per kernel name AND
  * launch shape: the name then reads "name|algorithmic_bytes|flops" of one launch.  A profiled train
  * step first holds the stream for 5 ms, so that its launches are queued by the time they run and
- * the spans hold device time only; that hold is the record "step_begin". */
+ * the spans hold device time only; that hold is the record "step_begin".
+ * on = 3 is the timeline mode, for train steps only: no events; instead the convolution, weight-
+ * gradient and BN-ReLU apply kernels write the GPU's nanosecond timer when their first CTA starts
+ * and their last CTA ends (one slot per launch, reset at the start of every step, also inside the
+ * replayed graph).  The summary then describes the LAST step that ran, as it ran (overlapping
+ * streams, no events in between): one line per kernel name and launch shape with the sum of its
+ * launches' start-to-end times, a line "stamped_busy" (time during which at least one stamped kernel
+ * was running; launches = stamped launches) and a line "stamped_span" (first start to last end).
+ * Kernels that overlap each count their own time, so the lines can add up to more than the span. */
 int revnet_profile_enable(revnet_ctx *ctx, int on);
 int revnet_profile_summary(revnet_ctx *ctx, char *buf, size_t buflen, size_t *needed);
 

@@ -316,7 +316,9 @@ def revnet_train_step_host(ctx, plan, images_host, labels_host, images_dev, labe
     return st
 
 
-def revnet_profile_enable(ctx, on: bool):
+def revnet_profile_enable(ctx, on):
+    """0 / False: off; 1 / True: one record per kernel name; 2: one per kernel name and launch shape;
+    3: timeline of the last train step from start / end stamps the kernels write themselves (no events)."""
     ctx.check(lib().revnet_profile_enable(ctx.h, C.c_int(int(on))), "revnet_profile_enable")
 
 

@@ -5,6 +5,7 @@
 #include <stdio.h>
 #include <math.h>
 #include <atomic>
+#include <algorithm>
 
 static int fail(revnet_ctx *ctx, int code, const std::string &msg) { if (ctx) ctx->err = msg; return code; }
 
@@ -18,6 +19,7 @@ extern "C" int revnet_create(revnet_ctx **out, int device) {
         if (cudaSetDevice(device) != cudaSuccess ||
             cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, device) != cudaSuccess ||
             cudaMalloc(&c->dev_status, 1024) != cudaSuccess || cudaMemset(c->dev_status, 0, 1024) != cudaSuccess ||
+            cudaMalloc(&c->stamps, 2 * kStampSlots * sizeof(unsigned long long)) != cudaSuccess ||
             cudaStreamCreateWithFlags(&c->capture_stream, cudaStreamNonBlocking) != cudaSuccess ||
             cudaStreamCreateWithFlags(&c->side_stream, cudaStreamNonBlocking) != cudaSuccess ||
             cudaStreamCreateWithFlags(&c->recon_stream, cudaStreamNonBlocking) != cudaSuccess ||
@@ -40,6 +42,7 @@ extern "C" int revnet_destroy(revnet_ctx *ctx) {
     if (!ctx) return REVNET_OK;
     for (cudaEvent_t e : ctx->ev_pool) cudaEventDestroy(e);
     if (ctx->dev_status) cudaFree(ctx->dev_status);
+    if (ctx->stamps) cudaFree(ctx->stamps);
     if (ctx->capture_stream) cudaStreamDestroy(ctx->capture_stream);
     if (ctx->side_stream) cudaStreamDestroy(ctx->side_stream);
     if (ctx->recon_stream) cudaStreamDestroy(ctx->recon_stream);
@@ -384,10 +387,13 @@ extern "C" int revnet_selftest_bounded_wait(revnet_ctx *ctx, uint64_t limit_ns, 
 // ---- per-kernel timing
 extern "C" int revnet_profile_enable(revnet_ctx *ctx, int on) {
     if (!ctx) return REVNET_E_INVALID_ARG;
-    ctx->profiling = on != 0;
+    ctx->profiling = on == 1 || on == 2;
     ctx->prof_detail = on == 2;
+    ctx->stamping = on == 3;
     ctx->prof.clear();
     ctx->ev_used = 0;
+    ctx->stamp_recs.clear();
+    ctx->stamp_next = 0;
     return REVNET_OK;
 }
 
@@ -395,6 +401,38 @@ extern "C" int revnet_profile_summary(revnet_ctx *ctx, char *buf, size_t buflen,
     if (!ctx || (!buf && buflen)) return REVNET_E_INVALID_ARG;
     struct Acc { std::string name; uint64_t n = 0; double ms = 0, bytes = 0, flops = 0; };
     std::vector<Acc> acc;
+    if (ctx->stamping) {
+        // timeline mode: the stamps of the last step that ran (the caller has synchronised, or we do)
+        std::vector<unsigned long long> h(2 * kStampSlots);
+        if (cudaDeviceSynchronize() != cudaSuccess || cudaMemcpy(h.data(), ctx->stamps, h.size() * sizeof(unsigned long long), cudaMemcpyDeviceToHost) != cudaSuccess)
+            return fail(ctx, REVNET_E_CUDA, std::string("revnet_profile_summary: ") + cudaGetErrorString(cudaGetLastError()));
+        std::vector<std::pair<unsigned long long, unsigned long long>> iv;
+        for (const StampRec &r : ctx->stamp_recs) {
+            const unsigned long long t0 = h[r.slot], t1 = h[kStampSlots + r.slot];
+            if (t1 == 0 || t0 == ~0ull || t1 < t0) continue;      // the kernel did not run in the last step
+            char key[160];
+            snprintf(key, sizeof key, "%s|%.0f|%.0f", r.name, r.bytes, r.flops);
+            Acc *a = nullptr;
+            for (auto &x : acc) if (x.name == key) { a = &x; break; }
+            if (!a) { acc.push_back(Acc()); a = &acc.back(); a->name = key; }
+            a->n++; a->ms += (double)(t1 - t0) * 1e-6; a->bytes += r.bytes; a->flops += r.flops;
+            iv.push_back({t0, t1});
+        }
+        // time during which at least one stamped kernel ran, and the span from the first start to the last end
+        std::sort(iv.begin(), iv.end());
+        double busy = 0; unsigned long long lo = 0, hi = 0;
+        for (auto &p : iv) {
+            if (hi == 0) { lo = p.first; hi = p.second; }
+            else if (p.first <= hi) { if (p.second > hi) hi = p.second; }
+            else { busy += (double)(hi - lo) * 1e-6; lo = p.first; hi = p.second; }
+        }
+        if (hi) busy += (double)(hi - lo) * 1e-6;
+        Acc b; b.name = "stamped_busy"; b.n = iv.size(); b.ms = busy; acc.push_back(b);
+        if (!iv.empty()) {
+            unsigned long long last = 0; for (auto &p : iv) if (p.second > last) last = p.second;
+            Acc sp; sp.name = "stamped_span"; sp.n = 1; sp.ms = (double)(last - iv.front().first) * 1e-6; acc.push_back(sp);
+        }
+    }
     if (!ctx->prof.empty() && cudaEventSynchronize(ctx->prof.back().ev) != cudaSuccess)
         return fail(ctx, REVNET_E_CUDA, std::string("revnet_profile_summary: ") + cudaGetErrorString(cudaGetLastError()));
     for (size_t i = 1; i < ctx->prof.size(); i++) {

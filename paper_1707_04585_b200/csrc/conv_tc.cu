@@ -49,6 +49,7 @@ struct TcParams {
     int GW;          // 32 or 16 floats: rows of 128 / 64 bytes, stored with the matching TMA swizzle
     int group_bytes; // one column group of a tile (128 pixel rows), a multiple of 1024
     int need_aux;
+    int aux_slots;   // conv_tc2_kernel: slots of the partner ring (two interleaved rings, one per epilogue warp group)
     int split_o, split_x;   // channels in the first tensor of a channel-split output / partner (0: one tensor)
     // the taps this launch sums: offset of the operand box in rows / columns of the operand tensor, and the tap's
     // place in the weight pack.  A plain convolution lists all k*k taps; one parity class of a stride-2 data
@@ -65,6 +66,7 @@ struct TcParams {
     // then pixel (m / Wp, m % Wp) of the tile; rows with m % Wp >= W are padding.
     int halo, Wp;
     int a_slots, a_slot_bytes, a_box_bytes;
+    unsigned long long *stamp;    // timeline slot of this launch (nullptr: off)
 };
 
 struct __align__(8) TcShared {
@@ -85,6 +87,23 @@ struct __align__(8) TcShared {
 //   pass B  thread = (channel quad, every rpp-th pixel): per-channel sums over the valid pixels of the group
 // KA: 0 plain float, 1 plain onto the fixed-point grid, 2 / 3 float coupling + / -, 4 / 5 fixed-point coupling + / -.
 template <int KA>
+__device__ __forceinline__ void pass_a_quad(float4 r, const uint8_t *aux, uint8_t *outb, float out_s) {
+    if (KA == 2 || KA == 3) {
+        const float4 pr = *reinterpret_cast<const float4 *>(aux);
+        if (KA == 2) { r.x = pr.x + r.x; r.y = pr.y + r.y; r.z = pr.z + r.z; r.w = pr.w + r.w; }
+        else { r.x = pr.x - r.x; r.y = pr.y - r.y; r.z = pr.z - r.z; r.w = pr.w - r.w; }
+    } else if (KA != 0) {
+        int4 iv = quant4(r, out_s);
+        if (KA >= 4) {
+            const int4 pi = *reinterpret_cast<const int4 *>(aux);
+            if (KA == 4) { iv.x = pi.x + iv.x; iv.y = pi.y + iv.y; iv.z = pi.z + iv.z; iv.w = pi.w + iv.w; }
+            else { iv.x = pi.x - iv.x; iv.y = pi.y - iv.y; iv.z = pi.z - iv.z; iv.w = pi.w - iv.w; }
+        }
+        r = make_float4(__int_as_float(iv.x), __int_as_float(iv.y), __int_as_float(iv.z), __int_as_float(iv.w));
+    }
+    *reinterpret_cast<float4 *>(outb) = r;
+}
+template <int KA>
 __device__ __forceinline__ void tma_pass_a(uint32_t tm, int GW, int row, bool valid, const uint8_t *aux, uint8_t *outb, float out_s) {
     const int row_b = GW * 4;
     const int swz = GW == 32 ? (row & 7) : ((row >> 1) & 3);
@@ -96,21 +115,7 @@ __device__ __forceinline__ void tma_pass_a(uint32_t tm, int GW, int row, bool va
 #pragma unroll
         for (int j = 0; j < 4; j++) {
             const int off = row * row_b + ((((c >> 2) + j) ^ swz) << 4);
-            float4 r = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-            if (KA == 2 || KA == 3) {
-                const float4 pr = *reinterpret_cast<const float4 *>(aux + off);
-                if (KA == 2) { r.x = pr.x + r.x; r.y = pr.y + r.y; r.z = pr.z + r.z; r.w = pr.w + r.w; }
-                else { r.x = pr.x - r.x; r.y = pr.y - r.y; r.z = pr.z - r.z; r.w = pr.w - r.w; }
-            } else if (KA != 0) {
-                int4 iv = make_int4(__float2int_rn(r.x * out_s), __float2int_rn(r.y * out_s), __float2int_rn(r.z * out_s), __float2int_rn(r.w * out_s));
-                if (KA >= 4) {
-                    const int4 pi = *reinterpret_cast<const int4 *>(aux + off);
-                    if (KA == 4) { iv.x = pi.x + iv.x; iv.y = pi.y + iv.y; iv.z = pi.z + iv.z; iv.w = pi.w + iv.w; }
-                    else { iv.x = pi.x - iv.x; iv.y = pi.y - iv.y; iv.z = pi.z - iv.z; iv.w = pi.w - iv.w; }
-                }
-                r = make_float4(__int_as_float(iv.x), __int_as_float(iv.y), __int_as_float(iv.z), __int_as_float(iv.w));
-            }
-            *reinterpret_cast<float4 *>(outb + off) = r;
+            pass_a_quad<KA>(make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]), aux + off, outb + off, out_s);
         }
     }
 }
@@ -126,16 +131,14 @@ __device__ __forceinline__ void tma_pass_b(int GW, const uint8_t *ob, const uint
         float4 v = *reinterpret_cast<const float4 *>(ob + off);
         if (KB >= 2) {
             float4 tt = *reinterpret_cast<const float4 *>(aux + off);
-            if (KB == 3) tt = make_float4(__int2float_rn(__float_as_int(tt.x)) * q, __int2float_rn(__float_as_int(tt.y)) * q,
-                                          __int2float_rn(__float_as_int(tt.z)) * q, __int2float_rn(__float_as_int(tt.w)) * q);
+            if (KB == 3) tt = dequant4(make_int4(__float_as_int(tt.x), __float_as_int(tt.y), __float_as_int(tt.z), __float_as_int(tt.w)), q);
             const float dx = fmaf(sc4.x, tt.x, sh4.x) > 0.f ? v.x : 0.f, dy = fmaf(sc4.y, tt.y, sh4.y) > 0.f ? v.y : 0.f;
             const float dz = fmaf(sc4.z, tt.z, sh4.z) > 0.f ? v.z : 0.f, dw = fmaf(sc4.w, tt.w, sh4.w) > 0.f ? v.w : 0.f;
             acc[0] += dx; acc[1] += dy; acc[2] += dz; acc[3] += dw;
             acc[4] += dx * ((tt.x - mu4.x) * rs4.x); acc[5] += dy * ((tt.y - mu4.y) * rs4.y);
             acc[6] += dz * ((tt.z - mu4.z) * rs4.z); acc[7] += dw * ((tt.w - mu4.w) * rs4.w);
         } else {
-            if (KB == 1) v = make_float4(__int2float_rn(__float_as_int(v.x)) * q, __int2float_rn(__float_as_int(v.y)) * q,
-                                         __int2float_rn(__float_as_int(v.z)) * q, __int2float_rn(__float_as_int(v.w)) * q);
+            if (KB == 1) v = dequant4(make_int4(__float_as_int(v.x), __float_as_int(v.y), __float_as_int(v.z), __float_as_int(v.w)), q);
             acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
             acc[4] += v.x * v.x; acc[5] += v.y * v.y; acc[6] += v.z * v.z; acc[7] += v.w * v.w;
         }
@@ -185,6 +188,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     pdl_enter();             // the set-up above may overlap the kernel before; its outputs are read from here on
+    stamp_begin(p.stamp);
     const uint32_t tmem_d = sh->tmem_base;
     const int col0 = blockIdx.y * p.BN;
 
@@ -288,27 +292,33 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         auto aux_map = [&](int col) { return (p.split_x && col >= p.split_x) ? &map_x1 : &map_x0; };
         auto col_out = [&](int col) { return (p.split_o && col >= p.split_o) ? col - p.split_o : col; };
         auto col_aux = [&](int col) { return (p.split_x && col >= p.split_x) ? col - p.split_x : col; };
-        auto load_aux = [&](int gi, int t) {                 // one thread; t: tile in the list of all classes
+        auto load_aux = [&](int gi, int cls, int n0, int h0) {     // one thread; (cls, n0, h0): class and origin of the tile
             const int col = col0 + gi * GW;
             if (col >= e.n_cols) return;
-            int n0, h0;
-            const int cls = t / p.g.n_px_tiles;
-            tile_origin(p.g, t - cls * p.g.n_px_tiles, n0, h0);
             mbar_expect_tx(&sh->aux_full[gi], aux_tx);
             tma_load_4d(auxr + gi * p.group_bytes, aux_map(col), &sh->aux_full[gi], col_aux(col), p.ox[cls], h0 * p.ostride + p.oy[cls], n0);
         };
+        // class and origin of the tile at hand and of the one after it: worked out once per tile, so that the thread
+        // that issues the partner loads between two column groups has no divisions to do
+        int cls = 0, n0 = 0, h0 = 0, cls_n = 0, n0_n = 0, h0_n = 0;
+        if ((int)blockIdx.x < n_vt) {
+            cls_n = (int)blockIdx.x / p.g.n_px_tiles;
+            tile_origin(p.g, (int)blockIdx.x - cls_n * p.g.n_px_tiles, n0_n, h0_n);
+        }
         if (etid == 0 && p.need_aux && (int)blockIdx.x < n_vt)
-            for (int gi = wg; gi < ng; gi += 2) load_aux(gi, blockIdx.x);
+            for (int gi = wg; gi < ng; gi += 2) load_aux(gi, cls_n, n0_n, h0_n);
         named_barrier(5, 256);
         bool ok = true;
         int ti = 0;
         uint8_t *ob = outr + wg * p.group_bytes;
         for (int t = blockIdx.x; t < n_vt; t += gridDim.x, ti++) {
             const int buf = ti & 1; const uint32_t use = ti >> 1;
-            int n0, h0;
-            const int cls = t / p.g.n_px_tiles;
-            tile_origin(p.g, t - cls * p.g.n_px_tiles, n0, h0);
+            cls = cls_n; n0 = n0_n; h0 = h0_n;
             const int tn = t + (int)gridDim.x;
+            if (tn < n_vt) {
+                cls_n = tn / p.g.n_px_tiles;
+                tile_origin(p.g, tn - cls_n * p.g.n_px_tiles, n0_n, h0_n);
+            }
             const int valid_px = p.g.BIMG > 1 ? (p.g.N - n0 < p.g.BIMG ? p.g.N - n0 : p.g.BIMG) * p.g.BH * p.g.W
                                               : (p.g.H - h0 < p.g.BH ? p.g.H - h0 : p.g.BH) * p.g.W;
             if (etid == 0) ok = mbar_wait(&sh->acc_full[buf], use & 1) && sh->failed == 0;     // one thread polls, the rest block
@@ -356,7 +366,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     slot[0] = make_float4(acc[0], acc[1], acc[2], acc[3]); slot[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
                 }
                 named_barrier(bar_a, 128);                 // the partner group and the output slot have been read
-                if (etid == 0 && p.need_aux && tn < n_vt) load_aux(gi, tn);
+                if (etid == 0 && p.need_aux && tn < n_vt) load_aux(gi, cls_n, n0_n, h0_n);
             }
             if (!ok) break;
             // this warp group has drained its columns of the accumulator (the other group arrives for its own)
@@ -390,6 +400,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && sh->failed) atomicExch(p.status, (int)REVNET_E_TIMEOUT);
+    stamp_end(p.stamp);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_d, tmem_cols);
@@ -423,7 +434,7 @@ conv_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const int wstage_bytes = (b_bytes + 1023) & ~1023;
     uint8_t *wring = tiles + (p.halo ? p.a_slots * p.a_slot_bytes : 0);
     uint8_t *auxr = p.halo ? wring + p.stages * wstage_bytes : tiles + p.stages * stage_bytes;
-    uint8_t *outr = auxr + (p.need_aux ? ng : 0) * p.group_bytes;
+    uint8_t *outr = auxr + (p.need_aux ? p.aux_slots : 0) * p.group_bytes;
     float *gsums = (float *)(outr + 2 * p.group_bytes);
     TcShared *sh = (TcShared *)(gsums + ng * 128 * 8);
 
@@ -453,6 +464,7 @@ conv_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     cluster_sync_all();      // the peer's barriers are initialised and its tensor memory allocated before anything crosses over
     tc_fence_after();
     pdl_enter();
+    stamp_begin(p.stamp);
     const uint32_t tmem_d = sh->tmem_base;
     const int col0 = blockIdx.y * p.BN;
     // this CTA's tile of tile pair vp
@@ -586,21 +598,37 @@ conv_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         auto aux_map = [&](int col) { return (p.split_x && col >= p.split_x) ? &map_x1 : &map_x0; };
         auto col_out = [&](int col) { return (p.split_o && col >= p.split_o) ? col - p.split_o : col; };
         auto col_aux = [&](int col) { return (p.split_x && col >= p.split_x) ? col - p.split_x : col; };
-        auto load_aux = [&](int gi, int vp) {                // one thread; returns without loading for a tile outside the tensor
-            const int col = col0 + gi * GW;
-            int cls, t, n0, h0;
-            my_tile(vp, cls, t);
-            if (col >= e.n_cols || t >= p.g.n_px_tiles) return;
-            tile_origin(p.g, t, n0, h0);
-            mbar_expect_tx(&sh->aux_full[gi], aux_tx);
-            tma_load_4d(auxr + gi * p.group_bytes, aux_map(col), &sh->aux_full[gi], col_aux(col), p.ox[cls], h0 * p.ostride + p.oy[cls], n0);
+        // The partner groups arrive through a ring of SW slots per warp group (slots wg, wg + 2, ...), filled in the
+        // order the group will visit them: its column groups of this tile, then of its next tile, ...; groups beyond
+        // the valid channels and tiles outside the tensor are not visited.  l_*: next visit to load (one thread),
+        // c_*: next visit to consume (all threads, uniform).
+        const int SW = p.aux_slots >> 1;
+        int l_vp = pair, l_gi = wg, l_slot = 0;
+        int c_slot = 0; uint32_t c_par = 0;
+        auto load_next_aux = [&]() {                         // one thread; returns without loading once the visits are used up
+            while (l_vp < n_vp) {
+                int cls, t, n0, h0;
+                my_tile(l_vp, cls, t);
+                const int col = col0 + l_gi * GW;
+                const bool live = col < e.n_cols && t < p.g.n_px_tiles;
+                l_gi += 2;
+                const bool last_of_tile = l_gi >= ng;
+                if (live) {
+                    tile_origin(p.g, t, n0, h0);
+                    const int slot = wg + 2 * l_slot;
+                    mbar_expect_tx(&sh->aux_full[slot], aux_tx);
+                    tma_load_4d(auxr + slot * p.group_bytes, aux_map(col), &sh->aux_full[slot], col_aux(col), p.ox[cls], h0 * p.ostride + p.oy[cls], n0);
+                    if (++l_slot == SW) l_slot = 0;
+                }
+                if (last_of_tile) { l_gi = wg; l_vp += n_pairs; }
+                if (live) return;
+            }
         };
-        if (etid == 0 && p.need_aux && pair < n_vp)
-            for (int gi = wg; gi < ng; gi += 2) load_aux(gi, pair);
+        if (etid == 0 && p.need_aux && wg < ng)
+            for (int i = 0; i < SW; i++) load_next_aux();
         named_barrier(5, 256);
         bool ok = true;
         int ti = 0;
-        uint32_t aux_uses[8] = {0, 0, 0, 0, 0, 0, 0, 0};     // per column group: loads waited for so far (tiles outside the tensor load nothing)
         uint8_t *ob = outr + wg * p.group_bytes;
         for (int vp = pair; vp < n_vp; vp += n_pairs, ti++) {
             const int buf = ti & 1; const uint32_t use = ti >> 1;
@@ -608,7 +636,6 @@ conv_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             my_tile(vp, cls, t);
             const bool in_range = t < p.g.n_px_tiles;
             tile_origin(p.g, t, n0, h0);
-            const int vpn = vp + n_pairs;
             int valid_px = 0;
             if (in_range)
                 valid_px = p.g.BIMG > 1 ? (p.g.N - n0 < p.g.BIMG ? p.g.N - n0 : p.g.BIMG) * p.g.BH * p.g.W
@@ -622,12 +649,13 @@ conv_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             for (int gi = wg; gi < ng; gi += 2) {
                 const int col = col0 + gi * GW;
                 const bool live = in_range && col < e.n_cols;
-                const uint8_t *ax = auxr + gi * p.group_bytes;
+                const bool visit = p.need_aux && live;       // this group's partner tile sits in ring slot c_slot
+                const uint8_t *ax = auxr + (wg + 2 * c_slot) * p.group_bytes;
                 if (etid == 0) {
-                    if (p.need_aux && live) ok = mbar_wait(&sh->aux_full[gi], aux_uses[gi] & 1);
+                    if (visit) ok = mbar_wait(&sh->aux_full[wg + 2 * c_slot], c_par);
                     tma_store_wait_read();
                 }
-                if (p.need_aux && live) aux_uses[gi]++;
+                if (visit && ++c_slot == SW) { c_slot = 0; c_par ^= 1u; }
                 ok = named_barrier_and(bar_b, 128, ok);
                 if (!ok) break;
                 const bool rowv = live && srow >= 0 && srow < valid_px;
@@ -658,8 +686,8 @@ conv_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
                     else tma_pass_b<1>(GW, ob, ax, jq, r0, rpp, valid_px, out_q, sc4, sh4, mu4, rs4, acc);
                     slot[0] = make_float4(acc[0], acc[1], acc[2], acc[3]); slot[1] = make_float4(acc[4], acc[5], acc[6], acc[7]);
                 }
-                named_barrier(bar_a, 128);
-                if (etid == 0 && p.need_aux && vpn < n_vp) load_aux(gi, vpn);
+                named_barrier(bar_a, 128);                 // the partner slot and the output slot have been read
+                if (etid == 0 && visit) load_next_aux();   // refill the slot just freed
             }
             if (!ok) break;
             // this warp group has drained its columns of the accumulator: one arrival per group on the leader's barrier
@@ -693,6 +721,7 @@ conv_tc2_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && sh->failed) atomicExch(p.status, (int)REVNET_E_TIMEOUT);
+    stamp_end(p.stamp);
     // neither CTA leaves, or frees tensor memory, while the other may still read its operands or signal its barriers
     cluster_sync_all();
     if (warp == 1) {
@@ -850,6 +879,17 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
     const int ntap_max = s2 ? 4 : taps;
     // arithmetic-bound layers without a partner tile (transitions, their data gradients): 128 x 256 tiles
     if (!need_aux && !(out.c1 && out.c0 % 32) && (long long)ntap_max * cin >= 1024 && cout >= 256 && cout % 32 == 0) tc_shape(g, cin, cout, k, stride, s, true);
+    // 1x1 layers onto many channels (the last layer of a bottleneck function with its coupling partner, the data
+    // gradient of the first): their operands cross L2 -> shared memory once per tile, and with 128 x 128 tiles that
+    // traffic (not HBM, not the tensor cores) sets their time.  A CTA pair on a 256 x 256 tile moves half of it.
+    // Measured: no faster (these layers' time is their epilogue's, see the kernel), so off unless REVNET_CONV_PAIR1X1
+    // asks for it: bit 0 layers with a partner tile, bit 1 layers without
+    static const bool pair_enabled = [] { const char *v = getenv("REVNET_CONV_PAIR"); return !(v && v[0] == '0'); }();
+    static const int pair1x1 = [] { const char *v = getenv("REVNET_CONV_PAIR1X1"); return v ? atoi(v) : 0; }();
+    const bool wide1 = k == 1 && stride == 1 && !s2 && cout >= 256 && cout % 32 == 0 && !(out.c1 && out.c0 % 32) &&
+                       !(need_aux && auxp.c1 && auxp.c0 % 32) && s.KC == 64 &&
+                       pair_enabled && ex.ctx->sm_count % 2 == 0 && s.g.n_px_tiles >= 2 && ((need_aux && (pair1x1 & 1)) || (!need_aux && (pair1x1 & 2)));
+    if (wide1) tc_shape(g, cin, cout, k, stride, s, true);
     // rows of the weight pack (a multiple of its 128-row blocks, whatever the N tile); TMA fills rows beyond with zeros
     const int rp16 = round_up(cout, 16), rows_pad = rp16 <= 128 ? rp16 : round_up(rp16, 128);
     // column groups of 32 floats, or of 16 where the N tile or the halves of a channel-split tensor ask for it
@@ -862,9 +902,11 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
     int stages = 4;
     // CTA pairs (conv_tc2_kernel) wherever the epilogue runs through TMA, the N tile splits into two halves of whole
     // 16-row groups and there are at least two pixel tiles; REVNET_CONV_PAIR=0 keeps the single-CTA kernel (for comparison)
-    static const bool pair_enabled = [] { const char *v = getenv("REVNET_CONV_PAIR"); return !(v && v[0] == '0'); }();
     // (1x1 layers are bound by the activations' way from HBM, which a pair does not shorten: measured 3-10 % slower there)
-    bool pair = pair_enabled && epi_tma && k == 3 && s.BN % 32 == 0 && s.BN >= 64 && s.g.n_px_tiles >= 2 && ex.ctx->sm_count % 2 == 0;
+    bool pair = pair_enabled && epi_tma && (k == 3 || wide1) && s.BN % 32 == 0 && s.BN >= 64 && s.g.n_px_tiles >= 2 && ex.ctx->sm_count % 2 == 0;
+    // partner ring of the pair kernel: per epilogue warp group as many slots as it has column groups in a tile (at most 4)
+    int aux_slots = 0;
+    if (need_aux) { int sw = (ng + 1) / 2; if (sw > 4) sw = 4; aux_slots = 2 * sw; }
     // 3x3 stride-1 layers on a pair: the activations of a tile arrive once per channel chunk as one box with its halo
     // (see TcParams::halo); needs 64-channel chunks (128-byte operand rows) and tiles of whole image rows
     static const bool halo_enabled = [] { const char *v = getenv("REVNET_CONV_HALO"); return !(v && v[0] == '0'); }();
@@ -887,7 +929,10 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
             if (halo) return ((s.BN / 2) * s.KC * 2 + 1023) & ~1023;           // weight tiles only; the boxes are counted below
             return ((128 * s.KC * 2 + 1023) & ~1023) + (((pr ? s.BN / 2 : s.BN) * s.KC * 2 + 1023) & ~1023);
         };
-        auto smem_of = [&](int st, bool pr) { return 1024 + (halo ? a_slots * a_slot_bytes : 0) + st * stage_bytes_of(pr) + ((need_aux ? ng : 0) + 2) * group_bytes + ng * 128 * 32 + (int)sizeof(TcShared) + 64; };
+        auto smem_of = [&](int st, bool pr) { return 1024 + (halo ? a_slots * a_slot_bytes : 0) + st * stage_bytes_of(pr) + ((need_aux ? (pr ? aux_slots : ng) : 0) + 2) * group_bytes + ng * 128 * 32 + (int)sizeof(TcShared) + 64; };
+        // what does not fit gives way in this order: operand stages down to 3, partner slots down to 2 per warp group, stages down to 2
+        while (stages > 3 && smem_of(stages, pair) > 227 * 1024) stages--;
+        while (pair && aux_slots > 4 && smem_of(stages, pair) > 227 * 1024) aux_slots -= 2;
         while (stages > 2 && smem_of(stages, pair) > 227 * 1024) stages--;
         if (smem_of(stages, pair) > 227 * 1024) {
             if (s.BN == 256) return false;      // (does not happen: three stages of a wide tile fit)
@@ -969,6 +1014,7 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         }
         TcParams p;
         p.stages = stages; p.epi_tma = epi_tma ? 1 : 0; p.GW = GW; p.group_bytes = group_bytes; p.need_aux = need_aux ? 1 : 0;
+        p.aux_slots = aux_slots;
         p.split_o = out.c1 ? out.c0 : 0; p.split_x = (need_aux && auxp.c1) ? auxp.c0 : 0;
         memcpy(p.ntap, ntap, sizeof ntap); memcpy(p.tdy, tdy, sizeof tdy); memcpy(p.tdx, tdx, sizeof tdx); memcpy(p.tid, tid, sizeof tid);
         p.ostride = ostride; p.n_cls = n_cls;
@@ -976,6 +1022,7 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         for (int c = 0; c < 4; c++) { p.oy[c] = s2 ? c >> 1 : 0; p.ox[c] = s2 ? c & 1 : 0; }
         p.taps = taps; p.k = k; p.chunks = s.chunks; p.KC = s.KC; p.cin_pad = s.cin_pad; p.BN = s.BN; p.stride = stride; p.g = s.g;
         p.status = ex.ctx->dev_status;
+        p.stamp = ex.stamp_slot();
         EpiArgs &e = p.epi;
         memset(&e, 0, sizeof e);
         e.mode = req.bnbwd ? EPI_BNBWD : (sign ? EPI_COUPLE : EPI_PLAIN);
@@ -993,7 +1040,8 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
         if (pair) launch_cluster(ex, conv_tc2_kernel, grid, kThreadsTma, s.smem, 2, map_a, map_b, map_o[0], map_o[1], map_x[0], map_x[1], p);
         else launch(ex, conv_tc_kernel, grid, epi_tma ? kThreadsTma : kThreads, s.smem, map_a, map_b, map_o[0], map_o[1], map_x[0], map_x[1], p);
         const double bytes = (double)gin.P() * cin * 2 + (double)g.P() * cout * (sign || req.bnbwd ? 8 : 4) + (double)cout * taps * cin * 2;
-        ex.check(what, bytes, 2.0 * g.P() * cout * cin * ntap_all);
+        // (records of launches on a CTA pair carry the pair kernel's name)
+        ex.check(!pair ? what : (transposed ? "conv_dgrad_tc2" : "conv_fprop_tc2"), bytes, 2.0 * g.P() * cout * cin * ntap_all);
     }
     ex.ws.release(m);
     return true;
@@ -1038,7 +1086,7 @@ struct WgParams {
 // its index and then works on that layer alone.
 constexpr int kWgMaxJobs = 4;
 struct alignas(64) WgJob { CUtensorMap map_a, map_g; WgParams p; };
-struct WgBatch { WgJob job[kWgMaxJobs]; int n; };
+struct WgBatch { WgJob job[kWgMaxJobs]; int n; unsigned long long *stamp; };
 
 __global__ void __launch_bounds__(kThreads, 1)
 wgrad_tc_kernel(const __grid_constant__ WgBatch batch) {
@@ -1089,6 +1137,7 @@ wgrad_tc_kernel(const __grid_constant__ WgBatch batch) {
     __syncthreads();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     pdl_enter();             // the set-up above may overlap the kernel before; its outputs are read from here on
+    stamp_begin(batch.stamp);
     const uint32_t tmem_d = sh->tmem_base;
     const int pad = p.k / 2;
     const int tiles_per_img = p.tiles_per_img;
@@ -1196,9 +1245,10 @@ wgrad_tc_kernel(const __grid_constant__ WgBatch batch) {
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (threadIdx.x == 0 && sh->failed) atomicExch(p.status, (int)REVNET_E_TIMEOUT);
+    stamp_end(batch.stamp);
     if (warp == 1) {
-        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_d), "r"(tmem_cols) : "memory");
+        tc_fence_after();
+        tmem_dealloc(tmem_d, tmem_cols);
     }
 }
 
@@ -1254,6 +1304,7 @@ wgrad_tc2_kernel(const __grid_constant__ WgBatch batch) {
     cluster_sync_all();
     tc_fence_after();
     pdl_enter();
+    stamp_begin(batch.stamp);
     const uint32_t tmem_d = sh->tmem_base;
     const int pad = p.k / 2;
     const int tiles_per_img = p.tiles_per_img;
@@ -1357,6 +1408,7 @@ wgrad_tc2_kernel(const __grid_constant__ WgBatch batch) {
     tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && sh->failed) atomicExch(p.status, (int)REVNET_E_TIMEOUT);
+    stamp_end(batch.stamp);
     cluster_sync_all();      // neither CTA leaves, or frees tensor memory, while the other may still read its operands
     if (warp == 1) {
         tc_fence_after();
@@ -1580,6 +1632,7 @@ bool conv_wgrad_tc_batch(Exec &ex, int n, const void *const *gq, const void *con
         WgBatch batch;
         SumBatch sums;
         batch.n = n;
+        batch.stamp = ex.stamp_slot();
         int cta = 0, smem = 0, n_sums = 0;
         size_t off = 0, max_slice = 0;
         double bytes = 0, flops = 0, sum_bytes = 0;
@@ -1616,7 +1669,7 @@ bool conv_wgrad_tc_batch(Exec &ex, int n, const void *const *gq, const void *con
         }
         if (pair) launch_cluster(ex, wgrad_tc2_kernel, (unsigned)cta, kThreads, smem, 2, batch);
         else launch(ex, wgrad_tc_kernel, (unsigned)cta, kThreads, smem, batch);
-        ex.check("conv_wgrad_tc", bytes, flops);
+        ex.check(pair ? "conv_wgrad_tc2" : "conv_wgrad_tc", bytes, flops);
         if (n_sums) {
             if (max_slice >= 524288) {
                 size_t tiles = (max_slice + 1023) / 1024; if (tiles > (size_t)ex.ctx->sm_count * 8) tiles = (size_t)ex.ctx->sm_count * 8;

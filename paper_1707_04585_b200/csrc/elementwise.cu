@@ -14,8 +14,15 @@ cudaEvent_t revnet_ctx::next_event() {
     return ev_pool[ev_used++];
 }
 
+unsigned long long *Exec::stamp_slot() {
+    if (dry || !ctx->stamping || !ctx->stamps || ctx->stamp_next >= kStampSlots) return nullptr;
+    pending_slot = ctx->stamp_next++;
+    return ctx->stamps + pending_slot;
+}
+
 void Exec::check(const char *what, double bytes, double flops) {
     launches++;
+    if (pending_slot >= 0) { ctx->stamp_recs.push_back(StampRec{what, bytes, flops, pending_slot}); pending_slot = -1; }
     cudaError_t e = cudaPeekAtLastError();
     if (e != cudaSuccess && !failed) {
         failed = true;
@@ -219,8 +226,9 @@ void bn_stats(Exec &ex, Pair t, size_t P, Moments mo) {
 // A thread keeps one channel quad (scale and shift stay in registers) and strides the rows, four rows in flight;
 // row_step = threads of the grid / C4 (the launch makes that a whole number): no division per element.
 template <class TO>
-__global__ void __launch_bounds__(256) bn_relu_apply_kernel(Pair t, size_t P, int C4, BnRef bn, TO *__restrict__ a) {
+__global__ void __launch_bounds__(256) bn_relu_apply_kernel(Pair t, size_t P, int C4, BnRef bn, TO *__restrict__ a, unsigned long long *stamp) {
     pdl_enter();
+    stamp_begin(stamp);
     const int C = C4 * 4;
     const size_t gtid = (size_t)blockIdx.x * blockDim.x + threadIdx.x, nth = (size_t)gridDim.x * blockDim.x;
     const int q = (int)(gtid % C4), c = q * 4;
@@ -244,6 +252,7 @@ __global__ void __launch_bounds__(256) bn_relu_apply_kernel(Pair t, size_t P, in
             st4(a + row * C + c, o);
         }
     }
+    stamp_end(stamp);
 }
 
 static int ew_grid(size_t n, int sm) {
@@ -262,8 +271,9 @@ void bn_relu_apply(Exec &ex, Pair t, size_t P, BnRef bn, void *a, bool a_bf16) {
     const int C4 = t.C() / 4;
     static const int occ16 = blocks_per_sm(bn_relu_apply_kernel<bf16>), occ32 = blocks_per_sm(bn_relu_apply_kernel<float>);
     const int g = row_grid(P, C4, ex.ctx->sm_count, a_bf16 ? occ16 : occ32);
-    if (a_bf16) launch(ex, bn_relu_apply_kernel<bf16>, g, 256, 0, t, P, C4, bn, (bf16 *)a);
-    else launch(ex, bn_relu_apply_kernel<float>, g, 256, 0, t, P, C4, bn, (float *)a);
+    unsigned long long *stamp = ex.stamp_slot();
+    if (a_bf16) launch(ex, bn_relu_apply_kernel<bf16>, g, 256, 0, t, P, C4, bn, (bf16 *)a, stamp);
+    else launch(ex, bn_relu_apply_kernel<float>, g, 256, 0, t, P, C4, bn, (float *)a, stamp);
     ex.check("bn_relu_apply", (double)P * t.C() * (a_bf16 ? 6 : 8));
 }
 
@@ -275,8 +285,9 @@ void bn_relu_apply(Exec &ex, Pair t, size_t P, BnRef bn, void *a, bool a_bf16) {
 template <class TO, int OUT, bool CAST>
 __global__ void __launch_bounds__(256, 3) bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, size_t P, int C4, BnRef bn,
                                          const float *__restrict__ coef, TO *__restrict__ out, Pair add, Pair outp,
-                                         bf16 *__restrict__ cast) {
+                                         bf16 *__restrict__ cast, unsigned long long *stamp) {
     pdl_enter();
+    stamp_begin(stamp);
     const int C = C4 * 4;
     const size_t gtid = (size_t)blockIdx.x * blockDim.x + threadIdx.x, nth = (size_t)gridDim.x * blockDim.x;
     const int q = (int)(gtid % C4), c = q * 4;
@@ -309,6 +320,7 @@ __global__ void __launch_bounds__(256, 3) bn_relu_bwd_apply_kernel(const float *
             if (CAST) st4(cast + row * C + c, o);
         }
     }
+    stamp_end(stamp);
 }
 
 // grid for the row-strided elementwise kernels: 256 threads per block, a thread count that is a multiple of C4
@@ -342,14 +354,15 @@ void bn_relu_bwd(Exec &ex, const float *da, Pair t, size_t P, BnRef bn, float *d
         static const int occ = blocks_per_sm(bn_relu_bwd_apply_kernel<float, 2, true>);      // the heaviest variant
         const int g = row_grid(P, C4, ex.ctx->sm_count, occ);
 #define RV_ARGS da, t, P, C4, bn, coef
+        unsigned long long *stamp = ex.stamp_slot();
         if (out_pair.p0 && add.p0) {
-            if (out_cast) launch(ex, bn_relu_bwd_apply_kernel<float, 2, true>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, out_cast);
-            else launch(ex, bn_relu_bwd_apply_kernel<float, 2, false>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, nullptr);
+            if (out_cast) launch(ex, bn_relu_bwd_apply_kernel<float, 2, true>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, out_cast, stamp);
+            else launch(ex, bn_relu_bwd_apply_kernel<float, 2, false>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, nullptr, stamp);
         } else if (out_pair.p0) {
-            if (out_cast) launch(ex, bn_relu_bwd_apply_kernel<float, 1, true>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, out_cast);
-            else launch(ex, bn_relu_bwd_apply_kernel<float, 1, false>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, nullptr);
-        } else if (out_bf16) launch(ex, bn_relu_bwd_apply_kernel<bf16, 0, false>, g, 256, 0, RV_ARGS, (bf16 *)out_single, add, out_pair, nullptr);
-        else launch(ex, bn_relu_bwd_apply_kernel<float, 0, false>, g, 256, 0, RV_ARGS, (float *)out_single, add, out_pair, nullptr);
+            if (out_cast) launch(ex, bn_relu_bwd_apply_kernel<float, 1, true>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, out_cast, stamp);
+            else launch(ex, bn_relu_bwd_apply_kernel<float, 1, false>, g, 256, 0, RV_ARGS, nullptr, add, out_pair, nullptr, stamp);
+        } else if (out_bf16) launch(ex, bn_relu_bwd_apply_kernel<bf16, 0, false>, g, 256, 0, RV_ARGS, (bf16 *)out_single, add, out_pair, nullptr, stamp);
+        else launch(ex, bn_relu_bwd_apply_kernel<float, 0, false>, g, 256, 0, RV_ARGS, (float *)out_single, add, out_pair, nullptr, stamp);
 #undef RV_ARGS
         ex.check("bn_relu_bwd_apply", (double)P * C * ((out_pair.p0 ? (add.p0 ? 16 : 12) : (out_bf16 ? 10 : 12)) + (out_cast ? 2 : 0)));
     }

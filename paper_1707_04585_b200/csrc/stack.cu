@@ -48,6 +48,7 @@ struct revnet_plan {
     bool bound = false;
     cudaGraphExec_t graph_exec = nullptr;
     const void *graph_key[10] = {};
+    bool graph_stamping = false;    // the captured step carries timeline stamps
     revnet_step_stats graph_stats = {};
 };
 
@@ -81,6 +82,13 @@ static void run_step(revnet_plan *pl, Exec &ex, const float *images, const int32
     const float q = ex.q;   // format of the stage buffers (the coupling state)
 
     ex.mark("step_begin");
+    if (!ex.dry && ex.ctx->stamping && ex.ctx->stamps) {
+        // a step's stamps start from "no start yet" (all ones) and "no end yet" (zero); part of the captured graph
+        cudaMemsetAsync(ex.ctx->stamps, 0xff, kStampSlots * sizeof(unsigned long long), ex.stream);
+        cudaMemsetAsync(ex.ctx->stamps + kStampSlots, 0, kStampSlots * sizeof(unsigned long long), ex.stream);
+        ex.ctx->stamp_next = 0;
+        ex.ctx->stamp_recs.clear();
+    }
     // ---- step-long scratch
     const size_t nseg = pl->seg_end.size();
     uint32_t *seg_end = ex.ws.get<uint32_t>(nseg);
@@ -539,7 +547,7 @@ extern "C" int revnet_train_step(revnet_ctx *ctx, revnet_plan *pl, const float *
                     std::to_string(pl->bound_ws) + " bytes (activations / workspace), the plan needs " + std::to_string(pl->act_bytes) + " / " + std::to_string(pl->ws_bytes));
     const bool use_graph = pl->d.use_cuda_graph && !pl->d.verify_reconstruction && !ctx->profiling && ctx->capture_stream;
     const void *key[10] = {images, labels, params, grads, momentum, activations, workspace, loss, pred, logits};
-    if (use_graph && pl->graph_exec && memcmp(key, pl->graph_key, sizeof key) == 0) {
+    if (use_graph && pl->graph_exec && memcmp(key, pl->graph_key, sizeof key) == 0 && pl->graph_stamping == ctx->stamping) {
         if (cudaGraphLaunch(pl->graph_exec, (cudaStream_t)stream) != cudaSuccess)
             return fail(ctx, REVNET_E_CUDA, std::string("revnet_train_step: graph launch: ") + cudaGetErrorString(cudaGetLastError()));
         if (stats) *stats = pl->graph_stats;
@@ -572,6 +580,7 @@ extern "C" int revnet_train_step(revnet_ctx *ctx, revnet_plan *pl, const float *
         cudaGraphDestroy(graph);
         if (e != cudaSuccess) { pl->graph_exec = nullptr; return fail(ctx, REVNET_E_CUDA, std::string("revnet_train_step: instantiate: ") + cudaGetErrorString(e)); }
         memcpy(pl->graph_key, key, sizeof key);
+        pl->graph_stamping = ctx->stamping;
         pl->graph_stats = local_stats;
         if (cudaGraphLaunch(pl->graph_exec, (cudaStream_t)stream) != cudaSuccess)
             return fail(ctx, REVNET_E_CUDA, std::string("revnet_train_step: graph launch: ") + cudaGetErrorString(cudaGetLastError()));

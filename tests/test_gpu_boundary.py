@@ -108,3 +108,37 @@ def test_declared_buffers_smaller_than_planned_are_refused():
     r.step()
     assert np.isfinite(r.results()["loss"])
     ctx.close()
+
+
+@pytest.mark.parametrize("use_graph", [False, True])
+def test_timeline_mode_describes_the_last_step_and_changes_no_result(use_graph):
+    """Timeline stamps: same bits as an unstamped step; every stamped launch has start <= end; the time with a
+    stamped kernel running is no longer than the span from the first start to the last end."""
+    ctx = B.Context(0)
+    st = (syn.StageCfg(2, 64, 16, "bottleneck", 3, 1), syn.StageCfg(2, 128, 32, "bottleneck", 3, 2))
+    cfg = syn.StackCfg("timeline", 8, 16, 10, 3, 1, 16, False, st, seed=5)
+    inp = syn.make_stack_inputs(cfg)
+    r = R.StackRunner(ctx, cfg, 0, use_cuda_graph=use_graph)
+    got = []
+    for stamped in (False, True, False):
+        B.revnet_profile_enable(ctx, 3 if stamped else 0)
+        r.load(inp["images"], inp["labels"], inp["params"])
+        for _ in range(3):                      # under a graph: capture, then replays
+            r.load(inp["images"], inp["labels"], inp["params"])
+            st = r.step()
+        torch.cuda.synchronize()
+        got.append((float(r.loss.item()), r.params.cpu().numpy().copy()))
+        if stamped:
+            tl = B.revnet_profile_summary(ctx)
+            span, busy = tl.pop("stamped_span"), tl.pop("stamped_busy")
+            assert 0 < busy["ms"] <= span["ms"] * (1 + 1e-9)
+            assert busy["launches"] == sum(v["launches"] for v in tl.values()) > 0
+            assert busy["launches"] <= st.kernel_launches
+            assert all(v["ms"] >= 0 and k.count("|") == 2 for k, v in tl.items())
+            assert any(k.startswith("conv_") for k in tl) and any(k.startswith("bn_relu") for k in tl)
+            assert span["ms"] < 1e3
+    B.revnet_profile_enable(ctx, 0)
+    for loss, params in got[1:]:
+        assert loss == got[0][0] and np.array_equal(params, got[0][1])
+    B.revnet_check_device(ctx)
+    ctx.close()

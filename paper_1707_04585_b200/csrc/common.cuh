@@ -106,9 +106,15 @@ struct Pair {
 #ifdef __CUDACC__
     __device__ __forceinline__ float4 ld4(size_t row, int ch) const {
         const float *p = at(row, ch);
-        if (q == 0.f) return *reinterpret_cast<const float4 *>(p);
-        int4 i = *reinterpret_cast<const int4 *>(p);
-        return dequant4(i, q);
+        return from_raw(*reinterpret_cast<const float4 *>(p));
+    }
+    // the 16 bytes as they are stored, and their values: split so that a streaming kernel can issue the loads of several
+    // rows before it converts any of them (branch-free: the conversion instruction, not the adder route above)
+    __device__ __forceinline__ float4 ld4_raw(size_t row, int ch) const { return *reinterpret_cast<const float4 *>(at(row, ch)); }
+    __device__ __forceinline__ float4 from_raw(float4 r) const {
+        if (q == 0.f) return r;
+        return make_float4(__int2float_rn(__float_as_int(r.x)) * q, __int2float_rn(__float_as_int(r.y)) * q,
+                           __int2float_rn(__float_as_int(r.z)) * q, __int2float_rn(__float_as_int(r.w)) * q);
     }
     // out = partner + sign * v on the stored representation (sign 0: out = v)
     __device__ __forceinline__ void couple(size_t row, int ch, float v, const Pair &partner, int sign) const {

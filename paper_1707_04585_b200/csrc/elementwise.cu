@@ -236,16 +236,18 @@ __global__ void __launch_bounds__(256) bn_relu_apply_kernel(Pair t, size_t P, in
     float4 sc, sh, mu, rs;
     bn_coef4(bn, c, sc, sh, mu, rs);
     for (size_t rb = row0; rb < P; rb += 4 * row_step) {
+        // all four loads leave before anything waits on one: rows beyond the end read the last row again and are not stored
         float4 v[4];
 #pragma unroll
         for (int j = 0; j < 4; j++) {
             const size_t row = rb + j * row_step;
-            if (row < P) v[j] = t.ld4(row, c);
+            v[j] = t.ld4_raw(row < P ? row : P - 1, c);
         }
 #pragma unroll
         for (int j = 0; j < 4; j++) {
             const size_t row = rb + j * row_step;
             if (row >= P) continue;
+            v[j] = t.from_raw(v[j]);
             float4 o;
             o.x = fmaxf(fmaf(sc.x, v[j].x, sh.x), 0.f); o.y = fmaxf(fmaf(sc.y, v[j].y, sh.y), 0.f);
             o.z = fmaxf(fmaf(sc.z, v[j].z, sh.z), 0.f); o.w = fmaxf(fmaf(sc.w, v[j].w, sh.w), 0.f);
@@ -283,7 +285,7 @@ void bn_relu_apply(Exec &ex, Pair t, size_t P, BnRef bn, void *a, bool a_bf16) {
 // A thread keeps one channel quad (its coefficients stay in registers) and strides the rows, four
 // rows in flight; row_step = threads of the grid / C4 (the launch makes that a whole number).
 template <class TO, int OUT, bool CAST>
-__global__ void __launch_bounds__(256, 3) bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, size_t P, int C4, BnRef bn,
+__global__ void __launch_bounds__(256, 2) bn_relu_bwd_apply_kernel(const float *__restrict__ da, Pair t, size_t P, int C4, BnRef bn,
                                          const float *__restrict__ coef, TO *__restrict__ out, Pair add, Pair outp,
                                          bf16 *__restrict__ cast, unsigned long long *stamp) {
     pdl_enter();
@@ -296,19 +298,21 @@ __global__ void __launch_bounds__(256, 3) bn_relu_bwd_apply_kernel(const float *
     bn_coef4(bn, c, sc, sh, mu, rs);
     const float4 k0 = ld4(coef + c), k1 = ld4(coef + C + c), k2 = ld4(coef + 2 * C + c);
     for (size_t rb = row0; rb < P; rb += 4 * row_step) {
+        // all loads of the four rows leave before anything waits on one: rows beyond the end read the last row again and
+        // are not stored
         float4 v[4], g[4], pa[4];
 #pragma unroll
         for (int j = 0; j < 4; j++) {
-            const size_t row = rb + j * row_step;
-            if (row < P) {
-                v[j] = t.ld4(row, c); g[j] = ld4(da + row * C + c);
-                if (OUT == 2) pa[j] = add.ld4(row, c);
-            }
+            const size_t row = rb + j * row_step, rr = row < P ? row : P - 1;
+            v[j] = t.ld4_raw(rr, c); g[j] = ld4(da + rr * C + c);
+            if (OUT == 2) pa[j] = add.ld4_raw(rr, c);
         }
 #pragma unroll
         for (int j = 0; j < 4; j++) {
             const size_t row = rb + j * row_step;
             if (row >= P) continue;
+            v[j] = t.from_raw(v[j]);
+            if (OUT == 2) pa[j] = add.from_raw(pa[j]);
             float4 o;
             o.x = k0.x * (fmaf(sc.x, v[j].x, sh.x) > 0.f ? g[j].x : 0.f) - k1.x - k2.x * ((v[j].x - mu.x) * rs.x);
             o.y = k0.y * (fmaf(sc.y, v[j].y, sh.y) > 0.f ? g[j].y : 0.f) - k1.y - k2.y * ((v[j].y - mu.y) * rs.y);

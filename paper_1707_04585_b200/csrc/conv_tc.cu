@@ -86,84 +86,37 @@ struct __align__(8) TcShared {
 //   store   one TMA store of the group
 //   pass B  thread = (channel quad, every rpp-th pixel): per-channel sums over the valid pixels of the group
 // KA: 0 plain float, 1 plain onto the fixed-point grid, 2 / 3 float coupling + / -, 4 / 5 fixed-point coupling + / -.
+// These two passes run once per column group between barriers, on two warps per scheduler: straight-line code that
+// is executed once per visit is paid for in instruction fetches, not in issue slots.  So they are kept SMALL (rolled
+// loops, the plain conversion instructions) rather than unrolled.
 template <int KA>
 __device__ __forceinline__ void tma_pass_a(uint32_t tm, int GW, int row, bool valid, const uint8_t *aux, uint8_t *outb, float out_s) {
     const int row_b = GW * 4;
     const int swz = GW == 32 ? (row & 7) : ((row >> 1) & 3);
 #pragma unroll 1
-    for (int c = 0; c < GW; c += 16) {
-        float v[16];
-        tmem_ld16(tm + (uint32_t)c, v);
+    for (int c = 0; c < GW; c += 8) {
+        float v[8];
+        tmem_ld8(tm + (uint32_t)c, v);
         if (!valid) continue;
-        int off[4];
 #pragma unroll
-        for (int j = 0; j < 4; j++) off[j] = row * row_b + ((((c >> 2) + j) ^ swz) << 4);
-        if (KA == 0) {
-#pragma unroll
-            for (int j = 0; j < 4; j++) *reinterpret_cast<float4 *>(outb + off[j]) = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-        } else if (KA == 2 || KA == 3) {
-            float4 pr[4];
-#pragma unroll
-            for (int j = 0; j < 4; j++) pr[j] = *reinterpret_cast<const float4 *>(aux + off[j]);
-#pragma unroll
-            for (int j = 0; j < 4; j++) {
-                float4 r = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
-                if (KA == 2) { r.x = pr[j].x + r.x; r.y = pr[j].y + r.y; r.z = pr[j].z + r.z; r.w = pr[j].w + r.w; }
-                else { r.x = pr[j].x - r.x; r.y = pr[j].y - r.y; r.z = pr[j].z - r.z; r.w = pr[j].w - r.w; }
-                *reinterpret_cast<float4 *>(outb + off[j]) = r;
+        for (int j = 0; j < 2; j++) {
+            const int off = row * row_b + ((((c >> 2) + j) ^ swz) << 4);
+            float4 r = make_float4(v[4 * j], v[4 * j + 1], v[4 * j + 2], v[4 * j + 3]);
+            if (KA == 2 || KA == 3) {
+                const float4 pr = *reinterpret_cast<const float4 *>(aux + off);
+                if (KA == 2) { r.x = pr.x + r.x; r.y = pr.y + r.y; r.z = pr.z + r.z; r.w = pr.w + r.w; }
+                else { r.x = pr.x - r.x; r.y = pr.y - r.y; r.z = pr.z - r.z; r.w = pr.w - r.w; }
+            } else if (KA != 0) {
+                int4 iv = make_int4(__float2int_rn(r.x * out_s), __float2int_rn(r.y * out_s), __float2int_rn(r.z * out_s), __float2int_rn(r.w * out_s));
+                if (KA >= 4) {
+                    const int4 pi = *reinterpret_cast<const int4 *>(aux + off);
+                    if (KA == 4) { iv.x = pi.x + iv.x; iv.y = pi.y + iv.y; iv.z = pi.z + iv.z; iv.w = pi.w + iv.w; }
+                    else { iv.x = pi.x - iv.x; iv.y = pi.y - iv.y; iv.z = pi.z - iv.z; iv.w = pi.w - iv.w; }
+                }
+                r = make_float4(__int_as_float(iv.x), __int_as_float(iv.y), __int_as_float(iv.z), __int_as_float(iv.w));
             }
-        } else {
-            // onto the fixed-point grid: the sixteen values through the float adder with ONE range test between them
-            // (see round4_to_int), the partner's quads fetched before the arithmetic starts
-            int4 pi[4];
-            if (KA >= 4) {
-#pragma unroll
-                for (int j = 0; j < 4; j++) pi[j] = *reinterpret_cast<const int4 *>(aux + off[j]);
-            }
-            int iv[16];
-            unsigned chk = 0u;
-#pragma unroll
-            for (int i = 0; i < 16; i++) {
-                iv[i] = __float_as_int(__fadd_rn(__fmul_rn(v[i], out_s), 12582912.f));
-                chk |= (unsigned)iv[i] ^ 0x4B000000u;
-            }
-            if ((chk & 0xFF800000u) == 0u) {
-#pragma unroll
-                for (int i = 0; i < 16; i++) iv[i] -= 0x4B400000;
-            } else {
-#pragma unroll
-                for (int i = 0; i < 16; i++) iv[i] = __float2int_rn(__fmul_rn(v[i], out_s));
-            }
-#pragma unroll
-            for (int j = 0; j < 4; j++) {
-                int4 o = make_int4(iv[4 * j], iv[4 * j + 1], iv[4 * j + 2], iv[4 * j + 3]);
-                if (KA == 4) { o.x = pi[j].x + o.x; o.y = pi[j].y + o.y; o.z = pi[j].z + o.z; o.w = pi[j].w + o.w; }
-                if (KA == 5) { o.x = pi[j].x - o.x; o.y = pi[j].y - o.y; o.z = pi[j].z - o.z; o.w = pi[j].w - o.w; }
-                *reinterpret_cast<int4 *>(outb + off[j]) = o;
-            }
+            *reinterpret_cast<float4 *>(outb + off) = r;
         }
-    }
-}
-// fixed point -> float for the eight quads a thread of pass B holds: one range test for all of them (see int4_to_float)
-__device__ __forceinline__ void dequant_rows8(float4 (&v)[8], float q) {
-    unsigned u[32], chk = 0u;
-#pragma unroll
-    for (int k = 0; k < 8; k++) {
-        u[4 * k] = __float_as_uint(v[k].x) + 0x4B400000u; u[4 * k + 1] = __float_as_uint(v[k].y) + 0x4B400000u;
-        u[4 * k + 2] = __float_as_uint(v[k].z) + 0x4B400000u; u[4 * k + 3] = __float_as_uint(v[k].w) + 0x4B400000u;
-    }
-#pragma unroll
-    for (int i = 0; i < 32; i++) chk |= u[i] ^ 0x4B000000u;
-    if ((chk & 0xFF800000u) == 0u) {
-#pragma unroll
-        for (int k = 0; k < 8; k++)
-            v[k] = make_float4(__fmul_rn(__fadd_rn(__uint_as_float(u[4 * k]), -12582912.f), q), __fmul_rn(__fadd_rn(__uint_as_float(u[4 * k + 1]), -12582912.f), q),
-                               __fmul_rn(__fadd_rn(__uint_as_float(u[4 * k + 2]), -12582912.f), q), __fmul_rn(__fadd_rn(__uint_as_float(u[4 * k + 3]), -12582912.f), q));
-    } else {
-#pragma unroll
-        for (int k = 0; k < 8; k++)
-            v[k] = make_float4(__fmul_rn(__int2float_rn(__float_as_int(v[k].x)), q), __fmul_rn(__int2float_rn(__float_as_int(v[k].y)), q),
-                               __fmul_rn(__int2float_rn(__float_as_int(v[k].z)), q), __fmul_rn(__int2float_rn(__float_as_int(v[k].w)), q));
     }
 }
 // KB 0 / 1: sums and second sums of the stored values (float / fixed point); 2 / 3: the two sums of the
@@ -171,49 +124,23 @@ __device__ __forceinline__ void dequant_rows8(float4 (&v)[8], float q) {
 template <int KB>
 __device__ __forceinline__ void tma_pass_b(int GW, const uint8_t *ob, const uint8_t *aux, int jq, int r0, int rpp, int valid_px,
                                            float q, float4 sc4, float4 sh4, float4 mu4, float4 rs4, float (&acc)[8]) {
-    if (GW == 32) {
-        // rows r0, r0 + 16, ..., r0 + 112 of the group (rows of 128 bytes, 16-byte quads swizzled by row & 7, which is r0 & 7
-        // for all of them): all eight quads are fetched before the arithmetic starts; rows beyond the tile's pixels do not count
-        const int base = r0 * 128 + ((jq ^ (r0 & 7)) << 4);
-        float4 v[8], tt[8];
-#pragma unroll
-        for (int k = 0; k < 8; k++) v[k] = *reinterpret_cast<const float4 *>(ob + base + k * 2048);
-        if (KB >= 2) {
-#pragma unroll
-            for (int k = 0; k < 8; k++) tt[k] = *reinterpret_cast<const float4 *>(aux + base + k * 2048);
-            if (KB == 3) dequant_rows8(tt, q);
-        } else if (KB == 1) dequant_rows8(v, q);
-#pragma unroll
-        for (int k = 0; k < 8; k++) {
-            if (r0 + 16 * k >= valid_px) continue;
-            if (KB >= 2) {
-                const float dx = fmaf(sc4.x, tt[k].x, sh4.x) > 0.f ? v[k].x : 0.f, dy = fmaf(sc4.y, tt[k].y, sh4.y) > 0.f ? v[k].y : 0.f;
-                const float dz = fmaf(sc4.z, tt[k].z, sh4.z) > 0.f ? v[k].z : 0.f, dw = fmaf(sc4.w, tt[k].w, sh4.w) > 0.f ? v[k].w : 0.f;
-                acc[0] += dx; acc[1] += dy; acc[2] += dz; acc[3] += dw;
-                acc[4] += dx * ((tt[k].x - mu4.x) * rs4.x); acc[5] += dy * ((tt[k].y - mu4.y) * rs4.y);
-                acc[6] += dz * ((tt[k].z - mu4.z) * rs4.z); acc[7] += dw * ((tt[k].w - mu4.w) * rs4.w);
-            } else {
-                acc[0] += v[k].x; acc[1] += v[k].y; acc[2] += v[k].z; acc[3] += v[k].w;
-                acc[4] += v[k].x * v[k].x; acc[5] += v[k].y * v[k].y; acc[6] += v[k].z * v[k].z; acc[7] += v[k].w * v[k].w;
-            }
-        }
-        return;
-    }
     const int row_b = GW * 4;
-#pragma unroll 4
+#pragma unroll 1
     for (int pl = r0; pl < valid_px; pl += rpp) {
-        const int off = pl * row_b + ((jq ^ ((pl >> 1) & 3)) << 4);
+        const int off = pl * row_b + ((jq ^ (GW == 32 ? (pl & 7) : ((pl >> 1) & 3))) << 4);
         float4 v = *reinterpret_cast<const float4 *>(ob + off);
         if (KB >= 2) {
             float4 tt = *reinterpret_cast<const float4 *>(aux + off);
-            if (KB == 3) tt = dequant4(make_int4(__float_as_int(tt.x), __float_as_int(tt.y), __float_as_int(tt.z), __float_as_int(tt.w)), q);
+            if (KB == 3) tt = make_float4(__int2float_rn(__float_as_int(tt.x)) * q, __int2float_rn(__float_as_int(tt.y)) * q,
+                                          __int2float_rn(__float_as_int(tt.z)) * q, __int2float_rn(__float_as_int(tt.w)) * q);
             const float dx = fmaf(sc4.x, tt.x, sh4.x) > 0.f ? v.x : 0.f, dy = fmaf(sc4.y, tt.y, sh4.y) > 0.f ? v.y : 0.f;
             const float dz = fmaf(sc4.z, tt.z, sh4.z) > 0.f ? v.z : 0.f, dw = fmaf(sc4.w, tt.w, sh4.w) > 0.f ? v.w : 0.f;
             acc[0] += dx; acc[1] += dy; acc[2] += dz; acc[3] += dw;
             acc[4] += dx * ((tt.x - mu4.x) * rs4.x); acc[5] += dy * ((tt.y - mu4.y) * rs4.y);
             acc[6] += dz * ((tt.z - mu4.z) * rs4.z); acc[7] += dw * ((tt.w - mu4.w) * rs4.w);
         } else {
-            if (KB == 1) v = dequant4(make_int4(__float_as_int(v.x), __float_as_int(v.y), __float_as_int(v.z), __float_as_int(v.w)), q);
+            if (KB == 1) v = make_float4(__int2float_rn(__float_as_int(v.x)) * q, __int2float_rn(__float_as_int(v.y)) * q,
+                                         __int2float_rn(__float_as_int(v.z)) * q, __int2float_rn(__float_as_int(v.w)) * q);
             acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
             acc[4] += v.x * v.x; acc[5] += v.y * v.y; acc[6] += v.z * v.z; acc[7] += v.w * v.w;
         }

@@ -57,39 +57,6 @@ struct OncePerDevice {
     }
 };
 
-#ifdef __CUDACC__
-// Exact float <-> integer conversions, four at a time, through the float adder instead of the quarter-rate
-// conversion unit: for |x| < 2^22 the sum x + 1.5 * 2^23 carries the integer nearest to x (ties to even, the
-// adder's rounding) in its low mantissa bits, and the float whose bits are 0x4B400000 + i is 1.5 * 2^23 + i.
-// A sum outside [2^23, 2^24) -- a larger value, or not a number -- sends all four through cvt, so the results are
-// those of cvt.rni.s32.f32 / cvt.rn.f32.s32 bit for bit.
-__device__ __forceinline__ int4 round4_to_int(float4 x) {
-    const float m = 12582912.f;
-    const int a = __float_as_int(__fadd_rn(x.x, m)), b = __float_as_int(__fadd_rn(x.y, m));
-    const int c = __float_as_int(__fadd_rn(x.z, m)), d = __float_as_int(__fadd_rn(x.w, m));
-    if ((((a ^ 0x4B000000) | (b ^ 0x4B000000) | (c ^ 0x4B000000) | (d ^ 0x4B000000)) & 0xFF800000) == 0)
-        return make_int4(a - 0x4B400000, b - 0x4B400000, c - 0x4B400000, d - 0x4B400000);
-    return make_int4(__float2int_rn(x.x), __float2int_rn(x.y), __float2int_rn(x.z), __float2int_rn(x.w));
-}
-__device__ __forceinline__ float4 int4_to_float(int4 i) {
-    const unsigned a = (unsigned)i.x + 0x4B400000u, b = (unsigned)i.y + 0x4B400000u;
-    const unsigned c = (unsigned)i.z + 0x4B400000u, d = (unsigned)i.w + 0x4B400000u;
-    if ((((a ^ 0x4B000000u) | (b ^ 0x4B000000u) | (c ^ 0x4B000000u) | (d ^ 0x4B000000u)) & 0xFF800000u) == 0u) {
-        const float m = -12582912.f;
-        return make_float4(__fadd_rn(__uint_as_float(a), m), __fadd_rn(__uint_as_float(b), m), __fadd_rn(__uint_as_float(c), m), __fadd_rn(__uint_as_float(d), m));
-    }
-    return make_float4(__int2float_rn(i.x), __int2float_rn(i.y), __int2float_rn(i.z), __int2float_rn(i.w));
-}
-// fixed point -> value (i * q) and value -> fixed point (nearest multiple of q = 1 / s)
-__device__ __forceinline__ float4 dequant4(int4 i, float q) {
-    const float4 f = int4_to_float(i);
-    return make_float4(__fmul_rn(f.x, q), __fmul_rn(f.y, q), __fmul_rn(f.z, q), __fmul_rn(f.w, q));
-}
-__device__ __forceinline__ int4 quant4(float4 v, float s) {
-    return round4_to_int(make_float4(__fmul_rn(v.x, s), __fmul_rn(v.y, s), __fmul_rn(v.z, s), __fmul_rn(v.w, s)));
-}
-#endif
-
 // A tensor of C = c0 + c1 channels stored as two NHWC tensors: channels [0,c0) in p0 (row
 // stride c0) and [c0,c0+c1) in p1 (row stride c1).  c1 == 0: one plain tensor.
 // q == 0: elements are float.  q > 0: elements are int32 fixed point, value = i * q with
@@ -133,9 +100,9 @@ struct Pair {
         float *o = at(row, ch);
         if (q == 0.f) { *reinterpret_cast<float4 *>(o) = v; return v; }
         const float s = 1.f / q;
-        int4 iv = quant4(v, s);
+        int4 iv = make_int4(__float2int_rn(v.x * s), __float2int_rn(v.y * s), __float2int_rn(v.z * s), __float2int_rn(v.w * s));
         *reinterpret_cast<int4 *>(o) = iv;
-        return dequant4(iv, q);
+        return make_float4(__int2float_rn(iv.x) * q, __int2float_rn(iv.y) * q, __int2float_rn(iv.z) * q, __int2float_rn(iv.w) * q);
     }
     // out = partner + sign * v with the partner's 16 raw bytes already loaded; returns the stored values (dequantised)
     __device__ __forceinline__ float4 couple4_with(size_t row, int ch, float4 v, float4 praw, int sign) const {
@@ -147,12 +114,12 @@ struct Pair {
             return v;
         }
         const float s = 1.f / q;
-        int4 iv = quant4(v, s);
+        int4 iv = make_int4(__float2int_rn(v.x * s), __float2int_rn(v.y * s), __float2int_rn(v.z * s), __float2int_rn(v.w * s));
         const int4 p = make_int4(__float_as_int(praw.x), __float_as_int(praw.y), __float_as_int(praw.z), __float_as_int(praw.w));
         if (sign > 0) { iv.x = p.x + iv.x; iv.y = p.y + iv.y; iv.z = p.z + iv.z; iv.w = p.w + iv.w; }
         else { iv.x = p.x - iv.x; iv.y = p.y - iv.y; iv.z = p.z - iv.z; iv.w = p.w - iv.w; }
         *reinterpret_cast<int4 *>(o) = iv;
-        return dequant4(iv, q);
+        return make_float4(__int2float_rn(iv.x) * q, __int2float_rn(iv.y) * q, __int2float_rn(iv.z) * q, __int2float_rn(iv.w) * q);
     }
     // four consecutive channels at once (ch % 4 == 0)
     __device__ __forceinline__ void couple4(size_t row, int ch, float4 v, const Pair &partner, int sign) const {
@@ -166,7 +133,7 @@ struct Pair {
             *reinterpret_cast<float4 *>(o) = v;
         } else {
             const float s = 1.f / q;
-            int4 iv = quant4(v, s);
+            int4 iv = make_int4(__float2int_rn(v.x * s), __float2int_rn(v.y * s), __float2int_rn(v.z * s), __float2int_rn(v.w * s));
             if (sign) {
                 int4 p = *reinterpret_cast<const int4 *>(partner.at(row, ch));
                 if (sign > 0) { iv.x = p.x + iv.x; iv.y = p.y + iv.y; iv.z = p.z + iv.z; iv.w = p.w + iv.w; }

@@ -156,9 +156,8 @@ __device__ __forceinline__ void build_tile(const FusedParams &p, FusedShared *sh
                     x[0] = __uint_as_float(lo.x); x[1] = __uint_as_float(lo.y); x[2] = __uint_as_float(lo.z); x[3] = __uint_as_float(lo.w);
                     x[4] = __uint_as_float(hi.x); x[5] = __uint_as_float(hi.y); x[6] = __uint_as_float(hi.z); x[7] = __uint_as_float(hi.w);
                 } else {
-                    const float4 f0 = int4_to_float(make_int4((int)lo.x, (int)lo.y, (int)lo.z, (int)lo.w));
-                    const float4 f1 = int4_to_float(make_int4((int)hi.x, (int)hi.y, (int)hi.z, (int)hi.w));
-                    x[0] = f0.x; x[1] = f0.y; x[2] = f0.z; x[3] = f0.w; x[4] = f1.x; x[5] = f1.y; x[6] = f1.z; x[7] = f1.w;
+                    x[0] = __int2float_rn((int)lo.x); x[1] = __int2float_rn((int)lo.y); x[2] = __int2float_rn((int)lo.z); x[3] = __int2float_rn((int)lo.w);
+                    x[4] = __int2float_rn((int)hi.x); x[5] = __int2float_rn((int)hi.y); x[6] = __int2float_rn((int)hi.z); x[7] = __int2float_rn((int)hi.w);
                 }
 #pragma unroll
                 for (int e = 0; e < 8; e++) x[e] = fmaf(sc[e], x[e], sf[e]);
@@ -209,7 +208,7 @@ __device__ __forceinline__ void pass_a(const FusedParams &p, uint32_t tm, int c0
                 if (KIND == 2) { r.x = pr.x + r.x; r.y = pr.y + r.y; r.z = pr.z + r.z; r.w = pr.w + r.w; }
                 else { r.x = pr.x - r.x; r.y = pr.y - r.y; r.z = pr.z - r.z; r.w = pr.w - r.w; }
             } else if (KIND != 0) {
-                int4 iv = quant4(r, out_s);
+                int4 iv = make_int4(__float2int_rn(r.x * out_s), __float2int_rn(r.y * out_s), __float2int_rn(r.z * out_s), __float2int_rn(r.w * out_s));
                 if (KIND >= 4) {
                     const int4 pi = *reinterpret_cast<const int4 *>(aux + off);
                     if (KIND == 4) { iv.x = pi.x + iv.x; iv.y = pi.y + iv.y; iv.z = pi.z + iv.z; iv.w = pi.w + iv.w; }
@@ -235,14 +234,16 @@ __device__ __forceinline__ void pass_b(const FusedParams &p, const uint8_t *ob, 
         float4 v = *reinterpret_cast<const float4 *>(ob + off);
         if (KIND >= 2) {
             float4 tt = *reinterpret_cast<const float4 *>(aux + off);
-            if (KIND == 3) tt = dequant4(make_int4(__float_as_int(tt.x), __float_as_int(tt.y), __float_as_int(tt.z), __float_as_int(tt.w)), q);
+            if (KIND == 3) tt = make_float4(__int2float_rn(__float_as_int(tt.x)) * q, __int2float_rn(__float_as_int(tt.y)) * q,
+                                            __int2float_rn(__float_as_int(tt.z)) * q, __int2float_rn(__float_as_int(tt.w)) * q);
             const float dx = fmaf(sc4.x, tt.x, sh4.x) > 0.f ? v.x : 0.f, dy = fmaf(sc4.y, tt.y, sh4.y) > 0.f ? v.y : 0.f;
             const float dz = fmaf(sc4.z, tt.z, sh4.z) > 0.f ? v.z : 0.f, dw = fmaf(sc4.w, tt.w, sh4.w) > 0.f ? v.w : 0.f;
             acc[0] += dx; acc[1] += dy; acc[2] += dz; acc[3] += dw;
             acc[4] += dx * ((tt.x - mu4.x) * rs4.x); acc[5] += dy * ((tt.y - mu4.y) * rs4.y);
             acc[6] += dz * ((tt.z - mu4.z) * rs4.z); acc[7] += dw * ((tt.w - mu4.w) * rs4.w);
         } else {
-            if (KIND == 1) v = dequant4(make_int4(__float_as_int(v.x), __float_as_int(v.y), __float_as_int(v.z), __float_as_int(v.w)), q);
+            if (KIND == 1) v = make_float4(__int2float_rn(__float_as_int(v.x)) * q, __int2float_rn(__float_as_int(v.y)) * q,
+                                           __int2float_rn(__float_as_int(v.z)) * q, __int2float_rn(__float_as_int(v.w)) * q);
             acc[0] += v.x; acc[1] += v.y; acc[2] += v.z; acc[3] += v.w;
             acc[4] += v.x * v.x; acc[5] += v.y * v.y; acc[6] += v.z * v.z; acc[7] += v.w * v.w;
         }

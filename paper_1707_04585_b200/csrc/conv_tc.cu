@@ -892,6 +892,12 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
                        !(need_aux && auxp.c1 && auxp.c0 % 32) && s.KC == 64 &&
                        pair_enabled && ex.ctx->sm_count % 2 == 0 && s.g.n_px_tiles >= 2 && ((need_aux && (pair1x1 & 1)) || (!need_aux && (pair1x1 & 2)));
     if (wide1) tc_shape(g, cin, cout, k, stride, s, true);
+    // 3x3 stride-1 layers with a partner tile (data gradients with the BN-backward sums fused) on a pair: 256-wide tiles
+    // too, the partner groups through a ring of two slots per warp group (REVNET_CONV_WIDE3X3=0: 128-wide, as before)
+    static const bool wide3_enabled = [] { const char *v = getenv("REVNET_CONV_WIDE3X3"); return !(v && v[0] == '0'); }();
+    const bool wide3 = wide3_enabled && k == 3 && stride == 1 && !s2 && need_aux && cout >= 256 && cout % 32 == 0 && !(out.c1 && out.c0 % 32) &&
+                       !(auxp.c1 && auxp.c0 % 32) && s.KC == 64 && pair_enabled && ex.ctx->sm_count % 2 == 0 && s.g.n_px_tiles >= 2;
+    if (wide3) tc_shape(g, cin, cout, k, stride, s, true);
     // rows of the weight pack (a multiple of its 128-row blocks, whatever the N tile); TMA fills rows beyond with zeros
     const int rp16 = round_up(cout, 16), rows_pad = rp16 <= 128 ? rp16 : round_up(rp16, 128);
     // column groups of 32 floats, or of 16 where the N tile or the halves of a channel-split tensor ask for it

@@ -881,13 +881,13 @@ bool run_conv_tc(Exec &ex, const char *what, const void *act, Geom gin, int cin,
     const int ntap_max = s2 ? 4 : taps;
     // arithmetic-bound layers without a partner tile (transitions, their data gradients): 128 x 256 tiles
     if (!need_aux && !(out.c1 && out.c0 % 32) && (long long)ntap_max * cin >= 1024 && cout >= 256 && cout % 32 == 0) tc_shape(g, cin, cout, k, stride, s, true);
-    // 1x1 layers onto many channels (the last layer of a bottleneck function with its coupling partner, the data
-    // gradient of the first): their operands cross L2 -> shared memory once per tile, and with 128 x 128 tiles that
-    // traffic (not HBM, not the tensor cores) sets their time.  A CTA pair on a 256 x 256 tile moves half of it.
-    // Measured: no faster (these layers' time is their epilogue's, see the kernel), so off unless REVNET_CONV_PAIR1X1
-    // asks for it: bit 0 layers with a partner tile, bit 1 layers without
+    // 1x1 layers onto 256 channels and more on a CTA pair with 256 x 256 tiles: half the operand traffic from L2 per flop.
+    // Measured on the large-image network: layers WITHOUT a partner tile (2048 -> 512 and the like, many channel chunks
+    // per tile) 8-12 % faster; layers WITH one (the last layer of a bottleneck function, epilogue-bound, and a partner
+    // ring that the wide tile leaves only two slots per warp group) 7-12 % slower.  REVNET_CONV_PAIR1X1 overrides:
+    // bit 0 layers with a partner tile, bit 1 layers without (default 2)
     static const bool pair_enabled = [] { const char *v = getenv("REVNET_CONV_PAIR"); return !(v && v[0] == '0'); }();
-    static const int pair1x1 = [] { const char *v = getenv("REVNET_CONV_PAIR1X1"); return v ? atoi(v) : 0; }();
+    static const int pair1x1 = [] { const char *v = getenv("REVNET_CONV_PAIR1X1"); return v ? atoi(v) : 2; }();
     const bool wide1 = k == 1 && stride == 1 && !s2 && cout >= 256 && cout % 32 == 0 && !(out.c1 && out.c0 % 32) &&
                        !(need_aux && auxp.c1 && auxp.c0 % 32) && s.KC == 64 &&
                        pair_enabled && ex.ctx->sm_count % 2 == 0 && s.g.n_px_tiles >= 2 && ((need_aux && (pair1x1 & 1)) || (!need_aux && (pair1x1 & 2)));
